@@ -1,0 +1,197 @@
+/*
+ * nvfp4.h — C ABI of the B200 (sm_100a) NVFP4 linear-layer library.
+ *
+ * The library implements the hot path of the TetraJet-v2 NVFP4 linear layer:
+ *   - double-block quantization to NVFP4 (paper Sec. 2.2): FP32 global scale per outer group, one E4M3 scale
+ *     per 16 elements, E2M1 codes; round-to-nearest or stochastic rounding (Sec. 2.1), along either axis;
+ *   - the three block-scaled FP4 matrix products of the layer (Sec. 2.3):
+ *         Y = Q1(X) Q2(W)^T,   dX = Q3(dY) Q4(W-hat),   dW = Q5(dY^T) Q6(X-hat),
+ *     where backward re-quantizes the dequantized forward operands X-hat, W-hat;
+ *   - OutControl's split (Sec. 4.2, without the Hadamard factors): a static set of outlier channels of X / W
+ *     stays in BF16 and goes through high-precision products.
+ *
+ * Conventions, valid for every entry point unless stated otherwise:
+ *   - All data pointers are DEVICE pointers owned by the caller. The library never allocates, frees or
+ *     synchronises; every call only enqueues work on `stream` (a cudaStream_t passed as void*).
+ *   - Arguments are validated on the host before anything is launched: a non-zero status means nothing ran.
+ *   - Matrices are row-major. BF16 matrices have a leading dimension `ld` in elements (multiple of 8) and a
+ *     16-byte aligned base.
+ *   - Non-finite inputs are outside the contract (results unspecified, no fault).
+ *   - Only compute capability 10.x devices are supported (NVFP4_ERR_ARCH otherwise). There is no CPU path.
+ */
+#ifndef NVFP4_H_
+#define NVFP4_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  NVFP4_OK = 0,
+  NVFP4_ERR_NULL = 1,      /* a required pointer is NULL */
+  NVFP4_ERR_SHAPE = 2,     /* a size is negative, zero where not allowed, or inconsistent */
+  NVFP4_ERR_ALIGN = 3,     /* a pointer or leading dimension breaks the alignment rules */
+  NVFP4_ERR_ENUM = 4,      /* an enum argument is out of range */
+  NVFP4_ERR_WORKSPACE = 5, /* workspace missing or smaller than nvfp4_*_workspace_bytes says */
+  NVFP4_ERR_ARCH = 6,      /* current device is not sm_100 */
+  NVFP4_ERR_CUDA = 7,      /* a CUDA runtime / driver call failed (launch error, tensor-map encode) */
+  NVFP4_ERR_TIMEOUT = 8    /* reported through dev_status only: a bounded device-side wait ran out */
+} nvfp4_status;
+
+typedef enum { NVFP4_ROUND_RTN = 0, NVFP4_ROUND_SR = 1 } nvfp4_round;
+
+/* Axis along which the 16-element groups run in the SOURCE matrix.
+ * ROW: groups along the columns of a row; the operand has the source's shape [rows, cols].
+ * COL: groups down the rows of a column; the operand is the transpose, shape [cols, rows]. */
+typedef enum { NVFP4_AXIS_ROW = 0, NVFP4_AXIS_COL = 1 } nvfp4_axis;
+
+/* Granularity of the FP32 "global" scale S_global of Sec. 2.2.
+ * TENSOR: one per tensor (needs an amax pre-pass). ROW: one per operand row. BLOCK128: one per 128 consecutive
+ * k of an operand row — the paper's 1x128 outer block. */
+typedef enum { NVFP4_GS_TENSOR = 0, NVFP4_GS_ROW = 1, NVFP4_GS_BLOCK128 = 2 } nvfp4_gs_mode;
+
+/* Memory layout of the E4M3 block scales of an operand [R, Kp].
+ * LINEAR:     row-major [R, Kp/16].
+ * TILED128x4: what the tensor core reads. 512-byte tiles cover 128 rows x 4 k-blocks; inside a tile the byte
+ *             of (r, kb) sits at (r % 32) * 16 + (r / 32) * 4 + (kb % 4); tiles are ordered k-tile fastest
+ *             within a 128-row tile; rows are padded to 128 and k-blocks to 16 (zero bytes). */
+typedef enum { NVFP4_SF_LINEAR = 0, NVFP4_SF_TILED128x4 = 1 } nvfp4_sf_layout;
+
+typedef enum { NVFP4_DT_BF16 = 0, NVFP4_DT_F32 = 1 } nvfp4_dtype;
+
+/* A quantized GEMM operand [R, K], groups along K. Kp = K rounded up to 128; padding codes and scales are 0.
+ *   codes : uint8 [R, Kp/2], two E2M1 codes per byte, low nibble = even k; code = sign<<3 | magnitude index
+ *           into {0, .5, 1, 1.5, 2, 3, 4, 6}.
+ *   sf    : E4M3 bytes, nvfp4_operand_sf_bytes() of them, layout per sf_layout.
+ *   gscale: 1 (TENSOR) | R (ROW) | R * (Kp/128) (BLOCK128) floats, row-major.
+ * The struct lives on the host; the three pointers are device memory owned by the caller. R, K, gs_mode and
+ * sf_layout are inputs to the quantize calls (they say what the caller allocated) and are validated there. */
+typedef struct {
+  uint8_t* codes;
+  uint8_t* sf;
+  float* gscale;
+  int64_t R, K;
+  int32_t gs_mode;   /* nvfp4_gs_mode */
+  int32_t sf_layout; /* nvfp4_sf_layout */
+} nvfp4_operand;
+
+/* Host-only size helpers (no CUDA call). K padded to 128; bytes of codes / scales; floats of gscale. */
+int64_t nvfp4_padded_k(int64_t K);
+size_t nvfp4_operand_codes_bytes(int64_t R, int64_t K);
+size_t nvfp4_operand_sf_bytes(int64_t R, int64_t K, int32_t sf_layout);
+size_t nvfp4_operand_gscale_count(int64_t R, int64_t K, int32_t gs_mode);
+
+const char* nvfp4_status_string(nvfp4_status s);
+
+/* ---------------------------------------------------------------------------------------------------------
+ * nvfp4_quantize — double-block quantization of a BF16 matrix (Sec. 2.2; rounding per Sec. 2.1).
+ *
+ *   src_bf16 [rows, cols], leading dimension ld.
+ *   axis     ROW -> out is [rows, n_keep or cols]; COL -> out is the transpose [n_keep or cols, rows].
+ *   rounding RTN: nearest E2M1 value, ties to the even code. SR: 16 random bits u per element from
+ *            Philox4x32-10 (key = seed, counter = (idx / 8, stream_id, 0), idx = r * Kp16 + k in the OPERAND,
+ *            Kp16 = K rounded up to 16); the magnitude rounds up iff (u + 0.5) / 65536 < (a - q1) / (q2 - q1).
+ *   keep_cols optional sorted list (device, int32) of the n_keep source columns that are kept; the others
+ *            (OutControl's outlier channels) are skipped and the kept ones are compacted. ROW axis: compacts K.
+ *            COL axis: compacts the operand rows. NULL keeps all columns (n_keep is ignored).
+ *   out      operand to fill; out->R / out->K must equal the shape stated above.
+ *   workspace at least nvfp4_quantize_workspace_bytes(out->R, gs_mode); holds the amax cells of the TENSOR
+ *            and ROW modes.
+ *
+ * Arithmetic (binary32, one rounding each, in this order): Sg = amax_g / 2688 (1 if the group is all zero);
+ * t = amax_b / Sg; s = t / 6; Sb = e4m3_rn_satfinite(s); d = Sg * Sb; r = 1 / d (0 if Sb = 0); y = x * r;
+ * magnitude = round(min(|y|, 6)); the input's sign bit is kept.
+ * --------------------------------------------------------------------------------------------------------- */
+size_t nvfp4_quantize_workspace_bytes(int64_t out_rows, int32_t gs_mode);
+nvfp4_status nvfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld, int32_t axis,
+                            int32_t rounding, uint64_t seed, uint32_t stream_id, const int32_t* keep_cols,
+                            int64_t n_keep, const nvfp4_operand* out, void* workspace, size_t ws_bytes,
+                            void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------
+ * nvfp4_requantize_t — the backward quantizers Q4 / Q6 of Sec. 2.3: dequantize a forward operand to the
+ * aligned tensor (x_hat = (P * S_block) * S_global, one binary32 rounding), and quantize its TRANSPOSE.
+ *
+ *   in       forward operand [R, K] (any gs_mode, either sf layout).
+ *   out      operand [n_rows_out, R]; without a row map n_rows_out = in->K.
+ *   row_map  optional (device, int32 [n_rows_out]): output row d takes column row_map[d] of `in` when
+ *            row_map[d] >= 0, and column d of the BF16 matrix hp_bf16 [R, >= n_rows_out] (leading dimension
+ *            hp_ld) when row_map[d] < 0 — OutControl's W-hat, whose outlier columns come from W itself
+ *            (Sec. 4.2). NULL: identity map, hp_bf16 unused.
+ *   rounding, seed, stream_id, workspace: as in nvfp4_quantize.
+ * --------------------------------------------------------------------------------------------------------- */
+nvfp4_status nvfp4_requantize_t(const nvfp4_operand* in, const void* hp_bf16, int64_t hp_ld,
+                                const int32_t* row_map, int64_t n_rows_out, int32_t rounding, uint64_t seed,
+                                uint32_t stream_id, const nvfp4_operand* out, void* workspace, size_t ws_bytes,
+                                void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------
+ * nvfp4_gemm — block-scaled FP4 product of two operands (the "FP4 MM" of Sec. 2.3):
+ *      C[m, n] (+)= sum_k  (Pa * Sba * Sga)[m, k] * (Pb * Sbb * Sgb)[n, k]
+ * FP32 accumulation on the tensor cores; TENSOR / ROW global scales are applied in the epilogue, BLOCK128
+ * scales per 128-wide k chunk.
+ *
+ *   A [M, K], B [N, K]: same K and gs_mode, sf_layout = TILED128x4.
+ *   C [M, N] row-major, leading dimension ldc (elements), dtype c_dtype; 16-byte aligned rows.
+ *   accumulate != 0 adds to the existing C (read in c_dtype, summed in FP32).
+ *   dev_status optional device int: set to NVFP4_ERR_TIMEOUT if a bounded wait inside the kernel ran out
+ *            (the kernel then drains and exits; C is unspecified). Never written otherwise.
+ *   workspace at least nvfp4_gemm_workspace_bytes(M, N, K) (split-K partials for small outputs).
+ * --------------------------------------------------------------------------------------------------------- */
+size_t nvfp4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+nvfp4_status nvfp4_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
+                        int32_t accumulate, int32_t* dev_status, void* workspace, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------
+ * The layer (Sec. 2.3; OutControl split of Sec. 4.2). X [N_tok, D], W [C, D], Y / dY [N_tok, C].
+ * --------------------------------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t gs_mode;     /* nvfp4_gs_mode, used by all six quantizers */
+  int32_t rounding[6]; /* nvfp4_round of Q1..Q6; the paper's assignment is RTN, RTN, SR, SR, SR, SR */
+  uint64_t seed;       /* Philox key; the six quantizers use stream ids 1..6 */
+  int32_t y_dtype, dx_dtype, dw_dtype; /* nvfp4_dtype of the three outputs */
+  /* OutControl (all NULL / 0 when unused); device int32 arrays prepared by the caller:                       */
+  int64_t n_out;               /* number of outlier channels |A|                                             */
+  const int32_t* outlier_cols; /* [n_out]      sorted outlier channel indices                                */
+  const int32_t* keep_cols;    /* [D - n_out]  sorted complement                                             */
+  const int32_t* col_map;      /* [D]          position of channel d in keep_cols, or -1 for an outlier      */
+  int32_t* dev_status;         /* optional, see nvfp4_gemm                                                   */
+} nvfp4_layer_cfg;
+
+/* What forward leaves for backward. qx [N_tok, D - n_out] and qw [C, D - n_out] are filled by
+ * nvfp4_linear_fwd (buffers are the caller's, sf_layout TILED128x4). X and W must stay valid until backward
+ * when n_out > 0 (their outlier columns are read again). */
+typedef struct {
+  nvfp4_operand qx, qw;
+  const void* X; /* BF16 [N_tok, D] */
+  const void* W; /* BF16 [C, D]     */
+  int64_t ldx, ldw;
+  int64_t N_tok, D, C;
+} nvfp4_saved;
+
+typedef enum { NVFP4_OP_FWD = 0, NVFP4_OP_BWD_DX = 1, NVFP4_OP_BWD_DW = 2 } nvfp4_op_kind;
+size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, int64_t C, int64_t n_out,
+                                    int32_t gs_mode);
+
+/* Y = Q1(X[:, keep]) Q2(W[:, keep])^T  +  X[:, outl] W[:, outl]^T (BF16 inputs, FP32 accumulate). */
+nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t ldw, int64_t N_tok, int64_t D,
+                              int64_t C, const nvfp4_layer_cfg* cfg, void* Y, int64_t ldy, nvfp4_saved* saved,
+                              void* workspace, size_t ws_bytes, void* stream);
+
+/* dX = Q3(dY) Q4(W-hat): one FP4 product over all D channels; W-hat's outlier columns are W's. */
+nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved* saved,
+                                 const nvfp4_layer_cfg* cfg, void* dX, int64_t lddx, void* workspace,
+                                 size_t ws_bytes, void* stream);
+
+/* dW[:, keep] = Q5(dY^T) Q6(X-hat[:, keep]);  dW[:, outl] = dY^T X[:, outl] (BF16 inputs, FP32 accumulate). */
+nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved* saved,
+                                 const nvfp4_layer_cfg* cfg, void* dW, int64_t lddw, void* workspace,
+                                 size_t ws_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NVFP4_H_ */

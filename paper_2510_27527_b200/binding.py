@@ -1,0 +1,292 @@
+"""Thin ctypes binding of the C-ABI library (``include/nvfp4.h``).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of ``libnvfp4_b200.so``. PyTorch is
+used for device memory and streams, nothing else. There is no fallback: importing this module raises if the
+shared library has not been built (``python -m paper_2510_27527_b200.build``).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnvfp4_b200.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_27527_b200.build` (no fallback exists)")
+_lib = ctypes.CDLL(LIB_PATH)
+
+# enums of include/nvfp4.h
+OK = 0
+ROUND_RTN, ROUND_SR = 0, 1
+AXIS_ROW, AXIS_COL = 0, 1
+GS_TENSOR, GS_ROW, GS_BLOCK128 = 0, 1, 2
+SF_LINEAR, SF_TILED128x4 = 0, 1
+DT_BF16, DT_F32 = 0, 1
+OP_FWD, OP_BWD_DX, OP_BWD_DW = 0, 1, 2
+ERR_TIMEOUT = 8
+
+c_i64, c_i32, c_u64, c_u32, c_vp, c_sz = (ctypes.c_int64, ctypes.c_int32, ctypes.c_uint64, ctypes.c_uint32,
+                                          ctypes.c_void_p, ctypes.c_size_t)
+
+
+class COperand(ctypes.Structure):
+    _fields_ = [("codes", c_vp), ("sf", c_vp), ("gscale", c_vp), ("R", c_i64), ("K", c_i64), ("gs_mode", c_i32),
+                ("sf_layout", c_i32)]
+
+
+class CLayerCfg(ctypes.Structure):
+    _fields_ = [("gs_mode", c_i32), ("rounding", c_i32 * 6), ("seed", c_u64), ("y_dtype", c_i32), ("dx_dtype", c_i32),
+                ("dw_dtype", c_i32), ("n_out", c_i64), ("outlier_cols", c_vp), ("keep_cols", c_vp), ("col_map", c_vp),
+                ("dev_status", c_vp)]
+
+
+class CSaved(ctypes.Structure):
+    _fields_ = [("qx", COperand), ("qw", COperand), ("X", c_vp), ("W", c_vp), ("ldx", c_i64), ("ldw", c_i64),
+                ("N_tok", c_i64), ("D", c_i64), ("C", c_i64)]
+
+
+EXPORTS = {
+    "nvfp4_padded_k": (c_i64, [c_i64]),
+    "nvfp4_operand_codes_bytes": (c_sz, [c_i64, c_i64]),
+    "nvfp4_operand_sf_bytes": (c_sz, [c_i64, c_i64, c_i32]),
+    "nvfp4_operand_gscale_count": (c_sz, [c_i64, c_i64, c_i32]),
+    "nvfp4_status_string": (ctypes.c_char_p, [c_i32]),
+    "nvfp4_quantize_workspace_bytes": (c_sz, [c_i64, c_i32]),
+    "nvfp4_quantize": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_u64, c_u32, c_vp, c_i64,
+                               ctypes.POINTER(COperand), c_vp, c_sz, c_vp]),
+    "nvfp4_requantize_t": (c_i32, [ctypes.POINTER(COperand), c_vp, c_i64, c_vp, c_i64, c_i32, c_u64, c_u32,
+                                   ctypes.POINTER(COperand), c_vp, c_sz, c_vp]),
+    "nvfp4_gemm_workspace_bytes": (c_sz, [c_i64, c_i64, c_i64]),
+    "nvfp4_gemm": (c_i32, [ctypes.POINTER(COperand), ctypes.POINTER(COperand), c_vp, c_i32, c_i64, c_i32, c_vp, c_vp,
+                           c_sz, c_vp]),
+    "nvfp4_linear_workspace_bytes": (c_sz, [c_i32, c_i64, c_i64, c_i64, c_i64, c_i32]),
+    "nvfp4_linear_fwd": (c_i32, [c_vp, c_i64, c_vp, c_i64, c_i64, c_i64, c_i64, ctypes.POINTER(CLayerCfg), c_vp, c_i64,
+                                 ctypes.POINTER(CSaved), c_vp, c_sz, c_vp]),
+    "nvfp4_linear_bwd_dx": (c_i32, [c_vp, c_i64, ctypes.POINTER(CSaved), ctypes.POINTER(CLayerCfg), c_vp, c_i64, c_vp,
+                                    c_sz, c_vp]),
+    "nvfp4_linear_bwd_dw": (c_i32, [c_vp, c_i64, ctypes.POINTER(CSaved), ctypes.POINTER(CLayerCfg), c_vp, c_i64, c_vp,
+                                    c_sz, c_vp]),
+}
+for _name, (_res, _args) in EXPORTS.items():
+    _f = getattr(_lib, _name)
+    _f.restype = _res
+    _f.argtypes = _args
+
+lib = _lib
+
+
+class Nvfp4Error(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {_lib.nvfp4_status_string(status).decode()} (status {status})")
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise Nvfp4Error(status, where)
+
+
+def _stream_ptr() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+# ------------------------------------------------------------------------------------------------------------
+# device-memory holders
+# ------------------------------------------------------------------------------------------------------------
+@dataclass
+class Operand:
+    """Device buffers of one quantized operand [R, K] (see nvfp4_operand in the header)."""
+
+    codes: torch.Tensor  # uint8 [R, Kp/2]
+    sf: torch.Tensor  # uint8, flat
+    gscale: torch.Tensor  # float32, flat
+    R: int
+    K: int
+    gs_mode: int
+    sf_layout: int
+
+    def c(self) -> COperand:
+        return COperand(_ptr(self.codes), _ptr(self.sf), _ptr(self.gscale), self.R, self.K, self.gs_mode, self.sf_layout)
+
+    @property
+    def Kp(self) -> int:
+        return _lib.nvfp4_padded_k(self.K)
+
+    def sf_linear(self) -> np.ndarray:
+        """Scales as a host array [R, Kp/16] whatever the device layout (index shuffling only)."""
+        nb = self.Kp // 16
+        raw = self.sf.cpu().numpy()
+        if self.sf_layout == SF_LINEAR:
+            return raw.reshape(self.R, nb)
+        nbp = (nb + 15) // 16 * 16
+        r = np.arange(self.R)[:, None]
+        kb = np.arange(nb)[None, :]
+        off = ((r >> 7) * (nbp >> 2) + (kb >> 2)) * 512 + (r & 31) * 16 + ((r >> 5) & 3) * 4 + (kb & 3)
+        return raw[off]
+
+
+def alloc_operand(R: int, K: int, gs_mode: int, sf_layout: int = SF_TILED128x4, device="cuda", poison: bool = False) -> Operand:
+    fill = 0xA5 if poison else 0
+    codes = torch.full((max(_lib.nvfp4_operand_codes_bytes(R, K), 1),), fill, dtype=torch.uint8, device=device)
+    sf = torch.full((max(_lib.nvfp4_operand_sf_bytes(R, K, sf_layout), 1),), fill, dtype=torch.uint8, device=device)
+    gs = torch.zeros(max(_lib.nvfp4_operand_gscale_count(R, K, gs_mode), 1), dtype=torch.float32, device=device)
+    return Operand(codes, sf, gs, R, K, gs_mode, sf_layout)
+
+
+def _workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+# ------------------------------------------------------------------------------------------------------------
+# entry points (same names as the C ABI)
+# ------------------------------------------------------------------------------------------------------------
+def nvfp4_quantize(src: torch.Tensor, axis: int = AXIS_ROW, rounding: int = ROUND_RTN, seed: int = 0, stream_id: int = 0,
+                   gs_mode: int = GS_TENSOR, sf_layout: int = SF_TILED128x4, keep_cols: torch.Tensor | None = None,
+                   out: Operand | None = None, workspace: torch.Tensor | None = None) -> Operand:
+    assert src.dtype == torch.bfloat16 and src.dim() == 2 and src.stride(1) == 1
+    rows, cols = src.shape
+    kept = cols if keep_cols is None else int(keep_cols.numel())
+    R, K = (rows, kept) if axis == AXIS_ROW else (kept, rows)
+    if out is None:
+        out = alloc_operand(R, K, gs_mode, sf_layout, src.device)
+    ws = workspace if workspace is not None else _workspace(_lib.nvfp4_quantize_workspace_bytes(R, gs_mode), src.device)
+    co = out.c()
+    _check(_lib.nvfp4_quantize(_ptr(src), rows, cols, src.stride(0), axis, rounding, seed, stream_id, _ptr(keep_cols), kept,
+                               ctypes.byref(co), _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_quantize")
+    return out
+
+
+def nvfp4_requantize_t(inp: Operand, rounding: int = ROUND_SR, seed: int = 0, stream_id: int = 0, gs_mode: int | None = None,
+                       sf_layout: int = SF_TILED128x4, hp: torch.Tensor | None = None, row_map: torch.Tensor | None = None,
+                       out: Operand | None = None, workspace: torch.Tensor | None = None) -> Operand:
+    gs_mode = inp.gs_mode if gs_mode is None else gs_mode
+    D = inp.K if row_map is None else int(row_map.numel())
+    if out is None:
+        out = alloc_operand(D, inp.R, gs_mode, sf_layout, inp.codes.device)
+    ws = workspace if workspace is not None else _workspace(_lib.nvfp4_quantize_workspace_bytes(D, gs_mode), inp.codes.device)
+    ci, co = inp.c(), out.c()
+    _check(_lib.nvfp4_requantize_t(ctypes.byref(ci), _ptr(hp), 0 if hp is None else hp.stride(0), _ptr(row_map), D, rounding,
+                                   seed, stream_id, ctypes.byref(co), _ptr(ws), ws.numel(), _stream_ptr()),
+           "nvfp4_requantize_t")
+    return out
+
+
+def nvfp4_gemm(A: Operand, B: Operand, c_dtype: int = DT_F32, out: torch.Tensor | None = None, accumulate: bool = False,
+               dev_status: torch.Tensor | None = None, workspace: torch.Tensor | None = None) -> torch.Tensor:
+    if out is None:
+        out = torch.empty((A.R, B.R), dtype=torch.float32 if c_dtype == DT_F32 else torch.bfloat16, device=A.codes.device)
+    ws = workspace if workspace is not None else _workspace(_lib.nvfp4_gemm_workspace_bytes(A.R, B.R, A.K), A.codes.device)
+    ca, cb = A.c(), B.c()
+    _check(_lib.nvfp4_gemm(ctypes.byref(ca), ctypes.byref(cb), _ptr(out), c_dtype, out.stride(0), int(accumulate),
+                           _ptr(dev_status), _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_gemm")
+    return out
+
+
+@dataclass
+class LayerConfig:
+    gs_mode: int = GS_TENSOR
+    seed: int = 0
+    rounding: tuple = (ROUND_RTN, ROUND_RTN, ROUND_SR, ROUND_SR, ROUND_SR, ROUND_SR)
+    y_dtype: int = DT_BF16
+    dx_dtype: int = DT_BF16
+    dw_dtype: int = DT_F32
+    outliers: np.ndarray | None = None  # sorted outlier channel indices (host)
+    dev_status: torch.Tensor | None = None
+    # device index arrays, built by prepare()
+    _outl: torch.Tensor | None = None
+    _keep: torch.Tensor | None = None
+    _map: torch.Tensor | None = None
+    _D: int = -1
+
+    def prepare(self, D: int, device="cuda"):
+        """Uploads the OutControl index arrays for hidden size D (index bookkeeping only)."""
+        if self.outliers is None or len(self.outliers) == 0 or self._D == D:
+            return
+        outl = np.asarray(self.outliers, dtype=np.int64)
+        mask = np.ones(D, dtype=bool)
+        mask[outl] = False
+        keep = np.nonzero(mask)[0]
+        cmap = np.full(D, -1, dtype=np.int32)
+        cmap[keep] = np.arange(len(keep), dtype=np.int32)
+        self._outl = torch.from_numpy(outl.astype(np.int32)).to(device)
+        self._keep = torch.from_numpy(keep.astype(np.int32)).to(device)
+        self._map = torch.from_numpy(cmap).to(device)
+        self._D = D
+
+    @property
+    def n_out(self) -> int:
+        return 0 if self.outliers is None else len(self.outliers)
+
+    def c(self) -> CLayerCfg:
+        return CLayerCfg(self.gs_mode, (c_i32 * 6)(*self.rounding), self.seed, self.y_dtype, self.dx_dtype, self.dw_dtype,
+                         self.n_out, _ptr(self._outl), _ptr(self._keep), _ptr(self._map), _ptr(self.dev_status))
+
+
+@dataclass
+class Saved:
+    qx: Operand
+    qw: Operand
+    X: torch.Tensor
+    W: torch.Tensor
+
+    def c(self) -> CSaved:
+        return CSaved(self.qx.c(), self.qw.c(), _ptr(self.X), _ptr(self.W), self.X.stride(0), self.W.stride(0),
+                      self.X.shape[0], self.X.shape[1], self.W.shape[0])
+
+
+def linear_workspace(op_kind: int, N_tok: int, D: int, C: int, cfg: LayerConfig, device="cuda") -> torch.Tensor:
+    return _workspace(_lib.nvfp4_linear_workspace_bytes(op_kind, N_tok, D, C, cfg.n_out, cfg.gs_mode), device)
+
+
+def nvfp4_linear_fwd(X: torch.Tensor, W: torch.Tensor, cfg: LayerConfig, Y: torch.Tensor | None = None,
+                     saved: Saved | None = None, workspace: torch.Tensor | None = None):
+    N_tok, D = X.shape
+    C = W.shape[0]
+    cfg.prepare(D, X.device)
+    Dk = D - cfg.n_out
+    if saved is None:
+        saved = Saved(alloc_operand(N_tok, Dk, cfg.gs_mode, SF_TILED128x4, X.device),
+                      alloc_operand(C, Dk, cfg.gs_mode, SF_TILED128x4, X.device), X, W)
+    else:
+        saved.X, saved.W = X, W
+    if Y is None:
+        Y = torch.empty((N_tok, C), dtype=torch.float32 if cfg.y_dtype == DT_F32 else torch.bfloat16, device=X.device)
+    ws = workspace if workspace is not None else linear_workspace(OP_FWD, N_tok, D, C, cfg, X.device)
+    cs, cc = saved.c(), cfg.c()
+    _check(_lib.nvfp4_linear_fwd(_ptr(X), X.stride(0), _ptr(W), W.stride(0), N_tok, D, C, ctypes.byref(cc), _ptr(Y),
+                                 Y.stride(0), ctypes.byref(cs), _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_linear_fwd")
+    return Y, saved
+
+
+def nvfp4_linear_bwd_dx(dY: torch.Tensor, saved: Saved, cfg: LayerConfig, dX: torch.Tensor | None = None,
+                        workspace: torch.Tensor | None = None) -> torch.Tensor:
+    N_tok, D = saved.X.shape
+    C = saved.W.shape[0]
+    if dX is None:
+        dX = torch.empty((N_tok, D), dtype=torch.float32 if cfg.dx_dtype == DT_F32 else torch.bfloat16, device=dY.device)
+    ws = workspace if workspace is not None else linear_workspace(OP_BWD_DX, N_tok, D, C, cfg, dY.device)
+    cs, cc = saved.c(), cfg.c()
+    _check(_lib.nvfp4_linear_bwd_dx(_ptr(dY), dY.stride(0), ctypes.byref(cs), ctypes.byref(cc), _ptr(dX), dX.stride(0),
+                                    _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_linear_bwd_dx")
+    return dX
+
+
+def nvfp4_linear_bwd_dw(dY: torch.Tensor, saved: Saved, cfg: LayerConfig, dW: torch.Tensor | None = None,
+                        workspace: torch.Tensor | None = None) -> torch.Tensor:
+    N_tok, D = saved.X.shape
+    C = saved.W.shape[0]
+    if dW is None:
+        dW = torch.empty((C, D), dtype=torch.float32 if cfg.dw_dtype == DT_F32 else torch.bfloat16, device=dY.device)
+    ws = workspace if workspace is not None else linear_workspace(OP_BWD_DW, N_tok, D, C, cfg, dY.device)
+    cs, cc = saved.c(), cfg.c()
+    _check(_lib.nvfp4_linear_bwd_dw(_ptr(dY), dY.stride(0), ctypes.byref(cs), ctypes.byref(cc), _ptr(dW), dW.stride(0),
+                                    _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_linear_bwd_dw")
+    return dW

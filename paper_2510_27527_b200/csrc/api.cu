@@ -1,0 +1,450 @@
+// C-ABI entry points: argument validation on the host, workspace carving, and the order in which the layer's
+// quantizers and products are enqueued (paper Sec. 2.3; OutControl split of Sec. 4.2). No allocation, no
+// synchronisation: everything is enqueued on the caller's stream.
+#include "../../include/nvfp4.h"
+
+#include "nvfp4_device.cuh"
+#include "nvfp4_internal.h"
+
+using namespace nvfp4;
+
+namespace {
+
+inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+nvfp4_status check_arch() {
+  static int cached_dev = -1;
+  static nvfp4_status cached = NVFP4_OK;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return NVFP4_ERR_CUDA;
+  if (dev == cached_dev) return cached;
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return NVFP4_ERR_CUDA;
+  cached_dev = dev;
+  cached = (major == 10) ? NVFP4_OK : NVFP4_ERR_ARCH;
+  return cached;
+}
+
+bool valid_operand_desc(const nvfp4_operand* o) {
+  return o->R >= 0 && o->K >= 0 && o->gs_mode >= 0 && o->gs_mode <= 2 && o->sf_layout >= 0 && o->sf_layout <= 1;
+}
+
+nvfp4_status check_operand_ptrs(const nvfp4_operand* o) {
+  if (!o) return NVFP4_ERR_NULL;
+  if (!valid_operand_desc(o)) return (o->R < 0 || o->K < 0) ? NVFP4_ERR_SHAPE : NVFP4_ERR_ENUM;
+  if (o->R == 0 || o->K == 0) return NVFP4_OK;
+  if (!o->codes || !o->sf || !o->gscale) return NVFP4_ERR_NULL;
+  if (!aligned16(o->codes) || !aligned16(o->sf) || (reinterpret_cast<uintptr_t>(o->gscale) & 3u)) return NVFP4_ERR_ALIGN;
+  return NVFP4_OK;
+}
+
+// The scale buffer of the tiled layout is padded (rows to 128, k-blocks to 16); kernels write only real entries.
+cudaError_t clear_sf_padding(const nvfp4_operand* o, cudaStream_t st) {
+  if (o->sf_layout != NVFP4_SF_TILED128x4) return cudaSuccess;
+  const int64_t nb = nvfp4_padded_k(o->K) / 16;
+  if ((o->R % 128) == 0 && (nb % 16) == 0) return cudaSuccess;
+  return cudaMemsetAsync(o->sf, 0, nvfp4_operand_sf_bytes(o->R, o->K, o->sf_layout), st);
+}
+
+struct Carver {
+  uint8_t* base;
+  size_t size, used;
+  Carver(void* p, size_t n) : base(static_cast<uint8_t*>(p)), size(n), used(0) {}
+  void* take(size_t bytes) {
+    const size_t start = (used + 255) & ~(size_t)255;
+    used = start + bytes;
+    return (base && used <= size) ? base + start : nullptr;
+  }
+};
+inline size_t carve_size(size_t& total, size_t bytes) {
+  total = ((total + 255) & ~(size_t)255) + bytes;
+  return total;
+}
+
+size_t cells_bytes(int64_t rows, int32_t gs_mode) {
+  return gs_mode == NVFP4_GS_ROW ? (size_t)std::max<int64_t>(rows, 1) * 4 : 4;
+}
+
+// Operand carved from a workspace (tiled scales).
+void operand_sizes(size_t& total, int64_t R, int64_t K, int32_t gs_mode) {
+  carve_size(total, nvfp4_operand_codes_bytes(R, K));
+  carve_size(total, nvfp4_operand_sf_bytes(R, K, NVFP4_SF_TILED128x4));
+  carve_size(total, nvfp4_operand_gscale_count(R, K, gs_mode) * 4);
+}
+bool carve_operand(Carver& c, nvfp4_operand* o, int64_t R, int64_t K, int32_t gs_mode) {
+  o->codes = static_cast<uint8_t*>(c.take(nvfp4_operand_codes_bytes(R, K)));
+  o->sf = static_cast<uint8_t*>(c.take(nvfp4_operand_sf_bytes(R, K, NVFP4_SF_TILED128x4)));
+  o->gscale = static_cast<float*>(c.take(nvfp4_operand_gscale_count(R, K, gs_mode) * 4));
+  o->R = R;
+  o->K = K;
+  o->gs_mode = gs_mode;
+  o->sf_layout = NVFP4_SF_TILED128x4;
+  return o->codes && o->sf && o->gscale;
+}
+
+nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, int32_t rounding,
+                              uint64_t seed, uint32_t stream_id, const int32_t* keep, int64_t n_keep,
+                              const nvfp4_operand* out, uint32_t* cells, cudaStream_t st) {
+  if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+  QuantRowsArgs a{};
+  a.src = src;
+  a.rows = rows;
+  a.K = keep ? n_keep : cols;
+  a.cols_src = cols;
+  a.ld = ld;
+  a.keep = keep;
+  a.seed = seed;
+  a.stream_id = stream_id;
+  a.gs_mode = out->gs_mode;
+  a.sr = rounding == NVFP4_ROUND_SR;
+  a.sf_tiled = out->sf_layout == NVFP4_SF_TILED128x4;
+  a.compute_amax = 1;
+  a.gs_cells = cells;
+  a.codes = out->codes;
+  a.sf = out->sf;
+  a.gscale = out->gscale;
+  return launch_quantize_rows(a, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status do_quantize_transpose(const TransposeSrc& src, int from_codes, int64_t rowsK, int64_t D, int32_t rounding,
+                                   uint64_t seed, uint32_t stream_id, const nvfp4_operand* out, uint32_t* cells,
+                                   cudaStream_t st) {
+  if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+  QuantTransposeArgs a{};
+  a.from_codes = from_codes;
+  a.rowsK = rowsK;
+  a.D = D;
+  a.src = src;
+  a.seed = seed;
+  a.stream_id = stream_id;
+  a.gs_mode = out->gs_mode;
+  a.sr = rounding == NVFP4_ROUND_SR;
+  a.sf_tiled = out->sf_layout == NVFP4_SF_TILED128x4;
+  a.compute_amax = 1;
+  a.gs_cells = cells;
+  a.codes = out->codes;
+  a.sf = out->sf;
+  a.gscale = out->gscale;
+  return launch_quantize_transpose(a, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status do_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
+                     int32_t accumulate, const float* addend, int64_t ld_add, int32_t* dev_status, cudaStream_t st) {
+  GemmArgs g{};
+  g.a_codes = A->codes;
+  g.a_sf = A->sf;
+  g.a_gscale = A->gscale;
+  g.b_codes = B->codes;
+  g.b_sf = B->sf;
+  g.b_gscale = B->gscale;
+  g.M = A->R;
+  g.N = B->R;
+  g.K = A->K;
+  g.gs_mode = A->gs_mode;
+  g.C = C;
+  g.c_is_f32 = c_dtype == NVFP4_DT_F32;
+  g.ldc = ldc;
+  g.accumulate = accumulate;
+  g.addend = addend;
+  g.ld_add = ld_add;
+  g.dev_status = dev_status;
+  return launch_gemm(g, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status check_cfg(const nvfp4_layer_cfg* cfg, int64_t D) {
+  if (!cfg) return NVFP4_ERR_NULL;
+  if (cfg->gs_mode < 0 || cfg->gs_mode > 2) return NVFP4_ERR_ENUM;
+  for (int i = 0; i < 6; ++i)
+    if (cfg->rounding[i] < 0 || cfg->rounding[i] > 1) return NVFP4_ERR_ENUM;
+  if (cfg->y_dtype < 0 || cfg->y_dtype > 1 || cfg->dx_dtype < 0 || cfg->dx_dtype > 1 || cfg->dw_dtype < 0 ||
+      cfg->dw_dtype > 1)
+    return NVFP4_ERR_ENUM;
+  if (cfg->n_out < 0 || cfg->n_out > D) return NVFP4_ERR_SHAPE;
+  if (cfg->n_out > 0 && (!cfg->outlier_cols || !cfg->keep_cols || !cfg->col_map)) return NVFP4_ERR_NULL;
+  return NVFP4_OK;
+}
+
+bool bad_matrix(const void* p, int64_t ld, int64_t cols, int elem_bytes) {
+  return !aligned16(p) || ld < cols || (ld * elem_bytes) % 16 != 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t nvfp4_padded_k(int64_t K) { return round_up(K, 128); }
+
+size_t nvfp4_operand_codes_bytes(int64_t R, int64_t K) { return (size_t)(R * (nvfp4_padded_k(K) / 2)); }
+
+size_t nvfp4_operand_sf_bytes(int64_t R, int64_t K, int32_t sf_layout) {
+  const int64_t nb = nvfp4_padded_k(K) / 16;
+  if (sf_layout == NVFP4_SF_TILED128x4) return (size_t)(round_up(R, 128) * round_up(nb, 16));
+  return (size_t)(R * nb);
+}
+
+size_t nvfp4_operand_gscale_count(int64_t R, int64_t K, int32_t gs_mode) {
+  if (gs_mode == NVFP4_GS_TENSOR) return 1;
+  if (gs_mode == NVFP4_GS_ROW) return (size_t)R;
+  return (size_t)(R * (nvfp4_padded_k(K) / 128));
+}
+
+const char* nvfp4_status_string(nvfp4_status s) {
+  switch (s) {
+    case NVFP4_OK: return "ok";
+    case NVFP4_ERR_NULL: return "null pointer";
+    case NVFP4_ERR_SHAPE: return "bad shape";
+    case NVFP4_ERR_ALIGN: return "bad alignment";
+    case NVFP4_ERR_ENUM: return "bad enum value";
+    case NVFP4_ERR_WORKSPACE: return "workspace too small";
+    case NVFP4_ERR_ARCH: return "device is not sm_100";
+    case NVFP4_ERR_CUDA: return "CUDA call failed";
+    case NVFP4_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+size_t nvfp4_quantize_workspace_bytes(int64_t out_rows, int32_t gs_mode) {
+  return round_up((int64_t)cells_bytes(out_rows, gs_mode), 256);
+}
+
+nvfp4_status nvfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld, int32_t axis,
+                            int32_t rounding, uint64_t seed, uint32_t stream_id, const int32_t* keep_cols,
+                            int64_t n_keep, const nvfp4_operand* out, void* workspace, size_t ws_bytes,
+                            void* stream) {
+  if (!src_bf16 || !out) return NVFP4_ERR_NULL;
+  if (axis < 0 || axis > 1 || rounding < 0 || rounding > 1) return NVFP4_ERR_ENUM;
+  if (rows < 0 || cols < 0 || (keep_cols && (n_keep < 0 || n_keep > cols))) return NVFP4_ERR_SHAPE;
+  if (keep_cols && axis != NVFP4_AXIS_ROW) return NVFP4_ERR_SHAPE;
+  nvfp4_status s = check_operand_ptrs(out);
+  if (s != NVFP4_OK) return s;
+  const int64_t kept = keep_cols ? n_keep : cols;
+  const int64_t R = axis == NVFP4_AXIS_ROW ? rows : kept;
+  const int64_t K = axis == NVFP4_AXIS_ROW ? kept : rows;
+  if (out->R != R || out->K != K) return NVFP4_ERR_SHAPE;
+  if (bad_matrix(src_bf16, ld, cols, 2)) return NVFP4_ERR_ALIGN;
+  if (!workspace || ws_bytes < nvfp4_quantize_workspace_bytes(R, out->gs_mode)) return NVFP4_ERR_WORKSPACE;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  if (R == 0 || K == 0) return NVFP4_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* cells = static_cast<uint32_t*>(workspace);
+  if (axis == NVFP4_AXIS_ROW)
+    return do_quantize_rows(static_cast<const uint16_t*>(src_bf16), rows, cols, ld, rounding, seed, stream_id, keep_cols,
+                            n_keep, out, cells, st);
+  TransposeSrc ts{};
+  ts.bf16 = static_cast<const uint16_t*>(src_bf16);
+  ts.ld = ld;
+  return do_quantize_transpose(ts, 0, rows, cols, rounding, seed, stream_id, out, cells, st);
+}
+
+nvfp4_status nvfp4_requantize_t(const nvfp4_operand* in, const void* hp_bf16, int64_t hp_ld, const int32_t* row_map,
+                                int64_t n_rows_out, int32_t rounding, uint64_t seed, uint32_t stream_id,
+                                const nvfp4_operand* out, void* workspace, size_t ws_bytes, void* stream) {
+  if (!in || !out) return NVFP4_ERR_NULL;
+  if (rounding < 0 || rounding > 1) return NVFP4_ERR_ENUM;
+  nvfp4_status s;
+  if ((s = check_operand_ptrs(in)) != NVFP4_OK) return s;
+  if ((s = check_operand_ptrs(out)) != NVFP4_OK) return s;
+  const int64_t D = row_map ? n_rows_out : in->K;
+  if (n_rows_out < 0 || out->R != D || out->K != in->R) return NVFP4_ERR_SHAPE;
+  if (row_map && !hp_bf16) return NVFP4_ERR_NULL;
+  if (row_map && bad_matrix(hp_bf16, hp_ld, D, 2)) return NVFP4_ERR_ALIGN;
+  if (!workspace || ws_bytes < nvfp4_quantize_workspace_bytes(D, out->gs_mode)) return NVFP4_ERR_WORKSPACE;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  if (D == 0 || in->R == 0) return NVFP4_OK;
+  TransposeSrc ts{};
+  ts.in_codes = in->codes;
+  ts.in_sf = in->sf;
+  ts.in_gscale = in->gscale;
+  ts.in_K = in->K;
+  ts.in_gs_mode = in->gs_mode;
+  ts.in_sf_tiled = in->sf_layout == NVFP4_SF_TILED128x4;
+  ts.row_map = row_map;
+  ts.hp = static_cast<const uint16_t*>(hp_bf16);
+  ts.hp_ld = hp_ld;
+  return do_quantize_transpose(ts, 1, in->R, D, rounding, seed, stream_id, out, static_cast<uint32_t*>(workspace),
+                               static_cast<cudaStream_t>(stream));
+}
+
+size_t nvfp4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) { return gemm_workspace_bytes(M, N, K); }
+
+nvfp4_status nvfp4_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
+                        int32_t accumulate, int32_t* dev_status, void* workspace, size_t ws_bytes, void* stream) {
+  if (!A || !B || !C) return NVFP4_ERR_NULL;
+  nvfp4_status s;
+  if ((s = check_operand_ptrs(A)) != NVFP4_OK) return s;
+  if ((s = check_operand_ptrs(B)) != NVFP4_OK) return s;
+  if (c_dtype < 0 || c_dtype > 1) return NVFP4_ERR_ENUM;
+  if (A->K != B->K || A->K <= 0) return NVFP4_ERR_SHAPE;
+  if (A->gs_mode != B->gs_mode) return NVFP4_ERR_ENUM;
+  if (A->sf_layout != NVFP4_SF_TILED128x4 || B->sf_layout != NVFP4_SF_TILED128x4) return NVFP4_ERR_ENUM;
+  if (bad_matrix(C, ldc, B->R, c_dtype == NVFP4_DT_F32 ? 4 : 2)) return NVFP4_ERR_ALIGN;
+  const size_t need = nvfp4_gemm_workspace_bytes(A->R, B->R, A->K);
+  if (need && (!workspace || ws_bytes < need)) return NVFP4_ERR_WORKSPACE;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  return do_gemm(A, B, C, c_dtype, ldc, accumulate, nullptr, 0, dev_status, static_cast<cudaStream_t>(stream));
+}
+
+size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, int64_t C, int64_t n_out,
+                                    int32_t gs_mode) {
+  size_t total = 0;
+  const int64_t Dk = D - n_out;
+  if (op_kind == NVFP4_OP_FWD) {
+    carve_size(total, cells_bytes(N_tok, gs_mode));
+    carve_size(total, cells_bytes(C, gs_mode));
+    if (n_out > 0) carve_size(total, (size_t)N_tok * (size_t)round_up(C, 4) * 4);
+  } else if (op_kind == NVFP4_OP_BWD_DX) {
+    carve_size(total, cells_bytes(N_tok, gs_mode));
+    carve_size(total, cells_bytes(D, gs_mode));
+    operand_sizes(total, N_tok, C, gs_mode);
+    operand_sizes(total, D, C, gs_mode);
+  } else {
+    carve_size(total, cells_bytes(C, gs_mode));
+    carve_size(total, cells_bytes(Dk, gs_mode));
+    operand_sizes(total, C, N_tok, gs_mode);
+    operand_sizes(total, Dk, N_tok, gs_mode);
+    if (n_out > 0) carve_size(total, (size_t)C * (size_t)round_up(Dk, 4) * 4);
+  }
+  return ((total + 255) & ~(size_t)255) + 256;
+}
+
+nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t ldw, int64_t N_tok, int64_t D,
+                              int64_t C, const nvfp4_layer_cfg* cfg, void* Y, int64_t ldy, nvfp4_saved* saved,
+                              void* workspace, size_t ws_bytes, void* stream) {
+  if (!X || !W || !Y || !saved) return NVFP4_ERR_NULL;
+  if (N_tok <= 0 || D <= 0 || C <= 0) return NVFP4_ERR_SHAPE;
+  nvfp4_status s;
+  if ((s = check_cfg(cfg, D)) != NVFP4_OK) return s;
+  const int64_t n_out = cfg->n_out, Dk = D - n_out;
+  if (Dk <= 0) return NVFP4_ERR_SHAPE;
+  if ((s = check_operand_ptrs(&saved->qx)) != NVFP4_OK) return s;
+  if ((s = check_operand_ptrs(&saved->qw)) != NVFP4_OK) return s;
+  if (saved->qx.R != N_tok || saved->qx.K != Dk || saved->qw.R != C || saved->qw.K != Dk) return NVFP4_ERR_SHAPE;
+  if (saved->qx.gs_mode != cfg->gs_mode || saved->qw.gs_mode != cfg->gs_mode ||
+      saved->qx.sf_layout != NVFP4_SF_TILED128x4 || saved->qw.sf_layout != NVFP4_SF_TILED128x4)
+    return NVFP4_ERR_ENUM;
+  if (bad_matrix(X, ldx, D, 2) || bad_matrix(W, ldw, D, 2) || bad_matrix(Y, ldy, C, cfg->y_dtype == NVFP4_DT_F32 ? 4 : 2))
+    return NVFP4_ERR_ALIGN;
+  if (!workspace || ws_bytes < nvfp4_linear_workspace_bytes(NVFP4_OP_FWD, N_tok, D, C, n_out, cfg->gs_mode))
+    return NVFP4_ERR_WORKSPACE;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Carver cv(workspace, ws_bytes);
+  uint32_t* cells_x = static_cast<uint32_t*>(cv.take(cells_bytes(N_tok, cfg->gs_mode)));
+  uint32_t* cells_w = static_cast<uint32_t*>(cv.take(cells_bytes(C, cfg->gs_mode)));
+  const int64_t ld_add = round_up(C, 4);
+  float* addend = n_out > 0 ? static_cast<float*>(cv.take((size_t)N_tok * ld_add * 4)) : nullptr;
+  if (!cells_x || !cells_w || (n_out > 0 && !addend)) return NVFP4_ERR_WORKSPACE;
+
+  const uint16_t* Xp = static_cast<const uint16_t*>(X);
+  const uint16_t* Wp = static_cast<const uint16_t*>(W);
+  const int32_t* keep = n_out > 0 ? cfg->keep_cols : nullptr;
+  if ((s = do_quantize_rows(Xp, N_tok, D, ldx, cfg->rounding[0], cfg->seed, 1, keep, Dk, &saved->qx, cells_x, st)) != NVFP4_OK)
+    return s;
+  if ((s = do_quantize_rows(Wp, C, D, ldw, cfg->rounding[1], cfg->seed, 2, keep, Dk, &saved->qw, cells_w, st)) != NVFP4_OK)
+    return s;
+  if (n_out > 0) {
+    HpFwdArgs h{};
+    h.X = Xp; h.W = Wp; h.ldx = ldx; h.ldw = ldw; h.M = N_tok; h.N = C; h.n_out = n_out;
+    h.outl = cfg->outlier_cols; h.Y = addend; h.ldy = ld_add;
+    if (launch_hp_fwd(h, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+  }
+  saved->X = X; saved->W = W; saved->ldx = ldx; saved->ldw = ldw;
+  saved->N_tok = N_tok; saved->D = D; saved->C = C;
+  return do_gemm(&saved->qx, &saved->qw, Y, cfg->y_dtype, ldy, 0, addend, ld_add, cfg->dev_status, st);
+}
+
+nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
+                                 void* dX, int64_t lddx, void* workspace, size_t ws_bytes, void* stream) {
+  if (!dY || !saved || !dX) return NVFP4_ERR_NULL;
+  const int64_t N_tok = saved->N_tok, D = saved->D, C = saved->C;
+  if (N_tok <= 0 || D <= 0 || C <= 0) return NVFP4_ERR_SHAPE;
+  nvfp4_status s;
+  if ((s = check_cfg(cfg, D)) != NVFP4_OK) return s;
+  const int64_t n_out = cfg->n_out;
+  if ((s = check_operand_ptrs(&saved->qw)) != NVFP4_OK) return s;
+  if (saved->qw.R != C || saved->qw.K != D - n_out) return NVFP4_ERR_SHAPE;
+  if (n_out > 0 && !saved->W) return NVFP4_ERR_NULL;
+  if (bad_matrix(dY, lddy, C, 2) || bad_matrix(dX, lddx, D, cfg->dx_dtype == NVFP4_DT_F32 ? 4 : 2)) return NVFP4_ERR_ALIGN;
+  if (!workspace || ws_bytes < nvfp4_linear_workspace_bytes(NVFP4_OP_BWD_DX, N_tok, D, C, n_out, cfg->gs_mode))
+    return NVFP4_ERR_WORKSPACE;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Carver cv(workspace, ws_bytes);
+  uint32_t* cells3 = static_cast<uint32_t*>(cv.take(cells_bytes(N_tok, cfg->gs_mode)));
+  uint32_t* cells4 = static_cast<uint32_t*>(cv.take(cells_bytes(D, cfg->gs_mode)));
+  nvfp4_operand q3, q4;
+  if (!carve_operand(cv, &q3, N_tok, C, cfg->gs_mode) || !carve_operand(cv, &q4, D, C, cfg->gs_mode) || !cells3 || !cells4)
+    return NVFP4_ERR_WORKSPACE;
+  if ((s = do_quantize_rows(static_cast<const uint16_t*>(dY), N_tok, C, lddy, cfg->rounding[2], cfg->seed, 3, nullptr, 0,
+                            &q3, cells3, st)) != NVFP4_OK)
+    return s;
+  TransposeSrc ts{};
+  ts.in_codes = saved->qw.codes;
+  ts.in_sf = saved->qw.sf;
+  ts.in_gscale = saved->qw.gscale;
+  ts.in_K = saved->qw.K;
+  ts.in_gs_mode = saved->qw.gs_mode;
+  ts.in_sf_tiled = saved->qw.sf_layout == NVFP4_SF_TILED128x4;
+  if (n_out > 0) {
+    ts.row_map = cfg->col_map;
+    ts.hp = static_cast<const uint16_t*>(saved->W);
+    ts.hp_ld = saved->ldw;
+  }
+  if ((s = do_quantize_transpose(ts, 1, C, D, cfg->rounding[3], cfg->seed, 4, &q4, cells4, st)) != NVFP4_OK) return s;
+  return do_gemm(&q3, &q4, dX, cfg->dx_dtype, lddx, 0, nullptr, 0, cfg->dev_status, st);
+}
+
+nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
+                                 void* dW, int64_t lddw, void* workspace, size_t ws_bytes, void* stream) {
+  if (!dY || !saved || !dW) return NVFP4_ERR_NULL;
+  const int64_t N_tok = saved->N_tok, D = saved->D, C = saved->C;
+  if (N_tok <= 0 || D <= 0 || C <= 0) return NVFP4_ERR_SHAPE;
+  nvfp4_status s;
+  if ((s = check_cfg(cfg, D)) != NVFP4_OK) return s;
+  const int64_t n_out = cfg->n_out, Dk = D - n_out;
+  if ((s = check_operand_ptrs(&saved->qx)) != NVFP4_OK) return s;
+  if (saved->qx.R != N_tok || saved->qx.K != Dk) return NVFP4_ERR_SHAPE;
+  if (n_out > 0 && !saved->X) return NVFP4_ERR_NULL;
+  const int dw_f32 = cfg->dw_dtype == NVFP4_DT_F32;
+  if (bad_matrix(dY, lddy, C, 2) || bad_matrix(dW, lddw, D, dw_f32 ? 4 : 2)) return NVFP4_ERR_ALIGN;
+  if (!workspace || ws_bytes < nvfp4_linear_workspace_bytes(NVFP4_OP_BWD_DW, N_tok, D, C, n_out, cfg->gs_mode))
+    return NVFP4_ERR_WORKSPACE;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Carver cv(workspace, ws_bytes);
+  uint32_t* cells5 = static_cast<uint32_t*>(cv.take(cells_bytes(C, cfg->gs_mode)));
+  uint32_t* cells6 = static_cast<uint32_t*>(cv.take(cells_bytes(Dk, cfg->gs_mode)));
+  nvfp4_operand q5, q6;
+  if (!carve_operand(cv, &q5, C, N_tok, cfg->gs_mode) || !carve_operand(cv, &q6, Dk, N_tok, cfg->gs_mode) || !cells5 ||
+      !cells6)
+    return NVFP4_ERR_WORKSPACE;
+  const int64_t ld_compact = round_up(Dk, 4);
+  float* compact = n_out > 0 ? static_cast<float*>(cv.take((size_t)C * ld_compact * 4)) : nullptr;
+  if (n_out > 0 && !compact) return NVFP4_ERR_WORKSPACE;
+
+  TransposeSrc t5{};
+  t5.bf16 = static_cast<const uint16_t*>(dY);
+  t5.ld = lddy;
+  if ((s = do_quantize_transpose(t5, 0, N_tok, C, cfg->rounding[4], cfg->seed, 5, &q5, cells5, st)) != NVFP4_OK) return s;
+  TransposeSrc t6{};
+  t6.in_codes = saved->qx.codes;
+  t6.in_sf = saved->qx.sf;
+  t6.in_gscale = saved->qx.gscale;
+  t6.in_K = saved->qx.K;
+  t6.in_gs_mode = saved->qx.gs_mode;
+  t6.in_sf_tiled = saved->qx.sf_layout == NVFP4_SF_TILED128x4;
+  if ((s = do_quantize_transpose(t6, 1, N_tok, Dk, cfg->rounding[5], cfg->seed, 6, &q6, cells6, st)) != NVFP4_OK) return s;
+  if (n_out == 0) return do_gemm(&q5, &q6, dW, cfg->dw_dtype, lddw, 0, nullptr, 0, cfg->dev_status, st);
+
+  if ((s = do_gemm(&q5, &q6, compact, NVFP4_DT_F32, ld_compact, 0, nullptr, 0, cfg->dev_status, st)) != NVFP4_OK) return s;
+  if (launch_scatter_cols(compact, ld_compact, 1, dW, lddw, dw_f32, C, Dk, cfg->keep_cols, st) != cudaSuccess)
+    return NVFP4_ERR_CUDA;
+  HpDwArgs h{};
+  h.dY = static_cast<const uint16_t*>(dY); h.X = static_cast<const uint16_t*>(saved->X);
+  h.lddy = lddy; h.ldx = saved->ldx; h.T = N_tok; h.C = C; h.n_out = n_out; h.outl = cfg->outlier_cols;
+  h.dW = dW; h.dw_is_f32 = dw_f32; h.lddw = lddw;
+  return launch_hp_dw(h, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,480 @@
+// Block-scaled FP4 GEMM for sm_100a (the "FP4 MM" of the paper's Sec. 2.3):
+//     C[m, n] = sum_k (Pa Sba Sga)[m, k] (Pb Sbb Sgb)[n, k],  both operands packed along k.
+//
+// Design (one CTA per SM, persistent over output tiles, warp-specialised):
+//   warp 0      TMA producer: per 256-wide k tile, two tiled bulk-tensor loads (A, B codes; 128-byte swizzle) and
+//               two plain bulk copies (the 2 KB of E4M3 scales each operand tile needs, contiguous in the
+//               TILED128x4 layout) into a ring of shared-memory stages, completion on an mbarrier.
+//   warp 1      MMA issuer: copies the scales shared -> tensor memory (tcgen05.cp) and issues
+//               tcgen05.mma kind::mxf4nvf4 block_scale (E2M1 data, UE4M3 scale per 16 elements, K = 64 per
+//               instruction, FP32 accumulators in tensor memory, two accumulator buffers).
+//   warps 2..5  epilogue: tcgen05.ld the accumulator, apply the FP32 global scales, add the optional addend,
+//               convert and store.
+// Every wait on an mbarrier is bounded; when a bound is hit the kernel raises a status word, all roles drain and
+// the CTA frees its tensor memory and exits.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "nvfp4_device.cuh"
+#include "nvfp4_internal.h"
+
+namespace nvfp4 {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 256;                                  // elements per k tile = one 128-byte swizzle row
+constexpr uint32_t A_BYTES = BM * BK / 2;                // 16 KB
+constexpr uint32_t SFA_BYTES = 2048;                     // 128 rows x 16 k-blocks
+constexpr int NUM_THREADS = 192;
+constexpr int EPI_WARP0 = 2;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;    // ~2 s
+
+template <int BN>
+struct Cfg {
+  static constexpr uint32_t B_BYTES = BN * BK / 2;
+  static constexpr uint32_t SFB_BYTES = (BN / 128) * 2048;
+  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;  // multiple of 1024
+  static constexpr int STAGES = (BN == 128) ? 5 : 4;
+  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
+  // tensor memory columns: two accumulators, then two scale buffers (A: 16 columns, B: 16 * BN / 128)
+  static constexpr uint32_t ACC_COLS = BN;
+  static constexpr uint32_t SF_COLS = 16 + 16 * (BN / 128);
+  static constexpr uint32_t TMEM_COLS = 512;
+  static_assert(2 * ACC_COLS + 2 * SF_COLS <= TMEM_COLS || BN == 256, "tensor memory budget");
+};
+
+struct Params {
+  const uint8_t* a_sf;
+  const uint8_t* b_sf;
+  const float* a_gscale;
+  const float* b_gscale;
+  const float* addend;  // optional FP32 [M, N] (leading dimension ld_add) added before the store
+  int64_t ld_add;
+  void* C;
+  int64_t ldc;
+  int64_t M, N;
+  int32_t k_tiles;        // number of 256-wide k tiles
+  int32_t sf_tiles_a;     // 512-byte scale tiles per 128-row tile of A (= padded k-blocks / 4)
+  int32_t sf_tiles_b;
+  int32_t m_tiles, n_tiles;
+  int32_t c_is_f32, accumulate;
+  int32_t* dev_status;
+};
+
+// ---------------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait. Returns false when the bound ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+    if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+      *abort_flag = 1;
+      if (dev_status) atomicExch(dev_status, 8 /* NVFP4_ERR_TIMEOUT */);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int32_t c0, int32_t c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(tm), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (start address, leading / stride byte offsets in 16-byte units, version 1).
+// Code tiles: k-major rows of 128 bytes with the 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t desc_sw128(uint32_t saddr) {
+  return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)1 << 16) | ((uint64_t)64 << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+// Scale tiles: 32 rows of 16 bytes, unswizzled, 8-row groups 128 bytes apart.
+__device__ __forceinline__ uint64_t desc_sf(uint32_t saddr) {
+  return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)8 << 32) | ((uint64_t)1 << 46);
+}
+// Instruction descriptor: E2M1 x E2M1, UE4M3 scales, M = 128, N = BN, both operands k-major, K = 64.
+template <int BN>
+__device__ __forceinline__ uint32_t instr_desc() {
+  return (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (0u << 23) | ((uint32_t)(BM >> 4) << 24);
+}
+
+template <int GS, int BN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
+  using C = Cfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = smem_base + C::STAGES * C::STAGE_BYTES;
+  // barriers: full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], drain
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };
+  auto acc_full_bar = [&](int b) { return bar_base + 8u * (2 * C::STAGES + b); };
+  auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * C::STAGES + 2 + b); };
+  const uint32_t drain_bar = bar_base + 8u * (2 * C::STAGES + 4);
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    for (int s = 0; s < C::STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(acc_full_bar(b), 1);
+      mbar_init(acc_empty_bar(b), 4);
+    }
+    mbar_init(drain_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                 "r"(C::TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  const int64_t num_tiles = (int64_t)p.m_tiles * p.n_tiles;
+
+  if (warp == 0) {
+    // ===================================== TMA producer ====================================================
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
+        const uint8_t* sfa_src = p.a_sf + (size_t)mt * p.sf_tiles_a * 512;
+        const uint8_t* sfb_src = p.b_sf + (size_t)nt * (BN / 128) * p.sf_tiles_b * 512;
+        for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
+          const int s = it % C::STAGES;
+          const uint32_t round = it / C::STAGES;
+          if (!(ok = mbar_wait(empty_bar(s), (round & 1) ^ 1, abort_flag, p.dev_status))) break;
+          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+          mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
+          tma_load_2d(st, &tmA, kt * (BK / 2), mt * BM, full_bar(s));
+          tma_load_2d(st + A_BYTES, &tmB, kt * (BK / 2), nt * BN, full_bar(s));
+          bulk_load(st + A_BYTES + C::B_BYTES, sfa_src + (size_t)kt * 2048, 2048, full_bar(s));
+#pragma unroll
+          for (int h = 0; h < BN / 128; ++h)
+            bulk_load(st + A_BYTES + C::B_BYTES + SFA_BYTES + h * 2048,
+                      sfb_src + ((size_t)h * p.sf_tiles_b * 512) + (size_t)kt * 2048, 2048, full_bar(s));
+        }
+      }
+      if (!ok) {
+        // give the copies already in flight a bounded time to land before the CTA may exit
+        const uint32_t n_back = it < (uint32_t)C::STAGES ? it : (uint32_t)C::STAGES;
+        for (uint32_t j = 0; j < n_back; ++j) {
+          const uint32_t f = it - 1 - j;
+          const long long t0 = clock64();
+          while (!mbar_try(full_bar(f % C::STAGES), (f / C::STAGES) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================================== MMA issuer ======================================================
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc<BN>();
+      uint32_t it = 0, tile_it = 0;
+      bool ok = true;
+      for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
+        const uint32_t ab = tile_it & 1;
+        if (!(ok = mbar_wait(acc_empty_bar(ab), ((tile_it >> 1) & 1) ^ 1, abort_flag, p.dev_status))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + ab * C::ACC_COLS;
+        for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
+          const int s = it % C::STAGES;
+          if (!(ok = mbar_wait(full_bar(s), (it / C::STAGES) & 1, abort_flag, p.dev_status))) break;
+          tc_fence_after();
+          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+          const uint32_t sf_tmem = tmem_base + 2 * C::ACC_COLS + (it & 1) * C::SF_COLS;
+#pragma unroll
+          for (int kk = 0; kk < BK / 64; ++kk) {
+            // scales of this 64-wide k step: 4 columns for 128 rows of A, 4 per 128 rows of B
+            tc_cp_sf(sf_tmem + kk * 4, desc_sf(st + A_BYTES + C::B_BYTES + kk * 512));
+#pragma unroll
+            for (int h = 0; h < BN / 128; ++h)
+              tc_cp_sf(sf_tmem + 16 + (kk * (BN / 128) + h) * 4,
+                       desc_sf(st + A_BYTES + C::B_BYTES + SFA_BYTES + h * 2048 + kk * 512));
+            tc_mma_nvf4(d_tmem, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc, sf_tmem + kk * 4,
+                        sf_tmem + 16 + kk * (BN / 128) * 4, (kt | kk) != 0);
+          }
+          tc_commit(empty_bar(s));  // stage reusable once these MMAs have read it
+        }
+        if (ok) tc_commit(acc_full_bar(ab));
+      }
+      // make sure nothing issued is still running before tensor memory is freed
+      tc_commit(drain_bar);
+      {
+        const long long t0 = clock64();
+        while (!mbar_try(drain_bar, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
+        }
+      }
+    }
+  } else {
+    // ===================================== epilogue ========================================================
+    const int quad = warp & 3;  // tensor-memory lane quadrant this warp may read
+    uint32_t tile_it = 0;
+    bool ok = true;
+    float alpha = 1.0f;
+    if (GS == kGsTensor) alpha = __fmul_rn(p.a_gscale[0], p.b_gscale[0]);
+    for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
+      const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
+      const uint32_t ab = tile_it & 1;
+      if (!(ok = mbar_wait(acc_full_bar(ab), (tile_it >> 1) & 1, abort_flag, p.dev_status))) break;
+      tc_fence_after();
+      const int64_t m = (int64_t)mt * BM + quad * 32 + lane;
+      float sa = 1.0f;
+      if (GS == kGsRow && m < p.M) sa = p.a_gscale[m];
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t v[32];
+        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + c0, v);
+        tc_wait_ld();
+        const int64_t n0 = (int64_t)nt * BN + c0;
+        if (m < p.M && n0 < p.N) {
+          float o[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            float sc = alpha;
+            if (GS == kGsRow) sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
+            o[j] = __uint_as_float(v[j]) * sc;
+          }
+          if (p.addend) {
+            const float* ad = p.addend + m * p.ld_add + n0;
+            if (n0 + 32 <= p.N) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                const float4 q = *reinterpret_cast<const float4*>(ad + j);
+                o[j] += q.x; o[j + 1] += q.y; o[j + 2] += q.z; o[j + 3] += q.w;
+              }
+            } else {
+              for (int j = 0; j < 32 && n0 + j < p.N; ++j) o[j] += ad[j];
+            }
+          }
+          if (p.c_is_f32) {
+            float* cp = reinterpret_cast<float*>(p.C) + m * p.ldc + n0;
+            if (n0 + 32 <= p.N) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                float4 q = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+                if (p.accumulate) {
+                  const float4 old = *reinterpret_cast<const float4*>(cp + j);
+                  q.x += old.x; q.y += old.y; q.z += old.z; q.w += old.w;
+                }
+                *reinterpret_cast<float4*>(cp + j) = q;
+              }
+            } else {
+              for (int j = 0; j < 32 && n0 + j < p.N; ++j) cp[j] = p.accumulate ? cp[j] + o[j] : o[j];
+            }
+          } else {
+            __nv_bfloat16* cp = reinterpret_cast<__nv_bfloat16*>(p.C) + m * p.ldc + n0;
+            if (n0 + 32 <= p.N) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                if (p.accumulate) {
+                  const uint4 old = *reinterpret_cast<const uint4*>(cp + j);
+                  const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) {
+                    o[j + 2 * q] += bf16_lo(ow[q]);
+                    o[j + 2 * q + 1] += bf16_hi(ow[q]);
+                  }
+                }
+                uint4 q;
+                __nv_bfloat162 h;
+                h = __floats2bfloat162_rn(o[j], o[j + 1]); q.x = *reinterpret_cast<uint32_t*>(&h);
+                h = __floats2bfloat162_rn(o[j + 2], o[j + 3]); q.y = *reinterpret_cast<uint32_t*>(&h);
+                h = __floats2bfloat162_rn(o[j + 4], o[j + 5]); q.z = *reinterpret_cast<uint32_t*>(&h);
+                h = __floats2bfloat162_rn(o[j + 6], o[j + 7]); q.w = *reinterpret_cast<uint32_t*>(&h);
+                *reinterpret_cast<uint4*>(cp + j) = q;
+              }
+            } else {
+              for (int j = 0; j < 32 && n0 + j < p.N; ++j) {
+                const float prev = p.accumulate ? __bfloat162float(cp[j]) : 0.0f;
+                cp[j] = __float2bfloat16_rn(o[j] + prev);
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty_bar(ab));
+    }
+  }
+
+  // ===================================== teardown ============================================================
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::TMEM_COLS) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// Codes of an operand [R, Kp/2 bytes] as a 2-D byte tensor; box = 128 bytes x box_rows; out-of-range reads give 0.
+bool make_codes_map(CUtensorMap* tm, const uint8_t* codes, int64_t R, int64_t Kp, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)(Kp / 2), (cuuint64_t)R};
+  const cuuint64_t strides[1] = {(cuuint64_t)(Kp / 2)};
+  const cuuint32_t box[2] = {128, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(codes), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+  }
+  return n;
+}
+
+template <int GS, int BN>
+cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
+  using C = Cfg<BN>;
+  const int64_t Kp = (a.K + 127) & ~(int64_t)127;
+  CUtensorMap tmA, tmB;
+  if (!make_codes_map(&tmA, a.a_codes, a.M, Kp, BM) || !make_codes_map(&tmB, a.b_codes, a.N, Kp, BN))
+    return cudaErrorInvalidValue;
+  Params p{};
+  p.a_sf = a.a_sf;
+  p.b_sf = a.b_sf;
+  p.a_gscale = a.a_gscale;
+  p.b_gscale = a.b_gscale;
+  p.addend = a.addend;
+  p.ld_add = a.ld_add;
+  p.C = a.C;
+  p.ldc = a.ldc;
+  p.M = a.M;
+  p.N = a.N;
+  p.k_tiles = (int32_t)((Kp + BK - 1) / BK);
+  const int64_t kb_padded = ((Kp >> 4) + 15) & ~(int64_t)15;
+  p.sf_tiles_a = p.sf_tiles_b = (int32_t)(kb_padded >> 2);
+  p.m_tiles = (int32_t)((a.M + BM - 1) / BM);
+  p.n_tiles = (int32_t)((a.N + BN - 1) / BN);
+  p.c_is_f32 = a.c_is_f32;
+  p.accumulate = a.accumulate;
+  p.dev_status = a.dev_status;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_kernel<GS, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)C::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
+  const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
+  gemm_nvfp4_kernel<GS, BN><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(tmA, tmB, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+size_t gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
+
+cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
+  if (a.M == 0 || a.N == 0) return cudaSuccess;
+  switch (a.gs_mode) {
+    case kGsTensor: return launch_variant<kGsTensor, 128>(a, st);
+    case kGsRow: return launch_variant<kGsRow, 128>(a, st);
+    default: return cudaErrorNotSupported;
+  }
+}
+
+}  // namespace nvfp4

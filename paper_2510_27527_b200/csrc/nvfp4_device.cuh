@@ -1,0 +1,157 @@
+// Device-side building blocks of the NVFP4 quantizers: format conversions, the element rounding rules and the
+// counter-based random generator. Everything that can change a code or a scale is an explicit IEEE binary32
+// operation (__fdiv_rn / __fmul_rn, no fast-math, no contraction), in the order the quantizer's contract fixes.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace nvfp4 {
+
+constexpr int kRoundRTN = 0;
+constexpr int kRoundSR = 1;
+constexpr int kGsTensor = 0;
+constexpr int kGsRow = 1;
+constexpr int kGsBlock128 = 2;
+constexpr int kSfLinear = 0;
+constexpr int kSfTiled = 1;
+
+// ---------------------------------------------------------------------------------------------------------
+// BF16 pairs packed in a 32-bit word
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+// |x| of both halves as 16-bit patterns; for finite BF16 the pattern order is the value order.
+__device__ __forceinline__ uint32_t bf16x2_abs_bits(uint32_t w) { return w & 0x7FFF7FFFu; }
+__device__ __forceinline__ uint32_t umax16x2(uint32_t a, uint32_t b) { return __vmaxu2(a, b); }
+__device__ __forceinline__ uint32_t hmax_of_pair(uint32_t m) { return max(m & 0xFFFFu, m >> 16); }
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b16) { return __uint_as_float(b16 << 16); }
+
+// FP32 -> BF16 bit pattern, round to nearest even (finite inputs).
+__device__ __forceinline__ uint16_t f32_to_bf16_bits(float v) {
+  const uint32_t b = __float_as_uint(v);
+  return (uint16_t)((b + 0x7FFFu + ((b >> 16) & 1u)) >> 16);
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// E4M3 (bias 7, max 448, no infinity): block scales
+// ---------------------------------------------------------------------------------------------------------
+// Non-negative float -> E4M3 byte: round to nearest, ties to even, saturate to 448.
+__device__ __forceinline__ uint32_t e4m3_encode(float s) {
+  uint16_t packed;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(packed) : "f"(0.0f), "f"(s));
+  return packed & 0xFFu;
+}
+// E4M3 byte -> float (exact).
+__device__ __forceinline__ float e4m3_decode(uint32_t byte) {
+  uint32_t h2;
+  asm("{.reg .b16 t; cvt.u16.u32 t, %1; cvt.rn.f16x2.e4m3x2 %0, t;}" : "=r"(h2) : "r"(byte & 0xFFu));
+  return __half2float(__ushort_as_half((unsigned short)(h2 & 0xFFFFu)));
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Scales of the double-block quantizer (paper Sec. 2.2): the pinned operation sequence.
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float global_scale_from_amax(float amax) {
+  return amax == 0.0f ? 1.0f : __fdiv_rn(amax, 2688.0f);  // 448 * 6
+}
+// Returns the E4M3 byte of the block scale and the reciprocal r that maps x to the FP4 grid (0 if the scale is 0).
+__device__ __forceinline__ uint32_t block_scale(float amax_b, float Sg, float& rcp) {
+  const float t = __fdiv_rn(amax_b, Sg);
+  const float s = __fdiv_rn(t, 6.0f);
+  const uint32_t sb = e4m3_encode(s);
+  const float Sbf = e4m3_decode(sb);
+  const float d = __fmul_rn(Sg, Sbf);
+  rcp = (Sbf == 0.0f) ? 0.0f : __fdiv_rn(1.0f, d);
+  return sb;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Philox4x32-10
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                               uint32_t k1) {
+#pragma unroll
+  for (int i = 0; i < 10; ++i) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0;
+    const uint32_t n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+// The four 32-bit words holding the 16-bit draws of elements idx8*8 .. idx8*8+7 of the operand.
+__device__ __forceinline__ uint4 sr_words(uint64_t seed, uint32_t stream_id, uint64_t idx8) {
+  return philox4x32_10((uint32_t)idx8, (uint32_t)(idx8 >> 32), stream_id, 0u, (uint32_t)seed,
+                       (uint32_t)(seed >> 32));
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Element rounding to E2M1 (paper Sec. 2.1). Codes: sign << 3 | magnitude index.
+// ---------------------------------------------------------------------------------------------------------
+// Stochastic rounding of one scaled value with a 16-bit draw u. Exact: the comparison
+//   (u + 0.5) / 65536 < (a - q1) / (q2 - q1)
+// is evaluated on integers (a >= 1, where the fraction is the low 22 mantissa bits) or on exactly
+// representable floats (a < 1, where the grid step is 0.5).
+__device__ __forceinline__ uint32_t e2m1_sr(float y, uint32_t u) {
+  const float a = fminf(fabsf(y), 6.0f);
+  const uint32_t bits = __float_as_uint(a);
+  const uint32_t t = 2u * u + 1u;
+  uint32_t idx, up;
+  if (a >= 1.0f) {
+    idx = (bits >> 22) - 252u;  // 1 -> 2, 1.5 -> 3, 2 -> 4, 3 -> 5, 4 -> 6, 6 -> 7
+    up = (t << 5) < (bits & 0x3FFFFFu);
+  } else {
+    idx = a >= 0.5f;
+    up = (float)t < (a - 0.5f * (float)idx) * 262144.0f;
+  }
+  return (idx + up) | ((__float_as_uint(y) >> 28) & 8u);
+}
+
+// Round-to-nearest (ties to the even code, saturating) of 8 scaled values, packed low nibble first.
+__device__ __forceinline__ uint32_t e2m1x8_rtn(const float (&y)[8]) {
+  uint32_t out;
+  asm("{\n"
+      ".reg .b8 b0, b1, b2, b3;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n"
+      "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n"
+      "mov.b32 %0, {b0, b1, b2, b3};\n"
+      "}"
+      : "=r"(out)
+      : "f"(y[0]), "f"(y[1]), "f"(y[2]), "f"(y[3]), "f"(y[4]), "f"(y[5]), "f"(y[6]), "f"(y[7]));
+  return out;
+}
+
+// Stochastic rounding of 8 scaled values with the draws packed in w (two 16-bit draws per word).
+__device__ __forceinline__ uint32_t e2m1x8_sr(const float (&y)[8], const uint4& w) {
+  const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+  uint32_t out = 0;
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const uint32_t u = (ww[e >> 1] >> (16 * (e & 1))) & 0xFFFFu;
+    out |= e2m1_sr(y[e], u) << (4 * e);
+  }
+  return out;
+}
+
+// E2M1 code -> value, as float.
+__device__ __forceinline__ float e2m1_decode(uint32_t code) {
+  const uint32_t m = code & 7u;
+  // magnitudes 0, .5, 1, 1.5, 2, 3, 4, 6: exponent field e = m >> 1, mantissa bit m & 1
+  const uint32_t e = m >> 1, f = m & 1u;
+  const uint32_t bits = (e == 0) ? (f ? 0x3F000000u : 0u) : (((126u + e) << 23) | (f << 22));
+  return __uint_as_float(bits | ((code & 8u) << 28));
+}
+
+// Byte offset of scale (r, kb) in the TILED128x4 layout with n_ktiles4 = (number of k-blocks, padded to 16) / 4.
+__device__ __forceinline__ size_t sf_tiled_offset(int64_t r, int64_t kb, int64_t kb_padded) {
+  const int64_t tile = (r >> 7) * (kb_padded >> 2) + (kb >> 2);
+  return (size_t)tile * 512 + (size_t)((r & 31) * 16 + ((r >> 5) & 3) * 4 + (kb & 3));
+}
+
+}  // namespace nvfp4

@@ -1,0 +1,101 @@
+// Internal (non-ABI) declarations shared by the library's translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <algorithm>
+
+namespace nvfp4 {
+
+struct QuantRowsArgs {
+  const uint16_t* src;  // BF16 [rows, cols_src], leading dimension ld
+  int64_t rows, K, cols_src, ld;
+  const int32_t* keep;  // optional column list of length K
+  uint64_t seed;
+  uint32_t stream_id;
+  int gs_mode, sr, sf_tiled;
+  int compute_amax;    // TENSOR mode: run the amax pre-pass (0: gs_cells[0] already holds the amax bits)
+  uint32_t* gs_cells;  // workspace: 1 cell (TENSOR) or `rows` cells (ROW)
+  uint8_t* codes;
+  uint8_t* sf;
+  float* gscale;
+};
+
+// Source of a transposing quantizer. Operand element (d, k) = source element (row k, column d).
+struct TransposeSrc {
+  // from BF16: matrix [rowsK, D], leading dimension ld
+  const uint16_t* bf16;
+  int64_t ld;
+  // from a forward operand [rowsK, in_K] (codes + scales + global scales), optionally remapped per d and
+  // mixed with the BF16 matrix hp for the rows whose map entry is negative
+  const uint8_t* in_codes;
+  const uint8_t* in_sf;
+  const float* in_gscale;
+  int64_t in_K;
+  int32_t in_gs_mode, in_sf_tiled;
+  const int32_t* row_map;  // [D] or null
+  const uint16_t* hp;      // BF16 [rowsK, >= D]
+  int64_t hp_ld;
+};
+
+struct QuantTransposeArgs {
+  int from_codes;
+  int64_t rowsK, D;  // operand [D, rowsK] = transpose of a [rowsK, D] source
+  TransposeSrc src;
+  uint64_t seed;
+  uint32_t stream_id;
+  int gs_mode, sr, sf_tiled;
+  int compute_amax;
+  uint32_t* gs_cells;  // 1 cell (TENSOR) or D cells (ROW)
+  uint8_t* codes;
+  uint8_t* sf;
+  float* gscale;
+};
+
+cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st);
+cudaError_t launch_quantize_transpose(const QuantTransposeArgs& a, cudaStream_t st);
+
+struct GemmArgs {
+  const uint8_t *a_codes, *a_sf, *b_codes, *b_sf;
+  const float *a_gscale, *b_gscale;
+  int64_t M, N, K;  // logical sizes; operand buffers are padded as the ABI header says
+  int gs_mode;
+  void* C;
+  int c_is_f32;
+  int64_t ldc;
+  int accumulate;
+  const float* addend;  // optional FP32 [M, N] added in the epilogue (leading dimension ld_add)
+  int64_t ld_add;
+  int32_t* dev_status;
+  void* workspace;
+  size_t ws_bytes;
+};
+size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
+
+// High-precision (BF16 inputs, FP32 accumulate) products over OutControl's outlier channels.
+//   fwd: Y[m, n] (+)= sum_j X[m, outl[j]] * W[n, outl[j]]
+//   dw : dW[c, outl[j]] = sum_t dY[t, c] * X[t, outl[j]]
+struct HpFwdArgs {
+  const uint16_t *X, *W;
+  int64_t ldx, ldw, M, N, n_out;
+  const int32_t* outl;
+  float* Y;  // FP32 [M, N], overwritten
+  int64_t ldy;
+};
+struct HpDwArgs {
+  const uint16_t *dY, *X;
+  int64_t lddy, ldx, T, C, n_out;
+  const int32_t* outl;
+  void* dW;
+  int dw_is_f32;
+  int64_t lddw;
+};
+cudaError_t launch_hp_fwd(const HpFwdArgs& a, cudaStream_t st);
+cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st);
+
+// Scatter a compact [C, n_keep] matrix into columns keep[j] of dW [C, D].
+cudaError_t launch_scatter_cols(const void* src, int64_t ld_src, int src_is_f32, void* dst, int64_t ld_dst,
+                                int dst_is_f32, int64_t rows, int64_t n_keep, const int32_t* keep, cudaStream_t st);
+
+}  // namespace nvfp4

@@ -1,0 +1,430 @@
+// Quantize kernels of the NVFP4 linear layer (paper Sec. 2.2 double-block quantization, Sec. 2.1 rounding):
+//   - amax pre-passes (whole tensor, per source row, per source column) for the TENSOR and ROW scale modes;
+//   - row-axis quantize from BF16 (Q1, Q2, Q3 of Sec. 2.3): one thread per 16-element inner block;
+//   - transposing quantize (Q5 from BF16; Q4, Q6 from the forward operand's codes, i.e. from X-hat / W-hat):
+//     a 128(k) x 64(operand rows) tile is staged in shared memory as FP32 and read back column-wise.
+// All of them are HBM streaming kernels; the launch wrappers at the bottom are called by the C-ABI layer.
+#include "nvfp4_device.cuh"
+#include "nvfp4_internal.h"
+
+namespace nvfp4 {
+
+// =========================================================================================================
+// amax pre-passes. Results are bit patterns of non-negative floats combined with atomicMax (order-free, hence
+// deterministic). The cells must be zero before the launch.
+// =========================================================================================================
+__global__ void __launch_bounds__(256) amax_tensor_bf16_kernel(const uint16_t* __restrict__ src, int64_t rows,
+                                                              int64_t cols, int64_t ld, uint32_t* amax_bits) {
+  // One 16-byte chunk (8 BF16) per thread per step; rows are walked through a flattened chunk index.
+  const int64_t chunks_per_row = (cols + 7) >> 3;
+  const int64_t total = rows * chunks_per_row;
+  uint32_t m = 0;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / chunks_per_row, c = (i - r * chunks_per_row) << 3;
+    const uint16_t* p = src + r * ld + c;
+    if (c + 8 <= cols) {
+      const uint4 v = *reinterpret_cast<const uint4*>(p);
+      m = umax16x2(m, umax16x2(umax16x2(bf16x2_abs_bits(v.x), bf16x2_abs_bits(v.y)),
+                               umax16x2(bf16x2_abs_bits(v.z), bf16x2_abs_bits(v.w))));
+    } else {
+      for (int64_t j = c; j < cols; ++j) m = umax16x2(m, (uint32_t)(p[j - c] & 0x7FFFu));
+    }
+  }
+  uint32_t a = hmax_of_pair(m);
+#pragma unroll
+  for (int o = 16; o; o >>= 1) a = max(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
+  __shared__ uint32_t warp_max[8];
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = a;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) a = max(a, warp_max[w]);
+    if (a) atomicMax(amax_bits, a << 16);  // BF16 pattern -> FP32 pattern
+  }
+}
+
+// amax of each source row over the kept columns -> cells[row] (ROW scale mode of the row-axis quantizer).
+__global__ void __launch_bounds__(256) amax_rows_bf16_kernel(const uint16_t* __restrict__ src, int64_t rows,
+                                                            int64_t cols, int64_t ld,
+                                                            const int32_t* __restrict__ keep, int64_t n_keep,
+                                                            uint32_t* cells, int single_cell) {
+  const int64_t r = blockIdx.x;
+  const uint16_t* p = src + r * ld;
+  uint32_t m = 0;
+  if (keep) {
+    for (int64_t j = threadIdx.x; j < n_keep; j += blockDim.x) m = max(m, (uint32_t)(p[keep[j]] & 0x7FFFu));
+  } else {
+    const int64_t nchunk = cols >> 3;
+    for (int64_t c = threadIdx.x; c < nchunk; c += blockDim.x) {
+      const uint4 v = *reinterpret_cast<const uint4*>(p + (c << 3));
+      m = umax16x2(m, umax16x2(umax16x2(bf16x2_abs_bits(v.x), bf16x2_abs_bits(v.y)),
+                               umax16x2(bf16x2_abs_bits(v.z), bf16x2_abs_bits(v.w))));
+    }
+    for (int64_t j = (nchunk << 3) + threadIdx.x; j < cols; j += blockDim.x) m = umax16x2(m, (uint32_t)(p[j] & 0x7FFFu));
+    m = hmax_of_pair(m);
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  __shared__ uint32_t warp_max[8];
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) m = max(m, warp_max[w]);
+    if (single_cell) {
+      if (m) atomicMax(cells, m << 16);
+    } else {
+      cells[r] = m << 16;
+    }
+  }
+}
+
+// =========================================================================================================
+// Shared epilogue of one 16-element inner block: scale, round, pack.
+// =========================================================================================================
+template <bool SR>
+__device__ __forceinline__ uint2 quantize_block16(const float (&x)[16], float rcp, uint64_t seed, uint32_t stream_id,
+                                                  uint64_t idx8) {
+  float y0[8], y1[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    y0[i] = __fmul_rn(x[i], rcp);
+    y1[i] = __fmul_rn(x[8 + i], rcp);
+  }
+  uint2 out;
+  if (SR) {
+    out.x = e2m1x8_sr(y0, sr_words(seed, stream_id, idx8));
+    out.y = e2m1x8_sr(y1, sr_words(seed, stream_id, idx8 + 1));
+  } else {
+    out.x = e2m1x8_rtn(y0);
+    out.y = e2m1x8_rtn(y1);
+  }
+  return out;
+}
+
+// =========================================================================================================
+// Row-axis quantize from BF16: one thread per inner block, eight neighbouring threads per 128-wide outer block.
+//   GS      scale mode. TENSOR reads the amax cell gs_cells[0]; ROW reads gs_cells[row]; BLOCK128 reduces the
+//           group amax over the 8 threads of the group with shuffles (single pass over the data).
+//   GATHER  columns come from the list `keep` (OutControl compaction) instead of 0..cols-1.
+// =========================================================================================================
+template <int GS, bool SR, bool TILED, bool GATHER>
+__global__ void __launch_bounds__(256)
+quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, int64_t ld,
+                     const int32_t* __restrict__ keep, uint64_t seed, uint32_t stream_id,
+                     const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
+                     float* __restrict__ gscale) {
+  const int64_t Kp = (K + 127) & ~(int64_t)127;
+  const int64_t nb = Kp >> 4;  // inner blocks per operand row (multiple of 8)
+  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t total = rows * nb;
+  const bool active = gid < total;
+  const int64_t r = active ? gid / nb : 0;
+  const int64_t b = active ? gid - r * nb : 0;
+  const int64_t k0 = b << 4;
+
+  // ---- load 16 elements (zero beyond K) -----------------------------------------------------------------
+  uint32_t w[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) w[i] = 0;
+  if (active && k0 < K) {
+    const uint16_t* p = src + r * ld;
+    if (!GATHER && k0 + 16 <= K) {
+      const uint4 v0 = *reinterpret_cast<const uint4*>(p + k0);
+      const uint4 v1 = *reinterpret_cast<const uint4*>(p + k0 + 8);
+      w[0] = v0.x; w[1] = v0.y; w[2] = v0.z; w[3] = v0.w;
+      w[4] = v1.x; w[5] = v1.y; w[6] = v1.z; w[7] = v1.w;
+    } else {
+      for (int i = 0; i < 16; ++i) {
+        if (k0 + i < K) {
+          const uint32_t e = GATHER ? p[keep[k0 + i]] : p[k0 + i];
+          w[i >> 1] |= e << (16 * (i & 1));
+        }
+      }
+    }
+  }
+  uint32_t m2 = 0;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) m2 = umax16x2(m2, bf16x2_abs_bits(w[i]));
+  const uint32_t amax_b_bits = hmax_of_pair(m2);
+
+  // ---- global scale ---------------------------------------------------------------------------------------
+  float Sg;
+  if (GS == kGsBlock128) {
+    uint32_t g = amax_b_bits;
+    g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
+    g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
+    g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 4));
+    Sg = global_scale_from_amax(bf16_bits_to_float(g));
+    if (active && (b & 7) == 0) gscale[r * (Kp >> 7) + (b >> 3)] = Sg;
+  } else if (GS == kGsRow) {
+    Sg = global_scale_from_amax(__uint_as_float(gs_cells[r]));
+    if (active && b == 0) gscale[r] = Sg;
+  } else {
+    Sg = global_scale_from_amax(__uint_as_float(gs_cells[0]));
+    if (gid == 0) gscale[0] = Sg;
+  }
+
+  // ---- block scale, rounding, packing -------------------------------------------------------------------
+  float rcp;
+  const uint32_t sb = block_scale(bf16_bits_to_float(amax_b_bits), Sg, rcp);
+  float x[16];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    x[2 * i] = bf16_lo(w[i]);
+    x[2 * i + 1] = bf16_hi(w[i]);
+  }
+  const int64_t K16 = (K + 15) & ~(int64_t)15;
+  const uint2 packed = quantize_block16<SR>(x, rcp, seed, stream_id, (uint64_t)((r * K16 + k0) >> 3));
+
+  // four neighbouring threads own the four scale bytes of one 32-bit word in either layout
+  uint32_t sf4 = sb << (8 * (b & 3));
+  sf4 |= __shfl_xor_sync(0xFFFFFFFFu, sf4, 1);
+  sf4 |= __shfl_xor_sync(0xFFFFFFFFu, sf4, 2);
+  if (!active) return;
+  *reinterpret_cast<uint2*>(codes + r * (Kp >> 1) + (k0 >> 1)) = packed;
+  if ((b & 3) == 0) {
+    const size_t off = TILED ? sf_tiled_offset(r, b, (nb + 15) & ~(int64_t)15) : (size_t)(r * nb + b);
+    *reinterpret_cast<uint32_t*>(sf + off) = sf4;
+  }
+}
+
+// =========================================================================================================
+// Transposing quantizers. Operand element (d, k) = source element (row k, column d).
+// Tile = 128 k x 64 d. Phase 1 stages the tile as FP32 in shared memory; phase 2 gives each thread one
+// (d, 16-k block); phase 3 writes the packed rows back in 16-byte pieces.
+//   SRC = 0: BF16 source matrix [rowsK, colsD] (Q5).
+//   SRC = 1: forward operand [rowsK, Kin] as codes + scales + global scales, optionally remapped per d and
+//            mixed with a BF16 matrix for the rows whose map entry is negative (Q4, Q6 of Sec. 2.3 / 4.2).
+// =========================================================================================================
+__device__ __forceinline__ float load_aligned_value(const TransposeSrc& s, int64_t k, int64_t j) {
+  // x_hat = (P * S_block) * S_global of input operand element (row k, column j): one binary32 rounding.
+  const int64_t Kp = (s.in_K + 127) & ~(int64_t)127;
+  const uint32_t byte = s.in_codes[k * (Kp >> 1) + (j >> 1)];
+  const uint32_t code = (byte >> (4 * (j & 1))) & 15u;
+  const int64_t nb = Kp >> 4;
+  const size_t sfo = s.in_sf_tiled ? sf_tiled_offset(k, j >> 4, (nb + 15) & ~(int64_t)15) : (size_t)(k * nb + (j >> 4));
+  const float sbf = e4m3_decode(s.in_sf[sfo]);
+  const float sg = s.in_gs_mode == kGsTensor ? s.in_gscale[0]
+                   : s.in_gs_mode == kGsRow  ? s.in_gscale[k]
+                                             : s.in_gscale[k * (Kp >> 7) + (j >> 7)];
+  return __fmul_rn(__fmul_rn(e2m1_decode(code), sbf), sg);
+}
+
+template <int SRC>
+__device__ __forceinline__ float load_transpose_elem(const TransposeSrc& s, int64_t k, int64_t d) {
+  if (SRC == 0) return bf16_bits_to_float(s.bf16[k * s.ld + d]);
+  int64_t j = d;
+  if (s.row_map) {
+    const int32_t mj = s.row_map[d];
+    if (mj < 0) return bf16_bits_to_float(s.hp[k * s.hp_ld + d]);
+    j = mj;
+  }
+  return load_aligned_value(s, k, j);
+}
+
+// Column amax of the aligned tensor (ROW scale mode of Q4 / Q6) and of its high-precision rows; also used for
+// TENSOR mode when a row map mixes BF16 rows in (cells has one entry then).
+template <int SRC>
+__global__ void __launch_bounds__(256) amax_cols_generic_kernel(TransposeSrc s, int64_t rowsK, int64_t D,
+                                                               uint32_t* cells, int per_column) {
+  const int64_t d = (int64_t)blockIdx.x * 64 + (threadIdx.x & 63);
+  const int64_t r0 = (int64_t)blockIdx.y * 256;
+  if (d >= D) return;
+  float m = 0.0f;
+  for (int64_t k = r0 + (threadIdx.x >> 6); k < min(r0 + 256, rowsK); k += 4) m = fmaxf(m, fabsf(load_transpose_elem<SRC>(s, k, d)));
+  if (m > 0.0f) atomicMax(cells + (per_column ? d : 0), __float_as_uint(m));
+}
+
+template <int SRC, int GS, bool SR, bool TILED>
+__global__ void __launch_bounds__(256)
+quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t seed, uint32_t stream_id,
+                          const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes,
+                          uint8_t* __restrict__ sf, float* __restrict__ gscale) {
+  __shared__ float tile[128][65];
+  __shared__ float blk_amax[8][64];
+  __shared__ __align__(16) uint8_t out_codes[64][64];
+  const int64_t K = rowsK;  // operand K
+  const int64_t Kp = (K + 127) & ~(int64_t)127;
+  const int64_t nb = Kp >> 4;
+  const int64_t k_base = (int64_t)blockIdx.x * 128;
+  const int64_t d_base = (int64_t)blockIdx.y * 64;
+  const int tid = threadIdx.x;
+
+  // ---- phase 1: stage (zero outside the matrix) ------------------------------------------------------------
+  if (SRC == 0 && d_base + 64 <= D && (s.ld & 7) == 0) {
+    // 128 rows x 8 chunks of 8 BF16
+    for (int c = tid; c < 1024; c += 256) {
+      const int kr = c >> 3, dc = (c & 7) << 3;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (k_base + kr < rowsK) v = *reinterpret_cast<const uint4*>(s.bf16 + (k_base + kr) * s.ld + d_base + dc);
+      tile[kr][dc + 0] = bf16_lo(v.x); tile[kr][dc + 1] = bf16_hi(v.x);
+      tile[kr][dc + 2] = bf16_lo(v.y); tile[kr][dc + 3] = bf16_hi(v.y);
+      tile[kr][dc + 4] = bf16_lo(v.z); tile[kr][dc + 5] = bf16_hi(v.z);
+      tile[kr][dc + 6] = bf16_lo(v.w); tile[kr][dc + 7] = bf16_hi(v.w);
+    }
+  } else {
+    for (int e = tid; e < 128 * 64; e += 256) {
+      const int kr = e >> 6, dl = e & 63;
+      const int64_t k = k_base + kr, d = d_base + dl;
+      tile[kr][dl] = (k < rowsK && d < D) ? load_transpose_elem<SRC>(s, k, d) : 0.0f;
+    }
+  }
+  __syncthreads();
+
+  // ---- phase 2: two (d, k-block) items per thread -----------------------------------------------------------
+  const int dl = tid & 63;
+  const int64_t d = d_base + dl;
+  float xs[2][16];
+  float am[2];
+#pragma unroll
+  for (int it = 0; it < 2; ++it) {
+    const int kb = (tid >> 6) + 4 * it;  // 0..7
+    float m = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      xs[it][i] = tile[kb * 16 + i][dl];
+      m = fmaxf(m, fabsf(xs[it][i]));
+    }
+    am[it] = m;
+    if (GS == kGsBlock128) blk_amax[kb][dl] = m;
+  }
+  float Sg;
+  if (GS == kGsBlock128) {
+    __syncthreads();
+    float g = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) g = fmaxf(g, blk_amax[j][dl]);
+    Sg = global_scale_from_amax(g);
+    if (d < D && tid < 64 && k_base < K) gscale[d * (Kp >> 7) + blockIdx.x] = Sg;
+  } else if (GS == kGsRow) {
+    Sg = global_scale_from_amax(d < D ? __uint_as_float(gs_cells[d]) : 0.0f);
+    if (d < D && tid < 64 && blockIdx.x == 0) gscale[d] = Sg;
+  } else {
+    Sg = global_scale_from_amax(__uint_as_float(gs_cells[0]));
+    if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) gscale[0] = Sg;
+  }
+  const int64_t K16 = (K + 15) & ~(int64_t)15;
+#pragma unroll
+  for (int it = 0; it < 2; ++it) {
+    const int kb = (tid >> 6) + 4 * it;
+    float rcp;
+    const uint32_t sb = block_scale(am[it], Sg, rcp);
+    const int64_t k0 = k_base + kb * 16;
+    const uint2 packed = quantize_block16<SR>(xs[it], rcp, seed, stream_id, (uint64_t)((d * K16 + k0) >> 3));
+    *reinterpret_cast<uint2*>(&out_codes[dl][kb * 8]) = packed;
+    if (d < D && k0 < Kp) {
+      const int64_t b = k0 >> 4;
+      const size_t off = TILED ? sf_tiled_offset(d, b, (nb + 15) & ~(int64_t)15) : (size_t)(d * nb + b);
+      sf[off] = (uint8_t)sb;
+    }
+  }
+  __syncthreads();
+
+  // ---- phase 3: 64 rows x 64 bytes, 16 bytes per thread ------------------------------------------------------
+  {
+    const int row = tid >> 2, piece = tid & 3;
+    const int64_t dd = d_base + row;
+    if (dd < D && k_base + piece * 32 < Kp)
+      *reinterpret_cast<uint4*>(codes + dd * (Kp >> 1) + (k_base >> 1) + piece * 16) =
+          *reinterpret_cast<const uint4*>(&out_codes[row][piece * 16]);
+  }
+}
+
+// =========================================================================================================
+// Host-side launchers
+// =========================================================================================================
+static inline unsigned blocks_for(int64_t n, int per) { return (unsigned)((n + per - 1) / per); }
+
+template <int GS, bool SR, bool TILED>
+static cudaError_t launch_rows_g(const QuantRowsArgs& a, cudaStream_t st) {
+  const int64_t Kp = (a.K + 127) & ~(int64_t)127;
+  const int64_t total = a.rows * (Kp >> 4);
+  const unsigned grid = blocks_for(total, 256);
+  if (a.keep)
+    quantize_rows_kernel<GS, SR, TILED, true><<<grid, 256, 0, st>>>(a.src, a.rows, a.K, a.ld, a.keep, a.seed, a.stream_id,
+                                                                   a.gs_cells, a.codes, a.sf, a.gscale);
+  else
+    quantize_rows_kernel<GS, SR, TILED, false><<<grid, 256, 0, st>>>(a.src, a.rows, a.K, a.ld, nullptr, a.seed,
+                                                                    a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale);
+  return cudaGetLastError();
+}
+
+template <int GS, bool SR>
+static cudaError_t launch_rows_t(const QuantRowsArgs& a, cudaStream_t st) {
+  return a.sf_tiled ? launch_rows_g<GS, SR, true>(a, st) : launch_rows_g<GS, SR, false>(a, st);
+}
+
+template <int GS>
+static cudaError_t launch_rows_r(const QuantRowsArgs& a, cudaStream_t st) {
+  return a.sr ? launch_rows_t<GS, true>(a, st) : launch_rows_t<GS, false>(a, st);
+}
+
+cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
+  if (a.rows == 0 || a.K == 0) return cudaSuccess;
+  cudaError_t e;
+  if (a.gs_mode == kGsTensor) {
+    if (a.compute_amax) {
+      if ((e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
+      if (a.keep) {  // amax over the kept columns only: one row per CTA, one atomic per row
+        amax_rows_bf16_kernel<<<(unsigned)a.rows, 256, 0, st>>>(a.src, a.rows, a.cols_src, a.ld, a.keep, a.K, a.gs_cells, 1);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        return launch_rows_r<kGsTensor>(a, st);
+      }
+      const int64_t chunks = a.rows * ((a.cols_src + 7) >> 3);
+      const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
+      amax_tensor_bf16_kernel<<<grid, 256, 0, st>>>(a.src, a.rows, a.cols_src, a.ld, a.gs_cells);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    return launch_rows_r<kGsTensor>(a, st);
+  }
+  if (a.gs_mode == kGsRow) {
+    amax_rows_bf16_kernel<<<(unsigned)a.rows, 256, 0, st>>>(a.src, a.rows, a.cols_src, a.ld, a.keep, a.K, a.gs_cells, 0);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    return launch_rows_r<kGsRow>(a, st);
+  }
+  return launch_rows_r<kGsBlock128>(a, st);
+}
+
+template <int SRC, int GS, bool SR>
+static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
+  const dim3 grid(blocks_for(a.rowsK, 128), blocks_for(a.D, 64));
+  if (a.sf_tiled)
+    quantize_transpose_kernel<SRC, GS, SR, true><<<grid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.seed, a.stream_id, a.gs_cells,
+                                                                      a.codes, a.sf, a.gscale);
+  else
+    quantize_transpose_kernel<SRC, GS, SR, false><<<grid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.seed, a.stream_id,
+                                                                       a.gs_cells, a.codes, a.sf, a.gscale);
+  return cudaGetLastError();
+}
+
+template <int SRC, int GS>
+static cudaError_t launch_tr_r(const QuantTransposeArgs& a, cudaStream_t st) {
+  return a.sr ? launch_tr_t<SRC, GS, true>(a, st) : launch_tr_t<SRC, GS, false>(a, st);
+}
+
+template <int SRC>
+static cudaError_t launch_tr_s(const QuantTransposeArgs& a, cudaStream_t st) {
+  cudaError_t e;
+  const dim3 agrid(blocks_for(a.D, 64), blocks_for(a.rowsK, 256));
+  if (a.gs_mode == kGsTensor) {
+    if (a.compute_amax) {
+      if ((e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
+      amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 0);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    return launch_tr_r<SRC, kGsTensor>(a, st);
+  }
+  if (a.gs_mode == kGsRow) {
+    if ((e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t) * (size_t)a.D, st)) != cudaSuccess) return e;
+    amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 1);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    return launch_tr_r<SRC, kGsRow>(a, st);
+  }
+  return launch_tr_r<SRC, kGsBlock128>(a, st);
+}
+
+cudaError_t launch_quantize_transpose(const QuantTransposeArgs& a, cudaStream_t st) {
+  if (a.rowsK == 0 || a.D == 0) return cudaSuccess;
+  return a.from_codes ? launch_tr_s<1>(a, st) : launch_tr_s<0>(a, st);
+}
+
+}  // namespace nvfp4

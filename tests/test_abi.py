@@ -1,0 +1,76 @@
+"""CPU-side checks of the boundary: the shared library loads, exports every symbol the header declares, its
+host-only helpers agree with the documented layout, and bad arguments are refused before anything launches."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2510_27527_b200 import build
+
+    build.build()
+    from paper_2510_27527_b200 import binding as b
+
+    return b
+
+
+def test_every_declared_symbol_is_exported(binding):
+    header = open(os.path.join(ROOT, "include", "nvfp4.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(nvfp4_[a-z0-9_]+)\s*\(", header))
+    assert {"nvfp4_quantize", "nvfp4_linear_fwd", "nvfp4_linear_bwd_dx", "nvfp4_linear_bwd_dw", "nvfp4_gemm",
+            "nvfp4_requantize_t"} <= declared
+    for name in declared:
+        assert hasattr(binding.lib, name), name
+    assert declared == set(binding.EXPORTS)
+
+
+def test_size_helpers(binding):
+    L = binding.lib
+    assert L.nvfp4_padded_k(1) == 128 and L.nvfp4_padded_k(128) == 128 and L.nvfp4_padded_k(129) == 256
+    assert L.nvfp4_operand_codes_bytes(3, 16) == 3 * 64
+    assert L.nvfp4_operand_sf_bytes(3, 16, binding.SF_LINEAR) == 3 * 8
+    assert L.nvfp4_operand_sf_bytes(3, 16, binding.SF_TILED128x4) == 128 * 16
+    assert L.nvfp4_operand_sf_bytes(129, 300, binding.SF_TILED128x4) == 256 * 32
+    assert L.nvfp4_operand_gscale_count(7, 300, binding.GS_TENSOR) == 1
+    assert L.nvfp4_operand_gscale_count(7, 300, binding.GS_ROW) == 7
+    assert L.nvfp4_operand_gscale_count(7, 300, binding.GS_BLOCK128) == 7 * 3
+    assert L.nvfp4_status_string(0) == b"ok" and b"workspace" in L.nvfp4_status_string(5)
+    assert L.nvfp4_linear_workspace_bytes(binding.OP_BWD_DX, 256, 512, 512, 0, 0) > 256 * 512 // 2
+
+
+def test_bad_arguments_are_refused_on_the_host(binding):
+    L, b = binding.lib, binding
+    op = b.COperand(0x1000, 0x2000, 0x3000, 4, 32, 0, 0)
+    ws = 0x4000
+    q = lambda *a: L.nvfp4_quantize(*a)
+    assert q(0, 4, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 1  # null source
+    assert q(0x100, 4, 32, 32, 2, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 4  # bad axis
+    assert q(0x100, 4, 32, 32, 0, 7, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 4  # bad rounding
+    assert q(0x100, -1, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 2  # negative size
+    assert q(0x100, 5, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 2  # out shape mismatch
+    assert q(0x104, 4, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 3  # misaligned source
+    assert q(0x100, 4, 32, 36, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 3  # ld not multiple of 8
+    assert q(0x100, 4, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 8, None) == 5  # workspace too small
+    bad = b.COperand(0x1000, 0x2000, 0x3000, 4, 32, 9, 0)
+    assert q(0x100, 4, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(bad), ws, 256, None) == 4  # bad gs_mode
+    a = b.COperand(0x1000, 0x2000, 0x3000, 4, 32, 0, 1)
+    c = b.COperand(0x1000, 0x2000, 0x3000, 4, 64, 0, 1)
+    assert L.nvfp4_gemm(ctypes.byref(a), ctypes.byref(c), 0x5000, 1, 4, 0, None, None, 0, None) == 2  # K mismatch
+    lin = b.COperand(0x1000, 0x2000, 0x3000, 4, 32, 0, 0)
+    assert L.nvfp4_gemm(ctypes.byref(a), ctypes.byref(lin), 0x5000, 1, 4, 0, None, None, 0, None) == 4  # linear scales
+
+
+def test_product_does_not_import_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2510_27527_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert not re.search(r"^\s*(from|import)\s+\S*oracle", text, flags=re.M), f
+                assert "nvfp4_oracle" not in text and "libnvfp4_oracle" not in text, f

@@ -1,0 +1,78 @@
+"""GPU parity of the whole layer (forward, dX, dW; with and without OutControl) on the small configuration:
+X 256x512 ~N(0,1) with 4 outlier channels x50, W 512x512 ~N(0,0.02), dY 256x512 Student-t(3) x 1e-3, seed 0."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import nvfp4_oracle as orc
+from paper_2510_27527_b200 import synth
+from tests.gpu_util import assert_operand_equal, bf16_ulp_close, rel_fro, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def B():
+    from paper_2510_27527_b200 import binding
+
+    return binding
+
+
+def run_layer(b, X, W, dY, gs_mode, outliers, f32_out=True, seed=0):
+    cfg = b.LayerConfig(gs_mode=gs_mode, seed=seed, outliers=outliers, y_dtype=b.DT_F32 if f32_out else b.DT_BF16,
+                        dx_dtype=b.DT_F32 if f32_out else b.DT_BF16, dw_dtype=b.DT_F32)
+    Xd, Wd, dYd = to_dev_bf16(X), to_dev_bf16(W), to_dev_bf16(dY)
+    Y, saved = b.nvfp4_linear_fwd(Xd, Wd, cfg)
+    dX = b.nvfp4_linear_bwd_dx(dYd, saved, cfg)
+    dW = b.nvfp4_linear_bwd_dw(dYd, saved, cfg)
+    torch.cuda.synchronize()
+    return Y.float().cpu().numpy(), dX.float().cpu().numpy(), dW.float().cpu().numpy(), saved
+
+
+@pytest.mark.parametrize("gs_mode", [0, 1])
+@pytest.mark.parametrize("outcontrol", [False, True])
+def test_config1_layer(gs_mode, outcontrol):
+    b = B()
+    c = synth.CONFIGS[1]
+    (_, D, C), = c["linears"]
+    X, W, dY, ch = synth.layer_inputs(1, c["tokens"], D, C, n_outlier=c["n_outlier"], factor=c["factor"],
+                                      grad_scale=c["grad_scale"])
+    outl = ch if outcontrol else None
+    ocfg = orc.LayerConfig(gs_mode=gs_mode, seed=0, outliers=outl)
+    Yo, so = orc.linear_fwd(X, W, ocfg)
+    dXo = orc.linear_bwd_dx(dY, so, ocfg)
+    dWo = orc.linear_bwd_dw(dY, so, ocfg)
+    Y, dX, dW, saved = run_layer(b, X, W, dY, gs_mode, outl)
+    assert_operand_equal(saved.qx, so.qx, "Q1(X)")
+    assert_operand_equal(saved.qw, so.qw, "Q2(W)")
+    for name, got, want in (("Y", Y, Yo), ("dX", dX, dXo), ("dW", dW, dWo)):
+        assert got.shape == want.shape
+        assert rel_fro(got, want) <= 1e-3, name
+        assert rel_fro(got, want) <= 2e-5, (name, rel_fro(got, want))
+    # BF16 outputs: one rounding of the same FP32 result
+    Y16, dX16, _, _ = run_layer(b, X, W, dY, gs_mode, outl, f32_out=False)
+    assert np.all(bf16_ulp_close(Y16, Yo, 1.0)) and np.all(bf16_ulp_close(dX16, dXo, 1.0))
+
+
+def test_layer_is_replayable_and_seed_dependent():
+    b = B()
+    X, W, dY, _ = synth.layer_inputs(1, 256, 512, 512, n_outlier=4, factor=50.0, grad_scale=1e-3)
+    a = run_layer(b, X, W, dY, 0, None, seed=5)
+    a2 = run_layer(b, X, W, dY, 0, None, seed=5)
+    c = run_layer(b, X, W, dY, 0, None, seed=6)
+    assert np.array_equal(a[0], c[0])  # forward is deterministic rounding
+    assert np.array_equal(a[1], a2[1]) and np.array_equal(a[2], a2[2])
+    assert not np.array_equal(a[1], c[1]) and not np.array_equal(a[2], c[2])
+
+
+def test_ragged_layer_shapes():
+    """Tokens / features that are not multiples of the tile sizes (partial 16-blocks, partial 128-row tiles)."""
+    b = B()
+    N_tok, D, C = 200, 272, 136
+    X, W, dY, ch = synth.layer_inputs(9, N_tok, D, C, n_outlier=3, factor=40.0, grad_scale=1e-3)
+    for outl in (None, ch):
+        for gs_mode in (0, 1):
+            ocfg = orc.LayerConfig(gs_mode=gs_mode, seed=3, outliers=outl)
+            Yo, so = orc.linear_fwd(X, W, ocfg)
+            dXo, dWo = orc.linear_bwd_dx(dY, so, ocfg), orc.linear_bwd_dw(dY, so, ocfg)
+            Y, dX, dW, _ = run_layer(b, X, W, dY, gs_mode, outl, seed=3)
+            assert rel_fro(Y, Yo) <= 2e-5 and rel_fro(dX, dXo) <= 2e-5 and rel_fro(dW, dWo) <= 2e-5
