@@ -141,6 +141,13 @@ def alloc_operand(R: int, K: int, gs_mode: int, sf_layout: int = SF_TILED128x4, 
     return Operand(codes, sf, gs, R, K, gs_mode, sf_layout)
 
 
+def _matrix(rows: int, cols: int, dtype_code: int, device) -> torch.Tensor:
+    """Row-major output whose rows start on 16-byte boundaries (leading dimension padded to 8 elements)."""
+    ld = (cols + 7) // 8 * 8
+    buf = torch.empty((rows, ld), dtype=torch.float32 if dtype_code == DT_F32 else torch.bfloat16, device=device)
+    return buf[:, :cols]
+
+
 def _workspace(nbytes: int, device="cuda") -> torch.Tensor:
     return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
 
@@ -182,7 +189,7 @@ def nvfp4_requantize_t(inp: Operand, rounding: int = ROUND_SR, seed: int = 0, st
 def nvfp4_gemm(A: Operand, B: Operand, c_dtype: int = DT_F32, out: torch.Tensor | None = None, accumulate: bool = False,
                dev_status: torch.Tensor | None = None, workspace: torch.Tensor | None = None) -> torch.Tensor:
     if out is None:
-        out = torch.empty((A.R, B.R), dtype=torch.float32 if c_dtype == DT_F32 else torch.bfloat16, device=A.codes.device)
+        out = _matrix(A.R, B.R, c_dtype, A.codes.device)
     ws = workspace if workspace is not None else _workspace(_lib.nvfp4_gemm_workspace_bytes(A.R, B.R, A.K), A.codes.device)
     ca, cb = A.c(), B.c()
     _check(_lib.nvfp4_gemm(ctypes.byref(ca), ctypes.byref(cb), _ptr(out), c_dtype, out.stride(0), int(accumulate),
@@ -258,7 +265,7 @@ def nvfp4_linear_fwd(X: torch.Tensor, W: torch.Tensor, cfg: LayerConfig, Y: torc
     else:
         saved.X, saved.W = X, W
     if Y is None:
-        Y = torch.empty((N_tok, C), dtype=torch.float32 if cfg.y_dtype == DT_F32 else torch.bfloat16, device=X.device)
+        Y = _matrix(N_tok, C, cfg.y_dtype, X.device)
     ws = workspace if workspace is not None else linear_workspace(OP_FWD, N_tok, D, C, cfg, X.device)
     cs, cc = saved.c(), cfg.c()
     _check(_lib.nvfp4_linear_fwd(_ptr(X), X.stride(0), _ptr(W), W.stride(0), N_tok, D, C, ctypes.byref(cc), _ptr(Y),
@@ -271,7 +278,7 @@ def nvfp4_linear_bwd_dx(dY: torch.Tensor, saved: Saved, cfg: LayerConfig, dX: to
     N_tok, D = saved.X.shape
     C = saved.W.shape[0]
     if dX is None:
-        dX = torch.empty((N_tok, D), dtype=torch.float32 if cfg.dx_dtype == DT_F32 else torch.bfloat16, device=dY.device)
+        dX = _matrix(N_tok, D, cfg.dx_dtype, dY.device)
     ws = workspace if workspace is not None else linear_workspace(OP_BWD_DX, N_tok, D, C, cfg, dY.device)
     cs, cc = saved.c(), cfg.c()
     _check(_lib.nvfp4_linear_bwd_dx(_ptr(dY), dY.stride(0), ctypes.byref(cs), ctypes.byref(cc), _ptr(dX), dX.stride(0),
@@ -284,7 +291,7 @@ def nvfp4_linear_bwd_dw(dY: torch.Tensor, saved: Saved, cfg: LayerConfig, dW: to
     N_tok, D = saved.X.shape
     C = saved.W.shape[0]
     if dW is None:
-        dW = torch.empty((C, D), dtype=torch.float32 if cfg.dw_dtype == DT_F32 else torch.bfloat16, device=dY.device)
+        dW = _matrix(C, D, cfg.dw_dtype, dY.device)
     ws = workspace if workspace is not None else linear_workspace(OP_BWD_DW, N_tok, D, C, cfg, dY.device)
     cs, cc = saved.c(), cfg.c()
     _check(_lib.nvfp4_linear_bwd_dw(_ptr(dY), dY.stride(0), ctypes.byref(cs), ctypes.byref(cc), _ptr(dW), dW.stride(0),

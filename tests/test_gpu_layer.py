@@ -50,7 +50,9 @@ def test_config1_layer(gs_mode, outcontrol):
         assert rel_fro(got, want) <= 2e-5, (name, rel_fro(got, want))
     # BF16 outputs: one rounding of the same FP32 result
     Y16, dX16, _, _ = run_layer(b, X, W, dY, gs_mode, outl, f32_out=False)
-    assert np.all(bf16_ulp_close(Y16, Yo, 1.0)) and np.all(bf16_ulp_close(dX16, dXo, 1.0))
+    # (noise term: FP32 accumulation error where a sum cancels, scaled by the output's typical magnitude)
+    assert np.all(bf16_ulp_close(Y16, Yo, 1.0, 1e-4 * np.abs(Yo).mean()))
+    assert np.all(bf16_ulp_close(dX16, dXo, 1.0, 1e-4 * np.abs(dXo).mean()))
 
 
 def test_layer_is_replayable_and_seed_dependent():
