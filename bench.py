@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the NVFP4 linear-layer hot path on B200.
+
+One "step" = forward + dX + dW (six quantizers, three FP4 GEMMs each) of every linear of the workload, through the
+C-ABI library. Default workload: LLaMA-style attention projections, hidden 1024, tokens 8192 (QKV 1024->3072 and
+O 1024->1024), seeded synthetic BF16 inputs. Prints ONE JSON line (see the keys below).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload attn|mlp|model370m] [--gs tensor|row]
+
+N > 1 (torchrun): every rank runs the same workload on its own GPU (independent replicas, no collective on the data
+path); the time is the max over ranks and the value the sum of all ranks' work.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2510_27527_b200 import synth  # noqa: E402
+
+WORKLOADS = {
+    # name: (config id of the input recipe, tokens, [(linear name, D_in, C_out, swiglu input?)])
+    "attn": (2, 8192, [("qkv", 1024, 3072, False), ("o", 1024, 1024, False)]),
+    "mlp": (3, 8192, [("gate", 1024, 2816, False), ("up", 1024, 2816, False), ("down", 2816, 1024, True)]),
+    "model370m": (4, 16384, [("qkv", 1024, 3072, False), ("o", 1024, 1024, False), ("gate", 1024, 2816, False),
+                             ("up", 1024, 2816, False), ("down", 2816, 1024, True)]),
+}
+LAYERS = {"attn": 1, "mlp": 1, "model370m": 24}
+GS = {"tensor": 0, "row": 1, "block128": 2}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], bf16=d["bf16_tflops"], bf16_sustained=d["bf16_tflops_sustained"], source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+def flops_of(tokens, linears, layers):
+    return layers * sum(6.0 * tokens * D * C for (_, D, C, _) in linears)
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read-only queries)."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._pump, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for l in self.lines:
+            f = [t.strip() for t in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# the oracle arm (CPU): used for --impl reference and for the cpu_baseline leg of the default arm
+# ---------------------------------------------------------------------------------------------------------------
+def oracle_sample_step(workload: str, gs_mode: int, sample_tokens: int = 256):
+    """One forward + dX + dW of the workload's first linear on a slab of `sample_tokens` tokens, through the
+    oracle as it stands. Returns (seconds, flops of the sample, description)."""
+    from oracle import nvfp4_oracle as orc
+
+    cfg_id, tokens, linears = WORKLOADS[workload]
+    name, D, C, swiglu = linears[0]
+    c = synth.CONFIGS[cfg_id]
+    X, W, dY, _ = synth.layer_inputs(cfg_id, sample_tokens, D, C, n_outlier=c["n_outlier"], factor=c["factor"],
+                                     grad_scale=c["grad_scale"], swiglu=swiglu)
+    orc.lib()
+    t0 = time.perf_counter()
+    ocfg = orc.LayerConfig(gs_mode=gs_mode, seed=0)
+    _, saved = orc.linear_fwd(X, W, ocfg)
+    orc.linear_bwd_dx(dY, saved, ocfg)
+    orc.linear_bwd_dw(dY, saved, ocfg)
+    dt = time.perf_counter() - t0
+    return dt, 6.0 * sample_tokens * D * C, f"{name} linear {D}->{C}, {sample_tokens}-token slab of the {tokens}-token workload, fwd+dX+dW"
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import nvfp4_oracle as orc
+
+    gs_mode = GS[args.gs]
+    cfg_id, tokens, linears = WORKLOADS[args.workload]
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_step(args.workload, gs_mode, 64)
+    times, fl, desc = [], 0.0, ""
+    for _ in range(args.steps):
+        dt, fl, desc = oracle_sample_step(args.workload, gs_mode, args.ref_tokens)
+        times.append(dt)
+    t = float(np.mean(times))
+    val = fl / t / 1e12
+    line = {
+        "impl": "reference", "metric": "nvfp4_linear_fwd_bwd_tflops", "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(args), "sample": desc, "gs_mode": args.gs},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": orc.threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_name(args):
+    cfg_id, tokens, linears = WORKLOADS[args.workload]
+    return (f"{args.workload}: tokens {tokens}, " + ", ".join(f"{n} {D}->{C}" for n, D, C, _ in linears) +
+            (f", x{LAYERS[args.workload]} layers" if LAYERS[args.workload] > 1 else "") + ", fwd+dX+dW per linear")
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ---------------------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2510_27527_b200 import binding as b
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl")
+    dev = torch.device("cuda", local)
+    gs_mode = GS[args.gs]
+    cfg_id, tokens, linears = WORKLOADS[args.workload]
+    layers = LAYERS[args.workload]
+    c = synth.CONFIGS[cfg_id]
+
+    # ---- inputs: activations / gradients per shape class, fresh weights per layer ------------------------------
+    class Lin:
+        pass
+
+    lins = []
+    host_inputs = {}
+    for li, (name, D, C, swiglu) in enumerate(linears):
+        X, W, dY, _ = synth.layer_inputs(cfg_id, tokens, D, C, n_outlier=max(1, D // 100), factor=c["factor"],
+                                         grad_scale=c["grad_scale"], weight_id=10 + li, swiglu=swiglu)
+        L = Lin()
+        L.name, L.D, L.C = name, D, C
+        L.Xh, L.dYh = X, dY
+        L.X, L.dY = b.upload_bf16(X, dev), b.upload_bf16(dY, dev)
+        L.W = [b.upload_bf16(W, dev)]
+        for extra in range(1, layers):
+            L.W.append(b.upload_bf16(synth.weights(C, D, synth.seed_of(cfg_id, 100 * extra + li)), dev))
+        L.cfg = b.LayerConfig(gs_mode=gs_mode, seed=0, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32)
+        L.saved = b.Saved(b.alloc_operand(tokens, D, gs_mode, device=dev), b.alloc_operand(C, D, gs_mode, device=dev), L.X, L.W[0])
+        L.Y = torch.empty((tokens, C), dtype=torch.bfloat16, device=dev)
+        L.dXo = torch.empty((tokens, D), dtype=torch.bfloat16, device=dev)
+        L.dWo = torch.empty((C, D), dtype=torch.float32, device=dev)
+        L.ws = [b.linear_workspace(k, tokens, D, C, L.cfg, dev) for k in (b.OP_FWD, b.OP_BWD_DX, b.OP_BWD_DW)]
+        lins.append(L)
+
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def flush_l2():
+        flush_buf.fill_(1)
+
+    def step():
+        for layer in range(layers):
+            for L in lins:
+                W = L.W[layer]
+                b.nvfp4_linear_fwd(L.X, W, L.cfg, Y=L.Y, saved=L.saved, workspace=L.ws[0])
+                b.nvfp4_linear_bwd_dx(L.dY, L.saved, L.cfg, dX=L.dXo, workspace=L.ws[1])
+                b.nvfp4_linear_bwd_dw(L.dY, L.saved, L.cfg, dW=L.dWo, workspace=L.ws[2])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn, steps, flush=True):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        barrier()
+        for s in range(steps):
+            if flush:
+                flush_l2()
+            ev[s][0].record()
+            fn()
+            ev[s][1].record()
+        barrier()
+        ms = [a.elapsed_time(bb) for a, bb in ev]
+        tot = torch.tensor([sum(ms)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(tot, op=dist.ReduceOp.MAX)
+        return float(tot.item()) / steps, ms
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    l0 = b.lib.nvfp4_launch_count()
+    ms_step, _ = timed(step, args.steps)
+    launches = b.lib.nvfp4_launch_count() - l0
+    clocks = sampler.stop() if rank == 0 else None
+    fl = flops_of(tokens, linears, layers)
+    value = world * fl / (ms_step * 1e-3) / 1e12
+
+    # ---- end to end: host buffers in, results out, copies inside the timed region -------------------------------
+    pinned_in, h2d, d2h = [], 0, 0
+    for L in lins:
+        xb = torch.from_numpy(synth.to_bf16_bits(L.Xh).view(np.int16)).view(torch.bfloat16).pin_memory()
+        gb = torch.from_numpy(synth.to_bf16_bits(L.dYh).view(np.int16)).view(torch.bfloat16).pin_memory()
+        L.pin = (xb, gb)
+        L.out_pin = (torch.empty_like(L.Y, device="cpu").pin_memory(), torch.empty_like(L.dXo, device="cpu").pin_memory(),
+                     torch.empty_like(L.dWo, device="cpu").pin_memory())
+        h2d += layers * (xb.numel() + gb.numel()) * 2
+        d2h += layers * (L.Y.numel() * 2 + L.dXo.numel() * 2 + L.dWo.numel() * 4)
+
+    def step_e2e():
+        for layer in range(layers):
+            for L in lins:
+                L.X.copy_(L.pin[0], non_blocking=True)
+                L.dY.copy_(L.pin[1], non_blocking=True)
+                W = L.W[layer]
+                b.nvfp4_linear_fwd(L.X, W, L.cfg, Y=L.Y, saved=L.saved, workspace=L.ws[0])
+                b.nvfp4_linear_bwd_dx(L.dY, L.saved, L.cfg, dX=L.dXo, workspace=L.ws[1])
+                b.nvfp4_linear_bwd_dw(L.dY, L.saved, L.cfg, dW=L.dWo, workspace=L.ws[2])
+                L.out_pin[0].copy_(L.Y, non_blocking=True)
+                L.out_pin[1].copy_(L.dXo, non_blocking=True)
+                L.out_pin[2].copy_(L.dWo, non_blocking=True)
+
+    e2e_steps = max(2, min(args.steps, 5))
+    step_e2e()
+    ms_e2e, _ = timed(step_e2e, e2e_steps)
+    e2e_value = world * fl / (ms_e2e * 1e-3) / 1e12
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- per-kernel breakdown on the largest linear (rank 0): which kernel dominates, and its roofline ----------
+    pk = peaks()
+    L = max(lins, key=lambda l: l.D * l.C)
+    ws_q = b._workspace(1 << 20, dev)
+
+    def t_of(fn, n=20):
+        for _ in range(3):
+            fn()
+        t, _ = timed(fn, n)
+        return t * 1e-3
+
+    T, D, C = tokens, L.D, L.C
+    q3 = b.alloc_operand(T, C, gs_mode, device=dev)
+    q4 = b.alloc_operand(D, C, gs_mode, device=dev)
+    q5 = b.alloc_operand(C, T, gs_mode, device=dev)
+    q6 = b.alloc_operand(D, T, gs_mode, device=dev)
+    b.nvfp4_linear_fwd(L.X, L.W[0], L.cfg, Y=L.Y, saved=L.saved, workspace=L.ws[0])
+    parts = {}
+
+    def add(name, fn, alg_bytes=None, flops=None):
+        t = t_of(fn)
+        parts[name] = dict(seconds=t, GBps=(alg_bytes / t / 1e9 if alg_bytes else None),
+                           TFLOPs=(flops / t / 1e12 if flops else None), bytes=alg_bytes, flops=flops)
+
+    qbytes = lambda n: n * (2 + 0.5 + 1.0 / 16)
+    rqbytes = lambda n: n * 2 * (0.5 + 1.0 / 16)
+    amax_extra = 2.0 if gs_mode != 2 else 0.0  # TENSOR / ROW modes read the source twice (amax pre-pass)
+    add("quantize_rows_X(Q1)", lambda: b.nvfp4_quantize(L.X, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, out=L.saved.qx, workspace=ws_q),
+        qbytes(T * D) + amax_extra * T * D)
+    add("quantize_rows_dY_SR(Q3)", lambda: b.nvfp4_quantize(L.dY, b.AXIS_ROW, b.ROUND_SR, 0, 3, gs_mode, out=q3, workspace=ws_q),
+        qbytes(T * C) + amax_extra * T * C)
+    add("quantize_cols_dY_SR(Q5)", lambda: b.nvfp4_quantize(L.dY, b.AXIS_COL, b.ROUND_SR, 0, 5, gs_mode, out=q5, workspace=ws_q),
+        qbytes(T * C) + amax_extra * T * C)
+    add("requantize_t_W(Q4)", lambda: b.nvfp4_requantize_t(L.saved.qw, b.ROUND_SR, 0, 4, out=q4, workspace=ws_q), rqbytes(C * D))
+    add("requantize_t_X(Q6)", lambda: b.nvfp4_requantize_t(L.saved.qx, b.ROUND_SR, 0, 6, out=q6, workspace=ws_q), rqbytes(T * D))
+    gemm_bytes = lambda M, N, K, ob: 0.5625 * (M + N) * K + ob * M * N
+    add("gemm_fwd", lambda: b.nvfp4_gemm(L.saved.qx, L.saved.qw, b.DT_BF16, out=L.Y), gemm_bytes(T, C, D, 2), 2.0 * T * C * D)
+    add("gemm_dx", lambda: b.nvfp4_gemm(q3, q4, b.DT_BF16, out=L.dXo), gemm_bytes(T, D, C, 2), 2.0 * T * C * D)
+    add("gemm_dw", lambda: b.nvfp4_gemm(q5, q6, b.DT_F32, out=L.dWo), gemm_bytes(C, D, T, 4), 2.0 * T * C * D)
+    dom = max(parts, key=lambda k: parts[k]["seconds"])
+    dp = parts[dom]
+    fp4_peak = pk["bf16"] * 4.0  # dense FP4 : dense BF16 nominal ratio 9 : 2.25
+    if dom.startswith("gemm"):
+        t_tensor = dp["flops"] / (fp4_peak * 1e12)
+        t_hbm = dp["bytes"] / (pk["hbm"] * 1e9)
+        if t_tensor >= t_hbm:
+            roof = dict(bound="tensor", achieved=dp["TFLOPs"], peak=fp4_peak, unit="TFLOP/s", frac=dp["TFLOPs"] / fp4_peak)
+        else:
+            roof = dict(bound="hbm", achieved=dp["GBps"], peak=pk["hbm"], unit="GB/s", frac=dp["GBps"] / pk["hbm"])
+    else:
+        roof = dict(bound="hbm", achieved=dp["GBps"], peak=pk["hbm"], unit="GB/s", frac=dp["GBps"] / pk["hbm"])
+    roof.update(kernel=f"{dom} on {L.name} {D}->{C}, tokens {T}", peak_source=f"of {pk['source']}", traffic=None,
+                algorithmic_bytes_per_launch=dp["bytes"], seconds_per_launch=dp["seconds"])
+    tj = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tj):
+        roof["traffic"] = json.load(open(tj)).get(dom)
+
+    # ---- the oracle beside it ------------------------------------------------------------------------------------
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        from oracle import nvfp4_oracle as orc
+
+        dt, sfl, desc = oracle_sample_step(args.workload, gs_mode, args.cpu_tokens)
+        cpu = {"value": sfl / dt / 1e12, "unit": "TFLOP/s", "cores": orc.threads(), "kind": "oracle", "sample": desc,
+               "seconds": dt}
+
+    line = {
+        "metric": "nvfp4_linear_fwd_bwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "fp4(e2m1)xfp4 with ue4m3 block scales, f32 accumulate", "data": "synthetic",
+        "config": {"workload": workload_name(args), "gs_mode": args.gs, "l2": "256 MiB flush write before every timed step",
+                   "timing": "CUDA events per step on the launch stream, summed"},
+        "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
+        "gpu_launches": int(launches), "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
+        "kernels": {k: {kk: (round(vv, 9) if isinstance(vv, float) else vv) for kk, vv in v.items() if kk in ("seconds", "GBps", "TFLOPs")}
+                    for k, v in parts.items()},
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="attn", choices=list(WORKLOADS))
+    ap.add_argument("--gs", default="tensor", choices=list(GS))
+    ap.add_argument("--ref-tokens", type=int, default=1024, help="token slab of one oracle step (reference arm)")
+    ap.add_argument("--cpu-tokens", type=int, default=4096, help="token slab of the cpu_baseline leg")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -86,6 +86,9 @@ size_t nvfp4_operand_gscale_count(int64_t R, int64_t K, int32_t gs_mode);
 
 const char* nvfp4_status_string(nvfp4_status s);
 
+/* Number of kernels the library has enqueued since it was loaded (a measurement aid; not thread-safe). */
+long long nvfp4_launch_count(void);
+
 /* ---------------------------------------------------------------------------------------------------------
  * nvfp4_quantize — double-block quantization of a BF16 matrix (Sec. 2.2; rounding per Sec. 2.1).
  *

@@ -55,6 +55,7 @@ EXPORTS = {
     "nvfp4_operand_sf_bytes": (c_sz, [c_i64, c_i64, c_i32]),
     "nvfp4_operand_gscale_count": (c_sz, [c_i64, c_i64, c_i32]),
     "nvfp4_status_string": (ctypes.c_char_p, [c_i32]),
+    "nvfp4_launch_count": (ctypes.c_longlong, []),
     "nvfp4_quantize_workspace_bytes": (c_sz, [c_i64, c_i32]),
     "nvfp4_quantize": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_u64, c_u32, c_vp, c_i64,
                                ctypes.POINTER(COperand), c_vp, c_sz, c_vp]),
@@ -146,6 +147,13 @@ def _matrix(rows: int, cols: int, dtype_code: int, device) -> torch.Tensor:
     ld = (cols + 7) // 8 * 8
     buf = torch.empty((rows, ld), dtype=torch.float32 if dtype_code == DT_F32 else torch.bfloat16, device=device)
     return buf[:, :cols]
+
+
+def upload_bf16(x: np.ndarray, device="cuda") -> torch.Tensor:
+    """float32 host array holding BF16-representable values -> bfloat16 device tensor (bit copy)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    bits = (x.view(np.uint32) >> 16).astype(np.uint16)
+    return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(device)
 
 
 def _workspace(nbytes: int, device="cuda") -> torch.Tensor:

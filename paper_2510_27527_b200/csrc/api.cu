@@ -8,6 +8,10 @@
 
 using namespace nvfp4;
 
+namespace nvfp4 {
+long long g_launch_count = 0;
+}
+
 namespace {
 
 inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
@@ -188,6 +192,8 @@ size_t nvfp4_operand_gscale_count(int64_t R, int64_t K, int32_t gs_mode) {
   if (gs_mode == NVFP4_GS_ROW) return (size_t)R;
   return (size_t)(R * (nvfp4_padded_k(K) / 128));
 }
+
+long long nvfp4_launch_count(void) { return g_launch_count; }
 
 const char* nvfp4_status_string(nvfp4_status s) {
   switch (s) {

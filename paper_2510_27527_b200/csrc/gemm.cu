@@ -461,6 +461,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
   gemm_nvfp4_kernel<GS, BN><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(tmA, tmB, p);
+  ++g_launch_count;
   return cudaGetLastError();
 }
 

@@ -118,6 +118,7 @@ cudaError_t launch_hp_fwd(const HpFwdArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;
   const dim3 grid((unsigned)((a.N + 63) / 64), (unsigned)((a.M + 63) / 64));
   hp_fwd_kernel<<<grid, 256, 0, st>>>(a);
+  ++g_launch_count;
   return cudaGetLastError();
 }
 
@@ -125,6 +126,7 @@ cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st) {
   if (a.C == 0 || a.n_out == 0) return cudaSuccess;
   const dim3 grid((unsigned)((a.C + 63) / 64), (unsigned)((a.n_out + 7) / 8));
   hp_dw_kernel<<<grid, 256, 0, st>>>(a);
+  ++g_launch_count;
   return cudaGetLastError();
 }
 
@@ -134,6 +136,7 @@ cudaError_t launch_scatter_cols(const void* src, int64_t ld_src, int src_is_f32,
   if (total == 0) return cudaSuccess;
   const unsigned grid = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 32);
   scatter_cols_kernel<<<grid, 256, 0, st>>>(src, ld_src, src_is_f32, dst, ld_dst, dst_is_f32, rows, n_keep, keep);
+  ++g_launch_count;
   return cudaGetLastError();
 }
 

@@ -7,6 +7,9 @@
 
 namespace nvfp4 {
 
+// Number of kernels this library has enqueued since it was loaded (measurement aid).
+extern long long g_launch_count;
+
 struct QuantRowsArgs {
   const uint16_t* src;  // BF16 [rows, cols_src], leading dimension ld
   int64_t rows, K, cols_src, ld;

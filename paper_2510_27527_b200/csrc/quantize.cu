@@ -345,6 +345,7 @@ static cudaError_t launch_rows_g(const QuantRowsArgs& a, cudaStream_t st) {
   else
     quantize_rows_kernel<GS, SR, TILED, false><<<grid, 256, 0, st>>>(a.src, a.rows, a.K, a.ld, nullptr, a.seed,
                                                                     a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale);
+  ++g_launch_count;
   return cudaGetLastError();
 }
 
@@ -366,18 +367,21 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
       if ((e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
       if (a.keep) {  // amax over the kept columns only: one row per CTA, one atomic per row
         amax_rows_bf16_kernel<<<(unsigned)a.rows, 256, 0, st>>>(a.src, a.rows, a.cols_src, a.ld, a.keep, a.K, a.gs_cells, 1);
+  ++g_launch_count;
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         return launch_rows_r<kGsTensor>(a, st);
       }
       const int64_t chunks = a.rows * ((a.cols_src + 7) >> 3);
       const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
       amax_tensor_bf16_kernel<<<grid, 256, 0, st>>>(a.src, a.rows, a.cols_src, a.ld, a.gs_cells);
+  ++g_launch_count;
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     return launch_rows_r<kGsTensor>(a, st);
   }
   if (a.gs_mode == kGsRow) {
     amax_rows_bf16_kernel<<<(unsigned)a.rows, 256, 0, st>>>(a.src, a.rows, a.cols_src, a.ld, a.keep, a.K, a.gs_cells, 0);
+  ++g_launch_count;
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     return launch_rows_r<kGsRow>(a, st);
   }
@@ -393,6 +397,7 @@ static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
   else
     quantize_transpose_kernel<SRC, GS, SR, false><<<grid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.seed, a.stream_id,
                                                                        a.gs_cells, a.codes, a.sf, a.gscale);
+  ++g_launch_count;
   return cudaGetLastError();
 }
 
@@ -409,6 +414,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a, cudaStream_t st) {
     if (a.compute_amax) {
       if ((e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
       amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 0);
+  ++g_launch_count;
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     return launch_tr_r<SRC, kGsTensor>(a, st);
@@ -416,6 +422,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a, cudaStream_t st) {
   if (a.gs_mode == kGsRow) {
     if ((e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t) * (size_t)a.D, st)) != cudaSuccess) return e;
     amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 1);
+  ++g_launch_count;
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     return launch_tr_r<SRC, kGsRow>(a, st);
   }
