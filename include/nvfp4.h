@@ -38,7 +38,8 @@ typedef enum {
   NVFP4_ERR_WORKSPACE = 5, /* workspace missing or smaller than nvfp4_*_workspace_bytes says */
   NVFP4_ERR_ARCH = 6,      /* current device is not sm_100 */
   NVFP4_ERR_CUDA = 7,      /* a CUDA runtime / driver call failed (launch error, tensor-map encode) */
-  NVFP4_ERR_TIMEOUT = 8    /* reported through dev_status only: a bounded device-side wait ran out */
+  NVFP4_ERR_TIMEOUT = 8,   /* reported through dev_status only: a bounded device-side wait ran out */
+  NVFP4_ERR_LIMIT = 9      /* a size exceeds a fixed capacity of the entry point (see nvfp4_quantize_static) */
 } nvfp4_status;
 
 typedef enum { NVFP4_ROUND_RTN = 0, NVFP4_ROUND_SR = 1 } nvfp4_round;
@@ -113,6 +114,29 @@ nvfp4_status nvfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, in
                             int32_t rounding, uint64_t seed, uint32_t stream_id, const int32_t* keep_cols,
                             int64_t n_keep, const nvfp4_operand* out, void* workspace, size_t ws_bytes,
                             void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------
+ * nvfp4_quantize_static — nvfp4_quantize without a workspace argument. (The paper has no counterpart: this is a
+ * packaging variant of the same quantizer, not a step of the method.)
+ *
+ * For callers that cannot obtain device memory where they call from — code inside an allocator hook or under a
+ * framework's no-allocation guard, a plugin that receives tensors but no allocator, a loop whose memory was fixed
+ * at start-up. The amax cells live in a fixed array inside the library image (NVFP4_STATIC_MAX_ROWS 32-bit cells,
+ * 256 KiB, held by every GPU that loads the library until the process exits). The call allocates and frees
+ * nothing. Inputs, outputs, arithmetic and results are those of nvfp4_quantize.
+ *   - Capacity: gs_mode ROW needs one cell per operand row; out->R > NVFP4_STATIC_MAX_ROWS returns NVFP4_ERR_LIMIT
+ *     and nothing is launched. TENSOR and BLOCK128 have no such limit.
+ *   - The first call made with a given device current looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - Every call on a device shares the one array. The cells a call uses are cleared on `stream` before use, so
+ *     calls that are ordered (same stream, or ordered by events) are independent; calls whose kernels can overlap
+ *     on the GPU (different streams, no ordering) race on the cells and give undefined scales.
+ * --------------------------------------------------------------------------------------------------------- */
+#define NVFP4_STATIC_MAX_ROWS 65536
+int64_t nvfp4_quantize_static_max_rows(void);
+nvfp4_status nvfp4_quantize_static(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld, int32_t axis,
+                                   int32_t rounding, uint64_t seed, uint32_t stream_id, const int32_t* keep_cols,
+                                   int64_t n_keep, const nvfp4_operand* out, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------
  * nvfp4_requantize_t — the backward quantizers Q4 / Q6 of Sec. 2.3: dequantize a forward operand to the

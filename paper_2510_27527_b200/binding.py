@@ -59,6 +59,9 @@ EXPORTS = {
     "nvfp4_quantize_workspace_bytes": (c_sz, [c_i64, c_i32]),
     "nvfp4_quantize": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_u64, c_u32, c_vp, c_i64,
                                ctypes.POINTER(COperand), c_vp, c_sz, c_vp]),
+    "nvfp4_quantize_static_max_rows": (c_i64, []),
+    "nvfp4_quantize_static": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_u64, c_u32, c_vp, c_i64,
+                                      ctypes.POINTER(COperand), c_vp]),
     "nvfp4_requantize_t": (c_i32, [ctypes.POINTER(COperand), c_vp, c_i64, c_vp, c_i64, c_i32, c_u64, c_u32,
                                    ctypes.POINTER(COperand), c_vp, c_sz, c_vp]),
     "nvfp4_gemm_workspace_bytes": (c_sz, [c_i64, c_i64, c_i64]),
@@ -176,6 +179,23 @@ def nvfp4_quantize(src: torch.Tensor, axis: int = AXIS_ROW, rounding: int = ROUN
     co = out.c()
     _check(_lib.nvfp4_quantize(_ptr(src), rows, cols, src.stride(0), axis, rounding, seed, stream_id, _ptr(keep_cols), kept,
                                ctypes.byref(co), _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_quantize")
+    return out
+
+
+def nvfp4_quantize_static(src: torch.Tensor, axis: int = AXIS_ROW, rounding: int = ROUND_RTN, seed: int = 0,
+                          stream_id: int = 0, gs_mode: int = GS_TENSOR, sf_layout: int = SF_TILED128x4,
+                          keep_cols: torch.Tensor | None = None, out: Operand | None = None) -> Operand:
+    """nvfp4_quantize for callers that cannot hand over scratch memory: the amax cells live inside the library.
+    `out` should be passed by such callers (allocating it here is a convenience for tests)."""
+    assert src.dtype == torch.bfloat16 and src.dim() == 2 and src.stride(1) == 1
+    rows, cols = src.shape
+    kept = cols if keep_cols is None else int(keep_cols.numel())
+    R, K = (rows, kept) if axis == AXIS_ROW else (kept, rows)
+    if out is None:
+        out = alloc_operand(R, K, gs_mode, sf_layout, src.device)
+    co = out.c()
+    _check(_lib.nvfp4_quantize_static(_ptr(src), rows, cols, src.stride(0), axis, rounding, seed, stream_id, _ptr(keep_cols),
+                                      kept, ctypes.byref(co), _stream_ptr()), "nvfp4_quantize_static")
     return out
 
 

@@ -206,6 +206,7 @@ const char* nvfp4_status_string(nvfp4_status s) {
     case NVFP4_ERR_ARCH: return "device is not sm_100";
     case NVFP4_ERR_CUDA: return "CUDA call failed";
     case NVFP4_ERR_TIMEOUT: return "device-side wait timed out";
+    case NVFP4_ERR_LIMIT: return "size exceeds the fixed capacity of this entry point";
   }
   return "unknown status";
 }
