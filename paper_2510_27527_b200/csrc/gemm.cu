@@ -27,7 +27,6 @@ constexpr int BK = 256;                                  // elements per k tile 
 constexpr uint32_t A_BYTES = BM * BK / 2;                // 16 KB
 constexpr uint32_t SFA_BYTES = 2048;                     // 128 rows x 16 k-blocks
 constexpr int NUM_THREADS = 192;
-constexpr int EPI_WARP0 = 2;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;    // ~2 s
 
 template <int BN>

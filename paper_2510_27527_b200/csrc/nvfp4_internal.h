@@ -49,6 +49,7 @@ struct QuantTransposeArgs {
   uint32_t stream_id;
   int gs_mode, sr, sf_tiled;
   int compute_amax;
+  int tensor_closed_form;  // set by the launcher
   uint32_t* gs_cells;  // 1 cell (TENSOR) or D cells (ROW)
   uint8_t* codes;
   uint8_t* sf;

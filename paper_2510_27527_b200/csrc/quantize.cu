@@ -221,23 +221,70 @@ __device__ __forceinline__ float load_transpose_elem(const TransposeSrc& s, int6
   return load_aligned_value(s, k, j);
 }
 
-// Column amax of the aligned tensor (ROW scale mode of Q4 / Q6) and of its high-precision rows; also used for
-// TENSOR mode when a row map mixes BF16 rows in (cells has one entry then).
+// Column amax of a transposing quantizer's source: per source column (ROW scale mode: operand row = column) or
+// folded into one cell. `only_hp` restricts the pass to the columns whose row-map entry is negative (the BF16 rows
+// that OutControl mixes into W-hat). 64 columns x 256 rows per CTA, reduced in the CTA before any atomic.
 template <int SRC>
 __global__ void __launch_bounds__(256) amax_cols_generic_kernel(TransposeSrc s, int64_t rowsK, int64_t D,
-                                                               uint32_t* cells, int per_column) {
-  const int64_t d = (int64_t)blockIdx.x * 64 + (threadIdx.x & 63);
+                                                               uint32_t* cells, int per_column, int only_hp) {
+  __shared__ float red[4][64];
+  __shared__ float fin[2];
+  const int dl = threadIdx.x & 63, g = threadIdx.x >> 6;
+  const int64_t d = (int64_t)blockIdx.x * 64 + dl;
   const int64_t r0 = (int64_t)blockIdx.y * 256;
-  if (d >= D) return;
   float m = 0.0f;
-  for (int64_t k = r0 + (threadIdx.x >> 6); k < min(r0 + 256, rowsK); k += 4) m = fmaxf(m, fabsf(load_transpose_elem<SRC>(s, k, d)));
-  if (m > 0.0f) atomicMax(cells + (per_column ? d : 0), __float_as_uint(m));
+  if (d < D && !(only_hp && s.row_map[d] >= 0))
+    for (int64_t k = r0 + g; k < min(r0 + 256, rowsK); k += 4) m = fmaxf(m, fabsf(load_transpose_elem<SRC>(s, k, d)));
+  red[g][dl] = m;
+  __syncthreads();
+  if (g == 0) {
+    m = fmaxf(fmaxf(red[0][dl], red[1][dl]), fmaxf(red[2][dl], red[3][dl]));
+    if (per_column) {
+      if (d < D && m > 0.0f) atomicMax(cells + d, __float_as_uint(m));
+    } else {
+#pragma unroll
+      for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+      if ((threadIdx.x & 31) == 0) fin[threadIdx.x >> 5] = m;
+    }
+  }
+  if (!per_column) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      m = fmaxf(fin[0], fin[1]);
+      if (m > 0.0f) atomicMax(cells, __float_as_uint(m));
+    }
+  }
+}
+
+// Decode 8 packed E2M1 codes times one E4M3 scale times the global scale into 8 floats:
+// x_hat = (P * S_block) * S_global; the inner product is exact in FP16 (6 significant bits, |value| <= 2688).
+__device__ __forceinline__ void decode8(uint32_t word, uint32_t sf_byte, float sg, float* out) {
+  uint32_t h[4];
+  asm("{\n"
+      ".reg .b8 b0, b1, b2, b3;\n"
+      "mov.b32 {b0, b1, b2, b3}, %4;\n"
+      "cvt.rn.f16x2.e2m1x2 %0, b0;\n"
+      "cvt.rn.f16x2.e2m1x2 %1, b1;\n"
+      "cvt.rn.f16x2.e2m1x2 %2, b2;\n"
+      "cvt.rn.f16x2.e2m1x2 %3, b3;\n"
+      "}"
+      : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3])
+      : "r"(word));
+  uint32_t s2;
+  asm("{.reg .b16 t; cvt.u16.u32 t, %1; cvt.rn.f16x2.e4m3x2 %0, t;}" : "=r"(s2) : "r"(sf_byte | (sf_byte << 8)));
+  const __half2 sb2 = *reinterpret_cast<__half2*>(&s2);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __half22float2(__hmul2(*reinterpret_cast<__half2*>(&h[i]), sb2));
+    out[2 * i] = __fmul_rn(f.x, sg);
+    out[2 * i + 1] = __fmul_rn(f.y, sg);
+  }
 }
 
 template <int SRC, int GS, bool SR, bool TILED>
 __global__ void __launch_bounds__(256)
 quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t seed, uint32_t stream_id,
-                          const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes,
+                          const uint32_t* __restrict__ gs_cells, int tensor_closed_form, uint8_t* __restrict__ codes,
                           uint8_t* __restrict__ sf, float* __restrict__ gscale) {
   __shared__ float tile[128][65];
   __shared__ float blk_amax[8][64];
@@ -261,6 +308,31 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
       tile[kr][dc + 4] = bf16_lo(v.z); tile[kr][dc + 5] = bf16_hi(v.z);
       tile[kr][dc + 6] = bf16_lo(v.w); tile[kr][dc + 7] = bf16_hi(v.w);
     }
+  } else if (SRC == 1 && !s.row_map && d_base + 64 <= D) {
+    // forward operand without a row map: 32 codes (16 bytes) and their two scale bytes per thread
+    const int kr = tid >> 1, half = tid & 1;
+    const int64_t k = k_base + kr;
+    float v[32];
+    if (k < rowsK) {
+      const int64_t in_Kp = (s.in_K + 127) & ~(int64_t)127;
+      const int64_t in_nb = in_Kp >> 4;
+      const uint4 c4 = *reinterpret_cast<const uint4*>(s.in_codes + k * (in_Kp >> 1) + (d_base >> 1) + half * 16);
+      const int64_t kb = (d_base >> 4) + half * 2;
+      const size_t sfo = s.in_sf_tiled ? sf_tiled_offset(k, kb, (in_nb + 15) & ~(int64_t)15) : (size_t)(k * in_nb + kb);
+      const uint32_t sf2 = *reinterpret_cast<const uint16_t*>(s.in_sf + sfo);
+      const float sg = s.in_gs_mode == kGsTensor ? s.in_gscale[0]
+                       : s.in_gs_mode == kGsRow  ? s.in_gscale[k]
+                                                 : s.in_gscale[k * (in_Kp >> 7) + (d_base >> 7)];
+      decode8(c4.x, sf2 & 0xFFu, sg, v);
+      decode8(c4.y, sf2 & 0xFFu, sg, v + 8);
+      decode8(c4.z, sf2 >> 8, sg, v + 16);
+      decode8(c4.w, sf2 >> 8, sg, v + 24);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = 0.0f;
+    }
+#pragma unroll
+    for (int i = 0; i < 32; ++i) tile[kr][half * 32 + i] = v[i];
   } else {
     for (int e = tid; e < 128 * 64; e += 256) {
       const int kr = e >> 6, dl = e & 63;
@@ -299,7 +371,11 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
     Sg = global_scale_from_amax(d < D ? __uint_as_float(gs_cells[d]) : 0.0f);
     if (d < D && tid < 64 && blockIdx.x == 0) gscale[d] = Sg;
   } else {
-    Sg = global_scale_from_amax(__uint_as_float(gs_cells[0]));
+    float amax = __uint_as_float(gs_cells[0]);
+    // TENSOR -> TENSOR re-quantization: the aligned tensor's maximum is float32(2688 * S_global) of the forward
+    // operand (its largest block has scale 448 and a magnitude-6 element); gs_cells[0] then only covers BF16 rows.
+    if (SRC == 1 && tensor_closed_form) amax = fmaxf(amax, __fmul_rn(2688.0f, s.in_gscale[0]));
+    Sg = global_scale_from_amax(amax);
     if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) gscale[0] = Sg;
   }
   const int64_t K16 = (K + 15) & ~(int64_t)15;
@@ -393,10 +469,10 @@ static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
   const dim3 grid(blocks_for(a.rowsK, 128), blocks_for(a.D, 64));
   if (a.sf_tiled)
     quantize_transpose_kernel<SRC, GS, SR, true><<<grid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.seed, a.stream_id, a.gs_cells,
-                                                                      a.codes, a.sf, a.gscale);
+                                                                      a.tensor_closed_form, a.codes, a.sf, a.gscale);
   else
-    quantize_transpose_kernel<SRC, GS, SR, false><<<grid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.seed, a.stream_id,
-                                                                       a.gs_cells, a.codes, a.sf, a.gscale);
+    quantize_transpose_kernel<SRC, GS, SR, false><<<grid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.seed, a.stream_id, a.gs_cells,
+                                                                       a.tensor_closed_form, a.codes, a.sf, a.gscale);
   ++g_launch_count;
   return cudaGetLastError();
 }
@@ -407,22 +483,37 @@ static cudaError_t launch_tr_r(const QuantTransposeArgs& a, cudaStream_t st) {
 }
 
 template <int SRC>
-static cudaError_t launch_tr_s(const QuantTransposeArgs& a, cudaStream_t st) {
+static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
+  QuantTransposeArgs a = a0;
+  a.tensor_closed_form = 0;
   cudaError_t e;
   const dim3 agrid(blocks_for(a.D, 64), blocks_for(a.rowsK, 256));
   if (a.gs_mode == kGsTensor) {
     if (a.compute_amax) {
       if ((e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
-      amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 0);
-  ++g_launch_count;
+      if (SRC == 0) {
+        const int64_t chunks = a.rowsK * ((a.D + 7) >> 3);
+        const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
+        amax_tensor_bf16_kernel<<<grid, 256, 0, st>>>(a.src.bf16, a.rowsK, a.D, a.src.ld, a.gs_cells);
+        ++g_launch_count;
+      } else if (a.src.in_gs_mode == kGsTensor) {
+        a.tensor_closed_form = 1;  // only the BF16 rows (if any) need a pass
+        if (a.src.row_map) {
+          amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 0, 1);
+          ++g_launch_count;
+        }
+      } else {
+        amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 0, 0);
+        ++g_launch_count;
+      }
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     return launch_tr_r<SRC, kGsTensor>(a, st);
   }
   if (a.gs_mode == kGsRow) {
     if ((e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t) * (size_t)a.D, st)) != cudaSuccess) return e;
-    amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 1);
-  ++g_launch_count;
+    amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 1, 0);
+    ++g_launch_count;
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     return launch_tr_r<SRC, kGsRow>(a, st);
   }
