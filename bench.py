@@ -366,6 +366,80 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Roofline sweep (square and skinny GEMMs with their quantizers), one JSON line with a list of shapes.
+    Not the headline line: a measurement aid for the large-shape roofline fractions."""
+    import torch
+
+    from paper_2510_27527_b200 import binding as b
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    gs_mode = GS[args.gs]
+    pk = peaks()
+    shapes = synth.CONFIGS[5]["shapes"] if not args.shapes else [tuple(int(v) for v in t.split("x")) for t in args.shapes.split(",")]
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    out = []
+
+    def t_of(fn, n):
+        for _ in range(3):
+            fn()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        torch.cuda.synchronize()
+        for i in range(n):
+            flush_buf.fill_(1)
+            ev[i][0].record()
+            fn()
+            ev[i][1].record()
+        torch.cuda.synchronize()
+        ms = sorted(a.elapsed_time(bb) for a, bb in ev)
+        return ms[len(ms) // 2] * 1e-3, ms[0] * 1e-3
+
+    g = torch.Generator(device=dev)
+    g.manual_seed(5)
+    for (M, N, K) in shapes:
+        A = torch.randn((M, K), device=dev, generator=g, dtype=torch.float32)
+        nch = max(1, int(K * 0.005))
+        A[:, torch.randperm(K, device=dev, generator=g)[:nch]] *= 100.0
+        A = A.to(torch.bfloat16)
+        Bm = torch.randn((N, K), device=dev, generator=g, dtype=torch.float32).to(torch.bfloat16)
+        qa, qb = b.alloc_operand(M, K, gs_mode, device=dev), b.alloc_operand(N, K, gs_mode, device=dev)
+        qat = b.alloc_operand(K, M, gs_mode, device=dev)
+        ws = b._workspace(1 << 20, dev)
+        C = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+        n = args.steps
+        r = {"M": M, "N": N, "K": K}
+        qbytes = lambda e: e * (2 + 0.5 + 1.0 / 16)
+        amax_extra = 2.0 if gs_mode != 2 else 0.0
+        for name, fn, nelem in (
+            ("quantize_rows_rtn_A", lambda: b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, out=qa, workspace=ws), M * K),
+            ("quantize_rows_sr_A", lambda: b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_SR, 0, 3, gs_mode, out=qa, workspace=ws), M * K),
+            ("quantize_cols_sr_A", lambda: b.nvfp4_quantize(A, b.AXIS_COL, b.ROUND_SR, 0, 5, gs_mode, out=qat, workspace=ws), M * K),
+        ):
+            med, best = t_of(fn, n)
+            r[name] = {"us": med * 1e6, "GBps": qbytes(nelem) / med / 1e9, "GBps_incl_amax_read": (qbytes(nelem) + amax_extra * nelem) / med / 1e9,
+                       "frac_hbm_measured": (qbytes(nelem) + amax_extra * nelem) / med / 1e9 / pk["hbm"]}
+        b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, out=qa, workspace=ws)
+        b.nvfp4_quantize(Bm, b.AXIS_ROW, b.ROUND_RTN, 0, 2, gs_mode, out=qb, workspace=ws)
+        med, best = t_of(lambda: b.nvfp4_requantize_t(qa, b.ROUND_SR, 0, 6, out=qat, workspace=ws), n)
+        r["requantize_t_A"] = {"us": med * 1e6, "GBps": M * K * 1.125 / med / 1e9, "Gelem_per_s": M * K / med / 1e9}
+        med, best = t_of(lambda: b.nvfp4_gemm(qa, qb, b.DT_BF16, out=C), n)
+        fl = 2.0 * M * N * K
+        r["gemm"] = {"us": med * 1e6, "best_us": best * 1e6, "TFLOPs": fl / med / 1e12, "frac_of_4x_bf16_measured": fl / med / 1e12 / (4 * pk["bf16"]),
+                     "frac_of_9PF_nominal": fl / med / 1e12 / 9000.0}
+
+        def fused():
+            b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, out=qa, workspace=ws)
+            b.nvfp4_quantize(Bm, b.AXIS_ROW, b.ROUND_RTN, 0, 2, gs_mode, out=qb, workspace=ws)
+            b.nvfp4_gemm(qa, qb, b.DT_BF16, out=C)
+
+        med, best = t_of(fused, n)
+        r["quantize_plus_gemm"] = {"us": med * 1e6, "TFLOPs": fl / med / 1e12}
+        out.append(r)
+        del A, Bm, qa, qb, qat, C
+    print(json.dumps({"sweep": out, "gs_mode": args.gs, "peaks": pk}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -377,8 +451,12 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=1024, help="token slab of one oracle step (reference arm)")
     ap.add_argument("--cpu-tokens", type=int, default=4096, help="token slab of the cpu_baseline leg")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="roofline sweep of the large GEMM shapes instead of the step benchmark")
+    ap.add_argument("--shapes", default="", help="with --sweep: comma list of MxNxK")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -36,11 +36,11 @@ struct Cfg {
   static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;  // multiple of 1024
   static constexpr int STAGES = (BN == 128) ? 5 : 4;
   static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
-  // tensor memory columns: two accumulators, then two scale buffers (A: 16 columns, B: 16 * BN / 128)
+  // tensor memory columns: two accumulators, then four scale buffers (A: 16 columns, B: 16 * BN / 128)
   static constexpr uint32_t ACC_COLS = BN;
   static constexpr uint32_t SF_COLS = 16 + 16 * (BN / 128);
   static constexpr uint32_t TMEM_COLS = 512;
-  static_assert(2 * ACC_COLS + 2 * SF_COLS <= TMEM_COLS || BN == 256, "tensor memory budget");
+  static_assert(2 * ACC_COLS + 4 * SF_COLS <= TMEM_COLS || BN == 256, "tensor memory budget");
 };
 
 struct Params {
@@ -69,8 +69,17 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+// The issuing warps stay converged; instructions that one thread must issue take a `leader` flag (1 in exactly one
+// lane) and are predicated inside the asm, so their operands remain warp-uniform values.
+__device__ __forceinline__ uint32_t elect_leader() {
+  uint32_t pred;
+  asm volatile("{\n.reg .pred P;\nelect.sync _|P, 0xFFFFFFFF;\nselp.u32 %0, 1, 0, P;\n}" : "=r"(pred));
+  return pred;
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes, uint32_t leader) {
+  asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %2, 0;\n@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n}" ::"r"(bar),
+               "r"(bytes), "r"(leader)
+               : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -101,33 +110,44 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int32_t c0, int32_t c1, uint32_t bar) {
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int32_t c0, int32_t c1, uint32_t bar,
+                                            uint32_t leader) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(tm), "r"(c0), "r"(c1), "r"(bar)
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %5, 0;\n"
+      "@q cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n}" ::"r"(dst),
+      "l"(tm), "r"(c0), "r"(c1), "r"(bar), "r"(leader)
       : "memory");
 }
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint32_t leader) {
+  asm volatile(
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %4, 0;\n"
+      "@q cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n}" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar), "r"(leader)
+      : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+__device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t leader) {
+  asm volatile(
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %1, 0;\n"
+      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(bar),
+      "r"(leader)
+      : "memory");
 }
-__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
-  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc, uint32_t leader) {
+  asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %2, 0;\n@q tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;\n}" ::"r"(taddr),
+               "l"(sdesc), "r"(leader)
+               : "memory");
 }
 __device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate, uint32_t leader) {
   asm volatile(
-      "{\n.reg .pred p;\n"
+      "{\n.reg .pred p, q;\n"
       "setp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+      "setp.ne.b32 q, %7, 0;\n"
+      "@q tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem), "r"(leader)
       : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
@@ -205,78 +225,82 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   const int64_t num_tiles = (int64_t)p.m_tiles * p.n_tiles;
 
   if (warp == 0) {
-    // ===================================== TMA producer ====================================================
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
-        const uint8_t* sfa_src = p.a_sf + (size_t)mt * p.sf_tiles_a * 512;
-        const uint8_t* sfb_src = p.b_sf + (size_t)nt * (BN / 128) * p.sf_tiles_b * 512;
-        for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
-          const int s = it % C::STAGES;
-          const uint32_t round = it / C::STAGES;
-          if (!(ok = mbar_wait(empty_bar(s), (round & 1) ^ 1, abort_flag, p.dev_status))) break;
-          const uint32_t st = smem_base + s * C::STAGE_BYTES;
-          mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
-          tma_load_2d(st, &tmA, kt * (BK / 2), mt * BM, full_bar(s));
-          tma_load_2d(st + A_BYTES, &tmB, kt * (BK / 2), nt * BN, full_bar(s));
-          bulk_load(st + A_BYTES + C::B_BYTES, sfa_src + (size_t)kt * 2048, 2048, full_bar(s));
+    // ===================================== TMA producer (warp stays converged) ===============================
+    const uint32_t leader = elect_leader();
+    uint32_t it = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+      const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
+      const uint8_t* sfa_src = p.a_sf + (size_t)mt * p.sf_tiles_a * 512;
+      const uint8_t* sfb_src = p.b_sf + (size_t)nt * (BN / 128) * p.sf_tiles_b * 512;
+      for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
+        const int s = it % C::STAGES;
+        const uint32_t round = it / C::STAGES;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), (round & 1) ^ 1, abort_flag, p.dev_status));
+        if (!ok) break;
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        mbar_expect_tx(full_bar(s), C::STAGE_BYTES, leader);
+        tma_load_2d(st, &tmA, kt * (BK / 2), mt * BM, full_bar(s), leader);
+        tma_load_2d(st + A_BYTES, &tmB, kt * (BK / 2), nt * BN, full_bar(s), leader);
+        bulk_load(st + A_BYTES + C::B_BYTES, sfa_src + (size_t)kt * 2048, 2048, full_bar(s), leader);
 #pragma unroll
-          for (int h = 0; h < BN / 128; ++h)
-            bulk_load(st + A_BYTES + C::B_BYTES + SFA_BYTES + h * 2048,
-                      sfb_src + ((size_t)h * p.sf_tiles_b * 512) + (size_t)kt * 2048, 2048, full_bar(s));
-        }
+        for (int h = 0; h < BN / 128; ++h)
+          bulk_load(st + A_BYTES + C::B_BYTES + SFA_BYTES + h * 2048,
+                    sfb_src + ((size_t)h * p.sf_tiles_b * 512) + (size_t)kt * 2048, 2048, full_bar(s), leader);
       }
-      if (!ok) {
-        // give the copies already in flight a bounded time to land before the CTA may exit
-        const uint32_t n_back = it < (uint32_t)C::STAGES ? it : (uint32_t)C::STAGES;
-        for (uint32_t j = 0; j < n_back; ++j) {
-          const uint32_t f = it - 1 - j;
-          const long long t0 = clock64();
-          while (!mbar_try(full_bar(f % C::STAGES), (f / C::STAGES) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
-          }
+    }
+    if (!ok) {
+      // give the copies already in flight a bounded time to land before the CTA may exit
+      const uint32_t n_back = it < (uint32_t)C::STAGES ? it : (uint32_t)C::STAGES;
+      for (uint32_t j = 0; j < n_back; ++j) {
+        const uint32_t f = it - 1 - j;
+        const long long t0 = clock64();
+        while (!mbar_try(full_bar(f % C::STAGES), (f / C::STAGES) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
         }
       }
     }
   } else if (warp == 1) {
-    // ===================================== MMA issuer ======================================================
-    if (lane == 0) {
-      const uint32_t idesc = instr_desc<BN>();
-      uint32_t it = 0, tile_it = 0;
-      bool ok = true;
-      for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
-        const uint32_t ab = tile_it & 1;
-        if (!(ok = mbar_wait(acc_empty_bar(ab), ((tile_it >> 1) & 1) ^ 1, abort_flag, p.dev_status))) break;
+    // ===================================== MMA issuer (warp stays converged) =================================
+    const uint32_t leader = elect_leader();
+    const uint32_t idesc = instr_desc<BN>();
+    uint32_t it = 0, tile_it = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
+      const uint32_t ab = tile_it & 1;
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar(ab), ((tile_it >> 1) & 1) ^ 1, abort_flag, p.dev_status));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + ab * C::ACC_COLS;
+      for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
+        const int s = it % C::STAGES;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / C::STAGES) & 1, abort_flag, p.dev_status));
+        if (!ok) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + ab * C::ACC_COLS;
-        for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
-          const int s = it % C::STAGES;
-          if (!(ok = mbar_wait(full_bar(s), (it / C::STAGES) & 1, abort_flag, p.dev_status))) break;
-          tc_fence_after();
-          const uint32_t st = smem_base + s * C::STAGE_BYTES;
-          const uint32_t sf_tmem = tmem_base + 2 * C::ACC_COLS + (it & 1) * C::SF_COLS;
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        const uint32_t sf_tmem = tmem_base + 2 * C::ACC_COLS + (it & 3) * C::SF_COLS;
+        // Scales of this k tile: shared memory -> tensor memory. Per 64-wide k step: 4 columns for the 128 rows
+        // of A, 4 per 128 rows of B.
 #pragma unroll
-          for (int kk = 0; kk < BK / 64; ++kk) {
-            // scales of this 64-wide k step: 4 columns for 128 rows of A, 4 per 128 rows of B
-            tc_cp_sf(sf_tmem + kk * 4, desc_sf(st + A_BYTES + C::B_BYTES + kk * 512));
+        for (int kk = 0; kk < BK / 64; ++kk) {
+          tc_cp_sf(sf_tmem + kk * 4, desc_sf(st + A_BYTES + C::B_BYTES + kk * 512), leader);
 #pragma unroll
-            for (int h = 0; h < BN / 128; ++h)
-              tc_cp_sf(sf_tmem + 16 + (kk * (BN / 128) + h) * 4,
-                       desc_sf(st + A_BYTES + C::B_BYTES + SFA_BYTES + h * 2048 + kk * 512));
-            tc_mma_nvf4(d_tmem, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc, sf_tmem + kk * 4,
-                        sf_tmem + 16 + kk * (BN / 128) * 4, (kt | kk) != 0);
-          }
-          tc_commit(empty_bar(s));  // stage reusable once these MMAs have read it
+          for (int h = 0; h < BN / 128; ++h)
+            tc_cp_sf(sf_tmem + 16 + (kk * (BN / 128) + h) * 4,
+                     desc_sf(st + A_BYTES + C::B_BYTES + SFA_BYTES + h * 2048 + kk * 512), leader);
         }
-        if (ok) tc_commit(acc_full_bar(ab));
+#pragma unroll
+        for (int kk = 0; kk < BK / 64; ++kk)
+          tc_mma_nvf4(d_tmem, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc, sf_tmem + kk * 4,
+                      sf_tmem + 16 + kk * (BN / 128) * 4, (kt | kk) != 0, leader);
+        tc_commit(empty_bar(s), leader);  // stage reusable once these MMAs have read it
       }
-      // make sure nothing issued is still running before tensor memory is freed
-      tc_commit(drain_bar);
-      {
-        const long long t0 = clock64();
-        while (!mbar_try(drain_bar, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
-        }
+      if (ok) tc_commit(acc_full_bar(ab), leader);
+    }
+    // make sure nothing issued is still running before tensor memory is freed
+    tc_commit(drain_bar, leader);
+    {
+      const long long t0 = clock64();
+      while (!mbar_try(drain_bar, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
       }
     }
   } else {
