@@ -159,7 +159,8 @@ nvfp4_status nvfp4_requantize_t(const nvfp4_operand* in, const void* hp_bf16, in
  * nvfp4_gemm — block-scaled FP4 product of two operands (the "FP4 MM" of Sec. 2.3):
  *      C[m, n] (+)= sum_k  (Pa * Sba * Sga)[m, k] * (Pb * Sbb * Sgb)[n, k]
  * FP32 accumulation on the tensor cores; TENSOR / ROW global scales are applied in the epilogue, BLOCK128
- * scales per 128-wide k chunk.
+ * scales per 128-wide k chunk (each chunk's partial product is promoted into FP32 registers; this variant takes
+ * K up to 16384 and returns NVFP4_ERR_LIMIT beyond).
  *
  *   A [M, K], B [N, K]: same K and gs_mode, sf_layout = TILED128x4.
  *   C [M, N] row-major, leading dimension ldc (elements), dtype c_dtype; 16-byte aligned rows.

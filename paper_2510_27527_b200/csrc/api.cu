@@ -135,6 +135,7 @@ nvfp4_status do_quantize_transpose(const TransposeSrc& src, int from_codes, int6
 
 nvfp4_status do_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
                      int32_t accumulate, const float* addend, int64_t ld_add, int32_t* dev_status, cudaStream_t st) {
+  if (A->gs_mode == NVFP4_GS_BLOCK128 && nvfp4_padded_k(A->K) > gemm_block128_max_k()) return NVFP4_ERR_LIMIT;
   GemmArgs g{};
   g.a_codes = A->codes;
   g.a_sf = A->sf;

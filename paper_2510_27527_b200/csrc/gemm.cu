@@ -14,6 +14,7 @@
 // the CTA frees its tensor memory and exits.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cstdlib>
 
 #include "nvfp4_device.cuh"
 #include "nvfp4_internal.h"
@@ -38,9 +39,10 @@ struct Cfg {
   static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
   // tensor memory columns: two accumulators, then four scale buffers (A: 16 columns, B: 16 * BN / 128)
   static constexpr uint32_t ACC_COLS = BN;
+  static constexpr uint32_t ACC_BUFS = (BN == 256) ? 1 : 2;  // 256-wide accumulators leave no room for a second one
   static constexpr uint32_t SF_COLS = 16 + 16 * (BN / 128);
   static constexpr uint32_t TMEM_COLS = 512;
-  static_assert(2 * ACC_COLS + 4 * SF_COLS <= TMEM_COLS || BN == 256, "tensor memory budget");
+  static_assert(ACC_BUFS * ACC_COLS + 4 * SF_COLS <= TMEM_COLS, "tensor memory budget");
 };
 
 struct Params {
@@ -54,6 +56,8 @@ struct Params {
   int64_t ldc;
   int64_t M, N;
   int32_t k_tiles;        // number of 256-wide k tiles
+  int32_t k_chunks;       // number of 128-wide k chunks (BLOCK128 variant)
+  int64_t g_per_row;      // global scales per operand row in BLOCK128 mode
   int32_t sf_tiles_a;     // 512-byte scale tiles per 128-row tile of A (= padded k-blocks / 4)
   int32_t sf_tiles_b;
   int32_t m_tiles, n_tiles;
@@ -179,6 +183,67 @@ __device__ __forceinline__ uint32_t instr_desc() {
   return (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (0u << 23) | ((uint32_t)(BM >> 4) << 24);
 }
 
+// One output row, 32 consecutive columns starting at n0 (m < M and n0 < N are the caller's business): add the optional
+// FP32 addend and the old C when accumulating, convert, store.
+__device__ __forceinline__ void store_row_chunk(const Params& p, int64_t m, int64_t n0, float (&o)[32]) {
+    if (p.addend) {
+      const float* ad = p.addend + m * p.ld_add + n0;
+      if (n0 + 32 <= p.N) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const float4 q = *reinterpret_cast<const float4*>(ad + j);
+          o[j] += q.x; o[j + 1] += q.y; o[j + 2] += q.z; o[j + 3] += q.w;
+        }
+      } else {
+        for (int j = 0; j < 32 && n0 + j < p.N; ++j) o[j] += ad[j];
+      }
+    }
+    if (p.c_is_f32) {
+      float* cp = reinterpret_cast<float*>(p.C) + m * p.ldc + n0;
+      if (n0 + 32 <= p.N) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          float4 q = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
+          if (p.accumulate) {
+            const float4 old = *reinterpret_cast<const float4*>(cp + j);
+            q.x += old.x; q.y += old.y; q.z += old.z; q.w += old.w;
+          }
+          *reinterpret_cast<float4*>(cp + j) = q;
+        }
+      } else {
+        for (int j = 0; j < 32 && n0 + j < p.N; ++j) cp[j] = p.accumulate ? cp[j] + o[j] : o[j];
+      }
+    } else {
+      __nv_bfloat16* cp = reinterpret_cast<__nv_bfloat16*>(p.C) + m * p.ldc + n0;
+      if (n0 + 32 <= p.N) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          if (p.accumulate) {
+            const uint4 old = *reinterpret_cast<const uint4*>(cp + j);
+            const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              o[j + 2 * q] += bf16_lo(ow[q]);
+              o[j + 2 * q + 1] += bf16_hi(ow[q]);
+            }
+          }
+          uint4 q;
+          __nv_bfloat162 h;
+          h = __floats2bfloat162_rn(o[j], o[j + 1]); q.x = *reinterpret_cast<uint32_t*>(&h);
+          h = __floats2bfloat162_rn(o[j + 2], o[j + 3]); q.y = *reinterpret_cast<uint32_t*>(&h);
+          h = __floats2bfloat162_rn(o[j + 4], o[j + 5]); q.z = *reinterpret_cast<uint32_t*>(&h);
+          h = __floats2bfloat162_rn(o[j + 6], o[j + 7]); q.w = *reinterpret_cast<uint32_t*>(&h);
+          *reinterpret_cast<uint4*>(cp + j) = q;
+        }
+      } else {
+        for (int j = 0; j < 32 && n0 + j < p.N; ++j) {
+          const float prev = p.accumulate ? __bfloat162float(cp[j]) : 0.0f;
+          cp[j] = __float2bfloat16_rn(o[j] + prev);
+        }
+      }
+    }
+}
+
 template <int GS, int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
@@ -266,8 +331,8 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     uint32_t it = 0, tile_it = 0;
     bool ok = true;
     for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
-      const uint32_t ab = tile_it & 1;
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar(ab), ((tile_it >> 1) & 1) ^ 1, abort_flag, p.dev_status));
+      const uint32_t ab = tile_it % C::ACC_BUFS;
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar(ab), ((tile_it / C::ACC_BUFS) & 1) ^ 1, abort_flag, p.dev_status));
       if (!ok) break;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + ab * C::ACC_COLS;
@@ -277,7 +342,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (!ok) break;
         tc_fence_after();
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
-        const uint32_t sf_tmem = tmem_base + 2 * C::ACC_COLS + (it & 3) * C::SF_COLS;
+        const uint32_t sf_tmem = tmem_base + C::ACC_BUFS * C::ACC_COLS + (it & 3) * C::SF_COLS;
         // Scales of this k tile: shared memory -> tensor memory. Per 64-wide k step: 4 columns for the 128 rows
         // of A, 4 per 128 rows of B.
 #pragma unroll
@@ -312,8 +377,8 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     if (GS == kGsTensor) alpha = __fmul_rn(p.a_gscale[0], p.b_gscale[0]);
     for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
       const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
-      const uint32_t ab = tile_it & 1;
-      if (!(ok = mbar_wait(acc_full_bar(ab), (tile_it >> 1) & 1, abort_flag, p.dev_status))) break;
+      const uint32_t ab = tile_it % C::ACC_BUFS;
+      if (!(ok = mbar_wait(acc_full_bar(ab), (tile_it / C::ACC_BUFS) & 1, abort_flag, p.dev_status))) break;
       tc_fence_after();
       const int64_t m = (int64_t)mt * BM + quad * 32 + lane;
       float sa = 1.0f;
@@ -332,62 +397,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (GS == kGsRow) sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
             o[j] = __uint_as_float(v[j]) * sc;
           }
-          if (p.addend) {
-            const float* ad = p.addend + m * p.ld_add + n0;
-            if (n0 + 32 <= p.N) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                const float4 q = *reinterpret_cast<const float4*>(ad + j);
-                o[j] += q.x; o[j + 1] += q.y; o[j + 2] += q.z; o[j + 3] += q.w;
-              }
-            } else {
-              for (int j = 0; j < 32 && n0 + j < p.N; ++j) o[j] += ad[j];
-            }
-          }
-          if (p.c_is_f32) {
-            float* cp = reinterpret_cast<float*>(p.C) + m * p.ldc + n0;
-            if (n0 + 32 <= p.N) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                float4 q = make_float4(o[j], o[j + 1], o[j + 2], o[j + 3]);
-                if (p.accumulate) {
-                  const float4 old = *reinterpret_cast<const float4*>(cp + j);
-                  q.x += old.x; q.y += old.y; q.z += old.z; q.w += old.w;
-                }
-                *reinterpret_cast<float4*>(cp + j) = q;
-              }
-            } else {
-              for (int j = 0; j < 32 && n0 + j < p.N; ++j) cp[j] = p.accumulate ? cp[j] + o[j] : o[j];
-            }
-          } else {
-            __nv_bfloat16* cp = reinterpret_cast<__nv_bfloat16*>(p.C) + m * p.ldc + n0;
-            if (n0 + 32 <= p.N) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                if (p.accumulate) {
-                  const uint4 old = *reinterpret_cast<const uint4*>(cp + j);
-                  const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
-#pragma unroll
-                  for (int q = 0; q < 4; ++q) {
-                    o[j + 2 * q] += bf16_lo(ow[q]);
-                    o[j + 2 * q + 1] += bf16_hi(ow[q]);
-                  }
-                }
-                uint4 q;
-                __nv_bfloat162 h;
-                h = __floats2bfloat162_rn(o[j], o[j + 1]); q.x = *reinterpret_cast<uint32_t*>(&h);
-                h = __floats2bfloat162_rn(o[j + 2], o[j + 3]); q.y = *reinterpret_cast<uint32_t*>(&h);
-                h = __floats2bfloat162_rn(o[j + 4], o[j + 5]); q.z = *reinterpret_cast<uint32_t*>(&h);
-                h = __floats2bfloat162_rn(o[j + 6], o[j + 7]); q.w = *reinterpret_cast<uint32_t*>(&h);
-                *reinterpret_cast<uint4*>(cp + j) = q;
-              }
-            } else {
-              for (int j = 0; j < 32 && n0 + j < p.N; ++j) {
-                const float prev = p.accumulate ? __bfloat162float(cp[j]) : 0.0f;
-                cp[j] = __float2bfloat16_rn(o[j] + prev);
-              }
-            }
-          }
+          store_row_chunk(p, m, n0, o);
         }
       }
       tc_fence_before();
@@ -402,6 +412,211 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::TMEM_COLS) : "memory");
+  }
+}
+
+// =========================================================================================================
+// BLOCK128 variant: the FP32 global scale changes every 128 k (the paper's 1x128 outer block, Sec. 2.2), so a
+// partial product can only be accumulated over 128 k inside tensor memory. The MMA warp writes each 128-k partial
+// (two K = 64 instructions) into one of three tensor-memory buffers; the epilogue warps pull it out and promote it
+// into FP32 register accumulators with the rank-1 scale SgA[m, kc] * SgB[n, kc] (packed f32x2 FMAs). The SgB values
+// of the tile, for all chunks, are staged in shared memory once per tile ([chunk][n] so a warp reads them as
+// broadcasts). 128 x 128 tiles, K <= 16384.
+// =========================================================================================================
+constexpr int B128_STAGES = 4;
+constexpr int B128_NBUF = 3;
+constexpr int B128_MAX_CHUNKS = 128;
+constexpr uint32_t B128_SGB_BYTES = B128_MAX_CHUNKS * 128 * 4;
+constexpr uint32_t B128_SMEM_BYTES = B128_STAGES * Cfg<128>::STAGE_BYTES + B128_SGB_BYTES + 1024 + 256;
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
+  using C = Cfg<128>;
+  constexpr int BN = 128;
+  constexpr int STAGES = B128_STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  float* sgb = reinterpret_cast<float*>(smem_gen + STAGES * C::STAGE_BYTES);
+  const uint32_t bar_base = smem_base + STAGES * C::STAGE_BYTES + B128_SGB_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+  auto part_full_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+  auto part_empty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + B128_NBUF + b); };
+  const uint32_t drain_bar = bar_base + 8u * (2 * STAGES + 2 * B128_NBUF);
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int b = 0; b < B128_NBUF; ++b) {
+      mbar_init(part_full_bar(b), 1);
+      mbar_init(part_empty_bar(b), 4);
+    }
+    mbar_init(drain_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  const int64_t num_tiles = (int64_t)p.m_tiles * p.n_tiles;
+  const int32_t chunks = p.k_chunks;  // 128-wide k chunks per tile
+
+  if (warp == 0) {
+    const uint32_t leader = elect_leader();
+    uint32_t it = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+      const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
+      const uint8_t* sfa_src = p.a_sf + (size_t)mt * p.sf_tiles_a * 512;
+      const uint8_t* sfb_src = p.b_sf + (size_t)nt * p.sf_tiles_b * 512;
+      for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
+        const int s = it % STAGES;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.dev_status));
+        if (!ok) break;
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        mbar_expect_tx(full_bar(s), C::STAGE_BYTES, leader);
+        tma_load_2d(st, &tmA, kt * (BK / 2), mt * BM, full_bar(s), leader);
+        tma_load_2d(st + A_BYTES, &tmB, kt * (BK / 2), nt * BN, full_bar(s), leader);
+        bulk_load(st + A_BYTES + C::B_BYTES, sfa_src + (size_t)kt * 2048, 2048, full_bar(s), leader);
+        bulk_load(st + A_BYTES + C::B_BYTES + SFA_BYTES, sfb_src + (size_t)kt * 2048, 2048, full_bar(s), leader);
+      }
+    }
+    if (!ok) {
+      const uint32_t n_back = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
+      for (uint32_t j = 0; j < n_back; ++j) {
+        const uint32_t f = it - 1 - j;
+        const long long t0 = clock64();
+        while (!mbar_try(full_bar(f % STAGES), (f / STAGES) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
+        }
+      }
+    }
+  } else if (warp == 1) {
+    const uint32_t leader = elect_leader();
+    const uint32_t idesc = instr_desc<BN>();
+    uint32_t it = 0, cit = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+      for (int32_t kt = 0; kt < p.k_tiles && ok; ++kt, ++it) {
+        const int s = it % STAGES;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.dev_status));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        const uint32_t sf_tmem = tmem_base + B128_NBUF * 128 + (it & 3) * C::SF_COLS;
+#pragma unroll
+        for (int kk = 0; kk < BK / 64; ++kk) {
+          tc_cp_sf(sf_tmem + kk * 4, desc_sf(st + A_BYTES + C::B_BYTES + kk * 512), leader);
+          tc_cp_sf(sf_tmem + 16 + kk * 4, desc_sf(st + A_BYTES + C::B_BYTES + SFA_BYTES + kk * 512), leader);
+        }
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          if (kt * 2 + half >= chunks) break;  // the padded half of the last k tile holds only zeros
+          const uint32_t buf = cit % B128_NBUF;
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(part_empty_bar(buf), ((cit / B128_NBUF) & 1) ^ 1, abort_flag, p.dev_status));
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + buf * 128;
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+            const int kk = 2 * half + q;
+            tc_mma_nvf4(d_tmem, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc, sf_tmem + kk * 4,
+                        sf_tmem + 16 + kk * 4, q, leader);
+          }
+          tc_commit(part_full_bar(buf), leader);
+          ++cit;
+        }
+        tc_commit(empty_bar(s), leader);
+      }
+    }
+    tc_commit(drain_bar, leader);
+    {
+      const long long t0 = clock64();
+      while (!mbar_try(drain_bar, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
+      }
+    }
+  } else {
+    // ---- promotion + epilogue: thread = one output row, 128 FP32 accumulators in registers -----------------
+    const int quad = warp & 3;
+    const int epi_tid = (warp - 2) * 32 + lane;  // 0..127
+    const int64_t G = p.g_per_row;               // global scales per operand row (= padded K / 128)
+    uint32_t cit = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+      const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
+      // stage SgB[n, :] of this tile as sgb[chunk][n]
+      asm volatile("bar.sync 1, 128;" ::: "memory");  // everyone is done with the previous tile's values
+      {
+        const int64_t n = (int64_t)nt * BN + epi_tid;
+        const float* src = p.b_gscale + n * G;
+        for (int32_t kc = 0; kc < chunks; ++kc) sgb[kc * 128 + epi_tid] = (n < p.N) ? __ldg(src + kc) : 0.0f;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      const int64_t m = (int64_t)mt * BM + quad * 32 + lane;
+      const float* sa_row = p.a_gscale + (m < p.M ? m : 0) * G;
+      float2 acc[64];
+#pragma unroll
+      for (int j = 0; j < 64; ++j) acc[j] = make_float2(0.0f, 0.0f);
+      for (int32_t kc = 0; kc < chunks && ok; ++kc, ++cit) {
+        const uint32_t buf = cit % B128_NBUF;
+        if (!(ok = mbar_wait(part_full_bar(buf), (cit / B128_NBUF) & 1, abort_flag, p.dev_status))) break;
+        tc_fence_after();
+        const float sa = __ldg(sa_row + kc);
+        const float2 sa2 = make_float2(sa, sa);
+        const float4* sb4 = reinterpret_cast<const float4*>(sgb + kc * 128);
+#pragma unroll
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          uint32_t v[32];
+          tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * 128 + c0, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 sb = sb4[(c0 + j) >> 2];
+            const float2 t0 = __fmul2_rn(make_float2(__uint_as_float(v[j]), __uint_as_float(v[j + 1])), sa2);
+            const float2 t1 = __fmul2_rn(make_float2(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])), sa2);
+            acc[(c0 + j) >> 1] = __ffma2_rn(t0, make_float2(sb.x, sb.y), acc[(c0 + j) >> 1]);
+            acc[((c0 + j) >> 1) + 1] = __ffma2_rn(t1, make_float2(sb.z, sb.w), acc[((c0 + j) >> 1) + 1]);
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(part_empty_bar(buf));
+      }
+      if (ok && m < p.M) {
+#pragma unroll
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+          const int64_t n0 = (int64_t)nt * BN + c0;
+          if (n0 < p.N) {
+            float o[32];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              o[2 * j] = acc[(c0 >> 1) + j].x;
+              o[2 * j + 1] = acc[(c0 >> 1) + j].y;
+            }
+            store_row_chunk(p, m, n0, o);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 
@@ -467,6 +682,8 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
   p.M = a.M;
   p.N = a.N;
   p.k_tiles = (int32_t)((Kp + BK - 1) / BK);
+  p.k_chunks = (int32_t)(Kp / 128);
+  p.g_per_row = Kp / 128;
   const int64_t kb_padded = ((Kp >> 4) + 15) & ~(int64_t)15;
   p.sf_tiles_a = p.sf_tiles_b = (int32_t)(kb_padded >> 2);
   p.m_tiles = (int32_t)((a.M + BM - 1) / BM);
@@ -488,16 +705,60 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+cudaError_t launch_block128(const GemmArgs& a, cudaStream_t st) {
+  const int64_t Kp = (a.K + 127) & ~(int64_t)127;
+  if (Kp / 128 > B128_MAX_CHUNKS) return cudaErrorInvalidValue;
+  CUtensorMap tmA, tmB;
+  if (!make_codes_map(&tmA, a.a_codes, a.M, Kp, BM) || !make_codes_map(&tmB, a.b_codes, a.N, Kp, 128)) return cudaErrorInvalidValue;
+  Params p{};
+  p.a_sf = a.a_sf;
+  p.b_sf = a.b_sf;
+  p.a_gscale = a.a_gscale;
+  p.b_gscale = a.b_gscale;
+  p.addend = a.addend;
+  p.ld_add = a.ld_add;
+  p.C = a.C;
+  p.ldc = a.ldc;
+  p.M = a.M;
+  p.N = a.N;
+  p.k_tiles = (int32_t)((Kp + BK - 1) / BK);
+  p.k_chunks = (int32_t)(Kp / 128);
+  p.g_per_row = Kp / 128;
+  const int64_t kb_padded = ((Kp >> 4) + 15) & ~(int64_t)15;
+  p.sf_tiles_a = p.sf_tiles_b = (int32_t)(kb_padded >> 2);
+  p.m_tiles = (int32_t)((a.M + BM - 1) / BM);
+  p.n_tiles = (int32_t)((a.N + 127) / 128);
+  p.c_is_f32 = a.c_is_f32;
+  p.accumulate = a.accumulate;
+  p.dev_status = a.dev_status;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_block128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)B128_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
+  const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
+  gemm_nvfp4_block128_kernel<<<grid, NUM_THREADS, B128_SMEM_BYTES, st>>>(tmA, tmB, p);
+  ++g_launch_count;
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 size_t gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
+int64_t gemm_block128_max_k() { return (int64_t)B128_MAX_CHUNKS * 128; }
 
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;
+  // 128 x 256 tiles halve the operand traffic per flop; they pay off once there are enough of them to fill the SMs.
+  const char* force = getenv("NVFP4_GEMM_BN");
+  const bool wide = force ? atoi(force) == 256 : (((a.M + 127) / 128) * ((a.N + 255) / 256) >= 2 * sm_count());
   switch (a.gs_mode) {
-    case kGsTensor: return launch_variant<kGsTensor, 128>(a, st);
-    case kGsRow: return launch_variant<kGsRow, 128>(a, st);
-    default: return cudaErrorNotSupported;
+    case kGsTensor: return wide ? launch_variant<kGsTensor, 256>(a, st) : launch_variant<kGsTensor, 128>(a, st);
+    case kGsRow: return wide ? launch_variant<kGsRow, 256>(a, st) : launch_variant<kGsRow, 128>(a, st);
+    default: return launch_block128(a, st);
   }
 }
 

@@ -75,6 +75,7 @@ struct GemmArgs {
   size_t ws_bytes;
 };
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int64_t gemm_block128_max_k();  // largest K the BLOCK128 GEMM variant takes
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
 
 // High-precision (BF16 inputs, FP32 accumulate) products over OutControl's outlier channels.

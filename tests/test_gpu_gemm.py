@@ -61,7 +61,7 @@ def test_code_layout_one_hot_probe():
         assert not C.any()
 
 
-@pytest.mark.parametrize("gs_mode", [0, 1])
+@pytest.mark.parametrize("gs_mode", [0, 1, 2])
 @pytest.mark.parametrize("shape", [(128, 128, 256), (256, 384, 1024), (130, 70, 144), (1, 8, 16), (300, 520, 640)])
 def test_exact_on_integer_valued_operands(gs_mode, shape):
     """Power-of-two scales and small-integer codes: every partial sum is an integer below 2^24, so FP32
@@ -76,7 +76,8 @@ def test_exact_on_integer_valued_operands(gs_mode, shape):
         nib[:, K:] = 0
         codes = (nib[:, 0::2] | (nib[:, 1::2] << 4)).astype(np.uint8)
         sf = rng.choice([0x30, 0x38, 0x40], size=(R, K16 // 16)).astype(np.uint8)  # 0.5, 1, 2
-        gs = {0: np.array([0.25], dtype=np.float32), 1: rng.choice([0.5, 1.0, 4.0], size=R).astype(np.float32)}[gs_mode]
+        gs = {0: np.array([0.25], dtype=np.float32), 1: rng.choice([0.5, 1.0, 4.0], size=R).astype(np.float32),
+              2: rng.choice([0.5, 1.0, 4.0], size=(R, (K + 127) // 128)).astype(np.float32)}[gs_mode]
         return orc.Operand(codes, sf, gs, R, K, gs_mode)
 
     a, bb = rnd_operand(M), rnd_operand(N)
@@ -85,7 +86,7 @@ def test_exact_on_integer_valued_operands(gs_mode, shape):
     assert np.array_equal(got.astype(np.float64), want)
 
 
-@pytest.mark.parametrize("gs_mode", [0, 1])
+@pytest.mark.parametrize("gs_mode", [0, 1, 2])
 @pytest.mark.parametrize("shape", [(256, 512, 512), (384, 256, 2048), (200, 136, 400), (512, 1024, 4096)])
 def test_random_operands_against_fp64(gs_mode, shape):
     b = B()
@@ -118,9 +119,40 @@ def test_gemm_consumes_device_quantizer_output():
     M, N, K = 384, 640, 1024
     x, _ = synth.activations(M, K, 5, n_outlier=8, factor=30.0)
     w = synth.weights(N, K, 6)
-    for gs_mode in (0, 1):
+    for gs_mode in (0, 1, 2):
         qa = b.nvfp4_quantize(to_dev_bf16(x), b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode)
         qb = b.nvfp4_quantize(to_dev_bf16(w), b.AXIS_ROW, b.ROUND_RTN, 0, 2, gs_mode)
         got = b.nvfp4_gemm(qa, qb, b.DT_F32).cpu().numpy()
         want = orc.gemm_operands(orc.quantize(x, gs_mode=gs_mode), orc.quantize(w, gs_mode=gs_mode))
         assert rel_fro(got, want) <= 1e-5
+
+
+def test_block128_gemm_k_limit_is_reported():
+    """The outer-block (BLOCK128) product keeps the tile's global scales in shared memory: K up to 16384."""
+    b = B()
+    a = b.alloc_operand(128, 16384 + 128, b.GS_BLOCK128)
+    with pytest.raises(b.Nvfp4Error) as e:
+        b.nvfp4_gemm(a, a, b.DT_F32)
+    assert e.value.status == 9
+    ok = b.alloc_operand(128, 16384, b.GS_BLOCK128)
+    ok.gscale.fill_(1.0)
+    C = b.nvfp4_gemm(ok, ok, b.DT_F32)
+    torch.cuda.synchronize()
+    assert not C.any()
+
+
+def test_block128_scale_layout_one_hot_probe():
+    """All codes and block scales 1.0; one outer-block scale of A (or B) doubled: exactly that row (column) of C
+    grows by 128."""
+    b = B()
+    M, N, K = 256, 128, 640
+    for which, (r, g) in (("A", (130, 3)), ("B", (77, 0)), ("A", (0, 4)), ("B", (127, 2))):
+        a, bb = const_operand(M, K, 2, 0x38, 2), const_operand(N, K, 2, 0x38, 2)
+        (a if which == "A" else bb).gscale[r, g] = 2.0
+        C = b.nvfp4_gemm(upload_operand(a, b), upload_operand(bb, b), b.DT_F32).cpu().numpy()
+        expect = np.full((M, N), float(K))
+        if which == "A":
+            expect[r, :] += 128
+        else:
+            expect[:, r] += 128
+        assert np.array_equal(C, expect), (which, r, g)

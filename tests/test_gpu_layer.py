@@ -28,7 +28,7 @@ def run_layer(b, X, W, dY, gs_mode, outliers, f32_out=True, seed=0):
     return Y.float().cpu().numpy(), dX.float().cpu().numpy(), dW.float().cpu().numpy(), saved
 
 
-@pytest.mark.parametrize("gs_mode", [0, 1])
+@pytest.mark.parametrize("gs_mode", [0, 1, 2])
 @pytest.mark.parametrize("outcontrol", [False, True])
 def test_config1_layer(gs_mode, outcontrol):
     b = B()
@@ -72,7 +72,7 @@ def test_ragged_layer_shapes():
     N_tok, D, C = 200, 272, 136
     X, W, dY, ch = synth.layer_inputs(9, N_tok, D, C, n_outlier=3, factor=40.0, grad_scale=1e-3)
     for outl in (None, ch):
-        for gs_mode in (0, 1):
+        for gs_mode in (0, 1, 2):
             ocfg = orc.LayerConfig(gs_mode=gs_mode, seed=3, outliers=outl)
             Yo, so = orc.linear_fwd(X, W, ocfg)
             dXo, dWo = orc.linear_bwd_dx(dY, so, ocfg), orc.linear_bwd_dw(dY, so, ocfg)
