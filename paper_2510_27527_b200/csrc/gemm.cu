@@ -754,7 +754,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;
   // 128 x 256 tiles halve the operand traffic per flop; they pay off once there are enough of them to fill the SMs.
   const char* force = getenv("NVFP4_GEMM_BN");
-  const bool wide = force ? atoi(force) == 256 : (((a.M + 127) / 128) * ((a.N + 255) / 256) >= 2 * sm_count());
+  const bool wide = force ? atoi(force) == 256 : (a.K >= 2048 && ((a.M + 127) / 128) * ((a.N + 255) / 256) >= 2 * sm_count());
   switch (a.gs_mode) {
     case kGsTensor: return wide ? launch_variant<kGsTensor, 256>(a, st) : launch_variant<kGsTensor, 128>(a, st);
     case kGsRow: return wide ? launch_variant<kGsRow, 256>(a, st) : launch_variant<kGsRow, 128>(a, st);

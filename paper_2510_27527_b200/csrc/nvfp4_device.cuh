@@ -92,23 +92,20 @@ __device__ __forceinline__ uint4 sr_words(uint64_t seed, uint32_t stream_id, uin
 // ---------------------------------------------------------------------------------------------------------
 // Element rounding to E2M1 (paper Sec. 2.1). Codes: sign << 3 | magnitude index.
 // ---------------------------------------------------------------------------------------------------------
-// Stochastic rounding of one scaled value with a 16-bit draw u. Exact: the comparison
-//   (u + 0.5) / 65536 < (a - q1) / (q2 - q1)
-// is evaluated on integers (a >= 1, where the fraction is the low 22 mantissa bits) or on exactly
-// representable floats (a < 1, where the grid step is 0.5).
-__device__ __forceinline__ uint32_t e2m1_sr(float y, uint32_t u) {
+// Stochastic rounding of one scaled value. `r22` carries the element's 16-bit draw u as
+//     r22 = 2^22 - 1 - ((2u + 1) << 5) = ((~u & 0xFFFF) << 6) | 0x1F.
+// The rule "round up iff (u + 0.5) / 65536 < (a - q1) / (q2 - q1)" is evaluated exactly with one integer add:
+//   * for a >= 1 the E2M1 cell of a is (bits >> 22) - 252 and the low 22 mantissa bits are the position inside the
+//     cell in units of 2^-22 of the cell width;
+//   * for a < 1 the cells [0, .5) and [.5, 1) are mapped onto [.5, .75) and [.75, 1) by z = 0.5 + a / 2, computed
+//     with round-up so that the low bits are ceil(position * 2^22) (an integer n is < x iff n < ceil(x); when the
+//     ceiling crosses into the next cell the true position was within 2^-24 of 1, where every draw rounds up);
+//   then position + r22 carries into the cell index iff position > (2u + 1) << 5.
+__device__ __forceinline__ uint32_t e2m1_sr(float y, uint32_t r22) {
   const float a = fminf(fabsf(y), 6.0f);
-  const uint32_t bits = __float_as_uint(a);
-  const uint32_t t = 2u * u + 1u;
-  uint32_t idx, up;
-  if (a >= 1.0f) {
-    idx = (bits >> 22) - 252u;  // 1 -> 2, 1.5 -> 3, 2 -> 4, 3 -> 5, 4 -> 6, 6 -> 7
-    up = (t << 5) < (bits & 0x3FFFFFu);
-  } else {
-    idx = a >= 0.5f;
-    up = (float)t < (a - 0.5f * (float)idx) * 262144.0f;
-  }
-  return (idx + up) | ((__float_as_uint(y) >> 28) & 8u);
+  const float z = (a < 1.0f) ? __fmaf_ru(a, 0.5f, 0.5f) : a;
+  const uint32_t m = ((__float_as_uint(z) + r22) >> 22) - 252u;
+  return m | ((__float_as_uint(y) >> 28) & 8u);
 }
 
 // Round-to-nearest (ties to the even code, saturating) of 8 scaled values, packed low nibble first.
@@ -133,8 +130,10 @@ __device__ __forceinline__ uint32_t e2m1x8_sr(const float (&y)[8], const uint4& 
   uint32_t out = 0;
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
-    const uint32_t u = (ww[e >> 1] >> (16 * (e & 1))) & 0xFFFFu;
-    out |= e2m1_sr(y[e], u) << (4 * e);
+    // ((~u & 0xFFFF) << 6) | 0x1F with u the low (even e) or high (odd e) half of the word
+    const uint32_t nw = ~ww[e >> 1];
+    const uint32_t r22 = (((e & 1) ? (nw >> 10) : (nw << 6)) & 0x3FFFC0u) | 0x1Fu;
+    out |= e2m1_sr(y[e], r22) << (4 * e);
   }
   return out;
 }
