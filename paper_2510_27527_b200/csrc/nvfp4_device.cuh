@@ -2,6 +2,7 @@
 // counter-based random generator. Everything that can change a code or a scale is an explicit IEEE binary32
 // operation (__fdiv_rn / __fmul_rn, no fast-math, no contraction), in the order the quantizer's contract fixes.
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -23,7 +24,11 @@ __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w 
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 // |x| of both halves as 16-bit patterns; for finite BF16 the pattern order is the value order.
 __device__ __forceinline__ uint32_t bf16x2_abs_bits(uint32_t w) { return w & 0x7FFF7FFFu; }
-__device__ __forceinline__ uint32_t umax16x2(uint32_t a, uint32_t b) { return __vmaxu2(a, b); }
+// max of two packed pairs of non-negative BF16 patterns (as 16-bit unsigned integers == as BF16 values)
+__device__ __forceinline__ uint32_t umax16x2(uint32_t a, uint32_t b) {
+  const __nv_bfloat162 r = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+  return *reinterpret_cast<const uint32_t*>(&r);
+}
 __device__ __forceinline__ uint32_t hmax_of_pair(uint32_t m) { return max(m & 0xFFFFu, m >> 16); }
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t b16) { return __uint_as_float(b16 << 16); }
 
@@ -92,20 +97,21 @@ __device__ __forceinline__ uint4 sr_words(uint64_t seed, uint32_t stream_id, uin
 // ---------------------------------------------------------------------------------------------------------
 // Element rounding to E2M1 (paper Sec. 2.1). Codes: sign << 3 | magnitude index.
 // ---------------------------------------------------------------------------------------------------------
-// Stochastic rounding of one scaled value. `r22` carries the element's 16-bit draw u as
-//     r22 = 2^22 - 1 - ((2u + 1) << 5) = ((~u & 0xFFFF) << 6) | 0x1F.
-// The rule "round up iff (u + 0.5) / 65536 < (a - q1) / (q2 - q1)" is evaluated exactly with one integer add:
-//   * for a >= 1 the E2M1 cell of a is (bits >> 22) - 252 and the low 22 mantissa bits are the position inside the
-//     cell in units of 2^-22 of the cell width;
-//   * for a < 1 the cells [0, .5) and [.5, 1) are mapped onto [.5, .75) and [.75, 1) by z = 0.5 + a / 2, computed
-//     with round-up so that the low bits are ceil(position * 2^22) (an integer n is < x iff n < ceil(x); when the
-//     ceiling crosses into the next cell the true position was within 2^-24 of 1, where every draw rounds up);
-//   then position + r22 carries into the cell index iff position > (2u + 1) << 5.
-__device__ __forceinline__ uint32_t e2m1_sr(float y, uint32_t r22) {
+// Stochastic rounding. For an element with 16-bit draw u the rule is
+//     round the magnitude up  iff  (u + 0.5) / 65536 < (a - q1) / (q2 - q1),   a = min(|y|, 6) in [q1, q2).
+// It is evaluated exactly with one integer add on the bits of a float z:
+//   * for a >= 1, z = a: the E2M1 cell of a is (bits >> 22) - 252 and the low 22 mantissa bits are the position inside
+//     the cell in units of 2^-22 of the cell width;
+//   * for a < 1 the cells [0, .5) and [.5, 1) are mapped onto [.5, .75) and [.75, 1) by z = 0.5 + a / 2, computed with
+//     round-up so that the low bits are ceil(position * 2^22) (an integer n is < x iff n < ceil(x); when the ceiling
+//     crosses into the next cell the true position was within 2^-24 of 1, where every draw rounds up);
+//     0.5 + a / 2 >= a exactly when a <= 1, so z = max(a, 0.5 + a / 2) picks the right branch;
+//   * adding r22 = 2^22 - 1 - ((2u + 1) << 5) = ((~u & 0xFFFF) << 6) | 0x1F carries into the cell index iff
+//     position > (2u + 1) << 5; adding -(252 << 22) as well leaves the magnitude index 0..7 in bits 22..24.
+__device__ __forceinline__ uint32_t e2m1_sr_bits(float y, uint32_t c) {
   const float a = fminf(fabsf(y), 6.0f);
-  const float z = (a < 1.0f) ? __fmaf_ru(a, 0.5f, 0.5f) : a;
-  const uint32_t m = ((__float_as_uint(z) + r22) >> 22) - 252u;
-  return m | ((__float_as_uint(y) >> 28) & 8u);
+  const float z = fmaxf(a, __fmaf_ru(a, 0.5f, 0.5f));
+  return __float_as_uint(z) + c;  // magnitude index in bits 22..24, nothing above
 }
 
 // Round-to-nearest (ties to the even code, saturating) of 8 scaled values, packed low nibble first.
@@ -124,16 +130,21 @@ __device__ __forceinline__ uint32_t e2m1x8_rtn(const float (&y)[8]) {
   return out;
 }
 
-// Stochastic rounding of 8 scaled values with the draws packed in w (two 16-bit draws per word).
+// Stochastic rounding of 8 scaled values with the draws packed in w (two 16-bit draws per word), packed low nibble
+// first. The sign bits are those of y.
 __device__ __forceinline__ uint32_t e2m1x8_sr(const float (&y)[8], const uint4& w) {
   const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
   uint32_t out = 0;
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
-    // ((~u & 0xFFFF) << 6) | 0x1F with u the low (even e) or high (odd e) half of the word
     const uint32_t nw = ~ww[e >> 1];
-    const uint32_t r22 = (((e & 1) ? (nw >> 10) : (nw << 6)) & 0x3FFFC0u) | 0x1Fu;
-    out |= e2m1_sr(y[e], r22) << (4 * e);
+    // ((~u & 0xFFFF) << 6) | 0x1F, minus 252 << 22 (the two fields do not overlap)
+    const uint32_t c = (((e & 1) ? (nw >> 10) : (nw << 6)) & 0x3FFFC0u) | 0xC100001Fu;
+    const uint32_t v = e2m1_sr_bits(y[e], c);
+    const int sh = 22 - 4 * e;
+    const uint32_t mag = (sh >= 0 ? (v >> sh) : (v << -sh)) & (7u << (4 * e));
+    const int ss = 28 - 4 * e;  // sign bit 31 -> bit 4e + 3
+    out |= mag | ((__float_as_uint(y[e]) >> ss) & (8u << (4 * e)));
   }
   return out;
 }

@@ -19,6 +19,23 @@ __global__ void __launch_bounds__(256) amax_tensor_bf16_kernel(const uint16_t* _
   const int64_t chunks_per_row = (cols + 7) >> 3;
   const int64_t total = rows * chunks_per_row;
   uint32_t m = 0;
+  if (ld == cols && (cols & 7) == 0) {  // one contiguous run of 16-byte chunks: no row arithmetic, four loads in flight
+    const uint4* p4 = reinterpret_cast<const uint4*>(src);
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + 3 * stride < total; i += 4 * stride) {
+      const uint4 v0 = p4[i], v1 = p4[i + stride], v2 = p4[i + 2 * stride], v3 = p4[i + 3 * stride];
+      const uint32_t a0 = umax16x2(umax16x2(bf16x2_abs_bits(v0.x), bf16x2_abs_bits(v0.y)), umax16x2(bf16x2_abs_bits(v0.z), bf16x2_abs_bits(v0.w)));
+      const uint32_t a1 = umax16x2(umax16x2(bf16x2_abs_bits(v1.x), bf16x2_abs_bits(v1.y)), umax16x2(bf16x2_abs_bits(v1.z), bf16x2_abs_bits(v1.w)));
+      const uint32_t a2 = umax16x2(umax16x2(bf16x2_abs_bits(v2.x), bf16x2_abs_bits(v2.y)), umax16x2(bf16x2_abs_bits(v2.z), bf16x2_abs_bits(v2.w)));
+      const uint32_t a3 = umax16x2(umax16x2(bf16x2_abs_bits(v3.x), bf16x2_abs_bits(v3.y)), umax16x2(bf16x2_abs_bits(v3.z), bf16x2_abs_bits(v3.w)));
+      m = umax16x2(m, umax16x2(umax16x2(a0, a1), umax16x2(a2, a3)));
+    }
+    for (; i < total; i += stride) {
+      const uint4 v = p4[i];
+      m = umax16x2(m, umax16x2(umax16x2(bf16x2_abs_bits(v.x), bf16x2_abs_bits(v.y)), umax16x2(bf16x2_abs_bits(v.z), bf16x2_abs_bits(v.w))));
+    }
+  } else
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / chunks_per_row, c = (i - r * chunks_per_row) << 3;
     const uint16_t* p = src + r * ld + c;
@@ -111,79 +128,118 @@ __global__ void __launch_bounds__(256)
 quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, int64_t ld,
                      const int32_t* __restrict__ keep, uint64_t seed, uint32_t stream_id,
                      const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
-                     float* __restrict__ gscale) {
+                     float* __restrict__ gscale, uint32_t div_mul, uint32_t div_shift, int wide_loads) {
+  constexpr int NB = 4;  // inner blocks per thread; all loads are issued before any arithmetic
   const int64_t Kp = (K + 127) & ~(int64_t)127;
+  const int64_t K16 = (K + 15) & ~(int64_t)15;
   const int64_t nb = Kp >> 4;  // inner blocks per operand row (multiple of 8)
-  const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t total = rows * nb;
-  const bool active = gid < total;
-  const int64_t r = active ? gid / nb : 0;
-  const int64_t b = active ? gid - r * nb : 0;
-  const int64_t k0 = b << 4;
+  const int64_t cta_base = (int64_t)blockIdx.x * (256 * NB) + threadIdx.x;
 
-  // ---- load 16 elements (zero beyond K) -----------------------------------------------------------------
-  uint32_t w[8];
+  uint32_t w[NB][8];
+  int64_t row[NB];
+  int32_t blk[NB];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) w[i] = 0;
-  if (active && k0 < K) {
-    const uint16_t* p = src + r * ld;
-    if (!GATHER && k0 + 16 <= K) {
-      const uint4 v0 = *reinterpret_cast<const uint4*>(p + k0);
-      const uint4 v1 = *reinterpret_cast<const uint4*>(p + k0 + 8);
-      w[0] = v0.x; w[1] = v0.y; w[2] = v0.z; w[3] = v0.w;
-      w[4] = v1.x; w[5] = v1.y; w[6] = v1.z; w[7] = v1.w;
-    } else {
-      for (int i = 0; i < 16; ++i) {
-        if (k0 + i < K) {
-          const uint32_t e = GATHER ? p[keep[k0 + i]] : p[k0 + i];
-          w[i >> 1] |= e << (16 * (i & 1));
+  for (int j = 0; j < NB; ++j) {
+    const int64_t gid = cta_base + j * 256;
+    const bool active = gid < total;
+    int64_t r = 0;
+    if (active) {
+      // gid / nb: by multiply-high when the launcher could prepare the constants (gid < 2^31), else plain division
+      if (div_mul) {
+        const uint32_t n = (uint32_t)gid, t = __umulhi(div_mul, n);
+        r = (t + ((n - t) >> 1)) >> div_shift;
+      } else if (div_shift != 0xFFFFFFFFu) {
+        r = (uint32_t)gid >> div_shift;
+      } else {
+        r = gid / nb;
+      }
+    }
+    row[j] = active ? r : -1;
+    blk[j] = active ? (int32_t)(gid - r * nb) : 0;
+    const int64_t k0 = (int64_t)blk[j] << 4;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w[j][i] = 0;
+    if (active && k0 < K) {
+      const uint16_t* p = src + r * ld;
+      if (!GATHER && k0 + 16 <= K) {
+        if (wide_loads) {  // rows start on 32-byte boundaries: one 256-bit load, a warp reads 1 KB contiguously
+          asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                       : "=r"(w[j][0]), "=r"(w[j][1]), "=r"(w[j][2]), "=r"(w[j][3]), "=r"(w[j][4]), "=r"(w[j][5]),
+                         "=r"(w[j][6]), "=r"(w[j][7])
+                       : "l"(p + k0));
+        } else {
+          const uint4 v0 = *reinterpret_cast<const uint4*>(p + k0);
+          const uint4 v1 = *reinterpret_cast<const uint4*>(p + k0 + 8);
+          w[j][0] = v0.x; w[j][1] = v0.y; w[j][2] = v0.z; w[j][3] = v0.w;
+          w[j][4] = v1.x; w[j][5] = v1.y; w[j][6] = v1.z; w[j][7] = v1.w;
+        }
+      } else {
+        for (int i = 0; i < 16; ++i) {
+          if (k0 + i < K) {
+            const uint32_t e = GATHER ? p[keep[k0 + i]] : p[k0 + i];
+            w[j][i >> 1] |= e << (16 * (i & 1));
+          }
         }
       }
     }
   }
-  uint32_t m2 = 0;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) m2 = umax16x2(m2, bf16x2_abs_bits(w[i]));
-  const uint32_t amax_b_bits = hmax_of_pair(m2);
 
-  // ---- global scale ---------------------------------------------------------------------------------------
-  float Sg;
-  if (GS == kGsBlock128) {
-    uint32_t g = amax_b_bits;
-    g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
-    g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
-    g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 4));
-    Sg = global_scale_from_amax(bf16_bits_to_float(g));
-    if (active && (b & 7) == 0) gscale[r * (Kp >> 7) + (b >> 3)] = Sg;
-  } else if (GS == kGsRow) {
-    Sg = global_scale_from_amax(__uint_as_float(gs_cells[r]));
-    if (active && b == 0) gscale[r] = Sg;
-  } else {
-    Sg = global_scale_from_amax(__uint_as_float(gs_cells[0]));
-    if (gid == 0) gscale[0] = Sg;
+  float Sg_t = 1.0f;
+  if (GS == kGsTensor) {
+    Sg_t = global_scale_from_amax(__uint_as_float(gs_cells[0]));
+    if (blockIdx.x == 0 && threadIdx.x == 0) gscale[0] = Sg_t;
   }
 
-  // ---- block scale, rounding, packing -------------------------------------------------------------------
-  float rcp;
-  const uint32_t sb = block_scale(bf16_bits_to_float(amax_b_bits), Sg, rcp);
-  float x[16];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    x[2 * i] = bf16_lo(w[i]);
-    x[2 * i + 1] = bf16_hi(w[i]);
-  }
-  const int64_t K16 = (K + 15) & ~(int64_t)15;
-  const uint2 packed = quantize_block16<SR>(x, rcp, seed, stream_id, (uint64_t)((r * K16 + k0) >> 3));
+  for (int j = 0; j < NB; ++j) {
+    const bool active = row[j] >= 0;
+    const int64_t r = active ? row[j] : 0;
+    const int64_t b = blk[j];
+    const int64_t k0 = b << 4;
+    uint32_t m2 = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m2 = umax16x2(m2, bf16x2_abs_bits(w[j][i]));
+    const uint32_t amax_b_bits = hmax_of_pair(m2);
 
-  // four neighbouring threads own the four scale bytes of one 32-bit word in either layout
-  uint32_t sf4 = sb << (8 * (b & 3));
-  sf4 |= __shfl_xor_sync(0xFFFFFFFFu, sf4, 1);
-  sf4 |= __shfl_xor_sync(0xFFFFFFFFu, sf4, 2);
-  if (!active) return;
-  *reinterpret_cast<uint2*>(codes + r * (Kp >> 1) + (k0 >> 1)) = packed;
-  if ((b & 3) == 0) {
-    const size_t off = TILED ? sf_tiled_offset(r, b, (nb + 15) & ~(int64_t)15) : (size_t)(r * nb + b);
-    *reinterpret_cast<uint32_t*>(sf + off) = sf4;
+    // ---- global scale -------------------------------------------------------------------------------------
+    float Sg;
+    if (GS == kGsBlock128) {
+      uint32_t g = amax_b_bits;
+      g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
+      g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
+      g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 4));
+      Sg = global_scale_from_amax(bf16_bits_to_float(g));
+      if (active && (b & 7) == 0) gscale[r * (Kp >> 7) + (b >> 3)] = Sg;
+    } else if (GS == kGsRow) {
+      Sg = global_scale_from_amax(__uint_as_float(gs_cells[r]));
+      if (active && b == 0) gscale[r] = Sg;
+    } else {
+      Sg = Sg_t;
+    }
+
+    // ---- block scale, rounding, packing -------------------------------------------------------------------
+    float rcp;
+    const uint32_t sb = block_scale(bf16_bits_to_float(amax_b_bits), Sg, rcp);
+    float x[16];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      x[2 * i] = bf16_lo(w[j][i]);
+      x[2 * i + 1] = bf16_hi(w[j][i]);
+    }
+    const uint2 packed = quantize_block16<SR>(x, rcp, seed, stream_id, (uint64_t)((r * K16 + k0) >> 3));
+
+    // four neighbouring threads own the four scale bytes of one 32-bit word in either layout
+    uint32_t sf4 = sb << (8 * (b & 3));
+    sf4 |= __shfl_xor_sync(0xFFFFFFFFu, sf4, 1);
+    sf4 |= __shfl_xor_sync(0xFFFFFFFFu, sf4, 2);
+    if (active) {
+      *reinterpret_cast<uint2*>(codes + r * (Kp >> 1) + (k0 >> 1)) = packed;
+      if ((b & 3) == 0) {
+        const size_t off = TILED ? sf_tiled_offset(r, b, (nb + 15) & ~(int64_t)15) : (size_t)(r * nb + b);
+        *reinterpret_cast<uint32_t*>(sf + off) = sf4;
+      }
+    }
   }
 }
 
@@ -414,13 +470,28 @@ template <int GS, bool SR, bool TILED>
 static cudaError_t launch_rows_g(const QuantRowsArgs& a, cudaStream_t st) {
   const int64_t Kp = (a.K + 127) & ~(int64_t)127;
   const int64_t total = a.rows * (Kp >> 4);
-  const unsigned grid = blocks_for(total, 256);
+  const unsigned grid = blocks_for(total, 256 * 4);
+  // constants for gid / nb without a hardware division (n / d = (t + ((n - t) >> 1)) >> (s - 1), t = mulhi(m, n))
+  uint32_t div_mul = 0, div_shift = 0xFFFFFFFFu;
+  const uint64_t d = (uint64_t)(Kp >> 4);
+  if (total + 1024 < (int64_t)1 << 31) {
+    if ((d & (d - 1)) == 0) {
+      div_shift = 0;
+      while (((uint64_t)1 << div_shift) < d) ++div_shift;
+    } else {
+      uint32_t sft = 0;
+      while (((uint64_t)1 << sft) < d) ++sft;
+      div_mul = (uint32_t)((((uint64_t)1 << 32) * (((uint64_t)1 << sft) - d)) / d + 1);
+      div_shift = sft - 1;
+    }
+  }
+  const int wide_loads = ((reinterpret_cast<uintptr_t>(a.src) & 31u) == 0 && (a.ld & 15) == 0) ? 1 : 0;
   if (a.keep)
     quantize_rows_kernel<GS, SR, TILED, true><<<grid, 256, 0, st>>>(a.src, a.rows, a.K, a.ld, a.keep, a.seed, a.stream_id,
-                                                                   a.gs_cells, a.codes, a.sf, a.gscale);
+                                                                   a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads);
   else
-    quantize_rows_kernel<GS, SR, TILED, false><<<grid, 256, 0, st>>>(a.src, a.rows, a.K, a.ld, nullptr, a.seed,
-                                                                    a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale);
+    quantize_rows_kernel<GS, SR, TILED, false><<<grid, 256, 0, st>>>(a.src, a.rows, a.K, a.ld, nullptr, a.seed, a.stream_id,
+                                                                    a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads);
   ++g_launch_count;
   return cudaGetLastError();
 }
