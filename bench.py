@@ -165,6 +165,7 @@ def run_ours(args):
     import torch.distributed as dist
 
     from paper_2510_27527_b200 import binding as b
+    from paper_2510_27527_b200 import multi
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -237,10 +238,7 @@ def run_ours(args):
             ev[s][1].record()
         barrier()
         ms = [a.elapsed_time(bb) for a, bb in ev]
-        tot = torch.tensor([sum(ms)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(tot, op=dist.ReduceOp.MAX)
-        return float(tot.item()) / steps, ms
+        return multi.max_over_ranks(sum(ms), dev) / steps, ms  # the job's time is the slowest rank's
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -253,6 +251,17 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     fl = flops_of(tokens, linears, layers)
     value = world * fl / (ms_step * 1e-3) / 1e12
+
+    if args.no_breakdown:
+        if rank != 0:
+            if world > 1:
+                dist.destroy_process_group()
+            return
+        print(json.dumps({"metric": "nvfp4_linear_fwd_bwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+                          "steps": args.steps, "ms_per_step": ms_step, "gpu_launches": int(launches), "note": "--no-breakdown run"}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # ---- end to end: host buffers in, results out, copies inside the timed region -------------------------------
     pinned_in, h2d, d2h = [], 0, 0
@@ -457,6 +466,7 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=1024, help="token slab of one oracle step (reference arm)")
     ap.add_argument("--cpu-tokens", type=int, default=4096, help="token slab of the cpu_baseline leg")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-breakdown", action="store_true", help="only warm-up + timed steps (used for ncu launch lists)")
     ap.add_argument("--sweep", action="store_true", help="roofline sweep of the large GEMM shapes instead of the step benchmark")
     ap.add_argument("--shapes", default="", help="with --sweep: comma list of MxNxK")
     args = ap.parse_args()

@@ -1,0 +1,107 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times (tiled scales, BF16 / FP32
+outputs, same entry points): quantizers bit-exact on the whole tensor, GEMM outputs on sampled entries and tiles
+that the oracle computes one by one (FP64 dot products of the dequantized operands)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import nvfp4_oracle as orc
+from paper_2510_27527_b200 import synth
+from tests.gpu_util import assert_operand_equal, to_dev_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+def B():
+    from paper_2510_27527_b200 import binding
+
+    return binding
+
+
+def sample_positions(M, N, rng, n_scatter=4096, n_tiles=4, tile=32):
+    ms = [rng.integers(0, M, n_scatter)]
+    ns = [rng.integers(0, N, n_scatter)]
+    for _ in range(n_tiles):
+        m0, n0 = rng.integers(0, M - tile + 1), rng.integers(0, N - tile + 1)
+        mm, nn = np.meshgrid(np.arange(m0, m0 + tile), np.arange(n0, n0 + tile), indexing="ij")
+        ms.append(mm.ravel())
+        ns.append(nn.ravel())
+    # always include the corners and the last row / column
+    ms.append(np.array([0, 0, M - 1, M - 1]))
+    ns.append(np.array([0, N - 1, 0, N - 1]))
+    return np.concatenate(ms).astype(np.int64), np.concatenate(ns).astype(np.int64)
+
+
+def check_sampled(got: torch.Tensor, A64, B64, rng, bf16_out, name):
+    M, N = got.shape
+    ms, ns = sample_positions(M, N, rng)
+    want, absdot = orc.gemm_tn_samples(A64, B64, ms, ns)
+    g = got[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].float().cpu().numpy().astype(np.float64)
+    tol = 1e-3 * absdot  # |err| <= 1e-3 * sum_k |a_k b_k| elementwise
+    if bf16_out:
+        tol = tol + np.abs(want) * 2.0 ** -8  # one BF16 rounding of the result
+    bad = np.abs(g - want) > tol + 1e-300
+    assert not bad.any(), (name, int(bad.sum()), float(np.abs(g - want).max()))
+    rel = np.linalg.norm(g - want) / np.linalg.norm(want)
+    assert rel <= (4e-3 if bf16_out else 1e-3), (name, rel)
+
+
+@pytest.mark.parametrize("gs_mode", [0, 2])
+def test_attention_projection_qkv_full_size(gs_mode):
+    """BASELINE config 2, the QKV linear: tokens 8192, 1024 -> 3072; forward, dX, dW through the layer entry points."""
+    b = B()
+    c = synth.CONFIGS[2]
+    T, D, C = c["tokens"], 1024, 3072
+    X, W, dY, _ = synth.layer_inputs(2, T, D, C, n_outlier=c["n_outlier"], factor=c["factor"], grad_scale=c["grad_scale"],
+                                     weight_id=10)
+    cfg = b.LayerConfig(gs_mode=gs_mode, seed=0, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32)
+    Xd, Wd, dYd = to_dev_bf16(X), to_dev_bf16(W), to_dev_bf16(dY)
+    Y, saved = b.nvfp4_linear_fwd(Xd, Wd, cfg)
+    dX = b.nvfp4_linear_bwd_dx(dYd, saved, cfg)
+    dW = b.nvfp4_linear_bwd_dw(dYd, saved, cfg)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(0)
+    # oracle operands (whole tensors), compared bit for bit where the device exposes them
+    q1 = orc.quantize(X, orc.AXIS_ROW, orc.RTN, gs_mode, 0, 1)
+    q2 = orc.quantize(W, orc.AXIS_ROW, orc.RTN, gs_mode, 0, 2)
+    assert_operand_equal(saved.qx, q1, "Q1(X) full size")
+    assert_operand_equal(saved.qw, q2, "Q2(W) full size")
+    check_sampled(Y, orc.dequantize(q1), orc.dequantize(q2), rng, True, "Y")
+    q3 = orc.quantize(dY, orc.AXIS_ROW, orc.SR, gs_mode, 0, 3)
+    q4 = orc.quantize(orc.rematerialize_f32(q2), orc.AXIS_COL, orc.SR, gs_mode, 0, 4)
+    check_sampled(dX, orc.dequantize(q3), orc.dequantize(q4), rng, True, "dX")
+    q5 = orc.quantize(dY, orc.AXIS_COL, orc.SR, gs_mode, 0, 5)
+    q6 = orc.quantize(orc.rematerialize_f32(q1), orc.AXIS_COL, orc.SR, gs_mode, 0, 6)
+    check_sampled(dW, orc.dequantize(q5), orc.dequantize(q6), rng, False, "dW")
+    # the backward operands themselves, bit for bit, through the operand-level entry points
+    g3 = b.nvfp4_quantize(dYd, b.AXIS_ROW, b.ROUND_SR, 0, 3, gs_mode)
+    assert_operand_equal(g3, q3, "Q3(dY) full size")
+    g5 = b.nvfp4_quantize(dYd, b.AXIS_COL, b.ROUND_SR, 0, 5, gs_mode)
+    assert_operand_equal(g5, q5, "Q5(dY^T) full size")
+    g4 = b.nvfp4_requantize_t(saved.qw, b.ROUND_SR, 0, 4)
+    assert_operand_equal(g4, q4, "Q4(W-hat) full size")
+    g6 = b.nvfp4_requantize_t(saved.qx, b.ROUND_SR, 0, 6)
+    assert_operand_equal(g6, q6, "Q6(X-hat) full size")
+
+
+def test_largest_sweep_shape_quantize_and_gemm():
+    """BASELINE config 5, the largest shape: M = 16384, N = K = 8192 (BF16 ~N(0,1), 0.5 % channels x100)."""
+    b = B()
+    M, N, K = 16384, 8192, 8192
+    A, _ = synth.activations(M, K, synth.seed_of(5, 1), n_outlier=41, factor=100.0)
+    Bm, _ = synth.activations(N, K, synth.seed_of(5, 2), n_outlier=41, factor=100.0)
+    Ad, Bd = to_dev_bf16(A), to_dev_bf16(Bm)
+    qa = b.nvfp4_quantize(Ad, b.AXIS_ROW, b.ROUND_RTN, 0, 1, b.GS_TENSOR)
+    qb = b.nvfp4_quantize(Bd, b.AXIS_ROW, b.ROUND_SR, 7, 2, b.GS_TENSOR)
+    oa = orc.quantize(A, orc.AXIS_ROW, orc.RTN, orc.GS_TENSOR, 0, 1)
+    ob = orc.quantize(Bm, orc.AXIS_ROW, orc.SR, orc.GS_TENSOR, 7, 2)
+    assert_operand_equal(qa, oa, "A 16384x8192 RTN")
+    assert_operand_equal(qb, ob, "B 8192x8192 SR")
+    C = b.nvfp4_gemm(qa, qb, b.DT_BF16)
+    torch.cuda.synchronize()
+    check_sampled(C, orc.dequantize(oa), orc.dequantize(ob), np.random.default_rng(1), True, "C 16384x8192x8192")
+    del C
+    # the transposed (column-axis) quantizer at the same size, bit for bit
+    qt = b.nvfp4_quantize(Bd, b.AXIS_COL, b.ROUND_SR, 9, 5, b.GS_BLOCK128)
+    ot = orc.quantize(Bm, orc.AXIS_COL, orc.SR, orc.GS_BLOCK128, 9, 5)
+    assert_operand_equal(qt, ot, "B^T 8192x8192 SR block128")
