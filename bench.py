@@ -38,6 +38,14 @@ LAYERS = {"attn": 1, "mlp": 1, "model370m": 24}
 GS = {"tensor": 0, "row": 1, "block128": 2}
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
+# (default workload, QKV linear, tokens 8192), keyed by the kernel labels of the per-kernel breakdown below.
+PROFILED_TRAFFIC = {
+    "quantize_cols_dY_SR(Q5)": (51153152, "profiles/quantize_transpose_bf16_sr_attn_dY_8192x3072.txt"),
+    "quantize_rows_dY_SR(Q3)": (50739712, "profiles/quantize_rows_sr_attn_dY_8192x3072.txt"),
+}
+
+
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -350,9 +358,8 @@ def run_ours(args):
         roof = dict(bound="hbm", achieved=dp["GBps"], peak=pk["hbm"], unit="GB/s", frac=dp["GBps"] / pk["hbm"])
     roof.update(kernel=f"{dom} on {L.name} {D}->{C}, tokens {T}", peak_source=f"of {pk['source']}", traffic=None,
                 algorithmic_bytes_per_launch=dp["bytes"], seconds_per_launch=dp["seconds"])
-    tj = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tj):
-        roof["traffic"] = json.load(open(tj)).get(dom)
+    if args.workload == "attn" and args.gs == "tensor" and dom in PROFILED_TRAFFIC:
+        roof["traffic"], roof["traffic_source"] = PROFILED_TRAFFIC[dom]
 
     # ---- the oracle beside it ------------------------------------------------------------------------------------
     cpu = None
