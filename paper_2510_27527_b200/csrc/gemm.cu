@@ -36,7 +36,11 @@ struct Cfg {
   static constexpr uint32_t SFB_BYTES = (BN / 128) * 2048;
   static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;  // multiple of 1024
   static constexpr int STAGES = (BN == 128) ? 5 : 4;
-  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
+  // epilogue staging for bulk tensor stores: per epilogue warp two 32-row x 128-byte buffers (128 x 128 tiles only;
+  // the 128 x 256 variant has no shared memory left and stores straight from registers)
+  static constexpr bool TMA_STORE = (BN == 128);
+  static constexpr uint32_t STAGING_BYTES = TMA_STORE ? 4 * 2 * 4096 : 0;
+  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
   // tensor memory columns: two accumulators, then four scale buffers (A: 16 columns, B: 16 * BN / 128)
   static constexpr uint32_t ACC_COLS = BN;
   static constexpr uint32_t ACC_BUFS = (BN == 256) ? 1 : 2;  // 256-wide accumulators leave no room for a second one
@@ -62,6 +66,7 @@ struct Params {
   int32_t sf_tiles_b;
   int32_t m_tiles, n_tiles;
   int32_t c_is_f32, accumulate;
+  int32_t use_tma_store;  // C is described by a tensor map: stage the epilogue in shared memory and bulk-store it
   int32_t* dev_status;
 };
 
@@ -183,6 +188,56 @@ __device__ __forceinline__ uint32_t instr_desc() {
   return (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (0u << 23) | ((uint32_t)(BM >> 4) << 24);
 }
 
+// Bulk tensor store of a staged [32 rows x 128 bytes] block (128-byte swizzle) to C; rows / columns outside C are clipped.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int32_t c0, int32_t c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tm), "r"(src), "r"(c0),
+               "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Adds the optional FP32 addend and, when accumulating, the old C to W consecutive values of output row m from column n0
+// (a full chunk inside C).
+template <int W>
+__device__ __forceinline__ void add_existing(const Params& p, int64_t m, int64_t n0, float (&o)[W]) {
+  if (p.addend) {
+    const float* ad = p.addend + m * p.ld_add + n0;
+#pragma unroll
+    for (int j = 0; j < W; j += 4) {
+      const float4 q = *reinterpret_cast<const float4*>(ad + j);
+      o[j] += q.x; o[j + 1] += q.y; o[j + 2] += q.z; o[j + 3] += q.w;
+    }
+  }
+  if (p.accumulate) {
+    if (p.c_is_f32) {
+      const float* cp = reinterpret_cast<const float*>(p.C) + m * p.ldc + n0;
+#pragma unroll
+      for (int j = 0; j < W; j += 4) {
+        const float4 q = *reinterpret_cast<const float4*>(cp + j);
+        o[j] += q.x; o[j + 1] += q.y; o[j + 2] += q.z; o[j + 3] += q.w;
+      }
+    } else {
+      const uint16_t* cp = reinterpret_cast<const uint16_t*>(p.C) + m * p.ldc + n0;
+#pragma unroll
+      for (int j = 0; j < W; j += 8) {
+        const uint4 old = *reinterpret_cast<const uint4*>(cp + j);
+        const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          o[j + 2 * q] += bf16_lo(ow[q]);
+          o[j + 2 * q + 1] += bf16_hi(ow[q]);
+        }
+      }
+    }
+  }
+}
+
 // One output row, 32 consecutive columns starting at n0 (m < M and n0 < N are the caller's business): add the optional
 // FP32 addend and the old C when accumulating, convert, store.
 __device__ __forceinline__ void store_row_chunk(const Params& p, int64_t m, int64_t n0, float (&o)[32]) {
@@ -246,11 +301,13 @@ __device__ __forceinline__ void store_row_chunk(const Params& p, int64_t m, int6
 
 template <int GS, int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
+gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmC, const Params p) {
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = smem_base + C::STAGES * C::STAGE_BYTES;
+  const uint32_t staging_base = smem_base + C::STAGES * C::STAGE_BYTES;
+  const uint32_t bar_base = staging_base + C::STAGING_BYTES;
   // barriers: full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], drain
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (C::STAGES + s); };
@@ -371,7 +428,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   } else {
     // ===================================== epilogue ========================================================
     const int quad = warp & 3;  // tensor-memory lane quadrant this warp may read
-    uint32_t tile_it = 0;
+    uint32_t tile_it = 0, chunk_it = 0;
     bool ok = true;
     float alpha = 1.0f;
     if (GS == kGsTensor) alpha = __fmul_rn(p.a_gscale[0], p.b_gscale[0]);
@@ -383,6 +440,116 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int64_t m = (int64_t)mt * BM + quad * 32 + lane;
       float sa = 1.0f;
       if (GS == kGsRow && m < p.M) sa = p.a_gscale[m];
+      if (C::TMA_STORE && p.use_tma_store) {
+        // Stage 128-byte row pieces (32 FP32 or 64 BF16 columns) in shared memory with the 128-byte swizzle and let the
+        // bulk-tensor engine write them: full lines, clipped at the edges of C, asynchronous.
+        const uint32_t my_stage = staging_base + (uint32_t)(warp - 2) * 8192u;
+        const int64_t m0 = (int64_t)mt * BM + quad * 32;
+        if (p.c_is_f32) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t v[32];
+            tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + c0, v);
+            tc_wait_ld();
+            const int64_t n0 = (int64_t)nt * BN + c0;
+            if (n0 >= p.N) break;
+            float o[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              float sc = alpha;
+              if (GS == kGsRow) sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
+              o[j] = __uint_as_float(v[j]) * sc;
+            }
+            if ((p.addend || p.accumulate) && m < p.M) {
+              if (n0 + 32 <= p.N) {
+                add_existing<32>(p, m, n0, o);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  if (n0 + j < p.N) {
+                    if (p.addend) o[j] += p.addend[m * p.ld_add + n0 + j];
+                    if (p.accumulate) o[j] += reinterpret_cast<const float*>(p.C)[m * p.ldc + n0 + j];
+                  }
+                }
+              }
+            }
+            const uint32_t buf = my_stage + (uint32_t)(chunk_it & 1) * 4096u;
+            if (lane == 0) bulk_wait_read<1>();  // the store that used this buffer two chunks ago has read it
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint32_t dst = buf + (uint32_t)lane * 128u + (uint32_t)((j ^ (lane & 7)) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(__float_as_uint(o[4 * j])),
+                           "r"(__float_as_uint(o[4 * j + 1])), "r"(__float_as_uint(o[4 * j + 2])),
+                           "r"(__float_as_uint(o[4 * j + 3]))
+                           : "memory");
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&tmC, buf, (int32_t)n0, (int32_t)m0);
+              bulk_commit();
+            }
+            ++chunk_it;
+          }
+        } else {
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN; c0 += 64) {
+            uint32_t v[32], v2[32];
+            tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + c0, v);
+            tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + c0 + 32, v2);
+            tc_wait_ld();
+            const int64_t n0 = (int64_t)nt * BN + c0;
+            if (n0 >= p.N) break;
+            float o[64];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              float sc = alpha, sc2 = alpha;
+              if (GS == kGsRow) {
+                sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
+                sc2 = __fmul_rn(sa, (n0 + 32 + j < p.N) ? __ldg(p.b_gscale + n0 + 32 + j) : 0.0f);
+              }
+              o[j] = __uint_as_float(v[j]) * sc;
+              o[32 + j] = __uint_as_float(v2[j]) * sc2;
+            }
+            if ((p.addend || p.accumulate) && m < p.M) {
+              if (n0 + 64 <= p.N) {
+                add_existing<64>(p, m, n0, o);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 64; ++j) {
+                  if (n0 + j < p.N) {
+                    if (p.addend) o[j] += p.addend[m * p.ld_add + n0 + j];
+                    if (p.accumulate) o[j] += __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.C)[m * p.ldc + n0 + j]);
+                  }
+                }
+              }
+            }
+            const uint32_t buf = my_stage + (uint32_t)(chunk_it & 1) * 4096u;
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              uint32_t q[4];
+#pragma unroll
+              for (int h = 0; h < 4; ++h) {
+                const __nv_bfloat162 hh = __floats2bfloat162_rn(o[8 * j + 2 * h], o[8 * j + 2 * h + 1]);
+                q[h] = *reinterpret_cast<const uint32_t*>(&hh);
+              }
+              const uint32_t dst = buf + (uint32_t)lane * 128u + (uint32_t)((j ^ (lane & 7)) << 4);
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(q[0]), "r"(q[1]), "r"(q[2]), "r"(q[3])
+                           : "memory");
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&tmC, buf, (int32_t)n0, (int32_t)m0);
+              bulk_commit();
+            }
+            ++chunk_it;
+          }
+        }
+      } else {
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
         uint32_t v[32];
@@ -400,10 +567,12 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           store_row_chunk(p, m, n0, o);
         }
       }
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty_bar(ab));
     }
+    if (C::TMA_STORE && lane == 0) bulk_wait_all();  // this lane's bulk stores are complete before the CTA may exit
   }
 
   // ===================================== teardown ============================================================
@@ -653,6 +822,20 @@ bool make_codes_map(CUtensorMap* tm, const uint8_t* codes, int64_t R, int64_t Kp
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// C [M, N] (BF16 or FP32, leading dimension ldc) as a 2-D tensor; box = 128 bytes of a row x 32 rows, 128-byte swizzle.
+bool make_c_map(CUtensorMap* tm, void* Cp, int64_t M, int64_t N, int64_t ldc, bool is_f32) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t esz = is_f32 ? 4 : 2;
+  const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)ldc * esz};
+  const cuuint32_t box[2] = {(cuuint32_t)(128 / esz), 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, is_f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Cp, dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int sm_count() {
   static int n = 0;
   if (!n) {
@@ -667,10 +850,13 @@ template <int GS, int BN>
 cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
   using C = Cfg<BN>;
   const int64_t Kp = (a.K + 127) & ~(int64_t)127;
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmB, tmC;
   if (!make_codes_map(&tmA, a.a_codes, a.M, Kp, BM) || !make_codes_map(&tmB, a.b_codes, a.N, Kp, BN))
     return cudaErrorInvalidValue;
+  const bool tma_store = C::TMA_STORE && make_c_map(&tmC, a.C, a.M, a.N, a.ldc, a.c_is_f32 != 0);
+  if (!tma_store) tmC = tmA;  // unused by the kernel then
   Params p{};
+  p.use_tma_store = tma_store ? 1 : 0;
   p.a_sf = a.a_sf;
   p.b_sf = a.b_sf;
   p.a_gscale = a.a_gscale;
@@ -700,7 +886,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
   }
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
-  gemm_nvfp4_kernel<GS, BN><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(tmA, tmB, p);
+  gemm_nvfp4_kernel<GS, BN><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(tmA, tmB, tmC, p);
   ++g_launch_count;
   return cudaGetLastError();
 }
