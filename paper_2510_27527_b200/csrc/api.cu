@@ -89,7 +89,7 @@ bool carve_operand(Carver& c, nvfp4_operand* o, int64_t R, int64_t K, int32_t gs
 
 nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, int32_t rounding,
                               uint64_t seed, uint32_t stream_id, const int32_t* keep, int64_t n_keep,
-                              const nvfp4_operand* out, uint32_t* cells, cudaStream_t st) {
+                              const nvfp4_operand* out, uint32_t* cells, cudaStream_t st, int cells_zeroed = 0) {
   if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   QuantRowsArgs a{};
   a.src = src;
@@ -104,6 +104,7 @@ nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, i
   a.sr = rounding == NVFP4_ROUND_SR;
   a.sf_tiled = out->sf_layout == NVFP4_SF_TILED128x4;
   a.compute_amax = 1;
+  a.cells_zeroed = cells_zeroed;
   a.gs_cells = cells;
   a.codes = out->codes;
   a.sf = out->sf;
@@ -113,7 +114,7 @@ nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, i
 
 nvfp4_status do_quantize_transpose(const TransposeSrc& src, int from_codes, int64_t rowsK, int64_t D, int32_t rounding,
                                    uint64_t seed, uint32_t stream_id, const nvfp4_operand* out, uint32_t* cells,
-                                   cudaStream_t st) {
+                                   cudaStream_t st, int cells_zeroed = 0) {
   if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   QuantTransposeArgs a{};
   a.from_codes = from_codes;
@@ -126,6 +127,7 @@ nvfp4_status do_quantize_transpose(const TransposeSrc& src, int from_codes, int6
   a.sr = rounding == NVFP4_ROUND_SR;
   a.sf_tiled = out->sf_layout == NVFP4_SF_TILED128x4;
   a.compute_amax = 1;
+  a.cells_zeroed = cells_zeroed;
   a.gs_cells = cells;
   a.codes = out->codes;
   a.sf = out->sf;
@@ -155,6 +157,13 @@ nvfp4_status do_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, in
   g.ld_add = ld_add;
   g.dev_status = dev_status;
   return launch_gemm(g, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+// Clears the amax cells of a layer call (two arrays carved back to back) with one memset, so that the kernels that follow
+// are launched kernel-after-kernel and can overlap their prologues with their predecessors' tails.
+bool zero_cells(uint32_t* first, uint32_t* second, size_t second_bytes, cudaStream_t st) {
+  const size_t span = (reinterpret_cast<uint8_t*>(second) - reinterpret_cast<uint8_t*>(first)) + second_bytes;
+  return cudaMemsetAsync(first, 0, span, st) == cudaSuccess;
 }
 
 nvfp4_status check_cfg(const nvfp4_layer_cfg* cfg, int64_t D) {
@@ -347,9 +356,10 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
   const uint16_t* Xp = static_cast<const uint16_t*>(X);
   const uint16_t* Wp = static_cast<const uint16_t*>(W);
   const int32_t* keep = n_out > 0 ? cfg->keep_cols : nullptr;
-  if ((s = do_quantize_rows(Xp, N_tok, D, ldx, cfg->rounding[0], cfg->seed, 1, keep, Dk, &saved->qx, cells_x, st)) != NVFP4_OK)
+  if (!zero_cells(cells_x, cells_w, cells_bytes(C, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
+  if ((s = do_quantize_rows(Xp, N_tok, D, ldx, cfg->rounding[0], cfg->seed, 1, keep, Dk, &saved->qx, cells_x, st, 1)) != NVFP4_OK)
     return s;
-  if ((s = do_quantize_rows(Wp, C, D, ldw, cfg->rounding[1], cfg->seed, 2, keep, Dk, &saved->qw, cells_w, st)) != NVFP4_OK)
+  if ((s = do_quantize_rows(Wp, C, D, ldw, cfg->rounding[1], cfg->seed, 2, keep, Dk, &saved->qw, cells_w, st, 1)) != NVFP4_OK)
     return s;
   if (n_out > 0) {
     HpFwdArgs h{};
@@ -384,8 +394,9 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
   nvfp4_operand q3, q4;
   if (!carve_operand(cv, &q3, N_tok, C, cfg->gs_mode) || !carve_operand(cv, &q4, D, C, cfg->gs_mode) || !cells3 || !cells4)
     return NVFP4_ERR_WORKSPACE;
+  if (!zero_cells(cells3, cells4, cells_bytes(D, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
   if ((s = do_quantize_rows(static_cast<const uint16_t*>(dY), N_tok, C, lddy, cfg->rounding[2], cfg->seed, 3, nullptr, 0,
-                            &q3, cells3, st)) != NVFP4_OK)
+                            &q3, cells3, st, 1)) != NVFP4_OK)
     return s;
   TransposeSrc ts{};
   ts.in_codes = saved->qw.codes;
@@ -399,7 +410,7 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
     ts.hp = static_cast<const uint16_t*>(saved->W);
     ts.hp_ld = saved->ldw;
   }
-  if ((s = do_quantize_transpose(ts, 1, C, D, cfg->rounding[3], cfg->seed, 4, &q4, cells4, st)) != NVFP4_OK) return s;
+  if ((s = do_quantize_transpose(ts, 1, C, D, cfg->rounding[3], cfg->seed, 4, &q4, cells4, st, 1)) != NVFP4_OK) return s;
   return do_gemm(&q3, &q4, dX, cfg->dx_dtype, lddx, 0, nullptr, 0, cfg->dev_status, st);
 }
 
@@ -434,7 +445,8 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
   TransposeSrc t5{};
   t5.bf16 = static_cast<const uint16_t*>(dY);
   t5.ld = lddy;
-  if ((s = do_quantize_transpose(t5, 0, N_tok, C, cfg->rounding[4], cfg->seed, 5, &q5, cells5, st)) != NVFP4_OK) return s;
+  if (!zero_cells(cells5, cells6, cells_bytes(Dk, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
+  if ((s = do_quantize_transpose(t5, 0, N_tok, C, cfg->rounding[4], cfg->seed, 5, &q5, cells5, st, 1)) != NVFP4_OK) return s;
   TransposeSrc t6{};
   t6.in_codes = saved->qx.codes;
   t6.in_sf = saved->qx.sf;
@@ -442,7 +454,7 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
   t6.in_K = saved->qx.K;
   t6.in_gs_mode = saved->qx.gs_mode;
   t6.in_sf_tiled = saved->qx.sf_layout == NVFP4_SF_TILED128x4;
-  if ((s = do_quantize_transpose(t6, 1, N_tok, Dk, cfg->rounding[5], cfg->seed, 6, &q6, cells6, st)) != NVFP4_OK) return s;
+  if ((s = do_quantize_transpose(t6, 1, N_tok, Dk, cfg->rounding[5], cfg->seed, 6, &q6, cells6, st, 1)) != NVFP4_OK) return s;
   if (n_out == 0) return do_gemm(&q5, &q6, dW, cfg->dw_dtype, lddw, 0, nullptr, 0, cfg->dev_status, st);
 
   if ((s = do_gemm(&q5, &q6, compact, NVFP4_DT_F32, ld_compact, 0, nullptr, 0, cfg->dev_status, st)) != NVFP4_OK) return s;

@@ -343,6 +343,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
+  pdl_prologue();  // everything above touched only shared and tensor memory
 
   const int64_t num_tiles = (int64_t)p.m_tiles * p.n_tiles;
 
@@ -640,6 +641,7 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
+  pdl_prologue();  // everything above touched only shared and tensor memory
   const int64_t num_tiles = (int64_t)p.m_tiles * p.n_tiles;
   const int32_t chunks = p.k_chunks;  // 128-wide k chunks per tile
 
@@ -886,8 +888,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
   }
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
-  gemm_nvfp4_kernel<GS, BN><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(tmA, tmB, tmC, p);
-  ++g_launch_count;
+  launch_kernel(gemm_nvfp4_kernel<GS, BN>, dim3(grid), dim3(NUM_THREADS), C::SMEM_BYTES, st, tmA, tmB, tmC, p);
   return cudaGetLastError();
 }
 
@@ -926,8 +927,7 @@ cudaError_t launch_block128(const GemmArgs& a, cudaStream_t st) {
   }
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
-  gemm_nvfp4_block128_kernel<<<grid, NUM_THREADS, B128_SMEM_BYTES, st>>>(tmA, tmB, p);
-  ++g_launch_count;
+  launch_kernel(gemm_nvfp4_block128_kernel, dim3(grid), dim3(NUM_THREADS), B128_SMEM_BYTES, st, tmA, tmB, p);
   return cudaGetLastError();
 }
 

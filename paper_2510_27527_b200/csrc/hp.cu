@@ -9,6 +9,7 @@ namespace nvfp4 {
 
 // Y[m, n] = sum_j X[m, outl[j]] * W[n, outl[j]].  CTA tile 64 x 64, outlier channels in chunks of 32.
 __global__ void __launch_bounds__(256) hp_fwd_kernel(HpFwdArgs a) {
+  pdl_prologue();
   __shared__ float xs[32][65];
   __shared__ float ws[32][65];
   const int64_t m0 = (int64_t)blockIdx.y * 64, n0 = (int64_t)blockIdx.x * 64;
@@ -56,6 +57,7 @@ __global__ void __launch_bounds__(256) hp_fwd_kernel(HpFwdArgs a) {
 // dW[c, outl[j]] = sum_t dY[t, c] * X[t, outl[j]].  One CTA per (64 output channels c, 8 outlier channels j);
 // four token groups per CTA reduced through shared memory in a fixed order.
 __global__ void __launch_bounds__(256) hp_dw_kernel(HpDwArgs a) {
+  pdl_prologue();
   __shared__ float red[4][8][64];
   const int cl = threadIdx.x & 63, tg = threadIdx.x >> 6;
   const int64_t c = (int64_t)blockIdx.x * 64 + cl;
@@ -93,6 +95,7 @@ __global__ void __launch_bounds__(256) hp_dw_kernel(HpDwArgs a) {
 __global__ void __launch_bounds__(256) scatter_cols_kernel(const void* src, int64_t ld_src, int src_is_f32, void* dst,
                                                           int64_t ld_dst, int dst_is_f32, int64_t rows, int64_t n_keep,
                                                           const int32_t* __restrict__ keep) {
+  pdl_prologue();
   const int64_t total = rows * n_keep;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = i / n_keep, j = i - r * n_keep;
@@ -117,16 +120,14 @@ __global__ void __launch_bounds__(256) scatter_cols_kernel(const void* src, int6
 cudaError_t launch_hp_fwd(const HpFwdArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;
   const dim3 grid((unsigned)((a.N + 63) / 64), (unsigned)((a.M + 63) / 64));
-  hp_fwd_kernel<<<grid, 256, 0, st>>>(a);
-  ++g_launch_count;
+  launch_kernel(hp_fwd_kernel, dim3(grid), dim3(256), 0, st, a);
   return cudaGetLastError();
 }
 
 cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st) {
   if (a.C == 0 || a.n_out == 0) return cudaSuccess;
   const dim3 grid((unsigned)((a.C + 63) / 64), (unsigned)((a.n_out + 7) / 8));
-  hp_dw_kernel<<<grid, 256, 0, st>>>(a);
-  ++g_launch_count;
+  launch_kernel(hp_dw_kernel, dim3(grid), dim3(256), 0, st, a);
   return cudaGetLastError();
 }
 
@@ -135,8 +136,7 @@ cudaError_t launch_scatter_cols(const void* src, int64_t ld_src, int src_is_f32,
   const int64_t total = rows * n_keep;
   if (total == 0) return cudaSuccess;
   const unsigned grid = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 32);
-  scatter_cols_kernel<<<grid, 256, 0, st>>>(src, ld_src, src_is_f32, dst, ld_dst, dst_is_f32, rows, n_keep, keep);
-  ++g_launch_count;
+  launch_kernel(scatter_cols_kernel, dim3(grid), dim3(256), 0, st, src, ld_src, src_is_f32, dst, ld_dst, dst_is_f32, rows, n_keep, keep);
   return cudaGetLastError();
 }
 

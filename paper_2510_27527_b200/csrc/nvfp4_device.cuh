@@ -9,6 +9,14 @@
 
 namespace nvfp4 {
 
+// Programmatic dependent launch: let the next kernel of the stream start its prologue, then wait until the previous
+// kernel has completed (its writes are visible, and it no longer reads what this kernel will overwrite). Must run
+// before the first global-memory access. A no-op when the kernel was launched without the attribute.
+__device__ __forceinline__ void pdl_prologue() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 constexpr int kRoundRTN = 0;
 constexpr int kRoundSR = 1;
 constexpr int kGsTensor = 0;

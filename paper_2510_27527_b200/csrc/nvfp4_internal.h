@@ -18,6 +18,7 @@ struct QuantRowsArgs {
   uint32_t stream_id;
   int gs_mode, sr, sf_tiled;
   int compute_amax;    // TENSOR mode: run the amax pre-pass (0: gs_cells[0] already holds the amax bits)
+  int cells_zeroed;    // the caller has already cleared gs_cells on this stream
   uint32_t* gs_cells;  // workspace: 1 cell (TENSOR) or `rows` cells (ROW)
   uint8_t* codes;
   uint8_t* sf;
@@ -49,12 +50,33 @@ struct QuantTransposeArgs {
   uint32_t stream_id;
   int gs_mode, sr, sf_tiled;
   int compute_amax;
+  int cells_zeroed;        // the caller has already cleared gs_cells on this stream
   int tensor_closed_form;  // set by the launcher
   uint32_t* gs_cells;  // 1 cell (TENSOR) or D cells (ROW)
   uint8_t* codes;
   uint8_t* sf;
   float* gscale;
 };
+
+// Every kernel of the library is launched with programmatic stream serialisation: its CTAs may be scheduled while the
+// previous kernel of the stream is still draining, run their prologue (barrier setup, tensor-memory allocation) and then
+// block in griddepcontrol.wait until that kernel has completed and its writes are visible. Each kernel calls
+// pdl_prologue() (see nvfp4_device.cuh) before its first global-memory access.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ++g_launch_count;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st);
 cudaError_t launch_quantize_transpose(const QuantTransposeArgs& a, cudaStream_t st);

@@ -15,6 +15,7 @@ namespace nvfp4 {
 // =========================================================================================================
 __global__ void __launch_bounds__(256) amax_tensor_bf16_kernel(const uint16_t* __restrict__ src, int64_t rows,
                                                               int64_t cols, int64_t ld, uint32_t* amax_bits) {
+  pdl_prologue();
   // One 16-byte chunk (8 BF16) per thread per step; rows are walked through a flattened chunk index.
   const int64_t chunks_per_row = (cols + 7) >> 3;
   const int64_t total = rows * chunks_per_row;
@@ -64,6 +65,7 @@ __global__ void __launch_bounds__(256) amax_rows_bf16_kernel(const uint16_t* __r
                                                             int64_t cols, int64_t ld,
                                                             const int32_t* __restrict__ keep, int64_t n_keep,
                                                             uint32_t* cells, int single_cell) {
+  pdl_prologue();
   const int64_t r = blockIdx.x;
   const uint16_t* p = src + r * ld;
   uint32_t m = 0;
@@ -129,6 +131,7 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
                      const int32_t* __restrict__ keep, uint64_t seed, uint32_t stream_id,
                      const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
                      float* __restrict__ gscale, uint32_t div_mul, uint32_t div_shift, int wide_loads) {
+  pdl_prologue();
   constexpr int NB = 4;  // inner blocks per thread; all loads are issued before any arithmetic
   const int64_t Kp = (K + 127) & ~(int64_t)127;
   const int64_t K16 = (K + 15) & ~(int64_t)15;
@@ -283,6 +286,7 @@ __device__ __forceinline__ float load_transpose_elem(const TransposeSrc& s, int6
 template <int SRC>
 __global__ void __launch_bounds__(256) amax_cols_generic_kernel(TransposeSrc s, int64_t rowsK, int64_t D,
                                                                uint32_t* cells, int per_column, int only_hp) {
+  pdl_prologue();
   __shared__ float red[4][64];
   __shared__ float fin[2];
   const int dl = threadIdx.x & 63, g = threadIdx.x >> 6;
@@ -342,6 +346,7 @@ __global__ void __launch_bounds__(256)
 quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t seed, uint32_t stream_id,
                           const uint32_t* __restrict__ gs_cells, int tensor_closed_form, uint8_t* __restrict__ codes,
                           uint8_t* __restrict__ sf, float* __restrict__ gscale) {
+  pdl_prologue();
   __shared__ float tile[128][65];
   __shared__ float blk_amax[8][64];
   __shared__ __align__(16) uint8_t out_codes[64][64];
@@ -487,12 +492,11 @@ static cudaError_t launch_rows_g(const QuantRowsArgs& a, cudaStream_t st) {
   }
   const int wide_loads = ((reinterpret_cast<uintptr_t>(a.src) & 31u) == 0 && (a.ld & 15) == 0) ? 1 : 0;
   if (a.keep)
-    quantize_rows_kernel<GS, SR, TILED, true><<<grid, 256, 0, st>>>(a.src, a.rows, a.K, a.ld, a.keep, a.seed, a.stream_id,
+    launch_kernel(quantize_rows_kernel<GS, SR, TILED, true>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, a.keep, a.seed, a.stream_id,
                                                                    a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads);
   else
-    quantize_rows_kernel<GS, SR, TILED, false><<<grid, 256, 0, st>>>(a.src, a.rows, a.K, a.ld, nullptr, a.seed, a.stream_id,
-                                                                    a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads);
-  ++g_launch_count;
+    launch_kernel(quantize_rows_kernel<GS, SR, TILED, false>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, nullptr, a.seed,
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads);
   return cudaGetLastError();
 }
 
@@ -511,24 +515,21 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
   cudaError_t e;
   if (a.gs_mode == kGsTensor) {
     if (a.compute_amax) {
-      if ((e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
+      if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
       if (a.keep) {  // amax over the kept columns only: one row per CTA, one atomic per row
-        amax_rows_bf16_kernel<<<(unsigned)a.rows, 256, 0, st>>>(a.src, a.rows, a.cols_src, a.ld, a.keep, a.K, a.gs_cells, 1);
-  ++g_launch_count;
+        launch_kernel(amax_rows_bf16_kernel, dim3((unsigned)a.rows), dim3(256), 0, st, a.src, a.rows, a.cols_src, a.ld, a.keep, a.K, a.gs_cells, 1);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         return launch_rows_r<kGsTensor>(a, st);
       }
       const int64_t chunks = a.rows * ((a.cols_src + 7) >> 3);
       const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
-      amax_tensor_bf16_kernel<<<grid, 256, 0, st>>>(a.src, a.rows, a.cols_src, a.ld, a.gs_cells);
-  ++g_launch_count;
+      launch_kernel(amax_tensor_bf16_kernel, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.cols_src, a.ld, a.gs_cells);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     return launch_rows_r<kGsTensor>(a, st);
   }
   if (a.gs_mode == kGsRow) {
-    amax_rows_bf16_kernel<<<(unsigned)a.rows, 256, 0, st>>>(a.src, a.rows, a.cols_src, a.ld, a.keep, a.K, a.gs_cells, 0);
-  ++g_launch_count;
+    launch_kernel(amax_rows_bf16_kernel, dim3((unsigned)a.rows), dim3(256), 0, st, a.src, a.rows, a.cols_src, a.ld, a.keep, a.K, a.gs_cells, 0);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     return launch_rows_r<kGsRow>(a, st);
   }
@@ -539,12 +540,11 @@ template <int SRC, int GS, bool SR>
 static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
   const dim3 grid(blocks_for(a.rowsK, 128), blocks_for(a.D, 64));
   if (a.sf_tiled)
-    quantize_transpose_kernel<SRC, GS, SR, true><<<grid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.seed, a.stream_id, a.gs_cells,
+    launch_kernel(quantize_transpose_kernel<SRC, GS, SR, true>, dim3(grid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.seed, a.stream_id, a.gs_cells,
                                                                       a.tensor_closed_form, a.codes, a.sf, a.gscale);
   else
-    quantize_transpose_kernel<SRC, GS, SR, false><<<grid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.seed, a.stream_id, a.gs_cells,
-                                                                       a.tensor_closed_form, a.codes, a.sf, a.gscale);
-  ++g_launch_count;
+    launch_kernel(quantize_transpose_kernel<SRC, GS, SR, false>, dim3(grid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.seed, a.stream_id,
+                  a.gs_cells, a.tensor_closed_form, a.codes, a.sf, a.gscale);
   return cudaGetLastError();
 }
 
@@ -561,30 +561,26 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
   const dim3 agrid(blocks_for(a.D, 64), blocks_for(a.rowsK, 256));
   if (a.gs_mode == kGsTensor) {
     if (a.compute_amax) {
-      if ((e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
+      if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
       if (SRC == 0) {
         const int64_t chunks = a.rowsK * ((a.D + 7) >> 3);
         const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
-        amax_tensor_bf16_kernel<<<grid, 256, 0, st>>>(a.src.bf16, a.rowsK, a.D, a.src.ld, a.gs_cells);
-        ++g_launch_count;
+        launch_kernel(amax_tensor_bf16_kernel, dim3(grid), dim3(256), 0, st, a.src.bf16, a.rowsK, a.D, a.src.ld, a.gs_cells);
       } else if (a.src.in_gs_mode == kGsTensor) {
         a.tensor_closed_form = 1;  // only the BF16 rows (if any) need a pass
         if (a.src.row_map) {
-          amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 0, 1);
-          ++g_launch_count;
+          launch_kernel(amax_cols_generic_kernel<SRC>, dim3(agrid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.gs_cells, 0, 1);
         }
       } else {
-        amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 0, 0);
-        ++g_launch_count;
+        launch_kernel(amax_cols_generic_kernel<SRC>, dim3(agrid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.gs_cells, 0, 0);
       }
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
     return launch_tr_r<SRC, kGsTensor>(a, st);
   }
   if (a.gs_mode == kGsRow) {
-    if ((e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t) * (size_t)a.D, st)) != cudaSuccess) return e;
-    amax_cols_generic_kernel<SRC><<<agrid, 256, 0, st>>>(a.src, a.rowsK, a.D, a.gs_cells, 1, 0);
-    ++g_launch_count;
+    if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t) * (size_t)a.D, st)) != cudaSuccess) return e;
+    launch_kernel(amax_cols_generic_kernel<SRC>, dim3(agrid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.gs_cells, 1, 0);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     return launch_tr_r<SRC, kGsRow>(a, st);
   }
