@@ -44,6 +44,10 @@ struct Cfg {
   // tensor memory columns: two accumulators, then four scale buffers (A: 16 columns, B: 16 * BN / 128)
   static constexpr uint32_t ACC_COLS = BN;
   static constexpr uint32_t ACC_BUFS = (BN == 256) ? 1 : 2;  // 256-wide accumulators leave no room for a second one
+  // The single-accumulator variant drains tensor memory into registers first (eight epilogue warps, 128 columns each),
+  // hands the accumulator back, and only then scales / converts / stores: the next tile's MMAs run under the stores.
+  static constexpr int EPI_WARPS = (BN == 256) ? 8 : 4;
+  static constexpr int THREADS = 64 + 32 * EPI_WARPS;
   static constexpr uint32_t SF_COLS = 16 + 16 * (BN / 128);
   static constexpr uint32_t TMEM_COLS = 512;
   static_assert(ACC_BUFS * ACC_COLS + 4 * SF_COLS <= TMEM_COLS, "tensor memory budget");
@@ -300,7 +304,7 @@ __device__ __forceinline__ void store_row_chunk(const Params& p, int64_t m, int6
 }
 
 template <int GS, int BN>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(Cfg<BN>::THREADS, 1)
 gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmC, const Params p) {
   using C = Cfg<BN>;
@@ -328,7 +332,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(acc_full_bar(b), 1);
-      mbar_init(acc_empty_bar(b), 4);
+      mbar_init(acc_empty_bar(b), C::EPI_WARPS);
     }
     mbar_init(drain_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -441,6 +445,33 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int64_t m = (int64_t)mt * BM + quad * 32 + lane;
       float sa = 1.0f;
       if (GS == kGsRow && m < p.M) sa = p.a_gscale[m];
+      if (C::EPI_WARPS == 8) {
+        // drain this warp's 32 lanes x 128 columns into registers, release the accumulator, then store
+        const int half = (warp - 2) >> 2;
+        uint32_t v[4][32];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + half * 128 + q * 32, v[q]);
+        tc_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty_bar(ab));
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int64_t n0 = (int64_t)nt * BN + half * 128 + q * 32;
+          if (m < p.M && n0 < p.N) {
+            float o[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              float sc = alpha;
+              if (GS == kGsRow) sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
+              o[j] = __uint_as_float(v[q][j]) * sc;
+            }
+            store_row_chunk(p, m, n0, o);
+          }
+        }
+        continue;
+      }
       if (C::TMA_STORE && p.use_tma_store) {
         // Stage 128-byte row pieces (32 FP32 or 64 BF16 columns) in shared memory with the 128-byte swizzle and let the
         // bulk-tensor engine write them: full lines, clipped at the edges of C, asynchronous.
@@ -888,7 +919,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
   }
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
-  launch_kernel(gemm_nvfp4_kernel<GS, BN>, dim3(grid), dim3(NUM_THREADS), C::SMEM_BYTES, st, tmA, tmB, tmC, p);
+  launch_kernel(gemm_nvfp4_kernel<GS, BN>, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, tmA, tmB, tmC, p);
   return cudaGetLastError();
 }
 
