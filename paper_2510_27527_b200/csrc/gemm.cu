@@ -822,6 +822,238 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
   }
 }
 
+// =========================================================================================================
+// Two-CTA variant (cta_group::2) for large products: a pair of CTAs on neighbouring SMs computes one 256 x 256 tile.
+// Each CTA loads its own 128 rows of A, HALF of the B tile (128 of the 256 rows) and the scales it needs; the pair's
+// tensor cores read both halves of B, so every SM pulls 38 KB per k tile instead of 54 KB (128 x 256 single-CTA
+// tiles) and five stages fit. The MMAs are issued by the leader CTA (cluster rank 0) only:
+//   - both CTAs' bulk-tensor loads complete on the LEADER's "full" barrier (armed for the bytes of both);
+//   - tcgen05.commit multicasts the "stage free" / "accumulator ready" arrivals to the same barrier in both CTAs;
+//   - both CTAs' epilogue warps arrive on the leader's "accumulator free" barrier (a remote arrive for the peer).
+// No load uses cluster multicast. Accumulator: 128 lanes x 256 columns per CTA, drained into registers by eight
+// epilogue warps before it is handed back (see the 128 x 256 variant above).
+// =========================================================================================================
+constexpr int C2_STAGES = 5;
+constexpr uint32_t C2_B_BYTES = 16384;                                  // this CTA's 128 rows of the B tile
+constexpr uint32_t C2_SFB_BYTES = 4096;                                 // scales of all 256 B rows
+constexpr uint32_t C2_STAGE_BYTES = A_BYTES + C2_B_BYTES + SFA_BYTES + C2_SFB_BYTES;  // 38 KB
+constexpr uint32_t C2_SMEM_BYTES = C2_STAGES * C2_STAGE_BYTES + 1024 + 256;
+constexpr int C2_THREADS = 64 + 256;
+constexpr uint32_t C2_SF_COLS = 16 + 32;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory location in the CTA with the given cluster rank.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Bulk-tensor load of one CTA of a pair; completes on an mbarrier that may live in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, int32_t c0, int32_t c1,
+                                                 uint32_t bar_cluster_addr, uint32_t leader) {
+  asm volatile(
+      "{\n.reg .pred q;\nsetp.ne.b32 q, %5, 0;\n"
+      "@q cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n}" ::"r"(dst),
+      "l"(tm), "r"(c0), "r"(c1), "r"(bar_cluster_addr), "r"(leader)
+      : "memory");
+}
+__device__ __forceinline__ void tc2_commit_both(uint32_t bar, uint32_t leader) {
+  asm volatile(
+      "{\n.reg .pred q;\n.reg .b16 m;\nsetp.ne.b32 q, %1, 0;\nmov.b16 m, 3;\n"
+      "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], m;\n}" ::"r"(bar),
+      "r"(leader)
+      : "memory");
+}
+__device__ __forceinline__ void tc2_cp_sf(uint32_t taddr, uint64_t sdesc, uint32_t leader) {
+  asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %2, 0;\n@q tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;\n}" ::"r"(taddr),
+               "l"(sdesc), "r"(leader)
+               : "memory");
+}
+__device__ __forceinline__ void tc2_mma_nvf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate, uint32_t leader) {
+  asm volatile(
+      "{\n.reg .pred p, q;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "setp.ne.b32 q, %7, 0;\n"
+      "@q tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem), "r"(leader)
+      : "memory");
+}
+
+template <int GS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(C2_THREADS, 1)
+gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                       const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB, const Params p) {
+  constexpr int STAGES = C2_STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar_base = smem_base + STAGES * C2_STAGE_BYTES;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };             // used in the leader CTA only
+  auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };  // one per CTA
+  const uint32_t acc_full_bar = bar_base + 8u * (2 * STAGES);            // one per CTA
+  const uint32_t acc_empty_bar = bar_base + 8u * (2 * STAGES + 1);       // leader CTA only (16 arrivals)
+  const uint32_t drain_bar = bar_base + 8u * (2 * STAGES + 2);
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(acc_full_bar, 1);
+    mbar_init(acc_empty_bar, 16);
+    mbar_init(drain_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers are initialised and its tensor memory allocated
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  pdl_prologue();
+
+  const int64_t num_tiles = (int64_t)p.m_tiles * p.n_tiles;  // 256 x 256 tiles
+  const int64_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+
+  if (warp == 0) {
+    // ===================================== TMA producer (both CTAs) ========================================
+    const uint32_t leader = elect_leader();
+    uint32_t it = 0;
+    bool ok = true;
+    for (int64_t t = pair; t < num_tiles && ok; t += num_pairs) {
+      const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
+      const int32_t a_row = mt * 256 + (int32_t)rank * 128, b_row = nt * 256 + (int32_t)rank * 128;
+      const int32_t sfa_row = ((mt * 2 + (int32_t)rank) * p.sf_tiles_a) * 4;  // in units of 128 bytes
+      const int32_t sfb_row0 = ((nt * 2) * p.sf_tiles_b) * 4, sfb_row1 = ((nt * 2 + 1) * p.sf_tiles_b) * 4;
+      for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
+        const int s = it % STAGES;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.dev_status));
+        if (!ok) break;
+        const uint32_t st = smem_base + s * C2_STAGE_BYTES;
+        const uint32_t full0 = map_to_cta(full_bar(s), 0);
+        if (rank == 0) mbar_expect_tx(full_bar(s), 2 * C2_STAGE_BYTES, leader);
+        tma_load_2d_pair(st, &tmA, kt * (BK / 2), a_row, full0, leader);
+        tma_load_2d_pair(st + A_BYTES, &tmB, kt * (BK / 2), b_row, full0, leader);
+        tma_load_2d_pair(st + A_BYTES + C2_B_BYTES, &tmSFA, 0, sfa_row + kt * 16, full0, leader);
+        tma_load_2d_pair(st + A_BYTES + C2_B_BYTES + SFA_BYTES, &tmSFB, 0, sfb_row0 + kt * 16, full0, leader);
+        tma_load_2d_pair(st + A_BYTES + C2_B_BYTES + SFA_BYTES + 2048, &tmSFB, 0, sfb_row1 + kt * 16, full0, leader);
+      }
+    }
+  } else if (warp == 1) {
+    // ===================================== MMA issuer (leader CTA only) ====================================
+    if (rank == 0) {
+      const uint32_t leader = elect_leader();
+      const uint32_t idesc = (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      uint32_t it = 0, tile_it = 0;
+      bool ok = true;
+      for (int64_t t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar, (tile_it & 1) ^ 1, abort_flag, p.dev_status));
+        if (!ok) break;
+        tc_fence_after();
+        for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
+          const int s = it % STAGES;
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.dev_status));
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t st = smem_base + s * C2_STAGE_BYTES;
+          const uint32_t sf_tmem = tmem_base + 256 + (it & 3) * C2_SF_COLS;
+#pragma unroll
+          for (int kk = 0; kk < BK / 64; ++kk) {
+            tc2_cp_sf(sf_tmem + kk * 4, desc_sf(st + A_BYTES + C2_B_BYTES + kk * 512), leader);
+            tc2_cp_sf(sf_tmem + 16 + kk * 8, desc_sf(st + A_BYTES + C2_B_BYTES + SFA_BYTES + kk * 512), leader);
+            tc2_cp_sf(sf_tmem + 16 + kk * 8 + 4, desc_sf(st + A_BYTES + C2_B_BYTES + SFA_BYTES + 2048 + kk * 512), leader);
+          }
+#pragma unroll
+          for (int kk = 0; kk < BK / 64; ++kk)
+            tc2_mma_nvf4(tmem_base, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc, sf_tmem + kk * 4,
+                         sf_tmem + 16 + kk * 8, (kt | kk) != 0, leader);
+          tc2_commit_both(empty_bar(s), leader);
+        }
+        if (ok) tc2_commit_both(acc_full_bar, leader);
+      }
+      // nothing issued may still be running when tensor memory is freed; the commit covers both CTAs' work
+      asm volatile(
+          "{\n.reg .pred q;\nsetp.ne.b32 q, %1, 0;\n"
+          "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(drain_bar),
+          "r"(leader)
+          : "memory");
+      {
+        const long long t0 = clock64();
+        while (!mbar_try(drain_bar, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
+        }
+      }
+    }
+  } else {
+    // ===================================== epilogue (both CTAs, eight warps) ================================
+    const int quad = warp & 3;
+    const int half = (warp - 2) >> 2;
+    const uint32_t acc_empty_leader = map_to_cta(acc_empty_bar, 0);
+    uint32_t tile_it = 0;
+    bool ok = true;
+    float alpha = 1.0f;
+    if (GS == kGsTensor) alpha = __fmul_rn(p.a_gscale[0], p.b_gscale[0]);
+    for (int64_t t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
+      const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
+      if (!(ok = mbar_wait(acc_full_bar, tile_it & 1, abort_flag, p.dev_status))) break;
+      tc_fence_after();
+      const int64_t m = (int64_t)mt * 256 + rank * 128 + quad * 32 + lane;
+      float sa = 1.0f;
+      if (GS == kGsRow && m < p.M) sa = p.a_gscale[m];
+      uint32_t v[4][32];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + half * 128 + q * 32, v[q]);
+      tc_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int64_t n0 = (int64_t)nt * 256 + half * 128 + q * 32;
+        if (m < p.M && n0 < p.N) {
+          float o[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            float sc = alpha;
+            if (GS == kGsRow) sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
+            o[j] = __uint_as_float(v[q][j]) * sc;
+          }
+          store_row_chunk(p, m, n0, o);
+        }
+      }
+    }
+  }
+
+  // ===================================== teardown ============================================================
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer may still be reading this CTA's shared memory through the pair's MMAs until here
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------------------
@@ -923,6 +1155,58 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// Scale bytes of an operand as a 2-D byte tensor of 128-byte rows; box = 16 rows = the 2 KB of one (row tile, k tile).
+bool make_sf_map(CUtensorMap* tm, const uint8_t* sf, int64_t total_bytes) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {128, (cuuint64_t)(total_bytes / 128)};
+  const cuuint64_t strides[1] = {128};
+  const cuuint32_t box[2] = {128, 16};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(sf), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int GS>
+cudaError_t launch_2cta(const GemmArgs& a, cudaStream_t st) {
+  const int64_t Kp = (a.K + 127) & ~(int64_t)127;
+  const int64_t kb_padded = ((Kp >> 4) + 15) & ~(int64_t)15;
+  const int64_t sfa_bytes = ((a.M + 127) / 128) * 128 * kb_padded, sfb_bytes = ((a.N + 127) / 128) * 128 * kb_padded;
+  CUtensorMap tmA, tmB, tmSFA, tmSFB;
+  if (!make_codes_map(&tmA, a.a_codes, a.M, Kp, 128) || !make_codes_map(&tmB, a.b_codes, a.N, Kp, 128) ||
+      !make_sf_map(&tmSFA, a.a_sf, sfa_bytes) || !make_sf_map(&tmSFB, a.b_sf, sfb_bytes))
+    return cudaErrorInvalidValue;
+  Params p{};
+  p.a_sf = a.a_sf;
+  p.b_sf = a.b_sf;
+  p.a_gscale = a.a_gscale;
+  p.b_gscale = a.b_gscale;
+  p.addend = a.addend;
+  p.ld_add = a.ld_add;
+  p.C = a.C;
+  p.ldc = a.ldc;
+  p.M = a.M;
+  p.N = a.N;
+  p.k_tiles = (int32_t)((Kp + BK - 1) / BK);
+  p.sf_tiles_a = p.sf_tiles_b = (int32_t)(kb_padded >> 2);
+  p.m_tiles = (int32_t)((a.M + 255) / 256);
+  p.n_tiles = (int32_t)((a.N + 255) / 256);
+  p.c_is_f32 = a.c_is_f32;
+  p.accumulate = a.accumulate;
+  p.dev_status = a.dev_status;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_2cta_kernel<GS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C2_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
+  const unsigned pairs = (unsigned)std::min<int64_t>(tiles, sm_count() / 2);
+  launch_kernel(gemm_nvfp4_2cta_kernel<GS>, dim3(2 * pairs), dim3(C2_THREADS), C2_SMEM_BYTES, st, tmA, tmB, tmSFA, tmSFB, p);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_block128(const GemmArgs& a, cudaStream_t st) {
   const int64_t Kp = (a.K + 127) & ~(int64_t)127;
   if (Kp / 128 > B128_MAX_CHUNKS) return cudaErrorInvalidValue;
@@ -972,6 +1256,13 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   // 128 x 256 tiles halve the operand traffic per flop; they pay off once there are enough of them to fill the SMs.
   const char* force = getenv("NVFP4_GEMM_BN");
   const bool wide = force ? atoi(force) == 256 : (a.K >= 2048 && ((a.M + 127) / 128) * ((a.N + 255) / 256) >= 2 * sm_count());
+  // Pairs of CTAs on 256 x 256 tiles for the largest products. A 256-row tile of an operand spans two 128-row scale
+  // tiles, and the last one must exist in full: rows are padded to 128 in the scale layout, so any M, N work.
+  const char* pair_env = getenv("NVFP4_GEMM_2CTA");
+  const bool pairs = pair_env ? atoi(pair_env) != 0
+                              : (a.K >= 2048 && ((a.M + 255) / 256) * ((a.N + 255) / 256) >= 2 * (sm_count() / 2));
+  if (pairs && a.gs_mode == kGsTensor) return launch_2cta<kGsTensor>(a, st);
+  if (pairs && a.gs_mode == kGsRow) return launch_2cta<kGsRow>(a, st);
   switch (a.gs_mode) {
     case kGsTensor: return wide ? launch_variant<kGsTensor, 256>(a, st) : launch_variant<kGsTensor, 128>(a, st);
     case kGsRow: return wide ? launch_variant<kGsRow, 256>(a, st) : launch_variant<kGsRow, 128>(a, st);
