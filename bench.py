@@ -204,8 +204,11 @@ def run_ours(args):
         L.W = [b.upload_bf16(W, dev)]
         for extra in range(1, layers):
             L.W.append(b.upload_bf16(synth.weights(C, D, synth.seed_of(cfg_id, 100 * extra + li)), dev))
-        L.cfg = b.LayerConfig(gs_mode=gs_mode, seed=0, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32)
-        L.saved = b.Saved(b.alloc_operand(tokens, D, gs_mode, device=dev), b.alloc_operand(C, D, gs_mode, device=dev), L.X, L.W[0])
+        n_out = int(round(args.outliers * D))
+        outl = synth.outlier_channels(D, n_out, synth.seed_of(cfg_id, 50 + li)) if n_out else None
+        L.cfg = b.LayerConfig(gs_mode=gs_mode, seed=0, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32, outliers=outl)
+        L.cfg.prepare(D, dev)
+        L.saved = b.alloc_saved(L.X, L.W[0], L.cfg)
         L.Y = torch.empty((tokens, C), dtype=torch.bfloat16, device=dev)
         L.dXo = torch.empty((tokens, D), dtype=torch.bfloat16, device=dev)
         L.dWo = torch.empty((C, D), dtype=torch.float32, device=dev)
@@ -374,7 +377,7 @@ def run_ours(args):
         "metric": "nvfp4_linear_fwd_bwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "fp4(e2m1)xfp4 with ue4m3 block scales, f32 accumulate", "data": "synthetic",
-        "config": {"workload": workload_name(args), "gs_mode": args.gs, "l2": "256 MiB write + 256 MiB read flush before every timed step",
+        "config": {"workload": workload_name(args), "gs_mode": args.gs, "outcontrol_fraction": args.outliers, "l2": "256 MiB write + 256 MiB read flush before every timed step",
                    "timing": "CUDA events per step on the launch stream, summed"},
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
@@ -473,6 +476,8 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=1024, help="token slab of one oracle step (reference arm)")
     ap.add_argument("--cpu-tokens", type=int, default=4096, help="token slab of the cpu_baseline leg")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--outliers", type=float, default=0.0,
+                    help="OutControl: fraction of input channels kept in BF16 (0 = off; the paper uses 0.10)")
     ap.add_argument("--no-breakdown", action="store_true", help="only warm-up + timed steps (used for ncu launch lists)")
     ap.add_argument("--sweep", action="store_true", help="roofline sweep of the large GEMM shapes instead of the step benchmark")
     ap.add_argument("--shapes", default="", help="with --sweep: comma list of MxNxK")

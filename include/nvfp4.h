@@ -190,15 +190,22 @@ typedef struct {
 } nvfp4_layer_cfg;
 
 /* What forward leaves for backward. qx [N_tok, D - n_out] and qw [C, D - n_out] are filled by
- * nvfp4_linear_fwd (buffers are the caller's, sf_layout TILED128x4). X and W must stay valid until backward
- * when n_out > 0 (their outlier columns are read again). */
+ * nvfp4_linear_fwd (buffers are the caller's, sf_layout TILED128x4). With OutControl (n_out > 0) forward also
+ * fills X_out [N_tok, Kh] and W_out [C, Kh]: compact BF16 copies of the outlier channels X[:, A], W[:, A], zero-padded
+ * to Kh = nvfp4_outlier_pad(n_out) columns (caller-owned device buffers, 16-byte aligned; NULL when n_out = 0).
+ * Backward reads only these and the operands; X and W themselves are not touched again. */
 typedef struct {
   nvfp4_operand qx, qw;
-  const void* X; /* BF16 [N_tok, D] */
+  const void* X; /* BF16 [N_tok, D] (recorded by forward; informational) */
   const void* W; /* BF16 [C, D]     */
   int64_t ldx, ldw;
   int64_t N_tok, D, C;
+  void* X_out; /* BF16 [N_tok, Kh] */
+  void* W_out; /* BF16 [C, Kh]     */
 } nvfp4_saved;
+
+/* Columns of the compact outlier-channel matrices: n_out rounded up to a multiple of 64 (0 for n_out = 0). */
+int64_t nvfp4_outlier_pad(int64_t n_out);
 
 typedef enum { NVFP4_OP_FWD = 0, NVFP4_OP_BWD_DX = 1, NVFP4_OP_BWD_DW = 2 } nvfp4_op_kind;
 size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, int64_t C, int64_t n_out,

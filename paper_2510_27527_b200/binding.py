@@ -46,11 +46,12 @@ class CLayerCfg(ctypes.Structure):
 
 class CSaved(ctypes.Structure):
     _fields_ = [("qx", COperand), ("qw", COperand), ("X", c_vp), ("W", c_vp), ("ldx", c_i64), ("ldw", c_i64),
-                ("N_tok", c_i64), ("D", c_i64), ("C", c_i64)]
+                ("N_tok", c_i64), ("D", c_i64), ("C", c_i64), ("X_out", c_vp), ("W_out", c_vp)]
 
 
 EXPORTS = {
     "nvfp4_padded_k": (c_i64, [c_i64]),
+    "nvfp4_outlier_pad": (c_i64, [c_i64]),
     "nvfp4_operand_codes_bytes": (c_sz, [c_i64, c_i64]),
     "nvfp4_operand_sf_bytes": (c_sz, [c_i64, c_i64, c_i32]),
     "nvfp4_operand_gscale_count": (c_sz, [c_i64, c_i64, c_i32]),
@@ -271,10 +272,24 @@ class Saved:
     qw: Operand
     X: torch.Tensor
     W: torch.Tensor
+    X_out: torch.Tensor | None = None  # [N_tok, Kh] bf16, OutControl only
+    W_out: torch.Tensor | None = None  # [C, Kh] bf16
 
     def c(self) -> CSaved:
         return CSaved(self.qx.c(), self.qw.c(), _ptr(self.X), _ptr(self.W), self.X.stride(0), self.W.stride(0),
-                      self.X.shape[0], self.X.shape[1], self.W.shape[0])
+                      self.X.shape[0], self.X.shape[1], self.W.shape[0], _ptr(self.X_out), _ptr(self.W_out))
+
+
+def alloc_saved(X: torch.Tensor, W: torch.Tensor, cfg: "LayerConfig") -> "Saved":
+    """Device buffers of everything forward leaves for backward."""
+    N_tok, D = X.shape
+    C = W.shape[0]
+    Dk = D - cfg.n_out
+    Kh = _lib.nvfp4_outlier_pad(cfg.n_out)
+    xo = torch.empty((N_tok, Kh), dtype=torch.bfloat16, device=X.device) if Kh else None
+    wo = torch.empty((C, Kh), dtype=torch.bfloat16, device=X.device) if Kh else None
+    return Saved(alloc_operand(N_tok, Dk, cfg.gs_mode, SF_TILED128x4, X.device), alloc_operand(C, Dk, cfg.gs_mode, SF_TILED128x4, X.device),
+                 X, W, xo, wo)
 
 
 def linear_workspace(op_kind: int, N_tok: int, D: int, C: int, cfg: LayerConfig, device="cuda") -> torch.Tensor:
@@ -288,8 +303,7 @@ def nvfp4_linear_fwd(X: torch.Tensor, W: torch.Tensor, cfg: LayerConfig, Y: torc
     cfg.prepare(D, X.device)
     Dk = D - cfg.n_out
     if saved is None:
-        saved = Saved(alloc_operand(N_tok, Dk, cfg.gs_mode, SF_TILED128x4, X.device),
-                      alloc_operand(C, Dk, cfg.gs_mode, SF_TILED128x4, X.device), X, W)
+        saved = alloc_saved(X, W, cfg)
     else:
         saved.X, saved.W = X, W
     if Y is None:

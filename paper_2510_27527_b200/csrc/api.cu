@@ -189,6 +189,8 @@ extern "C" {
 
 int64_t nvfp4_padded_k(int64_t K) { return round_up(K, 128); }
 
+int64_t nvfp4_outlier_pad(int64_t n_out) { return round_up(n_out, 64); }
+
 size_t nvfp4_operand_codes_bytes(int64_t R, int64_t K) { return (size_t)(R * (nvfp4_padded_k(K) / 2)); }
 
 size_t nvfp4_operand_sf_bytes(int64_t R, int64_t K, int32_t sf_layout) {
@@ -320,7 +322,10 @@ size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, i
     carve_size(total, cells_bytes(Dk, gs_mode));
     operand_sizes(total, C, N_tok, gs_mode);
     operand_sizes(total, Dk, N_tok, gs_mode);
-    if (n_out > 0) carve_size(total, (size_t)C * (size_t)round_up(Dk, 4) * 4);
+    if (n_out > 0) {
+      carve_size(total, (size_t)C * (size_t)round_up(Dk, 4) * 4);
+      carve_size(total, hp_dw_partial_floats(N_tok, C, nvfp4_outlier_pad(n_out)) * 4);
+    }
   }
   return ((total + 255) & ~(size_t)255) + 256;
 }
@@ -362,6 +367,11 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
   if ((s = do_quantize_rows(Wp, C, D, ldw, cfg->rounding[1], cfg->seed, 2, keep, Dk, &saved->qw, cells_w, st, 1)) != NVFP4_OK)
     return s;
   if (n_out > 0) {
+    if (!saved->X_out || !saved->W_out) return NVFP4_ERR_NULL;
+    const int64_t Kh = nvfp4_outlier_pad(n_out);
+    if (launch_gather_cols(Xp, ldx, N_tok, cfg->outlier_cols, n_out, static_cast<uint16_t*>(saved->X_out), Kh, st) != cudaSuccess ||
+        launch_gather_cols(Wp, ldw, C, cfg->outlier_cols, n_out, static_cast<uint16_t*>(saved->W_out), Kh, st) != cudaSuccess)
+      return NVFP4_ERR_CUDA;
     HpFwdArgs h{};
     h.X = Xp; h.W = Wp; h.ldx = ldx; h.ldw = ldw; h.M = N_tok; h.N = C; h.n_out = n_out;
     h.outl = cfg->outlier_cols; h.Y = addend; h.ldy = ld_add;
@@ -382,7 +392,6 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
   const int64_t n_out = cfg->n_out;
   if ((s = check_operand_ptrs(&saved->qw)) != NVFP4_OK) return s;
   if (saved->qw.R != C || saved->qw.K != D - n_out) return NVFP4_ERR_SHAPE;
-  if (n_out > 0 && !saved->W) return NVFP4_ERR_NULL;
   if (bad_matrix(dY, lddy, C, 2) || bad_matrix(dX, lddx, D, cfg->dx_dtype == NVFP4_DT_F32 ? 4 : 2)) return NVFP4_ERR_ALIGN;
   if (!workspace || ws_bytes < nvfp4_linear_workspace_bytes(NVFP4_OP_BWD_DX, N_tok, D, C, n_out, cfg->gs_mode))
     return NVFP4_ERR_WORKSPACE;
@@ -405,12 +414,56 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
   ts.in_K = saved->qw.K;
   ts.in_gs_mode = saved->qw.gs_mode;
   ts.in_sf_tiled = saved->qw.sf_layout == NVFP4_SF_TILED128x4;
-  if (n_out > 0) {
-    ts.row_map = cfg->col_map;
-    ts.hp = static_cast<const uint16_t*>(saved->W);
-    ts.hp_ld = saved->ldw;
+  if (n_out == 0) {
+    if ((s = do_quantize_transpose(ts, 1, C, D, cfg->rounding[3], cfg->seed, 4, &q4, cells4, st, 1)) != NVFP4_OK) return s;
+  } else {
+    // W-hat^T over all D channels in two passes that write disjoint operand rows: the kept channels from the forward
+    // operand (compact column j -> row keep[j]) and the outlier channels from the compact BF16 copy (column j -> row
+    // outl[j]). Rows are quantized independently; only the TENSOR-mode scale couples them: its maximum is the larger
+    // of float32(2688 * Sg) of the forward operand and the BF16 copy's amax, which both passes are told about.
+    if (!saved->W_out) return NVFP4_ERR_NULL;
+    const int64_t Kh = nvfp4_outlier_pad(n_out);
+    if (clear_sf_padding(&q4, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+    const bool closed = cfg->gs_mode == NVFP4_GS_TENSOR && saved->qw.gs_mode == NVFP4_GS_TENSOR;
+    TransposeSrc th{};
+    th.bf16 = static_cast<const uint16_t*>(saved->W_out);
+    th.ld = Kh;
+    th.out_rows = cfg->outlier_cols;
+    ts.out_rows = cfg->keep_cols;
+    QuantTransposeArgs qa{};
+    qa.seed = cfg->seed;
+    qa.stream_id = 4;
+    qa.gs_mode = cfg->gs_mode;
+    qa.sr = cfg->rounding[3] == NVFP4_ROUND_SR;
+    qa.sf_tiled = 1;
+    qa.cells_zeroed = 1;
+    qa.gs_cells = cells4;
+    qa.codes = q4.codes;
+    qa.sf = q4.sf;
+    qa.gscale = q4.gscale;
+    qa.rowsK = C;
+    if (cfg->gs_mode == NVFP4_GS_TENSOR) {
+      // one amax pass over the compact BF16 copy (and over the forward operand unless the closed form applies)
+      if (launch_amax_tensor(static_cast<const uint16_t*>(saved->W_out), C, Kh, Kh, cells4, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+      if (closed) {
+        th.closed_form_sg = saved->qw.gscale;
+        ts.closed_form_sg = saved->qw.gscale;
+      } else if (launch_amax_transpose_src(ts, 1, C, D - n_out, cells4, st) != cudaSuccess) {
+        return NVFP4_ERR_CUDA;
+      }
+      qa.compute_amax = 0;
+    } else {
+      qa.compute_amax = 1;  // ROW: per-row cells, each pass fills the rows it owns; BLOCK128: no pre-pass
+    }
+    qa.from_codes = 1;
+    qa.D = D - n_out;
+    qa.src = ts;
+    if (launch_quantize_transpose(qa, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+    qa.from_codes = 0;
+    qa.D = n_out;
+    qa.src = th;
+    if (launch_quantize_transpose(qa, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   }
-  if ((s = do_quantize_transpose(ts, 1, C, D, cfg->rounding[3], cfg->seed, 4, &q4, cells4, st, 1)) != NVFP4_OK) return s;
   return do_gemm(&q3, &q4, dX, cfg->dx_dtype, lddx, 0, nullptr, 0, cfg->dev_status, st);
 }
 
@@ -424,7 +477,7 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
   const int64_t n_out = cfg->n_out, Dk = D - n_out;
   if ((s = check_operand_ptrs(&saved->qx)) != NVFP4_OK) return s;
   if (saved->qx.R != N_tok || saved->qx.K != Dk) return NVFP4_ERR_SHAPE;
-  if (n_out > 0 && !saved->X) return NVFP4_ERR_NULL;
+  if (n_out > 0 && !saved->X_out) return NVFP4_ERR_NULL;
   const int dw_f32 = cfg->dw_dtype == NVFP4_DT_F32;
   if (bad_matrix(dY, lddy, C, 2) || bad_matrix(dW, lddw, D, dw_f32 ? 4 : 2)) return NVFP4_ERR_ALIGN;
   if (!workspace || ws_bytes < nvfp4_linear_workspace_bytes(NVFP4_OP_BWD_DW, N_tok, D, C, n_out, cfg->gs_mode))
@@ -439,8 +492,10 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
       !cells6)
     return NVFP4_ERR_WORKSPACE;
   const int64_t ld_compact = round_up(Dk, 4);
+  const int64_t Kh = nvfp4_outlier_pad(n_out);
   float* compact = n_out > 0 ? static_cast<float*>(cv.take((size_t)C * ld_compact * 4)) : nullptr;
-  if (n_out > 0 && !compact) return NVFP4_ERR_WORKSPACE;
+  float* hp_partial = n_out > 0 ? static_cast<float*>(cv.take(hp_dw_partial_floats(N_tok, C, Kh) * 4)) : nullptr;
+  if (n_out > 0 && (!compact || !hp_partial)) return NVFP4_ERR_WORKSPACE;
 
   TransposeSrc t5{};
   t5.bf16 = static_cast<const uint16_t*>(dY);
@@ -461,9 +516,9 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
   if (launch_scatter_cols(compact, ld_compact, 1, dW, lddw, dw_f32, C, Dk, cfg->keep_cols, st) != cudaSuccess)
     return NVFP4_ERR_CUDA;
   HpDwArgs h{};
-  h.dY = static_cast<const uint16_t*>(dY); h.X = static_cast<const uint16_t*>(saved->X);
-  h.lddy = lddy; h.ldx = saved->ldx; h.T = N_tok; h.C = C; h.n_out = n_out; h.outl = cfg->outlier_cols;
-  h.dW = dW; h.dw_is_f32 = dw_f32; h.lddw = lddw;
+  h.dY = static_cast<const uint16_t*>(dY); h.X_out = static_cast<const uint16_t*>(saved->X_out);
+  h.lddy = lddy; h.Kh = Kh; h.T = N_tok; h.C = C; h.n_out = n_out; h.outl = cfg->outlier_cols;
+  h.dW = dW; h.dw_is_f32 = dw_f32; h.lddw = lddw; h.partial = hp_partial;
   return launch_hp_dw(h, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 

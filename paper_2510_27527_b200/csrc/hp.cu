@@ -54,41 +54,99 @@ __global__ void __launch_bounds__(256) hp_fwd_kernel(HpFwdArgs a) {
   }
 }
 
-// dW[c, outl[j]] = sum_t dY[t, c] * X[t, outl[j]].  One CTA per (64 output channels c, 8 outlier channels j);
-// four token groups per CTA reduced through shared memory in a fixed order.
-__global__ void __launch_bounds__(256) hp_dw_kernel(HpDwArgs a) {
+// dW[c, outl[j]] = sum_t dY[t, c] * X_out[t, j]. The token range is split over blockIdx.y; each CTA owns 64 output
+// channels c and walks its tokens in chunks of 64 staged in shared memory (dY chunk [64 t x 64 c], X_out chunk
+// [64 t x 64 j]); a thread accumulates 16 outlier channels for one c. Partial sums go to a workspace and a second
+// kernel adds them in a fixed order (bit-reproducible results).
+constexpr int kHpDwSplit = 16;
+
+__global__ void __launch_bounds__(256) hp_dw_partial_kernel(HpDwArgs a, int64_t t_per_split) {
   pdl_prologue();
-  __shared__ float red[4][8][64];
-  const int cl = threadIdx.x & 63, tg = threadIdx.x >> 6;
-  const int64_t c = (int64_t)blockIdx.x * 64 + cl;
-  const int64_t j0 = (int64_t)blockIdx.y * 8;
-  int64_t cols[8];
+  __shared__ float dy_s[64][65];
+  __shared__ float x_s[64][64];
+  const int cl = threadIdx.x & 63, jg = threadIdx.x >> 6;  // jg: which 16 outlier channels of the 64-wide chunk
+  const int64_t c0 = (int64_t)blockIdx.x * 64;
+  const int64_t t_begin = (int64_t)blockIdx.y * t_per_split, t_end = min(a.T, t_begin + t_per_split);
+  for (int64_t j0 = 0; j0 < a.Kh; j0 += 64) {
+    if (j0 >= a.n_out) break;
+    const bool active = j0 + jg * 16 < a.n_out;
+    float acc[16];
 #pragma unroll
-  for (int j = 0; j < 8; ++j) cols[j] = (j0 + j < a.n_out) ? a.outl[j0 + j] : -1;
-  float acc[8] = {};
-  if (c < a.C) {
-    for (int64_t t = tg; t < a.T; t += 4) {
-      const float g = bf16_bits_to_float(a.dY[t * a.lddy + c]);
-      const uint16_t* xr = a.X + t * a.ldx;
+    for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
+    for (int64_t tc = t_begin; tc < t_end; tc += 64) {
+      __syncthreads();
+      for (int e = threadIdx.x; e < 64 * 8; e += 256) {  // 64 rows x 8 chunks of 8 BF16
+        const int tr = e >> 3, ch = (e & 7) << 3;
+        const int64_t t = tc + tr;
+        uint4 g = make_uint4(0, 0, 0, 0), x = make_uint4(0, 0, 0, 0);
+        if (t < t_end) {
+          if (c0 + ch + 8 <= a.C && (a.lddy & 7) == 0) {
+            g = *reinterpret_cast<const uint4*>(a.dY + t * a.lddy + c0 + ch);
+          } else {
+            uint32_t w[4] = {0, 0, 0, 0};
+            for (int q = 0; q < 8; ++q)
+              if (c0 + ch + q < a.C) w[q >> 1] |= (uint32_t)a.dY[t * a.lddy + c0 + ch + q] << (16 * (q & 1));
+            g = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+          x = *reinterpret_cast<const uint4*>(a.X_out + t * a.Kh + j0 + ch);
+        }
+        const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, xw[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-      for (int j = 0; j < 8; ++j)
-        if (cols[j] >= 0) acc[j] = fmaf(g, bf16_bits_to_float(xr[cols[j]]), acc[j]);
+        for (int q = 0; q < 4; ++q) {
+          dy_s[tr][ch + 2 * q] = bf16_lo(gw[q]);
+          dy_s[tr][ch + 2 * q + 1] = bf16_hi(gw[q]);
+          x_s[tr][ch + 2 * q] = bf16_lo(xw[q]);
+          x_s[tr][ch + 2 * q + 1] = bf16_hi(xw[q]);
+        }
+      }
+      __syncthreads();
+      if (active) {
+#pragma unroll 4
+        for (int tr = 0; tr < 64; ++tr) {
+          const float g = dy_s[tr][cl];
+          const float4* xr = reinterpret_cast<const float4*>(&x_s[tr][jg * 16]);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const float4 xv = xr[q];
+            acc[4 * q] = fmaf(g, xv.x, acc[4 * q]);
+            acc[4 * q + 1] = fmaf(g, xv.y, acc[4 * q + 1]);
+            acc[4 * q + 2] = fmaf(g, xv.z, acc[4 * q + 2]);
+            acc[4 * q + 3] = fmaf(g, xv.w, acc[4 * q + 3]);
+          }
+        }
+      }
+    }
+    if (active && c0 + cl < a.C) {
+      float* dst = a.partial + ((int64_t)blockIdx.y * a.C + c0 + cl) * a.Kh + j0 + jg * 16;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) dst[j] = acc[j];
     }
   }
-#pragma unroll
-  for (int j = 0; j < 8; ++j) red[tg][j][cl] = acc[j];
-  __syncthreads();
-  if (tg == 0 && c < a.C) {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      if (cols[j] < 0) continue;
-      const float v = ((red[0][j][cl] + red[1][j][cl]) + red[2][j][cl]) + red[3][j][cl];
-      if (a.dw_is_f32)
-        reinterpret_cast<float*>(a.dW)[c * a.lddw + cols[j]] = v;
-      else
-        reinterpret_cast<uint16_t*>(a.dW)[c * a.lddw + cols[j]] = f32_to_bf16_bits(v);
-    }
+}
+
+__global__ void __launch_bounds__(256) hp_dw_reduce_kernel(HpDwArgs a, int n_split) {
+  pdl_prologue();
+  const int64_t total = a.C * a.n_out;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t c = i / a.n_out, j = i - c * a.n_out;
+    float v = 0.0f;
+    for (int sp = 0; sp < n_split; ++sp) v += a.partial[((int64_t)sp * a.C + c) * a.Kh + j];
+    const int64_t o = c * a.lddw + a.outl[j];
+    if (a.dw_is_f32)
+      reinterpret_cast<float*>(a.dW)[o] = v;
+    else
+      reinterpret_cast<uint16_t*>(a.dW)[o] = f32_to_bf16_bits(v);
   }
+}
+
+// dst[r, j] = src[r, cols[j]] (j < n), 0 for n <= j < ld_dst. One warp per row.
+__global__ void __launch_bounds__(256) gather_cols_kernel(const uint16_t* __restrict__ src, int64_t ld_src, int64_t rows,
+                                                         const int32_t* __restrict__ cols, int64_t n, uint16_t* __restrict__ dst,
+                                                         int64_t ld_dst) {
+  pdl_prologue();
+  const int64_t r = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (r >= rows) return;
+  for (int64_t j = threadIdx.x & 31; j < ld_dst; j += 32) dst[r * ld_dst + j] = j < n ? src[r * ld_src + cols[j]] : (uint16_t)0;
 }
 
 // dst[r, keep[j]] = src[r, j]
@@ -124,10 +182,25 @@ cudaError_t launch_hp_fwd(const HpFwdArgs& a, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+size_t hp_dw_partial_floats(int64_t T, int64_t C, int64_t Kh) { return (size_t)kHpDwSplit * (size_t)C * (size_t)Kh; }
+
 cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st) {
   if (a.C == 0 || a.n_out == 0) return cudaSuccess;
-  const dim3 grid((unsigned)((a.C + 63) / 64), (unsigned)((a.n_out + 7) / 8));
-  launch_kernel(hp_dw_kernel, dim3(grid), dim3(256), 0, st, a);
+  const int64_t t_per_split = ((a.T + kHpDwSplit - 1) / kHpDwSplit + 63) / 64 * 64;
+  const int n_split = (int)((a.T + t_per_split - 1) / t_per_split);
+  const dim3 grid((unsigned)((a.C + 63) / 64), (unsigned)n_split);
+  launch_kernel(hp_dw_partial_kernel, dim3(grid), dim3(256), 0, st, a, t_per_split);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const int64_t total = a.C * a.n_out;
+  launch_kernel(hp_dw_reduce_kernel, dim3((unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8)), dim3(256), 0, st, a, n_split);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gather_cols(const uint16_t* src, int64_t ld_src, int64_t rows, const int32_t* cols, int64_t n, uint16_t* dst,
+                               int64_t ld_dst, cudaStream_t st) {
+  if (rows == 0 || ld_dst == 0) return cudaSuccess;
+  launch_kernel(gather_cols_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, st, src, ld_src, rows, cols, n, dst, ld_dst);
   return cudaGetLastError();
 }
 

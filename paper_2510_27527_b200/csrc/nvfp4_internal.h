@@ -40,6 +40,9 @@ struct TransposeSrc {
   const int32_t* row_map;  // [D] or null
   const uint16_t* hp;      // BF16 [rowsK, >= D]
   int64_t hp_ld;
+  // output placement and scale coupling (both optional)
+  const int32_t* out_rows;       // operand row that source column d produces (null: d itself)
+  const float* closed_form_sg;   // TENSOR mode: the tensor maximum is at least float32(2688 * *closed_form_sg)
 };
 
 struct QuantTransposeArgs {
@@ -80,6 +83,10 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
 
 cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st);
 cudaError_t launch_quantize_transpose(const QuantTransposeArgs& a, cudaStream_t st);
+// amax of a contiguous-row BF16 matrix folded into cells[0] (atomic max; the cell must already hold a valid value)
+cudaError_t launch_amax_tensor(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, uint32_t* cell, cudaStream_t st);
+// amax of a transposing quantizer's source (from codes or BF16) folded into cells[0]
+cudaError_t launch_amax_transpose_src(const TransposeSrc& s, int from_codes, int64_t rowsK, int64_t D, uint32_t* cell, cudaStream_t st);
 
 struct GemmArgs {
   const uint8_t *a_codes, *a_sf, *b_codes, *b_sf;
@@ -103,6 +110,10 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
 // High-precision (BF16 inputs, FP32 accumulate) products over OutControl's outlier channels.
 //   fwd: Y[m, n] (+)= sum_j X[m, outl[j]] * W[n, outl[j]]
 //   dw : dW[c, outl[j]] = sum_t dY[t, c] * X[t, outl[j]]
+// dst[r, j] = src[r, cols[j]] for j < n, zero for n <= j < ld_dst (compact BF16 copy of OutControl's outlier channels)
+cudaError_t launch_gather_cols(const uint16_t* src, int64_t ld_src, int64_t rows, const int32_t* cols, int64_t n, uint16_t* dst,
+                               int64_t ld_dst, cudaStream_t st);
+
 struct HpFwdArgs {
   const uint16_t *X, *W;
   int64_t ldx, ldw, M, N, n_out;
@@ -111,13 +122,15 @@ struct HpFwdArgs {
   int64_t ldy;
 };
 struct HpDwArgs {
-  const uint16_t *dY, *X;
-  int64_t lddy, ldx, T, C, n_out;
+  const uint16_t *dY, *X_out;  // dY [T, C]; X_out [T, Kh]: the outlier channels of X, compact, zero-padded to Kh (multiple of 64)
+  int64_t lddy, Kh, T, C, n_out;
   const int32_t* outl;
   void* dW;
   int dw_is_f32;
   int64_t lddw;
+  float* partial;  // workspace: hp_dw_partial_floats(T, C, Kh) floats
 };
+size_t hp_dw_partial_floats(int64_t T, int64_t C, int64_t Kh);
 cudaError_t launch_hp_fwd(const HpFwdArgs& a, cudaStream_t st);
 cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st);
 

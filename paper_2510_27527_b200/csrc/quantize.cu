@@ -130,14 +130,41 @@ __global__ void __launch_bounds__(256)
 quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, int64_t ld,
                      const int32_t* __restrict__ keep, uint64_t seed, uint32_t stream_id,
                      const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
-                     float* __restrict__ gscale, uint32_t div_mul, uint32_t div_shift, int wide_loads) {
+                     float* __restrict__ gscale, uint32_t div_mul, uint32_t div_shift, int wide_loads, int64_t cols_src,
+                     int64_t stage_cols8) {
   pdl_prologue();
   constexpr int NB = 4;  // inner blocks per thread; all loads are issued before any arithmetic
+  extern __shared__ uint16_t row_stage[];  // GATHER only: the source rows this CTA touches, [n_rows][cols_src8]
   const int64_t Kp = (K + 127) & ~(int64_t)127;
   const int64_t K16 = (K + 15) & ~(int64_t)15;
   const int64_t nb = Kp >> 4;  // inner blocks per operand row (multiple of 8)
   const int64_t total = rows * nb;
   const int64_t cta_base = (int64_t)blockIdx.x * (256 * NB) + threadIdx.x;
+  // GATHER (OutControl compaction): the CTA's blocks cover a few whole or partial source rows; copy those rows to
+  // shared memory with coalesced 16-byte loads, then pick the kept columns from there.
+  int64_t stage_row0 = 0;
+  if (GATHER && stage_cols8 > 0) {
+    const int64_t first = (int64_t)blockIdx.x * (256 * NB);
+    const int64_t last = min(first + 256 * NB, total) - 1;
+    stage_row0 = first / nb;
+    const int64_t n_rows = last / nb - stage_row0 + 1;
+    const int64_t chunks_per_row = stage_cols8 >> 3;
+    for (int64_t e = threadIdx.x; e < n_rows * chunks_per_row; e += 256) {
+      const int64_t rr = e / chunks_per_row, ch = (e - rr * chunks_per_row) << 3;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      const uint16_t* p = src + (stage_row0 + rr) * ld + ch;
+      if (ch + 8 <= cols_src) {
+        v = *reinterpret_cast<const uint4*>(p);
+      } else {
+        uint32_t t[4] = {0, 0, 0, 0};
+        for (int q = 0; q < 8; ++q)
+          if (ch + q < cols_src) t[q >> 1] |= (uint32_t)p[q] << (16 * (q & 1));
+        v = make_uint4(t[0], t[1], t[2], t[3]);
+      }
+      *reinterpret_cast<uint4*>(row_stage + rr * stage_cols8 + ch) = v;
+    }
+    __syncthreads();
+  }
 
   uint32_t w[NB][8];
   int64_t row[NB];
@@ -176,6 +203,15 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
           const uint4 v1 = *reinterpret_cast<const uint4*>(p + k0 + 8);
           w[j][0] = v0.x; w[j][1] = v0.y; w[j][2] = v0.z; w[j][3] = v0.w;
           w[j][4] = v1.x; w[j][5] = v1.y; w[j][6] = v1.z; w[j][7] = v1.w;
+        }
+      } else if (GATHER && stage_cols8 > 0 && k0 + 16 <= K) {
+        const uint16_t* sp = row_stage + (r - stage_row0) * stage_cols8;
+        const int4* kp = reinterpret_cast<const int4*>(keep + k0);  // keep is 16-byte aligned, k0 a multiple of 16
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int4 id = kp[q];
+          w[j][2 * q] = (uint32_t)sp[id.x] | ((uint32_t)sp[id.y] << 16);
+          w[j][2 * q + 1] = (uint32_t)sp[id.z] | ((uint32_t)sp[id.w] << 16);
         }
       } else {
         for (int i = 0; i < 16; ++i) {
@@ -300,7 +336,7 @@ __global__ void __launch_bounds__(256) amax_cols_generic_kernel(TransposeSrc s, 
   if (g == 0) {
     m = fmaxf(fmaxf(red[0][dl], red[1][dl]), fmaxf(red[2][dl], red[3][dl]));
     if (per_column) {
-      if (d < D && m > 0.0f) atomicMax(cells + d, __float_as_uint(m));
+      if (d < D && m > 0.0f) atomicMax(cells + (s.out_rows ? (int64_t)s.out_rows[d] : d), __float_as_uint(m));
     } else {
 #pragma unroll
       for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
@@ -406,6 +442,8 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
   // ---- phase 2: two (d, k-block) items per thread -----------------------------------------------------------
   const int dl = tid & 63;
   const int64_t d = d_base + dl;
+  // operand row produced by source column d (identity unless the caller scatters rows, as OutControl's W-hat does)
+  const int64_t o = (d < D && s.out_rows) ? (int64_t)s.out_rows[d] : d;
   float xs[2][16];
   float am[2];
 #pragma unroll
@@ -427,15 +465,16 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
 #pragma unroll
     for (int j = 0; j < 8; ++j) g = fmaxf(g, blk_amax[j][dl]);
     Sg = global_scale_from_amax(g);
-    if (d < D && tid < 64 && k_base < K) gscale[d * (Kp >> 7) + blockIdx.x] = Sg;
+    if (d < D && tid < 64 && k_base < K) gscale[o * (Kp >> 7) + blockIdx.x] = Sg;
   } else if (GS == kGsRow) {
-    Sg = global_scale_from_amax(d < D ? __uint_as_float(gs_cells[d]) : 0.0f);
-    if (d < D && tid < 64 && blockIdx.x == 0) gscale[d] = Sg;
+    Sg = global_scale_from_amax(d < D ? __uint_as_float(gs_cells[o]) : 0.0f);
+    if (d < D && tid < 64 && blockIdx.x == 0) gscale[o] = Sg;
   } else {
     float amax = __uint_as_float(gs_cells[0]);
     // TENSOR -> TENSOR re-quantization: the aligned tensor's maximum is float32(2688 * S_global) of the forward
     // operand (its largest block has scale 448 and a magnitude-6 element); gs_cells[0] then only covers BF16 rows.
     if (SRC == 1 && tensor_closed_form) amax = fmaxf(amax, __fmul_rn(2688.0f, s.in_gscale[0]));
+    if (s.closed_form_sg) amax = fmaxf(amax, __fmul_rn(2688.0f, s.closed_form_sg[0]));
     Sg = global_scale_from_amax(amax);
     if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) gscale[0] = Sg;
   }
@@ -446,11 +485,11 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
     float rcp;
     const uint32_t sb = block_scale(am[it], Sg, rcp);
     const int64_t k0 = k_base + kb * 16;
-    const uint2 packed = quantize_block16<SR>(xs[it], rcp, seed, stream_id, (uint64_t)((d * K16 + k0) >> 3));
+    const uint2 packed = quantize_block16<SR>(xs[it], rcp, seed, stream_id, (uint64_t)((o * K16 + k0) >> 3));
     *reinterpret_cast<uint2*>(&out_codes[dl][kb * 8]) = packed;
     if (d < D && k0 < Kp) {
       const int64_t b = k0 >> 4;
-      const size_t off = TILED ? sf_tiled_offset(d, b, (nb + 15) & ~(int64_t)15) : (size_t)(d * nb + b);
+      const size_t off = TILED ? sf_tiled_offset(o, b, (nb + 15) & ~(int64_t)15) : (size_t)(o * nb + b);
       sf[off] = (uint8_t)sb;
     }
   }
@@ -460,8 +499,9 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
   {
     const int row = tid >> 2, piece = tid & 3;
     const int64_t dd = d_base + row;
+    const int64_t oo = (dd < D && s.out_rows) ? (int64_t)s.out_rows[dd] : dd;
     if (dd < D && k_base + piece * 32 < Kp)
-      *reinterpret_cast<uint4*>(codes + dd * (Kp >> 1) + (k_base >> 1) + piece * 16) =
+      *reinterpret_cast<uint4*>(codes + oo * (Kp >> 1) + (k_base >> 1) + piece * 16) =
           *reinterpret_cast<const uint4*>(&out_codes[row][piece * 16]);
   }
 }
@@ -491,12 +531,30 @@ static cudaError_t launch_rows_g(const QuantRowsArgs& a, cudaStream_t st) {
     }
   }
   const int wide_loads = ((reinterpret_cast<uintptr_t>(a.src) & 31u) == 0 && (a.ld & 15) == 0) ? 1 : 0;
-  if (a.keep)
-    launch_kernel(quantize_rows_kernel<GS, SR, TILED, true>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, a.keep, a.seed, a.stream_id,
-                                                                   a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads);
-  else
+  if (a.keep) {
+    // rows a CTA can touch: its 1024 blocks span at most 1024 / nb + 2 rows; stage them if they fit in shared memory
+    const int64_t cols8 = (a.cols_src + 7) & ~(int64_t)7;
+    const int64_t max_rows = 1024 / (int64_t)d + 2;
+    size_t smem = (size_t)(max_rows * cols8 * 2);
+    int64_t stage_cols8 = cols8;
+    if (smem > 160 * 1024 || (reinterpret_cast<uintptr_t>(a.keep) & 15u) != 0 || (a.ld & 7) != 0) {
+      smem = 0;
+      stage_cols8 = 0;  // fall back to per-element global loads
+    } else if (smem > 48 * 1024) {
+      static size_t configured = 0;
+      if (smem > configured) {
+        cudaError_t e = cudaFuncSetAttribute(quantize_rows_kernel<GS, SR, TILED, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             160 * 1024);
+        if (e != cudaSuccess) return e;
+        configured = 160 * 1024;
+      }
+    }
+    launch_kernel(quantize_rows_kernel<GS, SR, TILED, true>, dim3(grid), dim3(256), smem, st, a.src, a.rows, a.K, a.ld, a.keep, a.seed,
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, stage_cols8);
+  } else {
     launch_kernel(quantize_rows_kernel<GS, SR, TILED, false>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, nullptr, a.seed,
-                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads);
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0);
+  }
   return cudaGetLastError();
 }
 
@@ -585,6 +643,25 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
     return launch_tr_r<SRC, kGsRow>(a, st);
   }
   return launch_tr_r<SRC, kGsBlock128>(a, st);
+}
+
+cudaError_t launch_amax_tensor(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, uint32_t* cell, cudaStream_t st) {
+  if (rows == 0 || cols == 0) return cudaSuccess;
+  const int64_t chunks = rows * ((cols + 7) >> 3);
+  const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
+  launch_kernel(amax_tensor_bf16_kernel, dim3(grid), dim3(256), 0, st, src, rows, cols, ld, cell);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_amax_transpose_src(const TransposeSrc& s, int from_codes, int64_t rowsK, int64_t D, uint32_t* cell,
+                                      cudaStream_t st) {
+  if (rowsK == 0 || D == 0) return cudaSuccess;
+  const dim3 agrid(blocks_for(D, 64), blocks_for(rowsK, 256));
+  if (from_codes)
+    launch_kernel(amax_cols_generic_kernel<1>, dim3(agrid), dim3(256), 0, st, s, rowsK, D, cell, 0, 0);
+  else
+    launch_kernel(amax_cols_generic_kernel<0>, dim3(agrid), dim3(256), 0, st, s, rowsK, D, cell, 0, 0);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_quantize_transpose(const QuantTransposeArgs& a, cudaStream_t st) {
