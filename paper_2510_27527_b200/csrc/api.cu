@@ -136,7 +136,8 @@ nvfp4_status do_quantize_transpose(const TransposeSrc& src, int from_codes, int6
 }
 
 nvfp4_status do_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
-                     int32_t accumulate, const float* addend, int64_t ld_add, int32_t* dev_status, cudaStream_t st) {
+                     int32_t accumulate, const float* addend, int64_t ld_add, int32_t* dev_status, cudaStream_t st,
+                     const void* hp_a = nullptr, const void* hp_b = nullptr, int64_t hp_Kh = 0) {
   if (A->gs_mode == NVFP4_GS_BLOCK128 && nvfp4_padded_k(A->K) > gemm_block128_max_k()) return NVFP4_ERR_LIMIT;
   GemmArgs g{};
   g.a_codes = A->codes;
@@ -156,6 +157,9 @@ nvfp4_status do_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, in
   g.addend = addend;
   g.ld_add = ld_add;
   g.dev_status = dev_status;
+  g.hp_a = hp_a;
+  g.hp_b = hp_b;
+  g.hp_Kh = hp_Kh;
   return launch_gemm(g, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
@@ -372,13 +376,19 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
     if (launch_gather_cols(Xp, ldx, N_tok, cfg->outlier_cols, n_out, static_cast<uint16_t*>(saved->X_out), Kh, st) != cudaSuccess ||
         launch_gather_cols(Wp, ldw, C, cfg->outlier_cols, n_out, static_cast<uint16_t*>(saved->W_out), Kh, st) != cudaSuccess)
       return NVFP4_ERR_CUDA;
-    HpFwdArgs h{};
-    h.X = Xp; h.W = Wp; h.ldx = ldx; h.ldw = ldw; h.M = N_tok; h.N = C; h.n_out = n_out;
-    h.outl = cfg->outlier_cols; h.Y = addend; h.ldy = ld_add;
-    if (launch_hp_fwd(h, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+    if (cfg->gs_mode == NVFP4_GS_BLOCK128) {
+      // the outer-block GEMM variant takes the side product as an FP32 addend computed beforehand
+      HpFwdArgs h{};
+      h.X = Xp; h.W = Wp; h.ldx = ldx; h.ldw = ldw; h.M = N_tok; h.N = C; h.n_out = n_out;
+      h.outl = cfg->outlier_cols; h.Y = addend; h.ldy = ld_add;
+      if (launch_hp_fwd(h, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+    }
   }
   saved->X = X; saved->W = W; saved->ldx = ldx; saved->ldw = ldw;
   saved->N_tok = N_tok; saved->D = D; saved->C = C;
+  if (n_out > 0 && cfg->gs_mode != NVFP4_GS_BLOCK128)  // Y = FP4 product + X_out W_out^T, both inside one kernel
+    return do_gemm(&saved->qx, &saved->qw, Y, cfg->y_dtype, ldy, 0, nullptr, 0, cfg->dev_status, st, saved->X_out, saved->W_out,
+                   nvfp4_outlier_pad(n_out));
   return do_gemm(&saved->qx, &saved->qw, Y, cfg->y_dtype, ldy, 0, addend, ld_add, cfg->dev_status, st);
 }
 

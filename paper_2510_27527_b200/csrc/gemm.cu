@@ -70,6 +70,7 @@ struct Params {
   int32_t sf_tiles_b;
   int32_t m_tiles, n_tiles;
   int32_t c_is_f32, accumulate;
+  int32_t hp_k_tiles;     // OutControl: 64-wide BF16 k tiles of the high-precision side product (0 = none)
   int32_t use_tma_store;  // C is described by a tensor map: stage the epilogue in shared memory and bulk-store it
   int32_t* dev_status;
 };
@@ -161,6 +162,17 @@ __device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t a_desc, ui
       "setp.ne.b32 q, %7, 0;\n"
       "@q tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n}" ::"r"(d_tmem),
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem), "r"(leader)
+      : "memory");
+}
+// BF16 x BF16 -> FP32 (kind::f16), K = 16 per instruction; used for OutControl's high-precision side product.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
+                                            uint32_t leader) {
+  asm volatile(
+      "{\n.reg .pred p, q;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "setp.ne.b32 q, %5, 0;\n"
+      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader)
       : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
@@ -306,7 +318,8 @@ __device__ __forceinline__ void store_row_chunk(const Params& p, int64_t m, int6
 template <int GS, int BN>
 __global__ void __launch_bounds__(Cfg<BN>::THREADS, 1)
 gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                  const __grid_constant__ CUtensorMap tmC, const Params p) {
+                  const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmAh,
+                  const __grid_constant__ CUtensorMap tmBh, const Params p) {
   using C = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -318,6 +331,11 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   auto acc_full_bar = [&](int b) { return bar_base + 8u * (2 * C::STAGES + b); };
   auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * C::STAGES + 2 + b); };
   const uint32_t drain_bar = bar_base + 8u * (2 * C::STAGES + 4);
+  const uint32_t hp_empty_bar = bar_base + 8u * (2 * C::STAGES + 5);  // high-precision accumulator drained
+  // tensor-memory columns of the optional high-precision accumulator (128 x 128 tiles only) and of the scale buffers
+  const uint32_t hp_cols = (BN == 128 && p.hp_k_tiles > 0) ? 128u : 0u;
+  const uint32_t hp_tmem_col = C::ACC_BUFS * C::ACC_COLS;
+  const uint32_t sf_tmem_col = C::ACC_BUFS * C::ACC_COLS + hp_cols;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   volatile int* abort_flag = &abort_flag_s;
@@ -335,6 +353,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       mbar_init(acc_empty_bar(b), C::EPI_WARPS);
     }
     mbar_init(drain_bar, 1);
+    mbar_init(hp_empty_bar, C::EPI_WARPS);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -375,6 +394,18 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           bulk_load(st + A_BYTES + C::B_BYTES + SFA_BYTES + h * 2048,
                     sfb_src + ((size_t)h * p.sf_tiles_b * 512) + (size_t)kt * 2048, 2048, full_bar(s), leader);
       }
+      if (BN == 128) {
+        // OutControl: the BF16 outlier channels of both operands, 64 per stage, into the same stage buffers
+        for (int32_t h = 0; h < p.hp_k_tiles && ok; ++h, ++it) {
+          const int s = it % C::STAGES;
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, abort_flag, p.dev_status));
+          if (!ok) break;
+          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+          mbar_expect_tx(full_bar(s), A_BYTES + C::B_BYTES, leader);
+          tma_load_2d(st, &tmAh, h * 64, mt * BM, full_bar(s), leader);
+          tma_load_2d(st + A_BYTES, &tmBh, h * 64, nt * BN, full_bar(s), leader);
+        }
+      }
     }
     if (!ok) {
       // give the copies already in flight a bounded time to land before the CTA may exit
@@ -404,7 +435,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (!ok) break;
         tc_fence_after();
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
-        const uint32_t sf_tmem = tmem_base + C::ACC_BUFS * C::ACC_COLS + (it & 3) * C::SF_COLS;
+        const uint32_t sf_tmem = tmem_base + sf_tmem_col + (it & 3) * C::SF_COLS;
         // Scales of this k tile: shared memory -> tensor memory. Per 64-wide k step: 4 columns for the 128 rows
         // of A, 4 per 128 rows of B.
 #pragma unroll
@@ -420,6 +451,27 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           tc_mma_nvf4(d_tmem, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc, sf_tmem + kk * 4,
                       sf_tmem + 16 + kk * (BN / 128) * 4, (kt | kk) != 0, leader);
         tc_commit(empty_bar(s), leader);  // stage reusable once these MMAs have read it
+      }
+      if (BN == 128 && p.hp_k_tiles > 0 && ok) {
+        // high-precision side product into its own accumulator (single buffer: wait until the previous tile's epilogue
+        // has drained it, which happened a whole main loop ago)
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(hp_empty_bar, (tile_it & 1) ^ 1, abort_flag, p.dev_status));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t idesc_bf16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        for (int32_t h = 0; h < p.hp_k_tiles; ++h, ++it) {
+          const int s = it % C::STAGES;
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / C::STAGES) & 1, abort_flag, p.dev_status));
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)  // 64 BF16 = one 128-byte swizzle row = four K = 16 steps of 32 bytes
+            tc_mma_bf16(tmem_base + hp_tmem_col, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc_bf16,
+                        (h | kk) != 0, leader);
+          tc_commit(empty_bar(s), leader);
+        }
+        if (!ok) break;
       }
       if (ok) tc_commit(acc_full_bar(ab), leader);
     }
@@ -492,6 +544,12 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               if (GS == kGsRow) sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
               o[j] = __uint_as_float(v[j]) * sc;
             }
+            if (hp_cols) {
+              tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + hp_tmem_col + c0, v);
+              tc_wait_ld();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) o[j] += __uint_as_float(v[j]);
+            }
             if ((p.addend || p.accumulate) && m < p.M) {
               if (n0 + 32 <= p.N) {
                 add_existing<32>(p, m, n0, o);
@@ -544,6 +602,16 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               o[j] = __uint_as_float(v[j]) * sc;
               o[32 + j] = __uint_as_float(v2[j]) * sc2;
             }
+            if (hp_cols) {
+              tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + hp_tmem_col + c0, v);
+              tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + hp_tmem_col + c0 + 32, v2);
+              tc_wait_ld();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                o[j] += __uint_as_float(v[j]);
+                o[32 + j] += __uint_as_float(v2[j]);
+              }
+            }
             if ((p.addend || p.accumulate) && m < p.M) {
               if (n0 + 64 <= p.N) {
                 add_existing<64>(p, m, n0, o);
@@ -584,8 +652,9 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       } else {
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t v[32];
+        uint32_t v[32], vh[32];
         tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + c0, v);
+        if (hp_cols) tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + hp_tmem_col + c0, vh);  // warp-uniform condition
         tc_wait_ld();
         const int64_t n0 = (int64_t)nt * BN + c0;
         if (m < p.M && n0 < p.N) {
@@ -596,13 +665,20 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (GS == kGsRow) sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
             o[j] = __uint_as_float(v[j]) * sc;
           }
+          if (hp_cols) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] += __uint_as_float(vh[j]);
+          }
           store_row_chunk(p, m, n0, o);
         }
       }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty_bar(ab));
+      if (lane == 0) {
+        mbar_arrive(acc_empty_bar(ab));
+        if (hp_cols) mbar_arrive(hp_empty_bar);
+      }
     }
     if (C::TMA_STORE && lane == 0) bulk_wait_all();  // this lane's bulk stores are complete before the CTA may exit
   }
@@ -1101,6 +1177,19 @@ bool make_c_map(CUtensorMap* tm, void* Cp, int64_t M, int64_t N, int64_t ldc, bo
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A compact BF16 side matrix [R, Kh] (Kh a multiple of 64) as a 2-D tensor; box = 64 columns (128 bytes) x 128 rows.
+bool make_hp_map(CUtensorMap* tm, const void* base, int64_t R, int64_t Kh) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)Kh, (cuuint64_t)R};
+  const cuuint64_t strides[1] = {(cuuint64_t)Kh * 2};
+  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int sm_count() {
   static int n = 0;
   if (!n) {
@@ -1120,8 +1209,13 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
     return cudaErrorInvalidValue;
   const bool tma_store = C::TMA_STORE && make_c_map(&tmC, a.C, a.M, a.N, a.ldc, a.c_is_f32 != 0);
   if (!tma_store) tmC = tmA;  // unused by the kernel then
+  CUtensorMap tmAh = tmA, tmBh = tmB;  // placeholders unless the high-precision side product is requested
   Params p{};
   p.use_tma_store = tma_store ? 1 : 0;
+  if (a.hp_Kh > 0) {
+    if (BN != 128 || !make_hp_map(&tmAh, a.hp_a, a.M, a.hp_Kh) || !make_hp_map(&tmBh, a.hp_b, a.N, a.hp_Kh)) return cudaErrorInvalidValue;
+    p.hp_k_tiles = (int32_t)(a.hp_Kh / 64);
+  }
   p.a_sf = a.a_sf;
   p.b_sf = a.b_sf;
   p.a_gscale = a.a_gscale;
@@ -1151,7 +1245,7 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
   }
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
-  launch_kernel(gemm_nvfp4_kernel<GS, BN>, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, tmA, tmB, tmC, p);
+  launch_kernel(gemm_nvfp4_kernel<GS, BN>, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, tmA, tmB, tmC, tmAh, tmBh, p);
   return cudaGetLastError();
 }
 
@@ -1261,6 +1355,8 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   const char* pair_env = getenv("NVFP4_GEMM_2CTA");
   const bool pairs = pair_env ? atoi(pair_env) != 0
                               : (a.K >= 2048 && ((a.M + 255) / 256) * ((a.N + 255) / 256) >= 2 * (sm_count() / 2));
+  if (a.hp_Kh > 0 && a.gs_mode != kGsBlock128)  // the fused high-precision side product lives in the 128 x 128 variant
+    return a.gs_mode == kGsTensor ? launch_variant<kGsTensor, 128>(a, st) : launch_variant<kGsRow, 128>(a, st);
   if (pairs && a.gs_mode == kGsTensor) return launch_2cta<kGsTensor>(a, st);
   if (pairs && a.gs_mode == kGsRow) return launch_2cta<kGsRow>(a, st);
   switch (a.gs_mode) {

@@ -99,6 +99,11 @@ struct GemmArgs {
   int accumulate;
   const float* addend;  // optional FP32 [M, N] added in the epilogue (leading dimension ld_add)
   int64_t ld_add;
+  // optional high-precision side product (OutControl): C += hp_a [M, hp_Kh] * hp_b [N, hp_Kh]^T, BF16 inputs, FP32
+  // accumulation on the tensor cores inside the same kernel (TENSOR / ROW modes)
+  const void* hp_a;
+  const void* hp_b;
+  int64_t hp_Kh;
   int32_t* dev_status;
   void* workspace;
   size_t ws_bytes;
