@@ -528,7 +528,7 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
   HpDwArgs h{};
   h.dY = static_cast<const uint16_t*>(dY); h.X_out = static_cast<const uint16_t*>(saved->X_out);
   h.lddy = lddy; h.Kh = Kh; h.T = N_tok; h.C = C; h.n_out = n_out; h.outl = cfg->outlier_cols;
-  h.dW = dW; h.dw_is_f32 = dw_f32; h.lddw = lddw; h.partial = hp_partial;
+  h.dW = dW; h.dw_is_f32 = dw_f32; h.lddw = lddw; h.partial = hp_partial; h.dev_status = cfg->dev_status;
   return launch_hp_dw(h, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 

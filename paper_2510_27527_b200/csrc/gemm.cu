@@ -1130,6 +1130,124 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   }
 }
 
+// =========================================================================================================
+// OutControl's high-precision weight-gradient columns (paper Sec. 4.2):  dW[:, A] = dY^T X[:, A], BF16 inputs, FP32
+// accumulation, on the tensor cores (tcgen05 kind::f16).  G[c, j] = sum_t dY[t, c] * X_out[t, j]  with
+// M = C, N = Kh (the compact outlier matrix, <= 256 columns), K = tokens. Both operands are stored with the
+// contraction index t as the SLOW index, i.e. "MN-major": a bulk-tensor box of 64 columns x 64 tokens lands in
+// shared memory as 64 rows of 128 bytes (8 swizzle atoms of 8 tokens), which is the MN-major 128-byte-swizzle
+// operand layout (leading byte offset = distance between 64-column boxes, stride byte offset = 1024).
+// Only C / 128 output tiles exist, so the token range is split over blockIdx.y; FP32 partial tiles go to a workspace
+// that hp_dw_reduce_kernel sums in a fixed order. One tile per CTA: no accumulator double buffering needed.
+// =========================================================================================================
+constexpr int HPDW_STAGES = 4;
+constexpr int HPDW_THREADS = 192;
+
+__global__ void __launch_bounds__(HPDW_THREADS, 1)
+hp_dw_mma_kernel(const __grid_constant__ CUtensorMap tmDY, const __grid_constant__ CUtensorMap tmXO, float* __restrict__ partial,
+                 int64_t C, int32_t Kh, int64_t T, int32_t t_per_split, int32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t b_bytes = (uint32_t)(Kh / 64) * 8192u;
+  const uint32_t stage_bytes = A_BYTES + b_bytes;  // A: two boxes of 64 channels x 64 tokens; B: Kh / 64 boxes
+  const uint32_t bar_base = smem_base + HPDW_STAGES * stage_bytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (HPDW_STAGES + s); };
+  const uint32_t acc_full_bar = bar_base + 8u * (2 * HPDW_STAGES);
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t tmem_cols = Kh <= 64 ? 64u : (Kh <= 128 ? 128u : 256u);
+
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    for (int s = 0; s < HPDW_STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    mbar_init(acc_full_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  pdl_prologue();
+
+  const int32_t c0 = (int32_t)blockIdx.x * 128;
+  const int64_t t_begin = (int64_t)blockIdx.y * t_per_split;
+  const int64_t t_end = min(T, t_begin + t_per_split);
+  const int32_t k_tiles = (int32_t)((t_end - t_begin + 63) / 64);  // tokens beyond T read as zero
+
+  if (warp == 0) {
+    const uint32_t leader = elect_leader();
+    for (int32_t kt = 0; kt < k_tiles; ++kt) {
+      const int s = kt % HPDW_STAGES;
+      if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((kt / HPDW_STAGES) & 1) ^ 1, abort_flag, dev_status))) break;
+      const uint32_t st = smem_base + s * stage_bytes;
+      const int32_t t0 = (int32_t)(t_begin + (int64_t)kt * 64);
+      mbar_expect_tx(full_bar(s), stage_bytes, leader);
+      tma_load_2d(st, &tmDY, c0, t0, full_bar(s), leader);
+      tma_load_2d(st + 8192, &tmDY, c0 + 64, t0, full_bar(s), leader);
+      for (int32_t h = 0; h < Kh / 64; ++h) tma_load_2d(st + A_BYTES + h * 8192, &tmXO, h * 64, t0, full_bar(s), leader);
+    }
+  } else if (warp == 1) {
+    const uint32_t leader = elect_leader();
+    // BF16 x BF16 -> FP32, M = 128, N = Kh, both operands MN-major
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(Kh >> 3) << 17) |
+                           ((uint32_t)(128 >> 4) << 24);
+    bool ok = true;
+    for (int32_t kt = 0; kt < k_tiles && ok; ++kt) {
+      const int s = kt % HPDW_STAGES;
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (kt / HPDW_STAGES) & 1, abort_flag, dev_status));
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t st = smem_base + s * stage_bytes;
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {  // 16 tokens = two 8-token swizzle atoms = 2048 bytes per step
+        const uint64_t adesc = (uint64_t)(((st + kk * 2048) >> 4) & 0x3FFFu) | ((uint64_t)(8192 >> 4) << 16) |
+                               ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+        const uint64_t bdesc = (uint64_t)(((st + A_BYTES + kk * 2048) >> 4) & 0x3FFFu) | ((uint64_t)(8192 >> 4) << 16) |
+                               ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+        tc_mma_bf16(tmem_base, adesc, bdesc, idesc, (kt | kk) != 0, leader);
+      }
+      tc_commit(empty_bar(s), leader);
+    }
+    tc_commit(acc_full_bar, leader);  // also covers the k_tiles == 0 case (arrives at once)
+  } else {
+    const int quad = warp & 3;
+    if (mbar_wait(acc_full_bar, 0, abort_flag, dev_status)) {
+      tc_fence_after();
+      const int64_t c = (int64_t)c0 + quad * 32 + lane;
+      float* dst = partial + ((int64_t)blockIdx.y * C + (c < C ? c : 0)) * Kh;
+      for (int j0 = 0; j0 < Kh; j0 += 32) {
+        uint32_t v[32];
+        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + j0, v);
+        tc_wait_ld();
+        if (c < C) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4)
+            *reinterpret_cast<float4*>(dst + j0 + j) = k_tiles > 0 ? make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                                                 __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]))
+                                                                   : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------------------
@@ -1340,7 +1458,41 @@ cudaError_t launch_block128(const GemmArgs& a, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// BF16 matrix [T, W] (leading dimension ld elements) as a 2-D tensor; box = 64 columns x 64 rows, 128-byte swizzle.
+bool make_tokens_map(CUtensorMap* tm, const void* base, int64_t T, int64_t W, int64_t ld) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)W, (cuuint64_t)T};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+  const cuuint32_t box[2] = {64, 64};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
+
+bool hp_dw_mma_supported(int64_t Kh) { return Kh >= 64 && Kh <= 256 && Kh % 64 == 0; }
+
+// partial[(split * C + c) * Kh + j] = sum over the split's tokens of dY[t, c] * X_out[t, j]
+cudaError_t launch_hp_dw_mma(const uint16_t* dY, int64_t lddy, const uint16_t* X_out, int64_t Kh, int64_t T, int64_t C,
+                             float* partial, int n_split, int64_t t_per_split, int32_t* dev_status, cudaStream_t st) {
+  CUtensorMap tmDY, tmXO;
+  if (!make_tokens_map(&tmDY, dY, T, C, lddy) || !make_tokens_map(&tmXO, X_out, T, Kh, Kh)) return cudaErrorInvalidValue;
+  const uint32_t stage_bytes = A_BYTES + (uint32_t)(Kh / 64) * 8192u;
+  const size_t smem = (size_t)HPDW_STAGES * stage_bytes + 1024 + 256;
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaError_t e = cudaFuncSetAttribute(hp_dw_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = smem;
+  }
+  const dim3 grid((unsigned)((C + 127) / 128), (unsigned)n_split);
+  launch_kernel(hp_dw_mma_kernel, dim3(grid), dim3(HPDW_THREADS), smem, st, tmDY, tmXO, partial, C, (int32_t)Kh, T, (int32_t)t_per_split,
+                dev_status);
+  return cudaGetLastError();
+}
 
 size_t gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
 int64_t gemm_block128_max_k() { return (int64_t)B128_MAX_CHUNKS * 128; }

@@ -188,9 +188,14 @@ cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st) {
   if (a.C == 0 || a.n_out == 0) return cudaSuccess;
   const int64_t t_per_split = ((a.T + kHpDwSplit - 1) / kHpDwSplit + 63) / 64 * 64;
   const int n_split = (int)((a.T + t_per_split - 1) / t_per_split);
-  const dim3 grid((unsigned)((a.C + 63) / 64), (unsigned)n_split);
-  launch_kernel(hp_dw_partial_kernel, dim3(grid), dim3(256), 0, st, a, t_per_split);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e;
+  if (hp_dw_mma_supported(a.Kh) && (a.lddy & 7) == 0) {  // tensor-core path (the CUDA-core kernel covers odd shapes)
+    e = launch_hp_dw_mma(a.dY, a.lddy, a.X_out, a.Kh, a.T, a.C, a.partial, n_split, t_per_split, a.dev_status, st);
+  } else {
+    const dim3 grid((unsigned)((a.C + 63) / 64), (unsigned)n_split);
+    launch_kernel(hp_dw_partial_kernel, dim3(grid), dim3(256), 0, st, a, t_per_split);
+    e = cudaGetLastError();
+  }
   if (e != cudaSuccess) return e;
   const int64_t total = a.C * a.n_out;
   launch_kernel(hp_dw_reduce_kernel, dim3((unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8)), dim3(256), 0, st, a, n_split);

@@ -134,8 +134,12 @@ struct HpDwArgs {
   int dw_is_f32;
   int64_t lddw;
   float* partial;  // workspace: hp_dw_partial_floats(T, C, Kh) floats
+  int32_t* dev_status;
 };
 size_t hp_dw_partial_floats(int64_t T, int64_t C, int64_t Kh);
+bool hp_dw_mma_supported(int64_t Kh);
+cudaError_t launch_hp_dw_mma(const uint16_t* dY, int64_t lddy, const uint16_t* X_out, int64_t Kh, int64_t T, int64_t C,
+                             float* partial, int n_split, int64_t t_per_split, int32_t* dev_status, cudaStream_t st);
 cudaError_t launch_hp_fwd(const HpFwdArgs& a, cudaStream_t st);
 cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st);
 
