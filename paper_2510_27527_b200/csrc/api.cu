@@ -89,7 +89,8 @@ bool carve_operand(Carver& c, nvfp4_operand* o, int64_t R, int64_t K, int32_t gs
 
 nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, int32_t rounding,
                               uint64_t seed, uint32_t stream_id, const int32_t* keep, int64_t n_keep,
-                              const nvfp4_operand* out, uint32_t* cells, cudaStream_t st, int cells_zeroed = 0) {
+                              const nvfp4_operand* out, uint32_t* cells, cudaStream_t st, int cells_zeroed = 0,
+                              const int32_t* excluded = nullptr) {
   if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   QuantRowsArgs a{};
   a.src = src;
@@ -98,6 +99,7 @@ nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, i
   a.cols_src = cols;
   a.ld = ld;
   a.keep = keep;
+  a.excluded = keep ? excluded : nullptr;
   a.seed = seed;
   a.stream_id = stream_id;
   a.gs_mode = out->gs_mode;
@@ -366,9 +368,11 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
   const uint16_t* Wp = static_cast<const uint16_t*>(W);
   const int32_t* keep = n_out > 0 ? cfg->keep_cols : nullptr;
   if (!zero_cells(cells_x, cells_w, cells_bytes(C, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
-  if ((s = do_quantize_rows(Xp, N_tok, D, ldx, cfg->rounding[0], cfg->seed, 1, keep, Dk, &saved->qx, cells_x, st, 1)) != NVFP4_OK)
+  if ((s = do_quantize_rows(Xp, N_tok, D, ldx, cfg->rounding[0], cfg->seed, 1, keep, Dk, &saved->qx, cells_x, st, 1,
+                            cfg->outlier_cols)) != NVFP4_OK)
     return s;
-  if ((s = do_quantize_rows(Wp, C, D, ldw, cfg->rounding[1], cfg->seed, 2, keep, Dk, &saved->qw, cells_w, st, 1)) != NVFP4_OK)
+  if ((s = do_quantize_rows(Wp, C, D, ldw, cfg->rounding[1], cfg->seed, 2, keep, Dk, &saved->qw, cells_w, st, 1,
+                            cfg->outlier_cols)) != NVFP4_OK)
     return s;
   if (n_out > 0) {
     if (!saved->X_out || !saved->W_out) return NVFP4_ERR_NULL;
@@ -522,6 +526,7 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
   if ((s = do_quantize_transpose(t6, 1, N_tok, Dk, cfg->rounding[5], cfg->seed, 6, &q6, cells6, st, 1)) != NVFP4_OK) return s;
   if (n_out == 0) return do_gemm(&q5, &q6, dW, cfg->dw_dtype, lddw, 0, nullptr, 0, cfg->dev_status, st);
 
+  // kept columns: compact product, then a column scatter (a scattering GEMM epilogue measured slower than this pair)
   if ((s = do_gemm(&q5, &q6, compact, NVFP4_DT_F32, ld_compact, 0, nullptr, 0, cfg->dev_status, st)) != NVFP4_OK) return s;
   if (launch_scatter_cols(compact, ld_compact, 1, dW, lddw, dw_f32, C, Dk, cfg->keep_cols, st) != cudaSuccess)
     return NVFP4_ERR_CUDA;

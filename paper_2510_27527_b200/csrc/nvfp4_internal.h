@@ -14,6 +14,7 @@ struct QuantRowsArgs {
   const uint16_t* src;  // BF16 [rows, cols_src], leading dimension ld
   int64_t rows, K, cols_src, ld;
   const int32_t* keep;  // optional column list of length K
+  const int32_t* excluded;  // optional: the sorted complement of `keep` (cols_src - K entries); enables the masked amax
   uint64_t seed;
   uint32_t stream_id;
   int gs_mode, sr, sf_tiled;

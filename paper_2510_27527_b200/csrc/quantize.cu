@@ -60,6 +60,53 @@ __global__ void __launch_bounds__(256) amax_tensor_bf16_kernel(const uint16_t* _
   }
 }
 
+// amax of a BF16 matrix over all columns EXCEPT a sorted list of excluded ones (OutControl: the outlier channels do not
+// take part in the FP4 operand's tensor scale). Each CTA builds a one-bit-per-column mask in shared memory from the
+// list, then streams whole rows with 16-byte loads, zeroing the excluded lanes. Folded into cells[0] by atomic max.
+__global__ void __launch_bounds__(256) amax_tensor_masked_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols,
+                                                                int64_t ld, const int32_t* __restrict__ excluded, int64_t n_excl,
+                                                                uint32_t* amax_bits) {
+  pdl_prologue();
+  extern __shared__ uint32_t keep_bits[];  // bit c = 1: column c takes part
+  const int64_t words = (cols + 31) >> 5;
+  for (int64_t i = threadIdx.x; i < words; i += 256) keep_bits[i] = 0xFFFFFFFFu;
+  __syncthreads();
+  for (int64_t i = threadIdx.x; i < n_excl; i += 256) atomicAnd(&keep_bits[excluded[i] >> 5], ~(1u << (excluded[i] & 31)));
+  __syncthreads();
+  const int64_t chunks = (cols + 7) >> 3;
+  uint32_t m = 0;
+  for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+    const uint16_t* p = src + r * ld;
+    for (int64_t c = threadIdx.x; c < chunks; c += 256) {
+      const uint32_t mask8 = (keep_bits[c >> 2] >> ((c & 3) * 8)) & 0xFFu;
+      uint32_t w[4] = {0, 0, 0, 0};
+      if ((c << 3) + 8 <= cols) {
+        const uint4 v = *reinterpret_cast<const uint4*>(p + (c << 3));
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+      } else {
+        for (int q = 0; q < 8; ++q)
+          if ((c << 3) + q < cols) w[q >> 1] |= (uint32_t)p[(c << 3) + q] << (16 * (q & 1));
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint32_t two = (mask8 >> (2 * q)) & 3u;
+        const uint32_t lanes = ((0u - (two & 1u)) & 0x0000FFFFu) | ((0u - (two >> 1)) & 0xFFFF0000u);
+        m = umax16x2(m, bf16x2_abs_bits(w[q]) & lanes);
+      }
+    }
+  }
+  uint32_t a = hmax_of_pair(m);
+#pragma unroll
+  for (int o = 16; o; o >>= 1) a = max(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
+  __shared__ uint32_t warp_max[8];
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = a;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) a = max(a, warp_max[w]);
+    if (a) atomicMax(amax_bits, a << 16);
+  }
+}
+
 // amax of each source row over the kept columns -> cells[row] (ROW scale mode of the row-axis quantizer).
 __global__ void __launch_bounds__(256) amax_rows_bf16_kernel(const uint16_t* __restrict__ src, int64_t rows,
                                                             int64_t cols, int64_t ld,
@@ -574,6 +621,15 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
   if (a.gs_mode == kGsTensor) {
     if (a.compute_amax) {
       if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
+      if (a.keep && a.excluded && (a.ld & 7) == 0 && a.cols_src <= 256 * 1024) {
+        // amax over the kept columns only: full-width vector loads with the excluded (outlier) columns masked out
+        const size_t smem = (size_t)((a.cols_src + 31) >> 5) * 4;
+        const unsigned grid = (unsigned)std::min<int64_t>(a.rows, 148 * 8);
+        launch_kernel(amax_tensor_masked_kernel, dim3(grid), dim3(256), smem, st, a.src, a.rows, a.cols_src, a.ld, a.excluded,
+                      a.cols_src - a.K, a.gs_cells);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        return launch_rows_r<kGsTensor>(a, st);
+      }
       if (a.keep) {  // amax over the kept columns only: one row per CTA, one atomic per row
         launch_kernel(amax_rows_bf16_kernel, dim3((unsigned)a.rows), dim3(256), 0, st, a.src, a.rows, a.cols_src, a.ld, a.keep, a.K, a.gs_cells, 1);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
