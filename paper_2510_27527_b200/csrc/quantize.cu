@@ -195,20 +195,21 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
     const int64_t last = min(first + 256 * NB, total) - 1;
     stage_row0 = first / nb;
     const int64_t n_rows = last / nb - stage_row0 + 1;
-    const int64_t chunks_per_row = stage_cols8 >> 3;
-    for (int64_t e = threadIdx.x; e < n_rows * chunks_per_row; e += 256) {
-      const int64_t rr = e / chunks_per_row, ch = (e - rr * chunks_per_row) << 3;
+    const uint32_t chunks_per_row = (uint32_t)(stage_cols8 >> 3);
+    const uint32_t n_chunks = (uint32_t)n_rows * chunks_per_row;
+    for (uint32_t e = threadIdx.x; e < n_chunks; e += 256) {
+      const uint32_t rr = e / chunks_per_row, ch = (e - rr * chunks_per_row) << 3;
       uint4 v = make_uint4(0, 0, 0, 0);
       const uint16_t* p = src + (stage_row0 + rr) * ld + ch;
-      if (ch + 8 <= cols_src) {
+      if ((int64_t)ch + 8 <= cols_src) {
         v = *reinterpret_cast<const uint4*>(p);
       } else {
         uint32_t t[4] = {0, 0, 0, 0};
         for (int q = 0; q < 8; ++q)
-          if (ch + q < cols_src) t[q >> 1] |= (uint32_t)p[q] << (16 * (q & 1));
+          if ((int64_t)ch + q < cols_src) t[q >> 1] |= (uint32_t)p[q] << (16 * (q & 1));
         v = make_uint4(t[0], t[1], t[2], t[3]);
       }
-      *reinterpret_cast<uint4*>(row_stage + rr * stage_cols8 + ch) = v;
+      *reinterpret_cast<uint4*>(row_stage + (size_t)rr * stage_cols8 + ch) = v;
     }
     __syncthreads();
   }
