@@ -25,6 +25,9 @@
  *   - Random bits: Philox4x32-10, key = seed, counter = (idx / 8, stream_id, 0), idx = row * K16 + k.
  *   - An all-zero outer group takes Sg = 1; a block whose scale rounds to 0 gets all-zero magnitudes.
  *
+ *   - Sec. 4.1 (Random Hadamard Transformation): A' = A S H with a block-diagonal Hadamard matrix of block size 16
+ *     and a random sign diagonal S, applied along the contraction axis to both operands of the two backward products.
+ *
  * Every function is pinned by tests that do not re-use its own formula (exhaustive format tables, hand-derived
  * golden blocks, Philox known-answer vectors, brute-force nearest-value search, unbiasedness statistics,
  * transposition/scaling/sign symmetries, brute-force triple-loop products).
@@ -274,6 +277,47 @@ void orc_rematerialize_f32(const uint8_t *codes, const uint8_t *sf, const float 
             const int code = (codes[(r * K16 + k) / 2] >> (4 * (k & 1))) & 15;
             const float ps = (float)(orc_e2m1_value(code) * orc_e4m3_value(sf[r * nb + k / 16]));
             out[r * K16 + k] = ps * gscale_at(gscale, gs_mode, r, k, ng);
+        }
+}
+
+/* ---------------------------------------------------------------------------------------------------------
+ * Random Hadamard transformation (Sec. 4.1), block size 16, along k:  out[r, 16g .. 16g+15] = (x[r, 16g ..] * s) H_16.
+ *   - H_16 is the orthonormal Sylvester matrix H_2 (x) H_2 (x) H_2 (x) H_2, entries +-1/4; it is symmetric.
+ *   - s_k = -1 iff bit (k % 128) of the Philox4x32-10 block with counter (k / 128, 0, stream_id, 0x5348) and key = seed
+ *     is set (word (k % 128) / 32, bit k % 32). The sign depends on k only: both operands of a product see the same S.
+ *   - Readings (the paper fixes only the mathematics): float32 arithmetic, the four butterfly stages in the order
+ *     h = 1, 2, 4, 8, each replacing (a, b) = (v[i], v[i + h]) for the i with (i & h) == 0 by (a + b, a - b), then one
+ *     multiplication by 0.25f. K is zero-extended to K16; the result has K16 columns.
+ * ------------------------------------------------------------------------------------------------------- */
+int orc_rht_sign_bit(uint64_t seed, uint32_t stream_id, uint64_t k) {
+    uint64_t g = k / 128;
+    uint32_t b = (uint32_t)(k % 128);
+    uint32_t ctr[4] = {(uint32_t)g, (uint32_t)(g >> 32), stream_id, 0x5348u};
+    uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+    uint32_t w[4];
+    orc_philox4x32_10(ctr, key, w);
+    return (int)((w[b / 32] >> (b % 32)) & 1u);
+}
+
+void orc_rht16(const float *x, int64_t R, int64_t K, uint64_t seed, uint32_t stream_id, float *out) {
+    const int64_t K16 = round_up(K, 16);
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < R; ++r)
+        for (int64_t k0 = 0; k0 < K16; k0 += 16) {
+            float v[16];
+            for (int i = 0; i < 16; ++i) {
+                const int64_t k = k0 + i;
+                const float xv = (k < K) ? x[r * K + k] : 0.0f;
+                v[i] = orc_rht_sign_bit(seed, stream_id, (uint64_t)k) ? -xv : xv;
+            }
+            for (int h = 1; h < 16; h <<= 1)
+                for (int i = 0; i < 16; ++i)
+                    if ((i & h) == 0) {
+                        const float a = v[i], b = v[i + h];
+                        v[i] = a + b;
+                        v[i + h] = a - b;
+                    }
+            for (int i = 0; i < 16; ++i) out[r * K16 + k0 + i] = v[i] * 0.25f;
         }
 }
 

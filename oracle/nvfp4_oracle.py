@@ -65,6 +65,10 @@ def lib():
         L.orc_dequantize.argtypes = [vp, vp, vp, c_i64, c_i64, c_int, vp]
         L.orc_rematerialize_f32.restype = None
         L.orc_rematerialize_f32.argtypes = [vp, vp, vp, c_i64, c_i64, c_int, vp]
+        L.orc_rht_sign_bit.restype = c_int
+        L.orc_rht_sign_bit.argtypes = [c_u64, c_u32, c_u64]
+        L.orc_rht16.restype = None
+        L.orc_rht16.argtypes = [vp, c_i64, c_i64, c_u64, c_u32, vp]
         L.orc_gemm_tn_f64.restype = None
         L.orc_gemm_tn_f64.argtypes = [vp, vp, c_i64, c_i64, c_i64, vp]
         L.orc_gemm_tn_f64_samples.restype = None
@@ -170,6 +174,21 @@ def rematerialize_f32(op: Operand) -> np.ndarray:
     return np.ascontiguousarray(out[:, : op.K])
 
 
+def rht_sign_bit(seed: int, stream_id: int, k: int) -> int:
+    return lib().orc_rht_sign_bit(int(seed), int(stream_id), int(k))
+
+
+def rht16(x: np.ndarray, seed: int, stream_id: int) -> np.ndarray:
+    """Random Hadamard transformation along k (Sec. 4.1, block size 16): (x * s) H_16 per 16 consecutive k.
+    Returns float32 [R, K16]."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    R, K = x.shape
+    K16 = (K + 15) // 16 * 16
+    out = np.zeros((R, K16), dtype=np.float32)
+    lib().orc_rht16(_p(x), R, K, seed, stream_id, _p(out))
+    return out
+
+
 def gemm_tn(A: np.ndarray, B: np.ndarray) -> np.ndarray:
     """C[m, n] = sum_k A[m, k] B[n, k] in float64."""
     A = np.ascontiguousarray(A, dtype=np.float64)
@@ -204,6 +223,7 @@ def gemm_operands(a: Operand, b: Operand) -> np.ndarray:
 # the linear layer (Sec. 2.3) with the optional OutControl split (Sec. 4.2, without the Hadamard factors)
 # ------------------------------------------------------------------------------------------------------------
 STREAM_Q3, STREAM_Q4, STREAM_Q5, STREAM_Q6 = 3, 4, 5, 6
+STREAM_RHT_DX, STREAM_RHT_DW = 7, 8  # sign diagonals S_C (dX product) and S_N (dW product)
 
 
 @dataclass
@@ -213,6 +233,7 @@ class LayerConfig:
     # rounding of Q1..Q6; the paper's assignment is deterministic in forward, stochastic in backward
     rounding: tuple = (RTN, RTN, SR, SR, SR, SR)
     outliers: np.ndarray | None = None  # sorted channel indices of the set A (columns of X / W), or None
+    rht: bool = False  # random Hadamard transformation of both operands of the two backward products (Sec. 4.1)
 
 
 @dataclass
@@ -266,8 +287,11 @@ def linear_bwd_dx(dY: np.ndarray, saved: Saved, cfg: LayerConfig) -> np.ndarray:
     """dX = Q3_S(dY) Q4_S(W-hat): one FP4 product over all D columns. dY [N_tok, C] -> dX [N_tok, D]."""
     dY = np.asarray(dY, dtype=np.float32)
     W_hat = aligned_full(saved.qw, saved.keep, saved.outl, saved.W_out, saved.D)  # [C, D]
-    q3 = quantize(dY, AXIS_ROW, cfg.rounding[2], cfg.gs_mode, cfg.seed, STREAM_Q3)  # [N_tok, C]
-    q4 = quantize(W_hat, AXIS_COL, cfg.rounding[3], cfg.gs_mode, cfg.seed, STREAM_Q4)  # [D, C]
+    A, B = dY, np.ascontiguousarray(W_hat.T)  # [N_tok, C], [D, C]: both along the contraction axis C
+    if cfg.rht:
+        A, B = rht16(A, cfg.seed, STREAM_RHT_DX), rht16(B, cfg.seed, STREAM_RHT_DX)
+    q3 = quantize(A, AXIS_ROW, cfg.rounding[2], cfg.gs_mode, cfg.seed, STREAM_Q3)
+    q4 = quantize(B, AXIS_ROW, cfg.rounding[3], cfg.gs_mode, cfg.seed, STREAM_Q4)
     return gemm_operands(q3, q4)
 
 
@@ -276,8 +300,11 @@ def linear_bwd_dw(dY: np.ndarray, saved: Saved, cfg: LayerConfig) -> np.ndarray:
     dY = np.asarray(dY, dtype=np.float32)
     C = dY.shape[1]
     X_hat_keep = rematerialize_f32(saved.qx)  # [N_tok, Dk]
-    q5 = quantize(dY, AXIS_COL, cfg.rounding[4], cfg.gs_mode, cfg.seed, STREAM_Q5)  # [C, N_tok]
-    q6 = quantize(X_hat_keep, AXIS_COL, cfg.rounding[5], cfg.gs_mode, cfg.seed, STREAM_Q6)  # [Dk, N_tok]
+    A, B = np.ascontiguousarray(dY.T), np.ascontiguousarray(X_hat_keep.T)  # [C, N_tok], [Dk, N_tok]: along tokens
+    if cfg.rht:
+        A, B = rht16(A, cfg.seed, STREAM_RHT_DW), rht16(B, cfg.seed, STREAM_RHT_DW)
+    q5 = quantize(A, AXIS_ROW, cfg.rounding[4], cfg.gs_mode, cfg.seed, STREAM_Q5)
+    q6 = quantize(B, AXIS_ROW, cfg.rounding[5], cfg.gs_mode, cfg.seed, STREAM_Q6)
     dW = np.zeros((C, saved.D), dtype=np.float64)
     dW[:, saved.keep] = gemm_operands(q5, q6)
     if len(saved.outl):
