@@ -111,7 +111,7 @@ class ClockSampler:
 # ---------------------------------------------------------------------------------------------------------------
 # the oracle arm (CPU): used for --impl reference and for the cpu_baseline leg of the default arm
 # ---------------------------------------------------------------------------------------------------------------
-def oracle_sample_step(workload: str, gs_mode: int, sample_tokens: int = 256):
+def oracle_sample_step(workload: str, gs_mode: int, sample_tokens: int = 256, rht: bool = False):
     """One forward + dX + dW of the workload's first linear on a slab of `sample_tokens` tokens, through the
     oracle as it stands. Returns (seconds, flops of the sample, description)."""
     from oracle import nvfp4_oracle as orc
@@ -123,7 +123,7 @@ def oracle_sample_step(workload: str, gs_mode: int, sample_tokens: int = 256):
                                      grad_scale=c["grad_scale"], swiglu=swiglu)
     orc.lib()
     t0 = time.perf_counter()
-    ocfg = orc.LayerConfig(gs_mode=gs_mode, seed=0)
+    ocfg = orc.LayerConfig(gs_mode=gs_mode, seed=0, rht=rht)
     _, saved = orc.linear_fwd(X, W, ocfg)
     orc.linear_bwd_dx(dY, saved, ocfg)
     orc.linear_bwd_dw(dY, saved, ocfg)
@@ -140,10 +140,10 @@ def run_reference(args):
     gs_mode = GS[args.gs]
     cfg_id, tokens, linears = WORKLOADS[args.workload]
     for _ in range(min(args.warmup, 1)):
-        oracle_sample_step(args.workload, gs_mode, 64)
+        oracle_sample_step(args.workload, gs_mode, 64, args.rht)
     times, fl, desc = [], 0.0, ""
     for _ in range(args.steps):
-        dt, fl, desc = oracle_sample_step(args.workload, gs_mode, args.ref_tokens)
+        dt, fl, desc = oracle_sample_step(args.workload, gs_mode, args.ref_tokens, args.rht)
         times.append(dt)
     t = float(np.mean(times))
     val = fl / t / 1e12
@@ -206,7 +206,7 @@ def run_ours(args):
             L.W.append(b.upload_bf16(synth.weights(C, D, synth.seed_of(cfg_id, 100 * extra + li)), dev))
         n_out = int(round(args.outliers * D))
         outl = synth.outlier_channels(D, n_out, synth.seed_of(cfg_id, 50 + li)) if n_out else None
-        L.cfg = b.LayerConfig(gs_mode=gs_mode, seed=0, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32, outliers=outl)
+        L.cfg = b.LayerConfig(gs_mode=gs_mode, seed=0, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32, outliers=outl, rht=args.rht)
         L.cfg.prepare(D, dev)
         L.saved = b.alloc_saved(L.X, L.W[0], L.cfg)
         L.Y = torch.empty((tokens, C), dtype=torch.bfloat16, device=dev)
@@ -369,7 +369,7 @@ def run_ours(args):
     if world == 1 and not args.no_cpu:
         from oracle import nvfp4_oracle as orc
 
-        dt, sfl, desc = oracle_sample_step(args.workload, gs_mode, args.cpu_tokens)
+        dt, sfl, desc = oracle_sample_step(args.workload, gs_mode, args.cpu_tokens, args.rht)
         cpu = {"value": sfl / dt / 1e12, "unit": "TFLOP/s", "cores": orc.threads(), "kind": "oracle", "sample": desc,
                "seconds": dt}
 
@@ -377,7 +377,7 @@ def run_ours(args):
         "metric": "nvfp4_linear_fwd_bwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "fp4(e2m1)xfp4 with ue4m3 block scales, f32 accumulate", "data": "synthetic",
-        "config": {"workload": workload_name(args), "gs_mode": args.gs, "outcontrol_fraction": args.outliers, "l2": "256 MiB write + 256 MiB read flush before every timed step",
+        "config": {"workload": workload_name(args), "gs_mode": args.gs, "outcontrol_fraction": args.outliers, "rht": bool(args.rht), "l2": "256 MiB write + 256 MiB read flush before every timed step",
                    "timing": "CUDA events per step on the launch stream, summed"},
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
@@ -478,6 +478,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--outliers", type=float, default=0.0,
                     help="OutControl: fraction of input channels kept in BF16 (0 = off; the paper uses 0.10)")
+    ap.add_argument("--rht", action="store_true", help="random Hadamard transformation (block 16) in the four backward quantizers")
     ap.add_argument("--no-breakdown", action="store_true", help="only warm-up + timed steps (used for ncu launch lists)")
     ap.add_argument("--sweep", action="store_true", help="roofline sweep of the large GEMM shapes instead of the step benchmark")
     ap.add_argument("--shapes", default="", help="with --sweep: comma list of MxNxK")

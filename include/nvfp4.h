@@ -98,9 +98,17 @@ long long nvfp4_launch_count(void);
  *   rounding RTN: nearest E2M1 value, ties to the even code. SR: 16 random bits u per element from
  *            Philox4x32-10 (key = seed, counter = (idx / 8, stream_id, 0), idx = r * Kp16 + k in the OPERAND,
  *            Kp16 = K rounded up to 16); the magnitude rounds up iff (u + 0.5) / 65536 < (a - q1) / (q2 - q1).
+ *   rht_stream_id  0: off. Otherwise the random Hadamard transformation of Sec. 4.1 is applied along the operand's K before
+ *            anything else: each aligned block of 16 consecutive k (zero-extended at the end of K) becomes (x S) H_16,
+ *            H_16 the orthonormal Sylvester matrix (entries +-1/4), S the sign diagonal with s_k = -1 iff bit (k % 128)
+ *            of the Philox block with counter (k / 128, 0, rht_stream_id, 0x5348) and key = seed is set. Binary32:
+ *            v_i = x_i * (s_i / 4), then the butterfly stages h = 1, 2, 4, 8, each (a, b) -> (a + b, a - b). Scales and
+ *            codes are those of the transformed matrix, whose columns K .. K16-1 are in general non-zero. Two operands
+ *            transformed with the same seed and stream multiply to the product of the untransformed ones (up to
+ *            rounding). Not combined with keep_cols (NVFP4_ERR_ENUM).
  *   keep_cols optional sorted list (device, int32) of the n_keep source columns that are kept; the others
- *            (OutControl's outlier channels) are skipped and the kept ones are compacted. ROW axis: compacts K.
- *            COL axis: compacts the operand rows. NULL keeps all columns (n_keep is ignored).
+ *            (OutControl's outlier channels) are skipped and the kept ones are compacted along K. ROW axis only
+ *            (NVFP4_ERR_SHAPE otherwise). NULL keeps all columns (n_keep is ignored).
  *   out      operand to fill; out->R / out->K must equal the shape stated above.
  *   workspace at least nvfp4_quantize_workspace_bytes(out->R, gs_mode); holds the amax cells of the TENSOR
  *            and ROW modes.
@@ -111,9 +119,9 @@ long long nvfp4_launch_count(void);
  * --------------------------------------------------------------------------------------------------------- */
 size_t nvfp4_quantize_workspace_bytes(int64_t out_rows, int32_t gs_mode);
 nvfp4_status nvfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld, int32_t axis,
-                            int32_t rounding, uint64_t seed, uint32_t stream_id, const int32_t* keep_cols,
-                            int64_t n_keep, const nvfp4_operand* out, void* workspace, size_t ws_bytes,
-                            void* stream);
+                            int32_t rounding, uint64_t seed, uint32_t stream_id, uint32_t rht_stream_id,
+                            const int32_t* keep_cols, int64_t n_keep, const nvfp4_operand* out, void* workspace,
+                            size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------
  * nvfp4_quantize_static — nvfp4_quantize without a workspace argument. (The paper has no counterpart: this is a
@@ -148,12 +156,13 @@ nvfp4_status nvfp4_quantize_static(const void* src_bf16, int64_t rows, int64_t c
  *            row_map[d] >= 0, and column d of the BF16 matrix hp_bf16 [R, >= n_rows_out] (leading dimension
  *            hp_ld) when row_map[d] < 0 — OutControl's W-hat, whose outlier columns come from W itself
  *            (Sec. 4.2). NULL: identity map, hp_bf16 unused.
- *   rounding, seed, stream_id, workspace: as in nvfp4_quantize.
+ *   rounding, seed, stream_id, rht_stream_id, workspace: as in nvfp4_quantize (the transformation runs along the
+ *            output operand's K, i.e. along the rows of `in`).
  * --------------------------------------------------------------------------------------------------------- */
 nvfp4_status nvfp4_requantize_t(const nvfp4_operand* in, const void* hp_bf16, int64_t hp_ld,
                                 const int32_t* row_map, int64_t n_rows_out, int32_t rounding, uint64_t seed,
-                                uint32_t stream_id, const nvfp4_operand* out, void* workspace, size_t ws_bytes,
-                                void* stream);
+                                uint32_t stream_id, uint32_t rht_stream_id, const nvfp4_operand* out,
+                                void* workspace, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------
  * nvfp4_gemm — block-scaled FP4 product of two operands (the "FP4 MM" of Sec. 2.3):
@@ -187,6 +196,9 @@ typedef struct {
   const int32_t* keep_cols;    /* [D - n_out]  sorted complement                                             */
   const int32_t* col_map;      /* [D]          position of channel d in keep_cols, or -1 for an outlier      */
   int32_t* dev_status;         /* optional, see nvfp4_gemm                                                   */
+  /* Random Hadamard transformation of both operands of the two backward products (Sec. 4.1): 0 off, 1 on.
+   * Q3 and Q4 use sign stream 7 along C, Q5 and Q6 sign stream 8 along the tokens; forward is never transformed. */
+  int32_t rht;
 } nvfp4_layer_cfg;
 
 /* What forward leaves for backward. qx [N_tok, D - n_out] and qw [C, D - n_out] are filled by
@@ -216,12 +228,14 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
                               int64_t C, const nvfp4_layer_cfg* cfg, void* Y, int64_t ldy, nvfp4_saved* saved,
                               void* workspace, size_t ws_bytes, void* stream);
 
-/* dX = Q3(dY) Q4(W-hat): one FP4 product over all D channels; W-hat's outlier columns are W's. */
+/* dX = Q3(dY S H) Q4(H^T S^T W-hat): one FP4 product over all D channels; W-hat's outlier columns are W's.
+ * (S H is the identity unless cfg->rht is set.) */
 nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved* saved,
                                  const nvfp4_layer_cfg* cfg, void* dX, int64_t lddx, void* workspace,
                                  size_t ws_bytes, void* stream);
 
-/* dW[:, keep] = Q5(dY^T) Q6(X-hat[:, keep]);  dW[:, outl] = dY^T X[:, outl] (BF16 inputs, FP32 accumulate). */
+/* dW[:, keep] = Q5(dY^T S H) Q6(H^T S^T X-hat[:, keep]);  dW[:, outl] = dY^T X[:, outl] (BF16 inputs, FP32 accumulate,
+ * never transformed). */
 nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved* saved,
                                  const nvfp4_layer_cfg* cfg, void* dW, int64_t lddw, void* workspace,
                                  size_t ws_bytes, void* stream);

@@ -285,9 +285,9 @@ void orc_rematerialize_f32(const uint8_t *codes, const uint8_t *sf, const float 
  *   - H_16 is the orthonormal Sylvester matrix H_2 (x) H_2 (x) H_2 (x) H_2, entries +-1/4; it is symmetric.
  *   - s_k = -1 iff bit (k % 128) of the Philox4x32-10 block with counter (k / 128, 0, stream_id, 0x5348) and key = seed
  *     is set (word (k % 128) / 32, bit k % 32). The sign depends on k only: both operands of a product see the same S.
- *   - Readings (the paper fixes only the mathematics): float32 arithmetic, the four butterfly stages in the order
- *     h = 1, 2, 4, 8, each replacing (a, b) = (v[i], v[i + h]) for the i with (i & h) == 0 by (a + b, a - b), then one
- *     multiplication by 0.25f. K is zero-extended to K16; the result has K16 columns.
+ *   - Readings (the paper fixes only the mathematics): float32 arithmetic; v[i] = x[i] * (s_i / 4) first (exact: a
+ *     power of two), then the four butterfly stages in the order h = 1, 2, 4, 8, each replacing (a, b) = (v[i], v[i + h])
+ *     for the i with (i & h) == 0 by (a + b, a - b). K is zero-extended to K16; the result has K16 columns.
  * ------------------------------------------------------------------------------------------------------- */
 int orc_rht_sign_bit(uint64_t seed, uint32_t stream_id, uint64_t k) {
     uint64_t g = k / 128;
@@ -308,7 +308,7 @@ void orc_rht16(const float *x, int64_t R, int64_t K, uint64_t seed, uint32_t str
             for (int i = 0; i < 16; ++i) {
                 const int64_t k = k0 + i;
                 const float xv = (k < K) ? x[r * K + k] : 0.0f;
-                v[i] = orc_rht_sign_bit(seed, stream_id, (uint64_t)k) ? -xv : xv;
+                v[i] = xv * (orc_rht_sign_bit(seed, stream_id, (uint64_t)k) ? -0.25f : 0.25f);
             }
             for (int h = 1; h < 16; h <<= 1)
                 for (int i = 0; i < 16; ++i)
@@ -317,7 +317,7 @@ void orc_rht16(const float *x, int64_t R, int64_t K, uint64_t seed, uint32_t str
                         v[i] = a + b;
                         v[i + h] = a - b;
                     }
-            for (int i = 0; i < 16; ++i) out[r * K16 + k0 + i] = v[i] * 0.25f;
+            for (int i = 0; i < 16; ++i) out[r * K16 + k0 + i] = v[i];
         }
 }
 

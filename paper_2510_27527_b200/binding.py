@@ -41,7 +41,7 @@ class COperand(ctypes.Structure):
 class CLayerCfg(ctypes.Structure):
     _fields_ = [("gs_mode", c_i32), ("rounding", c_i32 * 6), ("seed", c_u64), ("y_dtype", c_i32), ("dx_dtype", c_i32),
                 ("dw_dtype", c_i32), ("n_out", c_i64), ("outlier_cols", c_vp), ("keep_cols", c_vp), ("col_map", c_vp),
-                ("dev_status", c_vp)]
+                ("dev_status", c_vp), ("rht", c_i32)]
 
 
 class CSaved(ctypes.Structure):
@@ -58,12 +58,12 @@ EXPORTS = {
     "nvfp4_status_string": (ctypes.c_char_p, [c_i32]),
     "nvfp4_launch_count": (ctypes.c_longlong, []),
     "nvfp4_quantize_workspace_bytes": (c_sz, [c_i64, c_i32]),
-    "nvfp4_quantize": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_u64, c_u32, c_vp, c_i64,
+    "nvfp4_quantize": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_u64, c_u32, c_u32, c_vp, c_i64,
                                ctypes.POINTER(COperand), c_vp, c_sz, c_vp]),
     "nvfp4_quantize_static_max_rows": (c_i64, []),
     "nvfp4_quantize_static": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_u64, c_u32, c_vp, c_i64,
                                       ctypes.POINTER(COperand), c_vp]),
-    "nvfp4_requantize_t": (c_i32, [ctypes.POINTER(COperand), c_vp, c_i64, c_vp, c_i64, c_i32, c_u64, c_u32,
+    "nvfp4_requantize_t": (c_i32, [ctypes.POINTER(COperand), c_vp, c_i64, c_vp, c_i64, c_i32, c_u64, c_u32, c_u32,
                                    ctypes.POINTER(COperand), c_vp, c_sz, c_vp]),
     "nvfp4_gemm_workspace_bytes": (c_sz, [c_i64, c_i64, c_i64]),
     "nvfp4_gemm": (c_i32, [ctypes.POINTER(COperand), ctypes.POINTER(COperand), c_vp, c_i32, c_i64, c_i32, c_vp, c_vp,
@@ -169,7 +169,7 @@ def _workspace(nbytes: int, device="cuda") -> torch.Tensor:
 # ------------------------------------------------------------------------------------------------------------
 def nvfp4_quantize(src: torch.Tensor, axis: int = AXIS_ROW, rounding: int = ROUND_RTN, seed: int = 0, stream_id: int = 0,
                    gs_mode: int = GS_TENSOR, sf_layout: int = SF_TILED128x4, keep_cols: torch.Tensor | None = None,
-                   out: Operand | None = None, workspace: torch.Tensor | None = None) -> Operand:
+                   out: Operand | None = None, workspace: torch.Tensor | None = None, rht_stream_id: int = 0) -> Operand:
     assert src.dtype == torch.bfloat16 and src.dim() == 2 and src.stride(1) == 1
     rows, cols = src.shape
     kept = cols if keep_cols is None else int(keep_cols.numel())
@@ -178,8 +178,8 @@ def nvfp4_quantize(src: torch.Tensor, axis: int = AXIS_ROW, rounding: int = ROUN
         out = alloc_operand(R, K, gs_mode, sf_layout, src.device)
     ws = workspace if workspace is not None else _workspace(_lib.nvfp4_quantize_workspace_bytes(R, gs_mode), src.device)
     co = out.c()
-    _check(_lib.nvfp4_quantize(_ptr(src), rows, cols, src.stride(0), axis, rounding, seed, stream_id, _ptr(keep_cols), kept,
-                               ctypes.byref(co), _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_quantize")
+    _check(_lib.nvfp4_quantize(_ptr(src), rows, cols, src.stride(0), axis, rounding, seed, stream_id, rht_stream_id,
+                               _ptr(keep_cols), kept, ctypes.byref(co), _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_quantize")
     return out
 
 
@@ -202,7 +202,7 @@ def nvfp4_quantize_static(src: torch.Tensor, axis: int = AXIS_ROW, rounding: int
 
 def nvfp4_requantize_t(inp: Operand, rounding: int = ROUND_SR, seed: int = 0, stream_id: int = 0, gs_mode: int | None = None,
                        sf_layout: int = SF_TILED128x4, hp: torch.Tensor | None = None, row_map: torch.Tensor | None = None,
-                       out: Operand | None = None, workspace: torch.Tensor | None = None) -> Operand:
+                       out: Operand | None = None, workspace: torch.Tensor | None = None, rht_stream_id: int = 0) -> Operand:
     gs_mode = inp.gs_mode if gs_mode is None else gs_mode
     D = inp.K if row_map is None else int(row_map.numel())
     if out is None:
@@ -210,7 +210,7 @@ def nvfp4_requantize_t(inp: Operand, rounding: int = ROUND_SR, seed: int = 0, st
     ws = workspace if workspace is not None else _workspace(_lib.nvfp4_quantize_workspace_bytes(D, gs_mode), inp.codes.device)
     ci, co = inp.c(), out.c()
     _check(_lib.nvfp4_requantize_t(ctypes.byref(ci), _ptr(hp), 0 if hp is None else hp.stride(0), _ptr(row_map), D, rounding,
-                                   seed, stream_id, ctypes.byref(co), _ptr(ws), ws.numel(), _stream_ptr()),
+                                   seed, stream_id, rht_stream_id, ctypes.byref(co), _ptr(ws), ws.numel(), _stream_ptr()),
            "nvfp4_requantize_t")
     return out
 
@@ -236,6 +236,7 @@ class LayerConfig:
     dw_dtype: int = DT_F32
     outliers: np.ndarray | None = None  # sorted outlier channel indices (host)
     dev_status: torch.Tensor | None = None
+    rht: bool = False  # random Hadamard transformation of both operands of the two backward products
     # device index arrays, built by prepare()
     _outl: torch.Tensor | None = None
     _keep: torch.Tensor | None = None
@@ -263,7 +264,7 @@ class LayerConfig:
 
     def c(self) -> CLayerCfg:
         return CLayerCfg(self.gs_mode, (c_i32 * 6)(*self.rounding), self.seed, self.y_dtype, self.dx_dtype, self.dw_dtype,
-                         self.n_out, _ptr(self._outl), _ptr(self._keep), _ptr(self._map), _ptr(self.dev_status))
+                         self.n_out, _ptr(self._outl), _ptr(self._keep), _ptr(self._map), _ptr(self.dev_status), int(self.rht))
 
 
 @dataclass

@@ -14,6 +14,9 @@ long long g_launch_count = 0;
 
 namespace {
 
+// Philox stream ids of the two sign diagonals of the backward products (the six quantizers use 1..6)
+constexpr uint32_t kRhtStreamDx = 7, kRhtStreamDw = 8;
+
 inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -90,7 +93,7 @@ bool carve_operand(Carver& c, nvfp4_operand* o, int64_t R, int64_t K, int32_t gs
 nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, int32_t rounding,
                               uint64_t seed, uint32_t stream_id, const int32_t* keep, int64_t n_keep,
                               const nvfp4_operand* out, uint32_t* cells, cudaStream_t st, int cells_zeroed = 0,
-                              const int32_t* excluded = nullptr) {
+                              const int32_t* excluded = nullptr, uint32_t rht_stream = 0) {
   if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   QuantRowsArgs a{};
   a.src = src;
@@ -102,6 +105,7 @@ nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, i
   a.excluded = keep ? excluded : nullptr;
   a.seed = seed;
   a.stream_id = stream_id;
+  a.rht_stream = rht_stream;
   a.gs_mode = out->gs_mode;
   a.sr = rounding == NVFP4_ROUND_SR;
   a.sf_tiled = out->sf_layout == NVFP4_SF_TILED128x4;
@@ -116,7 +120,7 @@ nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, i
 
 nvfp4_status do_quantize_transpose(const TransposeSrc& src, int from_codes, int64_t rowsK, int64_t D, int32_t rounding,
                                    uint64_t seed, uint32_t stream_id, const nvfp4_operand* out, uint32_t* cells,
-                                   cudaStream_t st, int cells_zeroed = 0) {
+                                   cudaStream_t st, int cells_zeroed = 0, uint32_t rht_stream = 0) {
   if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   QuantTransposeArgs a{};
   a.from_codes = from_codes;
@@ -125,6 +129,7 @@ nvfp4_status do_quantize_transpose(const TransposeSrc& src, int from_codes, int6
   a.src = src;
   a.seed = seed;
   a.stream_id = stream_id;
+  a.rht_stream = rht_stream;
   a.gs_mode = out->gs_mode;
   a.sr = rounding == NVFP4_ROUND_SR;
   a.sf_tiled = out->sf_layout == NVFP4_SF_TILED128x4;
@@ -178,7 +183,7 @@ nvfp4_status check_cfg(const nvfp4_layer_cfg* cfg, int64_t D) {
   for (int i = 0; i < 6; ++i)
     if (cfg->rounding[i] < 0 || cfg->rounding[i] > 1) return NVFP4_ERR_ENUM;
   if (cfg->y_dtype < 0 || cfg->y_dtype > 1 || cfg->dx_dtype < 0 || cfg->dx_dtype > 1 || cfg->dw_dtype < 0 ||
-      cfg->dw_dtype > 1)
+      cfg->dw_dtype > 1 || cfg->rht < 0 || cfg->rht > 1)
     return NVFP4_ERR_ENUM;
   if (cfg->n_out < 0 || cfg->n_out > D) return NVFP4_ERR_SHAPE;
   if (cfg->n_out > 0 && (!cfg->outlier_cols || !cfg->keep_cols || !cfg->col_map)) return NVFP4_ERR_NULL;
@@ -234,11 +239,12 @@ size_t nvfp4_quantize_workspace_bytes(int64_t out_rows, int32_t gs_mode) {
 }
 
 nvfp4_status nvfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld, int32_t axis,
-                            int32_t rounding, uint64_t seed, uint32_t stream_id, const int32_t* keep_cols,
-                            int64_t n_keep, const nvfp4_operand* out, void* workspace, size_t ws_bytes,
-                            void* stream) {
+                            int32_t rounding, uint64_t seed, uint32_t stream_id, uint32_t rht_stream_id,
+                            const int32_t* keep_cols, int64_t n_keep, const nvfp4_operand* out, void* workspace,
+                            size_t ws_bytes, void* stream) {
   if (!src_bf16 || !out) return NVFP4_ERR_NULL;
   if (axis < 0 || axis > 1 || rounding < 0 || rounding > 1) return NVFP4_ERR_ENUM;
+  if (rht_stream_id && keep_cols) return NVFP4_ERR_ENUM;
   if (rows < 0 || cols < 0 || (keep_cols && (n_keep < 0 || n_keep > cols))) return NVFP4_ERR_SHAPE;
   if (keep_cols && axis != NVFP4_AXIS_ROW) return NVFP4_ERR_SHAPE;
   nvfp4_status s = check_operand_ptrs(out);
@@ -255,16 +261,17 @@ nvfp4_status nvfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, in
   uint32_t* cells = static_cast<uint32_t*>(workspace);
   if (axis == NVFP4_AXIS_ROW)
     return do_quantize_rows(static_cast<const uint16_t*>(src_bf16), rows, cols, ld, rounding, seed, stream_id, keep_cols,
-                            n_keep, out, cells, st);
+                            n_keep, out, cells, st, 0, nullptr, rht_stream_id);
   TransposeSrc ts{};
   ts.bf16 = static_cast<const uint16_t*>(src_bf16);
   ts.ld = ld;
-  return do_quantize_transpose(ts, 0, rows, cols, rounding, seed, stream_id, out, cells, st);
+  return do_quantize_transpose(ts, 0, rows, cols, rounding, seed, stream_id, out, cells, st, 0, rht_stream_id);
 }
 
 nvfp4_status nvfp4_requantize_t(const nvfp4_operand* in, const void* hp_bf16, int64_t hp_ld, const int32_t* row_map,
                                 int64_t n_rows_out, int32_t rounding, uint64_t seed, uint32_t stream_id,
-                                const nvfp4_operand* out, void* workspace, size_t ws_bytes, void* stream) {
+                                uint32_t rht_stream_id, const nvfp4_operand* out, void* workspace, size_t ws_bytes,
+                                void* stream) {
   if (!in || !out) return NVFP4_ERR_NULL;
   if (rounding < 0 || rounding > 1) return NVFP4_ERR_ENUM;
   nvfp4_status s;
@@ -288,7 +295,7 @@ nvfp4_status nvfp4_requantize_t(const nvfp4_operand* in, const void* hp_bf16, in
   ts.hp = static_cast<const uint16_t*>(hp_bf16);
   ts.hp_ld = hp_ld;
   return do_quantize_transpose(ts, 1, in->R, D, rounding, seed, stream_id, out, static_cast<uint32_t*>(workspace),
-                               static_cast<cudaStream_t>(stream));
+                               static_cast<cudaStream_t>(stream), 0, rht_stream_id);
 }
 
 size_t nvfp4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) { return gemm_workspace_bytes(M, N, K); }
@@ -418,8 +425,9 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
   if (!carve_operand(cv, &q3, N_tok, C, cfg->gs_mode) || !carve_operand(cv, &q4, D, C, cfg->gs_mode) || !cells3 || !cells4)
     return NVFP4_ERR_WORKSPACE;
   if (!zero_cells(cells3, cells4, cells_bytes(D, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
+  const uint32_t rht = cfg->rht ? kRhtStreamDx : 0u;
   if ((s = do_quantize_rows(static_cast<const uint16_t*>(dY), N_tok, C, lddy, cfg->rounding[2], cfg->seed, 3, nullptr, 0,
-                            &q3, cells3, st, 1)) != NVFP4_OK)
+                            &q3, cells3, st, 1, nullptr, rht)) != NVFP4_OK)
     return s;
   TransposeSrc ts{};
   ts.in_codes = saved->qw.codes;
@@ -429,7 +437,7 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
   ts.in_gs_mode = saved->qw.gs_mode;
   ts.in_sf_tiled = saved->qw.sf_layout == NVFP4_SF_TILED128x4;
   if (n_out == 0) {
-    if ((s = do_quantize_transpose(ts, 1, C, D, cfg->rounding[3], cfg->seed, 4, &q4, cells4, st, 1)) != NVFP4_OK) return s;
+    if ((s = do_quantize_transpose(ts, 1, C, D, cfg->rounding[3], cfg->seed, 4, &q4, cells4, st, 1, rht)) != NVFP4_OK) return s;
   } else {
     // W-hat^T over all D channels in two passes that write disjoint operand rows: the kept channels from the forward
     // operand (compact column j -> row keep[j]) and the outlier channels from the compact BF16 copy (column j -> row
@@ -438,7 +446,8 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
     if (!saved->W_out) return NVFP4_ERR_NULL;
     const int64_t Kh = nvfp4_outlier_pad(n_out);
     if (clear_sf_padding(&q4, st) != cudaSuccess) return NVFP4_ERR_CUDA;
-    const bool closed = cfg->gs_mode == NVFP4_GS_TENSOR && saved->qw.gs_mode == NVFP4_GS_TENSOR;
+    // (the closed form does not survive the Hadamard transformation: both sources then get a transformed amax pass)
+    const bool closed = cfg->gs_mode == NVFP4_GS_TENSOR && saved->qw.gs_mode == NVFP4_GS_TENSOR && !rht;
     TransposeSrc th{};
     th.bf16 = static_cast<const uint16_t*>(saved->W_out);
     th.ld = Kh;
@@ -447,6 +456,7 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
     QuantTransposeArgs qa{};
     qa.seed = cfg->seed;
     qa.stream_id = 4;
+    qa.rht_stream = rht;
     qa.gs_mode = cfg->gs_mode;
     qa.sr = cfg->rounding[3] == NVFP4_ROUND_SR;
     qa.sf_tiled = 1;
@@ -458,11 +468,15 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
     qa.rowsK = C;
     if (cfg->gs_mode == NVFP4_GS_TENSOR) {
       // one amax pass over the compact BF16 copy (and over the forward operand unless the closed form applies)
-      if (launch_amax_tensor(static_cast<const uint16_t*>(saved->W_out), C, Kh, Kh, cells4, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+      if (rht) {
+        if (launch_amax_transpose_src(th, 0, C, n_out, cells4, st, cfg->seed, rht) != cudaSuccess) return NVFP4_ERR_CUDA;
+      } else if (launch_amax_tensor(static_cast<const uint16_t*>(saved->W_out), C, Kh, Kh, cells4, st) != cudaSuccess) {
+        return NVFP4_ERR_CUDA;
+      }
       if (closed) {
         th.closed_form_sg = saved->qw.gscale;
         ts.closed_form_sg = saved->qw.gscale;
-      } else if (launch_amax_transpose_src(ts, 1, C, D - n_out, cells4, st) != cudaSuccess) {
+      } else if (launch_amax_transpose_src(ts, 1, C, D - n_out, cells4, st, cfg->seed, rht) != cudaSuccess) {
         return NVFP4_ERR_CUDA;
       }
       qa.compute_amax = 0;
@@ -515,7 +529,8 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
   t5.bf16 = static_cast<const uint16_t*>(dY);
   t5.ld = lddy;
   if (!zero_cells(cells5, cells6, cells_bytes(Dk, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
-  if ((s = do_quantize_transpose(t5, 0, N_tok, C, cfg->rounding[4], cfg->seed, 5, &q5, cells5, st, 1)) != NVFP4_OK) return s;
+  const uint32_t rht = cfg->rht ? kRhtStreamDw : 0u;
+  if ((s = do_quantize_transpose(t5, 0, N_tok, C, cfg->rounding[4], cfg->seed, 5, &q5, cells5, st, 1, rht)) != NVFP4_OK) return s;
   TransposeSrc t6{};
   t6.in_codes = saved->qx.codes;
   t6.in_sf = saved->qx.sf;
@@ -523,7 +538,7 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
   t6.in_K = saved->qx.K;
   t6.in_gs_mode = saved->qx.gs_mode;
   t6.in_sf_tiled = saved->qx.sf_layout == NVFP4_SF_TILED128x4;
-  if ((s = do_quantize_transpose(t6, 1, N_tok, Dk, cfg->rounding[5], cfg->seed, 6, &q6, cells6, st, 1)) != NVFP4_OK) return s;
+  if ((s = do_quantize_transpose(t6, 1, N_tok, Dk, cfg->rounding[5], cfg->seed, 6, &q6, cells6, st, 1, rht)) != NVFP4_OK) return s;
   if (n_out == 0) return do_gemm(&q5, &q6, dW, cfg->dw_dtype, lddw, 0, nullptr, 0, cfg->dev_status, st);
 
   // kept columns: compact product, then a column scatter (a scattering GEMM epilogue measured slower than this pair)

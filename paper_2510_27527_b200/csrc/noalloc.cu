@@ -50,7 +50,7 @@ nvfp4_status nvfp4_quantize_static(const void* src_bf16, int64_t rows, int64_t c
   if (s != NVFP4_OK) return s;
   // Same validation, same kernels, same order as nvfp4_quantize; only the scratch differs. The launchers zero the
   // cells they use on `stream` before the amax pass, so the previous call's contents never leak into this one.
-  return nvfp4_quantize(src_bf16, rows, cols, ld, axis, rounding, seed, stream_id, keep_cols, n_keep, out, cells,
+  return nvfp4_quantize(src_bf16, rows, cols, ld, axis, rounding, seed, stream_id, 0u, keep_cols, n_keep, out, cells,
                         (size_t)kStaticCells * sizeof(uint32_t), stream);
 }
 

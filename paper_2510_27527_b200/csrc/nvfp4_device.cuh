@@ -104,6 +104,46 @@ __device__ __forceinline__ uint4 sr_words(uint64_t seed, uint32_t stream_id, uin
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// Random Hadamard transformation along k (paper Sec. 4.1): x' = (x S) H with H = diag(H_16, H_16, ...), the orthonormal
+// Sylvester matrix (entries +-1/4), and S a random sign diagonal that depends on k only.
+//   * sign of k: bit (k % 128) of the Philox block with counter (k / 128, 0, rht_stream, 0x5348), key = seed; set = -1;
+//   * arithmetic: v[i] = x[i] * (s_i / 4) (exact), then four butterfly stages h = 1, 2, 4, 8 in binary32.
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 rht_sign_words(uint64_t seed, uint32_t rht_stream, uint64_t group128) {
+  return philox4x32_10((uint32_t)group128, (uint32_t)(group128 >> 32), rht_stream, 0x5348u, (uint32_t)seed,
+                       (uint32_t)(seed >> 32));
+}
+__device__ __forceinline__ uint32_t rht_pick_word(const uint4& w, uint32_t q) {
+  return q == 0 ? w.x : q == 1 ? w.y : q == 2 ? w.z : w.w;
+}
+// the 16 sign bits of k0 .. k0 + 15 (k0 a multiple of 16), bit i for k0 + i
+__device__ __forceinline__ uint32_t rht_sign16(uint64_t seed, uint32_t rht_stream, int64_t k0) {
+  const uint4 w = rht_sign_words(seed, rht_stream, (uint64_t)k0 >> 7);
+  return (rht_pick_word(w, ((uint32_t)k0 >> 5) & 3u) >> ((uint32_t)k0 & 16u)) & 0xFFFFu;
+}
+// +-1/4 for position kk (0..127) of a 128-group
+__device__ __forceinline__ float rht_factor(const uint4& w, uint32_t kk) {
+  return __uint_as_float(0x3E800000u | ((rht_pick_word(w, kk >> 5) >> (kk & 31u)) << 31));
+}
+__device__ __forceinline__ void rht_scale16(float (&v)[16], uint32_t sign16) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(v[i], __uint_as_float(0x3E800000u | ((sign16 << (31 - i)) & 0x80000000u)));
+}
+__device__ __forceinline__ void hadamard16_butterflies(float (&v)[16]) {
+#pragma unroll
+  for (int h = 1; h < 16; h <<= 1) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      if ((i & h) == 0) {
+        const float a = v[i], b = v[i + h];
+        v[i] = __fadd_rn(a, b);
+        v[i + h] = __fsub_rn(a, b);
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // Element rounding to E2M1 (paper Sec. 2.1). Codes: sign << 3 | magnitude index.
 // ---------------------------------------------------------------------------------------------------------
 // Stochastic rounding. For an element with 16-bit draw u the rule is

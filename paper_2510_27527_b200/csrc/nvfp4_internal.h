@@ -17,6 +17,7 @@ struct QuantRowsArgs {
   const int32_t* excluded;  // optional: the sorted complement of `keep` (cols_src - K entries); enables the masked amax
   uint64_t seed;
   uint32_t stream_id;
+  uint32_t rht_stream;  // non-zero: random Hadamard transformation along K with this sign stream (not with `keep`)
   int gs_mode, sr, sf_tiled;
   int compute_amax;    // TENSOR mode: run the amax pre-pass (0: gs_cells[0] already holds the amax bits)
   int cells_zeroed;    // the caller has already cleared gs_cells on this stream
@@ -52,6 +53,7 @@ struct QuantTransposeArgs {
   TransposeSrc src;
   uint64_t seed;
   uint32_t stream_id;
+  uint32_t rht_stream;  // non-zero: random Hadamard transformation along the operand's K (source rows) with this stream
   int gs_mode, sr, sf_tiled;
   int compute_amax;
   int cells_zeroed;        // the caller has already cleared gs_cells on this stream
@@ -86,8 +88,10 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st);
 cudaError_t launch_quantize_transpose(const QuantTransposeArgs& a, cudaStream_t st);
 // amax of a contiguous-row BF16 matrix folded into cells[0] (atomic max; the cell must already hold a valid value)
 cudaError_t launch_amax_tensor(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, uint32_t* cell, cudaStream_t st);
-// amax of a transposing quantizer's source (from codes or BF16) folded into cells[0]
-cudaError_t launch_amax_transpose_src(const TransposeSrc& s, int from_codes, int64_t rowsK, int64_t D, uint32_t* cell, cudaStream_t st);
+// amax of a transposing quantizer's source (from codes or BF16) folded into cells[0]; with a non-zero rht_stream, of the
+// source after the random Hadamard transformation along its rows (the operand's K)
+cudaError_t launch_amax_transpose_src(const TransposeSrc& s, int from_codes, int64_t rowsK, int64_t D, uint32_t* cell, cudaStream_t st,
+                                      uint64_t seed = 0, uint32_t rht_stream = 0);
 
 struct GemmArgs {
   const uint8_t *a_codes, *a_sf, *b_codes, *b_sf;

@@ -3,6 +3,8 @@
 //   - row-axis quantize from BF16 (Q1, Q2, Q3 of Sec. 2.3): one thread per 16-element inner block;
 //   - transposing quantize (Q5 from BF16; Q4, Q6 from the forward operand's codes, i.e. from X-hat / W-hat):
 //     a 128(k) x 64(operand rows) tile is staged in shared memory as FP32 and read back column-wise.
+// With a non-zero sign stream the backward quantizers first apply the random Hadamard transformation of Sec. 4.1 to each
+// 16-element block along K (the block a thread already holds in registers), and the amax pre-passes see transformed data.
 // All of them are HBM streaming kernels; the launch wrappers at the bottom are called by the C-ABI layer.
 #include "nvfp4_device.cuh"
 #include "nvfp4_internal.h"
@@ -143,6 +145,69 @@ __global__ void __launch_bounds__(256) amax_rows_bf16_kernel(const uint16_t* __r
   }
 }
 
+// amax of the transformed matrix (x S) H along the rows' K axis: per row (ROW mode) or folded into cells[0]. One thread
+// per 16-element block; atomic max on cells that are zero before the launch.
+__global__ void __launch_bounds__(256) amax_rows_rht_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, int64_t ld,
+                                                           uint64_t seed, uint32_t rht_stream, uint32_t* cells, int per_row) {
+  pdl_prologue();
+  const int64_t nb16 = (K + 15) >> 4;
+  const int64_t total = rows * nb16;
+  float acc = 0.0f;
+  for (int64_t base = (int64_t)blockIdx.x * 256; base < total; base += (int64_t)gridDim.x * 256) {
+    const int64_t gid = base + threadIdx.x;
+    const bool active = gid < total;
+    const int64_t r = active ? gid / nb16 : -1;
+    const int64_t k0 = active ? (gid - r * nb16) << 4 : 0;
+    float x[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x[i] = 0.0f;
+    if (active) {
+      const uint16_t* p = src + r * ld + k0;
+      if (k0 + 16 <= K && (ld & 7) == 0) {
+        const uint4 v0 = *reinterpret_cast<const uint4*>(p), v1 = *reinterpret_cast<const uint4*>(p + 8);
+        const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          x[2 * i] = bf16_lo(w[i]);
+          x[2 * i + 1] = bf16_hi(w[i]);
+        }
+      } else {
+        for (int i = 0; i < 16; ++i)
+          if (k0 + i < K) x[i] = bf16_bits_to_float(p[i]);
+      }
+    }
+    rht_scale16(x, rht_sign16(seed, rht_stream, k0));
+    hadamard16_butterflies(x);
+    float m = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(x[i]));
+    if (per_row) {
+      // a warp usually sits inside one row: one atomic per warp then, else one per block
+      const int64_t r0 = __shfl_sync(0xFFFFFFFFu, r, 0);
+      if (__all_sync(0xFFFFFFFFu, r == r0)) {
+#pragma unroll
+        for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+        if ((threadIdx.x & 31) == 0 && r0 >= 0 && m > 0.0f) atomicMax(cells + r0, __float_as_uint(m));
+      } else if (active && m > 0.0f) {
+        atomicMax(cells + r, __float_as_uint(m));
+      }
+    } else {
+      acc = fmaxf(acc, m);
+    }
+  }
+  if (!per_row) {
+#pragma unroll
+    for (int o = 16; o; o >>= 1) acc = fmaxf(acc, __shfl_xor_sync(0xFFFFFFFFu, acc, o));
+    __shared__ float warp_max[8];
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int w = 1; w < 8; ++w) acc = fmaxf(acc, warp_max[w]);
+      if (acc > 0.0f) atomicMax(cells, __float_as_uint(acc));
+    }
+  }
+}
+
 // =========================================================================================================
 // Shared epilogue of one 16-element inner block: scale, round, pack.
 // =========================================================================================================
@@ -171,14 +236,15 @@ __device__ __forceinline__ uint2 quantize_block16(const float (&x)[16], float rc
 //   GS      scale mode. TENSOR reads the amax cell gs_cells[0]; ROW reads gs_cells[row]; BLOCK128 reduces the
 //           group amax over the 8 threads of the group with shuffles (single pass over the data).
 //   GATHER  columns come from the list `keep` (OutControl compaction) instead of 0..cols-1.
+//   RHT     each block is replaced by (x S) H_16 before anything else looks at it (never together with GATHER).
 // =========================================================================================================
-template <int GS, bool SR, bool TILED, bool GATHER>
+template <int GS, bool SR, bool TILED, bool GATHER, bool RHT>
 __global__ void __launch_bounds__(256)
 quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, int64_t ld,
                      const int32_t* __restrict__ keep, uint64_t seed, uint32_t stream_id,
                      const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
                      float* __restrict__ gscale, uint32_t div_mul, uint32_t div_shift, int wide_loads, int64_t cols_src,
-                     int64_t stage_cols8) {
+                     int64_t stage_cols8, uint32_t rht_stream) {
   pdl_prologue();
   constexpr int NB = 4;  // inner blocks per thread; all loads are issued before any arithmetic
   extern __shared__ uint16_t row_stage[];  // GATHER only: the source rows this CTA touches, [n_rows][cols_src8]
@@ -284,10 +350,27 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
     const int64_t r = active ? row[j] : 0;
     const int64_t b = blk[j];
     const int64_t k0 = b << 4;
-    uint32_t m2 = 0;
+    float x[16];
+    uint32_t amax_b_bits;  // binary32 pattern of the block's amax (non-negative, so integer order = float order)
+    if (RHT) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) m2 = umax16x2(m2, bf16x2_abs_bits(w[j][i]));
-    const uint32_t amax_b_bits = hmax_of_pair(m2);
+      for (int i = 0; i < 8; ++i) {
+        x[2 * i] = bf16_lo(w[j][i]);
+        x[2 * i + 1] = bf16_hi(w[j][i]);
+      }
+      // blocks past K (layout padding up to 128) take no signs, so that they stay +0 and encode as zero bytes
+      rht_scale16(x, k0 < K ? rht_sign16(seed, rht_stream, k0) : 0u);
+      hadamard16_butterflies(x);
+      float m = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(x[i]));
+      amax_b_bits = __float_as_uint(m);
+    } else {
+      uint32_t m2 = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) m2 = umax16x2(m2, bf16x2_abs_bits(w[j][i]));
+      amax_b_bits = hmax_of_pair(m2) << 16;
+    }
 
     // ---- global scale -------------------------------------------------------------------------------------
     float Sg;
@@ -296,7 +379,7 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
       g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
       g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
       g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 4));
-      Sg = global_scale_from_amax(bf16_bits_to_float(g));
+      Sg = global_scale_from_amax(__uint_as_float(g));
       if (active && (b & 7) == 0) gscale[r * (Kp >> 7) + (b >> 3)] = Sg;
     } else if (GS == kGsRow) {
       Sg = global_scale_from_amax(__uint_as_float(gs_cells[r]));
@@ -307,12 +390,13 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
 
     // ---- block scale, rounding, packing -------------------------------------------------------------------
     float rcp;
-    const uint32_t sb = block_scale(bf16_bits_to_float(amax_b_bits), Sg, rcp);
-    float x[16];
+    const uint32_t sb = block_scale(__uint_as_float(amax_b_bits), Sg, rcp);
+    if (!RHT) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      x[2 * i] = bf16_lo(w[j][i]);
-      x[2 * i + 1] = bf16_hi(w[j][i]);
+      for (int i = 0; i < 8; ++i) {
+        x[2 * i] = bf16_lo(w[j][i]);
+        x[2 * i + 1] = bf16_hi(w[j][i]);
+      }
     }
     const uint2 packed = quantize_block16<SR>(x, rcp, seed, stream_id, (uint64_t)((r * K16 + k0) >> 3));
 
@@ -425,11 +509,15 @@ __device__ __forceinline__ void decode8(uint32_t word, uint32_t sf_byte, float s
   }
 }
 
-template <int SRC, int GS, bool SR, bool TILED>
+//   RHT        the 16-blocks along k are replaced by (x S) H_16: the sign and the 1/4 are applied while staging (one
+//              factor per source row), the butterflies on the 16 values a thread reads back.
+//   AMAX_ONLY  stop after the block maxima and fold them into the amax cells (pre-pass for TENSOR / ROW under RHT;
+//              gs_cells is then written, and codes / sf / gscale are not touched).
+template <int SRC, int GS, bool SR, bool TILED, bool RHT, bool AMAX_ONLY>
 __global__ void __launch_bounds__(256)
 quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t seed, uint32_t stream_id,
-                          const uint32_t* __restrict__ gs_cells, int tensor_closed_form, uint8_t* __restrict__ codes,
-                          uint8_t* __restrict__ sf, float* __restrict__ gscale) {
+                          uint32_t* __restrict__ gs_cells, int tensor_closed_form, uint8_t* __restrict__ codes,
+                          uint8_t* __restrict__ sf, float* __restrict__ gscale, uint32_t rht_stream) {
   pdl_prologue();
   __shared__ float tile[128][65];
   __shared__ float blk_amax[8][64];
@@ -440,6 +528,19 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
   const int64_t k_base = (int64_t)blockIdx.x * 128;
   const int64_t d_base = (int64_t)blockIdx.y * 64;
   const int tid = threadIdx.x;
+  uint4 sw = make_uint4(0, 0, 0, 0);  // the tile's 128 sign bits (k_base is a multiple of 128)
+  if (RHT) {
+    sw = rht_sign_words(seed, rht_stream, (uint64_t)blockIdx.x);
+    // rows past K rounded up to 16 are layout padding: no signs there, so that they stay +0 and encode as zero bytes
+    const int64_t live = ((rowsK + 15) & ~(int64_t)15) - k_base;
+    if (live < 128) {
+      const uint32_t n = live > 0 ? (uint32_t)live : 0u;
+      sw.x &= n >= 32 ? 0xFFFFFFFFu : (1u << n) - 1u;
+      sw.y &= n >= 64 ? 0xFFFFFFFFu : n > 32 ? (1u << (n - 32)) - 1u : 0u;
+      sw.z &= n >= 96 ? 0xFFFFFFFFu : n > 64 ? (1u << (n - 64)) - 1u : 0u;
+      sw.w &= n > 96 ? (1u << (n - 96)) - 1u : 0u;
+    }
+  }
 
   // ---- phase 1: stage (zero outside the matrix) ------------------------------------------------------------
   if (SRC == 0 && d_base + 64 <= D && (s.ld & 7) == 0) {
@@ -448,10 +549,14 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
       const int kr = c >> 3, dc = (c & 7) << 3;
       uint4 v = make_uint4(0, 0, 0, 0);
       if (k_base + kr < rowsK) v = *reinterpret_cast<const uint4*>(s.bf16 + (k_base + kr) * s.ld + d_base + dc);
-      tile[kr][dc + 0] = bf16_lo(v.x); tile[kr][dc + 1] = bf16_hi(v.x);
-      tile[kr][dc + 2] = bf16_lo(v.y); tile[kr][dc + 3] = bf16_hi(v.y);
-      tile[kr][dc + 4] = bf16_lo(v.z); tile[kr][dc + 5] = bf16_hi(v.z);
-      tile[kr][dc + 6] = bf16_lo(v.w); tile[kr][dc + 7] = bf16_hi(v.w);
+      float f8[8] = {bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y), bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w)};
+      if (RHT) {
+        const float f = rht_factor(sw, (uint32_t)kr);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f8[i] = __fmul_rn(f8[i], f);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) tile[kr][dc + i] = f8[i];
     }
   } else if (SRC == 1 && !s.row_map && d_base + 64 <= D) {
     // forward operand without a row map: 32 codes (16 bytes) and their two scale bytes per thread
@@ -476,13 +581,20 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
 #pragma unroll
       for (int i = 0; i < 32; ++i) v[i] = 0.0f;
     }
+    if (RHT) {
+      const float f = rht_factor(sw, (uint32_t)kr);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = __fmul_rn(v[i], f);
+    }
 #pragma unroll
     for (int i = 0; i < 32; ++i) tile[kr][half * 32 + i] = v[i];
   } else {
     for (int e = tid; e < 128 * 64; e += 256) {
       const int kr = e >> 6, dl = e & 63;
       const int64_t k = k_base + kr, d = d_base + dl;
-      tile[kr][dl] = (k < rowsK && d < D) ? load_transpose_elem<SRC>(s, k, d) : 0.0f;
+      float v = (k < rowsK && d < D) ? load_transpose_elem<SRC>(s, k, d) : 0.0f;
+      if (RHT) v = __fmul_rn(v, rht_factor(sw, (uint32_t)kr));
+      tile[kr][dl] = v;
     }
   }
   __syncthreads();
@@ -497,14 +609,35 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
 #pragma unroll
   for (int it = 0; it < 2; ++it) {
     const int kb = (tid >> 6) + 4 * it;  // 0..7
+#pragma unroll
+    for (int i = 0; i < 16; ++i) xs[it][i] = tile[kb * 16 + i][dl];
+    if (RHT) hadamard16_butterflies(xs[it]);
     float m = 0.0f;
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      xs[it][i] = tile[kb * 16 + i][dl];
-      m = fmaxf(m, fabsf(xs[it][i]));
-    }
+    for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(xs[it][i]));
     am[it] = m;
     if (GS == kGsBlock128) blk_amax[kb][dl] = m;
+  }
+  if (AMAX_ONLY) {
+    float m = fmaxf(am[0], am[1]);
+    if (GS == kGsRow) {  // one cell per operand row
+      blk_amax[tid >> 6][dl] = m;
+      __syncthreads();
+      if (tid < 64 && d < D) {
+        m = fmaxf(fmaxf(blk_amax[0][dl], blk_amax[1][dl]), fmaxf(blk_amax[2][dl], blk_amax[3][dl]));
+        if (m > 0.0f) atomicMax(gs_cells + o, __float_as_uint(m));
+      }
+    } else {
+#pragma unroll
+      for (int q = 16; q; q >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, q));
+      if ((tid & 31) == 0) blk_amax[0][tid >> 5] = m;
+      __syncthreads();
+      if (tid == 0) {
+        for (int q = 1; q < 8; ++q) m = fmaxf(m, blk_amax[0][q]);
+        if (m > 0.0f) atomicMax(gs_cells, __float_as_uint(m));
+      }
+    }
+    return;
   }
   float Sg;
   if (GS == kGsBlock128) {
@@ -591,17 +724,20 @@ static cudaError_t launch_rows_g(const QuantRowsArgs& a, cudaStream_t st) {
     } else if (smem > 48 * 1024) {
       static size_t configured = 0;
       if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(quantize_rows_kernel<GS, SR, TILED, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(quantize_rows_kernel<GS, SR, TILED, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              160 * 1024);
         if (e != cudaSuccess) return e;
         configured = 160 * 1024;
       }
     }
-    launch_kernel(quantize_rows_kernel<GS, SR, TILED, true>, dim3(grid), dim3(256), smem, st, a.src, a.rows, a.K, a.ld, a.keep, a.seed,
-                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, stage_cols8);
+    launch_kernel(quantize_rows_kernel<GS, SR, TILED, true, false>, dim3(grid), dim3(256), smem, st, a.src, a.rows, a.K, a.ld, a.keep, a.seed,
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, stage_cols8, 0u);
+  } else if (a.rht_stream) {
+    launch_kernel(quantize_rows_kernel<GS, SR, TILED, false, true>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, nullptr, a.seed,
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0, a.rht_stream);
   } else {
-    launch_kernel(quantize_rows_kernel<GS, SR, TILED, false>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, nullptr, a.seed,
-                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0);
+    launch_kernel(quantize_rows_kernel<GS, SR, TILED, false, false>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, nullptr, a.seed,
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0, 0u);
   }
   return cudaGetLastError();
 }
@@ -619,6 +755,20 @@ static cudaError_t launch_rows_r(const QuantRowsArgs& a, cudaStream_t st) {
 cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
   if (a.rows == 0 || a.K == 0) return cudaSuccess;
   cudaError_t e;
+  if (a.rht_stream) {  // the scales come from the transformed data; column lists are not combined with the transformation
+    if (a.keep) return cudaErrorInvalidValue;
+    if (a.gs_mode != kGsBlock128 && (a.gs_mode == kGsRow || a.compute_amax)) {
+      const int per_row = a.gs_mode == kGsRow;
+      if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t) * (size_t)(per_row ? a.rows : 1), st)) != cudaSuccess) return e;
+      const int64_t blocks16 = a.rows * ((a.K + 15) >> 4);
+      const unsigned grid = (unsigned)std::min<int64_t>((blocks16 + 255) / 256, 148 * 16);
+      launch_kernel(amax_rows_rht_kernel, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, a.seed, a.rht_stream, a.gs_cells, per_row);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    }
+    return a.gs_mode == kGsTensor ? launch_rows_r<kGsTensor>(a, st)
+           : a.gs_mode == kGsRow  ? launch_rows_r<kGsRow>(a, st)
+                                  : launch_rows_r<kGsBlock128>(a, st);
+  }
   if (a.gs_mode == kGsTensor) {
     if (a.compute_amax) {
       if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
@@ -654,12 +804,25 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
 template <int SRC, int GS, bool SR>
 static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
   const dim3 grid(blocks_for(a.rowsK, 128), blocks_for(a.D, 64));
-  if (a.sf_tiled)
-    launch_kernel(quantize_transpose_kernel<SRC, GS, SR, true>, dim3(grid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.seed, a.stream_id, a.gs_cells,
-                                                                      a.tensor_closed_form, a.codes, a.sf, a.gscale);
-  else
-    launch_kernel(quantize_transpose_kernel<SRC, GS, SR, false>, dim3(grid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.seed, a.stream_id,
-                  a.gs_cells, a.tensor_closed_form, a.codes, a.sf, a.gscale);
+#define NVFP4_LAUNCH_TR(TILED_, RHT_)                                                                                              \
+  launch_kernel(quantize_transpose_kernel<SRC, GS, SR, TILED_, RHT_, false>, dim3(grid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.seed, \
+                a.stream_id, a.gs_cells, a.tensor_closed_form, a.codes, a.sf, a.gscale, a.rht_stream)
+  if (a.sf_tiled) {
+    if (a.rht_stream) NVFP4_LAUNCH_TR(true, true); else NVFP4_LAUNCH_TR(true, false);
+  } else {
+    if (a.rht_stream) NVFP4_LAUNCH_TR(false, true); else NVFP4_LAUNCH_TR(false, false);
+  }
+#undef NVFP4_LAUNCH_TR
+  return cudaGetLastError();
+}
+
+// amax pre-pass over the transformed source: the quantizer's own tile walk, stopped after the block maxima
+template <int SRC, int GS>
+static cudaError_t launch_tr_amax_rht(const TransposeSrc& src, int64_t rowsK, int64_t D, uint64_t seed, uint32_t rht_stream,
+                                      uint32_t* cells, cudaStream_t st) {
+  const dim3 grid(blocks_for(rowsK, 128), blocks_for(D, 64));
+  launch_kernel(quantize_transpose_kernel<SRC, GS, false, false, true, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
+                0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), rht_stream);
   return cudaGetLastError();
 }
 
@@ -674,6 +837,16 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
   a.tensor_closed_form = 0;
   cudaError_t e;
   const dim3 agrid(blocks_for(a.D, 64), blocks_for(a.rowsK, 256));
+  if (a.rht_stream && a.gs_mode != kGsBlock128) {
+    const bool per_row = a.gs_mode == kGsRow;
+    if (per_row || a.compute_amax) {
+      if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t) * (size_t)(per_row ? a.D : 1), st)) != cudaSuccess) return e;
+      e = per_row ? launch_tr_amax_rht<SRC, kGsRow>(a.src, a.rowsK, a.D, a.seed, a.rht_stream, a.gs_cells, st)
+                  : launch_tr_amax_rht<SRC, kGsTensor>(a.src, a.rowsK, a.D, a.seed, a.rht_stream, a.gs_cells, st);
+      if (e != cudaSuccess) return e;
+    }
+    return per_row ? launch_tr_r<SRC, kGsRow>(a, st) : launch_tr_r<SRC, kGsTensor>(a, st);
+  }
   if (a.gs_mode == kGsTensor) {
     if (a.compute_amax) {
       if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
@@ -711,8 +884,11 @@ cudaError_t launch_amax_tensor(const uint16_t* src, int64_t rows, int64_t cols, 
 }
 
 cudaError_t launch_amax_transpose_src(const TransposeSrc& s, int from_codes, int64_t rowsK, int64_t D, uint32_t* cell,
-                                      cudaStream_t st) {
+                                      cudaStream_t st, uint64_t seed, uint32_t rht_stream) {
   if (rowsK == 0 || D == 0) return cudaSuccess;
+  if (rht_stream)
+    return from_codes ? launch_tr_amax_rht<1, kGsTensor>(s, rowsK, D, seed, rht_stream, cell, st)
+                      : launch_tr_amax_rht<0, kGsTensor>(s, rowsK, D, seed, rht_stream, cell, st);
   const dim3 agrid(blocks_for(D, 64), blocks_for(rowsK, 256));
   if (from_codes)
     launch_kernel(amax_cols_generic_kernel<1>, dim3(agrid), dim3(256), 0, st, s, rowsK, D, cell, 0, 0);

@@ -15,11 +15,12 @@ def to_dev_i32(a) -> torch.Tensor:
     return torch.from_numpy(np.asarray(a, dtype=np.int32)).cuda()
 
 
-def assert_operand_equal(gpu_op, ref: orc.Operand, what=""):
+def assert_operand_equal(gpu_op, ref: orc.Operand, what="", k_extended=False):
     """Bit-exact comparison of a device operand with an oracle operand: codes, scales, global scales; and the
-    padding the device layout adds (K up to 128) must be zero."""
+    padding the device layout adds (K up to 128) must be zero. `k_extended`: the reference was computed on a matrix
+    already zero-extended to a multiple of 16 columns (the Hadamard-transformed operands), the device operand keeps K."""
     torch.cuda.synchronize()
-    assert gpu_op.R == ref.R and gpu_op.K == ref.K, what
+    assert gpu_op.R == ref.R and (gpu_op.K == ref.K or (k_extended and (gpu_op.K + 15) // 16 * 16 == ref.K)), what
     Kp = gpu_op.Kp
     K16 = ref.K16
     codes = gpu_op.codes.cpu().numpy()[: ref.R * (Kp // 2)].reshape(ref.R, Kp // 2)

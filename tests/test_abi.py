@@ -49,16 +49,17 @@ def test_bad_arguments_are_refused_on_the_host(binding):
     op = b.COperand(0x1000, 0x2000, 0x3000, 4, 32, 0, 0)
     ws = 0x4000
     q = lambda *a: L.nvfp4_quantize(*a)
-    assert q(0, 4, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 1  # null source
-    assert q(0x100, 4, 32, 32, 2, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 4  # bad axis
-    assert q(0x100, 4, 32, 32, 0, 7, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 4  # bad rounding
-    assert q(0x100, -1, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 2  # negative size
-    assert q(0x100, 5, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 2  # out shape mismatch
-    assert q(0x104, 4, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 3  # misaligned source
-    assert q(0x100, 4, 32, 36, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 3  # ld not multiple of 8
-    assert q(0x100, 4, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 8, None) == 5  # workspace too small
+    assert q(0, 4, 32, 32, 0, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 1  # null source
+    assert q(0x100, 4, 32, 32, 2, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 4  # bad axis
+    assert q(0x100, 4, 32, 32, 0, 7, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 4  # bad rounding
+    assert q(0x100, -1, 32, 32, 0, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 2  # negative size
+    assert q(0x100, 5, 32, 32, 0, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 2  # out shape mismatch
+    assert q(0x104, 4, 32, 32, 0, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 3  # misaligned source
+    assert q(0x100, 4, 32, 36, 0, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 256, None) == 3  # ld not multiple of 8
+    assert q(0x100, 4, 32, 32, 0, 0, 0, 0, 0, None, 0, ctypes.byref(op), ws, 8, None) == 5  # workspace too small
+    assert q(0x100, 4, 32, 32, 0, 0, 0, 0, 7, 0x6000, 32, ctypes.byref(op), ws, 256, None) == 4  # transformation + column list
     bad = b.COperand(0x1000, 0x2000, 0x3000, 4, 32, 9, 0)
-    assert q(0x100, 4, 32, 32, 0, 0, 0, 0, None, 0, ctypes.byref(bad), ws, 256, None) == 4  # bad gs_mode
+    assert q(0x100, 4, 32, 32, 0, 0, 0, 0, 0, None, 0, ctypes.byref(bad), ws, 256, None) == 4  # bad gs_mode
     a = b.COperand(0x1000, 0x2000, 0x3000, 4, 32, 0, 1)
     c = b.COperand(0x1000, 0x2000, 0x3000, 4, 64, 0, 1)
     assert L.nvfp4_gemm(ctypes.byref(a), ctypes.byref(c), 0x5000, 1, 4, 0, None, None, 0, None) == 2  # K mismatch
