@@ -44,11 +44,12 @@ def outlier_channels(K: int, n: int, seed: int) -> np.ndarray:
     return np.sort(rng.choice(K, size=n, replace=False)).astype(np.int64)
 
 
-def activations(rows: int, cols: int, seed: int, n_outlier: int = 0, factor: float = 1.0):
-    """~N(0,1) with ``n_outlier`` channels multiplied by ``factor``. Returns (tensor, sorted channel list)."""
+def activations(rows: int, cols: int, seed: int, n_outlier: int = 0, factor: float = 1.0, channel_seed: int | None = None):
+    """~N(0,1) with ``n_outlier`` channels multiplied by ``factor``. Returns (tensor, sorted channel list).
+    ``channel_seed`` fixes the channel choice independently of the values (the same channels over several steps)."""
     rng = np.random.default_rng(seed)
     x = rng.standard_normal((rows, cols), dtype=np.float32)
-    ch = outlier_channels(cols, n_outlier, seed) if n_outlier else np.zeros(0, dtype=np.int64)
+    ch = outlier_channels(cols, n_outlier, seed if channel_seed is None else channel_seed) if n_outlier else np.zeros(0, dtype=np.int64)
     if n_outlier:
         x[:, ch] *= np.float32(factor)
     return round_to_bf16(x), ch
