@@ -240,6 +240,26 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
                                  const nvfp4_layer_cfg* cfg, void* dW, int64_t lddw, void* workspace,
                                  size_t ws_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------------------------
+ * OutControl calibration (Sec. 4.2, the paragraph defining the outlier index set A): the activation l2-norm of every
+ * channel is accumulated over a calibration window; the channels with the largest accumulated value form A.
+ *
+ * nvfp4_outlier_accumulate — one step of the window:  acc[d] += sqrt(sum_t X[t, d]^2),  X BF16 [N_tok, D] (device,
+ *   leading dimension ldx, 16-byte aligned rows), acc FP32 [D] (device, read and written). FP32 arithmetic with a fixed
+ *   summation order (bit-reproducible for a given shape). workspace: at least
+ *   nvfp4_outlier_accumulate_workspace_bytes(N_tok, D), 16-byte aligned.
+ * nvfp4_outlier_select — the n_out channels that come first in the order (acc descending, channel index ascending on
+ *   ties; NaN is outside the contract). Writes, all device int32: outlier_cols [n_out] sorted ascending, keep_cols
+ *   [D - n_out] sorted ascending, col_map [D] = position of channel d in keep_cols or -1 for an outlier — exactly the
+ *   three arrays nvfp4_layer_cfg takes. n_out is the caller's rounding of p % of D.
+ * Errors: NULL / SHAPE / ALIGN / WORKSPACE / ARCH as elsewhere; nothing is launched on an error.
+ * --------------------------------------------------------------------------------------------------------- */
+size_t nvfp4_outlier_accumulate_workspace_bytes(int64_t N_tok, int64_t D);
+nvfp4_status nvfp4_outlier_accumulate(const void* X_bf16, int64_t ldx, int64_t N_tok, int64_t D, float* acc,
+                                      void* workspace, size_t ws_bytes, void* stream);
+nvfp4_status nvfp4_outlier_select(const float* acc, int64_t D, int64_t n_out, int32_t* outlier_cols,
+                                  int32_t* keep_cols, int32_t* col_map, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -75,6 +75,9 @@ EXPORTS = {
                                     c_sz, c_vp]),
     "nvfp4_linear_bwd_dw": (c_i32, [c_vp, c_i64, ctypes.POINTER(CSaved), ctypes.POINTER(CLayerCfg), c_vp, c_i64, c_vp,
                                     c_sz, c_vp]),
+    "nvfp4_outlier_accumulate_workspace_bytes": (c_sz, [c_i64, c_i64]),
+    "nvfp4_outlier_accumulate": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_vp, c_vp, c_sz, c_vp]),
+    "nvfp4_outlier_select": (c_i32, [c_vp, c_i64, c_i64, c_vp, c_vp, c_vp, c_vp]),
 }
 for _name, (_res, _args) in EXPORTS.items():
     _f = getattr(_lib, _name)
@@ -224,6 +227,28 @@ def nvfp4_gemm(A: Operand, B: Operand, c_dtype: int = DT_F32, out: torch.Tensor 
     _check(_lib.nvfp4_gemm(ctypes.byref(ca), ctypes.byref(cb), _ptr(out), c_dtype, out.stride(0), int(accumulate),
                            _ptr(dev_status), _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_gemm")
     return out
+
+
+def nvfp4_outlier_accumulate(X: torch.Tensor, acc: torch.Tensor, workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """acc[d] += ||X[:, d]||_2 (one step of OutControl's calibration window); acc is float32 [D] on the device."""
+    assert X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    assert acc.dtype == torch.float32 and acc.is_contiguous() and acc.numel() == X.shape[1]
+    N_tok, D = X.shape
+    ws = workspace if workspace is not None else _workspace(_lib.nvfp4_outlier_accumulate_workspace_bytes(N_tok, D), X.device)
+    _check(_lib.nvfp4_outlier_accumulate(_ptr(X), X.stride(0), N_tok, D, _ptr(acc), _ptr(ws), ws.numel(), _stream_ptr()),
+           "nvfp4_outlier_accumulate")
+    return acc
+
+
+def nvfp4_outlier_select(acc: torch.Tensor, n_out: int):
+    """Top-n_out channels of acc -> (outlier_cols, keep_cols, col_map), int32 device tensors."""
+    assert acc.dtype == torch.float32 and acc.is_contiguous()
+    D = acc.numel()
+    outl = torch.empty(max(n_out, 1), dtype=torch.int32, device=acc.device)[:n_out]
+    keep = torch.empty(max(D - n_out, 1), dtype=torch.int32, device=acc.device)[: D - n_out]
+    cmap = torch.empty(max(D, 1), dtype=torch.int32, device=acc.device)[:D]
+    _check(_lib.nvfp4_outlier_select(_ptr(acc), D, n_out, _ptr(outl), _ptr(keep), _ptr(cmap), _stream_ptr()), "nvfp4_outlier_select")
+    return outl, keep, cmap
 
 
 @dataclass

@@ -196,6 +196,10 @@ bool bad_matrix(const void* p, int64_t ld, int64_t cols, int elem_bytes) {
 
 }  // namespace
 
+namespace nvfp4 {
+bool device_is_sm100() { return check_arch() == NVFP4_OK; }
+}  // namespace nvfp4
+
 extern "C" {
 
 int64_t nvfp4_padded_k(int64_t K) { return round_up(K, 128); }

@@ -10,6 +10,9 @@ namespace nvfp4 {
 // Number of kernels this library has enqueued since it was loaded (measurement aid).
 extern long long g_launch_count;
 
+// true if the current device has compute capability 10.x (cached per device)
+bool device_is_sm100();
+
 struct QuantRowsArgs {
   const uint16_t* src;  // BF16 [rows, cols_src], leading dimension ld
   int64_t rows, K, cols_src, ld;
