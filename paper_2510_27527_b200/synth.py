@@ -104,3 +104,22 @@ def layer_inputs(config: int, tokens: int, D: int, C: int, *, n_outlier: int, fa
     W = weights(C, D, seed_of(config, weight_id))
     dY = gradients(tokens, C, seed_of(config, 3) + 7 * C, grad_scale)
     return X, W, dY, ch
+
+
+def weight_trajectory(C: int, D: int, steps: int, seed: int, std: float = 0.02, step_scale: float = 2e-3, osc_fraction: float = 0.02):
+    """FP32 master weights over ``steps + 1`` optimizer steps, as a list of [C, D] float32 arrays.
+
+    Start ~N(0, std). Every step adds small Gaussian noise (step_scale * std). A planted ``osc_fraction`` of the
+    elements additionally alternates by +-1.5 % of its own magnitude from step to step (late-training oscillation:
+    the master weight moves little, its quantized value may flip between two bins). Returns (list, planted mask)."""
+    rng = np.random.default_rng(seed)
+    w = (rng.standard_normal((C, D), dtype=np.float32) * np.float32(std)).astype(np.float32)
+    planted = rng.random((C, D)) < osc_fraction
+    amp = (np.float32(0.015) * np.abs(w)).astype(np.float32)
+    out = [w.copy()]
+    for t in range(1, steps + 1):
+        w = w + rng.standard_normal((C, D), dtype=np.float32) * np.float32(step_scale * std)
+        sign = np.float32(1.0 if t % 2 else -1.0)
+        w = np.where(planted, w + sign * amp, w).astype(np.float32)
+        out.append(w.copy())
+    return out, planted
