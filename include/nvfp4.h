@@ -260,6 +260,31 @@ nvfp4_status nvfp4_outlier_accumulate(const void* X_bf16, int64_t ldx, int64_t N
 nvfp4_status nvfp4_outlier_select(const float* acc, int64_t D, int64_t n_out, int32_t* outlier_cols,
                                   int32_t* keep_cols, int32_t* col_map, void* stream);
 
+/* ---------------------------------------------------------------------------------------------------------
+ * OsciReset (Sec. 3.2-3.3): oscillation statistics of the master weights (appendix Algorithm 2,
+ * "UpdateOscillationStats") and the reset of high-risk weights to their bin centre (Algorithm 1,
+ * "OscillationSuppress"), for one weight matrix.
+ *
+ *   W      master weights, FP32 [C, D] (device), leading dimension ldw, 16-byte aligned rows for full speed.
+ *   W_prev, D_M, D_Q   the state of Algorithm 2: previous step's weights and the two accumulated path lengths, FP32
+ *          [C, D] contiguous (device, 16-byte aligned), owned by the caller, 12 B per parameter.
+ *   Q(.)   FP4 quant-dequant as the layer's forward weight quantizer defines it: cast to BF16 (nearest even), double-block
+ *          quantize along D with round-to-nearest in `gs_mode`, dequantize as float32((P * S_block) * S_global).
+ *
+ * nvfp4_osci_update, t0 = 0:  D_M = D_Q = 0, W_prev = W.
+ *                    t0 > 0:  D_M += |W - W_prev|;  D_Q += |Q(W) - Q(W_prev)|;  W_prev = W   (one binary32 operation each).
+ * nvfp4_osci_suppress:        W[i] = Q(W)[i] wherever float32(D_Q[i] / D_M[i]) >= tau (0 / 0 is no reset); Q is taken of
+ *                             the weights as they are before any reset. *n_reset (device, optional, 8-byte aligned) is
+ *                             incremented by the number of resets. The statistics are not modified.
+ * workspace: nvfp4_osci_workspace_bytes(C, gs_mode) bytes (amax cells of the TENSOR / ROW modes), 4-byte aligned.
+ * --------------------------------------------------------------------------------------------------------- */
+size_t nvfp4_osci_workspace_bytes(int64_t C, int32_t gs_mode);
+nvfp4_status nvfp4_osci_update(const float* W, int64_t ldw, int64_t C, int64_t D, int32_t gs_mode, int32_t t0,
+                               float* W_prev, float* D_M, float* D_Q, void* workspace, size_t ws_bytes, void* stream);
+nvfp4_status nvfp4_osci_suppress(float* W, int64_t ldw, int64_t C, int64_t D, int32_t gs_mode, const float* D_M,
+                                 const float* D_Q, float tau, unsigned long long* n_reset, void* workspace,
+                                 size_t ws_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

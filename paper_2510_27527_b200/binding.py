@@ -78,6 +78,9 @@ EXPORTS = {
     "nvfp4_outlier_accumulate_workspace_bytes": (c_sz, [c_i64, c_i64]),
     "nvfp4_outlier_accumulate": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_vp, c_vp, c_sz, c_vp]),
     "nvfp4_outlier_select": (c_i32, [c_vp, c_i64, c_i64, c_vp, c_vp, c_vp, c_vp]),
+    "nvfp4_osci_workspace_bytes": (c_sz, [c_i64, c_i32]),
+    "nvfp4_osci_update": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_vp, c_vp, c_vp, c_vp, c_sz, c_vp]),
+    "nvfp4_osci_suppress": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_vp, c_vp, ctypes.c_float, c_vp, c_vp, c_sz, c_vp]),
 }
 for _name, (_res, _args) in EXPORTS.items():
     _f = getattr(_lib, _name)
@@ -249,6 +252,39 @@ def nvfp4_outlier_select(acc: torch.Tensor, n_out: int):
     cmap = torch.empty(max(D, 1), dtype=torch.int32, device=acc.device)[:D]
     _check(_lib.nvfp4_outlier_select(_ptr(acc), D, n_out, _ptr(outl), _ptr(keep), _ptr(cmap), _stream_ptr()), "nvfp4_outlier_select")
     return outl, keep, cmap
+
+
+@dataclass
+class OsciState:
+    """State of the oscillation statistics for one weight matrix (float32 [C, D] each, device)."""
+
+    W_prev: torch.Tensor
+    D_M: torch.Tensor
+    D_Q: torch.Tensor
+
+
+def alloc_osci_state(W: torch.Tensor) -> OsciState:
+    mk = lambda: torch.empty(W.shape, dtype=torch.float32, device=W.device)
+    return OsciState(mk(), mk(), mk())
+
+
+def nvfp4_osci_update(W: torch.Tensor, state: OsciState, t0: int, gs_mode: int = GS_TENSOR, workspace: torch.Tensor | None = None) -> None:
+    assert W.dtype == torch.float32 and W.dim() == 2 and W.stride(1) == 1
+    C, D = W.shape
+    ws = workspace if workspace is not None else _workspace(_lib.nvfp4_osci_workspace_bytes(C, gs_mode), W.device)
+    _check(_lib.nvfp4_osci_update(_ptr(W), W.stride(0), C, D, gs_mode, t0, _ptr(state.W_prev), _ptr(state.D_M), _ptr(state.D_Q),
+                                  _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_osci_update")
+
+
+def nvfp4_osci_suppress(W: torch.Tensor, state: OsciState, tau: float, gs_mode: int = GS_TENSOR, n_reset: torch.Tensor | None = None,
+                        workspace: torch.Tensor | None = None) -> None:
+    """Resets, in place, the elements of W whose oscillation risk D_Q / D_M is at least tau."""
+    assert W.dtype == torch.float32 and W.dim() == 2 and W.stride(1) == 1
+    assert n_reset is None or (n_reset.dtype == torch.int64 and n_reset.numel() == 1)
+    C, D = W.shape
+    ws = workspace if workspace is not None else _workspace(_lib.nvfp4_osci_workspace_bytes(C, gs_mode), W.device)
+    _check(_lib.nvfp4_osci_suppress(_ptr(W), W.stride(0), C, D, gs_mode, _ptr(state.D_M), _ptr(state.D_Q), float(tau), _ptr(n_reset),
+                                    _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_osci_suppress")
 
 
 @dataclass

@@ -207,6 +207,31 @@ __device__ __forceinline__ float e2m1_decode(uint32_t code) {
   return __uint_as_float(bits | ((code & 8u) << 28));
 }
 
+// Decode 8 packed E2M1 codes times one E4M3 scale times the global scale into 8 floats:
+// x_hat = (P * S_block) * S_global; the inner product is exact in FP16 (6 significant bits, |value| <= 2688).
+__device__ __forceinline__ void decode8(uint32_t word, uint32_t sf_byte, float sg, float* out) {
+  uint32_t h[4];
+  asm("{\n"
+      ".reg .b8 b0, b1, b2, b3;\n"
+      "mov.b32 {b0, b1, b2, b3}, %4;\n"
+      "cvt.rn.f16x2.e2m1x2 %0, b0;\n"
+      "cvt.rn.f16x2.e2m1x2 %1, b1;\n"
+      "cvt.rn.f16x2.e2m1x2 %2, b2;\n"
+      "cvt.rn.f16x2.e2m1x2 %3, b3;\n"
+      "}"
+      : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3])
+      : "r"(word));
+  uint32_t s2;
+  asm("{.reg .b16 t; cvt.u16.u32 t, %1; cvt.rn.f16x2.e4m3x2 %0, t;}" : "=r"(s2) : "r"(sf_byte | (sf_byte << 8)));
+  const __half2 sb2 = *reinterpret_cast<__half2*>(&s2);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __half22float2(__hmul2(*reinterpret_cast<__half2*>(&h[i]), sb2));
+    out[2 * i] = __fmul_rn(f.x, sg);
+    out[2 * i + 1] = __fmul_rn(f.y, sg);
+  }
+}
+
 // Byte offset of scale (r, kb) in the TILED128x4 layout with n_ktiles4 = (number of k-blocks, padded to 16) / 4.
 __device__ __forceinline__ size_t sf_tiled_offset(int64_t r, int64_t kb, int64_t kb_padded) {
   const int64_t tile = (r >> 7) * (kb_padded >> 2) + (kb >> 2);

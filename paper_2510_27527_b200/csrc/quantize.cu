@@ -484,31 +484,6 @@ __global__ void __launch_bounds__(256) amax_cols_generic_kernel(TransposeSrc s, 
   }
 }
 
-// Decode 8 packed E2M1 codes times one E4M3 scale times the global scale into 8 floats:
-// x_hat = (P * S_block) * S_global; the inner product is exact in FP16 (6 significant bits, |value| <= 2688).
-__device__ __forceinline__ void decode8(uint32_t word, uint32_t sf_byte, float sg, float* out) {
-  uint32_t h[4];
-  asm("{\n"
-      ".reg .b8 b0, b1, b2, b3;\n"
-      "mov.b32 {b0, b1, b2, b3}, %4;\n"
-      "cvt.rn.f16x2.e2m1x2 %0, b0;\n"
-      "cvt.rn.f16x2.e2m1x2 %1, b1;\n"
-      "cvt.rn.f16x2.e2m1x2 %2, b2;\n"
-      "cvt.rn.f16x2.e2m1x2 %3, b3;\n"
-      "}"
-      : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3])
-      : "r"(word));
-  uint32_t s2;
-  asm("{.reg .b16 t; cvt.u16.u32 t, %1; cvt.rn.f16x2.e4m3x2 %0, t;}" : "=r"(s2) : "r"(sf_byte | (sf_byte << 8)));
-  const __half2 sb2 = *reinterpret_cast<__half2*>(&s2);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float2 f = __half22float2(__hmul2(*reinterpret_cast<__half2*>(&h[i]), sb2));
-    out[2 * i] = __fmul_rn(f.x, sg);
-    out[2 * i + 1] = __fmul_rn(f.y, sg);
-  }
-}
-
 //   RHT        the 16-blocks along k are replaced by (x S) H_16: the sign and the 1/4 are applied while staging (one
 //              factor per source row), the butterflies on the 16 values a thread reads back.
 //   AMAX_ONLY  stop after the block maxima and fold them into the amax cells (pre-pass for TENSOR / ROW under RHT;
