@@ -389,6 +389,72 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_aux(args):
+    """HBM roofline of the auxiliary kernels (OutControl calibration, OsciReset statistics / reset) on large matrices:
+    one JSON line. Not the headline line."""
+    import torch
+
+    from paper_2510_27527_b200 import binding as b
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    pk = peaks()
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    flush_src = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+
+    def t_of(fn, n):
+        for _ in range(3):
+            fn()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        torch.cuda.synchronize()
+        for i in range(n):
+            flush_buf.fill_(1)
+            flush_src.max()
+            ev[i][0].record()
+            fn()
+            ev[i][1].record()
+        torch.cuda.synchronize()
+        ms = sorted(a.elapsed_time(bb) for a, bb in ev)
+        return ms[len(ms) // 2] * 1e-3
+
+    g = torch.Generator(device=dev)
+    g.manual_seed(7)
+    out = {}
+    N, D = 16384, 8192
+    X = torch.randn((N, D), device=dev, generator=g, dtype=torch.float32).to(torch.bfloat16)
+    acc = torch.zeros(D, dtype=torch.float32, device=dev)
+    ws = b._workspace(b.lib.nvfp4_outlier_accumulate_workspace_bytes(N, D), dev)
+    sec = t_of(lambda: b.nvfp4_outlier_accumulate(X, acc, workspace=ws), args.steps)
+    out["outlier_accumulate_16384x8192"] = {"us": sec * 1e6, "GBps": 2.0 * N * D / sec / 1e9, "frac_hbm_measured": 2.0 * N * D / sec / 1e9 / pk["hbm"]}
+    sec = t_of(lambda: b.nvfp4_outlier_select(acc, D // 10), args.steps)
+    out["outlier_select_8192_top10pct"] = {"us": sec * 1e6}
+    del X
+    C, D = 8192, 8192
+    W = torch.randn((C, D), device=dev, generator=g, dtype=torch.float32) * 0.02
+    W1 = W + torch.randn((C, D), device=dev, generator=g, dtype=torch.float32) * 4e-5
+    st = b.alloc_osci_state(W)
+    for name, gs in GS.items():
+        wsp = b._workspace(b.lib.nvfp4_osci_workspace_bytes(C, gs), dev)
+        b.nvfp4_osci_update(W, st, 0, gs, workspace=wsp)
+        flip = [0]
+
+        def upd():
+            flip[0] ^= 1
+            b.nvfp4_osci_update(W1 if flip[0] else W, st, 1, gs, workspace=wsp)
+
+        sec = t_of(upd, args.steps)
+        # algorithmic bytes: read W, W', D_M, D_Q and write W', D_M, D_Q (7 x 4 B); TENSOR / ROW re-read W and W' for amax
+        alg = (28.0 + (8.0 if gs != 2 else 0.0)) * C * D
+        out[f"osci_update_8192x8192_{name}"] = {"us": sec * 1e6, "GBps": alg / sec / 1e9, "frac_hbm_measured": alg / sec / 1e9 / pk["hbm"]}
+        n = torch.zeros(1, dtype=torch.int64, device=dev)
+        Wc = W1.clone()
+        sec = t_of(lambda: b.nvfp4_osci_suppress(Wc, st, 8.0, gs, n_reset=n, workspace=wsp), args.steps)
+        # read W, D_M, D_Q (12 B) (+4 B amax pre-pass); writes only the few reset blocks
+        alg = (12.0 + (4.0 if gs != 2 else 0.0)) * C * D
+        out[f"osci_suppress_8192x8192_{name}"] = {"us": sec * 1e6, "GBps": alg / sec / 1e9, "frac_hbm_measured": alg / sec / 1e9 / pk["hbm"]}
+    print(json.dumps({"aux": out, "peaks": pk}))
+
+
 def run_sweep(args):
     """Roofline sweep (square and skinny GEMMs with their quantizers), one JSON line with a list of shapes.
     Not the headline line: a measurement aid for the large-shape roofline fractions."""
@@ -481,10 +547,13 @@ def main():
     ap.add_argument("--rht", action="store_true", help="random Hadamard transformation (block 16) in the four backward quantizers")
     ap.add_argument("--no-breakdown", action="store_true", help="only warm-up + timed steps (used for ncu launch lists)")
     ap.add_argument("--sweep", action="store_true", help="roofline sweep of the large GEMM shapes instead of the step benchmark")
+    ap.add_argument("--aux", action="store_true", help="HBM roofline of the calibration and OsciReset kernels instead of the step benchmark")
     ap.add_argument("--shapes", default="", help="with --sweep: comma list of MxNxK")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+    elif args.aux:
+        run_aux(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -34,15 +34,12 @@ __global__ void __launch_bounds__(256) colsq_partial_kernel(const uint16_t* __re
   };
   if (c0 + 8 <= D) {
     int64_t r = r_begin + ry;
-    for (; r + 24 < r_end; r += 32) {  // four rows in flight
-      const uint4 v0 = *reinterpret_cast<const uint4*>(X + r * ld + c0);
-      const uint4 v1 = *reinterpret_cast<const uint4*>(X + (r + 8) * ld + c0);
-      const uint4 v2 = *reinterpret_cast<const uint4*>(X + (r + 16) * ld + c0);
-      const uint4 v3 = *reinterpret_cast<const uint4*>(X + (r + 24) * ld + c0);
-      add8(v0);
-      add8(v1);
-      add8(v2);
-      add8(v3);
+    for (; r + 56 < r_end; r += 64) {  // eight rows in flight
+      uint4 v[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) v[q] = *reinterpret_cast<const uint4*>(X + (r + 8 * q) * ld + c0);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) add8(v[q]);
     }
     for (; r < r_end; r += 8) add8(*reinterpret_cast<const uint4*>(X + r * ld + c0));
   } else if (c0 < D) {  // ragged last chunk of a row

@@ -63,21 +63,25 @@ __device__ __forceinline__ void quant_dequant16(float (&w)[16], uint32_t amax_ce
   }
   float rcp;
   const uint32_t sb = block_scale(m, Sg, rcp);
-  float y0[8], y1[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    y0[i] = __fmul_rn(w[i], rcp);
-    y1[i] = __fmul_rn(w[8 + i], rcp);
-  }
-  // x_hat = (P * S_block) * S_global; P * S_block is exact in binary32 (2 + 4 significant bits). Decoded arithmetically:
-  // unpacking a word that the packing conversion produced in the same thread through byte registers (decode8) came
-  // back as zeros on the device, so that path is only used on words loaded from memory.
-  const uint32_t c0 = e2m1x8_rtn(y0), c1 = e2m1x8_rtn(y1);
+  // x_hat = (P * S_block) * S_global with P = the E2M1 value nearest to y (ties to the even code, saturating): the
+  // hardware conversion to a packed pair of codes followed by the conversion of that byte back to FP16, inside one asm
+  // block. (Packing the codes into a 32-bit word and unpacking that word through byte registers again in the same thread
+  // came back as zeros on the device; this form never leaves the byte register.) P * S_block is exact in binary32.
   const float Sbf = e4m3_decode(sb);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    w[i] = __fmul_rn(__fmul_rn(e2m1_decode((c0 >> (4 * i)) & 15u), Sbf), Sg);
-    w[8 + i] = __fmul_rn(__fmul_rn(e2m1_decode((c1 >> (4 * i)) & 15u), Sbf), Sg);
+    const float ylo = __fmul_rn(w[2 * i], rcp), yhi = __fmul_rn(w[2 * i + 1], rcp);
+    uint32_t h2;
+    asm("{\n"
+        ".reg .b8 t;\n"
+        "cvt.rn.satfinite.e2m1x2.f32 t, %2, %1;\n"
+        "cvt.rn.f16x2.e2m1x2 %0, t;\n"
+        "}"
+        : "=r"(h2)
+        : "f"(ylo), "f"(yhi));
+    const float2 pv = __half22float2(*reinterpret_cast<__half2*>(&h2));
+    w[2 * i] = __fmul_rn(__fmul_rn(pv.x, Sbf), Sg);
+    w[2 * i + 1] = __fmul_rn(__fmul_rn(pv.y, Sbf), Sg);
   }
 }
 
@@ -91,7 +95,20 @@ __global__ void __launch_bounds__(256) amax_f32_kernel(const float* __restrict__
   for (int64_t r = blockIdx.x; r < C; r += gridDim.x) {
     const float* p = W + r * ld;
     float mr = 0.0f;
-    for (int64_t c = threadIdx.x; c < chunks; c += 256) {
+    int64_t c = threadIdx.x;
+    if (vec) {
+      for (; ((c + 768) << 2) + 4 <= D; c += 1024) {  // four 16-byte loads in flight
+        const float4 v0 = *reinterpret_cast<const float4*>(p + (c << 2));
+        const float4 v1 = *reinterpret_cast<const float4*>(p + ((c + 256) << 2));
+        const float4 v2 = *reinterpret_cast<const float4*>(p + ((c + 512) << 2));
+        const float4 v3 = *reinterpret_cast<const float4*>(p + ((c + 768) << 2));
+        mr = fmaxf(mr, fmaxf(fmaxf(fabsf(v0.x), fabsf(v0.y)), fmaxf(fabsf(v0.z), fabsf(v0.w))));
+        mr = fmaxf(mr, fmaxf(fmaxf(fabsf(v1.x), fabsf(v1.y)), fmaxf(fabsf(v1.z), fabsf(v1.w))));
+        mr = fmaxf(mr, fmaxf(fmaxf(fabsf(v2.x), fabsf(v2.y)), fmaxf(fabsf(v2.z), fabsf(v2.w))));
+        mr = fmaxf(mr, fmaxf(fmaxf(fabsf(v3.x), fabsf(v3.y)), fmaxf(fabsf(v3.z), fabsf(v3.w))));
+      }
+    }
+    for (; c < chunks; c += 256) {
       if (vec && (c << 2) + 4 <= D) {
         const float4 v = *reinterpret_cast<const float4*>(p + (c << 2));
         mr = fmaxf(mr, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
@@ -153,6 +170,9 @@ __global__ void __launch_bounds__(256) osci_update_kernel(const float* __restric
   float w[16], p[16];
   load16f(W + r * ldw, k0, D, vw, w);
   load16f(Wp + r * D, k0, D, vs, p);
+  float a[16], aq[16];
+  load16f(DM + r * D, k0, D, vs, a);  // requested before the arithmetic
+  load16f(DQ + r * D, k0, D, vs, aq);
   float dm[16];
 #pragma unroll
   for (int i = 0; i < 16; ++i) dm[i] = fabsf(__fsub_rn(w[i], p[i]));
@@ -162,20 +182,17 @@ __global__ void __launch_bounds__(256) osci_update_kernel(const float* __restric
   quant_dequant16<GS>(w, cw);
   quant_dequant16<GS>(p, cp);
   if (!(active && k0 < D)) return;
-  float a[16];
-  load16f(DM + r * D, k0, D, vs, a);
 #pragma unroll
   for (int i = 0; i < 16; ++i) a[i] = __fadd_rn(a[i], dm[i]);
   store16f(DM + r * D, k0, D, vs, a);
-  load16f(DQ + r * D, k0, D, vs, a);
 #pragma unroll
-  for (int i = 0; i < 16; ++i) a[i] = __fadd_rn(a[i], fabsf(__fsub_rn(w[i], p[i])));
-  store16f(DQ + r * D, k0, D, vs, a);
+  for (int i = 0; i < 16; ++i) aq[i] = __fadd_rn(aq[i], fabsf(__fsub_rn(w[i], p[i])));
+  store16f(DQ + r * D, k0, D, vs, aq);
 }
 
 // Algorithm 1: w <- Q(w) where D_Q / D_M >= tau
 template <int GS>
-__global__ void __launch_bounds__(256) osci_suppress_kernel(float* __restrict__ W, int64_t ldw, int64_t C, int64_t D,
+__global__ void __launch_bounds__(256, 3) osci_suppress_kernel(float* __restrict__ W, int64_t ldw, int64_t C, int64_t D,
                                                            const float* __restrict__ DM, const float* __restrict__ DQ, float tau,
                                                            const uint32_t* __restrict__ cells, unsigned long long* n_reset) {
   pdl_prologue();
@@ -186,29 +203,34 @@ __global__ void __launch_bounds__(256) osci_suppress_kernel(float* __restrict__ 
   const int64_t k0 = active ? (gid - r * nb) << 4 : D;
   const bool vw = (ldw & 3) == 0, vs = (D & 3) == 0;
   float w[16], q[16];
-  load16f(W + r * ldw, k0, D, vw, w);
-#pragma unroll
-  for (int i = 0; i < 16; ++i) q[i] = w[i];
-  quant_dequant16<GS>(q, GS == kGsTensor ? cells[0] : GS == kGsRow ? cells[r] : 0u);
-  int n = 0;
-  if (active && k0 < D) {
+  uint32_t hits = 0;
+  {
     float dm[16], dq[16];
+    load16f(W + r * ldw, k0, D, vw, w);  // all three streams are requested before any arithmetic
     load16f(DM + r * D, k0, D, vs, dm);
     load16f(DQ + r * D, k0, D, vs, dq);
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-      const bool hit = (k0 + i < D) && (__fdiv_rn(dq[i], dm[i]) >= tau);  // NaN (0 / 0) compares false
-      if (hit) {
-        w[i] = q[i];
-        ++n;
-      }
+      // NaN (0 / 0) compares false; an element whose quantized value never moved has risk 0 (or 0 / 0): no division
+      const bool hit = (k0 + i < D) && ((dq[i] == 0.0f && tau > 0.0f) ? false : (__fdiv_rn(dq[i], dm[i]) >= tau));
+      hits |= (hit ? 1u : 0u) << i;
     }
-    if (n) store16f(W + r * ldw, k0, D, vw, w);
+  }
+#pragma unroll
+  for (int i = 0; i < 16; ++i) q[i] = w[i];
+  quant_dequant16<GS>(q, GS == kGsTensor ? cells[0] : GS == kGsRow ? cells[r] : 0u);
+  const int n = __popc(hits);
+  if (active && n) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+      if ((hits >> i) & 1u) w[i] = q[i];
+    store16f(W + r * ldw, k0, D, vw, w);
   }
   if (n_reset) {
+    int total = n;
 #pragma unroll
-    for (int o = 16; o; o >>= 1) n += __shfl_xor_sync(0xFFFFFFFFu, n, o);
-    if ((threadIdx.x & 31) == 0 && n) atomicAdd(n_reset, (unsigned long long)n);
+    for (int o = 16; o; o >>= 1) total += __shfl_xor_sync(0xFFFFFFFFu, total, o);
+    if ((threadIdx.x & 31) == 0 && total) atomicAdd(n_reset, (unsigned long long)total);
   }
 }
 
