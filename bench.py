@@ -212,7 +212,7 @@ def run_ours(args):
         L.Y = torch.empty((tokens, C), dtype=torch.bfloat16, device=dev)
         L.dXo = torch.empty((tokens, D), dtype=torch.bfloat16, device=dev)
         L.dWo = torch.empty((C, D), dtype=torch.float32, device=dev)
-        L.ws = [b.linear_workspace(k, tokens, D, C, L.cfg, dev) for k in (b.OP_FWD, b.OP_BWD_DX, b.OP_BWD_DW)]
+        L.ws = [b.linear_workspace(k, tokens, D, C, L.cfg, dev) for k in (b.OP_FWD, b.OP_BWD_DX, b.OP_BWD_DW, b.OP_BWD)]
         lins.append(L)
 
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
@@ -229,8 +229,7 @@ def run_ours(args):
             for L in lins:
                 W = L.W[layer]
                 b.nvfp4_linear_fwd(L.X, W, L.cfg, Y=L.Y, saved=L.saved, workspace=L.ws[0])
-                b.nvfp4_linear_bwd_dx(L.dY, L.saved, L.cfg, dX=L.dXo, workspace=L.ws[1])
-                b.nvfp4_linear_bwd_dw(L.dY, L.saved, L.cfg, dW=L.dWo, workspace=L.ws[2])
+                b.nvfp4_linear_bwd(L.dY, L.saved, L.cfg, dX=L.dXo, dW=L.dWo, workspace=L.ws[3])
 
     def barrier():
         torch.cuda.synchronize()
@@ -292,8 +291,7 @@ def run_ours(args):
                 L.dY.copy_(L.pin[1], non_blocking=True)
                 W = L.W[layer]
                 b.nvfp4_linear_fwd(L.X, W, L.cfg, Y=L.Y, saved=L.saved, workspace=L.ws[0])
-                b.nvfp4_linear_bwd_dx(L.dY, L.saved, L.cfg, dX=L.dXo, workspace=L.ws[1])
-                b.nvfp4_linear_bwd_dw(L.dY, L.saved, L.cfg, dW=L.dWo, workspace=L.ws[2])
+                b.nvfp4_linear_bwd(L.dY, L.saved, L.cfg, dX=L.dXo, dW=L.dWo, workspace=L.ws[3])
                 L.out_pin[0].copy_(L.Y, non_blocking=True)
                 L.out_pin[1].copy_(L.dXo, non_blocking=True)
                 L.out_pin[2].copy_(L.dWo, non_blocking=True)

@@ -219,7 +219,7 @@ typedef struct {
 /* Columns of the compact outlier-channel matrices: n_out rounded up to a multiple of 64 (0 for n_out = 0). */
 int64_t nvfp4_outlier_pad(int64_t n_out);
 
-typedef enum { NVFP4_OP_FWD = 0, NVFP4_OP_BWD_DX = 1, NVFP4_OP_BWD_DW = 2 } nvfp4_op_kind;
+typedef enum { NVFP4_OP_FWD = 0, NVFP4_OP_BWD_DX = 1, NVFP4_OP_BWD_DW = 2, NVFP4_OP_BWD = 3 } nvfp4_op_kind;
 size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, int64_t C, int64_t n_out,
                                     int32_t gs_mode);
 
@@ -239,6 +239,13 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
 nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved* saved,
                                  const nvfp4_layer_cfg* cfg, void* dW, int64_t lddw, void* workspace,
                                  size_t ws_bytes, void* stream);
+
+/* Both backward products of Sec. 2.3 in one call: exactly nvfp4_linear_bwd_dx followed by nvfp4_linear_bwd_dw (bit-identical
+ * outputs), except that in the TENSOR scale mode without the Hadamard transformation the per-tensor amax of dY, which Q3
+ * and Q5 share, is computed once. workspace: nvfp4_linear_workspace_bytes(NVFP4_OP_BWD, ...). */
+nvfp4_status nvfp4_linear_bwd(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
+                              void* dX, int64_t lddx, void* dW, int64_t lddw, void* workspace, size_t ws_bytes,
+                              void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------
  * OutControl calibration (Sec. 4.2, the paragraph defining the outlier index set A): the activation l2-norm of every

@@ -26,7 +26,7 @@ AXIS_ROW, AXIS_COL = 0, 1
 GS_TENSOR, GS_ROW, GS_BLOCK128 = 0, 1, 2
 SF_LINEAR, SF_TILED128x4 = 0, 1
 DT_BF16, DT_F32 = 0, 1
-OP_FWD, OP_BWD_DX, OP_BWD_DW = 0, 1, 2
+OP_FWD, OP_BWD_DX, OP_BWD_DW, OP_BWD = 0, 1, 2, 3
 ERR_TIMEOUT = 8
 
 c_i64, c_i32, c_u64, c_u32, c_vp, c_sz = (ctypes.c_int64, ctypes.c_int32, ctypes.c_uint64, ctypes.c_uint32,
@@ -75,6 +75,8 @@ EXPORTS = {
                                     c_sz, c_vp]),
     "nvfp4_linear_bwd_dw": (c_i32, [c_vp, c_i64, ctypes.POINTER(CSaved), ctypes.POINTER(CLayerCfg), c_vp, c_i64, c_vp,
                                     c_sz, c_vp]),
+    "nvfp4_linear_bwd": (c_i32, [c_vp, c_i64, ctypes.POINTER(CSaved), ctypes.POINTER(CLayerCfg), c_vp, c_i64, c_vp, c_i64, c_vp,
+                                 c_sz, c_vp]),
     "nvfp4_outlier_accumulate_workspace_bytes": (c_sz, [c_i64, c_i64]),
     "nvfp4_outlier_accumulate": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_vp, c_vp, c_sz, c_vp]),
     "nvfp4_outlier_select": (c_i32, [c_vp, c_i64, c_i64, c_vp, c_vp, c_vp, c_vp]),
@@ -401,3 +403,19 @@ def nvfp4_linear_bwd_dw(dY: torch.Tensor, saved: Saved, cfg: LayerConfig, dW: to
     _check(_lib.nvfp4_linear_bwd_dw(_ptr(dY), dY.stride(0), ctypes.byref(cs), ctypes.byref(cc), _ptr(dW), dW.stride(0),
                                     _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_linear_bwd_dw")
     return dW
+
+
+def nvfp4_linear_bwd(dY: torch.Tensor, saved: Saved, cfg: LayerConfig, dX: torch.Tensor | None = None, dW: torch.Tensor | None = None,
+                     workspace: torch.Tensor | None = None):
+    """Both backward products in one call (dX, dW); the per-tensor amax of dY is computed once where Q3 and Q5 share it."""
+    N_tok, D = saved.X.shape
+    C = saved.W.shape[0]
+    if dX is None:
+        dX = _matrix(N_tok, D, cfg.dx_dtype, dY.device)
+    if dW is None:
+        dW = _matrix(C, D, cfg.dw_dtype, dY.device)
+    ws = workspace if workspace is not None else linear_workspace(OP_BWD, N_tok, D, C, cfg, dY.device)
+    cs, cc = saved.c(), cfg.c()
+    _check(_lib.nvfp4_linear_bwd(_ptr(dY), dY.stride(0), ctypes.byref(cs), ctypes.byref(cc), _ptr(dX), dX.stride(0), _ptr(dW),
+                                 dW.stride(0), _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_linear_bwd")
+    return dX, dW

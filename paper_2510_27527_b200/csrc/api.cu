@@ -93,7 +93,7 @@ bool carve_operand(Carver& c, nvfp4_operand* o, int64_t R, int64_t K, int32_t gs
 nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, int32_t rounding,
                               uint64_t seed, uint32_t stream_id, const int32_t* keep, int64_t n_keep,
                               const nvfp4_operand* out, uint32_t* cells, cudaStream_t st, int cells_zeroed = 0,
-                              const int32_t* excluded = nullptr, uint32_t rht_stream = 0) {
+                              const int32_t* excluded = nullptr, uint32_t rht_stream = 0, int compute_amax = 1) {
   if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   QuantRowsArgs a{};
   a.src = src;
@@ -109,7 +109,7 @@ nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, i
   a.gs_mode = out->gs_mode;
   a.sr = rounding == NVFP4_ROUND_SR;
   a.sf_tiled = out->sf_layout == NVFP4_SF_TILED128x4;
-  a.compute_amax = 1;
+  a.compute_amax = compute_amax;
   a.cells_zeroed = cells_zeroed;
   a.gs_cells = cells;
   a.codes = out->codes;
@@ -120,7 +120,7 @@ nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, i
 
 nvfp4_status do_quantize_transpose(const TransposeSrc& src, int from_codes, int64_t rowsK, int64_t D, int32_t rounding,
                                    uint64_t seed, uint32_t stream_id, const nvfp4_operand* out, uint32_t* cells,
-                                   cudaStream_t st, int cells_zeroed = 0, uint32_t rht_stream = 0) {
+                                   cudaStream_t st, int cells_zeroed = 0, uint32_t rht_stream = 0, int compute_amax = 1) {
   if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   QuantTransposeArgs a{};
   a.from_codes = from_codes;
@@ -133,7 +133,7 @@ nvfp4_status do_quantize_transpose(const TransposeSrc& src, int from_codes, int6
   a.gs_mode = out->gs_mode;
   a.sr = rounding == NVFP4_ROUND_SR;
   a.sf_tiled = out->sf_layout == NVFP4_SF_TILED128x4;
-  a.compute_amax = 1;
+  a.compute_amax = compute_amax;
   a.cells_zeroed = cells_zeroed;
   a.gs_cells = cells;
   a.codes = out->codes;
@@ -334,6 +334,10 @@ size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, i
     carve_size(total, cells_bytes(D, gs_mode));
     operand_sizes(total, N_tok, C, gs_mode);
     operand_sizes(total, D, C, gs_mode);
+  } else if (op_kind == NVFP4_OP_BWD) {
+    // both halves back to back (each already a multiple of 256 bytes) plus the shared amax cell
+    return nvfp4_linear_workspace_bytes(NVFP4_OP_BWD_DX, N_tok, D, C, n_out, gs_mode) +
+           nvfp4_linear_workspace_bytes(NVFP4_OP_BWD_DW, N_tok, D, C, n_out, gs_mode) + 256;
   } else {
     carve_size(total, cells_bytes(C, gs_mode));
     carve_size(total, cells_bytes(Dk, gs_mode));
@@ -407,8 +411,10 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
   return do_gemm(&saved->qx, &saved->qw, Y, cfg->y_dtype, ldy, 0, addend, ld_add, cfg->dev_status, st);
 }
 
-nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
-                                 void* dX, int64_t lddx, void* workspace, size_t ws_bytes, void* stream) {
+// dy_amax: optional cell already holding the bit pattern of max |dY| (TENSOR mode without the Hadamard transformation):
+// the amax pre-pass of the dY quantizer is then skipped.
+static nvfp4_status bwd_dx_impl(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
+                                void* dX, int64_t lddx, void* workspace, size_t ws_bytes, void* stream, uint32_t* dy_amax) {
   if (!dY || !saved || !dX) return NVFP4_ERR_NULL;
   const int64_t N_tok = saved->N_tok, D = saved->D, C = saved->C;
   if (N_tok <= 0 || D <= 0 || C <= 0) return NVFP4_ERR_SHAPE;
@@ -431,7 +437,7 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
   if (!zero_cells(cells3, cells4, cells_bytes(D, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
   const uint32_t rht = cfg->rht ? kRhtStreamDx : 0u;
   if ((s = do_quantize_rows(static_cast<const uint16_t*>(dY), N_tok, C, lddy, cfg->rounding[2], cfg->seed, 3, nullptr, 0,
-                            &q3, cells3, st, 1, nullptr, rht)) != NVFP4_OK)
+                            &q3, dy_amax ? dy_amax : cells3, st, 1, nullptr, rht, dy_amax ? 0 : 1)) != NVFP4_OK)
     return s;
   TransposeSrc ts{};
   ts.in_codes = saved->qw.codes;
@@ -499,8 +505,13 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
   return do_gemm(&q3, &q4, dX, cfg->dx_dtype, lddx, 0, nullptr, 0, cfg->dev_status, st);
 }
 
-nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
-                                 void* dW, int64_t lddw, void* workspace, size_t ws_bytes, void* stream) {
+nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
+                                 void* dX, int64_t lddx, void* workspace, size_t ws_bytes, void* stream) {
+  return bwd_dx_impl(dY, lddy, saved, cfg, dX, lddx, workspace, ws_bytes, stream, nullptr);
+}
+
+static nvfp4_status bwd_dw_impl(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
+                                void* dW, int64_t lddw, void* workspace, size_t ws_bytes, void* stream, uint32_t* dy_amax) {
   if (!dY || !saved || !dW) return NVFP4_ERR_NULL;
   const int64_t N_tok = saved->N_tok, D = saved->D, C = saved->C;
   if (N_tok <= 0 || D <= 0 || C <= 0) return NVFP4_ERR_SHAPE;
@@ -534,7 +545,9 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
   t5.ld = lddy;
   if (!zero_cells(cells5, cells6, cells_bytes(Dk, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
   const uint32_t rht = cfg->rht ? kRhtStreamDw : 0u;
-  if ((s = do_quantize_transpose(t5, 0, N_tok, C, cfg->rounding[4], cfg->seed, 5, &q5, cells5, st, 1, rht)) != NVFP4_OK) return s;
+  if ((s = do_quantize_transpose(t5, 0, N_tok, C, cfg->rounding[4], cfg->seed, 5, &q5, dy_amax ? dy_amax : cells5, st, 1, rht,
+                                 dy_amax ? 0 : 1)) != NVFP4_OK)
+    return s;
   TransposeSrc t6{};
   t6.in_codes = saved->qx.codes;
   t6.in_sf = saved->qx.sf;
@@ -554,6 +567,38 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
   h.lddy = lddy; h.Kh = Kh; h.T = N_tok; h.C = C; h.n_out = n_out; h.outl = cfg->outlier_cols;
   h.dW = dW; h.dw_is_f32 = dw_f32; h.lddw = lddw; h.partial = hp_partial; h.dev_status = cfg->dev_status;
   return launch_hp_dw(h, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
+                                 void* dW, int64_t lddw, void* workspace, size_t ws_bytes, void* stream) {
+  return bwd_dw_impl(dY, lddy, saved, cfg, dW, lddw, workspace, ws_bytes, stream, nullptr);
+}
+
+nvfp4_status nvfp4_linear_bwd(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg, void* dX,
+                              int64_t lddx, void* dW, int64_t lddw, void* workspace, size_t ws_bytes, void* stream) {
+  if (!dY || !saved || !cfg || !dX || !dW) return NVFP4_ERR_NULL;
+  const int64_t N_tok = saved->N_tok, D = saved->D, C = saved->C;
+  if (N_tok <= 0 || D <= 0 || C <= 0) return NVFP4_ERR_SHAPE;
+  if (cfg->gs_mode < 0 || cfg->gs_mode > 2 || cfg->n_out < 0 || cfg->n_out > D) return NVFP4_ERR_ENUM;
+  const size_t need_dx = nvfp4_linear_workspace_bytes(NVFP4_OP_BWD_DX, N_tok, D, C, cfg->n_out, cfg->gs_mode);
+  const size_t need_dw = nvfp4_linear_workspace_bytes(NVFP4_OP_BWD_DW, N_tok, D, C, cfg->n_out, cfg->gs_mode);
+  if (!workspace || !aligned16(workspace) || ws_bytes < nvfp4_linear_workspace_bytes(NVFP4_OP_BWD, N_tok, D, C, cfg->n_out, cfg->gs_mode))
+    return NVFP4_ERR_WORKSPACE;
+  if (bad_matrix(dY, lddy, C, 2)) return NVFP4_ERR_ALIGN;
+  uint8_t* base = static_cast<uint8_t*>(workspace);
+  uint32_t* shared = nullptr;
+  if (cfg->gs_mode == NVFP4_GS_TENSOR && !cfg->rht) {
+    // Q3 and Q5 quantize the same tensor with the same per-tensor scale: one amax pass serves both
+    nvfp4_status s;
+    if ((s = check_arch()) != NVFP4_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    shared = reinterpret_cast<uint32_t*>(base + need_dx + need_dw);
+    if (cudaMemsetAsync(shared, 0, sizeof(uint32_t), st) != cudaSuccess) return NVFP4_ERR_CUDA;
+    if (launch_amax_tensor(static_cast<const uint16_t*>(dY), N_tok, C, lddy, shared, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+  }
+  nvfp4_status s = bwd_dx_impl(dY, lddy, saved, cfg, dX, lddx, base, need_dx, stream, shared);
+  if (s != NVFP4_OK) return s;
+  return bwd_dw_impl(dY, lddy, saved, cfg, dW, lddw, base + need_dx, need_dw, stream, shared);
 }
 
 }  // extern "C"

@@ -78,3 +78,21 @@ def test_ragged_layer_shapes():
             dXo, dWo = orc.linear_bwd_dx(dY, so, ocfg), orc.linear_bwd_dw(dY, so, ocfg)
             Y, dX, dW, _ = run_layer(b, X, W, dY, gs_mode, outl, seed=3)
             assert rel_fro(Y, Yo) <= 2e-5 and rel_fro(dX, dXo) <= 2e-5 and rel_fro(dW, dWo) <= 2e-5
+
+
+@pytest.mark.parametrize("gs_mode", [0, 1, 2])
+@pytest.mark.parametrize("outcontrol", [False, True])
+@pytest.mark.parametrize("rht", [False, True])
+def test_combined_backward_is_bit_identical_to_the_two_calls(gs_mode, outcontrol, rht):
+    """nvfp4_linear_bwd = bwd_dx then bwd_dw; sharing the per-tensor amax of dY changes no bit."""
+    b = B()
+    N_tok, D, C = 200, 272, 136
+    X, W, dY, ch = synth.layer_inputs(9, N_tok, D, C, n_outlier=3, factor=40.0, grad_scale=1e-3)
+    cfg = b.LayerConfig(gs_mode=gs_mode, seed=3, outliers=ch if outcontrol else None, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32, rht=rht)
+    Xd, Wd, dYd = to_dev_bf16(X), to_dev_bf16(W), to_dev_bf16(dY)
+    _, saved = b.nvfp4_linear_fwd(Xd, Wd, cfg)
+    dX1 = b.nvfp4_linear_bwd_dx(dYd, saved, cfg)
+    dW1 = b.nvfp4_linear_bwd_dw(dYd, saved, cfg)
+    dX2, dW2 = b.nvfp4_linear_bwd(dYd, saved, cfg)
+    torch.cuda.synchronize()
+    assert torch.equal(dX1, dX2) and torch.equal(dW1, dW2)
