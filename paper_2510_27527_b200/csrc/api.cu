@@ -383,11 +383,16 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
   const uint16_t* Wp = static_cast<const uint16_t*>(W);
   const int32_t* keep = n_out > 0 ? cfg->keep_cols : nullptr;
   if (!zero_cells(cells_x, cells_w, cells_bytes(C, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
+  int amax_pass = 1;
+  if (cfg->gs_mode == NVFP4_GS_TENSOR && !keep) {  // the two per-tensor maxima in one launch
+    if (launch_amax_tensor_pair(Xp, N_tok, D, ldx, cells_x, Wp, C, D, ldw, cells_w, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+    amax_pass = 0;
+  }
   if ((s = do_quantize_rows(Xp, N_tok, D, ldx, cfg->rounding[0], cfg->seed, 1, keep, Dk, &saved->qx, cells_x, st, 1,
-                            cfg->outlier_cols)) != NVFP4_OK)
+                            cfg->outlier_cols, 0, amax_pass)) != NVFP4_OK)
     return s;
   if ((s = do_quantize_rows(Wp, C, D, ldw, cfg->rounding[1], cfg->seed, 2, keep, Dk, &saved->qw, cells_w, st, 1,
-                            cfg->outlier_cols)) != NVFP4_OK)
+                            cfg->outlier_cols, 0, amax_pass)) != NVFP4_OK)
     return s;
   if (n_out > 0) {
     if (!saved->X_out || !saved->W_out) return NVFP4_ERR_NULL;

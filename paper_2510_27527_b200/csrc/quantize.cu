@@ -15,17 +15,16 @@ namespace nvfp4 {
 // amax pre-passes. Results are bit patterns of non-negative floats combined with atomicMax (order-free, hence
 // deterministic). The cells must be zero before the launch.
 // =========================================================================================================
-__global__ void __launch_bounds__(256) amax_tensor_bf16_kernel(const uint16_t* __restrict__ src, int64_t rows,
-                                                              int64_t cols, int64_t ld, uint32_t* amax_bits) {
-  pdl_prologue();
+__device__ __forceinline__ void amax_tensor_bf16_body(const uint16_t* __restrict__ src, int64_t rows, int64_t cols, int64_t ld,
+                                                      uint32_t* amax_bits, unsigned block, unsigned n_blocks) {
   // One 16-byte chunk (8 BF16) per thread per step; rows are walked through a flattened chunk index.
   const int64_t chunks_per_row = (cols + 7) >> 3;
   const int64_t total = rows * chunks_per_row;
   uint32_t m = 0;
   if (ld == cols && (cols & 7) == 0) {  // one contiguous run of 16-byte chunks: no row arithmetic, four loads in flight
     const uint4* p4 = reinterpret_cast<const uint4*>(src);
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t stride = (int64_t)n_blocks * blockDim.x;
+    int64_t i = (int64_t)block * blockDim.x + threadIdx.x;
     for (; i + 3 * stride < total; i += 4 * stride) {
       const uint4 v0 = p4[i], v1 = p4[i + stride], v2 = p4[i + 2 * stride], v3 = p4[i + 3 * stride];
       const uint32_t a0 = umax16x2(umax16x2(bf16x2_abs_bits(v0.x), bf16x2_abs_bits(v0.y)), umax16x2(bf16x2_abs_bits(v0.z), bf16x2_abs_bits(v0.w)));
@@ -39,7 +38,7 @@ __global__ void __launch_bounds__(256) amax_tensor_bf16_kernel(const uint16_t* _
       m = umax16x2(m, umax16x2(umax16x2(bf16x2_abs_bits(v.x), bf16x2_abs_bits(v.y)), umax16x2(bf16x2_abs_bits(v.z), bf16x2_abs_bits(v.w))));
     }
   } else
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+  for (int64_t i = (int64_t)block * blockDim.x + threadIdx.x; i < total; i += (int64_t)n_blocks * blockDim.x) {
     const int64_t r = i / chunks_per_row, c = (i - r * chunks_per_row) << 3;
     const uint16_t* p = src + r * ld + c;
     if (c + 8 <= cols) {
@@ -60,6 +59,23 @@ __global__ void __launch_bounds__(256) amax_tensor_bf16_kernel(const uint16_t* _
     for (int w = 1; w < 8; ++w) a = max(a, warp_max[w]);
     if (a) atomicMax(amax_bits, a << 16);  // BF16 pattern -> FP32 pattern
   }
+}
+
+__global__ void __launch_bounds__(256) amax_tensor_bf16_kernel(const uint16_t* __restrict__ src, int64_t rows,
+                                                              int64_t cols, int64_t ld, uint32_t* amax_bits) {
+  pdl_prologue();
+  amax_tensor_bf16_body(src, rows, cols, ld, amax_bits, blockIdx.x, gridDim.x);
+}
+
+// Two tensors in one launch (the forward pass's X and W): the first grid_a CTAs take A, the rest take B.
+__global__ void __launch_bounds__(256) amax_tensor_pair_kernel(const uint16_t* __restrict__ a, int64_t rows_a, int64_t cols_a, int64_t ld_a,
+                                                              uint32_t* cell_a, unsigned grid_a, const uint16_t* __restrict__ b,
+                                                              int64_t rows_b, int64_t cols_b, int64_t ld_b, uint32_t* cell_b) {
+  pdl_prologue();
+  if (blockIdx.x < grid_a)
+    amax_tensor_bf16_body(a, rows_a, cols_a, ld_a, cell_a, blockIdx.x, grid_a);
+  else
+    amax_tensor_bf16_body(b, rows_b, cols_b, ld_b, cell_b, blockIdx.x - grid_a, gridDim.x - grid_a);
 }
 
 // amax of a BF16 matrix over all columns EXCEPT a sorted list of excluded ones (OutControl: the outlier channels do not
@@ -855,6 +871,17 @@ cudaError_t launch_amax_tensor(const uint16_t* src, int64_t rows, int64_t cols, 
   const int64_t chunks = rows * ((cols + 7) >> 3);
   const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
   launch_kernel(amax_tensor_bf16_kernel, dim3(grid), dim3(256), 0, st, src, rows, cols, ld, cell);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_amax_tensor_pair(const uint16_t* a, int64_t rows_a, int64_t cols_a, int64_t ld_a, uint32_t* cell_a, const uint16_t* b,
+                                    int64_t rows_b, int64_t cols_b, int64_t ld_b, uint32_t* cell_b, cudaStream_t st) {
+  auto grid_of = [](int64_t rows, int64_t cols) {
+    const int64_t chunks = rows * ((cols + 7) >> 3);
+    return (unsigned)std::max<int64_t>(1, std::min<int64_t>((chunks + 255) / 256, 148 * 8));
+  };
+  const unsigned ga = grid_of(rows_a, cols_a), gb = grid_of(rows_b, cols_b);
+  launch_kernel(amax_tensor_pair_kernel, dim3(ga + gb), dim3(256), 0, st, a, rows_a, cols_a, ld_a, cell_a, ga, b, rows_b, cols_b, ld_b, cell_b);
   return cudaGetLastError();
 }
 
