@@ -439,7 +439,9 @@ static nvfp4_status bwd_dx_impl(const void* dY, int64_t lddy, const nvfp4_saved*
   nvfp4_operand q3, q4;
   if (!carve_operand(cv, &q3, N_tok, C, cfg->gs_mode) || !carve_operand(cv, &q4, D, C, cfg->gs_mode) || !cells3 || !cells4)
     return NVFP4_ERR_WORKSPACE;
-  if (!zero_cells(cells3, cells4, cells_bytes(D, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
+  // with a shared dY amax and a TENSOR -> TENSOR re-quantization (closed-form maximum) no cell of this call is read
+  const bool cells_unused = dy_amax && n_out == 0 && cfg->gs_mode == NVFP4_GS_TENSOR && saved->qw.gs_mode == NVFP4_GS_TENSOR && !cfg->rht;
+  if (!cells_unused && !zero_cells(cells3, cells4, cells_bytes(D, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
   const uint32_t rht = cfg->rht ? kRhtStreamDx : 0u;
   if ((s = do_quantize_rows(static_cast<const uint16_t*>(dY), N_tok, C, lddy, cfg->rounding[2], cfg->seed, 3, nullptr, 0,
                             &q3, dy_amax ? dy_amax : cells3, st, 1, nullptr, rht, dy_amax ? 0 : 1)) != NVFP4_OK)
@@ -548,7 +550,8 @@ static nvfp4_status bwd_dw_impl(const void* dY, int64_t lddy, const nvfp4_saved*
   TransposeSrc t5{};
   t5.bf16 = static_cast<const uint16_t*>(dY);
   t5.ld = lddy;
-  if (!zero_cells(cells5, cells6, cells_bytes(Dk, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
+  const bool cells_unused = dy_amax && cfg->gs_mode == NVFP4_GS_TENSOR && saved->qx.gs_mode == NVFP4_GS_TENSOR && !cfg->rht;
+  if (!cells_unused && !zero_cells(cells5, cells6, cells_bytes(Dk, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
   const uint32_t rht = cfg->rht ? kRhtStreamDw : 0u;
   if ((s = do_quantize_transpose(t5, 0, N_tok, C, cfg->rounding[4], cfg->seed, 5, &q5, dy_amax ? dy_amax : cells5, st, 1, rht,
                                  dy_amax ? 0 : 1)) != NVFP4_OK)

@@ -642,7 +642,8 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
     Sg = global_scale_from_amax(d < D ? __uint_as_float(gs_cells[o]) : 0.0f);
     if (d < D && tid < 64 && blockIdx.x == 0) gscale[o] = Sg;
   } else {
-    float amax = __uint_as_float(gs_cells[0]);
+    // (tensor_closed_form == 2: the cell carries nothing and may be uninitialised)
+    float amax = tensor_closed_form == 2 ? 0.0f : __uint_as_float(gs_cells[0]);
     // TENSOR -> TENSOR re-quantization: the aligned tensor's maximum is float32(2688 * S_global) of the forward
     // operand (its largest block has scale 448 and a magnitude-6 element); gs_cells[0] then only covers BF16 rows.
     if (SRC == 1 && tensor_closed_form) amax = fmaxf(amax, __fmul_rn(2688.0f, s.in_gscale[0]));
@@ -840,13 +841,14 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
   }
   if (a.gs_mode == kGsTensor) {
     if (a.compute_amax) {
-      if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
+      const bool cell_unused = SRC == 1 && a.src.in_gs_mode == kGsTensor && !a.src.row_map;
+      if (!cell_unused && !a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
       if (SRC == 0) {
         const int64_t chunks = a.rowsK * ((a.D + 7) >> 3);
         const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
         launch_kernel(amax_tensor_bf16_kernel, dim3(grid), dim3(256), 0, st, a.src.bf16, a.rowsK, a.D, a.src.ld, a.gs_cells);
       } else if (a.src.in_gs_mode == kGsTensor) {
-        a.tensor_closed_form = 1;  // only the BF16 rows (if any) need a pass
+        a.tensor_closed_form = a.src.row_map ? 1 : 2;  // only the BF16 rows (if any) need a pass
         if (a.src.row_map) {
           launch_kernel(amax_cols_generic_kernel<SRC>, dim3(agrid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.gs_cells, 0, 1);
         }
