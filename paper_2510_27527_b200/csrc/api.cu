@@ -174,7 +174,7 @@ nvfp4_status do_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, in
 // are launched kernel-after-kernel and can overlap their prologues with their predecessors' tails.
 bool zero_cells(uint32_t* first, uint32_t* second, size_t second_bytes, cudaStream_t st) {
   const size_t span = (reinterpret_cast<uint8_t*>(second) - reinterpret_cast<uint8_t*>(first)) + second_bytes;
-  return cudaMemsetAsync(first, 0, span, st) == cudaSuccess;
+  return launch_zero_words(first, (int64_t)((span + 3) / 4), st) == cudaSuccess;
 }
 
 nvfp4_status check_cfg(const nvfp4_layer_cfg* cfg, int64_t D) {
@@ -601,7 +601,7 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, int64_t lddy, const nvfp4_saved* s
     if ((s = check_arch()) != NVFP4_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     shared = reinterpret_cast<uint32_t*>(base + need_dx + need_dw);
-    if (cudaMemsetAsync(shared, 0, sizeof(uint32_t), st) != cudaSuccess) return NVFP4_ERR_CUDA;
+    if (launch_zero_words(shared, 1, st) != cudaSuccess) return NVFP4_ERR_CUDA;
     if (launch_amax_tensor(static_cast<const uint16_t*>(dY), N_tok, C, lddy, shared, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   }
   nvfp4_status s = bwd_dx_impl(dY, lddy, saved, cfg, dX, lddx, base, need_dx, stream, shared);

@@ -91,6 +91,8 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st);
 cudaError_t launch_quantize_transpose(const QuantTransposeArgs& a, cudaStream_t st);
 // amax of a contiguous-row BF16 matrix folded into cells[0] (atomic max; the cell must already hold a valid value)
 cudaError_t launch_amax_tensor(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, uint32_t* cell, cudaStream_t st);
+// p[0 .. n) = 0 by a kernel (keeps the programmatic launch chain intact where a memset node would break it)
+cudaError_t launch_zero_words(uint32_t* p, int64_t n, cudaStream_t st);
 // the same for two matrices in one launch
 cudaError_t launch_amax_tensor_pair(const uint16_t* a, int64_t rows_a, int64_t cols_a, int64_t ld_a, uint32_t* cell_a, const uint16_t* b,
                                     int64_t rows_b, int64_t cols_b, int64_t ld_b, uint32_t* cell_b, cudaStream_t st);

@@ -876,6 +876,17 @@ cudaError_t launch_amax_tensor(const uint16_t* src, int64_t rows, int64_t cols, 
   return cudaGetLastError();
 }
 
+// Clears amax cells with a kernel instead of a memset node, so that the programmatic launch chain is not interrupted.
+__global__ void __launch_bounds__(256) zero_words_kernel(uint32_t* p, int64_t n) {
+  pdl_prologue();
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n; i += (int64_t)gridDim.x * 256) p[i] = 0u;
+}
+cudaError_t launch_zero_words(uint32_t* p, int64_t n, cudaStream_t st) {
+  if (n <= 0) return cudaSuccess;
+  launch_kernel(zero_words_kernel, dim3((unsigned)std::min<int64_t>((n + 255) / 256, 148)), dim3(256), 0, st, p, n);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_amax_tensor_pair(const uint16_t* a, int64_t rows_a, int64_t cols_a, int64_t ld_a, uint32_t* cell_a, const uint16_t* b,
                                     int64_t rows_b, int64_t cols_b, int64_t ld_b, uint32_t* cell_b, cudaStream_t st) {
   auto grid_of = [](int64_t rows, int64_t cols) {
