@@ -37,6 +37,13 @@ __device__ __forceinline__ uint32_t umax16x2(uint32_t a, uint32_t b) {
   const __nv_bfloat162 r = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
   return *reinterpret_cast<const uint32_t*>(&r);
 }
+// max(|a|, |b|) of both halves in one instruction; the sign bits of the result are meaningless (xor of the inputs'),
+// callers mask them off once at the end with bf16x2_abs_bits
+__device__ __forceinline__ uint32_t amax16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
 __device__ __forceinline__ uint32_t hmax_of_pair(uint32_t m) { return max(m & 0xFFFFu, m >> 16); }
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t b16) { return __uint_as_float(b16 << 16); }
 

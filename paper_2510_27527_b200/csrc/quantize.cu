@@ -27,15 +27,15 @@ __device__ __forceinline__ void amax_tensor_bf16_body(const uint16_t* __restrict
     int64_t i = (int64_t)block * blockDim.x + threadIdx.x;
     for (; i + 3 * stride < total; i += 4 * stride) {
       const uint4 v0 = p4[i], v1 = p4[i + stride], v2 = p4[i + 2 * stride], v3 = p4[i + 3 * stride];
-      const uint32_t a0 = umax16x2(umax16x2(bf16x2_abs_bits(v0.x), bf16x2_abs_bits(v0.y)), umax16x2(bf16x2_abs_bits(v0.z), bf16x2_abs_bits(v0.w)));
-      const uint32_t a1 = umax16x2(umax16x2(bf16x2_abs_bits(v1.x), bf16x2_abs_bits(v1.y)), umax16x2(bf16x2_abs_bits(v1.z), bf16x2_abs_bits(v1.w)));
-      const uint32_t a2 = umax16x2(umax16x2(bf16x2_abs_bits(v2.x), bf16x2_abs_bits(v2.y)), umax16x2(bf16x2_abs_bits(v2.z), bf16x2_abs_bits(v2.w)));
-      const uint32_t a3 = umax16x2(umax16x2(bf16x2_abs_bits(v3.x), bf16x2_abs_bits(v3.y)), umax16x2(bf16x2_abs_bits(v3.z), bf16x2_abs_bits(v3.w)));
-      m = umax16x2(m, umax16x2(umax16x2(a0, a1), umax16x2(a2, a3)));
+      const uint32_t a0 = amax16x2(amax16x2(v0.x, v0.y), amax16x2(v0.z, v0.w));
+      const uint32_t a1 = amax16x2(amax16x2(v1.x, v1.y), amax16x2(v1.z, v1.w));
+      const uint32_t a2 = amax16x2(amax16x2(v2.x, v2.y), amax16x2(v2.z, v2.w));
+      const uint32_t a3 = amax16x2(amax16x2(v3.x, v3.y), amax16x2(v3.z, v3.w));
+      m = amax16x2(m, amax16x2(amax16x2(a0, a1), amax16x2(a2, a3)));
     }
     for (; i < total; i += stride) {
       const uint4 v = p4[i];
-      m = umax16x2(m, umax16x2(umax16x2(bf16x2_abs_bits(v.x), bf16x2_abs_bits(v.y)), umax16x2(bf16x2_abs_bits(v.z), bf16x2_abs_bits(v.w))));
+      m = amax16x2(m, amax16x2(amax16x2(v.x, v.y), amax16x2(v.z, v.w)));
     }
   } else
   for (int64_t i = (int64_t)block * blockDim.x + threadIdx.x; i < total; i += (int64_t)n_blocks * blockDim.x) {
@@ -43,13 +43,12 @@ __device__ __forceinline__ void amax_tensor_bf16_body(const uint16_t* __restrict
     const uint16_t* p = src + r * ld + c;
     if (c + 8 <= cols) {
       const uint4 v = *reinterpret_cast<const uint4*>(p);
-      m = umax16x2(m, umax16x2(umax16x2(bf16x2_abs_bits(v.x), bf16x2_abs_bits(v.y)),
-                               umax16x2(bf16x2_abs_bits(v.z), bf16x2_abs_bits(v.w))));
+      m = amax16x2(m, amax16x2(amax16x2(v.x, v.y), amax16x2(v.z, v.w)));
     } else {
-      for (int64_t j = c; j < cols; ++j) m = umax16x2(m, (uint32_t)(p[j - c] & 0x7FFFu));
+      for (int64_t j = c; j < cols; ++j) m = amax16x2(m, (uint32_t)p[j - c]);
     }
   }
-  uint32_t a = hmax_of_pair(m);
+  uint32_t a = hmax_of_pair(bf16x2_abs_bits(m));
 #pragma unroll
   for (int o = 16; o; o >>= 1) a = max(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
   __shared__ uint32_t warp_max[8];
@@ -384,8 +383,8 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
     } else {
       uint32_t m2 = 0;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) m2 = umax16x2(m2, bf16x2_abs_bits(w[j][i]));
-      amax_b_bits = hmax_of_pair(m2) << 16;
+      for (int i = 0; i < 8; ++i) m2 = amax16x2(m2, w[j][i]);
+      amax_b_bits = hmax_of_pair(bf16x2_abs_bits(m2)) << 16;
     }
 
     // ---- global scale -------------------------------------------------------------------------------------
