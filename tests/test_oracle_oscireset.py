@@ -85,3 +85,58 @@ def test_step_zero_clears_the_statistics():
     assert st.D_M.any()
     osc.update_stats(traj[1], st, 0, orc.GS_TENSOR)
     assert not st.D_M.any() and not st.D_Q.any() and np.array_equal(st.W_prev, traj[1])
+
+
+def test_sensitivity_on_a_hand_built_block():
+    """S_global = 1, S_block = 448 (largest element 2688): w / 448 = y sits at a known place in its bin.
+    y = 0.24 rounds to 0 (bin width 0.5): s = 0.48; y = 2.4 rounds to 2 (width 0.75): s = 0.4 / 0.75;
+    y = 3.0 exactly: s = 0; y = 4.9 rounds to 4 (width 1.5): s = 0.6; y = 5.5 rounds to 6 (width 2): s = 0.25."""
+    W = np.zeros((1, 16), dtype=np.float32)
+    W[0, 0] = 2688.0
+    ys = {1: 0.24, 2: 2.4, 3: 3.0, 4: 4.9, 5: 5.5, 6: -1.2}
+    for k, y in ys.items():
+        W[0, k] = np.float32(y * 448.0)
+    s = osc.sensitivity(W, orc.GS_TENSOR)
+    yb = {k: float(osc.bf16_round(np.array([W[0, k]]))[0]) / 448.0 for k in ys}  # what the quantizer sees
+    assert yb[1] < 0.25 and abs(s[0, 1] - abs(ys[1]) / 0.5) < 2e-3
+    assert abs(s[0, 2] - 0.4 / 0.75) < 2e-3 and s[0, 3] == 0.0
+    assert abs(s[0, 4] - 0.9 / 1.5) < 2e-3 and abs(s[0, 5] - 0.5 / 2.0) < 2e-3
+    assert abs(s[0, 6] - 0.2 / 0.5) < 2e-3 and s[0, 0] == 0.0 and s[0, 7] == 0.0
+    # scores never exceed ~2/3 (the wider side of the asymmetric bins of 2 and 4), up to the BF16 cast of the input
+    traj, _ = synth.weight_trajectory(32, 256, 0, seed=2)
+    for gs in MODES:
+        sm = osc.sensitivity(traj[0], gs)
+        assert np.all(sm >= 0) and sm.max() < 0.68 and np.all(np.isfinite(sm))
+
+
+def test_select_tracked_is_top_k_with_index_ties():
+    s = np.array([[0.1, 0.5, 0.5, 0.2], [0.5, 0.0, 0.3, 0.5]], dtype=np.float32)
+    assert osc.select_tracked(s, 3).tolist() == [1, 2, 4]  # three of the four 0.5 scores, lowest indices
+    assert osc.select_tracked(s, 5).tolist() == [1, 2, 4, 6, 7]
+    assert osc.select_tracked(s, 0).tolist() == []
+    rng = np.random.default_rng(0)
+    big = rng.random((7, 33)).astype(np.float32)
+    idx = osc.select_tracked(big, 20)
+    assert len(idx) == 20 and np.all(np.diff(idx) > 0)
+    assert big.reshape(-1)[idx].min() >= np.delete(big.reshape(-1), idx).max()
+
+
+@pytest.mark.parametrize("gs_mode", MODES)
+def test_sparse_statistics_equal_the_dense_ones_on_the_tracked_elements(gs_mode):
+    """Algorithm 3 restricted to idx is Algorithm 2 restricted to idx (same snapshots, same sums)."""
+    traj, _ = synth.weight_trajectory(24, 144, 6, seed=8)
+    dense = osc.Stats(traj[0].shape)
+    n_track = 24 * 144 // 10
+    sp = osc.SparseStats(n_track)
+    for t, W in enumerate(traj):
+        osc.update_stats(W, dense, t, gs_mode)
+        osc.update_stats_sparse(W, sp, t, gs_mode)
+    assert np.array_equal(sp.D_M, dense.D_M.reshape(-1)[sp.idx]) and np.array_equal(sp.D_Q, dense.D_Q.reshape(-1)[sp.idx])
+    # the tracked tenth is strongly enriched in the elements that the dense statistics flag at tau = 8 (base rate 0.1)
+    _, mask = osc.suppress(traj[-1], dense, 8.0, gs_mode)
+    flagged = np.nonzero(mask.reshape(-1))[0]
+    assert len(flagged) > 0 and np.isin(flagged, sp.idx).mean() > 0.3
+    out_s, hit = osc.suppress_sparse(traj[-1], sp, 8.0, gs_mode)
+    out_d, _ = osc.suppress(traj[-1], dense, 8.0, gs_mode)
+    changed = np.nonzero((out_s != traj[-1]).reshape(-1))[0]
+    assert np.all(np.isin(changed, sp.idx)) and np.array_equal(out_s.reshape(-1)[sp.idx], out_d.reshape(-1)[sp.idx])
