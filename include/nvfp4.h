@@ -292,6 +292,32 @@ nvfp4_status nvfp4_osci_suppress(float* W, int64_t ldw, int64_t C, int64_t D, in
                                  const float* D_Q, float tau, unsigned long long* n_reset, void* workspace,
                                  size_t ws_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------------------------
+ * OsciReset, memory-efficient statistics (appendix Algorithm 3, "UpdateOscillationStats_MemoryEfficient"): only the
+ * n_track elements with the largest sensitivity score at t0 = 0 are tracked,
+ *      s = |w - Q(w)| / binwidth(Q(w)),   binwidth = (upper - lower rounding threshold of the E2M1 value) * S_block * S_global
+ * (widths 0.5, 0.5, 0.5, 0.5, 0.75, 1, 1.5, 2 for |P| = 0 .. 6; a block with scale 0 scores 0; binary32, one operation each).
+ *
+ *   State, all caller-owned device arrays of n_track entries: idx (int32 linear index r * D + c, sorted ascending; ties in
+ *   s go to the lower index), WM_prev / WQ_prev (FP32 snapshots of w and Q(w)), D_M / D_Q (FP32 path lengths): 20 B per
+ *   tracked element. C * D must be below 2^31 (NVFP4_ERR_LIMIT).
+ *
+ * nvfp4_osci_sparse_update, t0 = 0: computes the scores, selects idx (radix select + ordered compaction), clears D_M, D_Q
+ *                                   and takes the snapshots.
+ *                           t0 > 0: D_M += |w - WM_prev|; D_Q += |Q(w) - WQ_prev|; snapshots <- current values.
+ * nvfp4_osci_sparse_suppress:       W[idx[i]] = Q(W)[idx[i]] wherever float32(D_Q[i] / D_M[i]) >= tau; Q is taken of the
+ *                                   matrix before any reset (two launches); *n_reset as in nvfp4_osci_suppress.
+ * workspace: nvfp4_osci_sparse_workspace_bytes(C, D, gs_mode, n_track, phase), 256-byte aligned; phase 0 = update with
+ * t0 = 0 (holds one 32-bit score per element of W for the selection), 1 = update with t0 > 0, 2 = suppress.
+ * --------------------------------------------------------------------------------------------------------- */
+size_t nvfp4_osci_sparse_workspace_bytes(int64_t C, int64_t D, int32_t gs_mode, int64_t n_track, int32_t phase);
+nvfp4_status nvfp4_osci_sparse_update(const float* W, int64_t ldw, int64_t C, int64_t D, int32_t gs_mode, int32_t t0,
+                                      int64_t n_track, int32_t* idx, float* WM_prev, float* WQ_prev, float* D_M,
+                                      float* D_Q, void* workspace, size_t ws_bytes, void* stream);
+nvfp4_status nvfp4_osci_sparse_suppress(float* W, int64_t ldw, int64_t C, int64_t D, int32_t gs_mode, int64_t n_track,
+                                        const int32_t* idx, const float* D_M, const float* D_Q, float tau,
+                                        unsigned long long* n_reset, void* workspace, size_t ws_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -83,6 +83,11 @@ EXPORTS = {
     "nvfp4_osci_workspace_bytes": (c_sz, [c_i64, c_i32]),
     "nvfp4_osci_update": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_vp, c_vp, c_vp, c_vp, c_sz, c_vp]),
     "nvfp4_osci_suppress": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_vp, c_vp, ctypes.c_float, c_vp, c_vp, c_sz, c_vp]),
+    "nvfp4_osci_sparse_workspace_bytes": (c_sz, [c_i64, c_i64, c_i32, c_i64, c_i32]),
+    "nvfp4_osci_sparse_update": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_i64, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_sz,
+                                         c_vp]),
+    "nvfp4_osci_sparse_suppress": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i64, c_vp, c_vp, c_vp, ctypes.c_float, c_vp, c_vp,
+                                           c_sz, c_vp]),
 }
 for _name, (_res, _args) in EXPORTS.items():
     _f = getattr(_lib, _name)
@@ -287,6 +292,46 @@ def nvfp4_osci_suppress(W: torch.Tensor, state: OsciState, tau: float, gs_mode: 
     ws = workspace if workspace is not None else _workspace(_lib.nvfp4_osci_workspace_bytes(C, gs_mode), W.device)
     _check(_lib.nvfp4_osci_suppress(_ptr(W), W.stride(0), C, D, gs_mode, _ptr(state.D_M), _ptr(state.D_Q), float(tau), _ptr(n_reset),
                                     _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_osci_suppress")
+
+
+@dataclass
+class OsciSparseState:
+    """State of the memory-efficient oscillation statistics: n_track tracked elements of one weight matrix."""
+
+    idx: torch.Tensor  # int32, linear indices, sorted
+    WM_prev: torch.Tensor
+    WQ_prev: torch.Tensor
+    D_M: torch.Tensor
+    D_Q: torch.Tensor
+
+
+def alloc_osci_sparse_state(n_track: int, device="cuda") -> OsciSparseState:
+    mk = lambda dt: torch.empty(max(n_track, 1), dtype=dt, device=device)[:n_track]
+    return OsciSparseState(mk(torch.int32), mk(torch.float32), mk(torch.float32), mk(torch.float32), mk(torch.float32))
+
+
+def nvfp4_osci_sparse_update(W: torch.Tensor, state: OsciSparseState, t0: int, gs_mode: int = GS_TENSOR,
+                             workspace: torch.Tensor | None = None) -> None:
+    assert W.dtype == torch.float32 and W.dim() == 2 and W.stride(1) == 1
+    C, D = W.shape
+    n = state.idx.numel()
+    ws = workspace if workspace is not None else _workspace(
+        _lib.nvfp4_osci_sparse_workspace_bytes(C, D, gs_mode, n, 0 if t0 == 0 else 1), W.device)
+    _check(_lib.nvfp4_osci_sparse_update(_ptr(W), W.stride(0), C, D, gs_mode, t0, n, _ptr(state.idx), _ptr(state.WM_prev),
+                                         _ptr(state.WQ_prev), _ptr(state.D_M), _ptr(state.D_Q), _ptr(ws), ws.numel(), _stream_ptr()),
+           "nvfp4_osci_sparse_update")
+
+
+def nvfp4_osci_sparse_suppress(W: torch.Tensor, state: OsciSparseState, tau: float, gs_mode: int = GS_TENSOR,
+                               n_reset: torch.Tensor | None = None, workspace: torch.Tensor | None = None) -> None:
+    assert W.dtype == torch.float32 and W.dim() == 2 and W.stride(1) == 1
+    assert n_reset is None or (n_reset.dtype == torch.int64 and n_reset.numel() == 1)
+    C, D = W.shape
+    n = state.idx.numel()
+    ws = workspace if workspace is not None else _workspace(_lib.nvfp4_osci_sparse_workspace_bytes(C, D, gs_mode, n, 2), W.device)
+    _check(_lib.nvfp4_osci_sparse_suppress(_ptr(W), W.stride(0), C, D, gs_mode, n, _ptr(state.idx), _ptr(state.D_M), _ptr(state.D_Q),
+                                           float(tau), _ptr(n_reset), _ptr(ws), ws.numel(), _stream_ptr()),
+           "nvfp4_osci_sparse_suppress")
 
 
 @dataclass

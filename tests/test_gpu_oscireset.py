@@ -90,3 +90,52 @@ def test_reset_leaves_the_forward_weight_operand_unchanged(gs_mode):
     torch.cuda.synchronize()
     assert int(n.item()) > 0
     assert torch.equal(before.codes, after.codes) and torch.equal(before.sf, after.sf) and torch.equal(before.gscale, after.gscale)
+
+
+@pytest.mark.parametrize("shape", [(1, 16), (5, 48), (48, 272), (130, 200), (64, 1024 + 36), (300, 520)])
+@pytest.mark.parametrize("gs_mode", MODES)
+def test_memory_efficient_statistics_bit_exact(shape, gs_mode):
+    """Algorithm 3: tracked index set, snapshots and path lengths identical to the oracle's; the reset as well."""
+    b = B()
+    C, D = shape
+    traj, _ = synth.weight_trajectory(C, D, 4, seed=5 + D)
+    n_track = max(1, (C * D) // 12)
+    ref = osc.SparseStats(n_track)
+    state = b.alloc_osci_sparse_state(n_track)
+    for t, W in enumerate(traj):
+        osc.update_stats_sparse(W, ref, t, gs_mode)
+        b.nvfp4_osci_sparse_update(dev(W, pad=4 if t % 2 else 0), state, t, gs_mode)
+        torch.cuda.synchronize()
+        got_idx = state.idx.cpu().numpy().astype(np.int64)
+        if t == 0:
+            bad = np.nonzero(got_idx != ref.idx)[0]
+            assert len(bad) == 0, f"idx: {len(bad)} differ, first at {bad[:4].tolist()}: {got_idx[bad[:4]].tolist()} vs {ref.idx[bad[:4]].tolist()}"
+        assert np.array_equal(bits(state.WM_prev.cpu().numpy()), bits(ref.WM_prev)), f"WM t={t}"
+        assert np.array_equal(bits(state.WQ_prev.cpu().numpy()), bits(ref.WQ_prev)), f"WQ t={t}"
+        assert np.array_equal(bits(state.D_M.cpu().numpy()), bits(ref.D_M)), f"D_M t={t}"
+        assert np.array_equal(bits(state.D_Q.cpu().numpy()), bits(ref.D_Q)), f"D_Q t={t}"
+    for tau in (8.0, 0.0):
+        want, hit = osc.suppress_sparse(traj[-1], ref, tau, gs_mode)
+        Wd = dev(traj[-1], pad=8)
+        n = torch.zeros(1, dtype=torch.int64, device="cuda")
+        b.nvfp4_osci_sparse_suppress(Wd, state, tau, gs_mode, n_reset=n)
+        torch.cuda.synchronize()
+        assert np.array_equal(bits(Wd.cpu().numpy()), bits(want)), f"sparse suppress tau={tau}"
+        assert int(n.item()) == int(hit.sum())
+
+
+def test_selection_with_massive_ties_and_extreme_counts():
+    """Scores with very few distinct values (a matrix that is already on the grid scores 0 everywhere): the tie rule
+    decides everything; also n_track = all elements."""
+    b = B()
+    C, D = 40, 64
+    W = np.zeros((C, D), dtype=np.float32)
+    W[:, 0] = 6.0  # every block: scale from 6, everything else exactly 0 -> all scores 0
+    W[3, 5] = 0.7  # a single positive score
+    for n_track in (1, 2, 100, C * D):
+        ref = osc.SparseStats(n_track)
+        osc.update_stats_sparse(W, ref, 0, orc.GS_TENSOR)
+        state = b.alloc_osci_sparse_state(n_track)
+        b.nvfp4_osci_sparse_update(dev(W), state, 0, b.GS_TENSOR)
+        torch.cuda.synchronize()
+        assert np.array_equal(state.idx.cpu().numpy().astype(np.int64), ref.idx), n_track
