@@ -450,6 +450,27 @@ def run_aux(args):
         # read W, D_M, D_Q (12 B) (+4 B amax pre-pass); writes only the few reset blocks
         alg = (12.0 + (4.0 if gs != 2 else 0.0)) * C * D
         out[f"osci_suppress_8192x8192_{name}"] = {"us": sec * 1e6, "GBps": alg / sec / 1e9, "frac_hbm_measured": alg / sec / 1e9 / pk["hbm"]}
+    # memory-efficient statistics: 5 % of the elements tracked
+    n_track = C * D // 20
+    for name, gs in GS.items():
+        sp = b.alloc_osci_sparse_state(n_track, dev)
+        ws0 = b._workspace(b.lib.nvfp4_osci_sparse_workspace_bytes(C, D, gs, n_track, 0), dev)
+        ws1 = b._workspace(b.lib.nvfp4_osci_sparse_workspace_bytes(C, D, gs, n_track, 1), dev)
+        sec = t_of(lambda: b.nvfp4_osci_sparse_update(W, sp, 0, gs, workspace=ws0), max(3, args.steps // 2))
+        out[f"osci_sparse_select_8192x8192_{name}"] = {"us": sec * 1e6}
+        flip = [0]
+
+        def upd_s():
+            flip[0] ^= 1
+            b.nvfp4_osci_sparse_update(W1 if flip[0] else W, sp, 1, gs, workspace=ws1)
+
+        sec = t_of(upd_s, args.steps)
+        # bytes moved at most: W read once for the amax pre-pass (per tensor, row or 128-group) + per tracked element its
+        # 64-byte block (blocks are shared between neighbours) and 36 B of state traffic
+        alg = 4.0 * C * D + n_track * (64.0 + 36.0)
+        out[f"osci_sparse_update_8192x8192_{name}"] = {"us": sec * 1e6, "state_bytes_per_param": 20.0 * n_track / (C * D),
+                                                        "GBps_upper_bound_bytes": alg / sec / 1e9}
+        del ws0
     print(json.dumps({"aux": out, "peaks": pk}))
 
 

@@ -40,27 +40,41 @@ __device__ __forceinline__ void store16f(float* __restrict__ row, int64_t k0, in
   }
 }
 
-// In place: w (master values) -> Q(w) for one 16-block. amax_cell: binary32 pattern of the group's amax over the master
-// values (TENSOR / ROW), unused for BLOCK128 where the 8 threads of a 128-group reduce their block maxima by shuffles.
-template <int GS>
-__device__ __forceinline__ void quant_dequant16(float (&w)[16], uint32_t amax_cell) {
+// Q(w) of one 16-block in three steps: BF16 cast + block amax, global scale of its group, scale / round / dequantize.
+// w <- BF16(w) in place; returns the block's amax
+__device__ __forceinline__ float round_block_bf16(float (&w)[16]) {
   float m = 0.0f;
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
     w[i] = bf16_bits_to_float(f32_to_bf16_bits(w[i]));
     m = fmaxf(m, fabsf(w[i]));
   }
-  float Sg;
+  return m;
+}
+// global scale of the block: from the 8 lanes of its 128-group (BLOCK128; every lane of the warp must call this), or from
+// the pre-pass cell, which holds max |w| over the master values (BF16 rounding is monotonic, so rounding it gives
+// max |bf16(w)|)
+template <int GS>
+__device__ __forceinline__ float group_scale(float m, uint32_t amax_cell) {
   if (GS == kGsBlock128) {
     uint32_t g = __float_as_uint(m);
     g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
     g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
     g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 4));
-    Sg = global_scale_from_amax(__uint_as_float(g));
-  } else {
-    // the cell holds max |w| over the master values; BF16 rounding is monotonic, so rounding it gives max |bf16(w)|
-    Sg = global_scale_from_amax(bf16_bits_to_float(f32_to_bf16_bits(__uint_as_float(amax_cell))));
+    return global_scale_from_amax(__uint_as_float(g));
   }
+  return global_scale_from_amax(bf16_bits_to_float(f32_to_bf16_bits(__uint_as_float(amax_cell))));
+}
+__device__ __forceinline__ void quant_block_with(float (&w)[16], float m, float Sg);
+
+template <int GS>
+__device__ __forceinline__ void quant_dequant16(float (&w)[16], uint32_t amax_cell) {
+  const float m = round_block_bf16(w);
+  quant_block_with(w, m, group_scale<GS>(m, amax_cell));
+}
+
+// w (already BF16-rounded, block amax m) -> x_hat for the global scale Sg
+__device__ __forceinline__ void quant_block_with(float (&w)[16], float m, float Sg) {
   float rcp;
   const uint32_t sb = block_scale(m, Sg, rcp);
   // x_hat = (P * S_block) * S_global with P = the E2M1 value nearest to y (ties to the even code, saturating): the
@@ -484,29 +498,46 @@ __global__ void __launch_bounds__(256) osci_scatter_kernel(const uint32_t* __res
   }
 }
 
-// One tracked element per thread (TENSOR / ROW) or per 8 lanes (BLOCK128: each lane quantizes one 16-block of the
-// element's 128-group, the group amax goes round by shuffles). Returns through wm / wq the master value and Q(w) of the
-// element in the lane that owns its block (`mine`); every lane of the warp must call it.
+// amax of every 128-group of a row (BLOCK128 scale mode) as binary32 patterns: cells[r * G + g], G = ceil(D / 128).
+__global__ void __launch_bounds__(256) amax_groups_f32_kernel(const float* __restrict__ W, int64_t ldw, int64_t C, int64_t D,
+                                                             uint32_t* __restrict__ cells) {
+  pdl_prologue();
+  const int64_t nb = ((D + 127) & ~(int64_t)127) >> 4;
+  const int64_t gid = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  const bool active = gid < C * nb;
+  const int64_t r = active ? gid / nb : 0;
+  const int64_t b = active ? gid - r * nb : 0;
+  float w[16];
+  load16f(W + r * ldw, active ? b << 4 : D, D, (ldw & 3) == 0, w);
+  float m = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(w[i]));
+  uint32_t g = __float_as_uint(m);
+  g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
+  g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
+  g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 4));
+  if (active && (b & 7) == 0) cells[r * (nb >> 3) + (b >> 3)] = g;
+}
+
+// One tracked element per thread: its 16-block is loaded and quantized with the global scale looked up in the amax
+// cells (tensor, row, or the element's 128-group). Returns the master value and Q(w) of the element.
 template <int GS>
 __device__ __forceinline__ void tracked_values(const float* __restrict__ W, int64_t ldw, int64_t C, int64_t D,
                                                const uint32_t* __restrict__ cells, int32_t e, bool valid, float& wm, float& wq,
                                                bool& mine) {
   const uint32_t ue = valid ? (uint32_t)e : 0u;
   const uint32_t r = ue / (uint32_t)D, c = ue - r * (uint32_t)D;
-  int64_t k0;
-  if (GS == kGsBlock128) {
-    const uint32_t j = threadIdx.x & 7u;
-    k0 = valid ? (int64_t)((c & ~127u) + 16u * j) : D;
-    mine = valid && j == ((c >> 4) & 7u);
-  } else {
-    k0 = valid ? (int64_t)(c & ~15u) : D;
-    mine = valid;
-  }
+  const int64_t k0 = valid ? (int64_t)(c & ~15u) : D;
+  mine = valid;
   float w[16], q[16];
   load16f(W + (int64_t)r * ldw, k0, D, (ldw & 3) == 0, w);
 #pragma unroll
   for (int i = 0; i < 16; ++i) q[i] = w[i];
-  quant_dequant16<GS>(q, GS == kGsTensor ? cells[0] : GS == kGsRow ? cells[r] : 0u);
+  const float m = round_block_bf16(q);
+  const int64_t G = (D + 127) >> 7;
+  const uint32_t cell = GS == kGsTensor ? cells[0] : GS == kGsRow ? cells[r] : cells[(int64_t)r * G + (c >> 7)];
+  const float Sg = group_scale<kGsTensor>(m, cell);  // the lookup form (no shuffles) in every mode
+  quant_block_with(q, m, Sg);
   wm = 0.0f;
   wq = 0.0f;
   const uint32_t pos = c & 15u;
@@ -526,7 +557,7 @@ __global__ void __launch_bounds__(256) osci_sparse_update_kernel(const float* __
                                                                 int init) {
   pdl_prologue();
   const int64_t gid = (int64_t)blockIdx.x * 256 + threadIdx.x;
-  const int64_t i = GS == kGsBlock128 ? gid >> 3 : gid;
+  const int64_t i = gid;
   const bool valid = i < n_track;
   const int32_t e = valid ? idx[i] : 0;
   float wm, wq;
@@ -553,7 +584,7 @@ __global__ void __launch_bounds__(256) osci_sparse_decide_kernel(const float* __
                                                                 const float* __restrict__ DQ, float tau, float* __restrict__ newval) {
   pdl_prologue();
   const int64_t gid = (int64_t)blockIdx.x * 256 + threadIdx.x;
-  const int64_t i = GS == kGsBlock128 ? gid >> 3 : gid;
+  const int64_t i = gid;
   const bool valid = i < n_track;
   const int32_t e = valid ? idx[i] : 0;
   float wm, wq;
@@ -674,7 +705,7 @@ nvfp4_status nvfp4_osci_suppress(float* W, int64_t ldw, int64_t C, int64_t D, in
 // ---- memory-efficient variant --------------------------------------------------------------------------------
 namespace {
 struct SparseWs {
-  uint32_t* cells;      // amax cells of W (1 word, or C words in the ROW mode)
+  uint32_t* cells;      // amax cells of W: 1 word (TENSOR), C words (ROW), C * ceil(D / 128) words (BLOCK128)
   uint32_t* sel;        // selection phase: 258 words of the radix select
   uint2* cta_counts;    // selection phase: one pair per 4096 elements
   uint32_t* scores;     // selection phase: C * D words
@@ -688,7 +719,7 @@ size_t sparse_ws_layout(int64_t C, int64_t D, int32_t gs_mode, int64_t n_track, 
     off = start + bytes;
     return base ? static_cast<uint8_t*>(base) + start : nullptr;
   };
-  uint8_t* p0 = take(osci_cells(C, gs_mode) * 4);
+  uint8_t* p0 = take((gs_mode == kGsBlock128 ? (size_t)C * (size_t)((D + 127) >> 7) : osci_cells(C, gs_mode)) * 4);
   uint8_t* p1 = take(258 * 4);
   const int64_t n = C * D;
   uint8_t* p2 = take(phase == 0 ? (size_t)((n + 4095) / 4096) * 8 : 0);
@@ -705,7 +736,11 @@ size_t sparse_ws_layout(int64_t C, int64_t D, int32_t gs_mode, int64_t n_track, 
 }
 
 nvfp4_status sparse_amax(const float* W, int64_t ldw, int64_t C, int64_t D, int32_t gs_mode, uint32_t* cells, cudaStream_t st) {
-  if (gs_mode == kGsBlock128) return NVFP4_OK;
+  if (gs_mode == kGsBlock128) {  // every group is written: no clearing needed
+    const int64_t nb = ((D + 127) & ~(int64_t)127) >> 4;
+    launch_kernel(amax_groups_f32_kernel, dim3((unsigned)((C * nb + 255) / 256)), dim3(256), 0, st, W, ldw, C, D, cells);
+    return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+  }
   const int per_row = gs_mode == kGsRow;
   if (launch_zero_words(cells, per_row ? C : 1, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   return run_amax(W, ldw, C, D, cells, per_row, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
@@ -761,7 +796,7 @@ nvfp4_status nvfp4_osci_sparse_update(const float* W, int64_t ldw, int64_t C, in
     if (cudaGetLastError() != cudaSuccess) return NVFP4_ERR_CUDA;
   }
   const int init = t0 == 0 ? 1 : 0;
-  const int64_t threads = gs_mode == kGsBlock128 ? n_track * 8 : n_track;
+  const int64_t threads = n_track;
   const dim3 grid((unsigned)((threads + 255) / 256));
   const int32_t* cidx = idx;
   if (gs_mode == kGsTensor)
@@ -792,7 +827,7 @@ nvfp4_status nvfp4_osci_sparse_suppress(float* W, int64_t ldw, int64_t C, int64_
   nvfp4_status s = sparse_amax(W, ldw, C, D, gs_mode, ws.cells, st);
   if (s != NVFP4_OK) return s;
   const uint32_t* cells = ws.cells;
-  const int64_t threads = gs_mode == kGsBlock128 ? n_track * 8 : n_track;
+  const int64_t threads = n_track;
   const dim3 grid((unsigned)((threads + 255) / 256));
   if (gs_mode == kGsTensor)
     launch_kernel(osci_sparse_decide_kernel<kGsTensor>, grid, dim3(256), 0, st, static_cast<const float*>(W), ldw, C, D, cells, n_track, idx, D_M, D_Q, tau, ws.newval);
