@@ -67,6 +67,29 @@ def test_bad_arguments_are_refused_on_the_host(binding):
     assert L.nvfp4_gemm(ctypes.byref(a), ctypes.byref(lin), 0x5000, 1, 4, 0, None, None, 0, None) == 4  # linear scales
 
 
+def test_bad_arguments_of_the_calibration_and_oscireset_entry_points(binding):
+    L = binding.lib
+    f32 = ctypes.c_float
+    assert L.nvfp4_outlier_accumulate(0, 64, 8, 64, 0x2000, 0x3000, 1 << 20, None) == 1  # null source
+    assert L.nvfp4_outlier_accumulate(0x1000, 60, 8, 64, 0x2000, 0x3000, 1 << 20, None) == 3  # ld < D
+    assert L.nvfp4_outlier_accumulate(0x1000, 64, 8, 64, 0x2000, 0x3000, 16, None) == 5  # workspace too small
+    assert L.nvfp4_outlier_select(0x1000, 8, 9, 0x2000, 0x3000, 0x4000, None) == 2  # n_out > D
+    assert L.nvfp4_outlier_select(0x1000, 8, 2, None, 0x3000, 0x4000, None) == 1  # missing output
+    assert L.nvfp4_osci_update(0x1000, 16, 4, 16, 7, 1, 0x2000, 0x3000, 0x4000, 0x5000, 256, None) == 4  # bad gs_mode
+    assert L.nvfp4_osci_update(0x1000, 8, 4, 16, 0, 1, 0x2000, 0x3000, 0x4000, 0x5000, 256, None) == 2  # ld < D
+    assert L.nvfp4_osci_update(0x1004, 16, 4, 16, 0, 1, 0x2000, 0x3000, 0x4000, 0x5000, 256, None) == 3  # misaligned
+    assert L.nvfp4_osci_suppress(0x1000, 16, 4, 16, 0, None, 0x4000, f32(8.0), None, 0x5000, 256, None) == 1
+    big = 1 << 16
+    assert L.nvfp4_osci_sparse_update(0x1000, big, big, big, 0, 0, 10, 0x2000, 0x3000, 0x4000, 0x5000, 0x6000, 0x7000, 1 << 40,
+                                      None) == 9  # C * D >= 2^31
+    assert L.nvfp4_osci_sparse_update(0x1000, 16, 4, 16, 0, 0, 65, 0x2000, 0x3000, 0x4000, 0x5000, 0x6000, 0x7000, 1 << 20,
+                                      None) == 2  # n_track > C * D
+    assert L.nvfp4_osci_sparse_workspace_bytes(64, 64, 0, 100, 0) > 64 * 64 * 4
+    assert L.nvfp4_osci_sparse_workspace_bytes(64, 64, 0, 100, 1) < 4096
+    assert L.nvfp4_linear_workspace_bytes(binding.OP_BWD, 256, 512, 512, 0, 0) > L.nvfp4_linear_workspace_bytes(
+        binding.OP_BWD_DX, 256, 512, 512, 0, 0)
+
+
 def test_product_does_not_import_the_oracle():
     pkg = os.path.join(ROOT, "paper_2510_27527_b200")
     for dirpath, _, files in os.walk(pkg):

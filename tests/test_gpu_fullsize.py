@@ -105,3 +105,77 @@ def test_largest_sweep_shape_quantize_and_gemm():
     qt = b.nvfp4_quantize(Bd, b.AXIS_COL, b.ROUND_SR, 9, 5, b.GS_BLOCK128)
     ot = orc.quantize(Bm, orc.AXIS_COL, orc.SR, orc.GS_BLOCK128, 9, 5)
     assert_operand_equal(qt, ot, "B^T 8192x8192 SR block128")
+
+
+def test_attention_projection_with_rht_full_size():
+    """The paper's base recipe at the benchmark's size: 1x128 outer-block scales, random Hadamard transformation in the
+    four backward quantizers, through the combined backward entry point that bench.py times."""
+    b = B()
+    c = synth.CONFIGS[2]
+    T, D, C = c["tokens"], 1024, 3072
+    gs_mode = orc.GS_BLOCK128
+    X, W, dY, _ = synth.layer_inputs(2, T, D, C, n_outlier=c["n_outlier"], factor=c["factor"], grad_scale=c["grad_scale"],
+                                     weight_id=10)
+    cfg = b.LayerConfig(gs_mode=gs_mode, seed=0, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32, rht=True)
+    Xd, Wd, dYd = to_dev_bf16(X), to_dev_bf16(W), to_dev_bf16(dY)
+    _, saved = b.nvfp4_linear_fwd(Xd, Wd, cfg)
+    dX, dW = b.nvfp4_linear_bwd(dYd, saved, cfg)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(3)
+    q1 = orc.quantize(X, orc.AXIS_ROW, orc.RTN, gs_mode, 0, 1)
+    q2 = orc.quantize(W, orc.AXIS_ROW, orc.RTN, gs_mode, 0, 2)
+    q3 = orc.quantize(orc.rht16(dY, 0, orc.STREAM_RHT_DX), orc.AXIS_ROW, orc.SR, gs_mode, 0, 3)
+    q4 = orc.quantize(orc.rht16(np.ascontiguousarray(orc.rematerialize_f32(q2).T), 0, orc.STREAM_RHT_DX), orc.AXIS_ROW, orc.SR,
+                      gs_mode, 0, 4)
+    check_sampled(dX, orc.dequantize(q3), orc.dequantize(q4), rng, True, "dX with RHT")
+    q5 = orc.quantize(orc.rht16(np.ascontiguousarray(dY.T), 0, orc.STREAM_RHT_DW), orc.AXIS_ROW, orc.SR, gs_mode, 0, 5)
+    q6 = orc.quantize(orc.rht16(np.ascontiguousarray(orc.rematerialize_f32(q1).T), 0, orc.STREAM_RHT_DW), orc.AXIS_ROW, orc.SR,
+                      gs_mode, 0, 6)
+    check_sampled(dW, orc.dequantize(q5), orc.dequantize(q6), rng, False, "dW with RHT")
+    g3 = b.nvfp4_quantize(dYd, b.AXIS_ROW, b.ROUND_SR, 0, 3, gs_mode, rht_stream_id=7)
+    assert_operand_equal(g3, q3, "Q3(dY S H) full size", k_extended=True)
+    g5 = b.nvfp4_quantize(dYd, b.AXIS_COL, b.ROUND_SR, 0, 5, gs_mode, rht_stream_id=8)
+    assert_operand_equal(g5, q5, "Q5(dY^T S H) full size", k_extended=True)
+    g6 = b.nvfp4_requantize_t(saved.qx, b.ROUND_SR, 0, 6, rht_stream_id=8)
+    assert_operand_equal(g6, q6, "Q6(X-hat^T S H) full size", k_extended=True)
+
+
+def test_oscireset_and_calibration_at_model_size():
+    """A 4096 x 4096 FP32 weight matrix through two statistics steps (dense and memory-efficient) and the reset, and a
+    8192 x 4096 activation through the calibration: bit-exact / within the float32 tolerance against the oracle."""
+    from oracle import calibration as cal
+    from oracle import oscireset as osc
+
+    b = B()
+    C, D = 4096, 4096
+    traj, _ = synth.weight_trajectory(C, D, 2, seed=77)
+    gs = orc.GS_BLOCK128
+    ref, sref = osc.Stats((C, D)), osc.SparseStats(C * D // 20)
+    st = b.alloc_osci_state(torch.from_numpy(traj[0]).cuda())
+    sp = b.alloc_osci_sparse_state(C * D // 20)
+    for t, Wt in enumerate(traj):
+        Wd = torch.from_numpy(Wt).cuda()
+        osc.update_stats(Wt, ref, t, gs)
+        osc.update_stats_sparse(Wt, sref, t, gs)
+        b.nvfp4_osci_update(Wd, st, t, gs)
+        b.nvfp4_osci_sparse_update(Wd, sp, t, gs)
+    torch.cuda.synchronize()
+    u32 = lambda a: np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    assert np.array_equal(u32(st.D_M.cpu().numpy()), u32(ref.D_M)) and np.array_equal(u32(st.D_Q.cpu().numpy()), u32(ref.D_Q))
+    assert np.array_equal(sp.idx.cpu().numpy().astype(np.int64), sref.idx)
+    assert np.array_equal(u32(sp.D_M.cpu().numpy()), u32(sref.D_M)) and np.array_equal(u32(sp.D_Q.cpu().numpy()), u32(sref.D_Q))
+    want, mask = osc.suppress(traj[-1], ref, 8.0, gs)
+    Wd = torch.from_numpy(traj[-1]).cuda()
+    n = torch.zeros(1, dtype=torch.int64, device="cuda")
+    b.nvfp4_osci_suppress(Wd, st, 8.0, gs, n_reset=n)
+    torch.cuda.synchronize()
+    assert np.array_equal(u32(Wd.cpu().numpy()), u32(want)) and int(n.item()) == int(mask.sum())
+    X, ch = synth.activations(8192, 4096, 5, n_outlier=20, factor=30.0)
+    acc = torch.zeros(4096, dtype=torch.float32, device="cuda")
+    b.nvfp4_outlier_accumulate(to_dev_bf16(X), acc)
+    want_acc = cal.accumulate(np.zeros(4096), X)
+    torch.cuda.synchronize()
+    got = acc.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - want_acc) <= 1e-5 * want_acc)
+    outl, _, _ = b.nvfp4_outlier_select(acc, 20)
+    assert outl.cpu().numpy().tolist() == sorted(ch.tolist())
