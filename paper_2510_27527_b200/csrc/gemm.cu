@@ -36,17 +36,19 @@ struct Cfg {
   static constexpr uint32_t SFB_BYTES = (BN / 128) * 2048;
   static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;  // multiple of 1024
   static constexpr int STAGES = (BN == 128) ? 5 : 4;
-  // epilogue staging for bulk tensor stores: per epilogue warp two 32-row x 128-byte buffers (128 x 128 tiles only;
+  // epilogue staging for bulk tensor stores: per epilogue warp one 32-row x 128-byte buffer (128 x 128 tiles only;
   // the 128 x 256 variant has no shared memory left and stores straight from registers)
   static constexpr bool TMA_STORE = (BN == 128);
-  static constexpr uint32_t STAGING_BYTES = TMA_STORE ? 4 * 2 * 4096 : 0;
+  static constexpr uint32_t STAGING_BYTES = TMA_STORE ? 8 * 4096 : 0;
   static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
   // tensor memory columns: two accumulators, then four scale buffers (A: 16 columns, B: 16 * BN / 128)
   static constexpr uint32_t ACC_COLS = BN;
   static constexpr uint32_t ACC_BUFS = (BN == 256) ? 1 : 2;  // 256-wide accumulators leave no room for a second one
   // The single-accumulator variant drains tensor memory into registers first (eight epilogue warps, 128 columns each),
   // hands the accumulator back, and only then scales / converts / stores: the next tile's MMAs run under the stores.
-  static constexpr int EPI_WARPS = (BN == 256) ? 8 : 4;
+  // Eight epilogue warps in both variants: two per tensor-memory lane quadrant, each taking half of the tile's columns
+  // (a 128 x 128 tile's epilogue with four warps took 1.9 us and bounded every product with K <= 1024).
+  static constexpr int EPI_WARPS = 8;
   static constexpr int THREADS = 64 + 32 * EPI_WARPS;
   static constexpr uint32_t SF_COLS = 16 + 16 * (BN / 128);
   static constexpr uint32_t TMEM_COLS = 512;
@@ -497,9 +499,9 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       const int64_t m = (int64_t)mt * BM + quad * 32 + lane;
       float sa = 1.0f;
       if (GS == kGsRow && m < p.M) sa = p.a_gscale[m];
-      if (C::EPI_WARPS == 8) {
+      const int half = (warp - 2) >> 2;  // which half of the tile's columns this warp owns
+      if (BN == 256) {
         // drain this warp's 32 lanes x 128 columns into registers, release the accumulator, then store
-        const int half = (warp - 2) >> 2;
         uint32_t v[4][32];
 #pragma unroll
         for (int q = 0; q < 4; ++q)
@@ -527,11 +529,11 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       if (C::TMA_STORE && p.use_tma_store) {
         // Stage 128-byte row pieces (32 FP32 or 64 BF16 columns) in shared memory with the 128-byte swizzle and let the
         // bulk-tensor engine write them: full lines, clipped at the edges of C, asynchronous.
-        const uint32_t my_stage = staging_base + (uint32_t)(warp - 2) * 8192u;
+        const uint32_t my_stage = staging_base + (uint32_t)(warp - 2) * 4096u;
         const int64_t m0 = (int64_t)mt * BM + quad * 32;
         if (p.c_is_f32) {
 #pragma unroll 1
-          for (int c0 = 0; c0 < BN; c0 += 32) {
+          for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
             uint32_t v[32];
             tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + c0, v);
             tc_wait_ld();
@@ -563,8 +565,8 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 }
               }
             }
-            const uint32_t buf = my_stage + (uint32_t)(chunk_it & 1) * 4096u;
-            if (lane == 0) bulk_wait_read<1>();  // the store that used this buffer two chunks ago has read it
+            const uint32_t buf = my_stage;
+            if (lane == 0) bulk_wait_read<0>();  // the previous store from this buffer has read it
             __syncwarp();
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -584,7 +586,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
           }
         } else {
 #pragma unroll 1
-          for (int c0 = 0; c0 < BN; c0 += 64) {
+          for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 64) {
             uint32_t v[32], v2[32];
             tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + c0, v);
             tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + c0 + 32, v2);
@@ -625,8 +627,8 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 }
               }
             }
-            const uint32_t buf = my_stage + (uint32_t)(chunk_it & 1) * 4096u;
-            if (lane == 0) bulk_wait_read<1>();
+            const uint32_t buf = my_stage;
+            if (lane == 0) bulk_wait_read<0>();
             __syncwarp();
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -651,7 +653,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         }
       } else {
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
+      for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
         uint32_t v[32], vh[32];
         tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + c0, v);
         if (hp_cols) tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + hp_tmem_col + c0, vh);  // warp-uniform condition
@@ -1501,12 +1503,14 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;
   // 128 x 256 tiles halve the operand traffic per flop; they pay off once there are enough of them to fill the SMs.
   const char* force = getenv("NVFP4_GEMM_BN");
-  const bool wide = force ? atoi(force) == 256 : (a.K >= 2048 && ((a.M + 127) / 128) * ((a.N + 255) / 256) >= 2 * sm_count());
+  // (measured on 8192 x 3072 x K: at K = 2048 the 128 x 128 variant, whose two accumulators overlap epilogue and MMAs, is
+  // 39 us against 45-48 us for the wider single-accumulator variants; from K = 4096 on the wider ones win)
+  const bool wide = force ? atoi(force) == 256 : (a.K >= 3072 && ((a.M + 127) / 128) * ((a.N + 255) / 256) >= 2 * sm_count());
   // Pairs of CTAs on 256 x 256 tiles for the largest products. A 256-row tile of an operand spans two 128-row scale
   // tiles, and the last one must exist in full: rows are padded to 128 in the scale layout, so any M, N work.
   const char* pair_env = getenv("NVFP4_GEMM_2CTA");
   const bool pairs = pair_env ? atoi(pair_env) != 0
-                              : (a.K >= 2048 && ((a.M + 255) / 256) * ((a.N + 255) / 256) >= 2 * (sm_count() / 2));
+                              : (a.K >= 3072 && ((a.M + 255) / 256) * ((a.N + 255) / 256) >= 2 * (sm_count() / 2));
   if (a.hp_Kh > 0 && a.gs_mode != kGsBlock128)  // the fused high-precision side product lives in the 128 x 128 variant
     return a.gs_mode == kGsTensor ? launch_variant<kGsTensor, 128>(a, st) : launch_variant<kGsRow, 128>(a, st);
   if (pairs && a.gs_mode == kGsTensor) return launch_2cta<kGsTensor>(a, st);
