@@ -706,10 +706,12 @@ constexpr int B128_STAGES = 4;
 constexpr int B128_NBUF = 3;
 constexpr int B128_MAX_CHUNKS = 128;
 constexpr uint32_t B128_SGB_BYTES = B128_MAX_CHUNKS * 128 * 4;
-constexpr uint32_t B128_SMEM_BYTES = B128_STAGES * Cfg<128>::STAGE_BYTES + B128_SGB_BYTES + 1024 + 256;
+constexpr uint32_t B128_STAGING_BYTES = 4 * 4096;  // one 32-row x 128-byte staging buffer per epilogue warp (bulk stores)
+constexpr uint32_t B128_SMEM_BYTES = B128_STAGES * Cfg<128>::STAGE_BYTES + B128_SGB_BYTES + B128_STAGING_BYTES + 1024 + 256;
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const Params p) {
+gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                           const __grid_constant__ CUtensorMap tmC, const Params p) {
   using C = Cfg<128>;
   constexpr int BN = 128;
   constexpr int STAGES = B128_STAGES;
@@ -717,7 +719,8 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   float* sgb = reinterpret_cast<float*>(smem_gen + STAGES * C::STAGE_BYTES);
-  const uint32_t bar_base = smem_base + STAGES * C::STAGE_BYTES + B128_SGB_BYTES;
+  const uint32_t staging_base = smem_base + STAGES * C::STAGE_BYTES + B128_SGB_BYTES;  // 1024-byte aligned
+  const uint32_t bar_base = staging_base + B128_STAGING_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
   auto part_full_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
@@ -874,7 +877,66 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
         __syncwarp();
         if (lane == 0) mbar_arrive(part_empty_bar(buf));
       }
-      if (ok && m < p.M) {
+      if (ok && p.use_tma_store && !p.addend && !p.accumulate) {
+        // 128-byte row pieces staged in shared memory with the 128-byte swizzle and written by the bulk-tensor engine:
+        // full lines, clipped at the edges of C (a thread-per-row store from registers took longer than the whole
+        // promotion loop of a K = 1024 tile)
+        const uint32_t buf = staging_base + (uint32_t)(warp - 2) * 4096u;
+        const int64_t m0 = (int64_t)mt * BM + quad * 32;
+        // (both loops are fully unrolled: the accumulators must be addressed with compile-time indices)
+        if (p.c_is_f32) {
+#pragma unroll
+          for (int c0 = 0; c0 < 128; c0 += 32) {
+            const int64_t n0 = (int64_t)nt * BN + c0;
+            if (n0 < p.N) {
+              if (lane == 0) bulk_wait_read<0>();  // the previous store from this buffer has read it
+              __syncwarp();
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const float2 a0 = acc[(c0 >> 1) + 2 * j], a1 = acc[(c0 >> 1) + 2 * j + 1];
+                const uint32_t dst = buf + (uint32_t)lane * 128u + (uint32_t)((j ^ (lane & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(__float_as_uint(a0.x)),
+                             "r"(__float_as_uint(a0.y)), "r"(__float_as_uint(a1.x)), "r"(__float_as_uint(a1.y))
+                             : "memory");
+              }
+              fence_async_smem();
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_2d(&tmC, buf, (int32_t)n0, (int32_t)m0);
+                bulk_commit();
+              }
+            }
+          }
+        } else {
+#pragma unroll
+          for (int c0 = 0; c0 < 128; c0 += 64) {
+            const int64_t n0 = (int64_t)nt * BN + c0;
+            if (n0 < p.N) {
+              if (lane == 0) bulk_wait_read<0>();
+              __syncwarp();
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                uint32_t q[4];
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                  const float2 a = acc[(c0 >> 1) + 4 * j + h];
+                  const __nv_bfloat162 hh = __floats2bfloat162_rn(a.x, a.y);
+                  q[h] = *reinterpret_cast<const uint32_t*>(&hh);
+                }
+                const uint32_t dst = buf + (uint32_t)lane * 128u + (uint32_t)((j ^ (lane & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(q[0]), "r"(q[1]), "r"(q[2]), "r"(q[3])
+                             : "memory");
+              }
+              fence_async_smem();
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_2d(&tmC, buf, (int32_t)n0, (int32_t)m0);
+                bulk_commit();
+              }
+            }
+          }
+        }
+      } else if (ok && m < p.M) {
 #pragma unroll
         for (int c0 = 0; c0 < 128; c0 += 32) {
           const int64_t n0 = (int64_t)nt * BN + c0;
@@ -890,6 +952,7 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
         }
       }
     }
+    if (lane == 0) bulk_wait_all();  // this lane's bulk stores are complete before the CTA may exit
   }
 
   tc_fence_before();
@@ -1424,9 +1487,11 @@ cudaError_t launch_2cta(const GemmArgs& a, cudaStream_t st) {
 cudaError_t launch_block128(const GemmArgs& a, cudaStream_t st) {
   const int64_t Kp = (a.K + 127) & ~(int64_t)127;
   if (Kp / 128 > B128_MAX_CHUNKS) return cudaErrorInvalidValue;
-  CUtensorMap tmA, tmB;
+  CUtensorMap tmA, tmB, tmC;
   if (!make_codes_map(&tmA, a.a_codes, a.M, Kp, BM) || !make_codes_map(&tmB, a.b_codes, a.N, Kp, 128)) return cudaErrorInvalidValue;
   Params p{};
+  p.use_tma_store = make_c_map(&tmC, a.C, a.M, a.N, a.ldc, a.c_is_f32 != 0) ? 1 : 0;
+  if (!p.use_tma_store) tmC = tmA;  // unused by the kernel then
   p.a_sf = a.a_sf;
   p.b_sf = a.b_sf;
   p.a_gscale = a.a_gscale;
@@ -1456,7 +1521,7 @@ cudaError_t launch_block128(const GemmArgs& a, cudaStream_t st) {
   }
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
-  launch_kernel(gemm_nvfp4_block128_kernel, dim3(grid), dim3(NUM_THREADS), B128_SMEM_BYTES, st, tmA, tmB, p);
+  launch_kernel(gemm_nvfp4_block128_kernel, dim3(grid), dim3(NUM_THREADS), B128_SMEM_BYTES, st, tmA, tmB, tmC, p);
   return cudaGetLastError();
 }
 
