@@ -382,7 +382,8 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
   const uint16_t* Xp = static_cast<const uint16_t*>(X);
   const uint16_t* Wp = static_cast<const uint16_t*>(W);
   const int32_t* keep = n_out > 0 ? cfg->keep_cols : nullptr;
-  if (!zero_cells(cells_x, cells_w, cells_bytes(C, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
+  // (the 1x128 outer-block mode has no amax cells: its scales come out of the quantizers' own pass)
+  if (cfg->gs_mode != NVFP4_GS_BLOCK128 && !zero_cells(cells_x, cells_w, cells_bytes(C, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
   int amax_pass = 1;
   if (cfg->gs_mode == NVFP4_GS_TENSOR && !keep) {  // the two per-tensor maxima in one launch
     if (launch_amax_tensor_pair(Xp, N_tok, D, ldx, cells_x, Wp, C, D, ldw, cells_w, st) != cudaSuccess) return NVFP4_ERR_CUDA;
@@ -440,7 +441,8 @@ static nvfp4_status bwd_dx_impl(const void* dY, int64_t lddy, const nvfp4_saved*
   if (!carve_operand(cv, &q3, N_tok, C, cfg->gs_mode) || !carve_operand(cv, &q4, D, C, cfg->gs_mode) || !cells3 || !cells4)
     return NVFP4_ERR_WORKSPACE;
   // with a shared dY amax and a TENSOR -> TENSOR re-quantization (closed-form maximum) no cell of this call is read
-  const bool cells_unused = dy_amax && n_out == 0 && cfg->gs_mode == NVFP4_GS_TENSOR && saved->qw.gs_mode == NVFP4_GS_TENSOR && !cfg->rht;
+  const bool cells_unused = cfg->gs_mode == NVFP4_GS_BLOCK128 ||
+                            (dy_amax && n_out == 0 && cfg->gs_mode == NVFP4_GS_TENSOR && saved->qw.gs_mode == NVFP4_GS_TENSOR && !cfg->rht);
   if (!cells_unused && !zero_cells(cells3, cells4, cells_bytes(D, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
   const uint32_t rht = cfg->rht ? kRhtStreamDx : 0u;
   if ((s = do_quantize_rows(static_cast<const uint16_t*>(dY), N_tok, C, lddy, cfg->rounding[2], cfg->seed, 3, nullptr, 0,
@@ -550,7 +552,8 @@ static nvfp4_status bwd_dw_impl(const void* dY, int64_t lddy, const nvfp4_saved*
   TransposeSrc t5{};
   t5.bf16 = static_cast<const uint16_t*>(dY);
   t5.ld = lddy;
-  const bool cells_unused = dy_amax && cfg->gs_mode == NVFP4_GS_TENSOR && saved->qx.gs_mode == NVFP4_GS_TENSOR && !cfg->rht;
+  const bool cells_unused = cfg->gs_mode == NVFP4_GS_BLOCK128 ||
+                            (dy_amax && cfg->gs_mode == NVFP4_GS_TENSOR && saved->qx.gs_mode == NVFP4_GS_TENSOR && !cfg->rht);
   if (!cells_unused && !zero_cells(cells5, cells6, cells_bytes(Dk, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
   const uint32_t rht = cfg->rht ? kRhtStreamDw : 0u;
   if ((s = do_quantize_transpose(t5, 0, N_tok, C, cfg->rounding[4], cfg->seed, 5, &q5, dy_amax ? dy_amax : cells5, st, 1, rht,
