@@ -40,9 +40,12 @@ GS = {"tensor": 0, "row": 1, "block128": 2}
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
 # (default workload, QKV linear, tokens 8192), keyed by the kernel labels of the per-kernel breakdown below.
+# DRAM traffic (dram__bytes_read + dram__bytes_write) of one call = its quantize kernel (ncu capture of this workload) plus
+# its amax pre-pass, which reads the source exactly once (268.4 MB for 134.2 M elements in the 16384 x 8192 capture, scaled
+# to this tensor's 25.17 M elements: 50.33 MB)
 PROFILED_TRAFFIC = {
-    "quantize_cols_dY_SR(Q5)": (51153152, "profiles/quantize_transpose_bf16_sr_attn_dY_8192x3072.txt"),
-    "quantize_rows_dY_SR(Q3)": (50739712, "profiles/quantize_rows_sr_attn_dY_8192x3072.txt"),
+    "quantize_cols_dY_SR(Q5)": (50355968 + 636416 + 50331648, "profiles/quantize_transpose_bf16_sr_attn_dY_8192x3072.txt"),
+    "quantize_rows_dY_SR(Q3)": (50380800 + 246272 + 50331648, "profiles/quantize_rows_sr_attn_dY_8192x3072.txt"),
 }
 
 
