@@ -656,7 +656,7 @@ nvfp4_status nvfp4_osci_update(const float* W, int64_t ldw, int64_t C, int64_t D
   uint32_t* cells = static_cast<uint32_t*>(workspace);
   if (gs_mode != kGsBlock128) {
     const int per_row = gs_mode == kGsRow;
-    if (cudaMemsetAsync(cells, 0, osci_cells(C, gs_mode) * 4, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+    if (launch_zero_words(cells, (int64_t)osci_cells(C, gs_mode), st) != cudaSuccess) return NVFP4_ERR_CUDA;
     if (run_amax(W, ldw, C, D, cells, per_row, st) != cudaSuccess) return NVFP4_ERR_CUDA;
     if (run_amax(W_prev, D, C, D, cells + (per_row ? C : 1), per_row, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   }
@@ -685,7 +685,7 @@ nvfp4_status nvfp4_osci_suppress(float* W, int64_t ldw, int64_t C, int64_t D, in
   uint32_t* cells = static_cast<uint32_t*>(workspace);
   if (gs_mode != kGsBlock128) {
     const int per_row = gs_mode == kGsRow;
-    if (cudaMemsetAsync(cells, 0, osci_cells(C, gs_mode) * 4, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+    if (launch_zero_words(cells, (int64_t)osci_cells(C, gs_mode), st) != cudaSuccess) return NVFP4_ERR_CUDA;
     if (run_amax(W, ldw, C, D, cells, per_row, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   }
   const int64_t nb = ((D + 127) & ~(int64_t)127) >> 4;

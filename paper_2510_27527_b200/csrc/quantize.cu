@@ -750,7 +750,7 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
     if (a.keep) return cudaErrorInvalidValue;
     if (a.gs_mode != kGsBlock128 && (a.gs_mode == kGsRow || a.compute_amax)) {
       const int per_row = a.gs_mode == kGsRow;
-      if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t) * (size_t)(per_row ? a.rows : 1), st)) != cudaSuccess) return e;
+      if (!a.cells_zeroed && (e = launch_zero_words(a.gs_cells, per_row ? a.rows : 1, st)) != cudaSuccess) return e;
       const int64_t blocks16 = a.rows * ((a.K + 15) >> 4);
       const unsigned grid = (unsigned)std::min<int64_t>((blocks16 + 255) / 256, 148 * 16);
       launch_kernel(amax_rows_rht_kernel, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, a.seed, a.rht_stream, a.gs_cells, per_row);
@@ -762,7 +762,7 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
   }
   if (a.gs_mode == kGsTensor) {
     if (a.compute_amax) {
-      if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
+      if (!a.cells_zeroed && (e = launch_zero_words(a.gs_cells, 1, st)) != cudaSuccess) return e;
       if (a.keep && a.excluded && (a.ld & 7) == 0 && a.cols_src <= 256 * 1024) {
         // amax over the kept columns only: full-width vector loads with the excluded (outlier) columns masked out
         const size_t smem = (size_t)((a.cols_src + 31) >> 5) * 4;
@@ -831,7 +831,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
   if (a.rht_stream && a.gs_mode != kGsBlock128) {
     const bool per_row = a.gs_mode == kGsRow;
     if (per_row || a.compute_amax) {
-      if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t) * (size_t)(per_row ? a.D : 1), st)) != cudaSuccess) return e;
+      if (!a.cells_zeroed && (e = launch_zero_words(a.gs_cells, per_row ? a.D : 1, st)) != cudaSuccess) return e;
       e = per_row ? launch_tr_amax_rht<SRC, kGsRow>(a.src, a.rowsK, a.D, a.seed, a.rht_stream, a.gs_cells, st)
                   : launch_tr_amax_rht<SRC, kGsTensor>(a.src, a.rowsK, a.D, a.seed, a.rht_stream, a.gs_cells, st);
       if (e != cudaSuccess) return e;
@@ -841,7 +841,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
   if (a.gs_mode == kGsTensor) {
     if (a.compute_amax) {
       const bool cell_unused = SRC == 1 && a.src.in_gs_mode == kGsTensor && !a.src.row_map;
-      if (!cell_unused && !a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t), st)) != cudaSuccess) return e;
+      if (!cell_unused && !a.cells_zeroed && (e = launch_zero_words(a.gs_cells, 1, st)) != cudaSuccess) return e;
       if (SRC == 0) {
         const int64_t chunks = a.rowsK * ((a.D + 7) >> 3);
         const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
@@ -859,7 +859,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
     return launch_tr_r<SRC, kGsTensor>(a, st);
   }
   if (a.gs_mode == kGsRow) {
-    if (!a.cells_zeroed && (e = cudaMemsetAsync(a.gs_cells, 0, sizeof(uint32_t) * (size_t)a.D, st)) != cudaSuccess) return e;
+    if (!a.cells_zeroed && (e = launch_zero_words(a.gs_cells, a.D, st)) != cudaSuccess) return e;
     launch_kernel(amax_cols_generic_kernel<SRC>, dim3(agrid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.gs_cells, 1, 0);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     return launch_tr_r<SRC, kGsRow>(a, st);
