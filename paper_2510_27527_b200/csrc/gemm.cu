@@ -8,8 +8,10 @@
 //   warp 1      MMA issuer: copies the scales shared -> tensor memory (tcgen05.cp) and issues
 //               tcgen05.mma kind::mxf4nvf4 block_scale (E2M1 data, UE4M3 scale per 16 elements, K = 64 per
 //               instruction, FP32 accumulators in tensor memory, two accumulator buffers).
-//   warps 2..5  epilogue: tcgen05.ld the accumulator, apply the FP32 global scales, add the optional addend,
-//               convert and store.
+//   warps 2..9  epilogue (two warps per tensor-memory lane quadrant, half of the tile's columns each): tcgen05.ld the
+//               accumulator, apply the FP32 global scales, add the optional addend, convert, stage 128-byte row pieces
+//               in shared memory and write them with bulk tensor stores. (The outer-block variant further down keeps
+//               four promotion warps, 2..5.)
 // Every wait on an mbarrier is bounded; when a bound is hit the kernel raises a status word, all roles drain and
 // the CTA frees its tensor memory and exits.
 #include <cuda.h>
@@ -487,7 +489,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   } else {
     // ===================================== epilogue ========================================================
     const int quad = warp & 3;  // tensor-memory lane quadrant this warp may read
-    uint32_t tile_it = 0, chunk_it = 0;
+    uint32_t tile_it = 0;
     bool ok = true;
     float alpha = 1.0f;
     if (GS == kGsTensor) alpha = __fmul_rn(p.a_gscale[0], p.b_gscale[0]);
@@ -582,7 +584,6 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               tma_store_2d(&tmC, buf, (int32_t)n0, (int32_t)m0);
               bulk_commit();
             }
-            ++chunk_it;
           }
         } else {
 #pragma unroll 1
@@ -648,7 +649,6 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               tma_store_2d(&tmC, buf, (int32_t)n0, (int32_t)m0);
               bulk_commit();
             }
-            ++chunk_it;
           }
         }
       } else {
