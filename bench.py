@@ -522,6 +522,11 @@ def run_sweep(args):
         ms = sorted(a.elapsed_time(bb) for a, bb in ev)
         return ms[len(ms) // 2] * 1e-3, ms[0] * 1e-3
 
+    # tensor-core ceiling of this machine under load: the issue loop without memory traffic (4 MMAs of 128 x 256 x 64 per turn)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    probe_flops = b.nvfp4_mma_issue_probe(2048, status)
+    sec, _ = t_of(lambda: b.nvfp4_mma_issue_probe(2048, status), 10)
+    issue_loop_tflops = probe_flops / sec / 1e12 if int(status.item()) == 0 else None
     g = torch.Generator(device=dev)
     g.manual_seed(5)
     for (M, N, K) in shapes:
@@ -553,7 +558,8 @@ def run_sweep(args):
         med, best = t_of(lambda: b.nvfp4_gemm(qa, qb, b.DT_BF16, out=C), n)
         fl = 2.0 * M * N * K
         r["gemm"] = {"us": med * 1e6, "best_us": best * 1e6, "TFLOPs": fl / med / 1e12, "frac_of_4x_bf16_measured": fl / med / 1e12 / (4 * pk["bf16"]),
-                     "frac_of_9PF_nominal": fl / med / 1e12 / 9000.0}
+                     "frac_of_9PF_nominal": fl / med / 1e12 / 9000.0,
+                     "frac_of_issue_loop": (fl / med / 1e12 / issue_loop_tflops) if issue_loop_tflops else None}
 
         def fused():
             b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, out=qa, workspace=ws)
@@ -564,7 +570,7 @@ def run_sweep(args):
         r["quantize_plus_gemm"] = {"us": med * 1e6, "TFLOPs": fl / med / 1e12}
         out.append(r)
         del A, Bm, qa, qb, qat, C
-    print(json.dumps({"sweep": out, "gs_mode": args.gs, "peaks": pk}))
+    print(json.dumps({"sweep": out, "gs_mode": args.gs, "peaks": pk, "mma_issue_loop_TFLOPs": issue_loop_tflops}))
 
 
 def main():

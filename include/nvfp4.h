@@ -182,6 +182,12 @@ size_t nvfp4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
 nvfp4_status nvfp4_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
                         int32_t accumulate, int32_t* dev_status, void* workspace, size_t ws_bytes, void* stream);
 
+/* Measurement aid (the paper has no counterpart): every SM issues iters x 4 block-scaled FP4 MMA instructions
+ * (M = 128, N = 256, K = 64) on tiles resident in shared / tensor memory, no global traffic in the loop. *flops_out (host,
+ * optional) receives the FP4 flops one launch performs; time the launch with events to get this device's tensor-core
+ * ceiling under load. dev_status as in nvfp4_gemm (the kernel's single wait is bounded). 1 <= iters <= 2^20. */
+nvfp4_status nvfp4_mma_issue_probe(int32_t iters, int32_t* dev_status, double* flops_out, void* stream);
+
 /* ---------------------------------------------------------------------------------------------------------
  * The layer (Sec. 2.3; OutControl split of Sec. 4.2). X [N_tok, D], W [C, D], Y / dY [N_tok, C].
  * --------------------------------------------------------------------------------------------------------- */

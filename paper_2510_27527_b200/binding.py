@@ -68,6 +68,7 @@ EXPORTS = {
     "nvfp4_gemm_workspace_bytes": (c_sz, [c_i64, c_i64, c_i64]),
     "nvfp4_gemm": (c_i32, [ctypes.POINTER(COperand), ctypes.POINTER(COperand), c_vp, c_i32, c_i64, c_i32, c_vp, c_vp,
                            c_sz, c_vp]),
+    "nvfp4_mma_issue_probe": (c_i32, [c_i32, c_vp, ctypes.POINTER(ctypes.c_double), c_vp]),
     "nvfp4_linear_workspace_bytes": (c_sz, [c_i32, c_i64, c_i64, c_i64, c_i64, c_i32]),
     "nvfp4_linear_fwd": (c_i32, [c_vp, c_i64, c_vp, c_i64, c_i64, c_i64, c_i64, ctypes.POINTER(CLayerCfg), c_vp, c_i64,
                                  ctypes.POINTER(CSaved), c_vp, c_sz, c_vp]),
@@ -259,6 +260,13 @@ def nvfp4_outlier_select(acc: torch.Tensor, n_out: int):
     cmap = torch.empty(max(D, 1), dtype=torch.int32, device=acc.device)[:D]
     _check(_lib.nvfp4_outlier_select(_ptr(acc), D, n_out, _ptr(outl), _ptr(keep), _ptr(cmap), _stream_ptr()), "nvfp4_outlier_select")
     return outl, keep, cmap
+
+
+def nvfp4_mma_issue_probe(iters: int, dev_status: torch.Tensor | None = None) -> float:
+    """Enqueues the tensor-core issue loop (no memory traffic); returns the FP4 flops the launch performs."""
+    fl = ctypes.c_double(0.0)
+    _check(_lib.nvfp4_mma_issue_probe(iters, _ptr(dev_status), ctypes.byref(fl), _stream_ptr()), "nvfp4_mma_issue_probe")
+    return fl.value
 
 
 @dataclass

@@ -585,6 +585,13 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
   return bwd_dw_impl(dY, lddy, saved, cfg, dW, lddw, workspace, ws_bytes, stream, nullptr);
 }
 
+nvfp4_status nvfp4_mma_issue_probe(int32_t iters, int32_t* dev_status, double* flops_out, void* stream) {
+  if (iters <= 0 || iters > (1 << 20)) return NVFP4_ERR_SHAPE;
+  nvfp4_status s = check_arch();
+  if (s != NVFP4_OK) return s;
+  return launch_mma_issue_probe(iters, dev_status, static_cast<cudaStream_t>(stream), flops_out) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
 nvfp4_status nvfp4_linear_bwd(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg, void* dX,
                               int64_t lddx, void* dW, int64_t lddw, void* workspace, size_t ws_bytes, void* stream) {
   if (!dY || !saved || !cfg || !dX || !dW) return NVFP4_ERR_NULL;

@@ -695,6 +695,69 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 }
 
 // =========================================================================================================
+// Issue-loop probe (a measurement aid, not a step of the method): every SM issues `iters` groups of four
+// tcgen05.mma kind::mxf4nvf4 instructions (M = 128, N = 256, K = 64 each) on operand and scale tiles that stay in
+// shared / tensor memory; no global memory is touched inside the loop. The rate it reaches is the tensor-core
+// ceiling this box gives the FP4 GEMMs at the clocks it runs under load.
+// =========================================================================================================
+constexpr uint32_t PROBE_SMEM_BYTES = 16384 + 32768 + 2048 + 4096 + 1024 + 64;
+
+__global__ void __launch_bounds__(64, 1) mma_issue_probe_kernel(int32_t iters, int32_t* dev_status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t a_tile = smem_base, b_tile = smem_base + 16384, sfa = smem_base + 49152, sfb = sfa + 2048;
+  const uint32_t done_bar = sfb + 4096;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+  const int warp = threadIdx.x >> 5;
+  // operands: the E2M1 code of 1.0 everywhere (0x22), scales: the E4M3 byte of 1.0 (0x38)
+  for (uint32_t i = threadIdx.x; i < (49152u >> 2); i += 64) reinterpret_cast<uint32_t*>(gen)[i] = 0x22222222u;
+  for (uint32_t i = threadIdx.x; i < (6144u >> 2); i += 64) reinterpret_cast<uint32_t*>(gen + 49152)[i] = 0x38383838u;
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    mbar_init(done_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes above, async-proxy reads below
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  pdl_prologue();
+  if (warp == 1) {
+    const uint32_t leader = elect_leader();
+    const uint32_t idesc = instr_desc<256>();
+    const uint32_t sf_tmem = tmem_base + 256;
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      tc_cp_sf(sf_tmem + kk * 4, desc_sf(sfa + kk * 512), leader);
+      tc_cp_sf(sf_tmem + 16 + kk * 8, desc_sf(sfb + kk * 512), leader);
+      tc_cp_sf(sf_tmem + 16 + kk * 8 + 4, desc_sf(sfb + 2048 + kk * 512), leader);
+    }
+    for (int32_t it = 0; it < iters; ++it) {
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk)
+        tc_mma_nvf4(tmem_base, desc_sw128(a_tile + kk * 32), desc_sw128(b_tile + kk * 32), idesc, sf_tmem + kk * 4,
+                    sf_tmem + 16 + kk * 8, (it | kk) != 0, leader);
+    }
+    tc_commit(done_bar, leader);
+    __all_sync(0xFFFFFFFFu, mbar_wait(done_bar, 0, &abort_flag_s, dev_status));  // bounded
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+  }
+}
+
+// =========================================================================================================
 // BLOCK128 variant: the FP32 global scale changes every 128 k (the paper's 1x128 outer block, Sec. 2.2), so a
 // partial product can only be accumulated over 128 k inside tensor memory. The MMA warp writes each 128-k partial
 // (two K = 64 instructions) into one of three tensor-memory buffers; the epilogue warps pull it out and promote it
@@ -1563,6 +1626,19 @@ cudaError_t launch_hp_dw_mma(const uint16_t* dY, int64_t lddy, const uint16_t* X
 
 size_t gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
 int64_t gemm_block128_max_k() { return (int64_t)B128_MAX_CHUNKS * 128; }
+
+cudaError_t launch_mma_issue_probe(int32_t iters, int32_t* dev_status, cudaStream_t st, double* flops) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(mma_issue_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PROBE_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int ctas = sm_count();
+  if (flops) *flops = (double)ctas * (double)iters * 4.0 * 2.0 * 128.0 * 256.0 * 64.0;
+  launch_kernel(mma_issue_probe_kernel, dim3((unsigned)ctas), dim3(64), PROBE_SMEM_BYTES, st, iters, dev_status);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;

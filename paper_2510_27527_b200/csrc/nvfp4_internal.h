@@ -124,6 +124,8 @@ struct GemmArgs {
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
 int64_t gemm_block128_max_k();  // largest K the BLOCK128 GEMM variant takes
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
+// Tensor-core issue loop without memory traffic (measurement aid); *flops = FP4 flops the launch performs.
+cudaError_t launch_mma_issue_probe(int32_t iters, int32_t* dev_status, cudaStream_t st, double* flops);
 
 // High-precision (BF16 inputs, FP32 accumulate) products over OutControl's outlier channels.
 //   fwd: Y[m, n] (+)= sum_j X[m, outl[j]] * W[n, outl[j]]

@@ -156,3 +156,16 @@ def test_block128_scale_layout_one_hot_probe():
         else:
             expect[:, r] += 128
         assert np.array_equal(C, expect), (which, r, g)
+
+
+def test_mma_issue_probe_runs_and_reports_its_work():
+    """The measurement aid: a short issue loop completes (its single wait is bounded) and reports 148-ish SMs' worth of
+    flops; the status word stays 0."""
+    from paper_2510_27527_b200 import binding as b
+
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fl = b.nvfp4_mma_issue_probe(8, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert fl == sms * 8 * 4 * 2.0 * 128 * 256 * 64
