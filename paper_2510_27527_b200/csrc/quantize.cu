@@ -778,7 +778,7 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
         return launch_rows_r<kGsTensor>(a, st);
       }
       const int64_t chunks = a.rows * ((a.cols_src + 7) >> 3);
-      const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
+      const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 8);
       launch_kernel(amax_tensor_bf16_kernel, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.cols_src, a.ld, a.gs_cells);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
@@ -844,7 +844,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
       if (!cell_unused && !a.cells_zeroed && (e = launch_zero_words(a.gs_cells, 1, st)) != cudaSuccess) return e;
       if (SRC == 0) {
         const int64_t chunks = a.rowsK * ((a.D + 7) >> 3);
-        const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
+        const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 8);
         launch_kernel(amax_tensor_bf16_kernel, dim3(grid), dim3(256), 0, st, a.src.bf16, a.rowsK, a.D, a.src.ld, a.gs_cells);
       } else if (a.src.in_gs_mode == kGsTensor) {
         a.tensor_closed_form = a.src.row_map ? 1 : 2;  // only the BF16 rows (if any) need a pass
@@ -870,7 +870,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
 cudaError_t launch_amax_tensor(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, uint32_t* cell, cudaStream_t st) {
   if (rows == 0 || cols == 0) return cudaSuccess;
   const int64_t chunks = rows * ((cols + 7) >> 3);
-  const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 16);
+  const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 8);
   launch_kernel(amax_tensor_bf16_kernel, dim3(grid), dim3(256), 0, st, src, rows, cols, ld, cell);
   return cudaGetLastError();
 }
