@@ -301,17 +301,48 @@ def run_ours(args):
         h2d += layers * (xb.numel() + gb.numel()) * 2
         d2h += layers * (L.Y.numel() * 2 + L.dXo.numel() * 2 + L.dWo.numel() * 4)
 
+    # Three streams: uploads, the library's kernels, downloads. A linear's inputs are uploaded while the previous one
+    # computes and its results are downloaded while the next one computes (the two copy directions use separate engines).
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    for L in lins:
+        L.ev_x, L.ev_dy, L.ev_fwd, L.ev_done, L.ev_drained = (torch.cuda.Event() for _ in range(5))
+        L.used = False
+
     def step_e2e():
+        cur = torch.cuda.current_stream()
+        ev_begin = torch.cuda.Event()
+        ev_begin.record(cur)
+        s_in.wait_event(ev_begin)
+        s_out.wait_event(ev_begin)
         for layer in range(layers):
             for L in lins:
-                L.X.copy_(L.pin[0], non_blocking=True)
-                L.dY.copy_(L.pin[1], non_blocking=True)
+                with torch.cuda.stream(s_in):
+                    if L.used:
+                        s_in.wait_event(L.ev_done)  # the kernels that read these input buffers have finished
+                    L.X.copy_(L.pin[0], non_blocking=True)
+                    L.ev_x.record(s_in)
+                    L.dY.copy_(L.pin[1], non_blocking=True)  # arrives while forward runs and Y leaves
+                    L.ev_dy.record(s_in)
+                cur.wait_event(L.ev_x)
+                if L.used:
+                    cur.wait_event(L.ev_drained)  # the previous results have left the output buffers
                 W = L.W[layer]
                 b.nvfp4_linear_fwd(L.X, W, L.cfg, Y=L.Y, saved=L.saved, workspace=L.ws[0])
+                L.ev_fwd.record(cur)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(L.ev_fwd)
+                    L.out_pin[0].copy_(L.Y, non_blocking=True)
+                cur.wait_event(L.ev_dy)
                 b.nvfp4_linear_bwd(L.dY, L.saved, L.cfg, dX=L.dXo, dW=L.dWo, workspace=L.ws[3])
-                L.out_pin[0].copy_(L.Y, non_blocking=True)
-                L.out_pin[1].copy_(L.dXo, non_blocking=True)
-                L.out_pin[2].copy_(L.dWo, non_blocking=True)
+                L.ev_done.record(cur)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(L.ev_done)
+                    L.out_pin[1].copy_(L.dXo, non_blocking=True)
+                    L.out_pin[2].copy_(L.dWo, non_blocking=True)
+                    L.ev_drained.record(s_out)
+                L.used = True
+        for L in lins:
+            cur.wait_event(L.ev_drained)  # the step ends when its last result is in host memory
 
     e2e_steps = max(2, min(args.steps, 5))
     step_e2e()
