@@ -6,6 +6,8 @@
 // With a non-zero sign stream the backward quantizers first apply the random Hadamard transformation of Sec. 4.1 to each
 // 16-element block along K (the block a thread already holds in registers), and the amax pre-passes see transformed data.
 // All of them are HBM streaming kernels; the launch wrappers at the bottom are called by the C-ABI layer.
+#include <type_traits>
+
 #include "nvfp4_device.cuh"
 #include "nvfp4_internal.h"
 
@@ -298,147 +300,157 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
   // Rows, K and the leading dimension are below 2^31 (checked by the launcher): row / block / column indices are 32-bit,
   // only the final byte offsets are formed in 64 bits (one widening multiply each).
   const uint32_t K32 = (uint32_t)K, ld32 = (uint32_t)ld, nb32 = (uint32_t)nb;
-  uint32_t w[NB][8];
-  int32_t row[NB];
-  uint32_t blk[NB];
-#pragma unroll
-  for (int j = 0; j < NB; ++j) {
-    const int64_t gid = cta_base + j * 256;
-    const bool active = gid < total;
-    uint32_t r = 0, b = 0;
-    if (active) {
-      // gid / nb: by multiply-high when the launcher could prepare the constants (gid < 2^31), else plain division
-      if (div_mul) {
-        const uint32_t n = (uint32_t)gid, t = __umulhi(div_mul, n);
-        r = (t + ((n - t) >> 1)) >> div_shift;
-        b = n - r * nb32;
-      } else if (div_shift != 0xFFFFFFFFu) {
-        r = (uint32_t)gid >> div_shift;
-        b = (uint32_t)gid & (nb32 - 1u);
-      } else {
-        r = (uint32_t)(gid / nb);
-        b = (uint32_t)(gid - (int64_t)r * nb);
-      }
-    }
-    row[j] = active ? (int32_t)r : -1;
-    blk[j] = b;
-    const uint32_t k0 = b << 4;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) w[j][i] = 0;
-    if (active && k0 < K32) {
-      const uint16_t* p = src + (size_t)r * ld32;
-      if (!GATHER && k0 + 16 <= K32) {
-        if (wide_loads) {  // rows start on 32-byte boundaries: one 256-bit load, a warp reads 1 KB contiguously
-          asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                       : "=r"(w[j][0]), "=r"(w[j][1]), "=r"(w[j][2]), "=r"(w[j][3]), "=r"(w[j][4]), "=r"(w[j][5]),
-                         "=r"(w[j][6]), "=r"(w[j][7])
-                       : "l"(p + k0));
+  // Interior CTAs (all of their 1024 blocks exist and are full 16-element blocks) run a copy of the body in which every
+  // bounds check is compiled out; only the last CTA and ragged shapes take the checked copy.
+  auto body = [&](auto full_tag) {
+    constexpr bool FULL = decltype(full_tag)::value;
+    uint32_t w[NB][8];
+    int32_t row[NB];
+    uint32_t blk[NB];
+  #pragma unroll
+    for (int j = 0; j < NB; ++j) {
+      const int64_t gid = cta_base + j * 256;
+      const bool active = FULL || gid < total;
+      uint32_t r = 0, b = 0;
+      if (active) {
+        // gid / nb: by multiply-high when the launcher could prepare the constants (gid < 2^31), else plain division
+        if (div_mul) {
+          const uint32_t n = (uint32_t)gid, t = __umulhi(div_mul, n);
+          r = (t + ((n - t) >> 1)) >> div_shift;
+          b = n - r * nb32;
+        } else if (div_shift != 0xFFFFFFFFu) {
+          r = (uint32_t)gid >> div_shift;
+          b = (uint32_t)gid & (nb32 - 1u);
         } else {
-          const uint4 v0 = *reinterpret_cast<const uint4*>(p + k0);
-          const uint4 v1 = *reinterpret_cast<const uint4*>(p + k0 + 8);
-          w[j][0] = v0.x; w[j][1] = v0.y; w[j][2] = v0.z; w[j][3] = v0.w;
-          w[j][4] = v1.x; w[j][5] = v1.y; w[j][6] = v1.z; w[j][7] = v1.w;
+          r = (uint32_t)(gid / nb);
+          b = (uint32_t)(gid - (int64_t)r * nb);
         }
-      } else if (GATHER && stage_cols8 > 0 && k0 + 16 <= K32) {
-        const uint16_t* sp = row_stage + ((int64_t)r - stage_row0) * stage_cols8;
-        const int4* kp = reinterpret_cast<const int4*>(keep + k0);  // keep is 16-byte aligned, k0 a multiple of 16
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int4 id = kp[q];
-          w[j][2 * q] = (uint32_t)sp[id.x] | ((uint32_t)sp[id.y] << 16);
-          w[j][2 * q + 1] = (uint32_t)sp[id.z] | ((uint32_t)sp[id.w] << 16);
-        }
-      } else {
-        for (int i = 0; i < 16; ++i) {
-          if (k0 + i < K32) {
-            const uint32_t e = GATHER ? p[keep[k0 + i]] : p[k0 + i];
-            w[j][i >> 1] |= e << (16 * (i & 1));
+      }
+      row[j] = active ? (int32_t)r : -1;
+      blk[j] = b;
+      const uint32_t k0 = b << 4;
+  #pragma unroll
+      for (int i = 0; i < 8; ++i) w[j][i] = 0;
+      if (FULL || (active && k0 < K32)) {
+        const uint16_t* p = src + (size_t)r * ld32;
+        if (!GATHER && (FULL || k0 + 16 <= K32)) {
+          if (wide_loads) {  // rows start on 32-byte boundaries: one 256-bit load, a warp reads 1 KB contiguously
+            asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                         : "=r"(w[j][0]), "=r"(w[j][1]), "=r"(w[j][2]), "=r"(w[j][3]), "=r"(w[j][4]), "=r"(w[j][5]),
+                           "=r"(w[j][6]), "=r"(w[j][7])
+                         : "l"(p + k0));
+          } else {
+            const uint4 v0 = *reinterpret_cast<const uint4*>(p + k0);
+            const uint4 v1 = *reinterpret_cast<const uint4*>(p + k0 + 8);
+            w[j][0] = v0.x; w[j][1] = v0.y; w[j][2] = v0.z; w[j][3] = v0.w;
+            w[j][4] = v1.x; w[j][5] = v1.y; w[j][6] = v1.z; w[j][7] = v1.w;
+          }
+        } else if (GATHER && stage_cols8 > 0 && k0 + 16 <= K32) {
+          const uint16_t* sp = row_stage + ((int64_t)r - stage_row0) * stage_cols8;
+          const int4* kp = reinterpret_cast<const int4*>(keep + k0);  // keep is 16-byte aligned, k0 a multiple of 16
+  #pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int4 id = kp[q];
+            w[j][2 * q] = (uint32_t)sp[id.x] | ((uint32_t)sp[id.y] << 16);
+            w[j][2 * q + 1] = (uint32_t)sp[id.z] | ((uint32_t)sp[id.w] << 16);
+          }
+        } else {
+          for (int i = 0; i < 16; ++i) {
+            if (k0 + i < K32) {
+              const uint32_t e = GATHER ? p[keep[k0 + i]] : p[k0 + i];
+              w[j][i >> 1] |= e << (16 * (i & 1));
+            }
           }
         }
       }
     }
-  }
 
-  float Sg_t = 1.0f;
-  if (GS == kGsTensor) {
-    Sg_t = global_scale_from_amax(__uint_as_float(gs_cells[0]));
-    if (blockIdx.x == 0 && threadIdx.x == 0) gscale[0] = Sg_t;
-  }
-
-#pragma unroll
-  for (int j = 0; j < NB; ++j) {
-    const bool active = row[j] >= 0;
-    const uint32_t r = active ? (uint32_t)row[j] : 0u;
-    const uint32_t b = blk[j];
-    const uint32_t k0 = b << 4;
-    float x[16];
-    uint32_t amax_b_bits;  // binary32 pattern of the block's amax (non-negative, so integer order = float order)
-    if (RHT) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        x[2 * i] = bf16_lo(w[j][i]);
-        x[2 * i + 1] = bf16_hi(w[j][i]);
-      }
-      // blocks past K (layout padding up to 128) take no signs, so that they stay +0 and encode as zero bytes
-      rht_scale16(x, k0 < K32 ? rht_sign16(seed, rht_stream, (int64_t)k0) : 0u);
-      hadamard16_butterflies(x);
-      float m = 0.0f;
-#pragma unroll
-      for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(x[i]));
-      amax_b_bits = __float_as_uint(m);
-    } else {
-      uint32_t m2 = 0;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) m2 = amax16x2(m2, w[j][i]);
-      amax_b_bits = hmax_of_pair(bf16x2_abs_bits(m2)) << 16;
+    float Sg_t = 1.0f;
+    if (GS == kGsTensor) {
+      Sg_t = global_scale_from_amax(__uint_as_float(gs_cells[0]));
+      if (blockIdx.x == 0 && threadIdx.x == 0) gscale[0] = Sg_t;
     }
 
-    // ---- global scale -------------------------------------------------------------------------------------
-    float Sg;
-    if (GS == kGsBlock128) {
-      uint32_t g = amax_b_bits;
-      g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
-      g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
-      g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 4));
-      Sg = global_scale_from_amax(__uint_as_float(g));
-      if (active && (b & 7) == 0) gscale[(size_t)r * (uint32_t)(Kp >> 7) + (b >> 3)] = Sg;
-    } else if (GS == kGsRow) {
-      Sg = global_scale_from_amax(__uint_as_float(gs_cells[r]));
-      if (active && b == 0) gscale[r] = Sg;
-    } else {
-      Sg = Sg_t;
-    }
-
-    // ---- block scale, rounding, packing -------------------------------------------------------------------
-    float rcp;
-    const uint32_t sb = block_scale(__uint_as_float(amax_b_bits), Sg, rcp);
-    if (!RHT) {
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        x[2 * i] = bf16_lo(w[j][i]);
-        x[2 * i + 1] = bf16_hi(w[j][i]);
-      }
-    }
-    const uint2 packed = quantize_block16<SR>(x, rcp, seed, stream_id, ((uint64_t)r * (uint32_t)K16 + k0) >> 3);
-
-    // four neighbouring threads own the four scale bytes of one 32-bit word in either layout
-    uint32_t sf4 = sb << (8 * (b & 3));
-    sf4 |= __shfl_xor_sync(0xFFFFFFFFu, sf4, 1);
-    sf4 |= __shfl_xor_sync(0xFFFFFFFFu, sf4, 2);
-    if (active) {
-      *reinterpret_cast<uint2*>(codes + (size_t)r * (uint32_t)(Kp >> 1) + (k0 >> 1)) = packed;
-      if ((b & 3) == 0) {
-        size_t off;
-        if (TILED) {
-          const uint32_t tile = (r >> 7) * (((nb32 + 15u) & ~15u) >> 2) + (b >> 2);  // 512-byte tiles, k fastest
-          off = (size_t)tile * 512u + ((r & 31u) * 16u + ((r >> 5) & 3u) * 4u);       // b & 3 == 0 here
-        } else {
-          off = (size_t)r * nb32 + b;
+  #pragma unroll
+    for (int j = 0; j < NB; ++j) {
+      const bool active = FULL || row[j] >= 0;
+      const uint32_t r = active ? (uint32_t)row[j] : 0u;
+      const uint32_t b = blk[j];
+      const uint32_t k0 = b << 4;
+      float x[16];
+      uint32_t amax_b_bits;  // binary32 pattern of the block's amax (non-negative, so integer order = float order)
+      if (RHT) {
+  #pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          x[2 * i] = bf16_lo(w[j][i]);
+          x[2 * i + 1] = bf16_hi(w[j][i]);
         }
-        *reinterpret_cast<uint32_t*>(sf + off) = sf4;
+        // blocks past K (layout padding up to 128) take no signs, so that they stay +0 and encode as zero bytes
+        rht_scale16(x, (FULL || k0 < K32) ? rht_sign16(seed, rht_stream, (int64_t)k0) : 0u);
+        hadamard16_butterflies(x);
+        float m = 0.0f;
+  #pragma unroll
+        for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(x[i]));
+        amax_b_bits = __float_as_uint(m);
+      } else {
+        uint32_t m2 = 0;
+  #pragma unroll
+        for (int i = 0; i < 8; ++i) m2 = amax16x2(m2, w[j][i]);
+        amax_b_bits = hmax_of_pair(bf16x2_abs_bits(m2)) << 16;
+      }
+
+      // ---- global scale -------------------------------------------------------------------------------------
+      float Sg;
+      if (GS == kGsBlock128) {
+        uint32_t g = amax_b_bits;
+        g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));
+        g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 2));
+        g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 4));
+        Sg = global_scale_from_amax(__uint_as_float(g));
+        if (active && (b & 7) == 0) gscale[(size_t)r * (uint32_t)(Kp >> 7) + (b >> 3)] = Sg;
+      } else if (GS == kGsRow) {
+        Sg = global_scale_from_amax(__uint_as_float(gs_cells[r]));
+        if (active && b == 0) gscale[r] = Sg;
+      } else {
+        Sg = Sg_t;
+      }
+
+      // ---- block scale, rounding, packing -------------------------------------------------------------------
+      float rcp;
+      const uint32_t sb = block_scale(__uint_as_float(amax_b_bits), Sg, rcp);
+      if (!RHT) {
+  #pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          x[2 * i] = bf16_lo(w[j][i]);
+          x[2 * i + 1] = bf16_hi(w[j][i]);
+        }
+      }
+      const uint2 packed = quantize_block16<SR>(x, rcp, seed, stream_id, ((uint64_t)r * (uint32_t)K16 + k0) >> 3);
+
+      // four neighbouring threads own the four scale bytes of one 32-bit word in either layout
+      uint32_t sf4 = sb << (8 * (b & 3));
+      sf4 |= __shfl_xor_sync(0xFFFFFFFFu, sf4, 1);
+      sf4 |= __shfl_xor_sync(0xFFFFFFFFu, sf4, 2);
+      if (active) {
+        *reinterpret_cast<uint2*>(codes + (size_t)r * (uint32_t)(Kp >> 1) + (k0 >> 1)) = packed;
+        if ((b & 3) == 0) {
+          size_t off;
+          if (TILED) {
+            const uint32_t tile = (r >> 7) * (((nb32 + 15u) & ~15u) >> 2) + (b >> 2);  // 512-byte tiles, k fastest
+            off = (size_t)tile * 512u + ((r & 31u) * 16u + ((r >> 5) & 3u) * 4u);       // b & 3 == 0 here
+          } else {
+            off = (size_t)r * nb32 + b;
+          }
+          *reinterpret_cast<uint32_t*>(sf + off) = sf4;
+        }
       }
     }
-  }
+  };
+  const bool full = !GATHER && K32 == (uint32_t)Kp && (int64_t)blockIdx.x * (256 * NB) + 256 * NB <= total;  // CTA-uniform
+  if (full)
+    body(std::true_type{});
+  else
+    body(std::false_type{});
 }
 
 // =========================================================================================================
