@@ -114,24 +114,29 @@ class ClockSampler:
 # ---------------------------------------------------------------------------------------------------------------
 # the oracle arm (CPU): used for --impl reference and for the cpu_baseline leg of the default arm
 # ---------------------------------------------------------------------------------------------------------------
-def oracle_sample_step(workload: str, gs_mode: int, sample_tokens: int = 256, rht: bool = False):
-    """One forward + dX + dW of the workload's first linear on a slab of `sample_tokens` tokens, through the
-    oracle as it stands. Returns (seconds, flops of the sample, description)."""
+def oracle_sample_step(workload: str, gs_mode: int, sample_tokens: int = 256, rht: bool = False, all_linears: bool = False):
+    """One forward + dX + dW on a slab of `sample_tokens` tokens, through the oracle as it stands: of the workload's first
+    linear, or (all_linears) of every linear of one layer. Returns (seconds, flops of the sample, description)."""
     from oracle import nvfp4_oracle as orc
 
     cfg_id, tokens, linears = WORKLOADS[workload]
-    name, D, C, swiglu = linears[0]
     c = synth.CONFIGS[cfg_id]
-    X, W, dY, _ = synth.layer_inputs(cfg_id, sample_tokens, D, C, n_outlier=c["n_outlier"], factor=c["factor"],
-                                     grad_scale=c["grad_scale"], swiglu=swiglu)
+    chosen = linears if all_linears else linears[:1]
+    inputs = []
+    for li, (name, D, C, swiglu) in enumerate(chosen):
+        inputs.append(synth.layer_inputs(cfg_id, sample_tokens, D, C, n_outlier=c["n_outlier"], factor=c["factor"],
+                                         grad_scale=c["grad_scale"], swiglu=swiglu, weight_id=10 + li))
     orc.lib()
     t0 = time.perf_counter()
     ocfg = orc.LayerConfig(gs_mode=gs_mode, seed=0, rht=rht)
-    _, saved = orc.linear_fwd(X, W, ocfg)
-    orc.linear_bwd_dx(dY, saved, ocfg)
-    orc.linear_bwd_dw(dY, saved, ocfg)
+    for X, W, dY, _ in inputs:
+        _, saved = orc.linear_fwd(X, W, ocfg)
+        orc.linear_bwd_dx(dY, saved, ocfg)
+        orc.linear_bwd_dw(dY, saved, ocfg)
     dt = time.perf_counter() - t0
-    return dt, 6.0 * sample_tokens * D * C, f"{name} linear {D}->{C}, {sample_tokens}-token slab of the {tokens}-token workload, fwd+dX+dW"
+    fl = sum(6.0 * sample_tokens * D * C for _, D, C, _ in chosen)
+    names = " + ".join(f"{name} {D}->{C}" for name, D, C, _ in chosen)
+    return dt, fl, f"linear(s) {names}, {sample_tokens}-token slab of the {tokens}-token workload, fwd+dX+dW"
 
 
 def run_reference(args):
@@ -415,7 +420,7 @@ def run_ours(args):
     if world == 1 and not args.no_cpu:
         from oracle import nvfp4_oracle as orc
 
-        dt, sfl, desc = oracle_sample_step(args.workload, gs_mode, args.cpu_tokens, args.rht)
+        dt, sfl, desc = oracle_sample_step(args.workload, gs_mode, args.cpu_tokens, args.rht, all_linears=True)
         cpu = {"value": sfl / dt / 1e12, "unit": "TFLOP/s", "cores": orc.threads(), "kind": "oracle", "sample": desc,
                "seconds": dt}
 
@@ -613,7 +618,7 @@ def main():
     ap.add_argument("--workload", default="attn", choices=list(WORKLOADS))
     ap.add_argument("--gs", default="tensor", choices=list(GS))
     ap.add_argument("--ref-tokens", type=int, default=1024, help="token slab of one oracle step (reference arm)")
-    ap.add_argument("--cpu-tokens", type=int, default=4096, help="token slab of the cpu_baseline leg")
+    ap.add_argument("--cpu-tokens", type=int, default=8192, help="token slab of the cpu_baseline leg (every linear of one layer)")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--outliers", type=float, default=0.0,
                     help="OutControl: fraction of input channels kept in BF16 (0 = off; the paper uses 0.10)")
