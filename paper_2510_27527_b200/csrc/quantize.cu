@@ -832,13 +832,19 @@ static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-// amax pre-pass over the transformed source: the quantizer's own tile walk, stopped after the block maxima
+// amax pre-pass with the quantizer's own tile walk, stopped after the block maxima (its vectorised staging decodes a
+// forward operand several times faster than the element-wise column kernel; under the Hadamard transformation it is the
+// only pass that sees the transformed values)
 template <int SRC, int GS>
 static cudaError_t launch_tr_amax_rht(const TransposeSrc& src, int64_t rowsK, int64_t D, uint64_t seed, uint32_t rht_stream,
                                       uint32_t* cells, cudaStream_t st) {
   const dim3 grid(blocks_for(rowsK, 128), blocks_for(D, 64));
-  launch_kernel(quantize_transpose_kernel<SRC, GS, false, false, true, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
-                0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), rht_stream);
+  if (rht_stream)
+    launch_kernel(quantize_transpose_kernel<SRC, GS, false, false, true, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
+                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), rht_stream);
+  else
+    launch_kernel(quantize_transpose_kernel<SRC, GS, false, false, false, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
+                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), 0u);
   return cudaGetLastError();
 }
 
@@ -877,7 +883,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
           launch_kernel(amax_cols_generic_kernel<SRC>, dim3(agrid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.gs_cells, 0, 1);
         }
       } else {
-        launch_kernel(amax_cols_generic_kernel<SRC>, dim3(agrid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.gs_cells, 0, 0);
+        if ((e = launch_tr_amax_rht<SRC, kGsTensor>(a.src, a.rowsK, a.D, a.seed, 0u, a.gs_cells, st)) != cudaSuccess) return e;
       }
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
@@ -885,8 +891,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
   }
   if (a.gs_mode == kGsRow) {
     if (!a.cells_zeroed && (e = launch_zero_words(a.gs_cells, a.D, st)) != cudaSuccess) return e;
-    launch_kernel(amax_cols_generic_kernel<SRC>, dim3(agrid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.gs_cells, 1, 0);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = launch_tr_amax_rht<SRC, kGsRow>(a.src, a.rowsK, a.D, a.seed, 0u, a.gs_cells, st)) != cudaSuccess) return e;
     return launch_tr_r<SRC, kGsRow>(a, st);
   }
   return launch_tr_r<SRC, kGsBlock128>(a, st);
