@@ -202,6 +202,21 @@ __device__ __forceinline__ uint64_t desc_sw128(uint32_t saddr) {
 __device__ __forceinline__ uint64_t desc_sf(uint32_t saddr) {
   return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)8 << 32) | ((uint64_t)1 << 46);
 }
+// The 32 per-row global scales SgB[n0 .. n0 + 32) of a ROW-mode B operand (0 beyond N); every lane reads the same values, in
+// four-wide loads when the run lies inside the matrix and is 16-byte aligned.
+__device__ __forceinline__ void load_sgb32(const float* __restrict__ g, int64_t n0, int64_t N, float (&out)[32]) {
+  if (n0 + 32 <= N && (reinterpret_cast<uintptr_t>(g + n0) & 15u) == 0) {
+    const float4* g4 = reinterpret_cast<const float4*>(g + n0);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const float4 t = __ldg(g4 + q);
+      out[4 * q] = t.x; out[4 * q + 1] = t.y; out[4 * q + 2] = t.z; out[4 * q + 3] = t.w;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) out[j] = (n0 + j < N) ? __ldg(g + n0 + j) : 0.0f;
+  }
+}
 // Instruction descriptor: E2M1 x E2M1, UE4M3 scales, M = 128, N = BN, both operands k-major, K = 64.
 template <int BN>
 __device__ __forceinline__ uint32_t instr_desc() {
@@ -516,11 +531,12 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         for (int q = 0; q < 4; ++q) {
           const int64_t n0 = (int64_t)nt * BN + half * 128 + q * 32;
           if (m < p.M && n0 < p.N) {
-            float o[32];
+            float o[32], sgb[32];
+            if (GS == kGsRow) load_sgb32(p.b_gscale, n0, p.N, sgb);
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               float sc = alpha;
-              if (GS == kGsRow) sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
+              if (GS == kGsRow) sc = __fmul_rn(sa, sgb[j]);
               o[j] = __uint_as_float(v[q][j]) * sc;
             }
             store_row_chunk(p, m, n0, o);
@@ -541,11 +557,12 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             tc_wait_ld();
             const int64_t n0 = (int64_t)nt * BN + c0;
             if (n0 >= p.N) break;
-            float o[32];
+            float o[32], sgb[32];
+            if (GS == kGsRow) load_sgb32(p.b_gscale, n0, p.N, sgb);
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               float sc = alpha;
-              if (GS == kGsRow) sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
+              if (GS == kGsRow) sc = __fmul_rn(sa, sgb[j]);
               o[j] = __uint_as_float(v[j]) * sc;
             }
             if (hp_cols) {
@@ -595,15 +612,14 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             const int64_t n0 = (int64_t)nt * BN + c0;
             if (n0 >= p.N) break;
             float o[64];
+            {
+              float sgb[32];
+              if (GS == kGsRow) load_sgb32(p.b_gscale, n0, p.N, sgb);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              float sc = alpha, sc2 = alpha;
-              if (GS == kGsRow) {
-                sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
-                sc2 = __fmul_rn(sa, (n0 + 32 + j < p.N) ? __ldg(p.b_gscale + n0 + 32 + j) : 0.0f);
-              }
-              o[j] = __uint_as_float(v[j]) * sc;
-              o[32 + j] = __uint_as_float(v2[j]) * sc2;
+              for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(v[j]) * (GS == kGsRow ? __fmul_rn(sa, sgb[j]) : alpha);
+              if (GS == kGsRow) load_sgb32(p.b_gscale, n0 + 32, p.N, sgb);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) o[32 + j] = __uint_as_float(v2[j]) * (GS == kGsRow ? __fmul_rn(sa, sgb[j]) : alpha);
             }
             if (hp_cols) {
               tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + hp_tmem_col + c0, v);
@@ -660,11 +676,12 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         tc_wait_ld();
         const int64_t n0 = (int64_t)nt * BN + c0;
         if (m < p.M && n0 < p.N) {
-          float o[32];
+          float o[32], sgb[32];
+          if (GS == kGsRow) load_sgb32(p.b_gscale, n0, p.N, sgb);
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             float sc = alpha;
-            if (GS == kGsRow) sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
+            if (GS == kGsRow) sc = __fmul_rn(sa, sgb[j]);
             o[j] = __uint_as_float(v[j]) * sc;
           }
           if (hp_cols) {
@@ -1235,11 +1252,12 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       for (int q = 0; q < 4; ++q) {
         const int64_t n0 = (int64_t)nt * 256 + half * 128 + q * 32;
         if (m < p.M && n0 < p.N) {
-          float o[32];
+          float o[32], sgb[32];
+          if (GS == kGsRow) load_sgb32(p.b_gscale, n0, p.N, sgb);
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             float sc = alpha;
-            if (GS == kGsRow) sc = __fmul_rn(sa, (n0 + j < p.N) ? __ldg(p.b_gscale + n0 + j) : 0.0f);
+            if (GS == kGsRow) sc = __fmul_rn(sa, sgb[j]);
             o[j] = __uint_as_float(v[q][j]) * sc;
           }
           store_row_chunk(p, m, n0, o);
