@@ -114,10 +114,36 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
   }
   return make_uint4(c0, c1, c2, c3);
 }
+// The ten round keys of a 64-bit Philox key, prepared on the host and handed to the kernels as a constant parameter:
+// the rounds then read them as constant-bank operands instead of carrying two running additions per round.
+struct PhiloxKeys {
+  uint32_t k0[10], k1[10];
+};
+inline PhiloxKeys make_philox_keys(uint64_t seed) {
+  PhiloxKeys r;
+  uint32_t a = (uint32_t)seed, b = (uint32_t)(seed >> 32);
+  for (int i = 0; i < 10; ++i) {
+    r.k0[i] = a;
+    r.k1[i] = b;
+    a += 0x9E3779B9u;
+    b += 0xBB67AE85u;
+  }
+  return r;
+}
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const PhiloxKeys& rk) {
+#pragma unroll
+  for (int i = 0; i < 10; ++i) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk.k0[i];
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk.k1[i];
+    c0 = n0; c1 = (uint32_t)p1; c2 = n2; c3 = (uint32_t)p0;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
 // The four 32-bit words holding the 16-bit draws of elements idx8*8 .. idx8*8+7 of the operand.
-__device__ __forceinline__ uint4 sr_words(uint64_t seed, uint32_t stream_id, uint64_t idx8) {
-  return philox4x32_10((uint32_t)idx8, (uint32_t)(idx8 >> 32), stream_id, 0u, (uint32_t)seed,
-                       (uint32_t)(seed >> 32));
+__device__ __forceinline__ uint4 sr_words(const PhiloxKeys& rk, uint32_t stream_id, uint64_t idx8) {
+  return philox4x32_10((uint32_t)idx8, (uint32_t)(idx8 >> 32), stream_id, 0u, rk);
 }
 
 // ---------------------------------------------------------------------------------------------------------

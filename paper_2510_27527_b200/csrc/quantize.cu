@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(256) amax_rows_rht_kernel(const uint16_t* __re
 // Shared epilogue of one 16-element inner block: scale, round, pack.
 // =========================================================================================================
 template <bool SR>
-__device__ __forceinline__ uint2 quantize_block16(const float (&x)[16], float rcp, uint64_t seed, uint32_t stream_id,
+__device__ __forceinline__ uint2 quantize_block16(const float (&x)[16], float rcp, const PhiloxKeys& pk, uint32_t stream_id,
                                                   uint64_t idx8) {
   float y0[8], y1[8];
 #pragma unroll
@@ -239,8 +239,8 @@ __device__ __forceinline__ uint2 quantize_block16(const float (&x)[16], float rc
   }
   uint2 out;
   if (SR) {
-    out.x = e2m1x8_sr(y0, sr_words(seed, stream_id, idx8));
-    out.y = e2m1x8_sr(y1, sr_words(seed, stream_id, idx8 + 1));
+    out.x = e2m1x8_sr(y0, sr_words(pk, stream_id, idx8));
+    out.y = e2m1x8_sr(y1, sr_words(pk, stream_id, idx8 + 1));
   } else {
     out.x = e2m1x8_rtn(y0);
     out.y = e2m1x8_rtn(y1);
@@ -261,7 +261,7 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
                      const int32_t* __restrict__ keep, uint64_t seed, uint32_t stream_id,
                      const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
                      float* __restrict__ gscale, uint32_t div_mul, uint32_t div_shift, int wide_loads, int64_t cols_src,
-                     int64_t stage_cols8, uint32_t rht_stream) {
+                     int64_t stage_cols8, uint32_t rht_stream, const __grid_constant__ PhiloxKeys pk) {
   pdl_prologue();
   constexpr int NB = 4;  // inner blocks per thread; all loads are issued before any arithmetic
   extern __shared__ uint16_t row_stage[];  // GATHER only: the source rows this CTA touches, [n_rows][cols_src8]
@@ -425,7 +425,7 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
           x[2 * i + 1] = bf16_hi(w[j][i]);
         }
       }
-      const uint2 packed = quantize_block16<SR>(x, rcp, seed, stream_id, ((uint64_t)r * (uint32_t)K16 + k0) >> 3);
+      const uint2 packed = quantize_block16<SR>(x, rcp, pk, stream_id, ((uint64_t)r * (uint32_t)K16 + k0) >> 3);
 
       // four neighbouring threads own the four scale bytes of one 32-bit word in either layout
       uint32_t sf4 = sb << (8 * (b & 3));
@@ -531,7 +531,8 @@ template <int SRC, int GS, bool SR, bool TILED, bool RHT, bool AMAX_ONLY>
 __global__ void __launch_bounds__(256)
 quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t seed, uint32_t stream_id,
                           uint32_t* __restrict__ gs_cells, int tensor_closed_form, uint8_t* __restrict__ codes,
-                          uint8_t* __restrict__ sf, float* __restrict__ gscale, uint32_t rht_stream) {
+                          uint8_t* __restrict__ sf, float* __restrict__ gscale, uint32_t rht_stream,
+                          const __grid_constant__ PhiloxKeys pk) {
   pdl_prologue();
   __shared__ float tile[128][65];
   __shared__ float blk_amax[8][64];
@@ -681,7 +682,7 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
     float rcp;
     const uint32_t sb = block_scale(am[it], Sg, rcp);
     const int64_t k0 = k_base + kb * 16;
-    const uint2 packed = quantize_block16<SR>(xs[it], rcp, seed, stream_id, (uint64_t)((o * K16 + k0) >> 3));
+    const uint2 packed = quantize_block16<SR>(xs[it], rcp, pk, stream_id, (uint64_t)((o * K16 + k0) >> 3));
     *reinterpret_cast<uint2*>(&out_codes[dl][kb * 8]) = packed;
     if (d < D && k0 < Kp) {
       const int64_t b = k0 >> 4;
@@ -746,13 +747,13 @@ static cudaError_t launch_rows_g(const QuantRowsArgs& a, cudaStream_t st) {
       }
     }
     launch_kernel(quantize_rows_kernel<GS, SR, TILED, true, false>, dim3(grid), dim3(256), smem, st, a.src, a.rows, a.K, a.ld, a.keep, a.seed,
-                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, stage_cols8, 0u);
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, stage_cols8, 0u, make_philox_keys(a.seed));
   } else if (a.rht_stream) {
     launch_kernel(quantize_rows_kernel<GS, SR, TILED, false, true>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, nullptr, a.seed,
-                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0, a.rht_stream);
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0, a.rht_stream, make_philox_keys(a.seed));
   } else {
     launch_kernel(quantize_rows_kernel<GS, SR, TILED, false, false>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, nullptr, a.seed,
-                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0, 0u);
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0, 0u, make_philox_keys(a.seed));
   }
   return cudaGetLastError();
 }
@@ -822,7 +823,7 @@ static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
   const dim3 grid(blocks_for(a.rowsK, 128), blocks_for(a.D, 64));
 #define NVFP4_LAUNCH_TR(TILED_, RHT_)                                                                                              \
   launch_kernel(quantize_transpose_kernel<SRC, GS, SR, TILED_, RHT_, false>, dim3(grid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.seed, \
-                a.stream_id, a.gs_cells, a.tensor_closed_form, a.codes, a.sf, a.gscale, a.rht_stream)
+                a.stream_id, a.gs_cells, a.tensor_closed_form, a.codes, a.sf, a.gscale, a.rht_stream, make_philox_keys(a.seed))
   if (a.sf_tiled) {
     if (a.rht_stream) NVFP4_LAUNCH_TR(true, true); else NVFP4_LAUNCH_TR(true, false);
   } else {
@@ -841,10 +842,10 @@ static cudaError_t launch_tr_amax_rht(const TransposeSrc& src, int64_t rowsK, in
   const dim3 grid(blocks_for(rowsK, 128), blocks_for(D, 64));
   if (rht_stream)
     launch_kernel(quantize_transpose_kernel<SRC, GS, false, false, true, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
-                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), rht_stream);
+                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), rht_stream, make_philox_keys(seed));
   else
     launch_kernel(quantize_transpose_kernel<SRC, GS, false, false, false, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
-                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), 0u);
+                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), 0u, make_philox_keys(seed));
   return cudaGetLastError();
 }
 
