@@ -256,7 +256,7 @@ __device__ __forceinline__ uint2 quantize_block16(const float (&x)[16], float rc
 //   RHT     each block is replaced by (x S) H_16 before anything else looks at it (never together with GATHER).
 // =========================================================================================================
 template <int GS, bool SR, bool TILED, bool GATHER, bool RHT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, int64_t ld,
                      const int32_t* __restrict__ keep, uint64_t seed, uint32_t stream_id,
                      const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
