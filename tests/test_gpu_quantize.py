@@ -146,3 +146,43 @@ def test_all_seven_rtn_ties_and_saturation_on_device():
     codes = out.codes.cpu().numpy()[:32]
     nib = np.stack([codes & 15, codes >> 4], axis=1).reshape(-1)
     assert list(nib[0:16]) == rows[0][2] and list(nib[32:48]) == rows[2][2]
+
+
+@pytest.mark.parametrize("shape", [(128, 128), (129, 128), (127, 128), (64, 256), (65, 256), (512, 256), (513, 256), (16, 1024),
+                                   (17, 1024), (1024, 128), (96, 384), (2048, 128 * 3)])
+@pytest.mark.parametrize("gs_mode", MODES)
+def test_row_axis_cta_boundaries(shape, gs_mode):
+    """Shapes around the 1024-block CTA granularity with K a multiple of 128: interior CTAs take the unchecked copy of
+    the kernel body, the last CTA the checked one; both must agree with the oracle bit for bit."""
+    b = B()
+    x = make(shape, 100 + shape[0], "grad")
+    for rounding in (orc.RTN, orc.SR):
+        ref = orc.quantize(x, orc.AXIS_ROW, rounding, gs_mode, seed=31, stream_id=3)
+        out = b.alloc_operand(shape[0], shape[1], gs_mode, b.SF_TILED128x4, poison=True)
+        b.nvfp4_quantize(to_dev_bf16(x), b.AXIS_ROW, rounding, 31, 3, gs_mode, out=out)
+        assert_operand_equal(out, ref, f"cta boundary {shape} gs{gs_mode} r{rounding}")
+
+
+def test_randomised_shapes_modes_and_axes():
+    """Forty random (shape, axis, rounding, scale mode, transformation) combinations with a fixed seed."""
+    b = B()
+    rng = np.random.default_rng(2024)
+    for case in range(40):
+        rows, cols = int(rng.integers(1, 700)), int(rng.integers(1, 90)) * 8
+        axis = int(rng.integers(0, 2))
+        rounding = int(rng.integers(0, 2))
+        gs_mode = int(rng.integers(0, 3))
+        rht = int(rng.integers(0, 2)) * 7
+        x = make((rows, cols), 500 + case, "grad")
+        seed = int(rng.integers(0, 2 ** 40))
+        if axis == orc.AXIS_ROW:
+            src = orc.rht16(x, seed, rht) if rht else x
+            R, K = rows, cols
+        else:
+            xt = np.ascontiguousarray(x.T)
+            src = orc.rht16(xt, seed, rht) if rht else xt
+            R, K = cols, rows
+        ref = orc.quantize(src, orc.AXIS_ROW, rounding, gs_mode, seed=seed, stream_id=3)
+        out = b.alloc_operand(R, K, gs_mode, b.SF_TILED128x4, poison=True)
+        b.nvfp4_quantize(to_dev_bf16(x), axis, rounding, seed, 3, gs_mode, out=out, rht_stream_id=rht)
+        assert_operand_equal(out, ref, f"case {case}: {rows}x{cols} axis{axis} r{rounding} gs{gs_mode} rht{rht}", k_extended=bool(rht))
