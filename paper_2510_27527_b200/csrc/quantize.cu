@@ -558,12 +558,22 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
   }
 
   // ---- phase 1: stage (zero outside the matrix) ------------------------------------------------------------
-  if (SRC == 0 && d_base + 64 <= D && (s.ld & 7) == 0) {
-    // 128 rows x 8 chunks of 8 BF16
+  if (SRC == 0 && (s.ld & 7) == 0) {
+    // 128 rows x 8 chunks of 8 BF16; the one chunk that straddles D (ragged last column tile) is read element by element
     for (int c = tid; c < 1024; c += 256) {
       const int kr = c >> 3, dc = (c & 7) << 3;
       uint4 v = make_uint4(0, 0, 0, 0);
-      if (k_base + kr < rowsK) v = *reinterpret_cast<const uint4*>(s.bf16 + (k_base + kr) * s.ld + d_base + dc);
+      if (k_base + kr < rowsK) {
+        const uint16_t* src = s.bf16 + (k_base + kr) * s.ld + d_base + dc;
+        if (d_base + dc + 8 <= D) {
+          v = *reinterpret_cast<const uint4*>(src);
+        } else if (d_base + dc < D) {
+          uint32_t w[4] = {0, 0, 0, 0};
+          const int n = (int)(D - d_base - dc);
+          for (int i = 0; i < n; ++i) w[i >> 1] |= (uint32_t)src[i] << (16 * (i & 1));
+          v = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
       float f8[8] = {bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y), bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w)};
       if (RHT) {
         const float f = rht_factor(sw, (uint32_t)kr);
@@ -573,8 +583,10 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
 #pragma unroll
       for (int i = 0; i < 8; ++i) tile[kr][dc + i] = f8[i];
     }
-  } else if (SRC == 1 && !s.row_map && d_base + 64 <= D) {
-    // forward operand without a row map: 32 codes (16 bytes) and their two scale bytes per thread
+  } else if (SRC == 1 && !s.row_map) {
+    // forward operand without a row map: 32 codes (16 bytes) and their two scale bytes per thread. A tile that sticks out
+    // past D still lies inside the operand's row (K is padded to 128 there, with zero codes and zero scales), so the last
+    // column tile is staged the same way and the columns past D simply hold zeros that nobody stores.
     const int kr = tid >> 1, half = tid & 1;
     const int64_t k = k_base + kr;
     float v[32];
