@@ -93,9 +93,12 @@ bool carve_operand(Carver& c, nvfp4_operand* o, int64_t R, int64_t K, int32_t gs
 nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, int32_t rounding,
                               uint64_t seed, uint32_t stream_id, const int32_t* keep, int64_t n_keep,
                               const nvfp4_operand* out, uint32_t* cells, cudaStream_t st, int cells_zeroed = 0,
-                              const int32_t* excluded = nullptr, uint32_t rht_stream = 0, int compute_amax = 1) {
+                              const int32_t* excluded = nullptr, uint32_t rht_stream = 0, int compute_amax = 1,
+                              uint16_t* excl_out = nullptr, int64_t ld_excl_out = 0) {
   if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   QuantRowsArgs a{};
+  a.excl_out = keep && excluded ? excl_out : nullptr;
+  a.ld_excl_out = ld_excl_out;
   a.src = src;
   a.rows = rows;
   a.K = keep ? n_keep : cols;
@@ -389,18 +392,16 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
     if (launch_amax_tensor_pair(Xp, N_tok, D, ldx, cells_x, Wp, C, D, ldw, cells_w, st) != cudaSuccess) return NVFP4_ERR_CUDA;
     amax_pass = 0;
   }
+  // with outlier channels, the quantizers also write the BF16 side operands X[:, outliers] and W[:, outliers]
+  const int64_t Kh = n_out > 0 ? nvfp4_outlier_pad(n_out) : 0;
+  if (n_out > 0 && (!saved->X_out || !saved->W_out)) return NVFP4_ERR_NULL;
   if ((s = do_quantize_rows(Xp, N_tok, D, ldx, cfg->rounding[0], cfg->seed, 1, keep, Dk, &saved->qx, cells_x, st, 1,
-                            cfg->outlier_cols, 0, amax_pass)) != NVFP4_OK)
+                            cfg->outlier_cols, 0, amax_pass, static_cast<uint16_t*>(saved->X_out), Kh)) != NVFP4_OK)
     return s;
   if ((s = do_quantize_rows(Wp, C, D, ldw, cfg->rounding[1], cfg->seed, 2, keep, Dk, &saved->qw, cells_w, st, 1,
-                            cfg->outlier_cols, 0, amax_pass)) != NVFP4_OK)
+                            cfg->outlier_cols, 0, amax_pass, static_cast<uint16_t*>(saved->W_out), Kh)) != NVFP4_OK)
     return s;
   if (n_out > 0) {
-    if (!saved->X_out || !saved->W_out) return NVFP4_ERR_NULL;
-    const int64_t Kh = nvfp4_outlier_pad(n_out);
-    if (launch_gather_cols(Xp, ldx, N_tok, cfg->outlier_cols, n_out, static_cast<uint16_t*>(saved->X_out), Kh, st) != cudaSuccess ||
-        launch_gather_cols(Wp, ldw, C, cfg->outlier_cols, n_out, static_cast<uint16_t*>(saved->W_out), Kh, st) != cudaSuccess)
-      return NVFP4_ERR_CUDA;
     if (cfg->gs_mode == NVFP4_GS_BLOCK128) {
       // the outer-block GEMM variant takes the side product as an FP32 addend computed beforehand
       HpFwdArgs h{};
@@ -569,14 +570,14 @@ static nvfp4_status bwd_dw_impl(const void* dY, int64_t lddy, const nvfp4_saved*
   if ((s = do_quantize_transpose(t6, 1, N_tok, Dk, cfg->rounding[5], cfg->seed, 6, &q6, cells6, st, 1, rht)) != NVFP4_OK) return s;
   if (n_out == 0) return do_gemm(&q5, &q6, dW, cfg->dw_dtype, lddw, 0, nullptr, 0, cfg->dev_status, st);
 
-  // kept columns: compact product, then a column scatter (a scattering GEMM epilogue measured slower than this pair)
+  // kept columns: compact product; one pass then writes dW row by row from it and from the outlier channels' side product
+  // (a scattering GEMM epilogue measured slower)
   if ((s = do_gemm(&q5, &q6, compact, NVFP4_DT_F32, ld_compact, 0, nullptr, 0, cfg->dev_status, st)) != NVFP4_OK) return s;
-  if (launch_scatter_cols(compact, ld_compact, 1, dW, lddw, dw_f32, C, Dk, cfg->keep_cols, st) != cudaSuccess)
-    return NVFP4_ERR_CUDA;
   HpDwArgs h{};
   h.dY = static_cast<const uint16_t*>(dY); h.X_out = static_cast<const uint16_t*>(saved->X_out);
   h.lddy = lddy; h.Kh = Kh; h.T = N_tok; h.C = C; h.n_out = n_out; h.outl = cfg->outlier_cols;
   h.dW = dW; h.dw_is_f32 = dw_f32; h.lddw = lddw; h.partial = hp_partial; h.dev_status = cfg->dev_status;
+  h.compact = compact; h.ld_compact = ld_compact; h.D = D; h.keep = cfg->keep_cols; h.col_map = cfg->col_map;
   return launch_hp_dw(h, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 

@@ -139,6 +139,80 @@ __global__ void __launch_bounds__(256) hp_dw_reduce_kernel(HpDwArgs a, int n_spl
   }
 }
 
+// dW[c, d] for whole output rows (OutControl's weight gradient): a kept channel takes its value from the compact FP4
+// product, an outlier channel the sum of the high-precision side product's token splits. One coalesced pass over dW
+// instead of a column scatter plus a scattered reduce. Each CTA first builds, in shared memory, where every channel comes
+// from: src_of[d] = position in the compact product (>= 0) or -(1 + rank among the outliers). Rows are then taken four at a
+// time: all threads first reduce the splits of the group's outlier channels into shared memory (fixed order), then all
+// threads assemble and store the four rows.
+constexpr int kAsmRows = 4;
+template <bool F32>
+__global__ void __launch_bounds__(256) dw_assemble_kernel(HpDwArgs a, int n_split, const float* __restrict__ compact, int64_t ld_compact,
+                                                         const int32_t* __restrict__ col_map, int64_t D, int vec) {
+  pdl_prologue();
+  extern __shared__ int32_t src_of[];                                       // [D]
+  float* osum = reinterpret_cast<float*>(src_of + ((D + 3) & ~(int64_t)3));  // [kAsmRows][n_out]
+  for (int64_t d = threadIdx.x; d < D; d += 256) src_of[d] = col_map[d];
+  __syncthreads();
+  for (int64_t j = threadIdx.x; j < a.n_out; j += 256) src_of[a.outl[j]] = -(int32_t)(1 + j);
+  __syncthreads();
+  const uint32_t n_out = (uint32_t)a.n_out, D32 = (uint32_t)D;
+  const uint32_t chunks = (D32 + 3) >> 2;
+  for (int64_t c0 = (int64_t)blockIdx.x * kAsmRows; c0 < a.C; c0 += (int64_t)gridDim.x * kAsmRows) {
+    const uint32_t nr = (uint32_t)min((int64_t)kAsmRows, a.C - c0);
+    for (uint32_t e = threadIdx.x; e < nr * n_out; e += 256) {
+      const uint32_t rr = e / n_out, j = e - rr * n_out;
+      const float* p = a.partial + (c0 + rr) * a.Kh + j;
+      float v = 0.0f;
+      for (int sp = 0; sp < n_split; ++sp) v += p[(int64_t)sp * a.C * a.Kh];  // fixed order
+      osum[rr * n_out + j] = v;
+    }
+    __syncthreads();
+    if (vec) {  // four channels per item, one 16-byte (FP32) or 8-byte (BF16) store
+      for (uint32_t e = threadIdx.x; e < nr * chunks; e += 256) {
+        const uint32_t rr = e / chunks, d = (e - rr * chunks) << 2;
+        const int64_t c = c0 + rr;
+        float v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          v[i] = 0.0f;
+          if (d + i < D32) {
+            const int32_t m = src_of[d + i];
+            v[i] = m >= 0 ? compact[c * ld_compact + m] : osum[rr * n_out + (uint32_t)(-m - 1)];
+          }
+        }
+        if (d + 4 <= D32) {
+          if (F32)
+            *reinterpret_cast<float4*>(reinterpret_cast<float*>(a.dW) + c * a.lddw + d) = make_float4(v[0], v[1], v[2], v[3]);
+          else
+            *reinterpret_cast<uint2*>(reinterpret_cast<uint16_t*>(a.dW) + c * a.lddw + d) =
+                make_uint2((uint32_t)f32_to_bf16_bits(v[0]) | ((uint32_t)f32_to_bf16_bits(v[1]) << 16),
+                           (uint32_t)f32_to_bf16_bits(v[2]) | ((uint32_t)f32_to_bf16_bits(v[3]) << 16));
+        } else {
+          for (int i = 0; d + i < D32; ++i) {
+            if (F32)
+              reinterpret_cast<float*>(a.dW)[c * a.lddw + d + i] = v[i];
+            else
+              reinterpret_cast<uint16_t*>(a.dW)[c * a.lddw + d + i] = f32_to_bf16_bits(v[i]);
+          }
+        }
+      }
+    } else {
+      for (uint32_t e = threadIdx.x; e < nr * D32; e += 256) {
+        const uint32_t rr = e / D32, d = e - rr * D32;
+        const int64_t c = c0 + rr;
+        const int32_t m = src_of[d];
+        const float v = m >= 0 ? compact[c * ld_compact + m] : osum[rr * n_out + (uint32_t)(-m - 1)];
+        if (F32)
+          reinterpret_cast<float*>(a.dW)[c * a.lddw + d] = v;
+        else
+          reinterpret_cast<uint16_t*>(a.dW)[c * a.lddw + d] = f32_to_bf16_bits(v);
+      }
+    }
+    __syncthreads();  // osum is rewritten by the next group
+  }
+}
+
 // dst[r, j] = src[r, cols[j]] (j < n), 0 for n <= j < ld_dst. One warp per row.
 __global__ void __launch_bounds__(256) gather_cols_kernel(const uint16_t* __restrict__ src, int64_t ld_src, int64_t rows,
                                                          const int32_t* __restrict__ cols, int64_t n, uint16_t* __restrict__ dst,
@@ -186,7 +260,9 @@ size_t hp_dw_partial_floats(int64_t T, int64_t C, int64_t Kh) { return (size_t)k
 
 cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st) {
   if (a.C == 0 || a.n_out == 0) return cudaSuccess;
-  const int64_t t_per_split = ((a.T + kHpDwSplit - 1) / kHpDwSplit + 63) / 64 * 64;
+  // token splits: as many as fill the SMs once with (C / 128) x splits CTAs, at most kHpDwSplit (the workspace's size)
+  const int64_t want = std::max<int64_t>(1, std::min<int64_t>(kHpDwSplit, 148 / std::max<int64_t>(1, (a.C + 127) / 128)));
+  const int64_t t_per_split = ((a.T + want - 1) / want + 63) / 64 * 64;
   const int n_split = (int)((a.T + t_per_split - 1) / t_per_split);
   cudaError_t e;
   if (hp_dw_mma_supported(a.Kh) && (a.lddy & 7) == 0) {  // tensor-core path (the CUDA-core kernel covers odd shapes)
@@ -197,6 +273,28 @@ cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st) {
     e = cudaGetLastError();
   }
   if (e != cudaSuccess) return e;
+  if (a.compact && a.col_map && a.D < ((int64_t)1 << 29) && (a.D + 4 + kAsmRows * a.n_out) * 4 <= 200 * 1024) {
+    // kept and outlier channels written together, row by row
+    const size_t smem = (size_t)(((a.D + 3) & ~(int64_t)3) + kAsmRows * a.n_out) * 4;
+    const int f32 = a.dw_is_f32;
+    const int elt = f32 ? 4 : 2;
+    const int vec = (a.lddw & 3) == 0 && (reinterpret_cast<uintptr_t>(a.dW) & (size_t)(4 * elt - 1)) == 0;
+    if (smem > 48 * 1024) {
+      e = f32 ? cudaFuncSetAttribute(dw_assemble_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+              : cudaFuncSetAttribute(dw_assemble_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+    }
+    const dim3 grid((unsigned)std::min<int64_t>((a.C + kAsmRows - 1) / kAsmRows, 148 * 8));
+    if (f32)
+      launch_kernel(dw_assemble_kernel<true>, grid, dim3(256), smem, st, a, n_split, a.compact, a.ld_compact, a.col_map, a.D, vec);
+    else
+      launch_kernel(dw_assemble_kernel<false>, grid, dim3(256), smem, st, a, n_split, a.compact, a.ld_compact, a.col_map, a.D, vec);
+    return cudaGetLastError();
+  }
+  if (a.compact) {
+    e = launch_scatter_cols(a.compact, a.ld_compact, 1, a.dW, a.lddw, a.dw_is_f32, a.C, a.D - a.n_out, a.keep, st);
+    if (e != cudaSuccess) return e;
+  }
   const int64_t total = a.C * a.n_out;
   launch_kernel(hp_dw_reduce_kernel, dim3((unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8)), dim3(256), 0, st, a, n_split);
   return cudaGetLastError();

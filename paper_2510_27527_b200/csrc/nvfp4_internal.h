@@ -18,6 +18,10 @@ struct QuantRowsArgs {
   int64_t rows, K, cols_src, ld;
   const int32_t* keep;  // optional column list of length K
   const int32_t* excluded;  // optional: the sorted complement of `keep` (cols_src - K entries); enables the masked amax
+  // optional (with `excluded`): excl_out[r, j] = src[r, excluded[j]], zero for cols_src - K <= j < ld_excl_out. Written by the
+  // masked amax pass where that runs (the matrix is read once for both), else by a separate gather launch.
+  uint16_t* excl_out;
+  int64_t ld_excl_out;
   uint64_t seed;
   uint32_t stream_id;
   uint32_t rht_stream;  // non-zero: random Hadamard transformation along K with this sign stream (not with `keep`)
@@ -150,6 +154,12 @@ struct HpDwArgs {
   int64_t lddw;
   float* partial;  // workspace: hp_dw_partial_floats(T, C, Kh) floats
   int32_t* dev_status;
+  // optional: the kept channels' product [C, D - n_out] (FP32, compact), placed into dW by the same pass that writes the
+  // outlier channels. keep [D - n_out] and col_map [D] describe the placement (D = all channels).
+  const float* compact;
+  int64_t ld_compact, D;
+  const int32_t* keep;
+  const int32_t* col_map;
 };
 size_t hp_dw_partial_floats(int64_t T, int64_t C, int64_t Kh);
 bool hp_dw_mma_supported(int64_t Kh);

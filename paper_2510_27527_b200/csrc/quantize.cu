@@ -81,10 +81,14 @@ __global__ void __launch_bounds__(256) amax_tensor_pair_kernel(const uint16_t* _
 
 // amax of a BF16 matrix over all columns EXCEPT a sorted list of excluded ones (OutControl: the outlier channels do not
 // take part in the FP4 operand's tensor scale). Each CTA builds a one-bit-per-column mask in shared memory from the
-// list, then streams whole rows with 16-byte loads, zeroing the excluded lanes. Folded into cells[0] by atomic max.
+// list, then streams a contiguous slab of rows with 16-byte loads (four in flight per thread), zeroing the excluded
+// lanes. Folded into cells[0] by atomic max.
+// With `out` the excluded columns of the slab are then copied, in list order, to out[r, 0 .. n_excl) (zero up to ld_out):
+// the high-precision side operand, picked from rows this CTA has just pulled through L1 / L2.
 __global__ void __launch_bounds__(256) amax_tensor_masked_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols,
                                                                 int64_t ld, const int32_t* __restrict__ excluded, int64_t n_excl,
-                                                                uint32_t* amax_bits) {
+                                                                uint32_t* amax_bits, uint16_t* __restrict__ out, int64_t ld_out,
+                                                                int64_t rows_per_cta) {
   pdl_prologue();
   extern __shared__ uint32_t keep_bits[];  // bit c = 1: column c takes part
   const int64_t words = (cols + 31) >> 5;
@@ -92,26 +96,47 @@ __global__ void __launch_bounds__(256) amax_tensor_masked_kernel(const uint16_t*
   __syncthreads();
   for (int64_t i = threadIdx.x; i < n_excl; i += 256) atomicAnd(&keep_bits[excluded[i] >> 5], ~(1u << (excluded[i] & 31)));
   __syncthreads();
-  const int64_t chunks = (cols + 7) >> 3;
+  const int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
+  const int64_t r1 = min(rows, r0 + rows_per_cta);
+  const uint32_t chunks = (uint32_t)((cols + 7) >> 3);
+  const uint32_t n_items = r1 > r0 ? (uint32_t)(r1 - r0) * chunks : 0u;  // (row, chunk) pairs of the slab, row-major
+  const uint64_t inv = (1ull << 32) / chunks + 1ull;                    // item / chunks by multiplication
   uint32_t m = 0;
-  for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
-    const uint16_t* p = src + r * ld;
-    for (int64_t c = threadIdx.x; c < chunks; c += 256) {
-      const uint32_t mask8 = (keep_bits[c >> 2] >> ((c & 3) * 8)) & 0xFFu;
-      uint32_t w[4] = {0, 0, 0, 0};
-      if ((c << 3) + 8 <= cols) {
-        const uint4 v = *reinterpret_cast<const uint4*>(p + (c << 3));
-        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
-      } else {
-        for (int q = 0; q < 8; ++q)
-          if ((c << 3) + q < cols) w[q >> 1] |= (uint32_t)p[(c << 3) + q] << (16 * (q & 1));
+  for (uint32_t e0 = threadIdx.x; e0 < n_items; e0 += 256 * 4) {
+    uint32_t w[4][4], mask8[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t e = e0 + u * 256;
+      w[u][0] = w[u][1] = w[u][2] = w[u][3] = 0;
+      mask8[u] = 0;
+      if (e < n_items) {
+        const uint32_t rr = (uint32_t)(((uint64_t)e * inv) >> 32), c = e - rr * chunks;
+        const uint16_t* p = src + (r0 + rr) * ld + ((int64_t)c << 3);
+        mask8[u] = (keep_bits[c >> 2] >> ((c & 3) * 8)) & 0xFFu;
+        if (((int64_t)c << 3) + 8 <= cols) {
+          const uint4 v = *reinterpret_cast<const uint4*>(p);
+          w[u][0] = v.x; w[u][1] = v.y; w[u][2] = v.z; w[u][3] = v.w;
+        } else {
+          for (int q = 0; q < 8; ++q)
+            if (((int64_t)c << 3) + q < cols) w[u][q >> 1] |= (uint32_t)p[q] << (16 * (q & 1));
+        }
       }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const uint32_t two = (mask8 >> (2 * q)) & 3u;
+        const uint32_t two = (mask8[u] >> (2 * q)) & 3u;
         const uint32_t lanes = ((0u - (two & 1u)) & 0x0000FFFFu) | ((0u - (two >> 1)) & 0xFFFF0000u);
-        m = umax16x2(m, bf16x2_abs_bits(w[q]) & lanes);
+        m = umax16x2(m, bf16x2_abs_bits(w[u][q]) & lanes);
       }
+  }
+  if (out && r1 > r0) {
+    const uint32_t ldo = (uint32_t)ld_out, n_out_items = (uint32_t)(r1 - r0) * ldo;
+    const uint64_t inv_o = (1ull << 32) / ldo + 1ull;
+    for (uint32_t e = threadIdx.x; e < n_out_items; e += 256) {
+      const uint32_t rr = (uint32_t)(((uint64_t)e * inv_o) >> 32), j = e - rr * ldo;
+      out[(r0 + rr) * ld_out + j] = j < n_excl ? src[(r0 + rr) * ld + excluded[j]] : (uint16_t)0;
     }
   }
   uint32_t a = hmax_of_pair(m);
@@ -280,19 +305,34 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
     const int64_t n_rows = last / nb - stage_row0 + 1;
     const uint32_t chunks_per_row = (uint32_t)(stage_cols8 >> 3);
     const uint32_t n_chunks = (uint32_t)n_rows * chunks_per_row;
-    for (uint32_t e = threadIdx.x; e < n_chunks; e += 256) {
-      const uint32_t rr = e / chunks_per_row, ch = (e - rr * chunks_per_row) << 3;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      const uint16_t* p = src + (stage_row0 + rr) * ld + ch;
-      if ((int64_t)ch + 8 <= cols_src) {
-        v = *reinterpret_cast<const uint4*>(p);
-      } else {
-        uint32_t t[4] = {0, 0, 0, 0};
-        for (int q = 0; q < 8; ++q)
-          if ((int64_t)ch + q < cols_src) t[q >> 1] |= (uint32_t)p[q] << (16 * (q & 1));
-        v = make_uint4(t[0], t[1], t[2], t[3]);
+    // e / chunks_per_row by multiplication (exact while e * chunks_per_row < 2^32, and a CTA stages a few thousand chunks)
+    const uint64_t inv = (1ull << 32) / chunks_per_row + 1ull;
+    // eight chunks per thread and pass, every load issued before the first store: one exposed memory latency per pass
+    for (uint32_t e0 = threadIdx.x; e0 < n_chunks; e0 += 256 * 8) {
+      uint4 v[8];
+      uint32_t off[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const uint32_t e = e0 + q * 256;
+        v[q] = make_uint4(0, 0, 0, 0);
+        off[q] = 0xFFFFFFFFu;
+        if (e < n_chunks) {
+          const uint32_t rr = (uint32_t)(((uint64_t)e * inv) >> 32), ch = (e - rr * chunks_per_row) << 3;
+          off[q] = rr * (uint32_t)stage_cols8 + ch;
+          const uint16_t* p = src + (stage_row0 + rr) * ld + ch;
+          if ((int64_t)ch + 8 <= cols_src) {
+            v[q] = *reinterpret_cast<const uint4*>(p);
+          } else {
+            uint32_t t[4] = {0, 0, 0, 0};
+            for (int i = 0; i < 8; ++i)
+              if ((int64_t)ch + i < cols_src) t[i >> 1] |= (uint32_t)p[i] << (16 * (i & 1));
+            v[q] = make_uint4(t[0], t[1], t[2], t[3]);
+          }
+        }
       }
-      *reinterpret_cast<uint4*>(row_stage + (size_t)rr * stage_cols8 + ch) = v;
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        if (off[q] != 0xFFFFFFFFu) *reinterpret_cast<uint4*>(row_stage + off[q]) = v[q];
     }
     __syncthreads();
   }
@@ -780,7 +820,7 @@ static cudaError_t launch_rows_r(const QuantRowsArgs& a, cudaStream_t st) {
   return a.sr ? launch_rows_t<GS, true>(a, st) : launch_rows_t<GS, false>(a, st);
 }
 
-cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
+static cudaError_t launch_quantize_rows_impl(const QuantRowsArgs& a, cudaStream_t st, bool& side_copy_done) {
   if (a.rows == 0 || a.K == 0) return cudaSuccess;
   if (a.rows >= ((int64_t)1 << 31) || a.cols_src >= ((int64_t)1 << 31) || a.ld >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
   cudaError_t e;
@@ -804,10 +844,16 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
       if (a.keep && a.excluded && (a.ld & 7) == 0 && a.cols_src <= 256 * 1024) {
         // amax over the kept columns only: full-width vector loads with the excluded (outlier) columns masked out
         const size_t smem = (size_t)((a.cols_src + 31) >> 5) * 4;
-        const unsigned grid = (unsigned)std::min<int64_t>(a.rows, 148 * 8);
+        // a contiguous slab of rows per CTA. The kernel divides item numbers by d = chunks per row (and by the side
+        // operand's width) through a 32-bit reciprocal, exact while items * d < 2^32: slabs stay below 2^32 / d^2 rows
+        int64_t rows_per_cta = (a.rows + 148 * 8 - 1) / (148 * 8);
+        const int64_t dmax = std::max<int64_t>((a.cols_src + 7) >> 3, a.excl_out ? a.ld_excl_out : 1);
+        rows_per_cta = std::max<int64_t>(1, std::min<int64_t>(rows_per_cta, (((int64_t)1 << 32) - 1) / (dmax * dmax)));
+        const unsigned grid = (unsigned)((a.rows + rows_per_cta - 1) / rows_per_cta);
         launch_kernel(amax_tensor_masked_kernel, dim3(grid), dim3(256), smem, st, a.src, a.rows, a.cols_src, a.ld, a.excluded,
-                      a.cols_src - a.K, a.gs_cells);
+                      a.cols_src - a.K, a.gs_cells, a.excl_out, a.ld_excl_out, rows_per_cta);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        side_copy_done = a.excl_out != nullptr;
         return launch_rows_r<kGsTensor>(a, st);
       }
       if (a.keep) {  // amax over the kept columns only: one row per CTA, one atomic per row
@@ -828,6 +874,15 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
     return launch_rows_r<kGsRow>(a, st);
   }
   return launch_rows_r<kGsBlock128>(a, st);
+}
+
+cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
+  bool side_copy_done = false;
+  cudaError_t e = launch_quantize_rows_impl(a, st, side_copy_done);
+  if (e != cudaSuccess) return e;
+  if (a.excl_out && a.excluded && !side_copy_done)
+    e = launch_gather_cols(a.src, a.ld, a.rows, a.excluded, a.cols_src - a.K, a.excl_out, a.ld_excl_out, st);
+  return e;
 }
 
 template <int SRC, int GS, bool SR>
