@@ -41,6 +41,7 @@
 
 #define ORC_ROUND_RTN 0
 #define ORC_ROUND_SR 1
+#define ORC_ROUND_SR_SCALE_UP 2 /* SR with S_block rounded up to E4M3: no element beyond +-6, E[Q(x)] = x for all */
 #define ORC_GS_TENSOR 0
 #define ORC_GS_ROW 1
 #define ORC_GS_BLOCK128 2
@@ -85,6 +86,15 @@ int orc_e4m3_encode(float s) {
         }
     }
     return best;
+}
+
+/* Non-negative float -> the smallest E4M3 value that is >= s (byte), 448 (0x7E) if there is none.
+ * Variant for strictly unbiased stochastic rounding: with S_block >= amax_b / (6 Sg) every |x| / (Sg S_block) <= 6 up to
+ * the float roundings of d, r and y, so the clamp at 6 never removes more than those. Written as the definition. */
+int orc_e4m3_encode_up(float s) {
+    for (int c = 0; c <= 0x7E; ++c)
+        if (orc_e4m3_value(c) >= (double)s) return c;
+    return 0x7E;
 }
 
 /* ---------------------------------------------------------------------------------------------------------
@@ -216,7 +226,7 @@ void orc_quantize(const float *x, int64_t R, int64_t K, int rounding, int gs_mod
             const float amax_b = group_amax(row + k0, len);
             const float t = amax_b / Sg;
             const float s = t / 6.0f;
-            const int sb = orc_e4m3_encode(s);
+            const int sb = (rounding == ORC_ROUND_SR_SCALE_UP) ? orc_e4m3_encode_up(s) : orc_e4m3_encode(s);
             const float Sbf = (float)orc_e4m3_value(sb);
             sf[r * nb + b] = (uint8_t)sb;
             const float d = Sg * Sbf;
@@ -228,7 +238,7 @@ void orc_quantize(const float *x, int64_t R, int64_t K, int rounding, int gs_mod
                 float a = fabsf(y);
                 if (a > 6.0f) a = 6.0f;
                 int m;
-                if (rounding == ORC_ROUND_SR) {
+                if (rounding == ORC_ROUND_SR || rounding == ORC_ROUND_SR_SCALE_UP) {
                     const uint64_t idx = (uint64_t)r * (uint64_t)K16 + (uint64_t)k;
                     m = orc_round_sr_mag(a, orc_sr_bits(seed, stream_id, idx));
                 } else {

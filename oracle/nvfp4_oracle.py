@@ -19,6 +19,7 @@ from dataclasses import dataclass
 import numpy as np
 
 RTN, SR = 0, 1
+SR_SCALE_UP = 2  # stochastic rounding with the block scale rounded up to E4M3 (strictly unbiased variant)
 GS_TENSOR, GS_ROW, GS_BLOCK128 = 0, 1, 2
 AXIS_ROW, AXIS_COL = 0, 1
 
@@ -51,6 +52,8 @@ def lib():
         L.orc_e4m3_value.argtypes = [c_int]
         L.orc_e4m3_encode.restype = c_int
         L.orc_e4m3_encode.argtypes = [ctypes.c_float]
+        L.orc_e4m3_encode_up.restype = c_int
+        L.orc_e4m3_encode_up.argtypes = [ctypes.c_float]
         L.orc_philox4x32_10.restype = None
         L.orc_philox4x32_10.argtypes = [vp, vp, vp]
         L.orc_sr_bits.restype = c_u32
@@ -100,6 +103,11 @@ def e4m3_value(byte: int) -> float:
 
 def e4m3_encode(s: float) -> int:
     return lib().orc_e4m3_encode(float(s))
+
+
+def e4m3_encode_up(s: float) -> int:
+    """Byte of the smallest E4M3 value >= s (0x7E if none): the block scale of the SR_SCALE_UP variant."""
+    return lib().orc_e4m3_encode_up(float(s))
 
 
 def philox4x32_10(ctr, key):
