@@ -42,7 +42,14 @@ typedef enum {
   NVFP4_ERR_LIMIT = 9      /* a size exceeds a fixed capacity of the entry point (see nvfp4_quantize_static) */
 } nvfp4_status;
 
-typedef enum { NVFP4_ROUND_RTN = 0, NVFP4_ROUND_SR = 1 } nvfp4_round;
+/* Element rounding (paper Sec. 2.1).
+ * RTN: round to nearest, ties to the even code. SR: stochastic rounding with 16 random bits per element.
+ * SR_SCALE_UP: SR, and the block scale S_block is the smallest E4M3 value >= amax_b / (6 S_global) instead of the nearest
+ *   one (448 stays the ceiling). With the nearest scale about half of the blocks get a scale rounded down, their
+ *   largest element lands in (6, 6.43] on the FP4 grid and is clamped, so E[Q(x)] = x (Sec. 2.1, stated for -6 <= x <= 6)
+ *   fails for it; with the rounded-up scale every element lies within +-6 and the expectation is exact. A variant the
+ *   paper's unbiasedness ablation motivates; not the default of any quantizer. */
+typedef enum { NVFP4_ROUND_RTN = 0, NVFP4_ROUND_SR = 1, NVFP4_ROUND_SR_SCALE_UP = 2 } nvfp4_round;
 
 /* Axis along which the 16-element groups run in the SOURCE matrix.
  * ROW: groups along the columns of a row; the operand has the source's shape [rows, cols].
@@ -98,6 +105,7 @@ long long nvfp4_launch_count(void);
  *   rounding RTN: nearest E2M1 value, ties to the even code. SR: 16 random bits u per element from
  *            Philox4x32-10 (key = seed, counter = (idx / 8, stream_id, 0), idx = r * Kp16 + k in the OPERAND,
  *            Kp16 = K rounded up to 16); the magnitude rounds up iff (u + 0.5) / 65536 < (a - q1) / (q2 - q1).
+ *            SR_SCALE_UP: the same draws and rule, with S_block rounded up instead of to nearest (see nvfp4_round).
  *   rht_stream_id  0: off. Otherwise the random Hadamard transformation of Sec. 4.1 is applied along the operand's K before
  *            anything else: each aligned block of 16 consecutive k (zero-extended at the end of K) becomes (x S) H_16,
  *            H_16 the orthonormal Sylvester matrix (entries +-1/4), S the sign diagonal with s_k = -1 iff bit (k % 128)

@@ -22,6 +22,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 # enums of include/nvfp4.h
 OK = 0
 ROUND_RTN, ROUND_SR = 0, 1
+ROUND_SR_SCALE_UP = 2  # stochastic rounding, block scale rounded up to E4M3 (every element within +-6)
 AXIS_ROW, AXIS_COL = 0, 1
 GS_TENSOR, GS_ROW, GS_BLOCK128 = 0, 1, 2
 SF_LINEAR, SF_TILED128x4 = 0, 1

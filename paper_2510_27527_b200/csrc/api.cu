@@ -110,7 +110,7 @@ nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, i
   a.stream_id = stream_id;
   a.rht_stream = rht_stream;
   a.gs_mode = out->gs_mode;
-  a.sr = rounding == NVFP4_ROUND_SR;
+  a.sr = rounding == NVFP4_ROUND_SR ? 1 : rounding == NVFP4_ROUND_SR_SCALE_UP ? 2 : 0;
   a.sf_tiled = out->sf_layout == NVFP4_SF_TILED128x4;
   a.compute_amax = compute_amax;
   a.cells_zeroed = cells_zeroed;
@@ -134,7 +134,7 @@ nvfp4_status do_quantize_transpose(const TransposeSrc& src, int from_codes, int6
   a.stream_id = stream_id;
   a.rht_stream = rht_stream;
   a.gs_mode = out->gs_mode;
-  a.sr = rounding == NVFP4_ROUND_SR;
+  a.sr = rounding == NVFP4_ROUND_SR ? 1 : rounding == NVFP4_ROUND_SR_SCALE_UP ? 2 : 0;
   a.sf_tiled = out->sf_layout == NVFP4_SF_TILED128x4;
   a.compute_amax = compute_amax;
   a.cells_zeroed = cells_zeroed;
@@ -184,7 +184,7 @@ nvfp4_status check_cfg(const nvfp4_layer_cfg* cfg, int64_t D) {
   if (!cfg) return NVFP4_ERR_NULL;
   if (cfg->gs_mode < 0 || cfg->gs_mode > 2) return NVFP4_ERR_ENUM;
   for (int i = 0; i < 6; ++i)
-    if (cfg->rounding[i] < 0 || cfg->rounding[i] > 1) return NVFP4_ERR_ENUM;
+    if (cfg->rounding[i] < 0 || cfg->rounding[i] > 2) return NVFP4_ERR_ENUM;
   if (cfg->y_dtype < 0 || cfg->y_dtype > 1 || cfg->dx_dtype < 0 || cfg->dx_dtype > 1 || cfg->dw_dtype < 0 ||
       cfg->dw_dtype > 1 || cfg->rht < 0 || cfg->rht > 1)
     return NVFP4_ERR_ENUM;
@@ -250,7 +250,7 @@ nvfp4_status nvfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, in
                             const int32_t* keep_cols, int64_t n_keep, const nvfp4_operand* out, void* workspace,
                             size_t ws_bytes, void* stream) {
   if (!src_bf16 || !out) return NVFP4_ERR_NULL;
-  if (axis < 0 || axis > 1 || rounding < 0 || rounding > 1) return NVFP4_ERR_ENUM;
+  if (axis < 0 || axis > 1 || rounding < 0 || rounding > 2) return NVFP4_ERR_ENUM;
   if (rht_stream_id && keep_cols) return NVFP4_ERR_ENUM;
   if (rows < 0 || cols < 0 || (keep_cols && (n_keep < 0 || n_keep > cols))) return NVFP4_ERR_SHAPE;
   if (keep_cols && axis != NVFP4_AXIS_ROW) return NVFP4_ERR_SHAPE;
@@ -280,7 +280,7 @@ nvfp4_status nvfp4_requantize_t(const nvfp4_operand* in, const void* hp_bf16, in
                                 uint32_t rht_stream_id, const nvfp4_operand* out, void* workspace, size_t ws_bytes,
                                 void* stream) {
   if (!in || !out) return NVFP4_ERR_NULL;
-  if (rounding < 0 || rounding > 1) return NVFP4_ERR_ENUM;
+  if (rounding < 0 || rounding > 2) return NVFP4_ERR_ENUM;
   nvfp4_status s;
   if ((s = check_operand_ptrs(in)) != NVFP4_OK) return s;
   if ((s = check_operand_ptrs(out)) != NVFP4_OK) return s;
@@ -478,7 +478,7 @@ static nvfp4_status bwd_dx_impl(const void* dY, int64_t lddy, const nvfp4_saved*
     qa.stream_id = 4;
     qa.rht_stream = rht;
     qa.gs_mode = cfg->gs_mode;
-    qa.sr = cfg->rounding[3] == NVFP4_ROUND_SR;
+    qa.sr = cfg->rounding[3] == NVFP4_ROUND_SR ? 1 : cfg->rounding[3] == NVFP4_ROUND_SR_SCALE_UP ? 2 : 0;
     qa.sf_tiled = 1;
     qa.cells_zeroed = 1;
     qa.gs_cells = cells4;

@@ -86,11 +86,17 @@ __device__ __forceinline__ float global_scale_from_amax(float amax) {
   return amax == 0.0f ? 1.0f : div_const(amax, 2688.0f, 0x1.861862p-12f);  // amax / (448 * 6)
 }
 // Returns the E4M3 byte of the block scale and the reciprocal r that maps x to the FP4 grid (0 if the scale is 0).
-__device__ __forceinline__ uint32_t block_scale(float amax_b, float Sg, float& rcp) {
+// round_up: take the smallest E4M3 value >= s instead of the nearest one (448 stays the ceiling), so that no element of
+// the block lands beyond +-6 on the FP4 grid and stochastic rounding is unbiased for every element.
+__device__ __forceinline__ uint32_t block_scale(float amax_b, float Sg, float& rcp, bool round_up = false) {
   const float t = __fdiv_rn(amax_b, Sg);
   const float s = div_const(t, 6.0f, 0x1.555556p-3f);
-  const uint32_t sb = e4m3_encode(s);
-  const float Sbf = e4m3_decode(sb);
+  uint32_t sb = e4m3_encode(s);
+  float Sbf = e4m3_decode(sb);
+  if (round_up && Sbf < s && sb < 0x7Eu) {  // non-negative E4M3 bytes are ordered like their values
+    sb += 1u;
+    Sbf = e4m3_decode(sb);
+  }
   const float d = __fmul_rn(Sg, Sbf);
   rcp = (Sbf == 0.0f) ? 0.0f : __frcp_rn(d);  // the correctly rounded 1 / d
   return sb;

@@ -25,7 +25,7 @@ struct QuantRowsArgs {
   uint64_t seed;
   uint32_t stream_id;
   uint32_t rht_stream;  // non-zero: random Hadamard transformation along K with this sign stream (not with `keep`)
-  int gs_mode, sr, sf_tiled;
+  int gs_mode, sr, sf_tiled;  // sr: 0 round to nearest, 1 stochastic, 2 stochastic with the block scale rounded up
   int compute_amax;    // TENSOR mode: run the amax pre-pass (0: gs_cells[0] already holds the amax bits)
   int cells_zeroed;    // the caller has already cleared gs_cells on this stream
   uint32_t* gs_cells;  // workspace: 1 cell (TENSOR) or `rows` cells (ROW)
@@ -61,7 +61,7 @@ struct QuantTransposeArgs {
   uint64_t seed;
   uint32_t stream_id;
   uint32_t rht_stream;  // non-zero: random Hadamard transformation along the operand's K (source rows) with this stream
-  int gs_mode, sr, sf_tiled;
+  int gs_mode, sr, sf_tiled;  // sr: 0 round to nearest, 1 stochastic, 2 stochastic with the block scale rounded up
   int compute_amax;
   int cells_zeroed;        // the caller has already cleared gs_cells on this stream
   int tensor_closed_form;  // set by the launcher

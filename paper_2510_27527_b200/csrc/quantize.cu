@@ -286,7 +286,7 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
                      const int32_t* __restrict__ keep, uint64_t seed, uint32_t stream_id,
                      const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
                      float* __restrict__ gscale, uint32_t div_mul, uint32_t div_shift, int wide_loads, int64_t cols_src,
-                     int64_t stage_cols8, uint32_t rht_stream, const __grid_constant__ PhiloxKeys pk) {
+                     int64_t stage_cols8, uint32_t rht_stream, int sb_up, const __grid_constant__ PhiloxKeys pk) {
   pdl_prologue();
   constexpr int NB = 4;  // inner blocks per thread; all loads are issued before any arithmetic
   extern __shared__ uint16_t row_stage[];  // GATHER only: the source rows this CTA touches, [n_rows][cols_src8]
@@ -457,7 +457,7 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
 
       // ---- block scale, rounding, packing -------------------------------------------------------------------
       float rcp;
-      const uint32_t sb = block_scale(__uint_as_float(amax_b_bits), Sg, rcp);
+      const uint32_t sb = block_scale(__uint_as_float(amax_b_bits), Sg, rcp, SR && sb_up);
       if (!RHT) {
   #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -571,7 +571,7 @@ template <int SRC, int GS, bool SR, bool TILED, bool RHT, bool AMAX_ONLY>
 __global__ void __launch_bounds__(256)
 quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t seed, uint32_t stream_id,
                           uint32_t* __restrict__ gs_cells, int tensor_closed_form, uint8_t* __restrict__ codes,
-                          uint8_t* __restrict__ sf, float* __restrict__ gscale, uint32_t rht_stream,
+                          uint8_t* __restrict__ sf, float* __restrict__ gscale, uint32_t rht_stream, int sb_up,
                           const __grid_constant__ PhiloxKeys pk) {
   pdl_prologue();
   __shared__ float tile[128][65];
@@ -732,7 +732,7 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
   for (int it = 0; it < 2; ++it) {
     const int kb = (tid >> 6) + 4 * it;
     float rcp;
-    const uint32_t sb = block_scale(am[it], Sg, rcp);
+    const uint32_t sb = block_scale(am[it], Sg, rcp, SR && sb_up);
     const int64_t k0 = k_base + kb * 16;
     const uint2 packed = quantize_block16<SR>(xs[it], rcp, pk, stream_id, (uint64_t)((o * K16 + k0) >> 3));
     *reinterpret_cast<uint2*>(&out_codes[dl][kb * 8]) = packed;
@@ -799,13 +799,13 @@ static cudaError_t launch_rows_g(const QuantRowsArgs& a, cudaStream_t st) {
       }
     }
     launch_kernel(quantize_rows_kernel<GS, SR, TILED, true, false>, dim3(grid), dim3(256), smem, st, a.src, a.rows, a.K, a.ld, a.keep, a.seed,
-                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, stage_cols8, 0u, make_philox_keys(a.seed));
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, stage_cols8, 0u, a.sr == 2, make_philox_keys(a.seed));
   } else if (a.rht_stream) {
     launch_kernel(quantize_rows_kernel<GS, SR, TILED, false, true>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, nullptr, a.seed,
-                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0, a.rht_stream, make_philox_keys(a.seed));
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0, a.rht_stream, a.sr == 2, make_philox_keys(a.seed));
   } else {
     launch_kernel(quantize_rows_kernel<GS, SR, TILED, false, false>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, nullptr, a.seed,
-                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0, 0u, make_philox_keys(a.seed));
+                  a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, (int64_t)0, 0u, a.sr == 2, make_philox_keys(a.seed));
   }
   return cudaGetLastError();
 }
@@ -890,7 +890,7 @@ static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
   const dim3 grid(blocks_for(a.rowsK, 128), blocks_for(a.D, 64));
 #define NVFP4_LAUNCH_TR(TILED_, RHT_)                                                                                              \
   launch_kernel(quantize_transpose_kernel<SRC, GS, SR, TILED_, RHT_, false>, dim3(grid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.seed, \
-                a.stream_id, a.gs_cells, a.tensor_closed_form, a.codes, a.sf, a.gscale, a.rht_stream, make_philox_keys(a.seed))
+                a.stream_id, a.gs_cells, a.tensor_closed_form, a.codes, a.sf, a.gscale, a.rht_stream, a.sr == 2, make_philox_keys(a.seed))
   if (a.sf_tiled) {
     if (a.rht_stream) NVFP4_LAUNCH_TR(true, true); else NVFP4_LAUNCH_TR(true, false);
   } else {
@@ -909,10 +909,10 @@ static cudaError_t launch_tr_amax_rht(const TransposeSrc& src, int64_t rowsK, in
   const dim3 grid(blocks_for(rowsK, 128), blocks_for(D, 64));
   if (rht_stream)
     launch_kernel(quantize_transpose_kernel<SRC, GS, false, false, true, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
-                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), rht_stream, make_philox_keys(seed));
+                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), rht_stream, 0, make_philox_keys(seed));
   else
     launch_kernel(quantize_transpose_kernel<SRC, GS, false, false, false, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
-                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), 0u, make_philox_keys(seed));
+                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), 0u, 0, make_philox_keys(seed));
   return cudaGetLastError();
 }
 

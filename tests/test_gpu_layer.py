@@ -96,3 +96,28 @@ def test_combined_backward_is_bit_identical_to_the_two_calls(gs_mode, outcontrol
     dX2, dW2 = b.nvfp4_linear_bwd(dYd, saved, cfg)
     torch.cuda.synchronize()
     assert torch.equal(dX1, dX2) and torch.equal(dW1, dW2)
+
+
+@pytest.mark.parametrize("gs_mode", [0, 1, 2])
+@pytest.mark.parametrize("outcontrol", [False, True])
+@pytest.mark.parametrize("rht", [False, True])
+def test_backward_with_rounded_up_block_scales(gs_mode, outcontrol, rht):
+    """The strictly unbiased variant (block scale rounded up) in all four backward quantizers, through the layer calls."""
+    b = B()
+    N_tok, D, C = 200, 272, 136
+    X, W, dY, ch = synth.layer_inputs(12, N_tok, D, C, n_outlier=3, factor=40.0, grad_scale=1e-3)
+    outl = ch if outcontrol else None
+    rounding = (orc.RTN, orc.RTN, orc.SR_SCALE_UP, orc.SR_SCALE_UP, orc.SR_SCALE_UP, orc.SR_SCALE_UP)
+    ocfg = orc.LayerConfig(gs_mode=gs_mode, seed=8, outliers=outl, rounding=rounding, rht=rht)
+    _, so = orc.linear_fwd(X, W, ocfg)
+    dXo, dWo = orc.linear_bwd_dx(dY, so, ocfg), orc.linear_bwd_dw(dY, so, ocfg)
+    plain = orc.LayerConfig(gs_mode=gs_mode, seed=8, outliers=outl, rht=rht)
+    assert rel_fro(orc.linear_bwd_dx(dY, so, plain), dXo) > 1e-3  # the variant is a different quantizer
+    cfg = b.LayerConfig(gs_mode=gs_mode, seed=8, outliers=outl, rounding=rounding, rht=rht, y_dtype=b.DT_F32, dx_dtype=b.DT_F32,
+                        dw_dtype=b.DT_F32)
+    Xd, Wd, dYd = to_dev_bf16(X), to_dev_bf16(W), to_dev_bf16(dY)
+    _, saved = b.nvfp4_linear_fwd(Xd, Wd, cfg)
+    dX, dW = b.nvfp4_linear_bwd(dYd, saved, cfg)
+    torch.cuda.synchronize()
+    assert rel_fro(dX.float().cpu().numpy(), dXo) <= 2e-5
+    assert rel_fro(dW.float().cpu().numpy(), dWo) <= 2e-5

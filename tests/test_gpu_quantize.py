@@ -29,7 +29,7 @@ def make(shape, seed, kind="act"):
 
 @pytest.mark.parametrize("shape", SHAPES)
 @pytest.mark.parametrize("gs_mode", MODES)
-@pytest.mark.parametrize("rounding", [orc.RTN, orc.SR])
+@pytest.mark.parametrize("rounding", [orc.RTN, orc.SR, orc.SR_SCALE_UP])
 def test_row_axis_bit_exact(shape, gs_mode, rounding):
     b = B()
     x = make(shape, 7 + shape[1], "act" if rounding == orc.RTN else "grad")
@@ -42,7 +42,7 @@ def test_row_axis_bit_exact(shape, gs_mode, rounding):
 
 @pytest.mark.parametrize("shape", [(16, 1), (48, 5), (144, 127), (272, 129), (512, 256), (1000, 72), (200, 333)])
 @pytest.mark.parametrize("gs_mode", MODES)
-@pytest.mark.parametrize("rounding", [orc.RTN, orc.SR])
+@pytest.mark.parametrize("rounding", [orc.RTN, orc.SR, orc.SR_SCALE_UP])
 def test_col_axis_bit_exact(shape, gs_mode, rounding):
     b = B()
     cols8 = (shape[1] + 7) // 8 * 8  # leading dimension must be a multiple of 8 elements
@@ -70,17 +70,18 @@ def test_keep_cols_compaction(gs_mode):
 @pytest.mark.parametrize("shape", [(16, 16), (130, 272), (256, 512), (520, 200)])
 @pytest.mark.parametrize("gs_mode", MODES)
 @pytest.mark.parametrize("in_layout", [0, 1])
-def test_requantize_transposed_bit_exact(shape, gs_mode, in_layout):
+@pytest.mark.parametrize("rounding", [orc.SR, orc.SR_SCALE_UP])
+def test_requantize_transposed_bit_exact(shape, gs_mode, in_layout, rounding):
     """Q4 / Q6: re-quantize the aligned tensor X-hat along the other axis, from the forward operand's codes."""
     b = B()
     x = make(shape, 21 + shape[0])
     fwd_ref = orc.quantize(x, orc.AXIS_ROW, orc.RTN, gs_mode)
-    ref = orc.quantize(orc.rematerialize_f32(fwd_ref), orc.AXIS_COL, orc.SR, gs_mode, seed=5, stream_id=6)
+    ref = orc.quantize(orc.rematerialize_f32(fwd_ref), orc.AXIS_COL, rounding, gs_mode, seed=5, stream_id=6)
     fwd = b.nvfp4_quantize(to_dev_bf16(x), b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, in_layout)
     assert_operand_equal(fwd, fwd_ref, "fwd operand")
     out = b.alloc_operand(shape[1], shape[0], gs_mode, poison=True)
-    b.nvfp4_requantize_t(fwd, b.ROUND_SR, 5, 6, out=out)
-    assert_operand_equal(out, ref, f"requantize_t {shape} gs{gs_mode}")
+    b.nvfp4_requantize_t(fwd, rounding, 5, 6, out=out)
+    assert_operand_equal(out, ref, f"requantize_t {shape} gs{gs_mode} r{rounding}")
 
 
 @pytest.mark.parametrize("gs_mode", MODES)
@@ -170,7 +171,7 @@ def test_randomised_shapes_modes_and_axes():
     for case in range(40):
         rows, cols = int(rng.integers(1, 700)), int(rng.integers(1, 90)) * 8
         axis = int(rng.integers(0, 2))
-        rounding = int(rng.integers(0, 2))
+        rounding = int(rng.integers(0, 3))
         gs_mode = int(rng.integers(0, 3))
         rht = int(rng.integers(0, 2)) * 7
         x = make((rows, cols), 500 + case, "grad")
