@@ -626,7 +626,8 @@ def main():
                     help="OutControl: fraction of input channels kept in BF16 (0 = off; the paper uses 0.10)")
     ap.add_argument("--rht", action="store_true", help="random Hadamard transformation (block 16) in the four backward quantizers")
     ap.add_argument("--sr-scale-up", action="store_true", help="backward quantizers round the block scale up (strictly unbiased variant)")
-    ap.add_argument("--graph", action="store_true", help="capture one step in a CUDA graph and time its replays")
+    ap.add_argument("--graph", action=argparse.BooleanOptionalAction, default=True,
+                    help="capture one step in a CUDA graph and time its replays (default; --no-graph launches every kernel from the host)")
     ap.add_argument("--no-breakdown", action="store_true", help="only warm-up + timed steps (used for ncu launch lists)")
     ap.add_argument("--sweep", action="store_true", help="roofline sweep of the large GEMM shapes instead of the step benchmark")
     ap.add_argument("--aux", action="store_true", help="HBM roofline of the calibration and OsciReset kernels instead of the step benchmark")
