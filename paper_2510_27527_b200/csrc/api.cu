@@ -369,7 +369,6 @@ size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, i
   if (op_kind == NVFP4_OP_FWD) {
     carve_size(total, cells_bytes(N_tok, gs_mode));
     carve_size(total, cells_bytes(C, gs_mode));
-    if (n_out > 0) carve_size(total, (size_t)N_tok * (size_t)round_up(C, 4) * 4);
   } else if (op_kind == NVFP4_OP_BWD_DX) {
     carve_size(total, cells_bytes(N_tok, gs_mode));
     carve_size(total, cells_bytes(D, gs_mode));
@@ -416,9 +415,7 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
   Carver cv(workspace, ws_bytes);
   uint32_t* cells_x = static_cast<uint32_t*>(cv.take(cells_bytes(N_tok, cfg->gs_mode)));
   uint32_t* cells_w = static_cast<uint32_t*>(cv.take(cells_bytes(C, cfg->gs_mode)));
-  const int64_t ld_add = round_up(C, 4);
-  float* addend = n_out > 0 ? static_cast<float*>(cv.take((size_t)N_tok * ld_add * 4)) : nullptr;
-  if (!cells_x || !cells_w || (n_out > 0 && !addend)) return NVFP4_ERR_WORKSPACE;
+  if (!cells_x || !cells_w) return NVFP4_ERR_WORKSPACE;
 
   const uint16_t* Xp = static_cast<const uint16_t*>(X);
   const uint16_t* Wp = static_cast<const uint16_t*>(W);
@@ -446,21 +443,12 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
     return NVFP4_ERR_CUDA;
   if (s_x != NVFP4_OK) return s_x;
   if (s_w != NVFP4_OK) return s_w;
-  if (n_out > 0) {
-    if (cfg->gs_mode == NVFP4_GS_BLOCK128) {
-      // the outer-block GEMM variant takes the side product as an FP32 addend computed beforehand
-      HpFwdArgs h{};
-      h.X = Xp; h.W = Wp; h.ldx = ldx; h.ldw = ldw; h.M = N_tok; h.N = C; h.n_out = n_out;
-      h.outl = cfg->outlier_cols; h.Y = addend; h.ldy = ld_add;
-      if (launch_hp_fwd(h, st) != cudaSuccess) return NVFP4_ERR_CUDA;
-    }
-  }
   saved->X = X; saved->W = W; saved->ldx = ldx; saved->ldw = ldw;
   saved->N_tok = N_tok; saved->D = D; saved->C = C;
-  if (n_out > 0 && cfg->gs_mode != NVFP4_GS_BLOCK128)  // Y = FP4 product + X_out W_out^T, both inside one kernel
+  if (n_out > 0)  // Y = FP4 product + X_out W_out^T, both inside one kernel
     return do_gemm(&saved->qx, &saved->qw, Y, cfg->y_dtype, ldy, 0, nullptr, 0, cfg->dev_status, st, saved->X_out, saved->W_out,
                    nvfp4_outlier_pad(n_out));
-  return do_gemm(&saved->qx, &saved->qw, Y, cfg->y_dtype, ldy, 0, addend, ld_add, cfg->dev_status, st);
+  return do_gemm(&saved->qx, &saved->qw, Y, cfg->y_dtype, ldy, 0, nullptr, 0, cfg->dev_status, st);
 }
 
 // dy_amax: optional cell already holding the bit pattern of max |dY| (TENSOR mode without the Hadamard transformation):

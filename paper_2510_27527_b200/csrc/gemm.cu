@@ -785,13 +785,14 @@ __global__ void __launch_bounds__(64, 1) mma_issue_probe_kernel(int32_t iters, i
 constexpr int B128_STAGES = 4;
 constexpr int B128_NBUF = 3;
 constexpr int B128_MAX_CHUNKS = 128;
-constexpr uint32_t B128_SGB_BYTES = B128_MAX_CHUNKS * 128 * 4;
+constexpr uint32_t B128_SGB_BYTES = (B128_MAX_CHUNKS + 1) * 128 * 4 + 512;  // + the high-precision partial; 1024-byte multiple
 constexpr uint32_t B128_STAGING_BYTES = 4 * 4096;  // one 32-row x 128-byte staging buffer per epilogue warp (bulk stores)
 constexpr uint32_t B128_SMEM_BYTES = B128_STAGES * Cfg<128>::STAGE_BYTES + B128_SGB_BYTES + B128_STAGING_BYTES + 1024 + 256;
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                           const __grid_constant__ CUtensorMap tmC, const Params p) {
+                           const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmAh,
+                           const __grid_constant__ CUtensorMap tmBh, const Params p) {
   using C = Cfg<128>;
   constexpr int BN = 128;
   constexpr int STAGES = B128_STAGES;
@@ -856,6 +857,16 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
         bulk_load(st + A_BYTES + C::B_BYTES, sfa_src + (size_t)kt * 2048, 2048, full_bar(s), leader);
         bulk_load(st + A_BYTES + C::B_BYTES + SFA_BYTES, sfb_src + (size_t)kt * 2048, 2048, full_bar(s), leader);
       }
+      // OutControl: the BF16 outlier channels of both operands, 64 per stage, into the same stage buffers
+      for (int32_t h = 0; h < p.hp_k_tiles && ok; ++h, ++it) {
+        const int s = it % STAGES;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.dev_status));
+        if (!ok) break;
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        mbar_expect_tx(full_bar(s), A_BYTES + C::B_BYTES, leader);
+        tma_load_2d(st, &tmAh, h * 64, mt * BM, full_bar(s), leader);
+        tma_load_2d(st + A_BYTES, &tmBh, h * 64, nt * BN, full_bar(s), leader);
+      }
     }
     if (!ok) {
       const uint32_t n_back = it < (uint32_t)STAGES ? it : (uint32_t)STAGES;
@@ -903,6 +914,29 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
         }
         tc_commit(empty_bar(s), leader);
       }
+      if (p.hp_k_tiles > 0 && ok) {
+        // high-precision side product: one more partial, handed to the promotion warps like a 128-k chunk (scale 1)
+        const uint32_t buf = cit % B128_NBUF;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(part_empty_bar(buf), ((cit / B128_NBUF) & 1) ^ 1, abort_flag, p.dev_status));
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t idesc_bf16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        for (int32_t h = 0; h < p.hp_k_tiles; ++h, ++it) {
+          const int s = it % STAGES;
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.dev_status));
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)  // 64 BF16 = one 128-byte swizzle row = four K = 16 steps of 32 bytes
+            tc_mma_bf16(tmem_base + buf * 128, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc_bf16,
+                        (h | kk) != 0, leader);
+          tc_commit(empty_bar(s), leader);
+        }
+        if (!ok) break;
+        tc_commit(part_full_bar(buf), leader);
+        ++cit;
+      }
     }
     tc_commit(drain_bar, leader);
     {
@@ -925,6 +959,7 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
         const int64_t n = (int64_t)nt * BN + epi_tid;
         const float* src = p.b_gscale + n * G;
         for (int32_t kc = 0; kc < chunks; ++kc) sgb[kc * 128 + epi_tid] = (n < p.N) ? __ldg(src + kc) : 0.0f;
+        if (p.hp_k_tiles > 0) sgb[chunks * 128 + epi_tid] = 1.0f;  // the high-precision partial carries no scale
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
       const int64_t m = (int64_t)mt * BM + quad * 32 + lane;
@@ -932,11 +967,12 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
       float2 acc[64];
 #pragma unroll
       for (int j = 0; j < 64; ++j) acc[j] = make_float2(0.0f, 0.0f);
-      for (int32_t kc = 0; kc < chunks && ok; ++kc, ++cit) {
+      const int32_t parts = chunks + (p.hp_k_tiles > 0 ? 1 : 0);
+      for (int32_t kc = 0; kc < parts && ok; ++kc, ++cit) {
         const uint32_t buf = cit % B128_NBUF;
         if (!(ok = mbar_wait(part_full_bar(buf), (cit / B128_NBUF) & 1, abort_flag, p.dev_status))) break;
         tc_fence_after();
-        const float sa = __ldg(sa_row + kc);
+        const float sa = kc < chunks ? __ldg(sa_row + kc) : 1.0f;
         const float2 sa2 = make_float2(sa, sa);
         const float4* sb4 = reinterpret_cast<const float4*>(sgb + kc * 128);
 #pragma unroll
@@ -1571,6 +1607,11 @@ cudaError_t launch_block128(const GemmArgs& a, cudaStream_t st) {
   CUtensorMap tmA, tmB, tmC;
   if (!make_codes_map(&tmA, a.a_codes, a.M, Kp, BM) || !make_codes_map(&tmB, a.b_codes, a.N, Kp, 128)) return cudaErrorInvalidValue;
   Params p{};
+  CUtensorMap tmAh = tmA, tmBh = tmB;  // placeholders unless the high-precision side product is requested
+  if (a.hp_Kh > 0) {
+    if (!make_hp_map(&tmAh, a.hp_a, a.M, a.hp_Kh) || !make_hp_map(&tmBh, a.hp_b, a.N, a.hp_Kh)) return cudaErrorInvalidValue;
+    p.hp_k_tiles = (int32_t)(a.hp_Kh / 64);
+  }
   p.use_tma_store = make_c_map(&tmC, a.C, a.M, a.N, a.ldc, a.c_is_f32 != 0) ? 1 : 0;
   if (!p.use_tma_store) tmC = tmA;  // unused by the kernel then
   p.a_sf = a.a_sf;
@@ -1602,7 +1643,7 @@ cudaError_t launch_block128(const GemmArgs& a, cudaStream_t st) {
   }
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
-  launch_kernel(gemm_nvfp4_block128_kernel, dim3(grid), dim3(NUM_THREADS), B128_SMEM_BYTES, st, tmA, tmB, tmC, p);
+  launch_kernel(gemm_nvfp4_block128_kernel, dim3(grid), dim3(NUM_THREADS), B128_SMEM_BYTES, st, tmA, tmB, tmC, tmAh, tmBh, p);
   return cudaGetLastError();
 }
 
@@ -1670,7 +1711,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   const char* pair_env = getenv("NVFP4_GEMM_2CTA");
   const bool pairs = pair_env ? atoi(pair_env) != 0
                               : (a.K >= 3072 && ((a.M + 255) / 256) * ((a.N + 255) / 256) >= 2 * (sm_count() / 2));
-  if (a.hp_Kh > 0 && a.gs_mode != kGsBlock128)  // the fused high-precision side product lives in the 128 x 128 variant
+  if (a.hp_Kh > 0 && a.gs_mode != kGsBlock128)  // the fused high-precision side product lives in the 128 x 128 variants
     return a.gs_mode == kGsTensor ? launch_variant<kGsTensor, 128>(a, st) : launch_variant<kGsRow, 128>(a, st);
   if (pairs && a.gs_mode == kGsTensor) return launch_2cta<kGsTensor>(a, st);
   if (pairs && a.gs_mode == kGsRow) return launch_2cta<kGsRow>(a, st);

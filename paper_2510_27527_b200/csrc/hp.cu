@@ -1,58 +1,11 @@
-// High-precision side of OutControl (paper Sec. 4.2): the few outlier channels of X / W stay in BF16 and their
-// products are accumulated in FP32 on the CUDA cores. With the paper-scale channel counts used here (about 1 % of
-// the hidden size) these products are a tiny fraction of the layer's flops; the kernels are bound by reading dY and
-// by writing the FP32 addend.
+// High-precision side of OutControl (paper Sec. 4.2): the outlier channels of X / W stay in BF16. The forward side
+// product runs on the tensor cores inside the FP4 GEMM kernels; here are the copies that build the compact side
+// operands, the CUDA-core fallback of dW[:, outliers] = dY^T X_out for shapes the tensor-core kernel does not take, and
+// the pass that assembles dW from the compact FP4 product and the side product.
 #include "nvfp4_device.cuh"
 #include "nvfp4_internal.h"
 
 namespace nvfp4 {
-
-// Y[m, n] = sum_j X[m, outl[j]] * W[n, outl[j]].  CTA tile 64 x 64, outlier channels in chunks of 32.
-__global__ void __launch_bounds__(256) hp_fwd_kernel(HpFwdArgs a) {
-  pdl_prologue();
-  __shared__ float xs[32][65];
-  __shared__ float ws[32][65];
-  const int64_t m0 = (int64_t)blockIdx.y * 64, n0 = (int64_t)blockIdx.x * 64;
-  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;  // 16 x 16 threads, 4 x 4 outputs each
-  float acc[4][4] = {};
-  for (int64_t j0 = 0; j0 < a.n_out; j0 += 32) {
-    for (int e = threadIdx.x; e < 32 * 64; e += 256) {
-      const int jj = e & 31, rr = e >> 5;
-      const int64_t j = j0 + jj;
-      float xv = 0.0f, wv = 0.0f;
-      if (j < a.n_out) {
-        const int64_t col = a.outl[j];
-        if (m0 + rr < a.M) xv = bf16_bits_to_float(a.X[(m0 + rr) * a.ldx + col]);
-        if (n0 + rr < a.N) wv = bf16_bits_to_float(a.W[(n0 + rr) * a.ldw + col]);
-      }
-      xs[jj][rr] = xv;
-      ws[jj][rr] = wv;
-    }
-    __syncthreads();
-#pragma unroll 4
-    for (int jj = 0; jj < 32; ++jj) {
-      float xv[4], wv[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        xv[i] = xs[jj][ty * 4 + i];
-        wv[i] = ws[jj][tx * 4 + i];
-      }
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int k = 0; k < 4; ++k) acc[i][k] = fmaf(xv[i], wv[k], acc[i][k]);
-    }
-    __syncthreads();
-  }
-  for (int i = 0; i < 4; ++i) {
-    const int64_t m = m0 + ty * 4 + i;
-    if (m >= a.M) continue;
-    for (int k = 0; k < 4; ++k) {
-      const int64_t n = n0 + tx * 4 + k;
-      if (n < a.N) a.Y[m * a.ldy + n] = acc[i][k];
-    }
-  }
-}
 
 // dW[c, outl[j]] = sum_t dY[t, c] * X_out[t, j]. The token range is split over blockIdx.y; each CTA owns 64 output
 // channels c and walks its tokens in chunks of 64 staged in shared memory (dY chunk [64 t x 64 c], X_out chunk
@@ -247,13 +200,6 @@ __global__ void __launch_bounds__(256) scatter_cols_kernel(const void* src, int6
         reinterpret_cast<uint16_t*>(dst)[o] = v;
     }
   }
-}
-
-cudaError_t launch_hp_fwd(const HpFwdArgs& a, cudaStream_t st) {
-  if (a.M == 0 || a.N == 0) return cudaSuccess;
-  const dim3 grid((unsigned)((a.N + 63) / 64), (unsigned)((a.M + 63) / 64));
-  launch_kernel(hp_fwd_kernel, dim3(grid), dim3(256), 0, st, a);
-  return cudaGetLastError();
 }
 
 size_t hp_dw_partial_floats(int64_t T, int64_t C, int64_t Kh) { return (size_t)kHpDwSplit * (size_t)C * (size_t)Kh; }

@@ -138,13 +138,6 @@ cudaError_t launch_mma_issue_probe(int32_t iters, int32_t* dev_status, cudaStrea
 cudaError_t launch_gather_cols(const uint16_t* src, int64_t ld_src, int64_t rows, const int32_t* cols, int64_t n, uint16_t* dst,
                                int64_t ld_dst, cudaStream_t st);
 
-struct HpFwdArgs {
-  const uint16_t *X, *W;
-  int64_t ldx, ldw, M, N, n_out;
-  const int32_t* outl;
-  float* Y;  // FP32 [M, N], overwritten
-  int64_t ldy;
-};
 struct HpDwArgs {
   const uint16_t *dY, *X_out;  // dY [T, C]; X_out [T, Kh]: the outlier channels of X, compact, zero-padded to Kh (multiple of 64)
   int64_t lddy, Kh, T, C, n_out;
@@ -165,7 +158,6 @@ size_t hp_dw_partial_floats(int64_t T, int64_t C, int64_t Kh);
 bool hp_dw_mma_supported(int64_t Kh);
 cudaError_t launch_hp_dw_mma(const uint16_t* dY, int64_t lddy, const uint16_t* X_out, int64_t Kh, int64_t T, int64_t C,
                              float* partial, int n_split, int64_t t_per_split, int32_t* dev_status, cudaStream_t st);
-cudaError_t launch_hp_fwd(const HpFwdArgs& a, cudaStream_t st);
 cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st);
 
 // Scatter a compact [C, n_keep] matrix into columns keep[j] of dW [C, D].
