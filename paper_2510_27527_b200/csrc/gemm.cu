@@ -958,7 +958,22 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
       {
         const int64_t n = (int64_t)nt * BN + epi_tid;
         const float* src = p.b_gscale + n * G;
-        for (int32_t kc = 0; kc < chunks; ++kc) sgb[kc * 128 + epi_tid] = (n < p.N) ? __ldg(src + kc) : 0.0f;
+        if (n < p.N) {
+          int32_t kc = 0;
+          if ((G & 3) == 0) {  // a row's scales as 16-byte loads, sixteen values in flight per thread
+#pragma unroll 4
+            for (; kc + 4 <= chunks; kc += 4) {
+              const float4 q = __ldg(reinterpret_cast<const float4*>(src + kc));
+              sgb[kc * 128 + epi_tid] = q.x;
+              sgb[(kc + 1) * 128 + epi_tid] = q.y;
+              sgb[(kc + 2) * 128 + epi_tid] = q.z;
+              sgb[(kc + 3) * 128 + epi_tid] = q.w;
+            }
+          }
+          for (; kc < chunks; ++kc) sgb[kc * 128 + epi_tid] = __ldg(src + kc);
+        } else {
+          for (int32_t kc = 0; kc < chunks; ++kc) sgb[kc * 128 + epi_tid] = 0.0f;
+        }
         if (p.hp_k_tiles > 0) sgb[chunks * 128 + epi_tid] = 1.0f;  // the high-precision partial carries no scale
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -968,11 +983,15 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
 #pragma unroll
       for (int j = 0; j < 64; ++j) acc[j] = make_float2(0.0f, 0.0f);
       const int32_t parts = chunks + (p.hp_k_tiles > 0 ? 1 : 0);
+      // SgA[m, kc] is fetched two chunks ahead: with one promotion warp per scheduler nothing else would hide the load
+      float sa_0 = chunks > 0 ? __ldg(sa_row) : 1.0f, sa_1 = chunks > 1 ? __ldg(sa_row + 1) : 1.0f;
       for (int32_t kc = 0; kc < parts && ok; ++kc, ++cit) {
+        const float sa = kc < chunks ? sa_0 : 1.0f;
+        sa_0 = sa_1;
+        if (kc + 2 < chunks) sa_1 = __ldg(sa_row + kc + 2);
         const uint32_t buf = cit % B128_NBUF;
         if (!(ok = mbar_wait(part_full_bar(buf), (cit / B128_NBUF) & 1, abort_flag, p.dev_status))) break;
         tc_fence_after();
-        const float sa = kc < chunks ? __ldg(sa_row + kc) : 1.0f;
         const float2 sa2 = make_float2(sa, sa);
         const float4* sb4 = reinterpret_cast<const float4*>(sgb + kc * 128);
 #pragma unroll
