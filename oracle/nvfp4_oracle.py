@@ -242,6 +242,9 @@ class LayerConfig:
     rounding: tuple = (RTN, RTN, SR, SR, SR, SR)
     outliers: np.ndarray | None = None  # sorted channel indices of the set A (columns of X / W), or None
     rht: bool = False  # random Hadamard transformation of both operands of the two backward products (Sec. 4.1)
+    # outlier channels on a per-tensor power-of-two scaled E4M3 grid instead of BF16 (oracle/fp8_outliers.py: this
+    # build's own FP8 recipe, the paper gives none)
+    outlier_fp8: bool = False
 
 
 @dataclass
@@ -277,6 +280,10 @@ def linear_fwd(X: np.ndarray, W: np.ndarray, cfg: LayerConfig):
     Y = gemm_operands(qx, qw)
     X_out = np.ascontiguousarray(X[:, outl])
     W_out = np.ascontiguousarray(W[:, outl])
+    if len(outl) and cfg.outlier_fp8:
+        from oracle import fp8_outliers  # (imports this module)
+
+        X_out, W_out = fp8_outliers.snap(X_out)[0], fp8_outliers.snap(W_out)[0]
     if len(outl):
         Y = Y + gemm_tn(X_out, W_out)
     return Y, Saved(qx, qw, keep, outl, X_out, W_out, D)
