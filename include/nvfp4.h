@@ -213,6 +213,13 @@ typedef struct {
   /* Random Hadamard transformation of both operands of the two backward products (Sec. 4.1): 0 off, 1 on.
    * Q3 and Q4 use sign stream 7 along C, Q5 and Q6 sign stream 8 along the tokens; forward is never transformed. */
   int32_t rht;
+  /* Precision of the outlier channels under OutControl (Sec. 4.2 allows "FP8, BF16"; the paper gives no FP8 recipe, this
+   * one is the library's): 0 = BF16 as they are. 1 = E4M3 with a per-tensor power-of-two scale: forward replaces
+   * X[:, A] and W[:, A] by T8 = E4M3(T / 2^e) 2^e, e the smallest integer with amax|T| / 2^e <= 448 (round to nearest
+   * even; exact scalings), and everything that uses the outlier part (forward side product, dW[:, A], W-hat[:, A]) uses
+   * T8. T8 is exactly representable in BF16, which is how X_out / W_out hold it; products of T8 accumulated in FP32 equal
+   * the FP8 tensor product times the two scales. */
+  int32_t outlier_format;
 } nvfp4_layer_cfg;
 
 /* What forward leaves for backward. qx [N_tok, D - n_out] and qw [C, D - n_out] are filled by

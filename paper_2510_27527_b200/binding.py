@@ -42,7 +42,7 @@ class COperand(ctypes.Structure):
 class CLayerCfg(ctypes.Structure):
     _fields_ = [("gs_mode", c_i32), ("rounding", c_i32 * 6), ("seed", c_u64), ("y_dtype", c_i32), ("dx_dtype", c_i32),
                 ("dw_dtype", c_i32), ("n_out", c_i64), ("outlier_cols", c_vp), ("keep_cols", c_vp), ("col_map", c_vp),
-                ("dev_status", c_vp), ("rht", c_i32)]
+                ("dev_status", c_vp), ("rht", c_i32), ("outlier_format", c_i32)]
 
 
 class CSaved(ctypes.Structure):
@@ -354,6 +354,7 @@ class LayerConfig:
     outliers: np.ndarray | None = None  # sorted outlier channel indices (host)
     dev_status: torch.Tensor | None = None
     rht: bool = False  # random Hadamard transformation of both operands of the two backward products
+    outlier_fp8: bool = False  # outlier channels on a per-tensor power-of-two scaled E4M3 grid instead of BF16
     # device index arrays, built by prepare()
     _outl: torch.Tensor | None = None
     _keep: torch.Tensor | None = None
@@ -381,7 +382,8 @@ class LayerConfig:
 
     def c(self) -> CLayerCfg:
         return CLayerCfg(self.gs_mode, (c_i32 * 6)(*self.rounding), self.seed, self.y_dtype, self.dx_dtype, self.dw_dtype,
-                         self.n_out, _ptr(self._outl), _ptr(self._keep), _ptr(self._map), _ptr(self.dev_status), int(self.rht))
+                         self.n_out, _ptr(self._outl), _ptr(self._keep), _ptr(self._map), _ptr(self.dev_status), int(self.rht),
+                         int(self.outlier_fp8))
 
 
 @dataclass

@@ -224,7 +224,7 @@ nvfp4_status check_cfg(const nvfp4_layer_cfg* cfg, int64_t D) {
   for (int i = 0; i < 6; ++i)
     if (cfg->rounding[i] < 0 || cfg->rounding[i] > 2) return NVFP4_ERR_ENUM;
   if (cfg->y_dtype < 0 || cfg->y_dtype > 1 || cfg->dx_dtype < 0 || cfg->dx_dtype > 1 || cfg->dw_dtype < 0 ||
-      cfg->dw_dtype > 1 || cfg->rht < 0 || cfg->rht > 1)
+      cfg->dw_dtype > 1 || cfg->rht < 0 || cfg->rht > 1 || cfg->outlier_format < 0 || cfg->outlier_format > 1)
     return NVFP4_ERR_ENUM;
   if (cfg->n_out < 0 || cfg->n_out > D) return NVFP4_ERR_SHAPE;
   if (cfg->n_out > 0 && (!cfg->outlier_cols || !cfg->keep_cols || !cfg->col_map)) return NVFP4_ERR_NULL;
@@ -369,6 +369,7 @@ size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, i
   if (op_kind == NVFP4_OP_FWD) {
     carve_size(total, cells_bytes(N_tok, gs_mode));
     carve_size(total, cells_bytes(C, gs_mode));
+    if (n_out > 0) carve_size(total, 16);  // amax cells of the FP8 outlier option
   } else if (op_kind == NVFP4_OP_BWD_DX) {
     carve_size(total, cells_bytes(N_tok, gs_mode));
     carve_size(total, cells_bytes(D, gs_mode));
@@ -443,6 +444,13 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
     return NVFP4_ERR_CUDA;
   if (s_x != NVFP4_OK) return s_x;
   if (s_w != NVFP4_OK) return s_w;
+  if (n_out > 0 && cfg->outlier_format == 1) {  // outlier channels on their scaled E4M3 grids from here on
+    uint32_t* cells_fp8 = static_cast<uint32_t*>(cv.take(16));
+    if (!cells_fp8) return NVFP4_ERR_WORKSPACE;
+    if (launch_fp8_snap_pair(static_cast<uint16_t*>(saved->X_out), N_tok, static_cast<uint16_t*>(saved->W_out), C, Kh, cells_fp8, st) !=
+        cudaSuccess)
+      return NVFP4_ERR_CUDA;
+  }
   saved->X = X; saved->W = W; saved->ldx = ldx; saved->ldw = ldw;
   saved->N_tok = N_tok; saved->D = D; saved->C = C;
   if (n_out > 0)  // Y = FP4 product + X_out W_out^T, both inside one kernel

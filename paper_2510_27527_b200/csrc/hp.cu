@@ -166,6 +166,53 @@ __global__ void __launch_bounds__(256) dw_assemble_kernel(HpDwArgs a, int n_spli
   }
 }
 
+// FP8 option for the outlier channels (paper Sec. 4.2 names FP8 as a possible precision of the outlier part; the recipe
+// is this library's): a compact side operand T (BF16, contiguous) is replaced in place by the values an E4M3 tensor
+// with a per-tensor power-of-two scale represents:  e = smallest integer with amax / 2^e <= 448,  T8 = E4M3(T / 2^e) 2^e.
+// Both scalings are exact and T8 is exactly representable in BF16, so the BF16 tensor-core products that consume the
+// side operands give what an FP8 product times the two scales would give. cell holds the float bits of amax(|T|).
+__device__ __forceinline__ void fp8_snap_body(uint16_t* __restrict__ t, int64_t n, const uint32_t* __restrict__ cell, unsigned block,
+                                              unsigned n_blocks) {
+  const uint32_t ab = cell[0];
+  int e = 0;
+  if (ab) {
+    const int k = (int)((ab >> 23) & 0xFFu) - 127;
+    e = (ab & 0x7FFFFFu) <= 0x600000u ? k - 8 : k - 7;  // mantissa <= 1.75: amax / 2^(k - 8) = m 2^8 <= 448
+  }
+  const float r = __uint_as_float((uint32_t)(127 - e) << 23), s = __uint_as_float((uint32_t)(127 + e) << 23);
+  const int64_t pairs = n >> 1;  // n is even (the padded width is a multiple of 64)
+  uint32_t* t2 = reinterpret_cast<uint32_t*>(t);
+  for (int64_t i = (int64_t)block * blockDim.x + threadIdx.x; i < pairs; i += (int64_t)n_blocks * blockDim.x) {
+    const uint32_t w = t2[i];
+    const float lo = __fmul_rn(bf16_lo(w), r), hi = __fmul_rn(bf16_hi(w), r);
+    uint32_t h2;
+    asm("{\n.reg .b16 q;\ncvt.rn.satfinite.e4m3x2.f32 q, %1, %2;\ncvt.rn.f16x2.e4m3x2 %0, q;\n}" : "=r"(h2) : "f"(hi), "f"(lo));
+    const float qlo = __half2float(__ushort_as_half((unsigned short)(h2 & 0xFFFFu)));
+    const float qhi = __half2float(__ushort_as_half((unsigned short)(h2 >> 16)));
+    t2[i] = (uint32_t)f32_to_bf16_bits(__fmul_rn(qlo, s)) | ((uint32_t)f32_to_bf16_bits(__fmul_rn(qhi, s)) << 16);
+  }
+}
+__global__ void __launch_bounds__(256) fp8_snap_pair_kernel(uint16_t* a, int64_t n_a, const uint32_t* cell_a, unsigned grid_a, uint16_t* b,
+                                                           int64_t n_b, const uint32_t* cell_b) {
+  pdl_prologue();
+  if (blockIdx.x < grid_a)
+    fp8_snap_body(a, n_a, cell_a, blockIdx.x, grid_a);
+  else
+    fp8_snap_body(b, n_b, cell_b, blockIdx.x - grid_a, gridDim.x - grid_a);
+}
+
+cudaError_t launch_fp8_snap_pair(uint16_t* a, int64_t rows_a, uint16_t* b, int64_t rows_b, int64_t Kh, uint32_t* cells2, cudaStream_t st) {
+  if (Kh == 0 || (rows_a == 0 && rows_b == 0)) return cudaSuccess;
+  cudaError_t e;
+  if ((e = launch_zero_words(cells2, 2, st)) != cudaSuccess) return e;
+  if ((e = launch_amax_tensor_pair(a, rows_a, Kh, Kh, cells2, b, rows_b, Kh, Kh, cells2 + 1, st)) != cudaSuccess) return e;
+  auto grid_of = [](int64_t n) { return (unsigned)std::max<int64_t>(1, std::min<int64_t>((n / 2 + 255) / 256, 148 * 4)); };
+  const unsigned ga = grid_of(rows_a * Kh), gb = grid_of(rows_b * Kh);
+  launch_kernel(fp8_snap_pair_kernel, dim3(ga + gb), dim3(256), 0, st, a, rows_a * Kh, static_cast<const uint32_t*>(cells2), ga, b,
+                rows_b * Kh, static_cast<const uint32_t*>(cells2 + 1));
+  return cudaGetLastError();
+}
+
 // dst[r, j] = src[r, cols[j]] (j < n), 0 for n <= j < ld_dst. One warp per row.
 __global__ void __launch_bounds__(256) gather_cols_kernel(const uint16_t* __restrict__ src, int64_t ld_src, int64_t rows,
                                                          const int32_t* __restrict__ cols, int64_t n, uint16_t* __restrict__ dst,

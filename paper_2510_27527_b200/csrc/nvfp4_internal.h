@@ -138,6 +138,10 @@ cudaError_t launch_mma_issue_probe(int32_t iters, int32_t* dev_status, cudaStrea
 cudaError_t launch_gather_cols(const uint16_t* src, int64_t ld_src, int64_t rows, const int32_t* cols, int64_t n, uint16_t* dst,
                                int64_t ld_dst, cudaStream_t st);
 
+// FP8 option of OutControl: both compact side operands ([rows, Kh] BF16, contiguous) snapped in place onto their per-tensor
+// power-of-two scaled E4M3 grids; cells2 = two workspace words.
+cudaError_t launch_fp8_snap_pair(uint16_t* a, int64_t rows_a, uint16_t* b, int64_t rows_b, int64_t Kh, uint32_t* cells2, cudaStream_t st);
+
 struct HpDwArgs {
   const uint16_t *dY, *X_out;  // dY [T, C]; X_out [T, Kh]: the outlier channels of X, compact, zero-padded to Kh (multiple of 64)
   int64_t lddy, Kh, T, C, n_out;

@@ -121,3 +121,52 @@ def test_backward_with_rounded_up_block_scales(gs_mode, outcontrol, rht):
     torch.cuda.synchronize()
     assert rel_fro(dX.float().cpu().numpy(), dXo) <= 2e-5
     assert rel_fro(dW.float().cpu().numpy(), dWo) <= 2e-5
+
+
+@pytest.mark.parametrize("gs_mode", [0, 1, 2])
+@pytest.mark.parametrize("rht", [False, True])
+def test_fp8_outlier_channels(gs_mode, rht):
+    """OutControl with the outlier channels on their per-tensor power-of-two scaled E4M3 grids: the side operands are the
+    oracle's bit for bit, and forward / dX / dW follow."""
+    from oracle import fp8_outliers as f8
+
+    b = B()
+    N_tok, D, C = 200, 272, 136
+    X, W, dY, ch = synth.layer_inputs(21, N_tok, D, C, n_outlier=5, factor=40.0, grad_scale=1e-3)
+    ocfg = orc.LayerConfig(gs_mode=gs_mode, seed=2, outliers=ch, rht=rht, outlier_fp8=True)
+    Yo, so = orc.linear_fwd(X, W, ocfg)
+    dXo, dWo = orc.linear_bwd_dx(dY, so, ocfg), orc.linear_bwd_dw(dY, so, ocfg)
+    cfg = b.LayerConfig(gs_mode=gs_mode, seed=2, outliers=ch, rht=rht, outlier_fp8=True, y_dtype=b.DT_F32, dx_dtype=b.DT_F32,
+                        dw_dtype=b.DT_F32)
+    Xd, Wd, dYd = to_dev_bf16(X), to_dev_bf16(W), to_dev_bf16(dY)
+    Y, saved = b.nvfp4_linear_fwd(Xd, Wd, cfg)
+    dX, dW = b.nvfp4_linear_bwd(dYd, saved, cfg)
+    torch.cuda.synchronize()
+    n = len(ch)
+    X8 = saved.X_out.float().cpu().numpy()
+    W8 = saved.W_out.float().cpu().numpy()
+    assert np.array_equal(X8[:, :n], f8.snap(X[:, ch])[0]) and np.all(X8[:, n:] == 0)
+    assert np.array_equal(W8[:, :n], f8.snap(W[:, ch])[0]) and np.all(W8[:, n:] == 0)
+    assert not np.array_equal(X8[:, :n], X[:, ch])  # the option does something on these inputs
+    assert rel_fro(Y.float().cpu().numpy(), Yo) <= 2e-5
+    assert rel_fro(dX.float().cpu().numpy(), dXo) <= 2e-5
+    assert rel_fro(dW.float().cpu().numpy(), dWo) <= 2e-5
+
+
+def test_fp8_outlier_snap_extremes():
+    """Scale exponents far from zero, an all-zero slice, exact powers of two and values that fall below the E4M3 grid."""
+    from oracle import fp8_outliers as f8
+
+    b = B()
+    rng = np.random.default_rng(77)
+    for scale in (2.0 ** -40, 1.0, 448.0, 2.0 ** 30, 0.0):
+        X = (rng.standard_normal((64, 32)) * scale).astype(np.float32)
+        X[:, 3] *= np.float32(2.0 ** -12)  # a column that lands in the subnormal range of the scaled grid or below it
+        X = torch.from_numpy(X).to(torch.bfloat16).float().numpy()
+        W = torch.from_numpy((rng.standard_normal((16, 32)) * 0.02).astype(np.float32)).to(torch.bfloat16).float().numpy()
+        ch = np.array([1, 3, 8, 30])
+        cfg = b.LayerConfig(gs_mode=0, seed=0, outliers=ch, outlier_fp8=True, y_dtype=b.DT_F32)
+        _, saved = b.nvfp4_linear_fwd(to_dev_bf16(X), to_dev_bf16(W), cfg)
+        torch.cuda.synchronize()
+        assert np.array_equal(saved.X_out.float().cpu().numpy()[:, :4], f8.snap(X[:, ch])[0]), scale
+        assert np.array_equal(saved.W_out.float().cpu().numpy()[:, :4], f8.snap(W[:, ch])[0]), scale
