@@ -80,9 +80,10 @@ __global__ void __launch_bounds__(256) amax_tensor_pair_kernel(const uint16_t* _
 }
 
 // amax of a BF16 matrix over all columns EXCEPT a sorted list of excluded ones (OutControl: the outlier channels do not
-// take part in the FP4 operand's tensor scale). Each CTA builds a one-bit-per-column mask in shared memory from the
-// list, then streams a contiguous slab of rows with 16-byte loads (four in flight per thread), zeroing the excluded
-// lanes. Folded into cells[0] by atomic max.
+// take part in the FP4 operand's tensor scale). Each CTA builds, in shared memory, one 16-byte AND mask per 8-column
+// chunk (0x7FFF for a column that takes part: the sign goes with it; 0 for an excluded one or one past the end), then
+// streams a contiguous slab of rows with 16-byte loads: per chunk one mask load, four ANDs and four packed maxima.
+// The (row, chunk) position of a thread advances by additions only. Folded into cells[0] by atomic max.
 // With `out` the excluded columns of the slab are then copied, in list order, to out[r, 0 .. n_excl) (zero up to ld_out):
 // the high-precision side operand, picked from rows this CTA has just pulled through L1 / L2.
 __global__ void __launch_bounds__(256) amax_tensor_masked_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols,
@@ -90,53 +91,46 @@ __global__ void __launch_bounds__(256) amax_tensor_masked_kernel(const uint16_t*
                                                                 uint32_t* amax_bits, uint16_t* __restrict__ out, int64_t ld_out,
                                                                 int64_t rows_per_cta) {
   pdl_prologue();
-  extern __shared__ uint32_t keep_bits[];  // bit c = 1: column c takes part
-  const int64_t words = (cols + 31) >> 5;
-  for (int64_t i = threadIdx.x; i < words; i += 256) keep_bits[i] = 0xFFFFFFFFu;
+  extern __shared__ __align__(16) uint16_t lane_mask[];  // [chunks * 8]
+  const uint32_t chunks = (uint32_t)((cols + 7) >> 3);
+  for (uint32_t i = threadIdx.x; i < chunks * 8; i += 256) lane_mask[i] = (int64_t)i < cols ? (uint16_t)0x7FFFu : (uint16_t)0;
   __syncthreads();
-  for (int64_t i = threadIdx.x; i < n_excl; i += 256) atomicAnd(&keep_bits[excluded[i] >> 5], ~(1u << (excluded[i] & 31)));
+  for (int64_t i = threadIdx.x; i < n_excl; i += 256) lane_mask[excluded[i]] = 0;
   __syncthreads();
   const int64_t r0 = (int64_t)blockIdx.x * rows_per_cta;
   const int64_t r1 = min(rows, r0 + rows_per_cta);
-  const uint32_t chunks = (uint32_t)((cols + 7) >> 3);
-  const uint32_t n_items = r1 > r0 ? (uint32_t)(r1 - r0) * chunks : 0u;  // (row, chunk) pairs of the slab, row-major
-  const uint64_t inv = (1ull << 32) / chunks + 1ull;                    // item / chunks by multiplication
+  const uint32_t n_rows = r1 > r0 ? (uint32_t)(r1 - r0) : 0u;
+  // thread t starts at item t of the slab (row-major (row, chunk) pairs) and advances by 256 items
+  const uint32_t step_r = 256u / chunks, step_c = 256u % chunks;
+  uint32_t rr = threadIdx.x / chunks, c = threadIdx.x % chunks;
+  const bool row_tail = (cols & 7) != 0;  // the last chunk of a row is ragged: read element by element
   uint32_t m = 0;
-  for (uint32_t e0 = threadIdx.x; e0 < n_items; e0 += 256 * 4) {
-    uint32_t w[4][4], mask8[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const uint32_t e = e0 + u * 256;
-      w[u][0] = w[u][1] = w[u][2] = w[u][3] = 0;
-      mask8[u] = 0;
-      if (e < n_items) {
-        const uint32_t rr = (uint32_t)(((uint64_t)e * inv) >> 32), c = e - rr * chunks;
-        const uint16_t* p = src + (r0 + rr) * ld + ((int64_t)c << 3);
-        mask8[u] = (keep_bits[c >> 2] >> ((c & 3) * 8)) & 0xFFu;
-        if (((int64_t)c << 3) + 8 <= cols) {
-          const uint4 v = *reinterpret_cast<const uint4*>(p);
-          w[u][0] = v.x; w[u][1] = v.y; w[u][2] = v.z; w[u][3] = v.w;
-        } else {
-          for (int q = 0; q < 8; ++q)
-            if (((int64_t)c << 3) + q < cols) w[u][q >> 1] |= (uint32_t)p[q] << (16 * (q & 1));
-        }
-      }
+  while (rr < n_rows) {
+    const uint16_t* p = src + (r0 + rr) * ld + ((int64_t)c << 3);
+    uint4 v;
+    if (!row_tail || c + 1 < chunks) {
+      v = *reinterpret_cast<const uint4*>(p);
+    } else {
+      uint32_t t[4] = {0, 0, 0, 0};
+      for (int q = 0; q < 8; ++q)
+        if (((int64_t)c << 3) + q < cols) t[q >> 1] |= (uint32_t)p[q] << (16 * (q & 1));
+      v = make_uint4(t[0], t[1], t[2], t[3]);
     }
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const uint32_t two = (mask8[u] >> (2 * q)) & 3u;
-        const uint32_t lanes = ((0u - (two & 1u)) & 0x0000FFFFu) | ((0u - (two >> 1)) & 0xFFFF0000u);
-        m = umax16x2(m, bf16x2_abs_bits(w[u][q]) & lanes);
-      }
+    const uint4 k = *reinterpret_cast<const uint4*>(lane_mask + (c << 3));
+    m = umax16x2(m, umax16x2(umax16x2(v.x & k.x, v.y & k.y), umax16x2(v.z & k.z, v.w & k.w)));
+    c += step_c;
+    rr += step_r;
+    if (c >= chunks) {
+      c -= chunks;
+      rr += 1;
+    }
   }
-  if (out && r1 > r0) {
-    const uint32_t ldo = (uint32_t)ld_out, n_out_items = (uint32_t)(r1 - r0) * ldo;
+  if (out && n_rows) {
+    const uint32_t ldo = (uint32_t)ld_out, n_out_items = n_rows * ldo;
     const uint64_t inv_o = (1ull << 32) / ldo + 1ull;
     for (uint32_t e = threadIdx.x; e < n_out_items; e += 256) {
-      const uint32_t rr = (uint32_t)(((uint64_t)e * inv_o) >> 32), j = e - rr * ldo;
-      out[(r0 + rr) * ld_out + j] = j < n_excl ? src[(r0 + rr) * ld + excluded[j]] : (uint16_t)0;
+      const uint32_t ro = (uint32_t)(((uint64_t)e * inv_o) >> 32), j = e - ro * ldo;
+      out[(r0 + ro) * ld_out + j] = j < n_excl ? src[(r0 + ro) * ld + excluded[j]] : (uint16_t)0;
     }
   }
   uint32_t a = hmax_of_pair(m);
@@ -841,11 +835,11 @@ static cudaError_t launch_quantize_rows_impl(const QuantRowsArgs& a, cudaStream_
   if (a.gs_mode == kGsTensor) {
     if (a.compute_amax) {
       if (!a.cells_zeroed && (e = launch_zero_words(a.gs_cells, 1, st)) != cudaSuccess) return e;
-      if (a.keep && a.excluded && (a.ld & 7) == 0 && a.cols_src <= 256 * 1024) {
+      if (a.keep && a.excluded && (a.ld & 7) == 0 && a.cols_src <= 20 * 1024) {
         // amax over the kept columns only: full-width vector loads with the excluded (outlier) columns masked out
-        const size_t smem = (size_t)((a.cols_src + 31) >> 5) * 4;
-        // a contiguous slab of rows per CTA. The kernel divides item numbers by d = chunks per row (and by the side
-        // operand's width) through a 32-bit reciprocal, exact while items * d < 2^32: slabs stay below 2^32 / d^2 rows
+        const size_t smem = (size_t)((a.cols_src + 7) >> 3) * 16;  // one 16-byte mask per chunk (at most 40 KB)
+        // a contiguous slab of rows per CTA. The side copy divides item numbers by the side operand's width through a
+        // 32-bit reciprocal, exact while items * width < 2^32: slabs stay below 2^32 / d^2 rows (d also covers the chunk count)
         int64_t rows_per_cta = (a.rows + 148 * 8 - 1) / (148 * 8);
         const int64_t dmax = std::max<int64_t>((a.cols_src + 7) >> 3, a.excl_out ? a.ld_excl_out : 1);
         rows_per_cta = std::max<int64_t>(1, std::min<int64_t>(rows_per_cta, (((int64_t)1 << 32) - 1) / (dmax * dmax)));
