@@ -245,6 +245,9 @@ class LayerConfig:
     # outlier channels on a per-tensor power-of-two scaled E4M3 grid instead of BF16 (oracle/fp8_outliers.py: this
     # build's own FP8 recipe, the paper gives none)
     outlier_fp8: bool = False
+    # weights in 16x16 scale squares (the recipe the paper compares its 1x16 blocks with; oracle/w16x16.py): per-tensor
+    # global scale only, no outlier channels; dX then uses the forward codes as they are (no Q4, no Hadamard factor)
+    w_block16: bool = False
 
 
 @dataclass
@@ -276,7 +279,13 @@ def linear_fwd(X: np.ndarray, W: np.ndarray, cfg: LayerConfig):
     D = X.shape[1]
     keep, outl = _split(D, cfg.outliers)
     qx = quantize(X[:, keep], AXIS_ROW, cfg.rounding[0], cfg.gs_mode, cfg.seed, 1)
-    qw = quantize(W[:, keep], AXIS_ROW, cfg.rounding[1], cfg.gs_mode, cfg.seed, 2)
+    if cfg.w_block16:
+        from oracle import w16x16  # (imports this module)
+
+        assert cfg.gs_mode == GS_TENSOR and len(outl) == 0 and cfg.rounding[1] == RTN
+        qw = w16x16.quantize(W)
+    else:
+        qw = quantize(W[:, keep], AXIS_ROW, cfg.rounding[1], cfg.gs_mode, cfg.seed, 2)
     Y = gemm_operands(qx, qw)
     X_out = np.ascontiguousarray(X[:, outl])
     W_out = np.ascontiguousarray(W[:, outl])
@@ -301,6 +310,11 @@ def aligned_full(op: Operand, keep: np.ndarray, outl: np.ndarray, hp_cols: np.nd
 def linear_bwd_dx(dY: np.ndarray, saved: Saved, cfg: LayerConfig) -> np.ndarray:
     """dX = Q3_S(dY) Q4_S(W-hat): one FP4 product over all D columns. dY [N_tok, C] -> dX [N_tok, D]."""
     dY = np.asarray(dY, dtype=np.float32)
+    if cfg.w_block16:
+        from oracle import w16x16
+
+        q3 = quantize(dY, AXIS_ROW, cfg.rounding[2], cfg.gs_mode, cfg.seed, STREAM_Q3)
+        return gemm_operands(q3, w16x16.transpose_operand(saved.qw))
     W_hat = aligned_full(saved.qw, saved.keep, saved.outl, saved.W_out, saved.D)  # [C, D]
     A, B = dY, np.ascontiguousarray(W_hat.T)  # [N_tok, C], [D, C]: both along the contraction axis C
     if cfg.rht:
