@@ -216,7 +216,7 @@ def run_ours(args):
         outl = synth.outlier_channels(D, n_out, synth.seed_of(cfg_id, 50 + li)) if n_out else None
         rounding = (b.ROUND_RTN, b.ROUND_RTN) + ((b.ROUND_SR_SCALE_UP,) * 4 if args.sr_scale_up else (b.ROUND_SR,) * 4)
         L.cfg = b.LayerConfig(gs_mode=gs_mode, seed=0, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32, outliers=outl, rht=args.rht,
-                              rounding=rounding, outlier_fp8=args.outlier_fp8)
+                              rounding=rounding, outlier_fp8=args.outlier_fp8, w_block16=args.w16x16)
         L.cfg.prepare(D, dev)
         L.saved = b.alloc_saved(L.X, L.W[0], L.cfg)
         L.Y = torch.empty((tokens, C), dtype=torch.bfloat16, device=dev)
@@ -430,7 +430,7 @@ def run_ours(args):
         "metric": "nvfp4_linear_fwd_bwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "fp4(e2m1)xfp4 with ue4m3 block scales, f32 accumulate", "data": "synthetic",
-        "config": {"workload": workload_name(args), "gs_mode": args.gs, "outcontrol_fraction": args.outliers, "rht": bool(args.rht), "sr_scale_up": bool(args.sr_scale_up), "outlier_fp8": bool(args.outlier_fp8), "launch": "cuda_graph_replay" if args.graph else "stream", "l2": "256 MiB write + 256 MiB read flush before every timed step",
+        "config": {"workload": workload_name(args), "gs_mode": args.gs, "outcontrol_fraction": args.outliers, "rht": bool(args.rht), "sr_scale_up": bool(args.sr_scale_up), "outlier_fp8": bool(args.outlier_fp8), "weight_block": "16x16" if args.w16x16 else "1x16", "launch": "cuda_graph_replay" if args.graph else "stream", "l2": "256 MiB write + 256 MiB read flush before every timed step",
                    "timing": "CUDA events per step on the launch stream, summed"},
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
@@ -626,6 +626,7 @@ def main():
                     help="OutControl: fraction of input channels kept in BF16 (0 = off; the paper uses 0.10)")
     ap.add_argument("--rht", action="store_true", help="random Hadamard transformation (block 16) in the four backward quantizers")
     ap.add_argument("--outlier-fp8", action="store_true", help="with --outliers: outlier channels on a power-of-two scaled E4M3 grid instead of BF16")
+    ap.add_argument("--w16x16", action="store_true", help="weights in 16x16 scale squares (the recipe the paper compares with): no Q4 in backward")
     ap.add_argument("--sr-scale-up", action="store_true", help="backward quantizers round the block scale up (strictly unbiased variant)")
     ap.add_argument("--graph", action=argparse.BooleanOptionalAction, default=True,
                     help="capture one step in a CUDA graph and time its replays (default; --no-graph launches every kernel from the host)")

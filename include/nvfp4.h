@@ -155,6 +155,21 @@ nvfp4_status nvfp4_quantize_static(const void* src_bf16, int64_t rows, int64_t c
                                    int64_t n_keep, const nvfp4_operand* out, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------
+ * nvfp4_quantize_w16x16 / nvfp4_transpose_operand16 -- the two pieces of the 16x16 weight-block recipe (see
+ * nvfp4_layer_cfg.weight_block), exposed for tests and for callers that drive the GEMMs themselves.
+ *
+ *   nvfp4_quantize_w16x16: W_bf16 [C, D] (leading dimension ldw, multiple of 8) -> out [C, D], gs_mode TENSOR, either scale
+ *     layout. amax_b is taken over 16x16 squares (ragged squares cover the rows / columns that exist); round to nearest.
+ *     workspace: nvfp4_quantize_workspace_bytes(C, NVFP4_GS_TENSOR).
+ *   nvfp4_transpose_operand16: in [C, D] made by nvfp4_quantize_w16x16 -> out [D, C] (gs_mode TENSOR): the operand of
+ *     W-hat^T with identical values; pure data movement. in and out must not overlap.
+ *   Errors: NVFP4_ERR_NULL, _SHAPE (out shape), _ENUM (gs_mode), _ALIGN, _WORKSPACE, _ARCH, _CUDA.
+ * ------------------------------------------------------------------------------------------------------- */
+nvfp4_status nvfp4_quantize_w16x16(const void* W_bf16, int64_t C, int64_t D, int64_t ldw, const nvfp4_operand* out,
+                                   void* workspace, size_t ws_bytes, void* stream);
+nvfp4_status nvfp4_transpose_operand16(const nvfp4_operand* in, const nvfp4_operand* out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------
  * nvfp4_requantize_t — the backward quantizers Q4 / Q6 of Sec. 2.3: dequantize a forward operand to the
  * aligned tensor (x_hat = (P * S_block) * S_global, one binary32 rounding), and quantize its TRANSPOSE.
  *
@@ -220,6 +235,12 @@ typedef struct {
    * T8. T8 is exactly representable in BF16, which is how X_out / W_out hold it; products of T8 accumulated in FP32 equal
    * the FP8 tensor product times the two scales. */
   int32_t outlier_format;
+  /* Weight scale group (Sec. 2.3, third difference to NVIDIA's recipe; appendix on the overhead of the 1x16 scheme):
+   * 0 = 1x16 blocks, the paper's choice. 1 = 16x16 squares, the recipe it is compared with: Q2 takes amax_b over the
+   * square (same pinned scale arithmetic, round to nearest), the 16 rows of a square repeat its scale byte, and dX uses
+   * the forward codes transposed as they are -- no Q4, so no rounding, no random bits and no Hadamard factor on the dX
+   * product (cfg.rht then applies to dW only). Requires gs_mode TENSOR, n_out = 0 and rounding[1] = RTN (NVFP4_ERR_ENUM). */
+  int32_t weight_block;
 } nvfp4_layer_cfg;
 
 /* What forward leaves for backward. qx [N_tok, D - n_out] and qw [C, D - n_out] are filled by

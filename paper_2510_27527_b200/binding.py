@@ -42,7 +42,7 @@ class COperand(ctypes.Structure):
 class CLayerCfg(ctypes.Structure):
     _fields_ = [("gs_mode", c_i32), ("rounding", c_i32 * 6), ("seed", c_u64), ("y_dtype", c_i32), ("dx_dtype", c_i32),
                 ("dw_dtype", c_i32), ("n_out", c_i64), ("outlier_cols", c_vp), ("keep_cols", c_vp), ("col_map", c_vp),
-                ("dev_status", c_vp), ("rht", c_i32), ("outlier_format", c_i32)]
+                ("dev_status", c_vp), ("rht", c_i32), ("outlier_format", c_i32), ("weight_block", c_i32)]
 
 
 class CSaved(ctypes.Structure):
@@ -66,6 +66,8 @@ EXPORTS = {
                                       ctypes.POINTER(COperand), c_vp]),
     "nvfp4_requantize_t": (c_i32, [ctypes.POINTER(COperand), c_vp, c_i64, c_vp, c_i64, c_i32, c_u64, c_u32, c_u32,
                                    ctypes.POINTER(COperand), c_vp, c_sz, c_vp]),
+    "nvfp4_quantize_w16x16": (c_i32, [c_vp, c_i64, c_i64, c_i64, ctypes.POINTER(COperand), c_vp, c_sz, c_vp]),
+    "nvfp4_transpose_operand16": (c_i32, [ctypes.POINTER(COperand), ctypes.POINTER(COperand), c_vp]),
     "nvfp4_gemm_workspace_bytes": (c_sz, [c_i64, c_i64, c_i64]),
     "nvfp4_gemm": (c_i32, [ctypes.POINTER(COperand), ctypes.POINTER(COperand), c_vp, c_i32, c_i64, c_i32, c_vp, c_vp,
                            c_sz, c_vp]),
@@ -230,6 +232,28 @@ def nvfp4_requantize_t(inp: Operand, rounding: int = ROUND_SR, seed: int = 0, st
     return out
 
 
+def nvfp4_quantize_w16x16(W: torch.Tensor, sf_layout: int = SF_TILED128x4, out: Operand | None = None,
+                          workspace: torch.Tensor | None = None) -> Operand:
+    """Q2 of the 16x16 weight-block recipe: one E4M3 scale per 16x16 square, per-tensor global scale, round to nearest."""
+    C, D = W.shape
+    if out is None:
+        out = alloc_operand(C, D, GS_TENSOR, sf_layout, W.device)
+    ws = workspace if workspace is not None else _workspace(_lib.nvfp4_quantize_workspace_bytes(C, GS_TENSOR), W.device)
+    co = out.c()
+    _check(_lib.nvfp4_quantize_w16x16(_ptr(W), C, D, W.stride(0), ctypes.byref(co), _ptr(ws), ws.numel(), _stream_ptr()),
+           "nvfp4_quantize_w16x16")
+    return out
+
+
+def nvfp4_transpose_operand16(inp: Operand, sf_layout: int = SF_TILED128x4, out: Operand | None = None) -> Operand:
+    """Operand of W-hat^T from the 16x16-block operand of W (codes transposed, scales re-indexed; no arithmetic)."""
+    if out is None:
+        out = alloc_operand(inp.K, inp.R, GS_TENSOR, sf_layout, inp.codes.device)
+    ci, co = inp.c(), out.c()
+    _check(_lib.nvfp4_transpose_operand16(ctypes.byref(ci), ctypes.byref(co), _stream_ptr()), "nvfp4_transpose_operand16")
+    return out
+
+
 def nvfp4_gemm(A: Operand, B: Operand, c_dtype: int = DT_F32, out: torch.Tensor | None = None, accumulate: bool = False,
                dev_status: torch.Tensor | None = None, workspace: torch.Tensor | None = None) -> torch.Tensor:
     if out is None:
@@ -355,6 +379,7 @@ class LayerConfig:
     dev_status: torch.Tensor | None = None
     rht: bool = False  # random Hadamard transformation of both operands of the two backward products
     outlier_fp8: bool = False  # outlier channels on a per-tensor power-of-two scaled E4M3 grid instead of BF16
+    w_block16: bool = False  # weights in 16x16 scale squares (comparison recipe): dX uses the forward codes transposed, no Q4
     # device index arrays, built by prepare()
     _outl: torch.Tensor | None = None
     _keep: torch.Tensor | None = None
@@ -383,7 +408,7 @@ class LayerConfig:
     def c(self) -> CLayerCfg:
         return CLayerCfg(self.gs_mode, (c_i32 * 6)(*self.rounding), self.seed, self.y_dtype, self.dx_dtype, self.dw_dtype,
                          self.n_out, _ptr(self._outl), _ptr(self._keep), _ptr(self._map), _ptr(self.dev_status), int(self.rht),
-                         int(self.outlier_fp8))
+                         int(self.outlier_fp8), int(self.w_block16))
 
 
 @dataclass

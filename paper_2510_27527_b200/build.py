@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnvfp4_b200.so")
-SOURCES = ["api.cu", "quantize.cu", "gemm.cu", "hp.cu", "noalloc.cu", "calib.cu", "osci.cu"]
+SOURCES = ["api.cu", "quantize.cu", "gemm.cu", "hp.cu", "noalloc.cu", "calib.cu", "osci.cu", "w16.cu"]
 HEADERS = ["nvfp4_device.cuh", "nvfp4_internal.h", os.path.join("..", "..", "include", "nvfp4.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

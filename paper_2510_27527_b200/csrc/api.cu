@@ -224,7 +224,10 @@ nvfp4_status check_cfg(const nvfp4_layer_cfg* cfg, int64_t D) {
   for (int i = 0; i < 6; ++i)
     if (cfg->rounding[i] < 0 || cfg->rounding[i] > 2) return NVFP4_ERR_ENUM;
   if (cfg->y_dtype < 0 || cfg->y_dtype > 1 || cfg->dx_dtype < 0 || cfg->dx_dtype > 1 || cfg->dw_dtype < 0 ||
-      cfg->dw_dtype > 1 || cfg->rht < 0 || cfg->rht > 1 || cfg->outlier_format < 0 || cfg->outlier_format > 1)
+      cfg->dw_dtype > 1 || cfg->rht < 0 || cfg->rht > 1 || cfg->outlier_format < 0 || cfg->outlier_format > 1 ||
+      cfg->weight_block < 0 || cfg->weight_block > 1)
+    return NVFP4_ERR_ENUM;
+  if (cfg->weight_block == 1 && (cfg->gs_mode != NVFP4_GS_TENSOR || cfg->n_out != 0 || cfg->rounding[1] != NVFP4_ROUND_RTN))
     return NVFP4_ERR_ENUM;
   if (cfg->n_out < 0 || cfg->n_out > D) return NVFP4_ERR_SHAPE;
   if (cfg->n_out > 0 && (!cfg->outlier_cols || !cfg->keep_cols || !cfg->col_map)) return NVFP4_ERR_NULL;
@@ -311,6 +314,49 @@ nvfp4_status nvfp4_quantize(const void* src_bf16, int64_t rows, int64_t cols, in
   ts.bf16 = static_cast<const uint16_t*>(src_bf16);
   ts.ld = ld;
   return do_quantize_transpose(ts, 0, rows, cols, rounding, seed, stream_id, out, cells, st, 0, rht_stream_id);
+}
+
+nvfp4_status nvfp4_quantize_w16x16(const void* W_bf16, int64_t C, int64_t D, int64_t ldw, const nvfp4_operand* out,
+                                   void* workspace, size_t ws_bytes, void* stream) {
+  if (!W_bf16 || !out) return NVFP4_ERR_NULL;
+  if (C < 0 || D < 0) return NVFP4_ERR_SHAPE;
+  nvfp4_status s;
+  if ((s = check_operand_ptrs(out)) != NVFP4_OK) return s;
+  if (out->R != C || out->K != D) return NVFP4_ERR_SHAPE;
+  if (out->gs_mode != NVFP4_GS_TENSOR) return NVFP4_ERR_ENUM;
+  if (bad_matrix(W_bf16, ldw, D, 2)) return NVFP4_ERR_ALIGN;
+  if (!workspace || !aligned16(workspace) || ws_bytes < nvfp4_quantize_workspace_bytes(C, NVFP4_GS_TENSOR)) return NVFP4_ERR_WORKSPACE;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  if (C == 0 || D == 0) return NVFP4_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t* cell = static_cast<uint32_t*>(workspace);
+  if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+  if (launch_zero_words(cell, 1, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+  if (launch_amax_tensor(static_cast<const uint16_t*>(W_bf16), C, D, ldw, cell, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+  return launch_quantize_w16(static_cast<const uint16_t*>(W_bf16), C, D, ldw, cell, out->codes, out->sf, out->gscale,
+                             out->sf_layout == NVFP4_SF_TILED128x4, st) == cudaSuccess
+             ? NVFP4_OK
+             : NVFP4_ERR_CUDA;
+}
+
+static nvfp4_status do_transpose_operand16(const nvfp4_operand* in, const nvfp4_operand* out, cudaStream_t st) {
+  if (clear_sf_padding(out, st) != cudaSuccess) return NVFP4_ERR_CUDA;
+  return launch_transpose_operand(in->codes, in->sf, in->sf_layout == NVFP4_SF_TILED128x4, in->gscale, in->R, in->K, out->codes, out->sf,
+                                  out->sf_layout == NVFP4_SF_TILED128x4, out->gscale, st) == cudaSuccess
+             ? NVFP4_OK
+             : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_transpose_operand16(const nvfp4_operand* in, const nvfp4_operand* out, void* stream) {
+  if (!in || !out) return NVFP4_ERR_NULL;
+  nvfp4_status s;
+  if ((s = check_operand_ptrs(in)) != NVFP4_OK) return s;
+  if ((s = check_operand_ptrs(out)) != NVFP4_OK) return s;
+  if (out->R != in->K || out->K != in->R) return NVFP4_ERR_SHAPE;
+  if (in->gs_mode != NVFP4_GS_TENSOR || out->gs_mode != NVFP4_GS_TENSOR) return NVFP4_ERR_ENUM;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  if (in->R == 0 || in->K == 0) return NVFP4_OK;
+  return do_transpose_operand16(in, out, static_cast<cudaStream_t>(stream));
 }
 
 nvfp4_status nvfp4_requantize_t(const nvfp4_operand* in, const void* hp_bf16, int64_t hp_ld, const int32_t* row_map,
@@ -437,9 +483,17 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
     return NVFP4_ERR_CUDA;
   const nvfp4_status s_x = do_quantize_rows(Xp, N_tok, D, ldx, cfg->rounding[0], cfg->seed, 1, keep, Dk, &saved->qx, cells_x, st, 1,
                                             cfg->outlier_cols, 0, amax_pass, static_cast<uint16_t*>(saved->X_out), Kh);
-  const nvfp4_status s_w = do_quantize_rows(Wp, C, D, ldw, cfg->rounding[1], cfg->seed, 2, keep, Dk, &saved->qw, cells_w,
-                                            side ? side->stream : st, 1, cfg->outlier_cols, 0, amax_pass,
-                                            static_cast<uint16_t*>(saved->W_out), Kh);
+  nvfp4_status s_w;
+  if (cfg->weight_block == 1) {  // 16x16 scale squares (TENSOR mode: amax(W) is already in cells_w)
+    cudaStream_t sw = side ? side->stream : st;
+    s_w = clear_sf_padding(&saved->qw, sw) == cudaSuccess &&
+                  launch_quantize_w16(Wp, C, D, ldw, cells_w, saved->qw.codes, saved->qw.sf, saved->qw.gscale, 1, sw) == cudaSuccess
+              ? NVFP4_OK
+              : NVFP4_ERR_CUDA;
+  } else {
+    s_w = do_quantize_rows(Wp, C, D, ldw, cfg->rounding[1], cfg->seed, 2, keep, Dk, &saved->qw, cells_w, side ? side->stream : st, 1,
+                           cfg->outlier_cols, 0, amax_pass, static_cast<uint16_t*>(saved->W_out), Kh);
+  }
   if (side && (cudaEventRecord(side->join, side->stream) != cudaSuccess || cudaStreamWaitEvent(st, side->join, 0) != cudaSuccess))
     return NVFP4_ERR_CUDA;
   if (s_x != NVFP4_OK) return s_x;
@@ -486,10 +540,15 @@ static nvfp4_status bwd_dx_impl(const void* dY, int64_t lddy, const nvfp4_saved*
   const bool cells_unused = cfg->gs_mode == NVFP4_GS_BLOCK128 ||
                             (dy_amax && n_out == 0 && cfg->gs_mode == NVFP4_GS_TENSOR && saved->qw.gs_mode == NVFP4_GS_TENSOR && !cfg->rht);
   if (!cells_unused && !zero_cells(cells3, cells4, cells_bytes(D, cfg->gs_mode), st)) return NVFP4_ERR_CUDA;
-  const uint32_t rht = cfg->rht ? kRhtStreamDx : 0u;
+  // (16x16 weight squares: W-hat^T is the forward operand transposed as it is, so this product takes no Hadamard factor)
+  const uint32_t rht = cfg->rht && cfg->weight_block == 0 ? kRhtStreamDx : 0u;
   if ((s = do_quantize_rows(static_cast<const uint16_t*>(dY), N_tok, C, lddy, cfg->rounding[2], cfg->seed, 3, nullptr, 0,
                             &q3, dy_amax ? dy_amax : cells3, st, 1, nullptr, rht, dy_amax ? 0 : 1)) != NVFP4_OK)
     return s;
+  if (cfg->weight_block == 1) {
+    if ((s = do_transpose_operand16(&saved->qw, &q4, st)) != NVFP4_OK) return s;
+    return do_gemm(&q3, &q4, dX, cfg->dx_dtype, lddx, 0, nullptr, 0, cfg->dev_status, st);
+  }
   TransposeSrc ts{};
   ts.in_codes = saved->qw.codes;
   ts.in_sf = saved->qw.sf;

@@ -281,6 +281,27 @@ __device__ __forceinline__ void decode8(uint32_t word, uint32_t sf_byte, float s
   }
 }
 
+// Scale, round and pack one 16-element inner block (two code words).
+template <bool SR>
+__device__ __forceinline__ uint2 quantize_block16(const float (&x)[16], float rcp, const PhiloxKeys& pk, uint32_t stream_id,
+                                                  uint64_t idx8) {
+  float y0[8], y1[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    y0[i] = __fmul_rn(x[i], rcp);
+    y1[i] = __fmul_rn(x[8 + i], rcp);
+  }
+  uint2 out;
+  if (SR) {
+    out.x = e2m1x8_sr(y0, sr_words(pk, stream_id, idx8));
+    out.y = e2m1x8_sr(y1, sr_words(pk, stream_id, idx8 + 1));
+  } else {
+    out.x = e2m1x8_rtn(y0);
+    out.y = e2m1x8_rtn(y1);
+  }
+  return out;
+}
+
 // Byte offset of scale (r, kb) in the TILED128x4 layout with n_ktiles4 = (number of k-blocks, padded to 16) / 4.
 __device__ __forceinline__ size_t sf_tiled_offset(int64_t r, int64_t kb, int64_t kb_padded) {
   const int64_t tile = (r >> 7) * (kb_padded >> 2) + (kb >> 2);

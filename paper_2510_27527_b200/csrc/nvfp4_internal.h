@@ -138,6 +138,13 @@ cudaError_t launch_mma_issue_probe(int32_t iters, int32_t* dev_status, cudaStrea
 cudaError_t launch_gather_cols(const uint16_t* src, int64_t ld_src, int64_t rows, const int32_t* cols, int64_t n, uint16_t* dst,
                                int64_t ld_dst, cudaStream_t st);
 
+// 16x16 weight-block recipe: Q2 with one E4M3 scale per 16x16 square (per-tensor global scale from amax_cell, round to
+// nearest), and the transposition of such an operand (codes transposed, scales re-indexed) that replaces Q4.
+cudaError_t launch_quantize_w16(const uint16_t* src, int64_t C, int64_t D, int64_t ld, const uint32_t* amax_cell, uint8_t* codes,
+                                uint8_t* sf, float* gscale, int tiled, cudaStream_t st);
+cudaError_t launch_transpose_operand(const uint8_t* in_codes, const uint8_t* in_sf, int in_tiled, const float* in_gscale, int64_t C, int64_t D,
+                                     uint8_t* out_codes, uint8_t* out_sf, int out_tiled, float* out_gscale, cudaStream_t st);
+
 // FP8 option of OutControl: both compact side operands ([rows, Kh] BF16, contiguous) snapped in place onto their per-tensor
 // power-of-two scaled E4M3 grids; cells2 = two workspace words.
 cudaError_t launch_fp8_snap_pair(uint16_t* a, int64_t rows_a, uint16_t* b, int64_t rows_b, int64_t Kh, uint32_t* cells2, cudaStream_t st);

@@ -247,26 +247,6 @@ __global__ void __launch_bounds__(256) amax_rows_rht_kernel(const uint16_t* __re
 // =========================================================================================================
 // Shared epilogue of one 16-element inner block: scale, round, pack.
 // =========================================================================================================
-template <bool SR>
-__device__ __forceinline__ uint2 quantize_block16(const float (&x)[16], float rcp, const PhiloxKeys& pk, uint32_t stream_id,
-                                                  uint64_t idx8) {
-  float y0[8], y1[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    y0[i] = __fmul_rn(x[i], rcp);
-    y1[i] = __fmul_rn(x[8 + i], rcp);
-  }
-  uint2 out;
-  if (SR) {
-    out.x = e2m1x8_sr(y0, sr_words(pk, stream_id, idx8));
-    out.y = e2m1x8_sr(y1, sr_words(pk, stream_id, idx8 + 1));
-  } else {
-    out.x = e2m1x8_rtn(y0);
-    out.y = e2m1x8_rtn(y1);
-  }
-  return out;
-}
-
 // =========================================================================================================
 // Row-axis quantize from BF16: one thread per inner block, eight neighbouring threads per 128-wide outer block.
 //   GS      scale mode. TENSOR reads the amax cell gs_cells[0]; ROW reads gs_cells[row]; BLOCK128 reduces the
