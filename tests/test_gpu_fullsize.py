@@ -179,3 +179,47 @@ def test_oscireset_and_calibration_at_model_size():
     assert np.all(np.abs(got - want_acc) <= 1e-5 * want_acc)
     outl, _, _ = b.nvfp4_outlier_select(acc, 20)
     assert outl.cpu().numpy().tolist() == sorted(ch.tolist())
+
+
+def test_variants_at_the_qkv_size():
+    """The options added around the hot path at the benchmark's QKV size (tokens 8192, 1024 -> 3072), in the launch
+    configuration bench.py times: rounded-up block scales in Q3 / Q5, FP8 outlier channels, 16x16 weight squares."""
+    from oracle import fp8_outliers as f8
+    from oracle import w16x16
+
+    b = B()
+    c = synth.CONFIGS[2]
+    T, D, C = c["tokens"], 1024, 3072
+    X, W, dY, ch = synth.layer_inputs(2, T, D, C, n_outlier=c["n_outlier"], factor=c["factor"], grad_scale=c["grad_scale"],
+                                      weight_id=10)
+    Xd, Wd, dYd = to_dev_bf16(X), to_dev_bf16(W), to_dev_bf16(dY)
+    rng = np.random.default_rng(1)
+    # rounded-up block scales, whole operands
+    q3 = orc.quantize(dY, orc.AXIS_ROW, orc.SR_SCALE_UP, orc.GS_TENSOR, 0, 3)
+    assert_operand_equal(b.nvfp4_quantize(dYd, b.AXIS_ROW, b.ROUND_SR_SCALE_UP, 0, 3, b.GS_TENSOR), q3, "Q3 scale-up full size")
+    q5 = orc.quantize(dY, orc.AXIS_COL, orc.SR_SCALE_UP, orc.GS_TENSOR, 0, 5)
+    assert_operand_equal(b.nvfp4_quantize(dYd, b.AXIS_COL, b.ROUND_SR_SCALE_UP, 0, 5, b.GS_TENSOR), q5, "Q5 scale-up full size")
+    # 16x16 weight squares: quantizer and transposition bit for bit, dX on sampled entries
+    qw = w16x16.quantize(W)
+    cfg = b.LayerConfig(gs_mode=b.GS_TENSOR, seed=0, w_block16=True, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32)
+    Y, saved = b.nvfp4_linear_fwd(Xd, Wd, cfg)
+    assert_operand_equal(saved.qw, qw, "Q2 16x16 full size")
+    assert_operand_equal(b.nvfp4_transpose_operand16(saved.qw), w16x16.transpose_operand(qw), "W-hat^T 16x16 full size")
+    dX, _ = b.nvfp4_linear_bwd(dYd, saved, cfg)
+    torch.cuda.synchronize()
+    q3p = orc.quantize(dY, orc.AXIS_ROW, orc.SR, orc.GS_TENSOR, 0, 3)
+    check_sampled(dX, orc.dequantize(q3p), orc.dequantize(w16x16.transpose_operand(qw)), rng, True, "dX 16x16")
+    # FP8 outlier channels (10 % of the channels, as bench.py --outliers 0.1 --outlier-fp8): side operands bit for bit
+    outl = synth.outlier_channels(D, 102, 77)
+    cfg8 = b.LayerConfig(gs_mode=b.GS_TENSOR, seed=0, outliers=outl, outlier_fp8=True, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16,
+                         dw_dtype=b.DT_F32)
+    Y8, saved8 = b.nvfp4_linear_fwd(Xd, Wd, cfg8)
+    torch.cuda.synchronize()
+    assert np.array_equal(saved8.X_out.float().cpu().numpy()[:, :102], f8.snap(X[:, outl])[0])
+    assert np.array_equal(saved8.W_out.float().cpu().numpy()[:, :102], f8.snap(W[:, outl])[0])
+    keep = np.setdiff1d(np.arange(D), outl)
+    q1 = orc.quantize(X[:, keep], orc.AXIS_ROW, orc.RTN, orc.GS_TENSOR, 0, 1)
+    q2 = orc.quantize(W[:, keep], orc.AXIS_ROW, orc.RTN, orc.GS_TENSOR, 0, 2)
+    A64 = np.concatenate([orc.dequantize(q1), f8.snap(X[:, outl])[0].astype(np.float64)], axis=1)
+    B64 = np.concatenate([orc.dequantize(q2), f8.snap(W[:, outl])[0].astype(np.float64)], axis=1)
+    check_sampled(Y8, A64, B64, rng, True, "Y with FP8 outlier channels")
