@@ -284,7 +284,14 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
 
 /* Both backward products of Sec. 2.3 in one call: exactly nvfp4_linear_bwd_dx followed by nvfp4_linear_bwd_dw (bit-identical
  * outputs), except that in the TENSOR scale mode without the Hadamard transformation the per-tensor amax of dY, which Q3
- * and Q5 share, is computed once. workspace: nvfp4_linear_workspace_bytes(NVFP4_OP_BWD, ...). */
+ * and Q5 share, is computed once. workspace: nvfp4_linear_workspace_bytes(NVFP4_OP_BWD, ...).
+ *
+ * Streams: the two products share nothing but their inputs, so the dX chain runs on a side stream that the library owns
+ * (one per host thread and device, created on the first call and kept), forked from `stream` by an event at entry and
+ * joined into it before the call returns: work queued on `stream` after the call sees all results, nothing else is
+ * observable. nvfp4_linear_fwd does the same for the weight quantizer. The fork / join pattern is legal under stream
+ * capture; make one call outside a capture first (stream creation is not capturable). The environment variable
+ * NVFP4_BWD_CONCURRENT=0 keeps everything on `stream`. */
 nvfp4_status nvfp4_linear_bwd(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
                               void* dX, int64_t lddx, void* dW, int64_t lddw, void* workspace, size_t ws_bytes,
                               void* stream);

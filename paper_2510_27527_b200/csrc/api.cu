@@ -119,7 +119,7 @@ static SideStream* side_stream_for_current_device() {
   }
   return &t;
 }
-// NVFP4_BWD_CONCURRENT=0 keeps both backward chains on the caller's stream.
+// NVFP4_BWD_CONCURRENT=0 keeps every chain of the layer calls on the caller's stream.
 static bool bwd_concurrency_enabled() {
   static const bool on = [] {
     const char* e = getenv("NVFP4_BWD_CONCURRENT");
