@@ -170,3 +170,46 @@ def test_fp8_outlier_snap_extremes():
         torch.cuda.synchronize()
         assert np.array_equal(saved.X_out.float().cpu().numpy()[:, :4], f8.snap(X[:, ch])[0]), scale
         assert np.array_equal(saved.W_out.float().cpu().numpy()[:, :4], f8.snap(W[:, ch])[0]), scale
+
+
+@pytest.mark.parametrize("outcontrol", [False, True])
+def test_graph_replay_and_second_stream_give_the_eager_bits(outcontrol):
+    """A captured step (fork / join of the library's side stream included) replays to the eager results bit for bit, and so
+    does a call issued on a user stream that is not the current one's default."""
+    b = B()
+    X, W, dY, ch = synth.layer_inputs(31, 256, 512, 384, n_outlier=4, factor=50.0, grad_scale=1e-3)
+    cfg = b.LayerConfig(gs_mode=0, seed=11, outliers=ch if outcontrol else None, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32)
+    Xd, Wd, dYd = to_dev_bf16(X), to_dev_bf16(W), to_dev_bf16(dY)
+    cfg.prepare(512)
+    saved = b.alloc_saved(Xd, Wd, cfg)
+    Y = torch.empty((256, 384), dtype=torch.bfloat16, device="cuda")
+    dX = torch.empty((256, 512), dtype=torch.bfloat16, device="cuda")
+    dW = torch.empty((384, 512), dtype=torch.float32, device="cuda")
+    ws_f = b.linear_workspace(b.OP_FWD, 256, 512, 384, cfg, Xd.device)
+    ws_b = b.linear_workspace(b.OP_BWD, 256, 512, 384, cfg, Xd.device)
+
+    def step():
+        b.nvfp4_linear_fwd(Xd, Wd, cfg, Y=Y, saved=saved, workspace=ws_f)
+        b.nvfp4_linear_bwd(dYd, saved, cfg, dX=dX, dW=dW, workspace=ws_b)
+
+    step()  # eager (also creates the side stream outside any capture)
+    torch.cuda.synchronize()
+    want = (Y.clone(), dX.clone(), dW.clone())
+    for t in (Y, dX, dW):
+        t.zero_()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    for t in (Y, dX, dW):
+        t.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, w) for a, w in zip((Y, dX, dW), want))
+    for t in (Y, dX, dW):
+        t.zero_()
+    s2 = torch.cuda.Stream()
+    s2.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s2):
+        step()
+    s2.synchronize()
+    assert all(torch.equal(a, w) for a, w in zip((Y, dX, dW), want))
