@@ -213,3 +213,38 @@ def test_graph_replay_and_second_stream_give_the_eager_bits(outcontrol):
         step()
     s2.synchronize()
     assert all(torch.equal(a, w) for a, w in zip((Y, dX, dW), want))
+
+
+def test_randomised_layer_configurations():
+    """Twenty random (shape, scale mode, OutControl, Hadamard, outlier format, rounding variant) layer configurations with a
+    fixed seed, forward / dX / dW against the oracle."""
+    b = B()
+    rng = np.random.default_rng(4242)
+    for case in range(20):
+        N_tok = int(rng.integers(1, 40)) * 8 + int(rng.integers(0, 8))
+        D = int(rng.integers(3, 60)) * 8
+        C = int(rng.integers(1, 40)) * 8
+        gs_mode = int(rng.integers(0, 3))
+        rht = bool(rng.integers(0, 2))
+        n_outl = int(rng.integers(0, 4)) * int(rng.integers(1, 6))
+        n_outl = min(n_outl, D - 16)
+        fp8 = bool(rng.integers(0, 2)) and n_outl > 0
+        scale_up = bool(rng.integers(0, 2))
+        w16 = gs_mode == 0 and n_outl == 0 and bool(rng.integers(0, 2))
+        X, W, dY, _ = synth.layer_inputs(100 + case, N_tok, D, C, n_outlier=min(3, D // 8), factor=30.0, grad_scale=1e-3)
+        outl = synth.outlier_channels(D, n_outl, 900 + case) if n_outl else None
+        sr = orc.SR_SCALE_UP if scale_up else orc.SR
+        rounding = (orc.RTN, orc.RTN, sr, sr, sr, sr)
+        ocfg = orc.LayerConfig(gs_mode=gs_mode, seed=case, outliers=outl, rht=rht, outlier_fp8=fp8, rounding=rounding, w_block16=w16)
+        Yo, so = orc.linear_fwd(X, W, ocfg)
+        dXo, dWo = orc.linear_bwd_dx(dY, so, ocfg), orc.linear_bwd_dw(dY, so, ocfg)
+        cfg = b.LayerConfig(gs_mode=gs_mode, seed=case, outliers=outl, rht=rht, outlier_fp8=fp8, rounding=rounding, w_block16=w16,
+                            y_dtype=b.DT_F32, dx_dtype=b.DT_F32, dw_dtype=b.DT_F32)
+        Xd, Wd, dYd = to_dev_bf16(X), to_dev_bf16(W), to_dev_bf16(dY)
+        Y, saved = b.nvfp4_linear_fwd(Xd, Wd, cfg)
+        dX, dW = b.nvfp4_linear_bwd(dYd, saved, cfg)
+        torch.cuda.synchronize()
+        tag = f"case {case}: {N_tok}x{D}->{C} gs{gs_mode} rht{rht} outl{n_outl} fp8{fp8} up{scale_up} w16{w16}"
+        assert rel_fro(Y.float().cpu().numpy(), Yo) <= 2e-5, tag
+        assert rel_fro(dX.float().cpu().numpy(), dXo) <= 2e-5, tag
+        assert rel_fro(dW.float().cpu().numpy(), dWo) <= 2e-5, tag
