@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(256) amax_tensor_pair_kernel(const uint16_t* _
 __global__ void __launch_bounds__(256) amax_tensor_masked_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols,
                                                                 int64_t ld, const int32_t* __restrict__ excluded, int64_t n_excl,
                                                                 uint32_t* amax_bits, uint16_t* __restrict__ out, int64_t ld_out,
-                                                                int64_t rows_per_cta) {
+                                                                int64_t rows_per_cta, uint64_t inv_o) {
   pdl_prologue();
   extern __shared__ __align__(16) uint16_t lane_mask[];  // [chunks * 8]
   const uint32_t chunks = (uint32_t)((cols + 7) >> 3);
@@ -106,34 +106,48 @@ __global__ void __launch_bounds__(256) amax_tensor_masked_kernel(const uint16_t*
   const bool row_tail = (cols & 7) != 0;  // the last chunk of a row is ragged: read element by element
   uint32_t m = 0;
   while (rr < n_rows) {
-    const uint16_t* p = src + (r0 + rr) * ld + ((int64_t)c << 3);
-    uint4 v;
-    if (!row_tail || c + 1 < chunks) {
-      v = *reinterpret_cast<const uint4*>(p);
-    } else {
-      uint32_t t[4] = {0, 0, 0, 0};
-      for (int q = 0; q < 8; ++q)
-        if (((int64_t)c << 3) + q < cols) t[q >> 1] |= (uint32_t)p[q] << (16 * (q & 1));
-      v = make_uint4(t[0], t[1], t[2], t[3]);
+    // four items per pass: positions first, then all loads, then the masks and maxima
+    uint4 v[4];
+    uint32_t cc[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      cc[u] = 0xFFFFFFFFu;
+      v[u] = make_uint4(0, 0, 0, 0);
+      if (rr < n_rows) {
+        cc[u] = c;
+        const uint16_t* p = src + (r0 + rr) * ld + ((int64_t)c << 3);
+        if (!row_tail || c + 1 < chunks) {
+          v[u] = *reinterpret_cast<const uint4*>(p);
+        } else {
+          uint32_t t[4] = {0, 0, 0, 0};
+          for (int q = 0; q < 8; ++q)
+            if (((int64_t)c << 3) + q < cols) t[q >> 1] |= (uint32_t)p[q] << (16 * (q & 1));
+          v[u] = make_uint4(t[0], t[1], t[2], t[3]);
+        }
+        c += step_c;
+        rr += step_r;
+        if (c >= chunks) {
+          c -= chunks;
+          rr += 1;
+        }
+      }
     }
-    const uint4 k = *reinterpret_cast<const uint4*>(lane_mask + (c << 3));
-    m = umax16x2(m, umax16x2(umax16x2(v.x & k.x, v.y & k.y), umax16x2(v.z & k.z, v.w & k.w)));
-    c += step_c;
-    rr += step_r;
-    if (c >= chunks) {
-      c -= chunks;
-      rr += 1;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (cc[u] != 0xFFFFFFFFu) {
+        const uint4 k = *reinterpret_cast<const uint4*>(lane_mask + (cc[u] << 3));
+        m = amax16x2(m, amax16x2(amax16x2(v[u].x & k.x, v[u].y & k.y), amax16x2(v[u].z & k.z, v[u].w & k.w)));  // (sign bits: see amax16x2)
+      }
     }
   }
   if (out && n_rows) {
-    const uint32_t ldo = (uint32_t)ld_out, n_out_items = n_rows * ldo;
-    const uint64_t inv_o = (1ull << 32) / ldo + 1ull;
+    const uint32_t ldo = (uint32_t)ld_out, n_out_items = n_rows * ldo;  // inv_o = 2^32 / ldo + 1, prepared by the launcher
     for (uint32_t e = threadIdx.x; e < n_out_items; e += 256) {
       const uint32_t ro = (uint32_t)(((uint64_t)e * inv_o) >> 32), j = e - ro * ldo;
       out[(r0 + ro) * ld_out + j] = j < n_excl ? src[(r0 + ro) * ld + excluded[j]] : (uint16_t)0;
     }
   }
-  uint32_t a = hmax_of_pair(m);
+  uint32_t a = hmax_of_pair(bf16x2_abs_bits(m));
 #pragma unroll
   for (int o = 16; o; o >>= 1) a = max(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
   __shared__ uint32_t warp_max[8];
@@ -160,11 +174,10 @@ __global__ void __launch_bounds__(256) amax_rows_bf16_kernel(const uint16_t* __r
     const int64_t nchunk = cols >> 3;
     for (int64_t c = threadIdx.x; c < nchunk; c += blockDim.x) {
       const uint4 v = *reinterpret_cast<const uint4*>(p + (c << 3));
-      m = umax16x2(m, umax16x2(umax16x2(bf16x2_abs_bits(v.x), bf16x2_abs_bits(v.y)),
-                               umax16x2(bf16x2_abs_bits(v.z), bf16x2_abs_bits(v.w))));
+      m = amax16x2(m, amax16x2(amax16x2(v.x, v.y), amax16x2(v.z, v.w)));
     }
-    for (int64_t j = (nchunk << 3) + threadIdx.x; j < cols; j += blockDim.x) m = umax16x2(m, (uint32_t)(p[j] & 0x7FFFu));
-    m = hmax_of_pair(m);
+    for (int64_t j = (nchunk << 3) + threadIdx.x; j < cols; j += blockDim.x) m = amax16x2(m, (uint32_t)p[j]);
+    m = hmax_of_pair(bf16x2_abs_bits(m));
   }
 #pragma unroll
   for (int o = 16; o; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
@@ -820,12 +833,13 @@ static cudaError_t launch_quantize_rows_impl(const QuantRowsArgs& a, cudaStream_
         const size_t smem = (size_t)((a.cols_src + 7) >> 3) * 16;  // one 16-byte mask per chunk (at most 40 KB)
         // a contiguous slab of rows per CTA. The side copy divides item numbers by the side operand's width through a
         // 32-bit reciprocal, exact while items * width < 2^32: slabs stay below 2^32 / d^2 rows (d also covers the chunk count)
-        int64_t rows_per_cta = (a.rows + 148 * 8 - 1) / (148 * 8);
+        int64_t rows_per_cta = (a.rows + 148 * 4 - 1) / (148 * 4);  // few, fat CTAs: the per-thread setup is paid once
         const int64_t dmax = std::max<int64_t>((a.cols_src + 7) >> 3, a.excl_out ? a.ld_excl_out : 1);
         rows_per_cta = std::max<int64_t>(1, std::min<int64_t>(rows_per_cta, (((int64_t)1 << 32) - 1) / (dmax * dmax)));
         const unsigned grid = (unsigned)((a.rows + rows_per_cta - 1) / rows_per_cta);
         launch_kernel(amax_tensor_masked_kernel, dim3(grid), dim3(256), smem, st, a.src, a.rows, a.cols_src, a.ld, a.excluded,
-                      a.cols_src - a.K, a.gs_cells, a.excl_out, a.ld_excl_out, rows_per_cta);
+                      a.cols_src - a.K, a.gs_cells, a.excl_out, a.ld_excl_out, rows_per_cta,
+                      (uint64_t)((1ull << 32) / (uint64_t)std::max<int64_t>(1, a.ld_excl_out) + 1ull));
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
         side_copy_done = a.excl_out != nullptr;
         return launch_rows_r<kGsTensor>(a, st);
