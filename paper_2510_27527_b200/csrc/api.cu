@@ -622,7 +622,7 @@ nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved
 
 static nvfp4_status bwd_dw_impl(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
                                 void* dW, int64_t lddw, void* workspace, size_t ws_bytes, void* stream, uint32_t* dy_amax,
-                                cudaEvent_t dy_amax_ready = nullptr) {
+                                cudaEvent_t dy_amax_ready = nullptr, HpDwArgs* deferred_hp = nullptr) {
   if (!dY || !saved || !dW) return NVFP4_ERR_NULL;
   const int64_t N_tok = saved->N_tok, D = saved->D, C = saved->C;
   if (N_tok <= 0 || D <= 0 || C <= 0) return NVFP4_ERR_SHAPE;
@@ -681,6 +681,10 @@ static nvfp4_status bwd_dw_impl(const void* dY, int64_t lddy, const nvfp4_saved*
   h.lddy = lddy; h.Kh = Kh; h.T = N_tok; h.C = C; h.n_out = n_out; h.outl = cfg->outlier_cols;
   h.dW = dW; h.dw_is_f32 = dw_f32; h.lddw = lddw; h.partial = hp_partial; h.dev_status = cfg->dev_status;
   h.compact = compact; h.ld_compact = ld_compact; h.D = D; h.keep = cfg->keep_cols; h.col_map = cfg->col_map;
+  if (deferred_hp) {  // the caller runs the side product on another stream and finishes dW after joining it
+    *deferred_hp = h;
+    return NVFP4_OK;
+  }
   return launch_hp_dw(h, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
@@ -743,10 +747,18 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, int64_t lddy, const nvfp4_saved* s
       amax_ready = side->amax;
     }
   }
-  const nvfp4_status s_dw = bwd_dw_impl(dY, lddy, saved, cfg, dW, lddw, base + need_dx, need_dw, stream, shared, amax_ready);
+  // With OutControl the BF16 side product dY^T X_out needs nothing of the FP4 chain: it runs at the end of the (shorter) dX
+  // chain on the side stream, and dW is assembled on the caller's stream after the join.
+  HpDwArgs hp{};
+  const bool defer_hp = side != nullptr && cfg->n_out > 0;
+  nvfp4_status s_dw = bwd_dw_impl(dY, lddy, saved, cfg, dW, lddw, base + need_dx, need_dw, stream, shared, amax_ready,
+                                  defer_hp ? &hp : nullptr);
   const nvfp4_status s_dx = bwd_dx_impl(dY, lddy, saved, cfg, dX, lddx, base, need_dx, st_dx, shared);
+  const bool hp_pending = defer_hp && s_dw == NVFP4_OK && hp.n_out > 0;
+  if (hp_pending && launch_hp_dw_product(hp, side->stream) != cudaSuccess) s_dw = NVFP4_ERR_CUDA;
   if (side && (cudaEventRecord(side->join, side->stream) != cudaSuccess || cudaStreamWaitEvent(st, side->join, 0) != cudaSuccess))
     return NVFP4_ERR_CUDA;
+  if (hp_pending && s_dw == NVFP4_OK && launch_hp_dw_finish(hp, st) != cudaSuccess) s_dw = NVFP4_ERR_CUDA;
   return s_dx != NVFP4_OK ? s_dx : s_dw;
 }
 

@@ -251,21 +251,34 @@ __global__ void __launch_bounds__(256) scatter_cols_kernel(const void* src, int6
 
 size_t hp_dw_partial_floats(int64_t T, int64_t C, int64_t Kh) { return (size_t)kHpDwSplit * (size_t)C * (size_t)Kh; }
 
-cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st) {
-  if (a.C == 0 || a.n_out == 0) return cudaSuccess;
-  // token splits: as many as fill the SMs once with (C / 128) x splits CTAs, at most kHpDwSplit (the workspace's size)
+// token splits of the side product: as many as fill the SMs once with (C / 128) x splits CTAs, at most kHpDwSplit (the
+// workspace's size)
+static void hp_dw_splits(const HpDwArgs& a, int64_t& t_per_split, int& n_split) {
   const int64_t want = std::max<int64_t>(1, std::min<int64_t>(kHpDwSplit, 148 / std::max<int64_t>(1, (a.C + 127) / 128)));
-  const int64_t t_per_split = ((a.T + want - 1) / want + 63) / 64 * 64;
-  const int n_split = (int)((a.T + t_per_split - 1) / t_per_split);
+  t_per_split = ((a.T + want - 1) / want + 63) / 64 * 64;
+  n_split = (int)((a.T + t_per_split - 1) / t_per_split);
+}
+
+// First half of dW under OutControl: the split partial sums of dY^T X_out (needs nothing of the FP4 product).
+cudaError_t launch_hp_dw_product(const HpDwArgs& a, cudaStream_t st) {
+  if (a.C == 0 || a.n_out == 0) return cudaSuccess;
+  int64_t t_per_split;
+  int n_split;
+  hp_dw_splits(a, t_per_split, n_split);
+  if (hp_dw_mma_supported(a.Kh) && (a.lddy & 7) == 0)  // tensor-core path (the CUDA-core kernel covers odd shapes)
+    return launch_hp_dw_mma(a.dY, a.lddy, a.X_out, a.Kh, a.T, a.C, a.partial, n_split, t_per_split, a.dev_status, st);
+  const dim3 grid((unsigned)((a.C + 63) / 64), (unsigned)n_split);
+  launch_kernel(hp_dw_partial_kernel, dim3(grid), dim3(256), 0, st, a, t_per_split);
+  return cudaGetLastError();
+}
+
+// Second half: dW from the compact FP4 product and the split partial sums.
+cudaError_t launch_hp_dw_finish(const HpDwArgs& a, cudaStream_t st) {
+  if (a.C == 0 || a.n_out == 0) return cudaSuccess;
+  int64_t t_per_split;
+  int n_split;
+  hp_dw_splits(a, t_per_split, n_split);
   cudaError_t e;
-  if (hp_dw_mma_supported(a.Kh) && (a.lddy & 7) == 0) {  // tensor-core path (the CUDA-core kernel covers odd shapes)
-    e = launch_hp_dw_mma(a.dY, a.lddy, a.X_out, a.Kh, a.T, a.C, a.partial, n_split, t_per_split, a.dev_status, st);
-  } else {
-    const dim3 grid((unsigned)((a.C + 63) / 64), (unsigned)n_split);
-    launch_kernel(hp_dw_partial_kernel, dim3(grid), dim3(256), 0, st, a, t_per_split);
-    e = cudaGetLastError();
-  }
-  if (e != cudaSuccess) return e;
   if (a.compact && a.col_map && a.D < ((int64_t)1 << 29) && (a.D + 4 + kAsmRows * a.n_out) * 4 <= 200 * 1024) {
     // kept and outlier channels written together, row by row
     const size_t smem = (size_t)(((a.D + 3) & ~(int64_t)3) + kAsmRows * a.n_out) * 4;
@@ -291,6 +304,11 @@ cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st) {
   const int64_t total = a.C * a.n_out;
   launch_kernel(hp_dw_reduce_kernel, dim3((unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8)), dim3(256), 0, st, a, n_split);
   return cudaGetLastError();
+}
+
+cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st) {
+  const cudaError_t e = launch_hp_dw_product(a, st);
+  return e != cudaSuccess ? e : launch_hp_dw_finish(a, st);
 }
 
 cudaError_t launch_gather_cols(const uint16_t* src, int64_t ld_src, int64_t rows, const int32_t* cols, int64_t n, uint16_t* dst,

@@ -169,7 +169,10 @@ size_t hp_dw_partial_floats(int64_t T, int64_t C, int64_t Kh);
 bool hp_dw_mma_supported(int64_t Kh);
 cudaError_t launch_hp_dw_mma(const uint16_t* dY, int64_t lddy, const uint16_t* X_out, int64_t Kh, int64_t T, int64_t C,
                              float* partial, int n_split, int64_t t_per_split, int32_t* dev_status, cudaStream_t st);
-cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st);
+cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st);  // product, then finish, on one stream
+// the two halves, for callers that overlap the side product (which needs only dY and X_out) with other work
+cudaError_t launch_hp_dw_product(const HpDwArgs& a, cudaStream_t st);
+cudaError_t launch_hp_dw_finish(const HpDwArgs& a, cudaStream_t st);
 
 // Scatter a compact [C, n_keep] matrix into columns keep[j] of dW [C, D].
 cudaError_t launch_scatter_cols(const void* src, int64_t ld_src, int src_is_f32, void* dst, int64_t ld_dst,
