@@ -194,6 +194,90 @@ __global__ void __launch_bounds__(256) amax_rows_bf16_kernel(const uint16_t* __r
   }
 }
 
+// amax of each source row, one warp per row (ROW scale mode of the row-axis quantizer without a column list): 16-byte
+// loads, four in flight per lane, packed maxima, one shuffle reduction; no shared memory, no barrier. cells[row] is
+// written, not accumulated. Needs ld % 8 == 0 and a 16-byte aligned base.
+__global__ void __launch_bounds__(256) amax_rows_warp_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t cols, int64_t ld,
+                                                            uint32_t* __restrict__ cells) {
+  pdl_prologue();
+  const int lane = threadIdx.x & 31;
+  const int64_t r = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (r >= rows) return;
+  const uint16_t* p = src + r * ld;
+  const int64_t nchunk = cols >> 3;
+  uint32_t m = 0;
+  int64_t c = lane;
+  for (; c + 96 < nchunk; c += 128) {
+    const uint4 v0 = *reinterpret_cast<const uint4*>(p + (c << 3)), v1 = *reinterpret_cast<const uint4*>(p + ((c + 32) << 3));
+    const uint4 v2 = *reinterpret_cast<const uint4*>(p + ((c + 64) << 3)), v3 = *reinterpret_cast<const uint4*>(p + ((c + 96) << 3));
+    const uint32_t a0 = amax16x2(amax16x2(v0.x, v0.y), amax16x2(v0.z, v0.w)), a1 = amax16x2(amax16x2(v1.x, v1.y), amax16x2(v1.z, v1.w));
+    const uint32_t a2 = amax16x2(amax16x2(v2.x, v2.y), amax16x2(v2.z, v2.w)), a3 = amax16x2(amax16x2(v3.x, v3.y), amax16x2(v3.z, v3.w));
+    m = amax16x2(m, amax16x2(amax16x2(a0, a1), amax16x2(a2, a3)));
+  }
+  for (; c < nchunk; c += 32) {
+    const uint4 v = *reinterpret_cast<const uint4*>(p + (c << 3));
+    m = amax16x2(m, amax16x2(amax16x2(v.x, v.y), amax16x2(v.z, v.w)));
+  }
+  for (int64_t j = (nchunk << 3) + lane; j < cols; j += 32) m = amax16x2(m, (uint32_t)p[j]);
+  uint32_t a = hmax_of_pair(bf16x2_abs_bits(m));
+#pragma unroll
+  for (int o = 16; o; o >>= 1) a = max(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
+  if (lane == 0) cells[r] = a << 16;
+}
+
+// amax of each COLUMN of a BF16 matrix [rowsK, D] (the per-row scales of the transposed operand in ROW mode). CTA = 32 lanes
+// x 8 row lanes over a strip of 256 columns and a slab of rows: a lane owns eight neighbouring columns (one 16-byte load
+// per row, a warp reads 512 contiguous bytes), keeps eight running maxima in four packed registers, the eight row lanes
+// are combined through shared memory and the slab's result is folded into cells[column] (zero before the launch) by one
+// atomic max per column. ld % 8 == 0, 16-byte aligned base.
+__global__ void __launch_bounds__(256) amax_cols_bf16_kernel(const uint16_t* __restrict__ src, int64_t rowsK, int64_t D, int64_t ld,
+                                                            int64_t rows_per_slab, uint32_t* cells) {
+  pdl_prologue();
+  const int lane = threadIdx.x & 31, ry = threadIdx.x >> 5;
+  const int64_t d0 = (int64_t)blockIdx.x * 256 + lane * 8;
+  const int64_t k0 = (int64_t)blockIdx.y * rows_per_slab, k1 = min(rowsK, k0 + rows_per_slab);
+  uint32_t m[4] = {0, 0, 0, 0};
+  if (d0 + 8 <= D) {
+    int64_t k = k0 + ry;
+    for (; k + 24 < k1; k += 32) {  // four rows in flight
+      const uint4 v0 = *reinterpret_cast<const uint4*>(src + k * ld + d0), v1 = *reinterpret_cast<const uint4*>(src + (k + 8) * ld + d0);
+      const uint4 v2 = *reinterpret_cast<const uint4*>(src + (k + 16) * ld + d0), v3 = *reinterpret_cast<const uint4*>(src + (k + 24) * ld + d0);
+      m[0] = amax16x2(amax16x2(m[0], v0.x), amax16x2(amax16x2(v1.x, v2.x), v3.x));
+      m[1] = amax16x2(amax16x2(m[1], v0.y), amax16x2(amax16x2(v1.y, v2.y), v3.y));
+      m[2] = amax16x2(amax16x2(m[2], v0.z), amax16x2(amax16x2(v1.z, v2.z), v3.z));
+      m[3] = amax16x2(amax16x2(m[3], v0.w), amax16x2(amax16x2(v1.w, v2.w), v3.w));
+    }
+    for (; k < k1; k += 8) {
+      const uint4 v = *reinterpret_cast<const uint4*>(src + k * ld + d0);
+      m[0] = amax16x2(m[0], v.x);
+      m[1] = amax16x2(m[1], v.y);
+      m[2] = amax16x2(m[2], v.z);
+      m[3] = amax16x2(m[3], v.w);
+    }
+  } else if (d0 < D) {  // ragged last chunk of the rows
+    for (int64_t k = k0 + ry; k < k1; k += 8)
+      for (int i = 0; d0 + i < D; ++i) m[i >> 1] = amax16x2(m[i >> 1], (uint32_t)src[k * ld + d0 + i] << (16 * (i & 1)));
+  }
+  __shared__ uint32_t red[8][4][32];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) red[ry][i][lane] = bf16x2_abs_bits(m[i]);
+  __syncthreads();
+  {
+    // thread t combines the eight row lanes of packed pair (t >> 5 & 3) of lane (t & 31); two threads share... keep it simple:
+    // 128 threads, one packed pair each
+    if (threadIdx.x < 128) {
+      const int i = threadIdx.x >> 5, ln = threadIdx.x & 31;
+      uint32_t a = red[0][i][ln];
+#pragma unroll
+      for (int y = 1; y < 8; ++y) a = umax16x2(a, red[y][i][ln]);
+      const int64_t d = (int64_t)blockIdx.x * 256 + ln * 8 + 2 * i;
+      const uint32_t lo = a & 0xFFFFu, hi = a >> 16;
+      if (d < D && lo) atomicMax(cells + d, lo << 16);
+      if (d + 1 < D && hi) atomicMax(cells + d + 1, hi << 16);
+    }
+  }
+}
+
 // amax of the transformed matrix (x S) H along the rows' K axis: per row (ROW mode) or folded into cells[0]. One thread
 // per 16-element block; atomic max on cells that are zero before the launch.
 __global__ void __launch_bounds__(256) amax_rows_rht_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, int64_t ld,
@@ -857,7 +941,10 @@ static cudaError_t launch_quantize_rows_impl(const QuantRowsArgs& a, cudaStream_
     return launch_rows_r<kGsTensor>(a, st);
   }
   if (a.gs_mode == kGsRow) {
-    launch_kernel(amax_rows_bf16_kernel, dim3((unsigned)a.rows), dim3(256), 0, st, a.src, a.rows, a.cols_src, a.ld, a.keep, a.K, a.gs_cells, 0);
+    if (!a.keep && (a.ld & 7) == 0 && (reinterpret_cast<uintptr_t>(a.src) & 15u) == 0)  // a warp per row
+      launch_kernel(amax_rows_warp_kernel, dim3((unsigned)((a.rows + 7) / 8)), dim3(256), 0, st, a.src, a.rows, a.cols_src, a.ld, a.gs_cells);
+    else
+      launch_kernel(amax_rows_bf16_kernel, dim3((unsigned)a.rows), dim3(256), 0, st, a.src, a.rows, a.cols_src, a.ld, a.keep, a.K, a.gs_cells, 0);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     return launch_rows_r<kGsRow>(a, st);
   }
@@ -947,7 +1034,18 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
   }
   if (a.gs_mode == kGsRow) {
     if (!a.cells_zeroed && (e = launch_zero_words(a.gs_cells, a.D, st)) != cudaSuccess) return e;
-    if ((e = launch_tr_amax_rht<SRC, kGsRow>(a.src, a.rowsK, a.D, a.seed, 0u, a.gs_cells, st)) != cudaSuccess) return e;
+    if (SRC == 0 && !a.src.out_rows && (a.src.ld & 7) == 0 && (reinterpret_cast<uintptr_t>(a.src.bf16) & 15u) == 0) {
+      // per-column maxima of the BF16 source by a streaming kernel (about 2 CTAs per SM worth of row slabs per column strip)
+      const int64_t strips = (a.D + 255) / 256;
+      int64_t slabs = std::max<int64_t>(1, (148 * 4 + strips - 1) / strips);
+      slabs = std::min<int64_t>(slabs, (a.rowsK + 63) / 64);
+      const int64_t rows_per_slab = ((a.rowsK + slabs - 1) / slabs + 7) / 8 * 8;
+      launch_kernel(amax_cols_bf16_kernel, dim3((unsigned)strips, (unsigned)((a.rowsK + rows_per_slab - 1) / rows_per_slab)), dim3(256), 0, st,
+                    a.src.bf16, a.rowsK, a.D, a.src.ld, rows_per_slab, a.gs_cells);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    } else if ((e = launch_tr_amax_rht<SRC, kGsRow>(a.src, a.rowsK, a.D, a.seed, 0u, a.gs_cells, st)) != cudaSuccess) {
+      return e;
+    }
     return launch_tr_r<SRC, kGsRow>(a, st);
   }
   return launch_tr_r<SRC, kGsBlock128>(a, st);
