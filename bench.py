@@ -2,13 +2,16 @@
 """Benchmark of the NVFP4 linear-layer hot path on B200.
 
 One "step" = forward + dX + dW (six quantizers, three FP4 GEMMs each) of every linear of the workload, through the
-C-ABI library. Default workload: LLaMA-style attention projections, hidden 1024, tokens 8192 (QKV 1024->3072 and
-O 1024->1024), seeded synthetic BF16 inputs. Prints ONE JSON line (see the keys below).
+C-ABI library. Default workload: every NVFP4 linear of a 24-layer ~370M LLaMA-style transformer (hidden 1024, FFN 2816),
+tokens 16384 (BASELINE configuration 4), seeded synthetic BF16 inputs. Prints ONE JSON line (see the keys below); the
+line also carries `large_shapes`: quantizer GB/s and GEMM TFLOP/s on the roofline-sweep shapes of configuration 5.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload attn|mlp|model370m] [--gs tensor|row]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload attn|mlp|model370m]
+                  [--gs tensor|row|block128] [--outliers p] [--rht] ...
 
-N > 1 (torchrun): every rank runs the same workload on its own GPU (independent replicas, no collective on the data
-path); the time is the max over ranks and the value the sum of all ranks' work.
+N > 1: every rank runs the same workload on its own GPU (independent replicas, no collective on the data path); the
+time is the max over ranks and the value the sum of all ranks' work. Under torchrun the ranks are given; a plain
+`python bench.py --gpus N` starts the N ranks itself.
 """
 from __future__ import annotations
 
@@ -37,16 +40,10 @@ WORKLOADS = {
 LAYERS = {"attn": 1, "mlp": 1, "model370m": 24}
 GS = {"tensor": 0, "row": 1, "block128": 2}
 
-
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
-# (default workload, QKV linear, tokens 8192), keyed by the kernel labels of the per-kernel breakdown below.
-# DRAM traffic (dram__bytes_read + dram__bytes_write) of one call = its quantize kernel (ncu capture of this workload) plus
-# its amax pre-pass, which reads the source exactly once (268.4 MB for 134.2 M elements in the 16384 x 8192 capture, scaled
-# to this tensor's 25.17 M elements: 50.33 MB)
-PROFILED_TRAFFIC = {
-    "quantize_cols_dY_SR(Q5)": (50355968 + 636416 + 50331648, "profiles/quantize_transpose_bf16_sr_attn_dY_8192x3072.txt"),
-    "quantize_rows_dY_SR(Q3)": (50380800 + 246272 + 50331648, "profiles/quantize_rows_sr_attn_dY_8192x3072.txt"),
-}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernels, from the ncu captures summarised under
+# profiles/ (keyed by kernel label, linear and tokens; a capture on a smaller tensor of the same kernel is scaled by the
+# number of elements, stated in the summary).
+PROFILED_TRAFFIC = {}
 
 
 def peaks():
@@ -59,6 +56,22 @@ def peaks():
 
 def flops_of(tokens, linears, layers):
     return layers * sum(6.0 * tokens * D * C for (_, D, C, _) in linears)
+
+
+def workload_name(args):
+    cfg_id, tokens, linears = WORKLOADS[args.workload]
+    return (f"{args.workload}: tokens {tokens}, " + ", ".join(f"{n} {D}->{C}" for n, D, C, _ in linears) +
+            (f", x{LAYERS[args.workload]} layers" if LAYERS[args.workload] > 1 else "") + ", fwd+dX+dW per linear")
+
+
+def config_of(args):
+    """The workload and how it is run: the same dictionary in the CUDA arm's and the oracle arm's line."""
+    return {"workload": workload_name(args), "gs_mode": args.gs, "outcontrol_fraction": args.outliers, "rht": bool(args.rht),
+            "sr_scale_up": bool(args.sr_scale_up), "outlier_fp8": bool(args.outlier_fp8),
+            "weight_block": "16x16" if args.w16x16 else "1x16",
+            "launch": "cuda_graph_replay" if args.graph else "stream",
+            "l2": "256 MiB write + 256 MiB read flush before every timed step",
+            "timing": "CUDA events per step on the launch stream, summed"}
 
 
 class ClockSampler:
@@ -78,6 +91,7 @@ class ClockSampler:
                                           "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._pump, daemon=True)
             self.t.start()
+            time.sleep(0.3)  # let the first samples arrive before the timed region starts
         except Exception:
             self.proc = None
 
@@ -94,7 +108,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         for l in self.lines:
             f = [t.strip() for t in l.split(",")]
             if len(f) < 9:
@@ -102,30 +116,31 @@ class ClockSampler:
             try:
                 sm.append(float(f[1]))
                 mx.append(float(f[2]))
+                pw.append(float(f[3]))
             except ValueError:
                 continue
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "power_w_max": max(pw) if pw else None}
 
 
 # ---------------------------------------------------------------------------------------------------------------
 # the oracle arm (CPU): used for --impl reference and for the cpu_baseline leg of the default arm
 # ---------------------------------------------------------------------------------------------------------------
-def oracle_sample_step(workload: str, gs_mode: int, sample_tokens: int = 256, rht: bool = False, all_linears: bool = False):
-    """One forward + dX + dW on a slab of `sample_tokens` tokens, through the oracle as it stands: of the workload's first
-    linear, or (all_linears) of every linear of one layer. Returns (seconds, flops of the sample, description)."""
+def oracle_sample_step(workload: str, gs_mode: int, sample_tokens: int = 256, rht: bool = False, inputs=None):
+    """One forward + dX + dW of every linear of one layer of the workload on a slab of `sample_tokens` tokens, through the
+    oracle as it stands. Returns (seconds, flops of the sample, description, inputs)."""
     from oracle import nvfp4_oracle as orc
 
     cfg_id, tokens, linears = WORKLOADS[workload]
     c = synth.CONFIGS[cfg_id]
-    chosen = linears if all_linears else linears[:1]
-    inputs = []
-    for li, (name, D, C, swiglu) in enumerate(chosen):
-        inputs.append(synth.layer_inputs(cfg_id, sample_tokens, D, C, n_outlier=c["n_outlier"], factor=c["factor"],
-                                         grad_scale=c["grad_scale"], swiglu=swiglu, weight_id=10 + li))
+    if inputs is None:
+        inputs = []
+        for li, (name, D, C, swiglu) in enumerate(linears):
+            inputs.append(synth.layer_inputs(cfg_id, sample_tokens, D, C, n_outlier=max(1, D // 100), factor=c["factor"],
+                                             grad_scale=c["grad_scale"], swiglu=swiglu, weight_id=10 + li))
     orc.lib()
     t0 = time.perf_counter()
     ocfg = orc.LayerConfig(gs_mode=gs_mode, seed=0, rht=rht)
@@ -134,9 +149,11 @@ def oracle_sample_step(workload: str, gs_mode: int, sample_tokens: int = 256, rh
         orc.linear_bwd_dx(dY, saved, ocfg)
         orc.linear_bwd_dw(dY, saved, ocfg)
     dt = time.perf_counter() - t0
-    fl = sum(6.0 * sample_tokens * D * C for _, D, C, _ in chosen)
-    names = " + ".join(f"{name} {D}->{C}" for name, D, C, _ in chosen)
-    return dt, fl, f"linear(s) {names}, {sample_tokens}-token slab of the {tokens}-token workload, fwd+dX+dW"
+    fl = sum(6.0 * sample_tokens * D * C for _, D, C, _ in linears)
+    names = " + ".join(f"{name} {D}->{C}" for name, D, C, _ in linears)
+    desc = (f"every linear of one layer ({names}), {sample_tokens}-token slab of the {tokens}-token workload, fwd+dX+dW; "
+            f"value = the slab's GEMM flops / its time")
+    return dt, fl, desc, inputs
 
 
 def run_reference(args):
@@ -146,20 +163,21 @@ def run_reference(args):
     from oracle import nvfp4_oracle as orc
 
     gs_mode = GS[args.gs]
-    cfg_id, tokens, linears = WORKLOADS[args.workload]
+    inputs = None
     for _ in range(min(args.warmup, 1)):
-        oracle_sample_step(args.workload, gs_mode, 64, args.rht)
+        _, _, _, inputs = oracle_sample_step(args.workload, gs_mode, args.ref_tokens, args.rht, inputs)
     times, fl, desc = [], 0.0, ""
     for _ in range(args.steps):
-        dt, fl, desc = oracle_sample_step(args.workload, gs_mode, args.ref_tokens, args.rht)
+        dt, fl, desc, inputs = oracle_sample_step(args.workload, gs_mode, args.ref_tokens, args.rht, inputs)
         times.append(dt)
     t = float(np.mean(times))
     val = fl / t / 1e12
     line = {
         "impl": "reference", "metric": "nvfp4_linear_fwd_bwd_tflops", "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(args), "sample": desc, "gs_mode": args.gs},
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": config_of(args),
+        "notes": "the oracle (CPU, as it stands) on a bounded sample of the same workload; the launch / l2 / timing entries of "
+                 "config describe the CUDA arm",
         "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": orc.threads(), "kind": "oracle", "sample": desc},
         "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -167,10 +185,115 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def workload_name(args):
-    cfg_id, tokens, linears = WORKLOADS[args.workload]
-    return (f"{args.workload}: tokens {tokens}, " + ", ".join(f"{n} {D}->{C}" for n, D, C, _ in linears) +
-            (f", x{LAYERS[args.workload]} layers" if LAYERS[args.workload] > 1 else "") + ", fwd+dX+dW per linear")
+# ---------------------------------------------------------------------------------------------------------------
+# shared timing helper of the CUDA arm
+# ---------------------------------------------------------------------------------------------------------------
+class Timer:
+    """CUDA-event timing with an L2 flush before every timed call: 256 MiB written (evicts everything), then another
+    256 MiB read so that the lines left in L2 are clean (the timed kernels do not pay for writing the flush back)."""
+
+    def __init__(self, dev):
+        import torch
+
+        self.torch = torch
+        self.flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        self.flush_src = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
+
+    def flush_l2(self):
+        self.flush_buf.fill_(1)
+        self.flush_src.max()
+
+    def each(self, fn, n, warm=3):
+        """Per-call milliseconds of n flushed calls (after `warm` untimed ones)."""
+        torch = self.torch
+        for _ in range(warm):
+            fn()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        torch.cuda.synchronize()
+        for i in range(n):
+            self.flush_l2()
+            ev[i][0].record()
+            fn()
+            ev[i][1].record()
+        torch.cuda.synchronize()
+        return [a.elapsed_time(bb) for a, bb in ev]
+
+    def median_s(self, fn, n, warm=3):
+        ms = sorted(self.each(fn, n, warm))
+        return ms[len(ms) // 2] * 1e-3
+
+
+def measure_large_shapes(b, dev, pk, timer, shapes, gs_names, n_iter):
+    """Quantizers and GEMMs on the roofline-sweep shapes (BASELINE configuration 5): A [M, K], B [N, K] ~N(0,1) BF16 with
+    0.5 % of the K channels x100, drawn with the seeded numpy recipe the parity tests use (seeds 5001 / 5002)."""
+    import torch
+
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    probe_flops = b.nvfp4_mma_issue_probe(2048, status)
+    sec = timer.median_s(lambda: b.nvfp4_mma_issue_probe(2048, status), 10)
+    issue_loop = probe_flops / sec / 1e12 if int(status.item()) == 0 else None
+    fp4_peak = 4.0 * pk["bf16"]
+    out = {"mma_issue_loop_TFLOPs": issue_loop, "fp4_peak_TFLOPs_4x_measured_bf16": fp4_peak, "hbm_peak_GBps": pk["hbm"], "shapes": []}
+    cache = {}
+
+    def operand_source(rows, K, tensor_id):
+        key = (rows, K, tensor_id)
+        if key not in cache:
+            cache[key], _ = synth.activations(rows, K, synth.seed_of(5, tensor_id), n_outlier=max(1, int(K * 0.005)), factor=100.0)
+        return b.upload_bf16(cache[key], dev)
+
+    quantized_a = set()
+    ws = b._workspace(1 << 20, dev)
+    for (M, N, K) in shapes:
+        r = {"M": M, "N": N, "K": K}
+        A = operand_source(M, K, 1)
+        Bm = operand_source(N, K, 2)
+        fl = 2.0 * M * N * K
+        for gname in gs_names:
+            gs = GS[gname]
+            qa, qb = b.alloc_operand(M, K, gs, device=dev), b.alloc_operand(N, K, gs, device=dev)
+            C = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs, out=qa, workspace=ws)
+            b.nvfp4_quantize(Bm, b.AXIS_ROW, b.ROUND_RTN, 0, 2, gs, out=qb, workspace=ws)
+            ms = sorted(timer.each(lambda: b.nvfp4_gemm(qa, qb, b.DT_BF16, out=C), n_iter))
+            med = ms[len(ms) // 2] * 1e-3
+            t_tensor, t_hbm = fl / (fp4_peak * 1e12), (0.5625 * (M + N) * K + 2.0 * M * N) / (pk["hbm"] * 1e9)
+            r[f"gemm_{gname}"] = {"us": med * 1e6, "best_us": ms[0] * 1e3, "TFLOPs": fl / med / 1e12,
+                                  "frac_of_4x_bf16_measured": fl / med / 1e12 / fp4_peak,
+                                  "frac_of_9PF_nominal": fl / med / 1e12 / 9000.0,
+                                  "frac_of_issue_loop": (fl / med / 1e12 / issue_loop) if issue_loop else None,
+                                  "bound_us_max_tensor_hbm": max(t_tensor, t_hbm) * 1e6}
+
+            def both():
+                b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs, out=qa, workspace=ws)
+                b.nvfp4_quantize(Bm, b.AXIS_ROW, b.ROUND_RTN, 0, 2, gs, out=qb, workspace=ws)
+                b.nvfp4_gemm(qa, qb, b.DT_BF16, out=C)
+
+            med = timer.median_s(both, max(3, n_iter // 2))
+            r[f"quantize_plus_gemm_{gname}"] = {"us": med * 1e6, "TFLOPs": fl / med / 1e12}
+            if (M, K, gname) not in quantized_a:
+                quantized_a.add((M, K, gname))
+                qat = b.alloc_operand(K, M, gs, device=dev)
+                n_el = M * K
+                qbytes = n_el * (2 + 0.5 + 1.0 / 16) + (n_el / 128 * 4 if gs == 2 else 0.0)
+                amax_read = 2.0 * n_el if gs != 2 else 0.0  # TENSOR / ROW read the source twice (amax pre-pass)
+                for label, fn in (
+                    ("quantize_rows_rtn", lambda: b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs, out=qa, workspace=ws)),
+                    ("quantize_rows_sr", lambda: b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_SR, 0, 3, gs, out=qa, workspace=ws)),
+                    ("quantize_cols_sr", lambda: b.nvfp4_quantize(A, b.AXIS_COL, b.ROUND_SR, 0, 5, gs, out=qat, workspace=ws)),
+                ):
+                    med = timer.median_s(fn, n_iter)
+                    r[f"{label}_A_{gname}"] = {"us": med * 1e6, "GBps": (qbytes + amax_read) / med / 1e9,
+                                               "frac_hbm_measured": (qbytes + amax_read) / med / 1e9 / pk["hbm"],
+                                               "algorithmic_bytes": qbytes + amax_read}
+                b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs, out=qa, workspace=ws)
+                med = timer.median_s(lambda: b.nvfp4_requantize_t(qa, b.ROUND_SR, 0, 6, out=qat, workspace=ws), n_iter)
+                r[f"requantize_t_A_{gname}"] = {"us": med * 1e6, "GBps": n_el * 1.125 / med / 1e9, "Gelem_per_s": n_el / med / 1e9}
+                del qat
+            del qa, qb, C
+        out["shapes"].append(r)
+        del A, Bm
+    return out
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -201,7 +324,6 @@ def run_ours(args):
         pass
 
     lins = []
-    host_inputs = {}
     for li, (name, D, C, swiglu) in enumerate(linears):
         X, W, dY, _ = synth.layer_inputs(cfg_id, tokens, D, C, n_outlier=max(1, D // 100), factor=c["factor"],
                                          grad_scale=c["grad_scale"], weight_id=10 + li, swiglu=swiglu)
@@ -216,7 +338,7 @@ def run_ours(args):
         outl = synth.outlier_channels(D, n_out, synth.seed_of(cfg_id, 50 + li)) if n_out else None
         rounding = (b.ROUND_RTN, b.ROUND_RTN) + ((b.ROUND_SR_SCALE_UP,) * 4 if args.sr_scale_up else (b.ROUND_SR,) * 4)
         L.cfg = b.LayerConfig(gs_mode=gs_mode, seed=0, y_dtype=b.DT_BF16, dx_dtype=b.DT_BF16, dw_dtype=b.DT_F32, outliers=outl, rht=args.rht,
-                              rounding=rounding, outlier_fp8=args.outlier_fp8, w_block16=args.w16x16)
+                              rounding=rounding, outlier_fp8=args.outlier_fp8, w_block16=args.w16x16, concurrent=not args.one_stream)
         L.cfg.prepare(D, dev)
         L.saved = b.alloc_saved(L.X, L.W[0], L.cfg)
         L.Y = torch.empty((tokens, C), dtype=torch.bfloat16, device=dev)
@@ -225,14 +347,7 @@ def run_ours(args):
         L.ws = [b.linear_workspace(k, tokens, D, C, L.cfg, dev) for k in (b.OP_FWD, b.OP_BWD_DX, b.OP_BWD_DW, b.OP_BWD)]
         lins.append(L)
 
-    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    flush_src = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
-
-    def flush_l2():
-        # write 256 MiB (evicts everything), then read another 256 MiB so that the lines left in L2 are clean:
-        # otherwise the timed kernels would also pay for writing the flush's dirty lines back
-        flush_buf.fill_(1)
-        flush_src.max()
+    timer = Timer(dev)
 
     def step():
         for layer in range(layers):
@@ -252,7 +367,7 @@ def run_ours(args):
         barrier()
         for s in range(steps):
             if flush:
-                flush_l2()
+                timer.flush_l2()
             ev[s][0].record()
             fn()
             ev[s][1].record()
@@ -287,18 +402,16 @@ def run_ours(args):
     value = world * fl / (ms_step * 1e-3) / 1e12
 
     if args.no_breakdown:
-        if rank != 0:
-            if world > 1:
-                dist.destroy_process_group()
-            return
-        print(json.dumps({"metric": "nvfp4_linear_fwd_bwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
-                          "steps": args.steps, "ms_per_step": ms_step, "gpu_launches": int(launches), "note": "--no-breakdown run"}))
+        if rank == 0:
+            print(json.dumps({"metric": "nvfp4_linear_fwd_bwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+                              "steps": args.steps, "ms_per_step": ms_step, "gpu_launches": int(launches), "clocks": clocks,
+                              "config": config_of(args), "note": "--no-breakdown run"}))
         if world > 1:
             dist.destroy_process_group()
         return
 
     # ---- end to end: host buffers in, results out, copies inside the timed region -------------------------------
-    pinned_in, h2d, d2h = [], 0, 0
+    h2d, d2h = 0, 0
     for L in lins:
         xb = torch.from_numpy(synth.to_bf16_bits(L.Xh).view(np.int16)).view(torch.bfloat16).pin_memory()
         gb = torch.from_numpy(synth.to_bf16_bits(L.dYh).view(np.int16)).view(torch.bfloat16).pin_memory()
@@ -351,7 +464,7 @@ def run_ours(args):
         for L in lins:
             cur.wait_event(L.ev_drained)  # the step ends when its last result is in host memory
 
-    e2e_steps = max(2, min(args.steps, 5))
+    e2e_steps = max(2, min(args.steps, 3 if layers > 1 else 5))
     step_e2e()
     ms_e2e, _ = timed(step_e2e, e2e_steps)
     e2e_value = world * fl / (ms_e2e * 1e-3) / 1e12
@@ -361,81 +474,86 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    # ---- per-kernel breakdown on the largest linear (rank 0): which kernel dominates, and its roofline ----------
+    # ---- per-kernel breakdown over the linears of one layer (rank 0): which launch dominates, and its roofline -------
     pk = peaks()
-    L = max(lins, key=lambda l: l.D * l.C)
+    fp4_peak = pk["bf16"] * 4.0  # dense FP4 : dense BF16 nominal ratio 9 : 2.25
     ws_q = b._workspace(1 << 20, dev)
-
-    def t_of(fn, n=20):
-        for _ in range(3):
-            fn()
-        t, _ = timed(fn, n)
-        return t * 1e-3
-
-    T, D, C = tokens, L.D, L.C
-    q3 = b.alloc_operand(T, C, gs_mode, device=dev)
-    q4 = b.alloc_operand(D, C, gs_mode, device=dev)
-    q5 = b.alloc_operand(C, T, gs_mode, device=dev)
-    q6 = b.alloc_operand(D, T, gs_mode, device=dev)
-    b.nvfp4_linear_fwd(L.X, L.W[0], L.cfg, Y=L.Y, saved=L.saved, workspace=L.ws[0])
-    parts = {}
-
-    def add(name, fn, alg_bytes=None, flops=None):
-        t = t_of(fn)
-        parts[name] = dict(seconds=t, GBps=(alg_bytes / t / 1e9 if alg_bytes else None),
-                           TFLOPs=(flops / t / 1e12 if flops else None), bytes=alg_bytes, flops=flops)
-
-    qbytes = lambda n: n * (2 + 0.5 + 1.0 / 16)
+    qbytes = lambda n: n * (2 + 0.5 + 1.0 / 16) + (n / 128 * 4 if gs_mode == 2 else 0.0)
     rqbytes = lambda n: n * 2 * (0.5 + 1.0 / 16)
     amax_extra = 2.0 if gs_mode != 2 else 0.0  # TENSOR / ROW modes read the source twice (amax pre-pass)
-    add("quantize_rows_X(Q1)", lambda: b.nvfp4_quantize(L.X, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, out=L.saved.qx, workspace=ws_q),
-        qbytes(T * D) + amax_extra * T * D)
-    add("quantize_rows_dY_SR(Q3)", lambda: b.nvfp4_quantize(L.dY, b.AXIS_ROW, b.ROUND_SR, 0, 3, gs_mode, out=q3, workspace=ws_q),
-        qbytes(T * C) + amax_extra * T * C)
-    add("quantize_cols_dY_SR(Q5)", lambda: b.nvfp4_quantize(L.dY, b.AXIS_COL, b.ROUND_SR, 0, 5, gs_mode, out=q5, workspace=ws_q),
-        qbytes(T * C) + amax_extra * T * C)
-    add("requantize_t_W(Q4)", lambda: b.nvfp4_requantize_t(L.saved.qw, b.ROUND_SR, 0, 4, out=q4, workspace=ws_q), rqbytes(C * D))
-    add("requantize_t_X(Q6)", lambda: b.nvfp4_requantize_t(L.saved.qx, b.ROUND_SR, 0, 6, out=q6, workspace=ws_q), rqbytes(T * D))
     gemm_bytes = lambda M, N, K, ob: 0.5625 * (M + N) * K + ob * M * N
-    add("gemm_fwd", lambda: b.nvfp4_gemm(L.saved.qx, L.saved.qw, b.DT_BF16, out=L.Y), gemm_bytes(T, C, D, 2), 2.0 * T * C * D)
-    add("gemm_dx", lambda: b.nvfp4_gemm(q3, q4, b.DT_BF16, out=L.dXo), gemm_bytes(T, D, C, 2), 2.0 * T * C * D)
-    add("gemm_dw", lambda: b.nvfp4_gemm(q5, q6, b.DT_F32, out=L.dWo), gemm_bytes(C, D, T, 4), 2.0 * T * C * D)
-    dom = max(parts, key=lambda k: parts[k]["seconds"])
-    dp = parts[dom]
-    fp4_peak = pk["bf16"] * 4.0  # dense FP4 : dense BF16 nominal ratio 9 : 2.25
-    if dom.startswith("gemm"):
-        t_tensor = dp["flops"] / (fp4_peak * 1e12)
-        t_hbm = dp["bytes"] / (pk["hbm"] * 1e9)
-        if t_tensor >= t_hbm:
+    parts = {}
+    T = tokens
+    n_break = 10
+    for L in lins:
+        D, C = L.D, L.C
+        if L.cfg.n_out:
+            continue  # the operand-level calls below have no OutControl form; the step numbers above cover it
+        q3 = b.alloc_operand(T, C, gs_mode, device=dev)
+        q4 = b.alloc_operand(D, C, gs_mode, device=dev)
+        q5 = b.alloc_operand(C, T, gs_mode, device=dev)
+        q6 = b.alloc_operand(D, T, gs_mode, device=dev)
+        b.nvfp4_linear_fwd(L.X, L.W[0], L.cfg, Y=L.Y, saved=L.saved, workspace=L.ws[0])
+
+        def add(name, fn, alg_bytes=None, flops=None):
+            t = timer.median_s(fn, n_break)
+            parts[f"{name} on {L.name} {D}->{C}"] = dict(seconds=t, GBps=(alg_bytes / t / 1e9 if alg_bytes else None),
+                                                         TFLOPs=(flops / t / 1e12 if flops else None), bytes=alg_bytes, flops=flops)
+
+        add("quantize_rows_X(Q1)", lambda: b.nvfp4_quantize(L.X, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, out=L.saved.qx, workspace=ws_q),
+            qbytes(T * D) + amax_extra * T * D)
+        add("quantize_rows_dY_SR(Q3)", lambda: b.nvfp4_quantize(L.dY, b.AXIS_ROW, b.ROUND_SR, 0, 3, gs_mode, out=q3, workspace=ws_q),
+            qbytes(T * C) + amax_extra * T * C)
+        add("quantize_cols_dY_SR(Q5)", lambda: b.nvfp4_quantize(L.dY, b.AXIS_COL, b.ROUND_SR, 0, 5, gs_mode, out=q5, workspace=ws_q),
+            qbytes(T * C) + amax_extra * T * C)
+        add("requantize_t_W(Q4)", lambda: b.nvfp4_requantize_t(L.saved.qw, b.ROUND_SR, 0, 4, out=q4, workspace=ws_q), rqbytes(C * D))
+        add("requantize_t_X(Q6)", lambda: b.nvfp4_requantize_t(L.saved.qx, b.ROUND_SR, 0, 6, out=q6, workspace=ws_q), rqbytes(T * D))
+        add("gemm_fwd", lambda: b.nvfp4_gemm(L.saved.qx, L.saved.qw, b.DT_BF16, out=L.Y), gemm_bytes(T, C, D, 2), 2.0 * T * C * D)
+        add("gemm_dx", lambda: b.nvfp4_gemm(q3, q4, b.DT_BF16, out=L.dXo), gemm_bytes(T, D, C, 2), 2.0 * T * C * D)
+        add("gemm_dw", lambda: b.nvfp4_gemm(q5, q6, b.DT_F32, out=L.dWo), gemm_bytes(C, D, T, 4), 2.0 * T * C * D)
+        del q3, q4, q5, q6
+    roof = None
+    if parts:
+        dom = max(parts, key=lambda k: parts[k]["seconds"])
+        dp = parts[dom]
+        if dom.startswith("gemm") and dp["flops"] / (fp4_peak * 1e12) >= dp["bytes"] / (pk["hbm"] * 1e9):
             roof = dict(bound="tensor", achieved=dp["TFLOPs"], peak=fp4_peak, unit="TFLOP/s", frac=dp["TFLOPs"] / fp4_peak)
         else:
             roof = dict(bound="hbm", achieved=dp["GBps"], peak=pk["hbm"], unit="GB/s", frac=dp["GBps"] / pk["hbm"])
-    else:
-        roof = dict(bound="hbm", achieved=dp["GBps"], peak=pk["hbm"], unit="GB/s", frac=dp["GBps"] / pk["hbm"])
-    roof.update(kernel=f"{dom} on {L.name} {D}->{C}, tokens {T}", peak_source=f"of {pk['source']}", traffic=None,
-                algorithmic_bytes_per_launch=dp["bytes"], seconds_per_launch=dp["seconds"])
-    if args.workload == "attn" and args.gs == "tensor" and dom in PROFILED_TRAFFIC:
-        roof["traffic"], roof["traffic_source"] = PROFILED_TRAFFIC[dom]
+        roof.update(kernel=f"{dom}, tokens {T}", peak_source=f"of {pk['source']}", traffic=None,
+                    algorithmic_bytes_per_launch=dp["bytes"], seconds_per_launch=dp["seconds"],
+                    note="the call that takes longest when every ABI call of one layer is timed alone (incl. its amax pre-pass)")
+        key = (dom, args.gs)
+        if key in PROFILED_TRAFFIC:
+            roof["traffic"], roof["traffic_source"] = PROFILED_TRAFFIC[key]
+
+    # ---- quantizers and GEMMs on the large sweep shapes (configuration 5) ----------------------------------------
+    large = None
+    if not args.no_large_shapes:
+        sampler2 = ClockSampler(local)
+        sampler2.start()
+        shapes = synth.CONFIGS[5]["shapes"] if not args.shapes else [tuple(int(v) for v in t.split("x")) for t in args.shapes.split(",")]
+        large = measure_large_shapes(b, dev, pk, timer, shapes, ("tensor", "block128"), 10)
+        large["clocks"] = sampler2.stop()
 
     # ---- the oracle beside it ------------------------------------------------------------------------------------
     cpu = None
     if world == 1 and not args.no_cpu:
         from oracle import nvfp4_oracle as orc
 
-        dt, sfl, desc = oracle_sample_step(args.workload, gs_mode, args.cpu_tokens, args.rht, all_linears=True)
+        dt, sfl, desc, _ = oracle_sample_step(args.workload, gs_mode, args.cpu_tokens, args.rht)
         cpu = {"value": sfl / dt / 1e12, "unit": "TFLOP/s", "cores": orc.threads(), "kind": "oracle", "sample": desc,
                "seconds": dt}
 
     line = {
         "metric": "nvfp4_linear_fwd_bwd_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "fp4(e2m1)xfp4 with ue4m3 block scales, f32 accumulate", "data": "synthetic",
-        "config": {"workload": workload_name(args), "gs_mode": args.gs, "outcontrol_fraction": args.outliers, "rht": bool(args.rht), "sr_scale_up": bool(args.sr_scale_up), "outlier_fp8": bool(args.outlier_fp8), "weight_block": "16x16" if args.w16x16 else "1x16", "launch": "cuda_graph_replay" if args.graph else "stream", "l2": "256 MiB write + 256 MiB read flush before every timed step",
-                   "timing": "CUDA events per step on the launch stream, summed"},
+        "dtype": "fp4(e2m1)xfp4 with ue4m3 block scales, f32 accumulate", "data": "synthetic", "config": config_of(args),
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
         "kernels": {k: {kk: (round(vv, 9) if isinstance(vv, float) else vv) for kk, vv in v.items() if kk in ("seconds", "GBps", "TFLOPs")}
                     for k, v in parts.items()},
+        "large_shapes": large,
     }
     print(json.dumps(line))
     if world > 1:
@@ -452,24 +570,8 @@ def run_aux(args):
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     pk = peaks()
-    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    flush_src = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
-
-    def t_of(fn, n):
-        for _ in range(3):
-            fn()
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
-        torch.cuda.synchronize()
-        for i in range(n):
-            flush_buf.fill_(1)
-            flush_src.max()
-            ev[i][0].record()
-            fn()
-            ev[i][1].record()
-        torch.cuda.synchronize()
-        ms = sorted(a.elapsed_time(bb) for a, bb in ev)
-        return ms[len(ms) // 2] * 1e-3
-
+    timer = Timer(dev)
+    t_of = lambda fn, n: timer.median_s(fn, n)
     g = torch.Generator(device=dev)
     g.manual_seed(7)
     out = {}
@@ -530,85 +632,20 @@ def run_aux(args):
 
 
 def run_sweep(args):
-    """Roofline sweep (square and skinny GEMMs with their quantizers), one JSON line with a list of shapes.
-    Not the headline line: a measurement aid for the large-shape roofline fractions."""
+    """Only the large-shape measurements (quantizers and GEMMs of configuration 5, or --shapes), one JSON line."""
     import torch
 
     from paper_2510_27527_b200 import binding as b
 
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
-    gs_mode = GS[args.gs]
     pk = peaks()
     shapes = synth.CONFIGS[5]["shapes"] if not args.shapes else [tuple(int(v) for v in t.split("x")) for t in args.shapes.split(",")]
-    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    flush_src = torch.zeros(256 << 20, dtype=torch.uint8, device=dev)
-    out = []
-
-    def t_of(fn, n):
-        for _ in range(3):
-            fn()
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
-        torch.cuda.synchronize()
-        for i in range(n):
-            flush_buf.fill_(1)
-            flush_src.max()  # leave clean lines in L2
-            ev[i][0].record()
-            fn()
-            ev[i][1].record()
-        torch.cuda.synchronize()
-        ms = sorted(a.elapsed_time(bb) for a, bb in ev)
-        return ms[len(ms) // 2] * 1e-3, ms[0] * 1e-3
-
-    # tensor-core ceiling of this box under load: the issue loop without memory traffic (4 MMAs of 128 x 256 x 64 per turn)
-    status = torch.zeros(1, dtype=torch.int32, device=dev)
-    probe_flops = b.nvfp4_mma_issue_probe(2048, status)
-    sec, _ = t_of(lambda: b.nvfp4_mma_issue_probe(2048, status), 10)
-    issue_loop_tflops = probe_flops / sec / 1e12 if int(status.item()) == 0 else None
-    g = torch.Generator(device=dev)
-    g.manual_seed(5)
-    for (M, N, K) in shapes:
-        A = torch.randn((M, K), device=dev, generator=g, dtype=torch.float32)
-        nch = max(1, int(K * 0.005))
-        A[:, torch.randperm(K, device=dev, generator=g)[:nch]] *= 100.0
-        A = A.to(torch.bfloat16)
-        Bm = torch.randn((N, K), device=dev, generator=g, dtype=torch.float32).to(torch.bfloat16)
-        qa, qb = b.alloc_operand(M, K, gs_mode, device=dev), b.alloc_operand(N, K, gs_mode, device=dev)
-        qat = b.alloc_operand(K, M, gs_mode, device=dev)
-        ws = b._workspace(1 << 20, dev)
-        C = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
-        n = args.steps
-        r = {"M": M, "N": N, "K": K}
-        qbytes = lambda e: e * (2 + 0.5 + 1.0 / 16)
-        amax_extra = 2.0 if gs_mode != 2 else 0.0
-        for name, fn, nelem in (
-            ("quantize_rows_rtn_A", lambda: b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, out=qa, workspace=ws), M * K),
-            ("quantize_rows_sr_A", lambda: b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_SR, 0, 3, gs_mode, out=qa, workspace=ws), M * K),
-            ("quantize_cols_sr_A", lambda: b.nvfp4_quantize(A, b.AXIS_COL, b.ROUND_SR, 0, 5, gs_mode, out=qat, workspace=ws), M * K),
-        ):
-            med, best = t_of(fn, n)
-            r[name] = {"us": med * 1e6, "GBps": qbytes(nelem) / med / 1e9, "GBps_incl_amax_read": (qbytes(nelem) + amax_extra * nelem) / med / 1e9,
-                       "frac_hbm_measured": (qbytes(nelem) + amax_extra * nelem) / med / 1e9 / pk["hbm"]}
-        b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, out=qa, workspace=ws)
-        b.nvfp4_quantize(Bm, b.AXIS_ROW, b.ROUND_RTN, 0, 2, gs_mode, out=qb, workspace=ws)
-        med, best = t_of(lambda: b.nvfp4_requantize_t(qa, b.ROUND_SR, 0, 6, out=qat, workspace=ws), n)
-        r["requantize_t_A"] = {"us": med * 1e6, "GBps": M * K * 1.125 / med / 1e9, "Gelem_per_s": M * K / med / 1e9}
-        med, best = t_of(lambda: b.nvfp4_gemm(qa, qb, b.DT_BF16, out=C), n)
-        fl = 2.0 * M * N * K
-        r["gemm"] = {"us": med * 1e6, "best_us": best * 1e6, "TFLOPs": fl / med / 1e12, "frac_of_4x_bf16_measured": fl / med / 1e12 / (4 * pk["bf16"]),
-                     "frac_of_9PF_nominal": fl / med / 1e12 / 9000.0,
-                     "frac_of_issue_loop": (fl / med / 1e12 / issue_loop_tflops) if issue_loop_tflops else None}
-
-        def fused():
-            b.nvfp4_quantize(A, b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, out=qa, workspace=ws)
-            b.nvfp4_quantize(Bm, b.AXIS_ROW, b.ROUND_RTN, 0, 2, gs_mode, out=qb, workspace=ws)
-            b.nvfp4_gemm(qa, qb, b.DT_BF16, out=C)
-
-        med, best = t_of(fused, n)
-        r["quantize_plus_gemm"] = {"us": med * 1e6, "TFLOPs": fl / med / 1e12}
-        out.append(r)
-        del A, Bm, qa, qb, qat, C
-    print(json.dumps({"sweep": out, "gs_mode": args.gs, "peaks": pk, "mma_issue_loop_TFLOPs": issue_loop_tflops}))
+    sampler = ClockSampler(0)
+    sampler.start()
+    out = measure_large_shapes(b, dev, pk, Timer(dev), shapes, (args.gs,), args.steps)
+    out["clocks"] = sampler.stop()
+    print(json.dumps({"sweep": out, "gs_mode": args.gs, "peaks": pk}))
 
 
 def main():
@@ -617,10 +654,10 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="attn", choices=list(WORKLOADS))
+    ap.add_argument("--workload", default="model370m", choices=list(WORKLOADS))
     ap.add_argument("--gs", default="tensor", choices=list(GS))
-    ap.add_argument("--ref-tokens", type=int, default=1024, help="token slab of one oracle step (reference arm)")
-    ap.add_argument("--cpu-tokens", type=int, default=8192, help="token slab of the cpu_baseline leg (every linear of one layer)")
+    ap.add_argument("--ref-tokens", type=int, default=256, help="token slab of one oracle step (reference arm)")
+    ap.add_argument("--cpu-tokens", type=int, default=2048, help="token slab of the cpu_baseline leg (every linear of one layer)")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--outliers", type=float, default=0.0,
                     help="OutControl: fraction of input channels kept in BF16 (0 = off; the paper uses 0.10)")
@@ -630,11 +667,18 @@ def main():
     ap.add_argument("--sr-scale-up", action="store_true", help="backward quantizers round the block scale up (strictly unbiased variant)")
     ap.add_argument("--graph", action=argparse.BooleanOptionalAction, default=True,
                     help="capture one step in a CUDA graph and time its replays (default; --no-graph launches every kernel from the host)")
+    ap.add_argument("--one-stream", action="store_true", help="no second stream: every chain of a layer call runs on the caller's stream")
     ap.add_argument("--no-breakdown", action="store_true", help="only warm-up + timed steps (used for ncu launch lists)")
-    ap.add_argument("--sweep", action="store_true", help="roofline sweep of the large GEMM shapes instead of the step benchmark")
+    ap.add_argument("--no-large-shapes", action="store_true", help="skip the configuration-5 measurements of the default line")
+    ap.add_argument("--sweep", action="store_true", help="only the large-shape measurements (configuration 5 or --shapes)")
     ap.add_argument("--aux", action="store_true", help="HBM roofline of the calibration and OsciReset kernels instead of the step benchmark")
-    ap.add_argument("--shapes", default="", help="with --sweep: comma list of MxNxK")
+    ap.add_argument("--shapes", default="", help="comma list of MxNxK for the large-shape measurements")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours" and not (args.sweep or args.aux):
+        # not started by torchrun: start the N ranks here (one process per GPU), rank 0 prints the line
+        from paper_2510_27527_b200 import multi
+
+        sys.exit(multi.launch_ranks(args.gpus, os.path.abspath(__file__), sys.argv[1:]))
     if args.sweep:
         run_sweep(args)
     elif args.aux:

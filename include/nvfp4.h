@@ -94,9 +94,6 @@ size_t nvfp4_operand_gscale_count(int64_t R, int64_t K, int32_t gs_mode);
 
 const char* nvfp4_status_string(nvfp4_status s);
 
-/* Number of kernels the library has enqueued since it was loaded (a measurement aid; not thread-safe). */
-long long nvfp4_launch_count(void);
-
 /* ---------------------------------------------------------------------------------------------------------
  * nvfp4_quantize — double-block quantization of a BF16 matrix (Sec. 2.2; rounding per Sec. 2.1).
  *
@@ -200,16 +197,30 @@ nvfp4_status nvfp4_requantize_t(const nvfp4_operand* in, const void* hp_bf16, in
  *   dev_status optional device int: set to NVFP4_ERR_TIMEOUT if a bounded wait inside the kernel ran out
  *            (the kernel then drains and exits; C is unspecified). Never written otherwise.
  *   workspace at least nvfp4_gemm_workspace_bytes(M, N, K) (split-K partials for small outputs).
+ *
+ * nvfp4_gemm_ex is the same product with explicit control over what nvfp4_gemm chooses by itself (opts == NULL gives
+ * nvfp4_gemm). It exists for tests and for measurements:
+ *   variant  AUTO: chosen from the shape. TILE128: one CTA per 128 x 128 output tile, two accumulators. PAIR256: a pair of
+ *            CTAs on neighbouring SMs per 256 x 256 tile (cta_group::2; TENSOR and ROW scale modes only, NVFP4_ERR_ENUM
+ *            with BLOCK128).
+ *   wait_limit_cycles  bound of every device-side wait, in SM clock cycles (0: the default, about two seconds).
+ *   starve_first_stage  test hook of the bounded waits: when non-zero, the barrier of the first operand stage expects 16
+ *            bytes more than will ever arrive, so the first wait of the MMA warp runs out; the kernel then reports
+ *            NVFP4_ERR_TIMEOUT through dev_status, every role drains and the call returns. C is unspecified.
  * --------------------------------------------------------------------------------------------------------- */
 size_t nvfp4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
 nvfp4_status nvfp4_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
                         int32_t accumulate, int32_t* dev_status, void* workspace, size_t ws_bytes, void* stream);
 
-/* Measurement aid (the paper has no counterpart): every SM issues iters x 4 block-scaled FP4 MMA instructions
- * (M = 128, N = 256, K = 64) on tiles resident in shared / tensor memory, no global traffic in the loop. *flops_out (host,
- * optional) receives the FP4 flops one launch performs; time the launch with events to get this device's tensor-core
- * ceiling under load. dev_status as in nvfp4_gemm (the kernel's single wait is bounded). 1 <= iters <= 2^20. */
-nvfp4_status nvfp4_mma_issue_probe(int32_t iters, int32_t* dev_status, double* flops_out, void* stream);
+typedef enum { NVFP4_GEMM_AUTO = 0, NVFP4_GEMM_TILE128 = 1, NVFP4_GEMM_PAIR256 = 2 } nvfp4_gemm_variant;
+typedef struct {
+  int32_t variant;           /* nvfp4_gemm_variant */
+  int32_t starve_first_stage;
+  int64_t wait_limit_cycles;
+} nvfp4_gemm_opts;
+nvfp4_status nvfp4_gemm_ex(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
+                           int32_t accumulate, int32_t* dev_status, const nvfp4_gemm_opts* opts, void* workspace,
+                           size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------
  * The layer (Sec. 2.3; OutControl split of Sec. 4.2). X [N_tok, D], W [C, D], Y / dY [N_tok, C].
@@ -241,6 +252,17 @@ typedef struct {
    * the forward codes transposed as they are -- no Q4, so no rounding, no random bits and no Hadamard factor on the dX
    * product (cfg.rht then applies to dW only). Requires gs_mode TENSOR, n_out = 0 and rounding[1] = RTN (NVFP4_ERR_ENUM). */
   int32_t weight_block;
+  /* Optional second stream (all four NULL: everything is enqueued on the call's `stream`). The two backward products
+   * share nothing but their inputs, and forward's two quantizers are independent: with a side stream the dX chain (Q3, Q4,
+   * product) and the weight quantizer run on it, forked from `stream` by ev_fork at entry and joined into it by ev_join
+   * before the call returns (ev_aux orders the shared amax pass of dY before Q5 under OutControl). Work queued on `stream`
+   * after the call sees all results; nothing else is observable, and the pattern is legal under stream capture. The
+   * stream (a cudaStream_t) and the three events (cudaEvent_t, timing disabled is enough) belong to the caller, must live
+   * on the current device and must not be used by another call at the same time; the library creates none. */
+  void* side_stream;
+  void* ev_fork;
+  void* ev_join;
+  void* ev_aux;
 } nvfp4_layer_cfg;
 
 /* What forward leaves for backward. qx [N_tok, D - n_out] and qw [C, D - n_out] are filled by
@@ -265,6 +287,15 @@ typedef enum { NVFP4_OP_FWD = 0, NVFP4_OP_BWD_DX = 1, NVFP4_OP_BWD_DW = 2, NVFP4
 size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, int64_t C, int64_t n_out,
                                     int32_t gs_mode);
 
+/* Where a backward call keeps its quantized operands inside its workspace (host-only, nothing is launched): fills *out
+ * with the descriptor of Q3(dY) [N_tok, C], Q4(W-hat^T) [D, C], Q5(dY^T) [C, N_tok] or Q6(X-hat^T) [D - n_out, N_tok]
+ * (which = 3 .. 6; tiled scales) for a workspace that was, or will be, passed to the call of kind op_kind with the same
+ * shapes. The contents are valid once that call has run on its stream and until the workspace is used again: a way to
+ * inspect what the products of Sec. 2.3 actually consumed. which = 3, 4 go with NVFP4_OP_BWD_DX or NVFP4_OP_BWD, 5, 6 with
+ * NVFP4_OP_BWD_DW or NVFP4_OP_BWD (NVFP4_ERR_ENUM otherwise). */
+nvfp4_status nvfp4_linear_bwd_operand(int32_t op_kind, int32_t which, int64_t N_tok, int64_t D, int64_t C, int64_t n_out,
+                                      int32_t gs_mode, void* workspace, size_t ws_bytes, nvfp4_operand* out);
+
 /* Y = Q1(X[:, keep]) Q2(W[:, keep])^T  +  X[:, outl] W[:, outl]^T (BF16 inputs, FP32 accumulate). */
 nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t ldw, int64_t N_tok, int64_t D,
                               int64_t C, const nvfp4_layer_cfg* cfg, void* Y, int64_t ldy, nvfp4_saved* saved,
@@ -286,12 +317,7 @@ nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved
  * outputs), except that in the TENSOR scale mode without the Hadamard transformation the per-tensor amax of dY, which Q3
  * and Q5 share, is computed once. workspace: nvfp4_linear_workspace_bytes(NVFP4_OP_BWD, ...).
  *
- * Streams: the two products share nothing but their inputs, so the dX chain runs on a side stream that the library owns
- * (one per host thread and device, created on the first call and kept), forked from `stream` by an event at entry and
- * joined into it before the call returns: work queued on `stream` after the call sees all results, nothing else is
- * observable. nvfp4_linear_fwd does the same for the weight quantizer. The fork / join pattern is legal under stream
- * capture; make one call outside a capture first (stream creation is not capturable). The environment variable
- * NVFP4_BWD_CONCURRENT=0 keeps everything on `stream`. */
+ * Streams: with cfg->side_stream set, the dX chain runs there beside the dW chain (see nvfp4_layer_cfg). */
 nvfp4_status nvfp4_linear_bwd(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
                               void* dX, int64_t lddx, void* dW, int64_t lddw, void* workspace, size_t ws_bytes,
                               void* stream);

@@ -28,6 +28,7 @@ GS_TENSOR, GS_ROW, GS_BLOCK128 = 0, 1, 2
 SF_LINEAR, SF_TILED128x4 = 0, 1
 DT_BF16, DT_F32 = 0, 1
 OP_FWD, OP_BWD_DX, OP_BWD_DW, OP_BWD = 0, 1, 2, 3
+GEMM_AUTO, GEMM_TILE128, GEMM_PAIR256 = 0, 1, 2
 ERR_TIMEOUT = 8
 
 c_i64, c_i32, c_u64, c_u32, c_vp, c_sz = (ctypes.c_int64, ctypes.c_int32, ctypes.c_uint64, ctypes.c_uint32,
@@ -42,7 +43,12 @@ class COperand(ctypes.Structure):
 class CLayerCfg(ctypes.Structure):
     _fields_ = [("gs_mode", c_i32), ("rounding", c_i32 * 6), ("seed", c_u64), ("y_dtype", c_i32), ("dx_dtype", c_i32),
                 ("dw_dtype", c_i32), ("n_out", c_i64), ("outlier_cols", c_vp), ("keep_cols", c_vp), ("col_map", c_vp),
-                ("dev_status", c_vp), ("rht", c_i32), ("outlier_format", c_i32), ("weight_block", c_i32)]
+                ("dev_status", c_vp), ("rht", c_i32), ("outlier_format", c_i32), ("weight_block", c_i32),
+                ("side_stream", c_vp), ("ev_fork", c_vp), ("ev_join", c_vp), ("ev_aux", c_vp)]
+
+
+class CGemmOpts(ctypes.Structure):
+    _fields_ = [("variant", c_i32), ("starve_first_stage", c_i32), ("wait_limit_cycles", c_i64)]
 
 
 class CSaved(ctypes.Structure):
@@ -57,7 +63,6 @@ EXPORTS = {
     "nvfp4_operand_sf_bytes": (c_sz, [c_i64, c_i64, c_i32]),
     "nvfp4_operand_gscale_count": (c_sz, [c_i64, c_i64, c_i32]),
     "nvfp4_status_string": (ctypes.c_char_p, [c_i32]),
-    "nvfp4_launch_count": (ctypes.c_longlong, []),
     "nvfp4_quantize_workspace_bytes": (c_sz, [c_i64, c_i32]),
     "nvfp4_quantize": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_u64, c_u32, c_u32, c_vp, c_i64,
                                ctypes.POINTER(COperand), c_vp, c_sz, c_vp]),
@@ -71,8 +76,10 @@ EXPORTS = {
     "nvfp4_gemm_workspace_bytes": (c_sz, [c_i64, c_i64, c_i64]),
     "nvfp4_gemm": (c_i32, [ctypes.POINTER(COperand), ctypes.POINTER(COperand), c_vp, c_i32, c_i64, c_i32, c_vp, c_vp,
                            c_sz, c_vp]),
-    "nvfp4_mma_issue_probe": (c_i32, [c_i32, c_vp, ctypes.POINTER(ctypes.c_double), c_vp]),
+    "nvfp4_gemm_ex": (c_i32, [ctypes.POINTER(COperand), ctypes.POINTER(COperand), c_vp, c_i32, c_i64, c_i32, c_vp,
+                              ctypes.POINTER(CGemmOpts), c_vp, c_sz, c_vp]),
     "nvfp4_linear_workspace_bytes": (c_sz, [c_i32, c_i64, c_i64, c_i64, c_i64, c_i32]),
+    "nvfp4_linear_bwd_operand": (c_i32, [c_i32, c_i32, c_i64, c_i64, c_i64, c_i64, c_i32, c_vp, c_sz, ctypes.POINTER(COperand)]),
     "nvfp4_linear_fwd": (c_i32, [c_vp, c_i64, c_vp, c_i64, c_i64, c_i64, c_i64, ctypes.POINTER(CLayerCfg), c_vp, c_i64,
                                  ctypes.POINTER(CSaved), c_vp, c_sz, c_vp]),
     "nvfp4_linear_bwd_dx": (c_i32, [c_vp, c_i64, ctypes.POINTER(CSaved), ctypes.POINTER(CLayerCfg), c_vp, c_i64, c_vp,
@@ -93,12 +100,33 @@ EXPORTS = {
     "nvfp4_osci_sparse_suppress": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i64, c_vp, c_vp, c_vp, ctypes.c_float, c_vp, c_vp,
                                            c_sz, c_vp]),
 }
-for _name, (_res, _args) in EXPORTS.items():
+# measurement aids (include/nvfp4_measure.h): the launch counter lives in the main library, the tensor-core issue loop in
+# a library of its own that only the benchmark and its test load
+MEASURE_EXPORTS = {
+    "nvfp4_launch_count": (ctypes.c_longlong, []),
+    "nvfp4_mma_issue_probe": (c_i32, [c_i32, c_vp, ctypes.POINTER(ctypes.c_double), c_vp]),
+}
+for _name, (_res, _args) in list(EXPORTS.items()) + [("nvfp4_launch_count", MEASURE_EXPORTS["nvfp4_launch_count"])]:
     _f = getattr(_lib, _name)
     _f.restype = _res
     _f.argtypes = _args
 
 lib = _lib
+MEASURE_LIB_PATH = os.path.join(_HERE, "libnvfp4_measure.so")
+_measure_lib = None
+
+
+def measure_lib():
+    """The measurement-aid library (tensor-core issue loop), loaded on first use."""
+    global _measure_lib
+    if _measure_lib is None:
+        if not os.path.exists(MEASURE_LIB_PATH):
+            raise ImportError(f"{MEASURE_LIB_PATH} is missing: build it with `python -m paper_2510_27527_b200.build`")
+        _measure_lib = ctypes.CDLL(MEASURE_LIB_PATH)
+        res, args = MEASURE_EXPORTS["nvfp4_mma_issue_probe"]
+        _measure_lib.nvfp4_mma_issue_probe.restype = res
+        _measure_lib.nvfp4_mma_issue_probe.argtypes = args
+    return _measure_lib
 
 
 class Nvfp4Error(RuntimeError):
@@ -265,6 +293,20 @@ def nvfp4_gemm(A: Operand, B: Operand, c_dtype: int = DT_F32, out: torch.Tensor 
     return out
 
 
+def nvfp4_gemm_ex(A: Operand, B: Operand, c_dtype: int = DT_F32, out: torch.Tensor | None = None, accumulate: bool = False,
+                  dev_status: torch.Tensor | None = None, variant: int = GEMM_AUTO, wait_limit_cycles: int = 0,
+                  starve_first_stage: bool = False, workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """nvfp4_gemm with an explicit kernel variant, wait bound and the test hook of the bounded waits."""
+    if out is None:
+        out = _matrix(A.R, B.R, c_dtype, A.codes.device)
+    ws = workspace if workspace is not None else _workspace(_lib.nvfp4_gemm_workspace_bytes(A.R, B.R, A.K), A.codes.device)
+    ca, cb = A.c(), B.c()
+    opts = CGemmOpts(variant, int(starve_first_stage), wait_limit_cycles)
+    _check(_lib.nvfp4_gemm_ex(ctypes.byref(ca), ctypes.byref(cb), _ptr(out), c_dtype, out.stride(0), int(accumulate),
+                              _ptr(dev_status), ctypes.byref(opts), _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_gemm_ex")
+    return out
+
+
 def nvfp4_outlier_accumulate(X: torch.Tensor, acc: torch.Tensor, workspace: torch.Tensor | None = None) -> torch.Tensor:
     """acc[d] += ||X[:, d]||_2 (one step of OutControl's calibration window); acc is float32 [D] on the device."""
     assert X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
@@ -290,7 +332,7 @@ def nvfp4_outlier_select(acc: torch.Tensor, n_out: int):
 def nvfp4_mma_issue_probe(iters: int, dev_status: torch.Tensor | None = None) -> float:
     """Enqueues the tensor-core issue loop (no memory traffic); returns the FP4 flops the launch performs."""
     fl = ctypes.c_double(0.0)
-    _check(_lib.nvfp4_mma_issue_probe(iters, _ptr(dev_status), ctypes.byref(fl), _stream_ptr()), "nvfp4_mma_issue_probe")
+    _check(measure_lib().nvfp4_mma_issue_probe(iters, _ptr(dev_status), ctypes.byref(fl), _stream_ptr()), "nvfp4_mma_issue_probe")
     return fl.value
 
 
@@ -380,14 +422,32 @@ class LayerConfig:
     rht: bool = False  # random Hadamard transformation of both operands of the two backward products
     outlier_fp8: bool = False  # outlier channels on a per-tensor power-of-two scaled E4M3 grid instead of BF16
     w_block16: bool = False  # weights in 16x16 scale squares (comparison recipe): dX uses the forward codes transposed, no Q4
+    # run the independent chains of a call (dX beside dW, the weight quantizer beside the activation quantizer) on a
+    # second stream: the stream and its three events are created here, with torch, and handed to the library
+    concurrent: bool = True
     # device index arrays, built by prepare()
     _outl: torch.Tensor | None = None
     _keep: torch.Tensor | None = None
     _map: torch.Tensor | None = None
     _D: int = -1
+    _side: tuple | None = None
+
+    def side(self, device):
+        """(stream, fork, join, aux) of the second stream for `device`, created on first use; None when not concurrent."""
+        if not self.concurrent:
+            return None
+        dev = torch.device(device)
+        dev = torch.device("cuda", torch.cuda.current_device()) if dev.index is None else dev
+        if self._side is None or self._side[0] != dev:
+            with torch.cuda.device(dev):
+                self._side = (dev, torch.cuda.Stream(device=dev), torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event())
+                for ev in self._side[2:]:
+                    ev.record(self._side[1])  # forces creation of the underlying CUDA events (torch makes them lazily)
+        return self._side[1:]
 
     def prepare(self, D: int, device="cuda"):
         """Uploads the OutControl index arrays for hidden size D (index bookkeeping only)."""
+        self.side(device)
         if self.outliers is None or len(self.outliers) == 0 or self._D == D:
             return
         outl = np.asarray(self.outliers, dtype=np.int64)
@@ -406,9 +466,11 @@ class LayerConfig:
         return 0 if self.outliers is None else len(self.outliers)
 
     def c(self) -> CLayerCfg:
+        side = self._side[1:] if (self.concurrent and self._side is not None) else None
+        sp = (side[0].cuda_stream, side[1].cuda_event, side[2].cuda_event, side[3].cuda_event) if side else (0, 0, 0, 0)
         return CLayerCfg(self.gs_mode, (c_i32 * 6)(*self.rounding), self.seed, self.y_dtype, self.dx_dtype, self.dw_dtype,
                          self.n_out, _ptr(self._outl), _ptr(self._keep), _ptr(self._map), _ptr(self.dev_status), int(self.rht),
-                         int(self.outlier_fp8), int(self.w_block16))
+                         int(self.outlier_fp8), int(self.w_block16), *sp)
 
 
 @dataclass
@@ -439,6 +501,24 @@ def alloc_saved(X: torch.Tensor, W: torch.Tensor, cfg: "LayerConfig") -> "Saved"
 
 def linear_workspace(op_kind: int, N_tok: int, D: int, C: int, cfg: LayerConfig, device="cuda") -> torch.Tensor:
     return _workspace(_lib.nvfp4_linear_workspace_bytes(op_kind, N_tok, D, C, cfg.n_out, cfg.gs_mode), device)
+
+
+def nvfp4_linear_bwd_operand(op_kind: int, which: int, N_tok: int, D: int, C: int, cfg: LayerConfig, workspace: torch.Tensor) -> Operand:
+    """View of backward operand Q3..Q6 (which = 3..6) inside the workspace of a backward call (no copy, nothing launched)."""
+    co = COperand()
+    _check(_lib.nvfp4_linear_bwd_operand(op_kind, which, N_tok, D, C, cfg.n_out, cfg.gs_mode, _ptr(workspace), workspace.numel(),
+                                         ctypes.byref(co)), "nvfp4_linear_bwd_operand")
+    base = workspace.data_ptr()
+
+    def view(ptr, nbytes, dtype):
+        off = ptr - base
+        return workspace[off: off + nbytes].view(dtype)
+
+    R, K = co.R, co.K
+    return Operand(view(co.codes, _lib.nvfp4_operand_codes_bytes(R, K), torch.uint8),
+                   view(co.sf, _lib.nvfp4_operand_sf_bytes(R, K, SF_TILED128x4), torch.uint8),
+                   view(co.gscale, 4 * _lib.nvfp4_operand_gscale_count(R, K, cfg.gs_mode), torch.float32), R, K, cfg.gs_mode,
+                   SF_TILED128x4)
 
 
 def nvfp4_linear_fwd(X: torch.Tensor, W: torch.Tensor, cfg: LayerConfig, Y: torch.Tensor | None = None,
@@ -491,6 +571,7 @@ def nvfp4_linear_bwd(dY: torch.Tensor, saved: Saved, cfg: LayerConfig, dX: torch
     """Both backward products in one call (dX, dW); the per-tensor amax of dY is computed once where Q3 and Q5 share it."""
     N_tok, D = saved.X.shape
     C = saved.W.shape[0]
+    cfg.prepare(D, dY.device)
     if dX is None:
         dX = _matrix(N_tok, D, cfg.dx_dtype, dY.device)
     if dW is None:

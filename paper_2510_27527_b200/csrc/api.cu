@@ -2,6 +2,10 @@
 // quantizers and products are enqueued (paper Sec. 2.3; OutControl split of Sec. 4.2). No allocation, no
 // synchronisation: everything is enqueued on the caller's stream.
 #include "../../include/nvfp4.h"
+#include "../../include/nvfp4_measure.h"
+
+#include <map>
+#include <mutex>
 
 #include "nvfp4_device.cuh"
 #include "nvfp4_internal.h"
@@ -9,8 +13,54 @@
 using namespace nvfp4;
 
 namespace nvfp4 {
-long long g_launch_count = 0;
+std::atomic<long long> g_launch_count{0};
+
+// Per-device facts and settings (a process may drive several GPUs): compute capability, SM count, and the dynamic
+// shared-memory limit already granted to each kernel.
+namespace {
+constexpr int kMaxDevices = 64;
+struct DeviceCache {
+  int cc_major = -1;
+  int sm_count = 0;
+  std::map<const void*, size_t> dyn_smem;
+};
+std::mutex g_device_mutex;
+DeviceCache g_device[kMaxDevices];
+
+DeviceCache* current_device_cache() {  // call with g_device_mutex held
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  DeviceCache& d = g_device[dev];
+  if (d.cc_major < 0) {
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return nullptr;
+    d.cc_major = major;
+    d.sm_count = sms;
+  }
+  return &d;
 }
+}  // namespace
+
+int device_sm_count() {
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  DeviceCache* d = current_device_cache();
+  return d && d->sm_count > 0 ? d->sm_count : 1;
+}
+
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
+  if (bytes <= 48 * 1024) return cudaSuccess;
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  DeviceCache* d = current_device_cache();
+  if (!d) return cudaErrorInvalidDevice;
+  size_t& have = d->dyn_smem[kernel];
+  if (bytes <= have) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) have = bytes;
+  return e;
+}
+}  // namespace nvfp4
 
 namespace {
 
@@ -21,16 +71,10 @@ inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 nvfp4_status check_arch() {
-  static int cached_dev = -1;
-  static nvfp4_status cached = NVFP4_OK;
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return NVFP4_ERR_CUDA;
-  if (dev == cached_dev) return cached;
-  int major = 0;
-  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return NVFP4_ERR_CUDA;
-  cached_dev = dev;
-  cached = (major == 10) ? NVFP4_OK : NVFP4_ERR_ARCH;
-  return cached;
+  std::lock_guard<std::mutex> lock(g_device_mutex);
+  DeviceCache* d = current_device_cache();
+  if (!d) return NVFP4_ERR_CUDA;
+  return d->cc_major == 10 ? NVFP4_OK : NVFP4_ERR_ARCH;
 }
 
 bool valid_operand_desc(const nvfp4_operand* o) {
@@ -90,42 +134,32 @@ bool carve_operand(Carver& c, nvfp4_operand* o, int64_t R, int64_t K, int32_t gs
   return o->codes && o->sf && o->gscale;
 }
 
-// Side stream of nvfp4_linear_bwd (one per host thread and device), with the two events of its fork / join.
+// Head of the workspace of the two backward calls: amax cells, then the two operands (the rest follows in the callers).
+bool carve_bwd_dx(Carver& cv, int64_t N_tok, int64_t D, int64_t C, int32_t gs_mode, uint32_t** cells3, uint32_t** cells4,
+                  nvfp4_operand* q3, nvfp4_operand* q4) {
+  *cells3 = static_cast<uint32_t*>(cv.take(cells_bytes(N_tok, gs_mode)));
+  *cells4 = static_cast<uint32_t*>(cv.take(cells_bytes(D, gs_mode)));
+  return carve_operand(cv, q3, N_tok, C, gs_mode) && carve_operand(cv, q4, D, C, gs_mode) && *cells3 && *cells4;
+}
+bool carve_bwd_dw(Carver& cv, int64_t N_tok, int64_t Dk, int64_t C, int32_t gs_mode, uint32_t** cells5, uint32_t** cells6,
+                  nvfp4_operand* q5, nvfp4_operand* q6) {
+  *cells5 = static_cast<uint32_t*>(cv.take(cells_bytes(C, gs_mode)));
+  *cells6 = static_cast<uint32_t*>(cv.take(cells_bytes(Dk, gs_mode)));
+  return carve_operand(cv, q5, C, N_tok, gs_mode) && carve_operand(cv, q6, Dk, N_tok, gs_mode) && *cells5 && *cells6;
+}
+
+// The caller's optional second stream with its three events (nvfp4_layer_cfg); null when the call runs on one stream.
 struct SideStream {
   cudaStream_t stream = nullptr;
   cudaEvent_t fork = nullptr, join = nullptr, amax = nullptr;
 };
-static SideStream* side_stream_for_current_device() {
-  constexpr int kMaxDevices = 64;
-  thread_local SideStream table[kMaxDevices];
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-  SideStream& t = table[dev];
-  if (!t.stream) {
-    cudaStream_t s = nullptr;
-    cudaEvent_t f = nullptr, j = nullptr, a = nullptr;
-    if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess ||
-        cudaEventCreateWithFlags(&f, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&j, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&a, cudaEventDisableTiming) != cudaSuccess) {
-      if (s) cudaStreamDestroy(s);
-      if (f) cudaEventDestroy(f);
-      if (j) cudaEventDestroy(j);
-      if (a) cudaEventDestroy(a);
-      cudaGetLastError();
-      return nullptr;  // the caller falls back to one stream
-    }
-    t.stream = s; t.fork = f; t.join = j; t.amax = a;
-  }
-  return &t;
-}
-// NVFP4_BWD_CONCURRENT=0 keeps every chain of the layer calls on the caller's stream.
-static bool bwd_concurrency_enabled() {
-  static const bool on = [] {
-    const char* e = getenv("NVFP4_BWD_CONCURRENT");
-    return !(e && atoi(e) == 0);
-  }();
-  return on;
+static bool side_stream_of(const nvfp4_layer_cfg* cfg, SideStream* out) {
+  if (!cfg->side_stream) return false;
+  out->stream = static_cast<cudaStream_t>(cfg->side_stream);
+  out->fork = static_cast<cudaEvent_t>(cfg->ev_fork);
+  out->join = static_cast<cudaEvent_t>(cfg->ev_join);
+  out->amax = static_cast<cudaEvent_t>(cfg->ev_aux);
+  return true;
 }
 
 nvfp4_status do_quantize_rows(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, int32_t rounding,
@@ -184,8 +218,8 @@ nvfp4_status do_quantize_transpose(const TransposeSrc& src, int from_codes, int6
 }
 
 nvfp4_status do_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
-                     int32_t accumulate, const float* addend, int64_t ld_add, int32_t* dev_status, cudaStream_t st,
-                     const void* hp_a = nullptr, const void* hp_b = nullptr, int64_t hp_Kh = 0) {
+                     int32_t accumulate, int32_t* dev_status, cudaStream_t st, const void* hp_a = nullptr,
+                     const void* hp_b = nullptr, int64_t hp_Kh = 0, const nvfp4_gemm_opts* opts = nullptr) {
   if (A->gs_mode == NVFP4_GS_BLOCK128 && nvfp4_padded_k(A->K) > gemm_block128_max_k()) return NVFP4_ERR_LIMIT;
   GemmArgs g{};
   g.a_codes = A->codes;
@@ -202,12 +236,15 @@ nvfp4_status do_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, in
   g.c_is_f32 = c_dtype == NVFP4_DT_F32;
   g.ldc = ldc;
   g.accumulate = accumulate;
-  g.addend = addend;
-  g.ld_add = ld_add;
   g.dev_status = dev_status;
   g.hp_a = hp_a;
   g.hp_b = hp_b;
   g.hp_Kh = hp_Kh;
+  if (opts) {
+    g.variant = opts->variant;
+    g.wait_limit = opts->wait_limit_cycles;
+    g.starve_first_stage = opts->starve_first_stage;
+  }
   return launch_gemm(g, st) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
@@ -231,6 +268,7 @@ nvfp4_status check_cfg(const nvfp4_layer_cfg* cfg, int64_t D) {
     return NVFP4_ERR_ENUM;
   if (cfg->n_out < 0 || cfg->n_out > D) return NVFP4_ERR_SHAPE;
   if (cfg->n_out > 0 && (!cfg->outlier_cols || !cfg->keep_cols || !cfg->col_map)) return NVFP4_ERR_NULL;
+  if (cfg->side_stream && (!cfg->ev_fork || !cfg->ev_join || !cfg->ev_aux)) return NVFP4_ERR_NULL;
   return NVFP4_OK;
 }
 
@@ -264,7 +302,7 @@ size_t nvfp4_operand_gscale_count(int64_t R, int64_t K, int32_t gs_mode) {
   return (size_t)(R * (nvfp4_padded_k(K) / 128));
 }
 
-long long nvfp4_launch_count(void) { return g_launch_count; }
+long long nvfp4_launch_count(void) { return g_launch_count.load(std::memory_order_relaxed); }
 
 const char* nvfp4_status_string(nvfp4_status s) {
   switch (s) {
@@ -393,7 +431,16 @@ size_t nvfp4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) { return gemm
 
 nvfp4_status nvfp4_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
                         int32_t accumulate, int32_t* dev_status, void* workspace, size_t ws_bytes, void* stream) {
+  return nvfp4_gemm_ex(A, B, C, c_dtype, ldc, accumulate, dev_status, nullptr, workspace, ws_bytes, stream);
+}
+
+nvfp4_status nvfp4_gemm_ex(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
+                           int32_t accumulate, int32_t* dev_status, const nvfp4_gemm_opts* opts, void* workspace,
+                           size_t ws_bytes, void* stream) {
   if (!A || !B || !C) return NVFP4_ERR_NULL;
+  if (opts && (opts->variant < 0 || opts->variant > 2 || opts->wait_limit_cycles < 0 ||
+               (opts->variant == NVFP4_GEMM_PAIR256 && A->gs_mode == NVFP4_GS_BLOCK128)))
+    return NVFP4_ERR_ENUM;
   nvfp4_status s;
   if ((s = check_operand_ptrs(A)) != NVFP4_OK) return s;
   if ((s = check_operand_ptrs(B)) != NVFP4_OK) return s;
@@ -405,7 +452,7 @@ nvfp4_status nvfp4_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C,
   const size_t need = nvfp4_gemm_workspace_bytes(A->R, B->R, A->K);
   if (need && (!workspace || ws_bytes < need)) return NVFP4_ERR_WORKSPACE;
   if ((s = check_arch()) != NVFP4_OK) return s;
-  return do_gemm(A, B, C, c_dtype, ldc, accumulate, nullptr, 0, dev_status, static_cast<cudaStream_t>(stream));
+  return do_gemm(A, B, C, c_dtype, ldc, accumulate, dev_status, static_cast<cudaStream_t>(stream), nullptr, nullptr, 0, opts);
 }
 
 size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, int64_t C, int64_t n_out,
@@ -436,6 +483,31 @@ size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, i
     }
   }
   return ((total + 255) & ~(size_t)255) + 256;
+}
+
+nvfp4_status nvfp4_linear_bwd_operand(int32_t op_kind, int32_t which, int64_t N_tok, int64_t D, int64_t C, int64_t n_out,
+                                      int32_t gs_mode, void* workspace, size_t ws_bytes, nvfp4_operand* out) {
+  if (!workspace || !out) return NVFP4_ERR_NULL;
+  if (gs_mode < 0 || gs_mode > 2 || which < 3 || which > 6) return NVFP4_ERR_ENUM;
+  if (N_tok <= 0 || D <= 0 || C <= 0 || n_out < 0 || n_out >= D) return NVFP4_ERR_SHAPE;
+  const bool dx = which <= 4;
+  if (!(op_kind == NVFP4_OP_BWD || (dx && op_kind == NVFP4_OP_BWD_DX) || (!dx && op_kind == NVFP4_OP_BWD_DW))) return NVFP4_ERR_ENUM;
+  if (ws_bytes < nvfp4_linear_workspace_bytes(op_kind, N_tok, D, C, n_out, gs_mode)) return NVFP4_ERR_WORKSPACE;
+  uint8_t* base = static_cast<uint8_t*>(workspace);
+  size_t size = ws_bytes;
+  if (op_kind == NVFP4_OP_BWD && !dx) {  // the dW half follows the dX half
+    const size_t need_dx = nvfp4_linear_workspace_bytes(NVFP4_OP_BWD_DX, N_tok, D, C, n_out, gs_mode);
+    base += need_dx;
+    size -= need_dx;
+  }
+  Carver cv(base, size);
+  uint32_t *ca, *cb;
+  nvfp4_operand qa, qb;
+  const bool ok = dx ? carve_bwd_dx(cv, N_tok, D, C, gs_mode, &ca, &cb, &qa, &qb)
+                     : carve_bwd_dw(cv, N_tok, D - n_out, C, gs_mode, &ca, &cb, &qa, &qb);
+  if (!ok) return NVFP4_ERR_WORKSPACE;
+  *out = (which == 3 || which == 5) ? qa : qb;
+  return NVFP4_OK;
 }
 
 nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t ldw, int64_t N_tok, int64_t D,
@@ -478,7 +550,8 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
   const int64_t Kh = n_out > 0 ? nvfp4_outlier_pad(n_out) : 0;
   if (n_out > 0 && (!saved->X_out || !saved->W_out)) return NVFP4_ERR_NULL;
   // Q1 and Q2 (each with its own amax pass where it has one) are independent: the weight side runs on the side stream
-  SideStream* side = bwd_concurrency_enabled() ? side_stream_for_current_device() : nullptr;
+  SideStream side_store;
+  SideStream* side = side_stream_of(cfg, &side_store) ? &side_store : nullptr;
   if (side && (cudaEventRecord(side->fork, st) != cudaSuccess || cudaStreamWaitEvent(side->stream, side->fork, 0) != cudaSuccess))
     return NVFP4_ERR_CUDA;
   const nvfp4_status s_x = do_quantize_rows(Xp, N_tok, D, ldx, cfg->rounding[0], cfg->seed, 1, keep, Dk, &saved->qx, cells_x, st, 1,
@@ -508,9 +581,9 @@ nvfp4_status nvfp4_linear_fwd(const void* X, int64_t ldx, const void* W, int64_t
   saved->X = X; saved->W = W; saved->ldx = ldx; saved->ldw = ldw;
   saved->N_tok = N_tok; saved->D = D; saved->C = C;
   if (n_out > 0)  // Y = FP4 product + X_out W_out^T, both inside one kernel
-    return do_gemm(&saved->qx, &saved->qw, Y, cfg->y_dtype, ldy, 0, nullptr, 0, cfg->dev_status, st, saved->X_out, saved->W_out,
+    return do_gemm(&saved->qx, &saved->qw, Y, cfg->y_dtype, ldy, 0, cfg->dev_status, st, saved->X_out, saved->W_out,
                    nvfp4_outlier_pad(n_out));
-  return do_gemm(&saved->qx, &saved->qw, Y, cfg->y_dtype, ldy, 0, nullptr, 0, cfg->dev_status, st);
+  return do_gemm(&saved->qx, &saved->qw, Y, cfg->y_dtype, ldy, 0, cfg->dev_status, st);
 }
 
 // dy_amax: optional cell already holding the bit pattern of max |dY| (TENSOR mode without the Hadamard transformation):
@@ -531,11 +604,9 @@ static nvfp4_status bwd_dx_impl(const void* dY, int64_t lddy, const nvfp4_saved*
   if ((s = check_arch()) != NVFP4_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   Carver cv(workspace, ws_bytes);
-  uint32_t* cells3 = static_cast<uint32_t*>(cv.take(cells_bytes(N_tok, cfg->gs_mode)));
-  uint32_t* cells4 = static_cast<uint32_t*>(cv.take(cells_bytes(D, cfg->gs_mode)));
+  uint32_t *cells3, *cells4;
   nvfp4_operand q3, q4;
-  if (!carve_operand(cv, &q3, N_tok, C, cfg->gs_mode) || !carve_operand(cv, &q4, D, C, cfg->gs_mode) || !cells3 || !cells4)
-    return NVFP4_ERR_WORKSPACE;
+  if (!carve_bwd_dx(cv, N_tok, D, C, cfg->gs_mode, &cells3, &cells4, &q3, &q4)) return NVFP4_ERR_WORKSPACE;
   // with a shared dY amax and a TENSOR -> TENSOR re-quantization (closed-form maximum) no cell of this call is read
   const bool cells_unused = cfg->gs_mode == NVFP4_GS_BLOCK128 ||
                             (dy_amax && n_out == 0 && cfg->gs_mode == NVFP4_GS_TENSOR && saved->qw.gs_mode == NVFP4_GS_TENSOR && !cfg->rht);
@@ -547,7 +618,7 @@ static nvfp4_status bwd_dx_impl(const void* dY, int64_t lddy, const nvfp4_saved*
     return s;
   if (cfg->weight_block == 1) {
     if ((s = do_transpose_operand16(&saved->qw, &q4, st)) != NVFP4_OK) return s;
-    return do_gemm(&q3, &q4, dX, cfg->dx_dtype, lddx, 0, nullptr, 0, cfg->dev_status, st);
+    return do_gemm(&q3, &q4, dX, cfg->dx_dtype, lddx, 0, cfg->dev_status, st);
   }
   TransposeSrc ts{};
   ts.in_codes = saved->qw.codes;
@@ -612,7 +683,7 @@ static nvfp4_status bwd_dx_impl(const void* dY, int64_t lddy, const nvfp4_saved*
     qa.src = th;
     if (launch_quantize_transpose(qa, st) != cudaSuccess) return NVFP4_ERR_CUDA;
   }
-  return do_gemm(&q3, &q4, dX, cfg->dx_dtype, lddx, 0, nullptr, 0, cfg->dev_status, st);
+  return do_gemm(&q3, &q4, dX, cfg->dx_dtype, lddx, 0, cfg->dev_status, st);
 }
 
 nvfp4_status nvfp4_linear_bwd_dx(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
@@ -632,6 +703,7 @@ static nvfp4_status bwd_dw_impl(const void* dY, int64_t lddy, const nvfp4_saved*
   if ((s = check_operand_ptrs(&saved->qx)) != NVFP4_OK) return s;
   if (saved->qx.R != N_tok || saved->qx.K != Dk) return NVFP4_ERR_SHAPE;
   if (n_out > 0 && !saved->X_out) return NVFP4_ERR_NULL;
+  if (n_out > 0 && !hp_dw_assemble_fits(D, n_out)) return NVFP4_ERR_LIMIT;
   const int dw_f32 = cfg->dw_dtype == NVFP4_DT_F32;
   if (bad_matrix(dY, lddy, C, 2) || bad_matrix(dW, lddw, D, dw_f32 ? 4 : 2)) return NVFP4_ERR_ALIGN;
   if (!workspace || ws_bytes < nvfp4_linear_workspace_bytes(NVFP4_OP_BWD_DW, N_tok, D, C, n_out, cfg->gs_mode))
@@ -639,12 +711,9 @@ static nvfp4_status bwd_dw_impl(const void* dY, int64_t lddy, const nvfp4_saved*
   if ((s = check_arch()) != NVFP4_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   Carver cv(workspace, ws_bytes);
-  uint32_t* cells5 = static_cast<uint32_t*>(cv.take(cells_bytes(C, cfg->gs_mode)));
-  uint32_t* cells6 = static_cast<uint32_t*>(cv.take(cells_bytes(Dk, cfg->gs_mode)));
+  uint32_t *cells5, *cells6;
   nvfp4_operand q5, q6;
-  if (!carve_operand(cv, &q5, C, N_tok, cfg->gs_mode) || !carve_operand(cv, &q6, Dk, N_tok, cfg->gs_mode) || !cells5 ||
-      !cells6)
-    return NVFP4_ERR_WORKSPACE;
+  if (!carve_bwd_dw(cv, N_tok, Dk, C, cfg->gs_mode, &cells5, &cells6, &q5, &q6)) return NVFP4_ERR_WORKSPACE;
   const int64_t ld_compact = round_up(Dk, 4);
   const int64_t Kh = nvfp4_outlier_pad(n_out);
   float* compact = n_out > 0 ? static_cast<float*>(cv.take((size_t)C * ld_compact * 4)) : nullptr;
@@ -671,11 +740,11 @@ static nvfp4_status bwd_dw_impl(const void* dY, int64_t lddy, const nvfp4_saved*
   if ((s = do_quantize_transpose(t5, 0, N_tok, C, cfg->rounding[4], cfg->seed, 5, &q5, dy_amax ? dy_amax : cells5, st, 1, rht,
                                  dy_amax ? 0 : 1)) != NVFP4_OK)
     return s;
-  if (n_out == 0) return do_gemm(&q5, &q6, dW, cfg->dw_dtype, lddw, 0, nullptr, 0, cfg->dev_status, st);
+  if (n_out == 0) return do_gemm(&q5, &q6, dW, cfg->dw_dtype, lddw, 0, cfg->dev_status, st);
 
   // kept columns: compact product; one pass then writes dW row by row from it and from the outlier channels' side product
   // (a scattering GEMM epilogue measured slower)
-  if ((s = do_gemm(&q5, &q6, compact, NVFP4_DT_F32, ld_compact, 0, nullptr, 0, cfg->dev_status, st)) != NVFP4_OK) return s;
+  if ((s = do_gemm(&q5, &q6, compact, NVFP4_DT_F32, ld_compact, 0, cfg->dev_status, st)) != NVFP4_OK) return s;
   HpDwArgs h{};
   h.dY = static_cast<const uint16_t*>(dY); h.X_out = static_cast<const uint16_t*>(saved->X_out);
   h.lddy = lddy; h.Kh = Kh; h.T = N_tok; h.C = C; h.n_out = n_out; h.outl = cfg->outlier_cols;
@@ -691,13 +760,6 @@ static nvfp4_status bwd_dw_impl(const void* dY, int64_t lddy, const nvfp4_saved*
 nvfp4_status nvfp4_linear_bwd_dw(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg,
                                  void* dW, int64_t lddw, void* workspace, size_t ws_bytes, void* stream) {
   return bwd_dw_impl(dY, lddy, saved, cfg, dW, lddw, workspace, ws_bytes, stream, nullptr);
-}
-
-nvfp4_status nvfp4_mma_issue_probe(int32_t iters, int32_t* dev_status, double* flops_out, void* stream) {
-  if (iters <= 0 || iters > (1 << 20)) return NVFP4_ERR_SHAPE;
-  nvfp4_status s = check_arch();
-  if (s != NVFP4_OK) return s;
-  return launch_mma_issue_probe(iters, dev_status, static_cast<cudaStream_t>(stream), flops_out) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
 nvfp4_status nvfp4_linear_bwd(const void* dY, int64_t lddy, const nvfp4_saved* saved, const nvfp4_layer_cfg* cfg, void* dX,
@@ -722,7 +784,9 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, int64_t lddy, const nvfp4_saved* s
   nvfp4_status s;
   if ((s = check_arch()) != NVFP4_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  SideStream* side = bwd_concurrency_enabled() ? side_stream_for_current_device() : nullptr;
+  if (cfg->side_stream && (!cfg->ev_fork || !cfg->ev_join || !cfg->ev_aux)) return NVFP4_ERR_NULL;
+  SideStream side_store;
+  SideStream* side = side_stream_of(cfg, &side_store) ? &side_store : nullptr;
   // Q3 and Q5 quantize the same tensor with the same per-tensor scale: one amax pass serves both. Without OutControl it
   // runs before the fork. With OutControl it runs at the head of the dX chain, and the dW chain, which starts with Q6 (no
   // dY involved), waits for it only before Q5: the bandwidth-bound amax pass and the arithmetic-bound Q6 overlap.

@@ -139,9 +139,12 @@ __global__ void __launch_bounds__(1024) outlier_compact_kernel(int64_t D, int32_
   }
 }
 
+// Row slabs of the partial-sum pass. A tuning constant, not a hardware query: the workspace size derived from it must not
+// depend on the device (about six CTAs per SM on a 148-SM part).
+constexpr int64_t kCalibTargetCtas = 888;
 static int64_t calib_slabs(int64_t N, int64_t D) {
   const int64_t col_ctas = (D + 255) / 256;
-  int64_t slabs = (148 * 6 + col_ctas - 1) / col_ctas;  // about six CTAs per SM in total
+  int64_t slabs = (kCalibTargetCtas + col_ctas - 1) / col_ctas;
   slabs = std::max<int64_t>(1, std::min<int64_t>(slabs, (N + 31) / 32));
   return slabs;
 }

@@ -9,52 +9,45 @@
 //               tcgen05.mma kind::mxf4nvf4 block_scale (E2M1 data, UE4M3 scale per 16 elements, K = 64 per
 //               instruction, FP32 accumulators in tensor memory, two accumulator buffers).
 //   warps 2..9  epilogue (two warps per tensor-memory lane quadrant, half of the tile's columns each): tcgen05.ld the
-//               accumulator, apply the FP32 global scales, add the optional addend, convert, stage 128-byte row pieces
-//               in shared memory and write them with bulk tensor stores. (The outer-block variant further down keeps
-//               four promotion warps, 2..5.)
-// Every wait on an mbarrier is bounded; when a bound is hit the kernel raises a status word, all roles drain and
-// the CTA frees its tensor memory and exits.
+//               accumulator, apply the FP32 global scales, convert, stage 128-byte row pieces in shared memory and
+//               write them with bulk tensor stores. (The outer-block variant further down keeps four promotion
+//               warps, 2..5.)
+// Every wait on an mbarrier is bounded (Params::wait_limit clock cycles); when a bound is hit the kernel raises a
+// status word, all roles drain and the CTA frees its tensor memory and exits.
 #include <cuda.h>
 #include <cuda_bf16.h>
-#include <cstdlib>
 
 #include "nvfp4_device.cuh"
 #include "nvfp4_internal.h"
+#include "nvfp4_tc.cuh"
 
 namespace nvfp4 {
 
 namespace {
 
-constexpr int BM = 128;
-constexpr int BK = 256;                                  // elements per k tile = one 128-byte swizzle row
-constexpr uint32_t A_BYTES = BM * BK / 2;                // 16 KB
-constexpr uint32_t SFA_BYTES = 2048;                     // 128 rows x 16 k-blocks
 constexpr int NUM_THREADS = 192;
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;    // ~2 s
 
-template <int BN>
+// Single-CTA kernel: 128 x 128 output tiles.
+constexpr int BN = 128;
 struct Cfg {
   static constexpr uint32_t B_BYTES = BN * BK / 2;
-  static constexpr uint32_t SFB_BYTES = (BN / 128) * 2048;
-  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;  // multiple of 1024
-  static constexpr int STAGES = (BN == 128) ? 5 : 4;
-  // epilogue staging for bulk tensor stores: per epilogue warp one 32-row x 128-byte buffer (128 x 128 tiles only;
-  // the 128 x 256 variant has no shared memory left and stores straight from registers)
-  static constexpr bool TMA_STORE = (BN == 128);
-  static constexpr uint32_t STAGING_BYTES = TMA_STORE ? 8 * 4096 : 0;
+  static constexpr uint32_t SFB_BYTES = 2048;
+  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;  // 36 KB, multiple of 1024
+  static constexpr int STAGES = 5;
+  // epilogue staging for bulk tensor stores: per epilogue warp one 32-row x 128-byte buffer
+  static constexpr uint32_t STAGING_BYTES = 8 * 4096;
   static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*align slack*/ + 256 /*barriers*/;
-  // tensor memory columns: two accumulators, then four scale buffers (A: 16 columns, B: 16 * BN / 128)
+  // tensor memory columns: two accumulators (a tile's epilogue runs under the next tile's MMAs), the optional
+  // high-precision accumulator, then four scale buffers (A: 16 columns, B: 16)
   static constexpr uint32_t ACC_COLS = BN;
-  static constexpr uint32_t ACC_BUFS = (BN == 256) ? 1 : 2;  // 256-wide accumulators leave no room for a second one
-  // The single-accumulator variant drains tensor memory into registers first (eight epilogue warps, 128 columns each),
-  // hands the accumulator back, and only then scales / converts / stores: the next tile's MMAs run under the stores.
-  // Eight epilogue warps in both variants: two per tensor-memory lane quadrant, each taking half of the tile's columns
-  // (a 128 x 128 tile's epilogue with four warps took 1.9 us and bounded every product with K <= 1024).
+  static constexpr uint32_t ACC_BUFS = 2;
+  // Eight epilogue warps: two per tensor-memory lane quadrant, each taking half of the tile's columns (a tile's
+  // epilogue with four warps took 1.9 us and bounded every product with K <= 1024).
   static constexpr int EPI_WARPS = 8;
   static constexpr int THREADS = 64 + 32 * EPI_WARPS;
-  static constexpr uint32_t SF_COLS = 16 + 16 * (BN / 128);
+  static constexpr uint32_t SF_COLS = 32;
   static constexpr uint32_t TMEM_COLS = 512;
-  static_assert(ACC_BUFS * ACC_COLS + 4 * SF_COLS <= TMEM_COLS, "tensor memory budget");
+  static_assert(ACC_BUFS * ACC_COLS + 128 + 4 * SF_COLS <= TMEM_COLS, "tensor memory budget");
 };
 
 struct Params {
@@ -62,8 +55,6 @@ struct Params {
   const uint8_t* b_sf;
   const float* a_gscale;
   const float* b_gscale;
-  const float* addend;  // optional FP32 [M, N] (leading dimension ld_add) added before the store
-  int64_t ld_add;
   void* C;
   int64_t ldc;
   int64_t M, N;
@@ -76,179 +67,14 @@ struct Params {
   int32_t c_is_f32, accumulate;
   int32_t hp_k_tiles;     // OutControl: 64-wide BF16 k tiles of the high-precision side product (0 = none)
   int32_t use_tma_store;  // C is described by a tensor map: stage the epilogue in shared memory and bulk-store it
+  int32_t starve;         // test hook: the first stage's "full" barrier expects 16 bytes more than will ever arrive
+  long long wait_limit;   // bound of every wait, in clock cycles
   int32_t* dev_status;
 };
 
-// ---------------------------------------------------------------------------------------------------------
-// PTX wrappers
-// ---------------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-// The issuing warps stay converged; instructions that one thread must issue take a `leader` flag (1 in exactly one
-// lane) and are predicated inside the asm, so their operands remain warp-uniform values.
-__device__ __forceinline__ uint32_t elect_leader() {
-  uint32_t pred;
-  asm volatile("{\n.reg .pred P;\nelect.sync _|P, 0xFFFFFFFF;\nselp.u32 %0, 1, 0, P;\n}" : "=r"(pred));
-  return pred;
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes, uint32_t leader) {
-  asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %2, 0;\n@q mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n}" ::"r"(bar),
-               "r"(bytes), "r"(leader)
-               : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait. Returns false when the bound ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
-  if (mbar_try(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (true) {
-    if (mbar_try(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-      *abort_flag = 1;
-      if (dev_status) atomicExch(dev_status, 8 /* NVFP4_ERR_TIMEOUT */);
-      return false;
-    }
-  }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int32_t c0, int32_t c1, uint32_t bar,
-                                            uint32_t leader) {
-  asm volatile(
-      "{\n.reg .pred q;\nsetp.ne.b32 q, %5, 0;\n"
-      "@q cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];\n}" ::"r"(dst),
-      "l"(tm), "r"(c0), "r"(c1), "r"(bar), "r"(leader)
-      : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint32_t leader) {
-  asm volatile(
-      "{\n.reg .pred q;\nsetp.ne.b32 q, %4, 0;\n"
-      "@q cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n}" ::"r"(dst),
-      "l"(src), "r"(bytes), "r"(bar), "r"(leader)
-      : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar, uint32_t leader) {
-  asm volatile(
-      "{\n.reg .pred q;\nsetp.ne.b32 q, %1, 0;\n"
-      "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(bar),
-      "r"(leader)
-      : "memory");
-}
-__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc, uint32_t leader) {
-  asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %2, 0;\n@q tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;\n}" ::"r"(taddr),
-               "l"(sdesc), "r"(leader)
-               : "memory");
-}
-__device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate, uint32_t leader) {
-  asm volatile(
-      "{\n.reg .pred p, q;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "setp.ne.b32 q, %7, 0;\n"
-      "@q tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem), "r"(leader)
-      : "memory");
-}
-// BF16 x BF16 -> FP32 (kind::f16), K = 16 per instruction; used for OutControl's high-precision side product.
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
-                                            uint32_t leader) {
-  asm volatile(
-      "{\n.reg .pred p, q;\n"
-      "setp.ne.b32 p, %4, 0;\n"
-      "setp.ne.b32 q, %5, 0;\n"
-      "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader)
-      : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptors (start address, leading / stride byte offsets in 16-byte units, version 1).
-// Code tiles: k-major rows of 128 bytes with the 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t desc_sw128(uint32_t saddr) {
-  return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)1 << 16) | ((uint64_t)64 << 32) | ((uint64_t)1 << 46) |
-         ((uint64_t)2 << 61);
-}
-// Scale tiles: 32 rows of 16 bytes, unswizzled, 8-row groups 128 bytes apart.
-__device__ __forceinline__ uint64_t desc_sf(uint32_t saddr) {
-  return (uint64_t)((saddr >> 4) & 0x3FFFu) | ((uint64_t)8 << 32) | ((uint64_t)1 << 46);
-}
-// The 32 per-row global scales SgB[n0 .. n0 + 32) of a ROW-mode B operand (0 beyond N); every lane reads the same values, in
-// four-wide loads when the run lies inside the matrix and is 16-byte aligned.
-__device__ __forceinline__ void load_sgb32(const float* __restrict__ g, int64_t n0, int64_t N, float (&out)[32]) {
-  if (n0 + 32 <= N && (reinterpret_cast<uintptr_t>(g + n0) & 15u) == 0) {
-    const float4* g4 = reinterpret_cast<const float4*>(g + n0);
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      const float4 t = __ldg(g4 + q);
-      out[4 * q] = t.x; out[4 * q + 1] = t.y; out[4 * q + 2] = t.z; out[4 * q + 3] = t.w;
-    }
-  } else {
-#pragma unroll
-    for (int j = 0; j < 32; ++j) out[j] = (n0 + j < N) ? __ldg(g + n0 + j) : 0.0f;
-  }
-}
-// Instruction descriptor: E2M1 x E2M1, UE4M3 scales, M = 128, N = BN, both operands k-major, K = 64.
-template <int BN>
-__device__ __forceinline__ uint32_t instr_desc() {
-  return (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (0u << 23) | ((uint32_t)(BM >> 4) << 24);
-}
-
-// Bulk tensor store of a staged [32 rows x 128 bytes] block (128-byte swizzle) to C; rows / columns outside C are clipped.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, uint32_t src, int32_t c0, int32_t c1) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(tm), "r"(src), "r"(c0),
-               "r"(c1)
-               : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() {
-  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-// Adds the optional FP32 addend and, when accumulating, the old C to W consecutive values of output row m from column n0
-// (a full chunk inside C).
+// When accumulating: adds the old C to W consecutive values of output row m from column n0 (a full chunk inside C).
 template <int W>
 __device__ __forceinline__ void add_existing(const Params& p, int64_t m, int64_t n0, float (&o)[W]) {
-  if (p.addend) {
-    const float* ad = p.addend + m * p.ld_add + n0;
-#pragma unroll
-    for (int j = 0; j < W; j += 4) {
-      const float4 q = *reinterpret_cast<const float4*>(ad + j);
-      o[j] += q.x; o[j + 1] += q.y; o[j + 2] += q.z; o[j + 3] += q.w;
-    }
-  }
   if (p.accumulate) {
     if (p.c_is_f32) {
       const float* cp = reinterpret_cast<const float*>(p.C) + m * p.ldc + n0;
@@ -273,21 +99,9 @@ __device__ __forceinline__ void add_existing(const Params& p, int64_t m, int64_t
   }
 }
 
-// One output row, 32 consecutive columns starting at n0 (m < M and n0 < N are the caller's business): add the optional
-// FP32 addend and the old C when accumulating, convert, store.
+// One output row, 32 consecutive columns starting at n0 (m < M and n0 < N are the caller's business): add the old C when
+// accumulating, convert, store.
 __device__ __forceinline__ void store_row_chunk(const Params& p, int64_t m, int64_t n0, float (&o)[32]) {
-    if (p.addend) {
-      const float* ad = p.addend + m * p.ld_add + n0;
-      if (n0 + 32 <= p.N) {
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          const float4 q = *reinterpret_cast<const float4*>(ad + j);
-          o[j] += q.x; o[j + 1] += q.y; o[j + 2] += q.z; o[j + 3] += q.w;
-        }
-      } else {
-        for (int j = 0; j < 32 && n0 + j < p.N; ++j) o[j] += ad[j];
-      }
-    }
     if (p.c_is_f32) {
       float* cp = reinterpret_cast<float*>(p.C) + m * p.ldc + n0;
       if (n0 + 32 <= p.N) {
@@ -334,12 +148,12 @@ __device__ __forceinline__ void store_row_chunk(const Params& p, int64_t m, int6
     }
 }
 
-template <int GS, int BN>
-__global__ void __launch_bounds__(Cfg<BN>::THREADS, 1)
+template <int GS>
+__global__ void __launch_bounds__(Cfg::THREADS, 1)
 gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmAh,
                   const __grid_constant__ CUtensorMap tmBh, const Params p) {
-  using C = Cfg<BN>;
+  using C = Cfg;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t staging_base = smem_base + C::STAGES * C::STAGE_BYTES;
@@ -351,8 +165,8 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * C::STAGES + 2 + b); };
   const uint32_t drain_bar = bar_base + 8u * (2 * C::STAGES + 4);
   const uint32_t hp_empty_bar = bar_base + 8u * (2 * C::STAGES + 5);  // high-precision accumulator drained
-  // tensor-memory columns of the optional high-precision accumulator (128 x 128 tiles only) and of the scale buffers
-  const uint32_t hp_cols = (BN == 128 && p.hp_k_tiles > 0) ? 128u : 0u;
+  // tensor-memory columns of the optional high-precision accumulator and of the scale buffers
+  const uint32_t hp_cols = p.hp_k_tiles > 0 ? 128u : 0u;
   const uint32_t hp_tmem_col = C::ACC_BUFS * C::ACC_COLS;
   const uint32_t sf_tmem_col = C::ACC_BUFS * C::ACC_COLS + hp_cols;
   __shared__ uint32_t tmem_base_slot;
@@ -397,33 +211,29 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
       const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
       const uint8_t* sfa_src = p.a_sf + (size_t)mt * p.sf_tiles_a * 512;
-      const uint8_t* sfb_src = p.b_sf + (size_t)nt * (BN / 128) * p.sf_tiles_b * 512;
+      const uint8_t* sfb_src = p.b_sf + (size_t)nt * p.sf_tiles_b * 512;
       for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
         const int s = it % C::STAGES;
         const uint32_t round = it / C::STAGES;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), (round & 1) ^ 1, abort_flag, p.dev_status));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), (round & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
-        mbar_expect_tx(full_bar(s), C::STAGE_BYTES, leader);
+        // (test hook of the bounded waits: with `starve` the very first stage never completes)
+        mbar_expect_tx(full_bar(s), C::STAGE_BYTES + ((p.starve && it == 0) ? 16u : 0u), leader);
         tma_load_2d(st, &tmA, kt * (BK / 2), mt * BM, full_bar(s), leader);
         tma_load_2d(st + A_BYTES, &tmB, kt * (BK / 2), nt * BN, full_bar(s), leader);
         bulk_load(st + A_BYTES + C::B_BYTES, sfa_src + (size_t)kt * 2048, 2048, full_bar(s), leader);
-#pragma unroll
-        for (int h = 0; h < BN / 128; ++h)
-          bulk_load(st + A_BYTES + C::B_BYTES + SFA_BYTES + h * 2048,
-                    sfb_src + ((size_t)h * p.sf_tiles_b * 512) + (size_t)kt * 2048, 2048, full_bar(s), leader);
+        bulk_load(st + A_BYTES + C::B_BYTES + SFA_BYTES, sfb_src + (size_t)kt * 2048, 2048, full_bar(s), leader);
       }
-      if (BN == 128) {
-        // OutControl: the BF16 outlier channels of both operands, 64 per stage, into the same stage buffers
-        for (int32_t h = 0; h < p.hp_k_tiles && ok; ++h, ++it) {
-          const int s = it % C::STAGES;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, abort_flag, p.dev_status));
-          if (!ok) break;
-          const uint32_t st = smem_base + s * C::STAGE_BYTES;
-          mbar_expect_tx(full_bar(s), A_BYTES + C::B_BYTES, leader);
-          tma_load_2d(st, &tmAh, h * 64, mt * BM, full_bar(s), leader);
-          tma_load_2d(st + A_BYTES, &tmBh, h * 64, nt * BN, full_bar(s), leader);
-        }
+      // OutControl: the BF16 outlier channels of both operands, 64 per stage, into the same stage buffers
+      for (int32_t h = 0; h < p.hp_k_tiles && ok; ++h, ++it) {
+        const int s = it % C::STAGES;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
+        if (!ok) break;
+        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        mbar_expect_tx(full_bar(s), A_BYTES + C::B_BYTES, leader);
+        tma_load_2d(st, &tmAh, h * 64, mt * BM, full_bar(s), leader);
+        tma_load_2d(st + A_BYTES, &tmBh, h * 64, nt * BN, full_bar(s), leader);
       }
     }
     if (!ok) {
@@ -432,7 +242,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       for (uint32_t j = 0; j < n_back; ++j) {
         const uint32_t f = it - 1 - j;
         const long long t0 = clock64();
-        while (!mbar_try(full_bar(f % C::STAGES), (f / C::STAGES) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
+        while (!mbar_try(full_bar(f % C::STAGES), (f / C::STAGES) & 1) && clock64() - t0 < p.wait_limit) {
         }
       }
     }
@@ -444,13 +254,13 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     bool ok = true;
     for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
       const uint32_t ab = tile_it % C::ACC_BUFS;
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar(ab), ((tile_it / C::ACC_BUFS) & 1) ^ 1, abort_flag, p.dev_status));
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar(ab), ((tile_it / C::ACC_BUFS) & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
       if (!ok) break;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + ab * C::ACC_COLS;
       for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
         const int s = it % C::STAGES;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / C::STAGES) & 1, abort_flag, p.dev_status));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / C::STAGES) & 1, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         tc_fence_after();
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
@@ -460,27 +270,24 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
         for (int kk = 0; kk < BK / 64; ++kk) {
           tc_cp_sf(sf_tmem + kk * 4, desc_sf(st + A_BYTES + C::B_BYTES + kk * 512), leader);
-#pragma unroll
-          for (int h = 0; h < BN / 128; ++h)
-            tc_cp_sf(sf_tmem + 16 + (kk * (BN / 128) + h) * 4,
-                     desc_sf(st + A_BYTES + C::B_BYTES + SFA_BYTES + h * 2048 + kk * 512), leader);
+          tc_cp_sf(sf_tmem + 16 + kk * 4, desc_sf(st + A_BYTES + C::B_BYTES + SFA_BYTES + kk * 512), leader);
         }
 #pragma unroll
         for (int kk = 0; kk < BK / 64; ++kk)
           tc_mma_nvf4(d_tmem, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc, sf_tmem + kk * 4,
-                      sf_tmem + 16 + kk * (BN / 128) * 4, (kt | kk) != 0, leader);
+                      sf_tmem + 16 + kk * 4, (kt | kk) != 0, leader);
         tc_commit(empty_bar(s), leader);  // stage reusable once these MMAs have read it
       }
-      if (BN == 128 && p.hp_k_tiles > 0 && ok) {
+      if (p.hp_k_tiles > 0 && ok) {
         // high-precision side product into its own accumulator (single buffer: wait until the previous tile's epilogue
         // has drained it, which happened a whole main loop ago)
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(hp_empty_bar, (tile_it & 1) ^ 1, abort_flag, p.dev_status));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(hp_empty_bar, (tile_it & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         tc_fence_after();
         const uint32_t idesc_bf16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
         for (int32_t h = 0; h < p.hp_k_tiles; ++h, ++it) {
           const int s = it % C::STAGES;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / C::STAGES) & 1, abort_flag, p.dev_status));
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / C::STAGES) & 1, abort_flag, p.dev_status, p.wait_limit));
           if (!ok) break;
           tc_fence_after();
           const uint32_t st = smem_base + s * C::STAGE_BYTES;
@@ -498,7 +305,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     tc_commit(drain_bar, leader);
     {
       const long long t0 = clock64();
-      while (!mbar_try(drain_bar, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
+      while (!mbar_try(drain_bar, 0) && clock64() - t0 < p.wait_limit) {
       }
     }
   } else {
@@ -511,40 +318,13 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
       const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
       const uint32_t ab = tile_it % C::ACC_BUFS;
-      if (!(ok = mbar_wait(acc_full_bar(ab), (tile_it / C::ACC_BUFS) & 1, abort_flag, p.dev_status))) break;
+      if (!(ok = mbar_wait(acc_full_bar(ab), (tile_it / C::ACC_BUFS) & 1, abort_flag, p.dev_status, p.wait_limit))) break;
       tc_fence_after();
       const int64_t m = (int64_t)mt * BM + quad * 32 + lane;
       float sa = 1.0f;
       if (GS == kGsRow && m < p.M) sa = p.a_gscale[m];
       const int half = (warp - 2) >> 2;  // which half of the tile's columns this warp owns
-      if (BN == 256) {
-        // drain this warp's 32 lanes x 128 columns into registers, release the accumulator, then store
-        uint32_t v[4][32];
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-          tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + half * 128 + q * 32, v[q]);
-        tc_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty_bar(ab));
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const int64_t n0 = (int64_t)nt * BN + half * 128 + q * 32;
-          if (m < p.M && n0 < p.N) {
-            float o[32], sgb[32];
-            if (GS == kGsRow) load_sgb32(p.b_gscale, n0, p.N, sgb);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              float sc = alpha;
-              if (GS == kGsRow) sc = __fmul_rn(sa, sgb[j]);
-              o[j] = __uint_as_float(v[q][j]) * sc;
-            }
-            store_row_chunk(p, m, n0, o);
-          }
-        }
-        continue;
-      }
-      if (C::TMA_STORE && p.use_tma_store) {
+      {
         // Stage 128-byte row pieces (32 FP32 or 64 BF16 columns) in shared memory with the 128-byte swizzle and let the
         // bulk-tensor engine write them: full lines, clipped at the edges of C, asynchronous.
         const uint32_t my_stage = staging_base + (uint32_t)(warp - 2) * 4096u;
@@ -571,17 +351,13 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 #pragma unroll
               for (int j = 0; j < 32; ++j) o[j] += __uint_as_float(v[j]);
             }
-            if ((p.addend || p.accumulate) && m < p.M) {
+            if (p.accumulate && m < p.M) {
               if (n0 + 32 <= p.N) {
                 add_existing<32>(p, m, n0, o);
               } else {
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                  if (n0 + j < p.N) {
-                    if (p.addend) o[j] += p.addend[m * p.ld_add + n0 + j];
-                    if (p.accumulate) o[j] += reinterpret_cast<const float*>(p.C)[m * p.ldc + n0 + j];
-                  }
-                }
+                for (int j = 0; j < 32; ++j)
+                  if (n0 + j < p.N) o[j] += reinterpret_cast<const float*>(p.C)[m * p.ldc + n0 + j];
               }
             }
             const uint32_t buf = my_stage;
@@ -631,17 +407,13 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 o[32 + j] += __uint_as_float(v2[j]);
               }
             }
-            if ((p.addend || p.accumulate) && m < p.M) {
+            if (p.accumulate && m < p.M) {
               if (n0 + 64 <= p.N) {
                 add_existing<64>(p, m, n0, o);
               } else {
 #pragma unroll
-                for (int j = 0; j < 64; ++j) {
-                  if (n0 + j < p.N) {
-                    if (p.addend) o[j] += p.addend[m * p.ld_add + n0 + j];
-                    if (p.accumulate) o[j] += __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.C)[m * p.ldc + n0 + j]);
-                  }
-                }
+                for (int j = 0; j < 64; ++j)
+                  if (n0 + j < p.N) o[j] += __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.C)[m * p.ldc + n0 + j]);
               }
             }
             const uint32_t buf = my_stage;
@@ -667,30 +439,6 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             }
           }
         }
-      } else {
-#pragma unroll 1
-      for (int c0 = half * (BN / 2); c0 < (half + 1) * (BN / 2); c0 += 32) {
-        uint32_t v[32], vh[32];
-        tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * C::ACC_COLS + c0, v);
-        if (hp_cols) tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + hp_tmem_col + c0, vh);  // warp-uniform condition
-        tc_wait_ld();
-        const int64_t n0 = (int64_t)nt * BN + c0;
-        if (m < p.M && n0 < p.N) {
-          float o[32], sgb[32];
-          if (GS == kGsRow) load_sgb32(p.b_gscale, n0, p.N, sgb);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            float sc = alpha;
-            if (GS == kGsRow) sc = __fmul_rn(sa, sgb[j]);
-            o[j] = __uint_as_float(v[j]) * sc;
-          }
-          if (hp_cols) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] += __uint_as_float(vh[j]);
-          }
-          store_row_chunk(p, m, n0, o);
-        }
-      }
       }
       tc_fence_before();
       __syncwarp();
@@ -699,7 +447,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         if (hp_cols) mbar_arrive(hp_empty_bar);
       }
     }
-    if (C::TMA_STORE && lane == 0) bulk_wait_all();  // this lane's bulk stores are complete before the CTA may exit
+    if (lane == 0) bulk_wait_all();  // this lane's bulk stores are complete before the CTA may exit
   }
 
   // ===================================== teardown ============================================================
@@ -708,69 +456,6 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::TMEM_COLS) : "memory");
-  }
-}
-
-// =========================================================================================================
-// Issue-loop probe (a measurement aid, not a step of the method): every SM issues `iters` groups of four
-// tcgen05.mma kind::mxf4nvf4 instructions (M = 128, N = 256, K = 64 each) on operand and scale tiles that stay in
-// shared / tensor memory; no global memory is touched inside the loop. The rate it reaches is the tensor-core
-// ceiling this box gives the FP4 GEMMs at the clocks it runs under load.
-// =========================================================================================================
-constexpr uint32_t PROBE_SMEM_BYTES = 16384 + 32768 + 2048 + 4096 + 1024 + 64;
-
-__global__ void __launch_bounds__(64, 1) mma_issue_probe_kernel(int32_t iters, int32_t* dev_status) {
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t a_tile = smem_base, b_tile = smem_base + 16384, sfa = smem_base + 49152, sfb = sfa + 2048;
-  const uint32_t done_bar = sfb + 4096;
-  __shared__ uint32_t tmem_base_slot;
-  __shared__ int abort_flag_s;
-  const int warp = threadIdx.x >> 5;
-  // operands: the E2M1 code of 1.0 everywhere (0x22), scales: the E4M3 byte of 1.0 (0x38)
-  for (uint32_t i = threadIdx.x; i < (49152u >> 2); i += 64) reinterpret_cast<uint32_t*>(gen)[i] = 0x22222222u;
-  for (uint32_t i = threadIdx.x; i < (6144u >> 2); i += 64) reinterpret_cast<uint32_t*>(gen + 49152)[i] = 0x38383838u;
-  if (threadIdx.x == 0) {
-    abort_flag_s = 0;
-    mbar_init(done_bar, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes above, async-proxy reads below
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = tmem_base_slot;
-  pdl_prologue();
-  if (warp == 1) {
-    const uint32_t leader = elect_leader();
-    const uint32_t idesc = instr_desc<256>();
-    const uint32_t sf_tmem = tmem_base + 256;
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-      tc_cp_sf(sf_tmem + kk * 4, desc_sf(sfa + kk * 512), leader);
-      tc_cp_sf(sf_tmem + 16 + kk * 8, desc_sf(sfb + kk * 512), leader);
-      tc_cp_sf(sf_tmem + 16 + kk * 8 + 4, desc_sf(sfb + 2048 + kk * 512), leader);
-    }
-    for (int32_t it = 0; it < iters; ++it) {
-#pragma unroll
-      for (int kk = 0; kk < 4; ++kk)
-        tc_mma_nvf4(tmem_base, desc_sw128(a_tile + kk * 32), desc_sw128(b_tile + kk * 32), idesc, sf_tmem + kk * 4,
-                    sf_tmem + 16 + kk * 8, (it | kk) != 0, leader);
-    }
-    tc_commit(done_bar, leader);
-    __all_sync(0xFFFFFFFFu, mbar_wait(done_bar, 0, &abort_flag_s, dev_status));  // bounded
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 1) {
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
   }
 }
 
@@ -787,13 +472,13 @@ constexpr int B128_NBUF = 3;
 constexpr int B128_MAX_CHUNKS = 128;
 constexpr uint32_t B128_SGB_BYTES = (B128_MAX_CHUNKS + 1) * 128 * 4 + 512;  // + the high-precision partial; 1024-byte multiple
 constexpr uint32_t B128_STAGING_BYTES = 4 * 4096;  // one 32-row x 128-byte staging buffer per epilogue warp (bulk stores)
-constexpr uint32_t B128_SMEM_BYTES = B128_STAGES * Cfg<128>::STAGE_BYTES + B128_SGB_BYTES + B128_STAGING_BYTES + 1024 + 256;
+constexpr uint32_t B128_SMEM_BYTES = B128_STAGES * Cfg::STAGE_BYTES + B128_SGB_BYTES + B128_STAGING_BYTES + 1024 + 256;
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                            const __grid_constant__ CUtensorMap tmC, const __grid_constant__ CUtensorMap tmAh,
                            const __grid_constant__ CUtensorMap tmBh, const Params p) {
-  using C = Cfg<128>;
+  using C = Cfg;
   constexpr int BN = 128;
   constexpr int STAGES = B128_STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -848,7 +533,7 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
       const uint8_t* sfb_src = p.b_sf + (size_t)nt * p.sf_tiles_b * 512;
       for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
         const int s = it % STAGES;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.dev_status));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
         mbar_expect_tx(full_bar(s), C::STAGE_BYTES, leader);
@@ -860,7 +545,7 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
       // OutControl: the BF16 outlier channels of both operands, 64 per stage, into the same stage buffers
       for (int32_t h = 0; h < p.hp_k_tiles && ok; ++h, ++it) {
         const int s = it % STAGES;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.dev_status));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
         mbar_expect_tx(full_bar(s), A_BYTES + C::B_BYTES, leader);
@@ -873,7 +558,7 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
       for (uint32_t j = 0; j < n_back; ++j) {
         const uint32_t f = it - 1 - j;
         const long long t0 = clock64();
-        while (!mbar_try(full_bar(f % STAGES), (f / STAGES) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
+        while (!mbar_try(full_bar(f % STAGES), (f / STAGES) & 1) && clock64() - t0 < p.wait_limit) {
         }
       }
     }
@@ -885,7 +570,7 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
       for (int32_t kt = 0; kt < p.k_tiles && ok; ++kt, ++it) {
         const int s = it % STAGES;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.dev_status));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         tc_fence_after();
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
@@ -899,7 +584,7 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
         for (int half = 0; half < 2; ++half) {
           if (kt * 2 + half >= chunks) break;  // the padded half of the last k tile holds only zeros
           const uint32_t buf = cit % B128_NBUF;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(part_empty_bar(buf), ((cit / B128_NBUF) & 1) ^ 1, abort_flag, p.dev_status));
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(part_empty_bar(buf), ((cit / B128_NBUF) & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
           if (!ok) break;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * 128;
@@ -917,13 +602,13 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
       if (p.hp_k_tiles > 0 && ok) {
         // high-precision side product: one more partial, handed to the promotion warps like a 128-k chunk (scale 1)
         const uint32_t buf = cit % B128_NBUF;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(part_empty_bar(buf), ((cit / B128_NBUF) & 1) ^ 1, abort_flag, p.dev_status));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(part_empty_bar(buf), ((cit / B128_NBUF) & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         tc_fence_after();
         const uint32_t idesc_bf16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
         for (int32_t h = 0; h < p.hp_k_tiles; ++h, ++it) {
           const int s = it % STAGES;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.dev_status));
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.dev_status, p.wait_limit));
           if (!ok) break;
           tc_fence_after();
           const uint32_t st = smem_base + s * C::STAGE_BYTES;
@@ -941,7 +626,7 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
     tc_commit(drain_bar, leader);
     {
       const long long t0 = clock64();
-      while (!mbar_try(drain_bar, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
+      while (!mbar_try(drain_bar, 0) && clock64() - t0 < p.wait_limit) {
       }
     }
   } else {
@@ -990,7 +675,7 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
         sa_0 = sa_1;
         if (kc + 2 < chunks) sa_1 = __ldg(sa_row + kc + 2);
         const uint32_t buf = cit % B128_NBUF;
-        if (!(ok = mbar_wait(part_full_bar(buf), (cit / B128_NBUF) & 1, abort_flag, p.dev_status))) break;
+        if (!(ok = mbar_wait(part_full_bar(buf), (cit / B128_NBUF) & 1, abort_flag, p.dev_status, p.wait_limit))) break;
         tc_fence_after();
         const float2 sa2 = make_float2(sa, sa);
         const float4* sb4 = reinterpret_cast<const float4*>(sgb + kc * 128);
@@ -1012,7 +697,7 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
         __syncwarp();
         if (lane == 0) mbar_arrive(part_empty_bar(buf));
       }
-      if (ok && p.use_tma_store && !p.addend && !p.accumulate) {
+      if (ok && p.use_tma_store && !p.accumulate) {
         // 128-byte row pieces staged in shared memory with the 128-byte swizzle and written by the bulk-tensor engine:
         // full lines, clipped at the edges of C (a thread-per-row store from registers took longer than the whole
         // promotion loop of a K = 1024 tile)
@@ -1224,16 +909,23 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       const int32_t sfb_row0 = ((nt * 2) * p.sf_tiles_b) * 4, sfb_row1 = ((nt * 2 + 1) * p.sf_tiles_b) * 4;
       for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
         const int s = it % STAGES;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.dev_status));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         const uint32_t st = smem_base + s * C2_STAGE_BYTES;
         const uint32_t full0 = map_to_cta(full_bar(s), 0);
-        if (rank == 0) mbar_expect_tx(full_bar(s), 2 * C2_STAGE_BYTES, leader);
+        if (rank == 0) mbar_expect_tx(full_bar(s), 2 * C2_STAGE_BYTES + ((p.starve && it == 0) ? 16u : 0u), leader);
         tma_load_2d_pair(st, &tmA, kt * (BK / 2), a_row, full0, leader);
         tma_load_2d_pair(st + A_BYTES, &tmB, kt * (BK / 2), b_row, full0, leader);
         tma_load_2d_pair(st + A_BYTES + C2_B_BYTES, &tmSFA, 0, sfa_row + kt * 16, full0, leader);
         tma_load_2d_pair(st + A_BYTES + C2_B_BYTES + SFA_BYTES, &tmSFB, 0, sfb_row0 + kt * 16, full0, leader);
         tma_load_2d_pair(st + A_BYTES + C2_B_BYTES + SFA_BYTES + 2048, &tmSFB, 0, sfb_row1 + kt * 16, full0, leader);
+      }
+    }
+    if (!ok) {
+      // a wait ran out: this CTA's copies in flight complete on the leader's barrier, which the peer cannot poll, so give
+      // them a fixed time (far more than a copy takes) to land before the CTA may exit
+      const long long t0 = clock64();
+      while (clock64() - t0 < 400000) {
       }
     }
   } else if (warp == 1) {
@@ -1244,12 +936,12 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       uint32_t it = 0, tile_it = 0;
       bool ok = true;
       for (int64_t t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar, (tile_it & 1) ^ 1, abort_flag, p.dev_status));
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar, (tile_it & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         tc_fence_after();
         for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
           const int s = it % STAGES;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.dev_status));
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.dev_status, p.wait_limit));
           if (!ok) break;
           tc_fence_after();
           const uint32_t st = smem_base + s * C2_STAGE_BYTES;
@@ -1276,7 +968,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           : "memory");
       {
         const long long t0 = clock64();
-        while (!mbar_try(drain_bar, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {
+        while (!mbar_try(drain_bar, 0) && clock64() - t0 < p.wait_limit) {
         }
       }
     }
@@ -1291,7 +983,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     if (GS == kGsTensor) alpha = __fmul_rn(p.a_gscale[0], p.b_gscale[0]);
     for (int64_t t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
       const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
-      if (!(ok = mbar_wait(acc_full_bar, tile_it & 1, abort_flag, p.dev_status))) break;
+      if (!(ok = mbar_wait(acc_full_bar, tile_it & 1, abort_flag, p.dev_status, p.wait_limit))) break;
       tc_fence_after();
       const int64_t m = (int64_t)mt * 256 + rank * 128 + quad * 32 + lane;
       float sa = 1.0f;
@@ -1346,7 +1038,7 @@ constexpr int HPDW_THREADS = 192;
 
 __global__ void __launch_bounds__(HPDW_THREADS, 1)
 hp_dw_mma_kernel(const __grid_constant__ CUtensorMap tmDY, const __grid_constant__ CUtensorMap tmXO, float* __restrict__ partial,
-                 int64_t C, int32_t Kh, int64_t T, int32_t t_per_split, int32_t* dev_status) {
+                 int64_t C, int32_t Kh, int64_t ld_partial, int64_t T, int32_t t_per_split, int32_t* dev_status, long long wait_limit) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t b_bytes = (uint32_t)(Kh / 64) * 8192u;
@@ -1390,7 +1082,7 @@ hp_dw_mma_kernel(const __grid_constant__ CUtensorMap tmDY, const __grid_constant
     const uint32_t leader = elect_leader();
     for (int32_t kt = 0; kt < k_tiles; ++kt) {
       const int s = kt % HPDW_STAGES;
-      if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((kt / HPDW_STAGES) & 1) ^ 1, abort_flag, dev_status))) break;
+      if (!__all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((kt / HPDW_STAGES) & 1) ^ 1, abort_flag, dev_status, wait_limit))) break;
       const uint32_t st = smem_base + s * stage_bytes;
       const int32_t t0 = (int32_t)(t_begin + (int64_t)kt * 64);
       mbar_expect_tx(full_bar(s), stage_bytes, leader);
@@ -1406,7 +1098,7 @@ hp_dw_mma_kernel(const __grid_constant__ CUtensorMap tmDY, const __grid_constant
     bool ok = true;
     for (int32_t kt = 0; kt < k_tiles && ok; ++kt) {
       const int s = kt % HPDW_STAGES;
-      ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (kt / HPDW_STAGES) & 1, abort_flag, dev_status));
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (kt / HPDW_STAGES) & 1, abort_flag, dev_status, wait_limit));
       if (!ok) break;
       tc_fence_after();
       const uint32_t st = smem_base + s * stage_bytes;
@@ -1423,10 +1115,10 @@ hp_dw_mma_kernel(const __grid_constant__ CUtensorMap tmDY, const __grid_constant
     tc_commit(acc_full_bar, leader);  // also covers the k_tiles == 0 case (arrives at once)
   } else {
     const int quad = warp & 3;
-    if (mbar_wait(acc_full_bar, 0, abort_flag, dev_status)) {
+    if (mbar_wait(acc_full_bar, 0, abort_flag, dev_status, wait_limit)) {
       tc_fence_after();
       const int64_t c = (int64_t)c0 + quad * 32 + lane;
-      float* dst = partial + ((int64_t)blockIdx.y * C + (c < C ? c : 0)) * Kh;
+      float* dst = partial + ((int64_t)blockIdx.y * C + (c < C ? c : 0)) * ld_partial;
       for (int j0 = 0; j0 < Kh; j0 += 32) {
         uint32_t v[32];
         tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + j0, v);
@@ -1509,38 +1201,30 @@ bool make_hp_map(CUtensorMap* tm, const void* base, int64_t R, int64_t Kh) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-  }
-  return n;
-}
+inline int sm_count() { return device_sm_count(); }
+inline long long wait_limit_of(const GemmArgs& a) { return a.wait_limit > 0 ? a.wait_limit : DEFAULT_WAIT_LIMIT_CYCLES; }
 
-template <int GS, int BN>
-cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
-  using C = Cfg<BN>;
+template <int GS>
+cudaError_t launch_tile128(const GemmArgs& a, cudaStream_t st) {
+  using C = Cfg;
   const int64_t Kp = (a.K + 127) & ~(int64_t)127;
   CUtensorMap tmA, tmB, tmC;
   if (!make_codes_map(&tmA, a.a_codes, a.M, Kp, BM) || !make_codes_map(&tmB, a.b_codes, a.N, Kp, BN))
     return cudaErrorInvalidValue;
-  const bool tma_store = C::TMA_STORE && make_c_map(&tmC, a.C, a.M, a.N, a.ldc, a.c_is_f32 != 0);
-  if (!tma_store) tmC = tmA;  // unused by the kernel then
+  if (!make_c_map(&tmC, a.C, a.M, a.N, a.ldc, a.c_is_f32 != 0)) return cudaErrorInvalidValue;
   CUtensorMap tmAh = tmA, tmBh = tmB;  // placeholders unless the high-precision side product is requested
   Params p{};
-  p.use_tma_store = tma_store ? 1 : 0;
+  p.use_tma_store = 1;
+  p.starve = a.starve_first_stage;
+  p.wait_limit = wait_limit_of(a);
   if (a.hp_Kh > 0) {
-    if (BN != 128 || !make_hp_map(&tmAh, a.hp_a, a.M, a.hp_Kh) || !make_hp_map(&tmBh, a.hp_b, a.N, a.hp_Kh)) return cudaErrorInvalidValue;
+    if (!make_hp_map(&tmAh, a.hp_a, a.M, a.hp_Kh) || !make_hp_map(&tmBh, a.hp_b, a.N, a.hp_Kh)) return cudaErrorInvalidValue;
     p.hp_k_tiles = (int32_t)(a.hp_Kh / 64);
   }
   p.a_sf = a.a_sf;
   p.b_sf = a.b_sf;
   p.a_gscale = a.a_gscale;
   p.b_gscale = a.b_gscale;
-  p.addend = a.addend;
-  p.ld_add = a.ld_add;
   p.C = a.C;
   p.ldc = a.ldc;
   p.M = a.M;
@@ -1555,16 +1239,11 @@ cudaError_t launch_variant(const GemmArgs& a, cudaStream_t st) {
   p.c_is_f32 = a.c_is_f32;
   p.accumulate = a.accumulate;
   p.dev_status = a.dev_status;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_kernel<GS, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)C::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(gemm_nvfp4_kernel<GS>), C::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
-  launch_kernel(gemm_nvfp4_kernel<GS, BN>, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, tmA, tmB, tmC, tmAh, tmBh, p);
+  launch_kernel(gemm_nvfp4_kernel<GS>, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, tmA, tmB, tmC, tmAh, tmBh, p);
   return cudaGetLastError();
 }
 
@@ -1595,8 +1274,6 @@ cudaError_t launch_2cta(const GemmArgs& a, cudaStream_t st) {
   p.b_sf = a.b_sf;
   p.a_gscale = a.a_gscale;
   p.b_gscale = a.b_gscale;
-  p.addend = a.addend;
-  p.ld_add = a.ld_add;
   p.C = a.C;
   p.ldc = a.ldc;
   p.M = a.M;
@@ -1608,12 +1285,10 @@ cudaError_t launch_2cta(const GemmArgs& a, cudaStream_t st) {
   p.c_is_f32 = a.c_is_f32;
   p.accumulate = a.accumulate;
   p.dev_status = a.dev_status;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_2cta_kernel<GS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C2_SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  p.starve = a.starve_first_stage;
+  p.wait_limit = wait_limit_of(a);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(gemm_nvfp4_2cta_kernel<GS>), C2_SMEM_BYTES);
+  if (e != cudaSuccess) return e;
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned pairs = (unsigned)std::min<int64_t>(tiles, sm_count() / 2);
   launch_kernel(gemm_nvfp4_2cta_kernel<GS>, dim3(2 * pairs), dim3(C2_THREADS), C2_SMEM_BYTES, st, tmA, tmB, tmSFA, tmSFB, p);
@@ -1637,8 +1312,6 @@ cudaError_t launch_block128(const GemmArgs& a, cudaStream_t st) {
   p.b_sf = a.b_sf;
   p.a_gscale = a.a_gscale;
   p.b_gscale = a.b_gscale;
-  p.addend = a.addend;
-  p.ld_add = a.ld_add;
   p.C = a.C;
   p.ldc = a.ldc;
   p.M = a.M;
@@ -1653,13 +1326,9 @@ cudaError_t launch_block128(const GemmArgs& a, cudaStream_t st) {
   p.c_is_f32 = a.c_is_f32;
   p.accumulate = a.accumulate;
   p.dev_status = a.dev_status;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_nvfp4_block128_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)B128_SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  p.wait_limit = wait_limit_of(a);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(gemm_nvfp4_block128_kernel), B128_SMEM_BYTES);
+  if (e != cudaSuccess) return e;
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
   launch_kernel(gemm_nvfp4_block128_kernel, dim3(grid), dim3(NUM_THREADS), B128_SMEM_BYTES, st, tmA, tmB, tmC, tmAh, tmBh, p);
@@ -1681,64 +1350,49 @@ bool make_tokens_map(CUtensorMap* tm, const void* base, int64_t T, int64_t W, in
 
 }  // namespace
 
-bool hp_dw_mma_supported(int64_t Kh) { return Kh >= 64 && Kh <= 256 && Kh % 64 == 0; }
-
-// partial[(split * C + c) * Kh + j] = sum over the split's tokens of dY[t, c] * X_out[t, j]
+// partial[(split * C + c) * Kh + j] = sum over the split's tokens of dY[t, c] * X_out[t, j]. Kh is any multiple of 64:
+// the outlier channels are taken in slabs of at most 256 (the widest MMA), one launch per slab.
 cudaError_t launch_hp_dw_mma(const uint16_t* dY, int64_t lddy, const uint16_t* X_out, int64_t Kh, int64_t T, int64_t C,
                              float* partial, int n_split, int64_t t_per_split, int32_t* dev_status, cudaStream_t st) {
+  if (Kh <= 0 || Kh % 64 != 0) return cudaErrorInvalidValue;
   CUtensorMap tmDY, tmXO;
-  if (!make_tokens_map(&tmDY, dY, T, C, lddy) || !make_tokens_map(&tmXO, X_out, T, Kh, Kh)) return cudaErrorInvalidValue;
-  const uint32_t stage_bytes = A_BYTES + (uint32_t)(Kh / 64) * 8192u;
-  const size_t smem = (size_t)HPDW_STAGES * stage_bytes + 1024 + 256;
-  static size_t configured = 0;
-  if (smem > configured) {
-    cudaError_t e = cudaFuncSetAttribute(hp_dw_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (!make_tokens_map(&tmDY, dY, T, C, lddy)) return cudaErrorInvalidValue;
+  for (int64_t j0 = 0; j0 < Kh; j0 += 256) {
+    const int64_t w = std::min<int64_t>(256, Kh - j0);
+    if (!make_tokens_map(&tmXO, X_out + j0, T, w, Kh)) return cudaErrorInvalidValue;
+    const uint32_t stage_bytes = A_BYTES + (uint32_t)(w / 64) * 8192u;
+    const size_t smem = (size_t)HPDW_STAGES * stage_bytes + 1024 + 256;
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(hp_dw_mma_kernel), smem);
     if (e != cudaSuccess) return e;
-    configured = smem;
+    const dim3 grid((unsigned)((C + 127) / 128), (unsigned)n_split);
+    launch_kernel(hp_dw_mma_kernel, dim3(grid), dim3(HPDW_THREADS), smem, st, tmDY, tmXO, partial + j0, C, (int32_t)w, Kh, T,
+                  (int32_t)t_per_split, dev_status, DEFAULT_WAIT_LIMIT_CYCLES);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
-  const dim3 grid((unsigned)((C + 127) / 128), (unsigned)n_split);
-  launch_kernel(hp_dw_mma_kernel, dim3(grid), dim3(HPDW_THREADS), smem, st, tmDY, tmXO, partial, C, (int32_t)Kh, T, (int32_t)t_per_split,
-                dev_status);
-  return cudaGetLastError();
+  return cudaSuccess;
 }
 
 size_t gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
 int64_t gemm_block128_max_k() { return (int64_t)B128_MAX_CHUNKS * 128; }
 
-cudaError_t launch_mma_issue_probe(int32_t iters, int32_t* dev_status, cudaStream_t st, double* flops) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(mma_issue_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PROBE_SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
-  const int ctas = sm_count();
-  if (flops) *flops = (double)ctas * (double)iters * 4.0 * 2.0 * 128.0 * 256.0 * 64.0;
-  launch_kernel(mma_issue_probe_kernel, dim3((unsigned)ctas), dim3(64), PROBE_SMEM_BYTES, st, iters, dev_status);
-  return cudaGetLastError();
-}
-
+// Variant choice. 128 x 128 single-CTA tiles with two accumulators (a tile's epilogue overlaps the next tile's MMAs) win for
+// short K; pairs of CTAs on 256 x 256 tiles (half the operand traffic per flop and SM) win once K is long and there are
+// enough tiles for every pair (measured on 8192 x 3072 x K: K = 2048 -> 39 us against 48 us, K = 4096 -> 60 against 57.5,
+// 16384 x 8192 x 8192 -> 477 against 380 us). A 256-row tile of an operand spans two 128-row scale tiles, and rows are padded
+// to 128 in the scale layout, so any M, N work. The fused high-precision side product and the outer-block scales live in
+// the single-CTA kernels only.
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;
-  // 128 x 256 tiles halve the operand traffic per flop; they pay off once there are enough of them to fill the SMs.
-  const char* force = getenv("NVFP4_GEMM_BN");
-  // (measured on 8192 x 3072 x K: at K = 2048 the 128 x 128 variant, whose two accumulators overlap epilogue and MMAs, is
-  // 39 us against 45-48 us for the wider single-accumulator variants; from K = 4096 on the wider ones win)
-  const bool wide = force ? atoi(force) == 256 : (a.K >= 3072 && ((a.M + 127) / 128) * ((a.N + 255) / 256) >= 2 * sm_count());
-  // Pairs of CTAs on 256 x 256 tiles for the largest products. A 256-row tile of an operand spans two 128-row scale
-  // tiles, and the last one must exist in full: rows are padded to 128 in the scale layout, so any M, N work.
-  const char* pair_env = getenv("NVFP4_GEMM_2CTA");
-  const bool pairs = pair_env ? atoi(pair_env) != 0
-                              : (a.K >= 3072 && ((a.M + 255) / 256) * ((a.N + 255) / 256) >= 2 * (sm_count() / 2));
-  if (a.hp_Kh > 0 && a.gs_mode != kGsBlock128)  // the fused high-precision side product lives in the 128 x 128 variants
-    return a.gs_mode == kGsTensor ? launch_variant<kGsTensor, 128>(a, st) : launch_variant<kGsRow, 128>(a, st);
-  if (pairs && a.gs_mode == kGsTensor) return launch_2cta<kGsTensor>(a, st);
-  if (pairs && a.gs_mode == kGsRow) return launch_2cta<kGsRow>(a, st);
-  switch (a.gs_mode) {
-    case kGsTensor: return wide ? launch_variant<kGsTensor, 256>(a, st) : launch_variant<kGsTensor, 128>(a, st);
-    case kGsRow: return wide ? launch_variant<kGsRow, 256>(a, st) : launch_variant<kGsRow, 128>(a, st);
-    default: return launch_block128(a, st);
+  if (a.gs_mode == kGsBlock128) return a.variant == 2 ? cudaErrorInvalidValue : launch_block128(a, st);
+  bool pairs = a.K >= 3072 && ((a.M + 255) / 256) * ((a.N + 255) / 256) >= 2 * (sm_count() / 2);
+  if (a.variant == 1) pairs = false;
+  if (a.variant == 2) pairs = true;
+  if (a.hp_Kh > 0) {
+    if (a.variant == 2) return cudaErrorInvalidValue;
+    pairs = false;
   }
+  if (pairs) return a.gs_mode == kGsTensor ? launch_2cta<kGsTensor>(a, st) : launch_2cta<kGsRow>(a, st);
+  return a.gs_mode == kGsTensor ? launch_tile128<kGsTensor>(a, st) : launch_tile128<kGsRow>(a, st);
 }
 
 }  // namespace nvfp4

@@ -1,96 +1,15 @@
 // High-precision side of OutControl (paper Sec. 4.2): the outlier channels of X / W stay in BF16. The forward side
-// product runs on the tensor cores inside the FP4 GEMM kernels; here are the copies that build the compact side
-// operands, the CUDA-core fallback of dW[:, outliers] = dY^T X_out for shapes the tensor-core kernel does not take, and
-// the pass that assembles dW from the compact FP4 product and the side product.
+// product runs on the tensor cores inside the FP4 GEMM kernels and dW[:, outliers] = dY^T X_out in a BF16 tensor-core
+// kernel of its own (gemm.cu); here are the copy that builds a compact side operand, the FP8 snap of the side operands,
+// and the pass that assembles dW from the compact FP4 product and the side product's token splits.
 #include "nvfp4_device.cuh"
 #include "nvfp4_internal.h"
 
 namespace nvfp4 {
 
-// dW[c, outl[j]] = sum_t dY[t, c] * X_out[t, j]. The token range is split over blockIdx.y; each CTA owns 64 output
-// channels c and walks its tokens in chunks of 64 staged in shared memory (dY chunk [64 t x 64 c], X_out chunk
-// [64 t x 64 j]); a thread accumulates 16 outlier channels for one c. Partial sums go to a workspace and a second
-// kernel adds them in a fixed order (bit-reproducible results).
+// Token splits of the side product dW[c, outl[j]] = sum_t dY[t, c] * X_out[t, j]: at most kHpDwSplit partial sums per output
+// element go to a workspace and are added in a fixed order (bit-reproducible results).
 constexpr int kHpDwSplit = 16;
-
-__global__ void __launch_bounds__(256) hp_dw_partial_kernel(HpDwArgs a, int64_t t_per_split) {
-  pdl_prologue();
-  __shared__ float dy_s[64][65];
-  __shared__ float x_s[64][64];
-  const int cl = threadIdx.x & 63, jg = threadIdx.x >> 6;  // jg: which 16 outlier channels of the 64-wide chunk
-  const int64_t c0 = (int64_t)blockIdx.x * 64;
-  const int64_t t_begin = (int64_t)blockIdx.y * t_per_split, t_end = min(a.T, t_begin + t_per_split);
-  for (int64_t j0 = 0; j0 < a.Kh; j0 += 64) {
-    if (j0 >= a.n_out) break;
-    const bool active = j0 + jg * 16 < a.n_out;
-    float acc[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j) acc[j] = 0.0f;
-    for (int64_t tc = t_begin; tc < t_end; tc += 64) {
-      __syncthreads();
-      for (int e = threadIdx.x; e < 64 * 8; e += 256) {  // 64 rows x 8 chunks of 8 BF16
-        const int tr = e >> 3, ch = (e & 7) << 3;
-        const int64_t t = tc + tr;
-        uint4 g = make_uint4(0, 0, 0, 0), x = make_uint4(0, 0, 0, 0);
-        if (t < t_end) {
-          if (c0 + ch + 8 <= a.C && (a.lddy & 7) == 0) {
-            g = *reinterpret_cast<const uint4*>(a.dY + t * a.lddy + c0 + ch);
-          } else {
-            uint32_t w[4] = {0, 0, 0, 0};
-            for (int q = 0; q < 8; ++q)
-              if (c0 + ch + q < a.C) w[q >> 1] |= (uint32_t)a.dY[t * a.lddy + c0 + ch + q] << (16 * (q & 1));
-            g = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-          x = *reinterpret_cast<const uint4*>(a.X_out + t * a.Kh + j0 + ch);
-        }
-        const uint32_t gw[4] = {g.x, g.y, g.z, g.w}, xw[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          dy_s[tr][ch + 2 * q] = bf16_lo(gw[q]);
-          dy_s[tr][ch + 2 * q + 1] = bf16_hi(gw[q]);
-          x_s[tr][ch + 2 * q] = bf16_lo(xw[q]);
-          x_s[tr][ch + 2 * q + 1] = bf16_hi(xw[q]);
-        }
-      }
-      __syncthreads();
-      if (active) {
-#pragma unroll 4
-        for (int tr = 0; tr < 64; ++tr) {
-          const float g = dy_s[tr][cl];
-          const float4* xr = reinterpret_cast<const float4*>(&x_s[tr][jg * 16]);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const float4 xv = xr[q];
-            acc[4 * q] = fmaf(g, xv.x, acc[4 * q]);
-            acc[4 * q + 1] = fmaf(g, xv.y, acc[4 * q + 1]);
-            acc[4 * q + 2] = fmaf(g, xv.z, acc[4 * q + 2]);
-            acc[4 * q + 3] = fmaf(g, xv.w, acc[4 * q + 3]);
-          }
-        }
-      }
-    }
-    if (active && c0 + cl < a.C) {
-      float* dst = a.partial + ((int64_t)blockIdx.y * a.C + c0 + cl) * a.Kh + j0 + jg * 16;
-#pragma unroll
-      for (int j = 0; j < 16; ++j) dst[j] = acc[j];
-    }
-  }
-}
-
-__global__ void __launch_bounds__(256) hp_dw_reduce_kernel(HpDwArgs a, int n_split) {
-  pdl_prologue();
-  const int64_t total = a.C * a.n_out;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t c = i / a.n_out, j = i - c * a.n_out;
-    float v = 0.0f;
-    for (int sp = 0; sp < n_split; ++sp) v += a.partial[((int64_t)sp * a.C + c) * a.Kh + j];
-    const int64_t o = c * a.lddw + a.outl[j];
-    if (a.dw_is_f32)
-      reinterpret_cast<float*>(a.dW)[o] = v;
-    else
-      reinterpret_cast<uint16_t*>(a.dW)[o] = f32_to_bf16_bits(v);
-  }
-}
 
 // dW[c, d] for whole output rows (OutControl's weight gradient): a kept channel takes its value from the compact FP4
 // product, an outlier channel the sum of the high-precision side product's token splits. One coalesced pass over dW
@@ -206,7 +125,8 @@ cudaError_t launch_fp8_snap_pair(uint16_t* a, int64_t rows_a, uint16_t* b, int64
   cudaError_t e;
   if ((e = launch_zero_words(cells2, 2, st)) != cudaSuccess) return e;
   if ((e = launch_amax_tensor_pair(a, rows_a, Kh, Kh, cells2, b, rows_b, Kh, Kh, cells2 + 1, st)) != cudaSuccess) return e;
-  auto grid_of = [](int64_t n) { return (unsigned)std::max<int64_t>(1, std::min<int64_t>((n / 2 + 255) / 256, 148 * 4)); };
+  const int64_t cap = (int64_t)device_sm_count() * 4;
+  auto grid_of = [cap](int64_t n) { return (unsigned)std::max<int64_t>(1, std::min<int64_t>((n / 2 + 255) / 256, cap)); };
   const unsigned ga = grid_of(rows_a * Kh), gb = grid_of(rows_b * Kh);
   launch_kernel(fp8_snap_pair_kernel, dim3(ga + gb), dim3(256), 0, st, a, rows_a * Kh, static_cast<const uint32_t*>(cells2), ga, b,
                 rows_b * Kh, static_cast<const uint32_t*>(cells2 + 1));
@@ -223,38 +143,12 @@ __global__ void __launch_bounds__(256) gather_cols_kernel(const uint16_t* __rest
   for (int64_t j = threadIdx.x & 31; j < ld_dst; j += 32) dst[r * ld_dst + j] = j < n ? src[r * ld_src + cols[j]] : (uint16_t)0;
 }
 
-// dst[r, keep[j]] = src[r, j]
-__global__ void __launch_bounds__(256) scatter_cols_kernel(const void* src, int64_t ld_src, int src_is_f32, void* dst,
-                                                          int64_t ld_dst, int dst_is_f32, int64_t rows, int64_t n_keep,
-                                                          const int32_t* __restrict__ keep) {
-  pdl_prologue();
-  const int64_t total = rows * n_keep;
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t r = i / n_keep, j = i - r * n_keep;
-    const int64_t o = r * ld_dst + keep[j];
-    if (src_is_f32) {
-      const float v = reinterpret_cast<const float*>(src)[r * ld_src + j];
-      if (dst_is_f32) {
-        reinterpret_cast<float*>(dst)[o] = v;
-      } else {
-        reinterpret_cast<uint16_t*>(dst)[o] = f32_to_bf16_bits(v);
-      }
-    } else {
-      const uint16_t v = reinterpret_cast<const uint16_t*>(src)[r * ld_src + j];
-      if (dst_is_f32)
-        reinterpret_cast<float*>(dst)[o] = bf16_bits_to_float(v);
-      else
-        reinterpret_cast<uint16_t*>(dst)[o] = v;
-    }
-  }
-}
-
 size_t hp_dw_partial_floats(int64_t T, int64_t C, int64_t Kh) { return (size_t)kHpDwSplit * (size_t)C * (size_t)Kh; }
 
 // token splits of the side product: as many as fill the SMs once with (C / 128) x splits CTAs, at most kHpDwSplit (the
 // workspace's size)
 static void hp_dw_splits(const HpDwArgs& a, int64_t& t_per_split, int& n_split) {
-  const int64_t want = std::max<int64_t>(1, std::min<int64_t>(kHpDwSplit, 148 / std::max<int64_t>(1, (a.C + 127) / 128)));
+  const int64_t want = std::max<int64_t>(1, std::min<int64_t>(kHpDwSplit, device_sm_count() / std::max<int64_t>(1, (a.C + 127) / 128)));
   t_per_split = ((a.T + want - 1) / want + 63) / 64 * 64;
   n_split = (int)((a.T + t_per_split - 1) / t_per_split);
 }
@@ -265,11 +159,7 @@ cudaError_t launch_hp_dw_product(const HpDwArgs& a, cudaStream_t st) {
   int64_t t_per_split;
   int n_split;
   hp_dw_splits(a, t_per_split, n_split);
-  if (hp_dw_mma_supported(a.Kh) && (a.lddy & 7) == 0)  // tensor-core path (the CUDA-core kernel covers odd shapes)
-    return launch_hp_dw_mma(a.dY, a.lddy, a.X_out, a.Kh, a.T, a.C, a.partial, n_split, t_per_split, a.dev_status, st);
-  const dim3 grid((unsigned)((a.C + 63) / 64), (unsigned)n_split);
-  launch_kernel(hp_dw_partial_kernel, dim3(grid), dim3(256), 0, st, a, t_per_split);
-  return cudaGetLastError();
+  return launch_hp_dw_mma(a.dY, a.lddy, a.X_out, a.Kh, a.T, a.C, a.partial, n_split, t_per_split, a.dev_status, st);
 }
 
 // Second half: dW from the compact FP4 product and the split partial sums.
@@ -278,33 +168,25 @@ cudaError_t launch_hp_dw_finish(const HpDwArgs& a, cudaStream_t st) {
   int64_t t_per_split;
   int n_split;
   hp_dw_splits(a, t_per_split, n_split);
-  cudaError_t e;
-  if (a.compact && a.col_map && a.D < ((int64_t)1 << 29) && (a.D + 4 + kAsmRows * a.n_out) * 4 <= 200 * 1024) {
-    // kept and outlier channels written together, row by row
-    const size_t smem = (size_t)(((a.D + 3) & ~(int64_t)3) + kAsmRows * a.n_out) * 4;
-    const int f32 = a.dw_is_f32;
-    const int elt = f32 ? 4 : 2;
-    const int vec = (a.lddw & 3) == 0 && (reinterpret_cast<uintptr_t>(a.dW) & (size_t)(4 * elt - 1)) == 0;
-    if (smem > 48 * 1024) {
-      e = f32 ? cudaFuncSetAttribute(dw_assemble_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-              : cudaFuncSetAttribute(dw_assemble_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-    }
-    const dim3 grid((unsigned)std::min<int64_t>((a.C + kAsmRows - 1) / kAsmRows, 148 * 8));
-    if (f32)
-      launch_kernel(dw_assemble_kernel<true>, grid, dim3(256), smem, st, a, n_split, a.compact, a.ld_compact, a.col_map, a.D, vec);
-    else
-      launch_kernel(dw_assemble_kernel<false>, grid, dim3(256), smem, st, a, n_split, a.compact, a.ld_compact, a.col_map, a.D, vec);
-    return cudaGetLastError();
-  }
-  if (a.compact) {
-    e = launch_scatter_cols(a.compact, a.ld_compact, 1, a.dW, a.lddw, a.dw_is_f32, a.C, a.D - a.n_out, a.keep, st);
-    if (e != cudaSuccess) return e;
-  }
-  const int64_t total = a.C * a.n_out;
-  launch_kernel(hp_dw_reduce_kernel, dim3((unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8)), dim3(256), 0, st, a, n_split);
+  if (!a.compact || !a.col_map || !hp_dw_assemble_fits(a.D, a.n_out)) return cudaErrorInvalidValue;
+  // kept and outlier channels written together, row by row
+  const size_t smem = (size_t)(((a.D + 3) & ~(int64_t)3) + kAsmRows * a.n_out) * 4;
+  const int f32 = a.dw_is_f32;
+  const int elt = f32 ? 4 : 2;
+  const int vec = (a.lddw & 3) == 0 && (reinterpret_cast<uintptr_t>(a.dW) & (size_t)(4 * elt - 1)) == 0;
+  const cudaError_t e = ensure_dynamic_smem(f32 ? reinterpret_cast<const void*>(dw_assemble_kernel<true>)
+                                                : reinterpret_cast<const void*>(dw_assemble_kernel<false>), smem);
+  if (e != cudaSuccess) return e;
+  const dim3 grid((unsigned)std::min<int64_t>((a.C + kAsmRows - 1) / kAsmRows, (int64_t)device_sm_count() * 8));
+  if (f32)
+    launch_kernel(dw_assemble_kernel<true>, grid, dim3(256), smem, st, a, n_split, a.compact, a.ld_compact, a.col_map, a.D, vec);
+  else
+    launch_kernel(dw_assemble_kernel<false>, grid, dim3(256), smem, st, a, n_split, a.compact, a.ld_compact, a.col_map, a.D, vec);
   return cudaGetLastError();
 }
+
+// The assembling pass keeps one source index per channel and kAsmRows sums per outlier channel in shared memory.
+bool hp_dw_assemble_fits(int64_t D, int64_t n_out) { return (D + 4 + kAsmRows * n_out) * 4 <= 200 * 1024; }
 
 cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st) {
   const cudaError_t e = launch_hp_dw_product(a, st);
@@ -315,15 +197,6 @@ cudaError_t launch_gather_cols(const uint16_t* src, int64_t ld_src, int64_t rows
                                int64_t ld_dst, cudaStream_t st) {
   if (rows == 0 || ld_dst == 0) return cudaSuccess;
   launch_kernel(gather_cols_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, st, src, ld_src, rows, cols, n, dst, ld_dst);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_scatter_cols(const void* src, int64_t ld_src, int src_is_f32, void* dst, int64_t ld_dst,
-                                int dst_is_f32, int64_t rows, int64_t n_keep, const int32_t* keep, cudaStream_t st) {
-  const int64_t total = rows * n_keep;
-  if (total == 0) return cudaSuccess;
-  const unsigned grid = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 32);
-  launch_kernel(scatter_cols_kernel, dim3(grid), dim3(256), 0, st, src, ld_src, src_is_f32, dst, ld_dst, dst_is_f32, rows, n_keep, keep);
   return cudaGetLastError();
 }
 

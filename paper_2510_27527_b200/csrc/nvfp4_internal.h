@@ -4,14 +4,20 @@
 #include <stdint.h>
 
 #include <algorithm>
+#include <atomic>
 
 namespace nvfp4 {
 
 // Number of kernels this library has enqueued since it was loaded (measurement aid).
-extern long long g_launch_count;
+extern std::atomic<long long> g_launch_count;
 
 // true if the current device has compute capability 10.x (cached per device)
 bool device_is_sm100();
+// Number of SMs of the current device (queried once per device).
+int device_sm_count();
+// Raises a kernel's dynamic shared-memory limit to at least `bytes` on the current device; remembered per device and
+// kernel, so the attribute call is made once per pair.
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes);
 
 struct QuantRowsArgs {
   const uint16_t* src;  // BF16 [rows, cols_src], leading dimension ld
@@ -87,7 +93,7 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  ++g_launch_count;
+  g_launch_count.fetch_add(1, std::memory_order_relaxed);
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
@@ -114,8 +120,6 @@ struct GemmArgs {
   int c_is_f32;
   int64_t ldc;
   int accumulate;
-  const float* addend;  // optional FP32 [M, N] added in the epilogue (leading dimension ld_add)
-  int64_t ld_add;
   // optional high-precision side product (OutControl): C += hp_a [M, hp_Kh] * hp_b [N, hp_Kh]^T, BF16 inputs, FP32
   // accumulation on the tensor cores inside the same kernel (TENSOR / ROW modes)
   const void* hp_a;
@@ -124,12 +128,13 @@ struct GemmArgs {
   int32_t* dev_status;
   void* workspace;
   size_t ws_bytes;
+  int variant;               // nvfp4_gemm_variant of the ABI header (0 = chosen from the shape)
+  long long wait_limit;      // bound of every device-side wait in clock cycles (<= 0: the default, about two seconds)
+  int starve_first_stage;    // test hook of the bounded waits: the first stage's barrier expects bytes that never arrive
 };
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
 int64_t gemm_block128_max_k();  // largest K the BLOCK128 GEMM variant takes
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
-// Tensor-core issue loop without memory traffic (measurement aid); *flops = FP4 flops the launch performs.
-cudaError_t launch_mma_issue_probe(int32_t iters, int32_t* dev_status, cudaStream_t st, double* flops);
 
 // High-precision (BF16 inputs, FP32 accumulate) products over OutControl's outlier channels.
 //   fwd: Y[m, n] (+)= sum_j X[m, outl[j]] * W[n, outl[j]]
@@ -166,16 +171,12 @@ struct HpDwArgs {
   const int32_t* col_map;
 };
 size_t hp_dw_partial_floats(int64_t T, int64_t C, int64_t Kh);
-bool hp_dw_mma_supported(int64_t Kh);
+bool hp_dw_assemble_fits(int64_t D, int64_t n_out);  // the assembling pass of dW handles this many channels
 cudaError_t launch_hp_dw_mma(const uint16_t* dY, int64_t lddy, const uint16_t* X_out, int64_t Kh, int64_t T, int64_t C,
                              float* partial, int n_split, int64_t t_per_split, int32_t* dev_status, cudaStream_t st);
 cudaError_t launch_hp_dw(const HpDwArgs& a, cudaStream_t st);  // product, then finish, on one stream
 // the two halves, for callers that overlap the side product (which needs only dY and X_out) with other work
 cudaError_t launch_hp_dw_product(const HpDwArgs& a, cudaStream_t st);
 cudaError_t launch_hp_dw_finish(const HpDwArgs& a, cudaStream_t st);
-
-// Scatter a compact [C, n_keep] matrix into columns keep[j] of dW [C, D].
-cudaError_t launch_scatter_cols(const void* src, int64_t ld_src, int src_is_f32, void* dst, int64_t ld_dst,
-                                int dst_is_f32, int64_t rows, int64_t n_keep, const int32_t* keep, cudaStream_t st);
 
 }  // namespace nvfp4

@@ -623,7 +623,7 @@ size_t osci_cells(int64_t C, int32_t gs_mode) { return gs_mode == kGsRow ? (size
 bool bad_f32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
 cudaError_t run_amax(const float* W, int64_t ld, int64_t C, int64_t D, uint32_t* cells, int per_row, cudaStream_t st) {
-  const unsigned grid = (unsigned)std::min<int64_t>(C, 148 * 8);
+  const unsigned grid = (unsigned)std::min<int64_t>(C, device_sm_count() * 8);
   launch_kernel(amax_f32_kernel, dim3(grid), dim3(256), 0, st, W, ld, C, D, cells, per_row);
   return cudaGetLastError();
 }
@@ -782,7 +782,7 @@ nvfp4_status nvfp4_osci_sparse_update(const float* W, int64_t ldw, int64_t C, in
     else if (gs_mode == kGsRow) launch_kernel(osci_score_kernel<kGsRow>, sgrid, dim3(256), 0, st, W, ldw, C, D, cells, ws.scores);
     else launch_kernel(osci_score_kernel<kGsBlock128>, sgrid, dim3(256), 0, st, W, ldw, C, D, cells, ws.scores);
     launch_kernel(osci_sel_init_kernel, dim3(1), dim3(256), 0, st, ws.sel, (uint32_t)n_track);
-    const unsigned hgrid = (unsigned)std::min<int64_t>((n + 255) / 256, 148 * 8);
+    const unsigned hgrid = (unsigned)std::min<int64_t>((n + 255) / 256, device_sm_count() * 8);
     for (int shift = 24; shift >= 0; shift -= 8) {
       launch_kernel(osci_hist_kernel, dim3(hgrid), dim3(256), 0, st, static_cast<const uint32_t*>(ws.scores), n, ws.sel, shift);
       launch_kernel(osci_pick_kernel, dim3(1), dim3(32), 0, st, ws.sel, shift);

@@ -860,14 +860,9 @@ static cudaError_t launch_rows_g(const QuantRowsArgs& a, cudaStream_t st) {
     if (smem > 160 * 1024 || (reinterpret_cast<uintptr_t>(a.keep) & 15u) != 0 || (a.ld & 7) != 0) {
       smem = 0;
       stage_cols8 = 0;  // fall back to per-element global loads
-    } else if (smem > 48 * 1024) {
-      static size_t configured = 0;
-      if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(quantize_rows_kernel<GS, SR, TILED, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             160 * 1024);
-        if (e != cudaSuccess) return e;
-        configured = 160 * 1024;
-      }
+    } else {
+      cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(quantize_rows_kernel<GS, SR, TILED, true, false>), smem);
+      if (e != cudaSuccess) return e;
     }
     launch_kernel(quantize_rows_kernel<GS, SR, TILED, true, false>, dim3(grid), dim3(256), smem, st, a.src, a.rows, a.K, a.ld, a.keep, a.seed,
                   a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.cols_src, stage_cols8, 0u, a.sr == 2, make_philox_keys(a.seed));
@@ -901,7 +896,7 @@ static cudaError_t launch_quantize_rows_impl(const QuantRowsArgs& a, cudaStream_
       const int per_row = a.gs_mode == kGsRow;
       if (!a.cells_zeroed && (e = launch_zero_words(a.gs_cells, per_row ? a.rows : 1, st)) != cudaSuccess) return e;
       const int64_t blocks16 = a.rows * ((a.K + 15) >> 4);
-      const unsigned grid = (unsigned)std::min<int64_t>((blocks16 + 255) / 256, 148 * 16);
+      const unsigned grid = (unsigned)std::min<int64_t>((blocks16 + 255) / 256, device_sm_count() * 16);
       launch_kernel(amax_rows_rht_kernel, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, a.seed, a.rht_stream, a.gs_cells, per_row);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
@@ -917,7 +912,7 @@ static cudaError_t launch_quantize_rows_impl(const QuantRowsArgs& a, cudaStream_
         const size_t smem = (size_t)((a.cols_src + 7) >> 3) * 16;  // one 16-byte mask per chunk (at most 40 KB)
         // a contiguous slab of rows per CTA. The side copy divides item numbers by the side operand's width through a
         // 32-bit reciprocal, exact while items * width < 2^32: slabs stay below 2^32 / d^2 rows (d also covers the chunk count)
-        int64_t rows_per_cta = (a.rows + 148 * 4 - 1) / (148 * 4);  // few, fat CTAs: the per-thread setup is paid once
+        int64_t rows_per_cta = (a.rows + device_sm_count() * 4 - 1) / (device_sm_count() * 4);  // few, fat CTAs: the per-thread setup is paid once
         const int64_t dmax = std::max<int64_t>((a.cols_src + 7) >> 3, a.excl_out ? a.ld_excl_out : 1);
         rows_per_cta = std::max<int64_t>(1, std::min<int64_t>(rows_per_cta, (((int64_t)1 << 32) - 1) / (dmax * dmax)));
         const unsigned grid = (unsigned)((a.rows + rows_per_cta - 1) / rows_per_cta);
@@ -934,7 +929,7 @@ static cudaError_t launch_quantize_rows_impl(const QuantRowsArgs& a, cudaStream_
         return launch_rows_r<kGsTensor>(a, st);
       }
       const int64_t chunks = a.rows * ((a.cols_src + 7) >> 3);
-      const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 8);
+      const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, device_sm_count() * 8);
       launch_kernel(amax_tensor_bf16_kernel, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.cols_src, a.ld, a.gs_cells);
       if ((e = cudaGetLastError()) != cudaSuccess) return e;
     }
@@ -1018,7 +1013,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
       if (!cell_unused && !a.cells_zeroed && (e = launch_zero_words(a.gs_cells, 1, st)) != cudaSuccess) return e;
       if (SRC == 0) {
         const int64_t chunks = a.rowsK * ((a.D + 7) >> 3);
-        const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 8);
+        const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, device_sm_count() * 8);
         launch_kernel(amax_tensor_bf16_kernel, dim3(grid), dim3(256), 0, st, a.src.bf16, a.rowsK, a.D, a.src.ld, a.gs_cells);
       } else if (a.src.in_gs_mode == kGsTensor) {
         a.tensor_closed_form = a.src.row_map ? 1 : 2;  // only the BF16 rows (if any) need a pass
@@ -1037,7 +1032,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
     if (SRC == 0 && !a.src.out_rows && (a.src.ld & 7) == 0 && (reinterpret_cast<uintptr_t>(a.src.bf16) & 15u) == 0) {
       // per-column maxima of the BF16 source by a streaming kernel (about 2 CTAs per SM worth of row slabs per column strip)
       const int64_t strips = (a.D + 255) / 256;
-      int64_t slabs = std::max<int64_t>(1, (148 * 4 + strips - 1) / strips);
+      int64_t slabs = std::max<int64_t>(1, (device_sm_count() * 4 + strips - 1) / strips);
       slabs = std::min<int64_t>(slabs, (a.rowsK + 63) / 64);
       const int64_t rows_per_slab = ((a.rowsK + slabs - 1) / slabs + 7) / 8 * 8;
       launch_kernel(amax_cols_bf16_kernel, dim3((unsigned)strips, (unsigned)((a.rowsK + rows_per_slab - 1) / rows_per_slab)), dim3(256), 0, st,
@@ -1054,7 +1049,7 @@ static cudaError_t launch_tr_s(const QuantTransposeArgs& a0, cudaStream_t st) {
 cudaError_t launch_amax_tensor(const uint16_t* src, int64_t rows, int64_t cols, int64_t ld, uint32_t* cell, cudaStream_t st) {
   if (rows == 0 || cols == 0) return cudaSuccess;
   const int64_t chunks = rows * ((cols + 7) >> 3);
-  const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, 148 * 8);
+  const unsigned grid = (unsigned)std::min<int64_t>((chunks + 255) / 256, device_sm_count() * 8);
   launch_kernel(amax_tensor_bf16_kernel, dim3(grid), dim3(256), 0, st, src, rows, cols, ld, cell);
   return cudaGetLastError();
 }
@@ -1066,7 +1061,7 @@ __global__ void __launch_bounds__(256) zero_words_kernel(uint32_t* p, int64_t n)
 }
 cudaError_t launch_zero_words(uint32_t* p, int64_t n, cudaStream_t st) {
   if (n <= 0) return cudaSuccess;
-  launch_kernel(zero_words_kernel, dim3((unsigned)std::min<int64_t>((n + 255) / 256, 148)), dim3(256), 0, st, p, n);
+  launch_kernel(zero_words_kernel, dim3((unsigned)std::min<int64_t>((n + 255) / 256, (int64_t)device_sm_count())), dim3(256), 0, st, p, n);
   return cudaGetLastError();
 }
 
@@ -1074,7 +1069,7 @@ cudaError_t launch_amax_tensor_pair(const uint16_t* a, int64_t rows_a, int64_t c
                                     int64_t rows_b, int64_t cols_b, int64_t ld_b, uint32_t* cell_b, cudaStream_t st) {
   auto grid_of = [](int64_t rows, int64_t cols) {
     const int64_t chunks = rows * ((cols + 7) >> 3);
-    return (unsigned)std::max<int64_t>(1, std::min<int64_t>((chunks + 255) / 256, 148 * 8));
+    return (unsigned)std::max<int64_t>(1, std::min<int64_t>((chunks + 255) / 256, device_sm_count() * 8));
   };
   const unsigned ga = grid_of(rows_a, cols_a), gb = grid_of(rows_b, cols_b);
   launch_kernel(amax_tensor_pair_kernel, dim3(ga + gb), dim3(256), 0, st, a, rows_a, cols_a, ld_a, cell_a, ga, b, rows_b, cols_b, ld_b, cell_b);

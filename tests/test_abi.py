@@ -19,15 +19,26 @@ def binding():
     return b
 
 
-def test_every_declared_symbol_is_exported(binding):
-    header = open(os.path.join(ROOT, "include", "nvfp4.h")).read()
+def _declared(header_name):
+    header = open(os.path.join(ROOT, "include", header_name)).read()
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
-    declared = set(re.findall(r"\b(nvfp4_[a-z0-9_]+)\s*\(", header))
+    return set(re.findall(r"\b(nvfp4_[a-z0-9_]+)\s*\(", header))
+
+
+def test_every_declared_symbol_is_exported(binding):
+    declared = _declared("nvfp4.h")
     assert {"nvfp4_quantize", "nvfp4_linear_fwd", "nvfp4_linear_bwd_dx", "nvfp4_linear_bwd_dw", "nvfp4_gemm",
-            "nvfp4_requantize_t"} <= declared
+            "nvfp4_requantize_t", "nvfp4_gemm_ex", "nvfp4_quantize_static"} <= declared
     for name in declared:
         assert hasattr(binding.lib, name), name
     assert declared == set(binding.EXPORTS)
+    # the measurement aids: the launch counter in the main library, the issue loop in a library of its own
+    aids = _declared("nvfp4_measure.h")
+    assert aids == set(binding.MEASURE_EXPORTS) == {"nvfp4_launch_count", "nvfp4_mma_issue_probe"}
+    assert hasattr(binding.lib, "nvfp4_launch_count") and not hasattr(binding.lib, "nvfp4_mma_issue_probe")
+    assert hasattr(binding.measure_lib(), "nvfp4_mma_issue_probe")
+    # headers of the include directory are exactly these two
+    assert sorted(os.listdir(os.path.join(ROOT, "include"))) == ["nvfp4.h", "nvfp4_measure.h"]
 
 
 def test_size_helpers(binding):
@@ -65,6 +76,18 @@ def test_bad_arguments_are_refused_on_the_host(binding):
     assert L.nvfp4_gemm(ctypes.byref(a), ctypes.byref(c), 0x5000, 1, 4, 0, None, None, 0, None) == 2  # K mismatch
     lin = b.COperand(0x1000, 0x2000, 0x3000, 4, 32, 0, 0)
     assert L.nvfp4_gemm(ctypes.byref(a), ctypes.byref(lin), 0x5000, 1, 4, 0, None, None, 0, None) == 4  # linear scales
+    a2 = b.COperand(0x1000, 0x2000, 0x3000, 4, 32, 0, 1)
+    bad_variant = b.CGemmOpts(7, 0, 0)
+    assert L.nvfp4_gemm_ex(ctypes.byref(a), ctypes.byref(a2), 0x5000, 1, 4, 0, None, ctypes.byref(bad_variant), None, 0, None) == 4
+    neg_limit = b.CGemmOpts(0, 0, -5)
+    assert L.nvfp4_gemm_ex(ctypes.byref(a), ctypes.byref(a2), 0x5000, 1, 4, 0, None, ctypes.byref(neg_limit), None, 0, None) == 4
+    g2 = b.COperand(0x1000, 0x2000, 0x3000, 4, 32, 2, 1)
+    pair = b.CGemmOpts(b.GEMM_PAIR256, 0, 0)
+    assert L.nvfp4_gemm_ex(ctypes.byref(g2), ctypes.byref(g2), 0x5000, 1, 4, 0, None, ctypes.byref(pair), None, 0, None) == 4
+    # a side stream without its events is refused
+    cfg = b.CLayerCfg(0, (ctypes.c_int32 * 6)(0, 0, 1, 1, 1, 1), 0, 0, 0, 1, 0, None, None, None, None, 0, 0, 0, 0x7000, None, None, None)
+    sv = b.CSaved(a, a2, 0x100, 0x200, 32, 32, 4, 32, 4, None, None)
+    assert L.nvfp4_linear_fwd(0x100, 32, 0x200, 32, 4, 32, 4, ctypes.byref(cfg), 0x300, 8, ctypes.byref(sv), 0x400, 1 << 20, None) == 1
 
 
 def test_bad_arguments_of_the_calibration_and_oscireset_entry_points(binding):

@@ -7,7 +7,7 @@ import torch
 
 from oracle import nvfp4_oracle as orc
 from paper_2510_27527_b200 import synth
-from tests.gpu_util import assert_operand_equal, to_dev_bf16
+from tests.gpu_util import assert_operand_equal, check_sampled, to_dev_bf16
 
 pytestmark = pytest.mark.gpu
 
@@ -16,34 +16,6 @@ def B():
     from paper_2510_27527_b200 import binding
 
     return binding
-
-
-def sample_positions(M, N, rng, n_scatter=4096, n_tiles=4, tile=32):
-    ms = [rng.integers(0, M, n_scatter)]
-    ns = [rng.integers(0, N, n_scatter)]
-    for _ in range(n_tiles):
-        m0, n0 = rng.integers(0, M - tile + 1), rng.integers(0, N - tile + 1)
-        mm, nn = np.meshgrid(np.arange(m0, m0 + tile), np.arange(n0, n0 + tile), indexing="ij")
-        ms.append(mm.ravel())
-        ns.append(nn.ravel())
-    # always include the corners and the last row / column
-    ms.append(np.array([0, 0, M - 1, M - 1]))
-    ns.append(np.array([0, N - 1, 0, N - 1]))
-    return np.concatenate(ms).astype(np.int64), np.concatenate(ns).astype(np.int64)
-
-
-def check_sampled(got: torch.Tensor, A64, B64, rng, bf16_out, name):
-    M, N = got.shape
-    ms, ns = sample_positions(M, N, rng)
-    want, absdot = orc.gemm_tn_samples(A64, B64, ms, ns)
-    g = got[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].float().cpu().numpy().astype(np.float64)
-    tol = 1e-3 * absdot  # |err| <= 1e-3 * sum_k |a_k b_k| elementwise
-    if bf16_out:
-        tol = tol + np.abs(want) * 2.0 ** -8  # one BF16 rounding of the result
-    bad = np.abs(g - want) > tol + 1e-300
-    assert not bad.any(), (name, int(bad.sum()), float(np.abs(g - want).max()))
-    rel = np.linalg.norm(g - want) / np.linalg.norm(want)
-    assert rel <= (4e-3 if bf16_out else 1e-3), (name, rel)
 
 
 @pytest.mark.parametrize("gs_mode", [0, 2])

@@ -59,3 +59,56 @@ def test_single_process_is_the_identity():
     assert multi.world_info() == (0, 1)
     assert multi.max_over_ranks(0.5) == 0.5
     assert multi.job_throughput(10.0, 0.5) == 20.0
+
+
+_RANK_SCRIPT = """
+import json, os, sys
+sys.path.insert(0, {root!r})
+import torch.distributed as dist
+from paper_2510_27527_b200 import multi
+dist.init_process_group("gloo")
+rank, world = multi.world_info()
+assert world == int(os.environ["WORLD_SIZE"]) == int(sys.argv[sys.argv.index("--gpus") + 1])
+slowest = multi.max_over_ranks(0.010 * (rank + 1))
+thr = multi.job_throughput(100.0, 0.010 * (rank + 1))
+dist.barrier()
+if rank == 0:
+    open(sys.argv[sys.argv.index("--out") + 1], "w").write(json.dumps({{"world": world, "slowest": slowest, "thr": thr}}))
+dist.destroy_process_group()
+"""
+
+
+def test_launch_ranks_starts_one_process_per_rank(tmp_path):
+    """`bench.py --gpus N` without torchrun starts its ranks through multi.launch_ranks: here with two gloo ranks on CPU."""
+    import json
+
+    sys.path.insert(0, ROOT)
+    from paper_2510_27527_b200 import multi
+
+    script = tmp_path / "rank_script.py"
+    script.write_text(_RANK_SCRIPT.format(root=ROOT))
+    out = tmp_path / "out.json"
+    rc = multi.launch_ranks(2, str(script), ["--gpus", "2", "--out", str(out)], timeout=300)
+    assert rc == 0
+    got = json.loads(out.read_text())
+    assert got["world"] == 2
+    assert got["slowest"] == pytest.approx(0.020)
+    assert got["thr"] == pytest.approx(2 * 100.0 / 0.020)
+
+
+def test_bench_parses_gpus_and_would_spawn(monkeypatch):
+    """bench.py hands `--gpus N > 1` to launch_ranks when it was not started by torchrun (no WORLD_SIZE in the environment)."""
+    import importlib
+
+    sys.path.insert(0, ROOT)
+    bench = importlib.import_module("bench")
+    from paper_2510_27527_b200 import multi
+
+    calls = []
+    monkeypatch.setattr(multi, "launch_ranks", lambda n, script, argv, timeout=None: calls.append((n, script, list(argv))) or 0)
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4", "--steps", "2"])
+    with pytest.raises(SystemExit) as e:
+        bench.main()
+    assert e.value.code == 0
+    assert calls == [(4, os.path.join(ROOT, "bench.py"), ["--gpus", "4", "--steps", "2"])]

@@ -5,7 +5,9 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import nvfp4_oracle as orc
 from paper_2510_27527_b200 import synth
+from tests.gpu_util import assert_operand_equal
 
 pytestmark = pytest.mark.gpu
 
@@ -29,6 +31,9 @@ def test_static_scratch_quantize_matches_workspace_quantize_twice_in_a_row():
                 ref = b.nvfp4_quantize(d, axis, rounding, seed, 3, mode)
                 got = b.nvfp4_quantize_static(d, axis, rounding, seed, 3, mode)  # consecutive calls share the cells
                 assert same(got, ref), (mode, axis, rounding)
+    # and against the oracle itself, not only against the sibling entry point
+    want = orc.quantize(x1, orc.AXIS_ROW, orc.SR, orc.GS_ROW, 78, 3)
+    assert_operand_equal(b.nvfp4_quantize_static(d1, b.AXIS_ROW, b.ROUND_SR, 78, 3, b.GS_ROW), want, "static scratch, ROW mode, SR")
 
 
 def test_static_scratch_capacity_is_enforced_before_any_launch():
