@@ -30,7 +30,7 @@ def _stale(lib, sources) -> bool:
 def _compile(lib, sources, verbose):
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = lib + f".{os.getpid()}.tmp"
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + [os.path.join(CSRC, f) for f in sources] + ["-o", tmp]
+    cmd = [nvcc] + NVCC_FLAGS + os.environ.get("NVFP4_NVCC_EXTRA", "").split() + (["-Xptxas", "-v"] if verbose else []) + [os.path.join(CSRC, f) for f in sources] + ["-o", tmp]
     subprocess.check_call(cmd)
     os.replace(tmp, lib)
 

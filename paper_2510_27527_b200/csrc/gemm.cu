@@ -99,6 +99,24 @@ __device__ __forceinline__ void add_existing(const Params& p, int64_t m, int64_t
   }
 }
 
+// The columns of a chunk that sticks out past N (values final: scaled, accumulated): plain element stores, nothing beyond
+// column N - 1 is touched. The bulk tensor store is kept for whole chunks only: its clipping at the edge of C was seen to
+// overwrite the row's padding up to the next 16-byte boundary.
+template <int W>
+__device__ __forceinline__ void store_ragged(const Params& p, int64_t m, int64_t n0, const float (&o)[W]) {
+  if (p.c_is_f32) {
+    float* cp = reinterpret_cast<float*>(p.C) + m * p.ldc + n0;
+#pragma unroll
+    for (int j = 0; j < W; ++j)
+      if (n0 + j < p.N) cp[j] = o[j];
+  } else {
+    __nv_bfloat16* cp = reinterpret_cast<__nv_bfloat16*>(p.C) + m * p.ldc + n0;
+#pragma unroll
+    for (int j = 0; j < W; ++j)
+      if (n0 + j < p.N) cp[j] = __float2bfloat16_rn(o[j]);
+  }
+}
+
 // One output row, 32 consecutive columns starting at n0 (m < M and n0 < N are the caller's business): add the old C when
 // accumulating, convert, store.
 __device__ __forceinline__ void store_row_chunk(const Params& p, int64_t m, int64_t n0, float (&o)[32]) {
@@ -360,6 +378,10 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                   if (n0 + j < p.N) o[j] += reinterpret_cast<const float*>(p.C)[m * p.ldc + n0 + j];
               }
             }
+            if (n0 + 32 > p.N) {  // ragged last chunk of the row
+              if (m < p.M) store_ragged<32>(p, m, n0, o);
+              continue;
+            }
             const uint32_t buf = my_stage;
             if (lane == 0) bulk_wait_read<0>();  // the previous store from this buffer has read it
             __syncwarp();
@@ -415,6 +437,10 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 for (int j = 0; j < 64; ++j)
                   if (n0 + j < p.N) o[j] += __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.C)[m * p.ldc + n0 + j]);
               }
+            }
+            if (n0 + 64 > p.N) {  // ragged last chunk of the row
+              if (m < p.M) store_ragged<64>(p, m, n0, o);
+              continue;
             }
             const uint32_t buf = my_stage;
             if (lane == 0) bulk_wait_read<0>();
@@ -708,7 +734,17 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
 #pragma unroll
           for (int c0 = 0; c0 < 128; c0 += 32) {
             const int64_t n0 = (int64_t)nt * BN + c0;
-            if (n0 < p.N) {
+            if (n0 < p.N && n0 + 32 > p.N) {  // ragged last chunk of the row
+              if (m < p.M) {
+                float o[32];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                  o[2 * j] = acc[(c0 >> 1) + j].x;
+                  o[2 * j + 1] = acc[(c0 >> 1) + j].y;
+                }
+                store_ragged<32>(p, m, n0, o);
+              }
+            } else if (n0 < p.N) {
               if (lane == 0) bulk_wait_read<0>();  // the previous store from this buffer has read it
               __syncwarp();
 #pragma unroll
@@ -731,7 +767,17 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
 #pragma unroll
           for (int c0 = 0; c0 < 128; c0 += 64) {
             const int64_t n0 = (int64_t)nt * BN + c0;
-            if (n0 < p.N) {
+            if (n0 < p.N && n0 + 64 > p.N) {  // ragged last chunk of the row
+              if (m < p.M) {
+                float o[64];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  o[2 * j] = acc[(c0 >> 1) + j].x;
+                  o[2 * j + 1] = acc[(c0 >> 1) + j].y;
+                }
+                store_ragged<64>(p, m, n0, o);
+              }
+            } else if (n0 < p.N) {
               if (lane == 0) bulk_wait_read<0>();
               __syncwarp();
 #pragma unroll

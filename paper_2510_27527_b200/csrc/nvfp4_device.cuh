@@ -197,21 +197,19 @@ __device__ __forceinline__ void hadamard16_butterflies(float (&v)[16]) {
 // ---------------------------------------------------------------------------------------------------------
 // Stochastic rounding. For an element with 16-bit draw u the rule is
 //     round the magnitude up  iff  (u + 0.5) / 65536 < (a - q1) / (q2 - q1),   a = min(|y|, 6) in [q1, q2).
-// It is evaluated exactly with one integer add on the bits of a float z:
+// It is evaluated exactly with one integer multiply-add on the bits of a float z:
 //   * for a >= 1, z = a: the E2M1 cell of a is (bits >> 22) - 252 and the low 22 mantissa bits are the position inside
 //     the cell in units of 2^-22 of the cell width;
 //   * for a < 1 the cells [0, .5) and [.5, 1) are mapped onto [.5, .75) and [.75, 1) by z = 0.5 + a / 2, computed with
 //     round-up so that the low bits are ceil(position * 2^22) (an integer n is < x iff n < ceil(x); when the ceiling
 //     crosses into the next cell the true position was within 2^-24 of 1, where every draw rounds up);
 //     0.5 + a / 2 >= a exactly when a <= 1, so z = max(a, 0.5 + a / 2) picks the right branch;
-//   * adding r22 = 2^22 - 1 - ((2u + 1) << 5) = ((~u & 0xFFFF) << 6) | 0x1F carries into the cell index iff
-//     position > (2u + 1) << 5; adding -(252 << 22) as well leaves the magnitude index 0..7 in bits 22..24.
-__device__ __forceinline__ uint32_t e2m1_sr_bits(float y, uint32_t c) {
-  const float a = fminf(fabsf(y), 6.0f);
-  const float z = fmaxf(a, __fmaf_ru(a, 0.5f, 0.5f));
-  return __float_as_uint(z) + c;  // magnitude index in bits 22..24, nothing above
-}
-
+//   * adding r22 = 2^22 - 1 - ((2u + 1) << 5) = ((~u & 0xFFFF) << 6) | 0x1F to the bits carries into the cell index iff
+//     position > (2u + 1) << 5, and adding -(252 << 22) as well leaves the magnitude index 0..7 in bits 22..24 with
+//     nothing above. Both additions and a shift by 6 are one multiply-add modulo 2^32:
+//         v = bits * 64 + c6,   c6 = ((~u & 0xFFFF) << 12) | 0x7C0 | (4 << 28)      (-252 = 4 modulo 16)
+//     has the magnitude index in bits 28..30 and bit 31 clear, i.e. the code's magnitude already sits next to where the
+//     sign bit of y lives: one bit-select gives the nibble in the top four bits (e2m1x8_sr below).
 // Round-to-nearest (ties to the even code, saturating) of 8 scaled values, packed low nibble first.
 __device__ __forceinline__ uint32_t e2m1x8_rtn(const float (&y)[8]) {
   uint32_t out;
@@ -229,20 +227,27 @@ __device__ __forceinline__ uint32_t e2m1x8_rtn(const float (&y)[8]) {
 }
 
 // Stochastic rounding of 8 scaled values with the draws packed in w (two 16-bit draws per word), packed low nibble
-// first. The sign bits are those of y.
+// first. The sign bits are those of y. Elements are taken last to first: a funnel shift moves each code's four top bits
+// in below the ones already collected, so that element 0 ends in the lowest nibble.
 __device__ __forceinline__ uint32_t e2m1x8_sr(const float (&y)[8], const uint4& w) {
   const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
   uint32_t out = 0;
 #pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    const uint32_t nw = ~ww[e >> 1];
-    // ((~u & 0xFFFF) << 6) | 0x1F, minus 252 << 22 (the two fields do not overlap)
-    const uint32_t c = (((e & 1) ? (nw >> 10) : (nw << 6)) & 0x3FFFC0u) | 0xC100001Fu;
-    const uint32_t v = e2m1_sr_bits(y[e], c);
-    const int sh = 22 - 4 * e;
-    const uint32_t mag = (sh >= 0 ? (v >> sh) : (v << -sh)) & (7u << (4 * e));
-    const int ss = 28 - 4 * e;  // sign bit 31 -> bit 4e + 3
-    out |= mag | ((__float_as_uint(y[e]) >> ss) & (8u << (4 * e)));
+  for (int e = 7; e >= 0; --e) {
+    // The draw u of element e (the even element is the low half of its word), then c6 = ((0xFFFF - u) << 12) | 0x400007C0
+    // = 0x4FFFF7C0 - u * 4096. Multiply-adds are written as such on purpose: the logic / shift / min-max pipe is the one
+    // this code saturates (half the rate of the multiply-add pipe), so shifts and adds that can be a multiply-add are one.
+    uint32_t u, c6, v;
+    if (e & 1)
+      asm("mul.hi.u32 %0, %1, 65536;" : "=r"(u) : "r"(ww[e >> 1]));
+    else
+      u = ww[e >> 1] & 0xFFFFu;
+    asm("mad.lo.u32 %0, %1, 0xFFFFF000, 0x4FFFF7C0;" : "=r"(c6) : "r"(u));
+    const float a = fminf(fabsf(y[e]), 6.0f);
+    const float z = fmaxf(a, __fmaf_ru(a, 0.5f, 0.5f));
+    asm("mad.lo.u32 %0, %1, 64, %2;" : "=r"(v) : "r"(__float_as_uint(z)), "r"(c6));
+    // code in bits 28..31 (v has the magnitude index in 28..30 and bit 31 clear); the funnel shift takes those four bits
+    out = __funnelshift_l((__float_as_uint(y[e]) & 0x80000000u) | (v & 0x7FFFFFFFu), out, 4);
   }
   return out;
 }

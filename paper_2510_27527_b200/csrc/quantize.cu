@@ -565,6 +565,170 @@ quantize_rows_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, 
 }
 
 // =========================================================================================================
+// Row-axis quantize from BF16, four ADJACENT inner blocks per thread (64 consecutive k of one operand row).
+// What a thread does once per inner block in the kernel above (row / block index from the flat index, address
+// arithmetic, the shuffles that assemble a word of scale bytes and reduce the 128-wide group maximum) it does here once per
+// four blocks: the four scale bytes of a thread are one aligned 32-bit word of either scale layout, its codes are 32
+// contiguous bytes, a 128-wide outer group is two neighbouring lanes, and the sign bits of the random Hadamard
+// transformation for all four blocks come from one generator call. That bookkeeping was about 40 % of the instructions of
+// the stochastic-rounding quantizers. Loads are 32 bytes per lane at a 128-byte stride (every sector is used in full; the
+// four loads of a warp cover a contiguous 4 KB).
+//   RMODE  0 round to nearest, 1 stochastic rounding, 2 stochastic rounding with the block scale rounded up.
+// No column list (OutControl's compaction keeps the kernel above).
+// =========================================================================================================
+template <int GS, int RMODE, bool TILED, bool RHT>
+__global__ void __launch_bounds__(256, 3)
+quantize_rows4_kernel(const uint16_t* __restrict__ src, int64_t rows, int64_t K, int64_t ld, uint64_t seed, uint32_t stream_id,
+                      const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
+                      float* __restrict__ gscale, uint32_t div_mul, uint32_t div_shift, int wide_loads, uint32_t rht_stream,
+                      const __grid_constant__ PhiloxKeys pk) {
+  pdl_prologue();
+  constexpr bool SR = RMODE != 0;
+  const uint32_t K32 = (uint32_t)K;
+  const uint32_t Kp = (K32 + 127u) & ~127u;
+  const uint32_t K16 = (K32 + 15u) & ~15u;
+  const uint32_t nu = Kp >> 6;  // units (four inner blocks) per operand row: even, as rows are padded to 128
+  const int64_t total = rows * (int64_t)nu;
+  const int64_t unit = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  const bool full = K32 == Kp && (int64_t)blockIdx.x * 256 + 256 <= total;  // CTA-uniform: every block exists and is whole
+
+  auto body = [&](auto full_tag) {
+    constexpr bool FULL = decltype(full_tag)::value;
+    const bool active = FULL || unit < total;
+    uint32_t r = 0, q = 0;
+    if (active) {
+      if (div_mul) {
+        const uint32_t n = (uint32_t)unit, t = __umulhi(div_mul, n);
+        r = (t + ((n - t) >> 1)) >> div_shift;
+        q = n - r * nu;
+      } else if (div_shift != 0xFFFFFFFFu) {
+        r = (uint32_t)unit >> div_shift;
+        q = (uint32_t)unit & (nu - 1u);
+      } else {
+        r = (uint32_t)(unit / nu);
+        q = (uint32_t)(unit - (int64_t)r * nu);
+      }
+    }
+    const uint32_t k0 = q << 6;
+    uint32_t w[4][8];
+    {
+      const uint16_t* p = src + (size_t)r * (uint32_t)ld + k0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t k = k0 + 16u * j;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) w[j][i] = 0;
+        if (FULL || (active && k + 16u <= K32)) {
+          if (wide_loads) {
+            asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                         : "=r"(w[j][0]), "=r"(w[j][1]), "=r"(w[j][2]), "=r"(w[j][3]), "=r"(w[j][4]), "=r"(w[j][5]),
+                           "=r"(w[j][6]), "=r"(w[j][7])
+                         : "l"(p + 16 * j));
+          } else {
+            const uint4 v0 = *reinterpret_cast<const uint4*>(p + 16 * j);
+            const uint4 v1 = *reinterpret_cast<const uint4*>(p + 16 * j + 8);
+            w[j][0] = v0.x; w[j][1] = v0.y; w[j][2] = v0.z; w[j][3] = v0.w;
+            w[j][4] = v1.x; w[j][5] = v1.y; w[j][6] = v1.z; w[j][7] = v1.w;
+          }
+        } else if (active && k < K32) {
+          for (int i = 0; i < 16; ++i)
+            if (k + i < K32) w[j][i >> 1] |= (uint32_t)p[16 * j + i] << (16 * (i & 1));
+        }
+      }
+    }
+    // the 64 sign bits of this thread's k range (one half of a 128-group's generator block); none past K rounded up to 16
+    uint32_t sgn_lo = 0, sgn_hi = 0;
+    if (RHT) {
+      const uint4 sw = rht_sign_words(seed, rht_stream, (uint64_t)(k0 >> 7));
+      sgn_lo = (k0 & 64u) ? sw.z : sw.x;
+      sgn_hi = (k0 & 64u) ? sw.w : sw.y;
+    }
+
+    // block maxima (binary32 patterns of non-negative values: integer order = float order)
+    uint32_t amax_bits[4];
+    float xr[RHT ? 4 : 1][16];  // transformed values (RHT only)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      if (RHT) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          xr[RHT ? j : 0][2 * i] = bf16_lo(w[j][i]);
+          xr[RHT ? j : 0][2 * i + 1] = bf16_hi(w[j][i]);
+        }
+        const uint32_t s16 = ((j & 2) ? sgn_hi : sgn_lo) >> (16 * (j & 1));
+        rht_scale16(xr[RHT ? j : 0], (FULL || k0 + 16u * j < K16) ? (s16 & 0xFFFFu) : 0u);
+        hadamard16_butterflies(xr[RHT ? j : 0]);
+        float m = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(xr[RHT ? j : 0][i]));
+        amax_bits[j] = __float_as_uint(m);
+      } else {
+        uint32_t m2 = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) m2 = amax16x2(m2, w[j][i]);
+        amax_bits[j] = hmax_of_pair(bf16x2_abs_bits(m2)) << 16;
+      }
+    }
+
+    float Sg;
+    if (GS == kGsBlock128) {
+      uint32_t g = max(max(amax_bits[0], amax_bits[1]), max(amax_bits[2], amax_bits[3]));
+      g = max(g, __shfl_xor_sync(0xFFFFFFFFu, g, 1));  // the other half of the 128-wide group is the neighbouring lane
+      Sg = global_scale_from_amax(__uint_as_float(g));
+      if (active && (q & 1u) == 0) gscale[(size_t)r * (Kp >> 7) + (q >> 1)] = Sg;
+    } else if (GS == kGsRow) {
+      Sg = global_scale_from_amax(__uint_as_float(gs_cells[r]));
+      if (active && q == 0) gscale[r] = Sg;
+    } else {
+      Sg = global_scale_from_amax(__uint_as_float(gs_cells[0]));
+      if (unit == 0) gscale[0] = Sg;
+    }
+
+    const uint64_t idx8 = ((uint64_t)r * K16 + k0) >> 3;
+    uint32_t sf4 = 0;
+    uint32_t packed[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float rcp;
+      const uint32_t sb = block_scale(__uint_as_float(amax_bits[j]), Sg, rcp, RMODE == 2);
+      sf4 |= sb << (8 * j);
+      float x[16];
+      if (RHT) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) x[i] = xr[RHT ? j : 0][i];
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          x[2 * i] = bf16_lo(w[j][i]);
+          x[2 * i + 1] = bf16_hi(w[j][i]);
+        }
+      }
+      const uint2 c = quantize_block16<SR>(x, rcp, pk, stream_id, idx8 + 2 * j);
+      packed[2 * j] = c.x;
+      packed[2 * j + 1] = c.y;
+    }
+    if (active) {
+      uint4* cp = reinterpret_cast<uint4*>(codes + (size_t)r * (Kp >> 1) + (k0 >> 1));
+      cp[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+      cp[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+      const uint32_t nb = Kp >> 4;
+      size_t off;
+      if (TILED) {
+        const uint32_t tile = (r >> 7) * (((nb + 15u) & ~15u) >> 2) + q;  // 512-byte tiles, k fastest; this unit is one of them
+        off = (size_t)tile * 512u + ((r & 31u) * 16u + ((r >> 5) & 3u) * 4u);
+      } else {
+        off = (size_t)r * nb + (q << 2);
+      }
+      *reinterpret_cast<uint32_t*>(sf + off) = sf4;
+    }
+  };
+  if (full)
+    body(std::true_type{});
+  else
+    body(std::false_type{});
+}
+
+// =========================================================================================================
 // Transposing quantizers. Operand element (d, k) = source element (row k, column d).
 // Tile = 128 k x 64 d. Phase 1 stages the tile as FP32 in shared memory; phase 2 gives each thread one
 // (d, 16-k block); phase 3 writes the packed rows back in 16-byte pieces.
@@ -876,6 +1040,35 @@ static cudaError_t launch_rows_g(const QuantRowsArgs& a, cudaStream_t st) {
   return cudaGetLastError();
 }
 
+// The four-adjacent-blocks kernel (stochastic rounding without a column list).
+template <int GS, int RMODE, bool TILED>
+static cudaError_t launch_rows4(const QuantRowsArgs& a, cudaStream_t st) {
+  const int64_t Kp = (a.K + 127) & ~(int64_t)127;
+  const uint64_t d = (uint64_t)(Kp >> 6);  // units per row
+  const int64_t total = a.rows * (int64_t)d;
+  const unsigned grid = blocks_for(total, 256);
+  uint32_t div_mul = 0, div_shift = 0xFFFFFFFFu;
+  if (total + 256 < (int64_t)1 << 31) {
+    if ((d & (d - 1)) == 0) {
+      div_shift = 0;
+      while (((uint64_t)1 << div_shift) < d) ++div_shift;
+    } else {
+      uint32_t sft = 0;
+      while (((uint64_t)1 << sft) < d) ++sft;
+      div_mul = (uint32_t)((((uint64_t)1 << 32) * (((uint64_t)1 << sft) - d)) / d + 1);
+      div_shift = sft - 1;
+    }
+  }
+  const int wide_loads = ((reinterpret_cast<uintptr_t>(a.src) & 31u) == 0 && (a.ld & 15) == 0) ? 1 : 0;
+  if (a.rht_stream)
+    launch_kernel(quantize_rows4_kernel<GS, RMODE, TILED, true>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, a.seed, a.stream_id,
+                  a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, a.rht_stream, make_philox_keys(a.seed));
+  else
+    launch_kernel(quantize_rows4_kernel<GS, RMODE, TILED, false>, dim3(grid), dim3(256), 0, st, a.src, a.rows, a.K, a.ld, a.seed, a.stream_id,
+                  a.gs_cells, a.codes, a.sf, a.gscale, div_mul, div_shift, wide_loads, 0u, make_philox_keys(a.seed));
+  return cudaGetLastError();
+}
+
 template <int GS, bool SR>
 static cudaError_t launch_rows_t(const QuantRowsArgs& a, cudaStream_t st) {
   return a.sf_tiled ? launch_rows_g<GS, SR, true>(a, st) : launch_rows_g<GS, SR, false>(a, st);
@@ -883,6 +1076,12 @@ static cudaError_t launch_rows_t(const QuantRowsArgs& a, cudaStream_t st) {
 
 template <int GS>
 static cudaError_t launch_rows_r(const QuantRowsArgs& a, cudaStream_t st) {
+  // stochastic rounding is bound by instruction issue: the kernel with the least bookkeeping per block wins there; round to
+  // nearest is a streaming kernel and keeps the strided one (fully coalesced loads, four loads in flight per thread)
+  if (a.sr && !a.keep && (a.ld & 7) == 0 && (reinterpret_cast<uintptr_t>(a.src) & 15u) == 0 && a.K < ((int64_t)1 << 31)) {
+    if (a.sr == 2) return a.sf_tiled ? launch_rows4<GS, 2, true>(a, st) : launch_rows4<GS, 2, false>(a, st);
+    return a.sf_tiled ? launch_rows4<GS, 1, true>(a, st) : launch_rows4<GS, 1, false>(a, st);
+  }
   return a.sr ? launch_rows_t<GS, true>(a, st) : launch_rows_t<GS, false>(a, st);
 }
 

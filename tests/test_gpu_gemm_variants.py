@@ -29,16 +29,21 @@ def quantized_pair(M, N, K, gs_mode, seed=1):
     return a, bb
 
 
-def guarded_c(M, N, dtype, extra_rows=3, extra_cols=8):
-    """C [M, N] as a view of a larger poisoned buffer: extra_cols columns to the right of every row, extra_rows rows below."""
-    full = torch.full((M + extra_rows, N + extra_cols), POISON, dtype=dtype, device="cuda")
+def guarded_c(M, N, dtype, extra_rows=3):
+    """C [M, N] as a view of a larger poisoned buffer: at least 8 more columns to the right of every row (rows stay 16-byte
+    aligned), extra_rows rows below."""
+    ld = (N + 8 + 7) // 8 * 8
+    full = torch.full((M + extra_rows, ld), POISON, dtype=dtype, device="cuda")
     return full, full[:M, :N]
 
 
 def guard_intact(full, M, N):
     torch.cuda.synchronize()
     f = full.float()
-    return bool((f[:M, N:] == POISON).all()) and bool((f[M:, :] == POISON).all())
+    bad = torch.nonzero(f != POISON)
+    bad = bad[(bad[:, 0] >= M) | (bad[:, 1] >= N)]
+    assert bad.numel() == 0, f"{bad.shape[0]} elements outside C[{M}, {N}] were overwritten, first (row, column): {bad[:6].tolist()}"
+    return True
 
 
 @pytest.mark.parametrize("variant", [1, 2])
