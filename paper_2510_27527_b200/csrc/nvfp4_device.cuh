@@ -286,6 +286,30 @@ __device__ __forceinline__ void decode8(uint32_t word, uint32_t sf_byte, float s
   }
 }
 
+// Decode 8 packed E2M1 codes times one E4M3 scale into four packed FP16 pairs (element 2i in the low half of word i):
+// P * S_block, exact in FP16 (at most 7 significant bits, 2^-10 <= |value| <= 2688 or zero).
+__device__ __forceinline__ void decode8_h2(uint32_t word, uint32_t sf_byte, uint32_t (&out)[4]) {
+  uint32_t h[4];
+  asm("{\n"
+      ".reg .b8 b0, b1, b2, b3;\n"
+      "mov.b32 {b0, b1, b2, b3}, %4;\n"
+      "cvt.rn.f16x2.e2m1x2 %0, b0;\n"
+      "cvt.rn.f16x2.e2m1x2 %1, b1;\n"
+      "cvt.rn.f16x2.e2m1x2 %2, b2;\n"
+      "cvt.rn.f16x2.e2m1x2 %3, b3;\n"
+      "}"
+      : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3])
+      : "r"(word));
+  uint32_t s2;
+  asm("{.reg .b16 t; cvt.u16.u32 t, %1; cvt.rn.f16x2.e4m3x2 %0, t;}" : "=r"(s2) : "r"(sf_byte | (sf_byte << 8)));
+  const __half2 sb2 = *reinterpret_cast<__half2*>(&s2);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __half2 p = __hmul2(*reinterpret_cast<__half2*>(&h[i]), sb2);
+    out[i] = *reinterpret_cast<const uint32_t*>(&p);
+  }
+}
+
 // Scale, round and pack one 16-element inner block (two code words).
 template <bool SR>
 __device__ __forceinline__ uint2 quantize_block16(const float (&x)[16], float rcp, const PhiloxKeys& pk, uint32_t stream_id,

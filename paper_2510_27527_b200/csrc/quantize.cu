@@ -804,7 +804,7 @@ __global__ void __launch_bounds__(256) amax_cols_generic_kernel(TransposeSrc s, 
 //              gs_cells is then written, and codes / sf / gscale are not touched).
 template <int SRC, int GS, bool SR, bool TILED, bool RHT, bool AMAX_ONLY>
 __global__ void __launch_bounds__(256)
-quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t seed, uint32_t stream_id,
+quantize_transpose_generic_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t seed, uint32_t stream_id,
                           uint32_t* __restrict__ gs_cells, int tensor_closed_form, uint8_t* __restrict__ codes,
                           uint8_t* __restrict__ sf, float* __restrict__ gscale, uint32_t rht_stream, int sb_up,
                           const __grid_constant__ PhiloxKeys pk) {
@@ -991,6 +991,254 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
 }
 
 // =========================================================================================================
+// Transposing quantizers, fast path (no per-column remapping of the source). The 128 k x 64 d tile is staged as 16-bit
+// values: the BF16 source as it is (SRC = 0), or P * S_block of the forward operand as FP16 (SRC = 1, exact; the FP32
+// global scale of the source row is applied after the transposition, which is the same single rounding
+// x_hat = (P * S_block) * S_global). A tile row is 128 bytes; its 16-byte chunks are XOR-swizzled with the row number so that
+// both the row-wise 16-byte stores of the staging phase and the column-wise 4-byte reads of the quantizing phase are free of
+// bank conflicts. Each thread then owns TWO neighbouring operand rows (one 32-bit word per k holds both values) and one
+// 16-k block of each: half the shared-memory loads, packed maxima for BF16 sources, and all bookkeeping once per two blocks.
+// Codes and scale bytes are collected in shared memory and written as 16-byte / 4-byte pieces.
+//   RMODE  0 round to nearest, 1 stochastic rounding, 2 stochastic rounding with the block scale rounded up.
+// =========================================================================================================
+template <int SRC, int GS, int RMODE, bool TILED, bool RHT, bool AMAX_ONLY>
+__global__ void __launch_bounds__(256, 3)
+quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t seed, uint32_t stream_id,
+                          uint32_t* __restrict__ gs_cells, int tensor_closed_form, uint8_t* __restrict__ codes,
+                          uint8_t* __restrict__ sf, float* __restrict__ gscale, uint32_t rht_stream,
+                          const __grid_constant__ PhiloxKeys pk) {
+  pdl_prologue();
+  constexpr bool SR = RMODE != 0;
+  __shared__ __align__(16) uint32_t tile[128 * 32];
+  __shared__ float sg_row[128];
+  __shared__ float blk_amax[8][64];
+  __shared__ __align__(16) uint8_t out_codes[64][80];  // 64 code bytes per operand row (+16: spreads the rows over the banks)
+  __shared__ __align__(4) uint8_t out_sf[64][8];
+  // Sizes and indices are below 2^31 (checked by the launcher): 32-bit arithmetic throughout, 64 bits only where a byte
+  // offset is formed (one widening multiply each).
+  const uint32_t K = (uint32_t)rowsK;  // operand K
+  const uint32_t D32 = (uint32_t)D;
+  const uint32_t Kp = (K + 127u) & ~127u;
+  const uint32_t nb = Kp >> 4;
+  const uint32_t nbp4 = ((nb + 15u) & ~15u) >> 2;  // 512-byte scale tiles per 128-row tile of the output operand
+  const uint32_t k_base = blockIdx.x * 128u;
+  const uint32_t d_base = blockIdx.y * 64u;
+  const int tid = threadIdx.x;
+  uint4 sw = make_uint4(0, 0, 0, 0);  // the tile's 128 sign bits (k_base is a multiple of 128)
+  if (RHT) {
+    sw = rht_sign_words(seed, rht_stream, (uint64_t)blockIdx.x);
+    // rows past K rounded up to 16 are layout padding: no signs there, so that they stay +0 and encode as zero bytes
+    const int32_t live = (int32_t)((K + 15u) & ~15u) - (int32_t)k_base;
+    if (live < 128) {
+      const uint32_t n = live > 0 ? (uint32_t)live : 0u;
+      sw.x &= n >= 32 ? 0xFFFFFFFFu : (1u << n) - 1u;
+      sw.y &= n >= 64 ? 0xFFFFFFFFu : n > 32 ? (1u << (n - 32)) - 1u : 0u;
+      sw.z &= n >= 96 ? 0xFFFFFFFFu : n > 64 ? (1u << (n - 64)) - 1u : 0u;
+      sw.w &= n > 96 ? (1u << (n - 96)) - 1u : 0u;
+    }
+  }
+
+  // ---- phase 1: stage (zero outside the matrix) ------------------------------------------------------------
+  if (SRC == 0) {
+    // 128 rows x 8 chunks of 8 BF16, four chunks per thread, all loads first; the chunk that straddles D is read by element
+    uint4 v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t c = tid + 256 * i, kr = c >> 3, dc = (c & 7) << 3;
+      v[i] = make_uint4(0, 0, 0, 0);
+      if (k_base + kr < K) {
+        const uint16_t* src = s.bf16 + (size_t)(k_base + kr) * (uint32_t)s.ld + (d_base + dc);
+        if (d_base + dc + 8 <= D32) {
+          v[i] = *reinterpret_cast<const uint4*>(src);
+        } else if (d_base + dc < D32) {
+          uint32_t t[4] = {0, 0, 0, 0};
+          const int n = (int)(D32 - d_base - dc);
+          for (int e = 0; e < n; ++e) t[e >> 1] |= (uint32_t)src[e] << (16 * (e & 1));
+          v[i] = make_uint4(t[0], t[1], t[2], t[3]);
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int c = tid + 256 * i, kr = c >> 3, ch = c & 7;
+      *reinterpret_cast<uint4*>(&tile[kr * 32 + ((ch ^ (kr & 7)) << 2)]) = v[i];
+    }
+  } else {
+    // forward operand: 32 codes (16 bytes) and their two scale bytes per thread. A tile that sticks out past D still lies
+    // inside the operand's row (K is padded to 128 there, with zero codes and zero scales): the columns past D hold zeros
+    // that nobody stores.
+    const int kr = tid >> 1, half = tid & 1;
+    const uint32_t k = k_base + kr;
+    uint32_t h[4][4];
+    float sg = 0.0f;
+    if (k < K) {
+      const uint32_t in_Kp = ((uint32_t)s.in_K + 127u) & ~127u;
+      const uint32_t in_nb = in_Kp >> 4;
+      const uint4 c4 = *reinterpret_cast<const uint4*>(s.in_codes + (size_t)k * (in_Kp >> 1) + ((d_base >> 1) + half * 16));
+      const uint32_t kb = (d_base >> 4) + half * 2;
+      const size_t sfo = s.in_sf_tiled ? (size_t)((k >> 7) * (((in_nb + 15u) & ~15u) >> 2) + (kb >> 2)) * 512u +
+                                             ((k & 31u) * 16u + ((k >> 5) & 3u) * 4u + (kb & 3u))
+                                       : (size_t)k * in_nb + kb;
+      const uint32_t sf2 = *reinterpret_cast<const uint16_t*>(s.in_sf + sfo);
+      sg = s.in_gs_mode == kGsTensor ? s.in_gscale[0]
+           : s.in_gs_mode == kGsRow  ? s.in_gscale[k]
+                                     : s.in_gscale[(size_t)k * (in_Kp >> 7) + (d_base >> 7)];
+      decode8_h2(c4.x, sf2 & 0xFFu, h[0]);
+      decode8_h2(c4.y, sf2 & 0xFFu, h[1]);
+      decode8_h2(c4.z, sf2 >> 8, h[2]);
+      decode8_h2(c4.w, sf2 >> 8, h[3]);
+    } else {
+#pragma unroll
+      for (int w = 0; w < 4; ++w)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) h[w][i] = 0u;
+    }
+    if (half == 0) sg_row[kr] = sg;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const int ch = half * 4 + w;
+      *reinterpret_cast<uint4*>(&tile[kr * 32 + ((ch ^ (kr & 7)) << 2)]) = make_uint4(h[w][0], h[w][1], h[w][2], h[w][3]);
+    }
+  }
+  __syncthreads();
+
+  // ---- phase 2: per thread two neighbouring operand rows (d, d + 1), one 16-k block of each ------------------
+  const int dp = tid & 31, kb = tid >> 5;
+  uint32_t hw[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) hw[i] = tile[(kb * 16 + i) * 32 + ((((dp >> 2) ^ (i & 7)) << 2) | (dp & 3))];  // row & 7 = i & 7
+  const uint32_t s16 = RHT ? ((rht_pick_word(sw, (uint32_t)kb >> 1) >> (16 * (kb & 1))) & 0xFFFFu) : 0u;
+  float xs[2][16];
+  float am[2];
+  if (SRC == 0 && !RHT) {
+    // block maxima of both rows at once on the packed pairs; the values are expanded further down, one row at a time
+    uint32_t m2 = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) m2 = amax16x2(m2, hw[i]);
+    m2 = bf16x2_abs_bits(m2);
+    am[0] = __uint_as_float(m2 << 16);
+    am[1] = __uint_as_float(m2 & 0xFFFF0000u);
+  } else {
+    const bool uniform_sg = SRC == 1 && s.in_gs_mode == kGsTensor;
+    const float sg_t = uniform_sg ? s.in_gscale[0] : 1.0f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      if (SRC == 0) {
+        xs[0][i] = bf16_lo(hw[i]);
+        xs[1][i] = bf16_hi(hw[i]);
+      } else {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hw[i]));
+        const float sgk = uniform_sg ? sg_t : sg_row[kb * 16 + i];
+        xs[0][i] = __fmul_rn(f.x, sgk);
+        xs[1][i] = __fmul_rn(f.y, sgk);
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      if (RHT) {
+        rht_scale16(xs[c], s16);
+        hadamard16_butterflies(xs[c]);
+      }
+      float m = 0.0f;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) m = fmaxf(m, fabsf(xs[c][i]));
+      am[c] = m;
+    }
+  }
+  const uint32_t d0 = d_base + 2 * dp;
+  // operand rows produced by source columns d0, d0 + 1 (identity unless the caller scatters rows, as OutControl's W-hat does)
+  uint32_t o[2];
+#pragma unroll
+  for (int c = 0; c < 2; ++c) o[c] = (d0 + c < D32 && s.out_rows) ? (uint32_t)s.out_rows[d0 + c] : d0 + c;
+  if (GS == kGsBlock128 || (AMAX_ONLY && GS == kGsRow)) {
+    blk_amax[kb][2 * dp] = am[0];
+    blk_amax[kb][2 * dp + 1] = am[1];
+  }
+  if (AMAX_ONLY) {
+    if (GS == kGsRow) {  // one cell per operand row
+      __syncthreads();
+      if (tid < 64 && d_base + tid < D32) {
+        float m = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) m = fmaxf(m, blk_amax[j][tid]);
+        const uint32_t oo = s.out_rows ? (uint32_t)s.out_rows[d_base + tid] : d_base + tid;
+        if (m > 0.0f) atomicMax(gs_cells + oo, __float_as_uint(m));
+      }
+    } else {
+      float m = fmaxf(am[0], am[1]);
+#pragma unroll
+      for (int q = 16; q; q >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, q));
+      if ((tid & 31) == 0) blk_amax[0][tid >> 5] = m;
+      __syncthreads();
+      if (tid == 0) {
+        for (int q = 1; q < 8; ++q) m = fmaxf(m, blk_amax[0][q]);
+        if (m > 0.0f) atomicMax(gs_cells, __float_as_uint(m));
+      }
+    }
+    return;
+  }
+  float Sg[2];
+  if (GS == kGsBlock128) {
+    __syncthreads();
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      float g = 0.0f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) g = fmaxf(g, blk_amax[j][2 * dp + c]);
+      Sg[c] = global_scale_from_amax(g);
+      if (d0 + c < D32 && kb == 0 && k_base < K) gscale[(size_t)o[c] * (Kp >> 7) + blockIdx.x] = Sg[c];
+    }
+  } else if (GS == kGsRow) {
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      Sg[c] = global_scale_from_amax(d0 + c < D32 ? __uint_as_float(gs_cells[o[c]]) : 0.0f);
+      if (d0 + c < D32 && kb == 0 && blockIdx.x == 0) gscale[o[c]] = Sg[c];
+    }
+  } else {
+    // (tensor_closed_form == 2: the cell carries nothing and may be uninitialised)
+    float amax = tensor_closed_form == 2 ? 0.0f : __uint_as_float(gs_cells[0]);
+    // TENSOR -> TENSOR re-quantization: the aligned tensor's maximum is float32(2688 * S_global) of the forward
+    // operand (its largest block has scale 448 and a magnitude-6 element); gs_cells[0] then only covers BF16 rows.
+    if (SRC == 1 && tensor_closed_form) amax = fmaxf(amax, __fmul_rn(2688.0f, s.in_gscale[0]));
+    if (s.closed_form_sg) amax = fmaxf(amax, __fmul_rn(2688.0f, s.closed_form_sg[0]));
+    Sg[0] = Sg[1] = global_scale_from_amax(amax);
+    if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) gscale[0] = Sg[0];
+  }
+  const uint32_t K16 = (K + 15u) & ~15u;
+  const uint32_t k0 = k_base + kb * 16u;
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    float rcp;
+    const uint32_t sb = block_scale(am[c], Sg[c], rcp, RMODE == 2);
+    if (SRC == 0 && !RHT) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) xs[c][i] = c ? bf16_hi(hw[i]) : bf16_lo(hw[i]);
+    }
+    const uint2 packed = quantize_block16<SR>(xs[c], rcp, pk, stream_id, ((uint64_t)o[c] * K16 + k0) >> 3);
+    *reinterpret_cast<uint2*>(&out_codes[2 * dp + c][kb * 8]) = packed;
+    out_sf[2 * dp + c][kb] = (uint8_t)sb;
+  }
+  __syncthreads();
+
+  // ---- phase 3: 64 rows x 64 code bytes, 16 bytes per thread; 64 rows x 8 scale bytes, 4 bytes per thread -----
+  {
+    const int row = tid >> 2, piece = tid & 3;
+    const uint32_t dd = d_base + row;
+    if (dd < D32) {
+      const uint32_t oo = s.out_rows ? (uint32_t)s.out_rows[dd] : dd;
+      *reinterpret_cast<uint4*>(codes + (size_t)oo * (Kp >> 1) + ((k_base >> 1) + piece * 16)) =
+          *reinterpret_cast<const uint4*>(&out_codes[row][piece * 16]);
+      if (piece < 2) {  // scale bytes of k blocks 4 * piece .. 4 * piece + 3 of this tile: one aligned word in either layout
+        const uint32_t b = (k_base >> 4) + 4 * piece;
+        const size_t off = TILED ? (size_t)((oo >> 7) * nbp4 + (b >> 2)) * 512u + ((oo & 31u) * 16u + ((oo >> 5) & 3u) * 4u)
+                                 : (size_t)oo * nb + b;
+        *reinterpret_cast<uint32_t*>(sf + off) = *reinterpret_cast<const uint32_t*>(&out_sf[row][4 * piece]);
+      }
+    }
+  }
+}
+
+// =========================================================================================================
 // Host-side launchers
 // =========================================================================================================
 static inline unsigned blocks_for(int64_t n, int per) { return (unsigned)((n + per - 1) / per); }
@@ -1154,16 +1402,31 @@ cudaError_t launch_quantize_rows(const QuantRowsArgs& a, cudaStream_t st) {
   return e;
 }
 
-template <int SRC, int GS, bool SR>
+// The fast kernel takes every source that needs no per-column choice between the forward operand and a BF16 matrix
+// (nvfp4_requantize_t with a row map is the one caller that does) and whose BF16 rows can be read in 16-byte pieces.
+static bool transpose_fast_path(const TransposeSrc& s, int from_codes) {
+  if (s.ld >= ((int64_t)1 << 31) || s.in_K >= ((int64_t)1 << 31)) return false;
+  if (from_codes) return s.row_map == nullptr;
+  return (s.ld & 7) == 0 && (reinterpret_cast<uintptr_t>(s.bf16) & 15u) == 0;
+}
+
+template <int SRC, int GS, int RMODE>
 static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
   const dim3 grid(blocks_for(a.rowsK, 128), blocks_for(a.D, 64));
-#define NVFP4_LAUNCH_TR(TILED_, RHT_)                                                                                              \
-  launch_kernel(quantize_transpose_kernel<SRC, GS, SR, TILED_, RHT_, false>, dim3(grid), dim3(256), 0, st, a.src, a.rowsK, a.D, a.seed, \
-                a.stream_id, a.gs_cells, a.tensor_closed_form, a.codes, a.sf, a.gscale, a.rht_stream, a.sr == 2, make_philox_keys(a.seed))
+  const bool fast = transpose_fast_path(a.src, SRC);
+#define NVFP4_LAUNCH_TR(TILED_, RHT_)                                                                                                  \
+  if (fast)                                                                                                                            \
+    launch_kernel(quantize_transpose_kernel<SRC, GS, RMODE, TILED_, RHT_, false>, dim3(grid), dim3(256), 0, st, a.src, a.rowsK, a.D,    \
+                  a.seed, a.stream_id, a.gs_cells, a.tensor_closed_form, a.codes, a.sf, a.gscale, a.rht_stream,                        \
+                  make_philox_keys(a.seed));                                                                                           \
+  else                                                                                                                                 \
+    launch_kernel(quantize_transpose_generic_kernel<SRC, GS, RMODE != 0, TILED_, RHT_, false>, dim3(grid), dim3(256), 0, st, a.src,     \
+                  a.rowsK, a.D, a.seed, a.stream_id, a.gs_cells, a.tensor_closed_form, a.codes, a.sf, a.gscale, a.rht_stream,          \
+                  RMODE == 2, make_philox_keys(a.seed))
   if (a.sf_tiled) {
-    if (a.rht_stream) NVFP4_LAUNCH_TR(true, true); else NVFP4_LAUNCH_TR(true, false);
+    if (a.rht_stream) { NVFP4_LAUNCH_TR(true, true); } else { NVFP4_LAUNCH_TR(true, false); }
   } else {
-    if (a.rht_stream) NVFP4_LAUNCH_TR(false, true); else NVFP4_LAUNCH_TR(false, false);
+    if (a.rht_stream) { NVFP4_LAUNCH_TR(false, true); } else { NVFP4_LAUNCH_TR(false, false); }
   }
 #undef NVFP4_LAUNCH_TR
   return cudaGetLastError();
@@ -1176,18 +1439,28 @@ template <int SRC, int GS>
 static cudaError_t launch_tr_amax_rht(const TransposeSrc& src, int64_t rowsK, int64_t D, uint64_t seed, uint32_t rht_stream,
                                       uint32_t* cells, cudaStream_t st) {
   const dim3 grid(blocks_for(rowsK, 128), blocks_for(D, 64));
-  if (rht_stream)
-    launch_kernel(quantize_transpose_kernel<SRC, GS, false, false, true, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
-                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), rht_stream, 0, make_philox_keys(seed));
-  else
-    launch_kernel(quantize_transpose_kernel<SRC, GS, false, false, false, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
-                  0, static_cast<uint8_t*>(nullptr), static_cast<uint8_t*>(nullptr), static_cast<float*>(nullptr), 0u, 0, make_philox_keys(seed));
+  uint8_t* const no_bytes = nullptr;
+  float* const no_floats = nullptr;
+  if (transpose_fast_path(src, SRC)) {
+    if (rht_stream)
+      launch_kernel(quantize_transpose_kernel<SRC, GS, 0, false, true, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells, 0,
+                    no_bytes, no_bytes, no_floats, rht_stream, make_philox_keys(seed));
+    else
+      launch_kernel(quantize_transpose_kernel<SRC, GS, 0, false, false, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells, 0,
+                    no_bytes, no_bytes, no_floats, 0u, make_philox_keys(seed));
+  } else if (rht_stream) {
+    launch_kernel(quantize_transpose_generic_kernel<SRC, GS, false, false, true, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
+                  0, no_bytes, no_bytes, no_floats, rht_stream, 0, make_philox_keys(seed));
+  } else {
+    launch_kernel(quantize_transpose_generic_kernel<SRC, GS, false, false, false, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells,
+                  0, no_bytes, no_bytes, no_floats, 0u, 0, make_philox_keys(seed));
+  }
   return cudaGetLastError();
 }
 
 template <int SRC, int GS>
 static cudaError_t launch_tr_r(const QuantTransposeArgs& a, cudaStream_t st) {
-  return a.sr ? launch_tr_t<SRC, GS, true>(a, st) : launch_tr_t<SRC, GS, false>(a, st);
+  return a.sr == 2 ? launch_tr_t<SRC, GS, 2>(a, st) : a.sr ? launch_tr_t<SRC, GS, 1>(a, st) : launch_tr_t<SRC, GS, 0>(a, st);
 }
 
 template <int SRC>
@@ -1291,6 +1564,7 @@ cudaError_t launch_amax_transpose_src(const TransposeSrc& s, int from_codes, int
 
 cudaError_t launch_quantize_transpose(const QuantTransposeArgs& a, cudaStream_t st) {
   if (a.rowsK == 0 || a.D == 0) return cudaSuccess;
+  if (a.rowsK >= ((int64_t)1 << 31) - 128 || a.D >= ((int64_t)1 << 31) - 128) return cudaErrorInvalidValue;
   return a.from_codes ? launch_tr_s<1>(a, st) : launch_tr_s<0>(a, st);
 }
 
