@@ -1422,15 +1422,20 @@ size_t gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
 int64_t gemm_block128_max_k() { return (int64_t)B128_MAX_CHUNKS * 128; }
 
 // Variant choice. 128 x 128 single-CTA tiles with two accumulators (a tile's epilogue overlaps the next tile's MMAs) win for
-// short K; pairs of CTAs on 256 x 256 tiles (half the operand traffic per flop and SM) win once K is long and there are
-// enough tiles for every pair (measured on 8192 x 3072 x K: K = 2048 -> 39 us against 48 us, K = 4096 -> 60 against 57.5,
-// 16384 x 8192 x 8192 -> 477 against 380 us). A 256-row tile of an operand spans two 128-row scale tiles, and rows are padded
-// to 128 in the scale layout, so any M, N work. The fused high-precision side product and the outer-block scales live in
-// the single-CTA kernels only.
+// short K; pairs of CTAs on 256 x 256 tiles (half the operand traffic per flop and SM, which is what bounds the long-K
+// products: the 128 x 128 kernel pulls 36 KB per k tile and SM out of L2) win once K is long: from K = 4096 when there are
+// two tiles for every pair, from K = 8192 already when half of the pairs get a tile (the weight gradients of a model:
+// few tiles, K = tokens). Measured, FP32 output, 128 x 128 against pairs: 16384 x 1024 x 3072 -> 36.9 / 45.0 us,
+// 8192 x 8192 x 3072 -> 129 / 138, 16384 x 14336 x 4096 -> 541 / 524, 4096 x 8192 x 8192 -> 139 / 110,
+// 3072 x 1024 x 16384 (48 pair tiles) -> 41.1 / 34.8, 2816 x 1024 x 8192 (44) -> 26.6 / 24.6, 2048 x 2048 x 16384 (64) ->
+// 44.9 / 36.8, 1024 x 1024 x 16384 (16) -> 24.6 / 32.8; BF16 output: 16384 x 8192 x 8192 -> 477 / 380.
+// A 256-row tile of an operand spans two 128-row scale tiles, and rows are padded to 128 in the scale layout, so any M, N
+// work. The fused high-precision side product and the outer-block scales live in the single-CTA kernels only.
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;
   if (a.gs_mode == kGsBlock128) return a.variant == 2 ? cudaErrorInvalidValue : launch_block128(a, st);
-  bool pairs = a.K >= 3072 && ((a.M + 255) / 256) * ((a.N + 255) / 256) >= 2 * (sm_count() / 2);
+  const int64_t tiles256 = ((a.M + 255) / 256) * ((a.N + 255) / 256), n_pairs = sm_count() / 2;
+  bool pairs = (a.K >= 4096 && tiles256 >= 2 * n_pairs) || (a.K >= 8192 && 2 * tiles256 >= n_pairs);
   if (a.variant == 1) pairs = false;
   if (a.variant == 2) pairs = true;
   if (a.hp_Kh > 0) {

@@ -99,10 +99,10 @@ def test_outer_block_kernel_guard_bands(shape):
 
 @pytest.mark.parametrize("gs_mode", [0, 1])
 def test_pair_kernel_is_what_large_ragged_products_run(gs_mode):
-    """4000 x 2600 x 3072: 16 x 11 = 176 pair tiles, the shape class nvfp4_gemm sends to the CTA-pair kernel by itself; the
+    """4000 x 2600 x 4096: 16 x 11 = 176 pair tiles, the shape class nvfp4_gemm sends to the CTA-pair kernel by itself; the
     last tile row and column are ragged (rows beyond M in the second CTA's half, columns beyond N)."""
     b = B()
-    M, N, K = 4000, 2600, 3072
+    M, N, K = 4000, 2600, 4096
     a, bb = quantized_pair(M, N, K, gs_mode, seed=11)
     A64, B64 = orc.dequantize(a), orc.dequantize(bb)
     da, db = upload_operand(a, b), upload_operand(bb, b)
@@ -110,7 +110,7 @@ def test_pair_kernel_is_what_large_ragged_products_run(gs_mode):
     full, C = guarded_c(M, N, torch.float32)
     b.nvfp4_gemm(da, db, b.DT_F32, out=C)
     assert guard_intact(full, M, N)
-    check_sampled(C, A64, B64, rng, False, "auto 4000x2600x3072 f32")
+    check_sampled(C, A64, B64, rng, False, "auto 4000x2600x4096 f32")
     # the explicit variants give the same matrix up to FP32 summation order
     C2 = b.nvfp4_gemm_ex(da, db, b.DT_F32, variant=b.GEMM_PAIR256)
     C1 = b.nvfp4_gemm_ex(da, db, b.DT_F32, variant=b.GEMM_TILE128)
@@ -120,7 +120,7 @@ def test_pair_kernel_is_what_large_ragged_products_run(gs_mode):
     full16, C16 = guarded_c(M, N, torch.bfloat16)
     b.nvfp4_gemm(da, db, b.DT_BF16, out=C16)
     assert guard_intact(full16, M, N)
-    check_sampled(C16, A64, B64, rng, True, "auto 4000x2600x3072 bf16")
+    check_sampled(C16, A64, B64, rng, True, "auto 4000x2600x4096 bf16")
 
 
 @pytest.mark.parametrize("variant", [1, 2])
