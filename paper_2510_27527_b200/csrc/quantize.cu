@@ -1239,6 +1239,201 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
 }
 
 // =========================================================================================================
+// Column-axis quantize from BF16 without a shared-memory transposition (Q5 of Sec. 2.3: the operand is dY^T, its blocks
+// run along the tokens). A lane owns FOUR neighbouring source columns (= operand rows) and 64 consecutive source rows
+// (= operand k). It reads 8 bytes per source row, so one warp instruction covers two source rows of 128 contiguous bytes
+// (lanes 0..15: rows k .. , lanes 16..31: rows k + 64 ..), and the 16 values of an inner block are the same half of 16 loaded
+// words: the transposition is the choice of that half. Per 16 source rows the lane quantizes four blocks (one per column)
+// and stores 8 code bytes to each of its four operand rows; the four scale bytes of an operand row (64 k) are one aligned
+// word of either scale layout. The two lanes that share a 128-wide outer group exchange their maxima with one shuffle;
+// BLOCK128 therefore walks its 64 rows twice (maxima, then codes; the second walk is served by L2). No barrier, no shared
+// memory, and the index arithmetic is paid once per 256 elements.
+//   RMODE  0 round to nearest, 1 stochastic rounding, 2 stochastic rounding with the block scale rounded up.
+// Preconditions (the launcher falls back to the staged kernel otherwise): D and ld multiples of 4, src 8-byte aligned,
+// identity row order, no Hadamard transformation.
+// =========================================================================================================
+__device__ __forceinline__ uint2 ld_nc_8(const uint16_t* p) {
+  uint2 v;
+  asm volatile("ld.global.nc.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+  return v;
+}
+
+template <int GS, int RMODE, bool TILED>
+__global__ void __launch_bounds__(128, 4)
+quantize_cols4_kernel(const uint16_t* __restrict__ src, uint32_t K, uint32_t D, uint32_t ld, uint32_t stream_id,
+                      const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
+                      float* __restrict__ gscale, const __grid_constant__ PhiloxKeys pk) {
+  pdl_prologue();
+  constexpr bool SR = RMODE != 0;
+  const uint32_t Kp = (K + 127u) & ~127u;
+  const uint32_t K16 = (K + 15u) & ~15u;
+  const uint32_t nb = Kp >> 4;
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  const uint32_t d0 = blockIdx.y * 64u + (lane & 15u) * 4u;                          // first of this lane's operand rows
+  const uint32_t k_start = blockIdx.x * 512u + warp * 128u + (lane >> 4) * 64u;      // first of its 64 k
+  const bool live = d0 < D && k_start < Kp;  // (all four rows exist or none: D is a multiple of 4)
+  const uint16_t* p = src + (size_t)k_start * ld + d0;
+
+  float Sg[4];
+  if (GS == kGsBlock128) {
+    uint32_t mx = 0, my = 0;
+    if (live) {
+#pragma unroll 16
+      for (uint32_t t = 0; t < 64; ++t) {
+        if (k_start + t < K) {
+          const uint2 v = ld_nc_8(p + (size_t)t * ld);
+          mx = amax16x2(mx, v.x);
+          my = amax16x2(my, v.y);
+        }
+      }
+    }
+    mx = amax16x2(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));  // the other half of the 128-wide group
+    my = amax16x2(my, __shfl_xor_sync(0xFFFFFFFFu, my, 16));
+    mx = bf16x2_abs_bits(mx);
+    my = bf16x2_abs_bits(my);
+    Sg[0] = global_scale_from_amax(__uint_as_float(mx << 16));
+    Sg[1] = global_scale_from_amax(__uint_as_float(mx & 0xFFFF0000u));
+    Sg[2] = global_scale_from_amax(__uint_as_float(my << 16));
+    Sg[3] = global_scale_from_amax(__uint_as_float(my & 0xFFFF0000u));
+    if (live && (lane >> 4) == 0) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) gscale[(size_t)(d0 + c) * (Kp >> 7) + (k_start >> 7)] = Sg[c];
+    }
+  } else if (GS == kGsRow) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      Sg[c] = global_scale_from_amax(live ? __uint_as_float(gs_cells[d0 + c]) : 0.0f);
+      if (live && k_start == 0) gscale[d0 + c] = Sg[c];
+    }
+  } else {
+    Sg[0] = Sg[1] = Sg[2] = Sg[3] = global_scale_from_amax(__uint_as_float(gs_cells[0]));
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) gscale[0] = Sg[0];
+  }
+  if (!live) return;
+
+  uint32_t sfw[4] = {0u, 0u, 0u, 0u};
+#pragma unroll 1
+  for (uint32_t tb = 0; tb < 4; ++tb) {
+    const uint32_t k0 = k_start + 16u * tb;
+    uint2 w[16];
+    if (k0 + 16u <= K) {
+#pragma unroll
+      for (int t = 0; t < 16; ++t) w[t] = ld_nc_8(p + (size_t)(16u * tb + t) * ld);
+    } else {
+#pragma unroll
+      for (int t = 0; t < 16; ++t) w[t] = k0 + t < K ? ld_nc_8(p + (size_t)(16u * tb + t) * ld) : make_uint2(0u, 0u);
+    }
+    uint32_t mx = 0, my = 0;
+#pragma unroll
+    for (int t = 0; t < 16; ++t) {
+      mx = amax16x2(mx, w[t].x);
+      my = amax16x2(my, w[t].y);
+    }
+    mx = bf16x2_abs_bits(mx);
+    my = bf16x2_abs_bits(my);
+    const float am[4] = {__uint_as_float(mx << 16), __uint_as_float(mx & 0xFFFF0000u), __uint_as_float(my << 16),
+                         __uint_as_float(my & 0xFFFF0000u)};
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float rcp;
+      const uint32_t sb = block_scale(am[c], Sg[c], rcp, RMODE == 2);
+      sfw[c] |= sb << (8u * tb);
+      float x[16];
+#pragma unroll
+      for (int t = 0; t < 16; ++t) {
+        const uint32_t word = c < 2 ? w[t].x : w[t].y;
+        x[t] = (c & 1) ? bf16_hi(word) : bf16_lo(word);
+      }
+      const uint2 packed = quantize_block16<SR>(x, rcp, pk, stream_id, ((uint64_t)(d0 + c) * K16 + k0) >> 3);
+      *reinterpret_cast<uint2*>(codes + (size_t)(d0 + c) * (Kp >> 1) + (k0 >> 1)) = packed;
+    }
+  }
+  const uint32_t b = k_start >> 4;  // first of this lane's four k blocks: a multiple of 4
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const uint32_t o = d0 + c;
+    const size_t off = TILED ? (size_t)((o >> 7) * (((nb + 15u) & ~15u) >> 2) + (b >> 2)) * 512u + ((o & 31u) * 16u + ((o >> 5) & 3u) * 4u)
+                             : (size_t)o * nb + b;
+    *reinterpret_cast<uint32_t*>(sf + off) = sfw[c];
+  }
+}
+
+// The same for the 1 x 128 outer block (BLOCK128), where the scale of a block depends on all 128 k of its group: a lane owns
+// TWO neighbouring source columns and keeps its 64 source rows in registers (one 32-bit word per row), so the data is read
+// once; the two lanes of a group exchange the group maximum with one shuffle. A warp instruction covers two source rows of
+// 64 contiguous bytes.
+template <int RMODE, bool TILED>
+__global__ void __launch_bounds__(128, 3)
+quantize_cols2_block128_kernel(const uint16_t* __restrict__ src, uint32_t K, uint32_t D, uint32_t ld, uint32_t stream_id,
+                               uint8_t* __restrict__ codes, uint8_t* __restrict__ sf, float* __restrict__ gscale,
+                               const __grid_constant__ PhiloxKeys pk) {
+  pdl_prologue();
+  constexpr bool SR = RMODE != 0;
+  const uint32_t Kp = (K + 127u) & ~127u;
+  const uint32_t K16 = (K + 15u) & ~15u;
+  const uint32_t nb = Kp >> 4;
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  const uint32_t d0 = blockIdx.y * 32u + (lane & 15u) * 2u;
+  const uint32_t k_start = blockIdx.x * 512u + warp * 128u + (lane >> 4) * 64u;
+  const bool live = d0 < D && k_start < Kp;  // (both rows exist or none: D is even)
+  const uint16_t* p = src + (size_t)k_start * ld + d0;
+
+  uint32_t w[64];
+  if (live && k_start + 64u <= K) {
+#pragma unroll
+    for (int t = 0; t < 64; ++t) asm volatile("ld.global.nc.L1::no_allocate.b32 %0, [%1];" : "=r"(w[t]) : "l"(p + (size_t)t * ld));
+  } else {
+#pragma unroll
+    for (int t = 0; t < 64; ++t) {
+      w[t] = 0u;
+      if (live && k_start + t < K) asm volatile("ld.global.nc.L1::no_allocate.b32 %0, [%1];" : "=r"(w[t]) : "l"(p + (size_t)t * ld));
+    }
+  }
+  uint32_t bm[4];  // packed block maxima (sign bits meaningless until masked)
+#pragma unroll
+  for (int tb = 0; tb < 4; ++tb) {
+    uint32_t m = 0;
+#pragma unroll
+    for (int t = 0; t < 16; ++t) m = amax16x2(m, w[16 * tb + t]);
+    bm[tb] = m;
+  }
+  uint32_t g = amax16x2(amax16x2(bm[0], bm[1]), amax16x2(bm[2], bm[3]));
+  g = bf16x2_abs_bits(amax16x2(g, __shfl_xor_sync(0xFFFFFFFFu, g, 16)));  // the other half of the 128-wide group
+  if (!live) return;
+  const float Sg[2] = {global_scale_from_amax(__uint_as_float(g << 16)), global_scale_from_amax(__uint_as_float(g & 0xFFFF0000u))};
+  if ((lane >> 4) == 0) {
+    gscale[(size_t)d0 * (Kp >> 7) + (k_start >> 7)] = Sg[0];
+    gscale[(size_t)(d0 + 1) * (Kp >> 7) + (k_start >> 7)] = Sg[1];
+  }
+  uint32_t sfw[2] = {0u, 0u};
+#pragma unroll
+  for (int tb = 0; tb < 4; ++tb) {
+    const uint32_t k0 = k_start + 16u * tb;
+    const uint32_t m = bf16x2_abs_bits(bm[tb]);
+    const float am[2] = {__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u)};
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      float rcp;
+      const uint32_t sb = block_scale(am[c], Sg[c], rcp, RMODE == 2);
+      sfw[c] |= sb << (8 * tb);
+      float x[16];
+#pragma unroll
+      for (int t = 0; t < 16; ++t) x[t] = c ? bf16_hi(w[16 * tb + t]) : bf16_lo(w[16 * tb + t]);
+      const uint2 packed = quantize_block16<SR>(x, rcp, pk, stream_id, ((uint64_t)(d0 + c) * K16 + k0) >> 3);
+      *reinterpret_cast<uint2*>(codes + (size_t)(d0 + c) * (Kp >> 1) + (k0 >> 1)) = packed;
+    }
+  }
+  const uint32_t b = k_start >> 4;
+#pragma unroll
+  for (int c = 0; c < 2; ++c) {
+    const uint32_t o = d0 + c;
+    const size_t off = TILED ? (size_t)((o >> 7) * (((nb + 15u) & ~15u) >> 2) + (b >> 2)) * 512u + ((o & 31u) * 16u + ((o >> 5) & 3u) * 4u)
+                             : (size_t)o * nb + b;
+    *reinterpret_cast<uint32_t*>(sf + off) = sfw[c];
+  }
+}
+
+// =========================================================================================================
 // Host-side launchers
 // =========================================================================================================
 static inline unsigned blocks_for(int64_t n, int per) { return (unsigned)((n + per - 1) / per); }
@@ -1410,10 +1605,39 @@ static bool transpose_fast_path(const TransposeSrc& s, int from_codes) {
   return (s.ld & 7) == 0 && (reinterpret_cast<uintptr_t>(s.bf16) & 15u) == 0;
 }
 
+// The register-transposing kernel takes a plain BF16 source whose rows can be read in 8-byte pieces: identity row order, no
+// Hadamard transformation, no closed-form maximum handed in by OutControl's two-pass W-hat.
+static bool cols4_path(const QuantTransposeArgs& a) {
+  const TransposeSrc& s = a.src;
+  return !a.rht_stream && !s.out_rows && !s.closed_form_sg && !a.tensor_closed_form && (a.D & 3) == 0 && (s.ld & 3) == 0 &&
+         (reinterpret_cast<uintptr_t>(s.bf16) & 7u) == 0 && s.ld < ((int64_t)1 << 31) && a.rowsK < ((int64_t)1 << 31) - 1024 &&
+         a.D < ((int64_t)1 << 31) - 64;
+}
+
 template <int SRC, int GS, int RMODE>
 static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
   const dim3 grid(blocks_for(a.rowsK, 128), blocks_for(a.D, 64));
   const bool fast = transpose_fast_path(a.src, SRC);
+  if (SRC == 0 && GS == kGsBlock128 && cols4_path(a)) {
+    const dim3 g2(blocks_for(a.rowsK, 512), blocks_for(a.D, 32));
+    if (a.sf_tiled)
+      launch_kernel(quantize_cols2_block128_kernel<RMODE, true>, g2, dim3(128), 0, st, a.src.bf16, (uint32_t)a.rowsK, (uint32_t)a.D,
+                    (uint32_t)a.src.ld, a.stream_id, a.codes, a.sf, a.gscale, make_philox_keys(a.seed));
+    else
+      launch_kernel(quantize_cols2_block128_kernel<RMODE, false>, g2, dim3(128), 0, st, a.src.bf16, (uint32_t)a.rowsK, (uint32_t)a.D,
+                    (uint32_t)a.src.ld, a.stream_id, a.codes, a.sf, a.gscale, make_philox_keys(a.seed));
+    return cudaGetLastError();
+  }
+  if (SRC == 0 && cols4_path(a)) {
+    const dim3 g4(blocks_for(a.rowsK, 512), blocks_for(a.D, 64));
+    if (a.sf_tiled)
+      launch_kernel(quantize_cols4_kernel<GS, RMODE, true>, g4, dim3(128), 0, st, a.src.bf16, (uint32_t)a.rowsK, (uint32_t)a.D,
+                    (uint32_t)a.src.ld, a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, make_philox_keys(a.seed));
+    else
+      launch_kernel(quantize_cols4_kernel<GS, RMODE, false>, g4, dim3(128), 0, st, a.src.bf16, (uint32_t)a.rowsK, (uint32_t)a.D,
+                    (uint32_t)a.src.ld, a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, make_philox_keys(a.seed));
+    return cudaGetLastError();
+  }
 #define NVFP4_LAUNCH_TR(TILED_, RHT_)                                                                                                  \
   if (fast)                                                                                                                            \
     launch_kernel(quantize_transpose_kernel<SRC, GS, RMODE, TILED_, RHT_, false>, dim3(grid), dim3(256), 0, st, a.src, a.rowsK, a.D,    \

@@ -40,7 +40,11 @@ def test_row_axis_bit_exact(shape, gs_mode, rounding):
         assert_operand_equal(out, ref, f"row {shape} gs{gs_mode} r{rounding} layout{layout}")
 
 
-@pytest.mark.parametrize("shape", [(16, 1), (48, 5), (144, 127), (272, 129), (512, 256), (1000, 72), (200, 333)])
+# (rows, columns) of the source; the operand is its transpose. Column counts that are multiples of 4 take the kernels that
+# transpose in registers (ragged token counts: 1000, 700, 1040 end inside a 16-block, a lane's 64 rows, a warp's 128 and a
+# CTA's 512; 68 and 132 columns leave most lanes of the last CTA without work); the others take the staged kernels.
+@pytest.mark.parametrize("shape", [(16, 1), (48, 5), (144, 127), (272, 129), (512, 256), (1000, 72), (200, 333), (700, 68),
+                                   (1040, 132), (64, 4)])
 @pytest.mark.parametrize("gs_mode", MODES)
 @pytest.mark.parametrize("rounding", [orc.RTN, orc.SR, orc.SR_SCALE_UP])
 def test_col_axis_bit_exact(shape, gs_mode, rounding):
@@ -50,9 +54,10 @@ def test_col_axis_bit_exact(shape, gs_mode, rounding):
     x = np.ascontiguousarray(full[:, : shape[1]])
     ref = orc.quantize(x, orc.AXIS_COL, rounding, gs_mode, seed=99, stream_id=5)
     src = to_dev_bf16(full)[:, : shape[1]]
-    out = b.alloc_operand(shape[1], shape[0], gs_mode, b.SF_TILED128x4, poison=True)
-    b.nvfp4_quantize(src, b.AXIS_COL, rounding, 99, 5, gs_mode, out=out)
-    assert_operand_equal(out, ref, f"col {shape} gs{gs_mode} r{rounding}")
+    for layout in (b.SF_TILED128x4, b.SF_LINEAR):
+        out = b.alloc_operand(shape[1], shape[0], gs_mode, layout, poison=True)
+        b.nvfp4_quantize(src, b.AXIS_COL, rounding, 99, 5, gs_mode, layout, out=out)
+        assert_operand_equal(out, ref, f"col {shape} gs{gs_mode} r{rounding} layout{layout}")
 
 
 @pytest.mark.parametrize("gs_mode", MODES)
