@@ -43,7 +43,19 @@ GS = {"tensor": 0, "row": 1, "block128": 2}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernels, from the ncu captures summarised under
 # profiles/ (keyed by kernel label, linear and tokens; a capture on a smaller tensor of the same kernel is scaled by the
 # number of elements, stated in the summary).
+# Stochastic-rounding quantizer calls in TENSOR mode = amax pre-pass + quantizer. Captured on 8192 x 8192 (67.1 M elements):
+# amax 138.0 MB, quantize_cols4 151.0 MB, quantize_rows4 157.3 MB per launch (profiles/quantizers_tensor_mode_8192x8192.txt,
+# profiles/quantizers_block128_8192x8192.txt); both kernels stream, so traffic scales with the element count.
+def _scaled_traffic(mb_per_67m, rows, cols):
+    return sum(mb_per_67m) * 1e6 * (rows * cols) / (8192.0 * 8192.0)
+
+
 PROFILED_TRAFFIC = {}
+for _name, _d, _c in (("qkv", 1024, 3072), ("gate", 1024, 2816), ("up", 1024, 2816)):
+    PROFILED_TRAFFIC[(f"quantize_cols_dY_SR(Q5) on {_name} {_d}->{_c}", "tensor")] = (
+        _scaled_traffic((138.0, 151.0), 16384, _c), "ncu on 8192x8192 (amax_tensor_bf16 + quantize_cols4), scaled by the element count")
+    PROFILED_TRAFFIC[(f"quantize_rows_dY_SR(Q3) on {_name} {_d}->{_c}", "tensor")] = (
+        _scaled_traffic((138.0, 157.3), 16384, _c), "ncu on 8192x8192 (amax_tensor_bf16 + quantize_rows4), scaled by the element count")
 
 
 def peaks():

@@ -196,7 +196,8 @@ nvfp4_status nvfp4_requantize_t(const nvfp4_operand* in, const void* hp_bf16, in
  *   accumulate != 0 adds to the existing C (read in c_dtype, summed in FP32).
  *   dev_status optional device int: set to NVFP4_ERR_TIMEOUT if a bounded wait inside the kernel ran out
  *            (the kernel then drains and exits; C is unspecified). Never written otherwise.
- *   workspace at least nvfp4_gemm_workspace_bytes(M, N, K) (split-K partials for small outputs).
+ *   workspace at least nvfp4_gemm_workspace_bytes(M, N, K) bytes; the present kernels need none (the query returns 0 for
+ *            every shape and workspace may then be NULL).
  *
  * nvfp4_gemm_ex is the same product with explicit control over what nvfp4_gemm chooses by itself (opts == NULL gives
  * nvfp4_gemm). It exists for tests and for measurements:

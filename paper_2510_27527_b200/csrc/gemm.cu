@@ -1072,12 +1072,12 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
 // =========================================================================================================
 // OutControl's high-precision weight-gradient columns (paper Sec. 4.2):  dW[:, A] = dY^T X[:, A], BF16 inputs, FP32
 // accumulation, on the tensor cores (tcgen05 kind::f16).  G[c, j] = sum_t dY[t, c] * X_out[t, j]  with
-// M = C, N = Kh (the compact outlier matrix, <= 256 columns), K = tokens. Both operands are stored with the
+// M = C, N = Kh (a slab of at most 256 columns of the compact outlier matrix), K = tokens. Both operands are stored with the
 // contraction index t as the SLOW index, i.e. "MN-major": a bulk-tensor box of 64 columns x 64 tokens lands in
 // shared memory as 64 rows of 128 bytes (8 swizzle atoms of 8 tokens), which is the MN-major 128-byte-swizzle
 // operand layout (leading byte offset = distance between 64-column boxes, stride byte offset = 1024).
 // Only C / 128 output tiles exist, so the token range is split over blockIdx.y; FP32 partial tiles go to a workspace
-// that hp_dw_reduce_kernel sums in a fixed order. One tile per CTA: no accumulator double buffering needed.
+// that dw_assemble_kernel sums in a fixed order. One tile per CTA: no accumulator double buffering needed.
 // =========================================================================================================
 constexpr int HPDW_STAGES = 4;
 constexpr int HPDW_THREADS = 192;
