@@ -324,6 +324,49 @@ nvfp4_status nvfp4_linear_bwd(const void* dY, int64_t lddy, const nvfp4_saved* s
                               void* stream);
 
 /* ---------------------------------------------------------------------------------------------------------
+ * Simulated FP6 x FP4 products (Sec. 5.4, paragraph "Precision Switching in Final Stage"):
+ *     Y = Q6_D(X) Q4_D(W^T),   dX = Q6_S(dY) Q4_S(W-hat),   dW = Q4_S(dY^T) Q6_S(X-hat)
+ * (D deterministic, S stochastic rounding; X-hat / W-hat the dequantized forward operands). The paper names FP6 and gives
+ * these three products, nothing more; the FP6 quantizer is this library's definition: element format E2M3 (sign, two
+ * exponent bits with bias 1, three mantissa bits: 32 magnitudes 0, 1/8, ..., 7/8, 1 ... 1.875, 2 ... 3.75, 4 ... 7.5), the
+ * FP4 quantizer's scale sequence (Sec. 2.2) with Q_max = 7.5 in place of 6 (Sg = amax / 3360, t = amax_b / Sg,
+ * s = t / 7.5, Sb = e4m3(s), d = Sg Sb, r = 1 / d, y = x r, each one binary32 operation, |y| clamped to 7.5), a per-tensor
+ * global scale (TENSOR mode only), NVFP4_ROUND_RTN (ties to the even code) or NVFP4_ROUND_SR with the FP4 quantizer's
+ * rule, 16-bit draws and Philox addressing (element idx = row * K16 + k of the operand).
+ *
+ * No tensor-core instruction multiplies E2M3 by E2M1 values under E4M3 block scales, and the paper simulates as well: the
+ * operands of these products are "dense" -- vals = P * S_block as BF16 [R, ld] (exact: at most 4 + 4 significant bits),
+ * ld = nvfp4_dense_ld(K) = K rounded up to 64, columns K .. ld - 1 zero, rows 16-byte aligned, plus one FP32 global scale.
+ *   nvfp4_fp6_quantize      Q6 along the rows of a BF16 matrix [rows, cols] (leading dimension ld, 16-byte aligned rows as for
+ *                           nvfp4_quantize: NVFP4_ERR_ALIGN otherwise; operand K = cols).
+ *   nvfp4_fp6_requantize_t  Q6 of the transposed aligned tensor float32(vals * gscale) of a dense operand `in` [R, K]:
+ *                           out is [K, R], its blocks run along R (Q6_S(X-hat) of the dW product).
+ *   nvfp4_expand_operand    an ordinary FP4 operand (TENSOR mode, either scale layout) as a dense operand: no arithmetic
+ *                           beyond P * S_block.
+ *   nvfp4_dense_gemm        C [A.R, B.R] = (A.gscale B.gscale) A.vals B.vals^T, A.K == B.K: BF16 tensor-core product with
+ *                           FP32 accumulation (the BF16 path of the 128 x 128 GEMM kernel), C BF16 or FP32 with leading
+ *                           dimension ldc, 16-byte aligned rows; dev_status as for nvfp4_gemm.
+ * workspace (the two quantizers): at least nvfp4_fp6_workspace_bytes() bytes, 16-byte aligned. All pointers device.
+ * Errors: NULL / SHAPE / ALIGN / ENUM (rounding, c_dtype, an operand that is not TENSOR mode) / WORKSPACE / ARCH; nothing is
+ * launched on an error.
+ * --------------------------------------------------------------------------------------------------------- */
+typedef struct {
+  void* vals;       /* BF16 [R, ld] */
+  float* gscale;    /* FP32 [1] */
+  int64_t R, K, ld; /* ld == nvfp4_dense_ld(K) */
+} nvfp4_dense_operand;
+int64_t nvfp4_dense_ld(int64_t K);
+size_t nvfp4_fp6_workspace_bytes(void);
+nvfp4_status nvfp4_fp6_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld, int32_t rounding, uint64_t seed,
+                                uint32_t stream_id, const nvfp4_dense_operand* out, void* workspace, size_t ws_bytes,
+                                void* stream);
+nvfp4_status nvfp4_fp6_requantize_t(const nvfp4_dense_operand* in, int32_t rounding, uint64_t seed, uint32_t stream_id,
+                                    const nvfp4_dense_operand* out, void* workspace, size_t ws_bytes, void* stream);
+nvfp4_status nvfp4_expand_operand(const nvfp4_operand* in, const nvfp4_dense_operand* out, void* stream);
+nvfp4_status nvfp4_dense_gemm(const nvfp4_dense_operand* A, const nvfp4_dense_operand* B, void* C, int32_t c_dtype, int64_t ldc,
+                              int32_t* dev_status, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------
  * OutControl calibration (Sec. 4.2, the paragraph defining the outlier index set A): the activation l2-norm of every
  * channel is accumulated over a calibration window; the channels with the largest accumulated value form A.
  *

@@ -51,6 +51,10 @@ class CGemmOpts(ctypes.Structure):
     _fields_ = [("variant", c_i32), ("starve_first_stage", c_i32), ("wait_limit_cycles", c_i64)]
 
 
+class CDenseOperand(ctypes.Structure):
+    _fields_ = [("vals", c_vp), ("gscale", c_vp), ("R", c_i64), ("K", c_i64), ("ld", c_i64)]
+
+
 class CSaved(ctypes.Structure):
     _fields_ = [("qx", COperand), ("qw", COperand), ("X", c_vp), ("W", c_vp), ("ldx", c_i64), ("ldw", c_i64),
                 ("N_tok", c_i64), ("D", c_i64), ("C", c_i64), ("X_out", c_vp), ("W_out", c_vp)]
@@ -97,6 +101,13 @@ EXPORTS = {
     "nvfp4_osci_sparse_workspace_bytes": (c_sz, [c_i64, c_i64, c_i32, c_i64, c_i32]),
     "nvfp4_osci_sparse_update": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i32, c_i64, c_vp, c_vp, c_vp, c_vp, c_vp, c_vp, c_sz,
                                          c_vp]),
+    "nvfp4_dense_ld": (c_i64, [c_i64]),
+    "nvfp4_fp6_workspace_bytes": (c_sz, []),
+    "nvfp4_fp6_quantize": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_u64, c_u32, ctypes.POINTER(CDenseOperand), c_vp, c_sz, c_vp]),
+    "nvfp4_fp6_requantize_t": (c_i32, [ctypes.POINTER(CDenseOperand), c_i32, c_u64, c_u32, ctypes.POINTER(CDenseOperand), c_vp, c_sz,
+                                       c_vp]),
+    "nvfp4_expand_operand": (c_i32, [ctypes.POINTER(COperand), ctypes.POINTER(CDenseOperand), c_vp]),
+    "nvfp4_dense_gemm": (c_i32, [ctypes.POINTER(CDenseOperand), ctypes.POINTER(CDenseOperand), c_vp, c_i32, c_i64, c_vp, c_vp]),
     "nvfp4_osci_sparse_suppress": (c_i32, [c_vp, c_i64, c_i64, c_i64, c_i32, c_i64, c_vp, c_vp, c_vp, ctypes.c_float, c_vp, c_vp,
                                            c_sz, c_vp]),
 }
@@ -581,3 +592,91 @@ def nvfp4_linear_bwd(dY: torch.Tensor, saved: Saved, cfg: LayerConfig, dX: torch
     _check(_lib.nvfp4_linear_bwd(_ptr(dY), dY.stride(0), ctypes.byref(cs), ctypes.byref(cc), _ptr(dX), dX.stride(0), _ptr(dW),
                                  dW.stride(0), _ptr(ws), ws.numel(), _stream_ptr()), "nvfp4_linear_bwd")
     return dX, dW
+
+
+# ------------------------------------------------------------------------------------------------------------
+# simulated FP6 x FP4 products (paper Sec. 5.4, "Precision Switching in Final Stage")
+# ------------------------------------------------------------------------------------------------------------
+@dataclass
+class DenseOperand:
+    """Device buffers of a dense simulation operand [R, K]: vals = P * S_block as BF16 [R, ld], one FP32 global scale."""
+
+    vals: torch.Tensor  # bfloat16 [R, ld]
+    gscale: torch.Tensor  # float32 [1]
+    R: int
+    K: int
+
+    @property
+    def ld(self) -> int:
+        return _lib.nvfp4_dense_ld(self.K)
+
+    def c(self) -> CDenseOperand:
+        return CDenseOperand(_ptr(self.vals), _ptr(self.gscale), self.R, self.K, self.ld)
+
+
+def alloc_dense(R: int, K: int, device="cuda", poison: bool = False) -> DenseOperand:
+    vals = torch.full((R, _lib.nvfp4_dense_ld(K)), 7.0 if poison else 0.0, dtype=torch.bfloat16, device=device)
+    return DenseOperand(vals, torch.zeros(1, dtype=torch.float32, device=device), R, K)
+
+
+def nvfp4_fp6_quantize(src: torch.Tensor, rounding: int = ROUND_RTN, seed: int = 0, stream_id: int = 0,
+                       out: DenseOperand | None = None, workspace: torch.Tensor | None = None) -> DenseOperand:
+    assert src.dtype == torch.bfloat16 and src.dim() == 2 and src.stride(1) == 1
+    rows, cols = src.shape
+    if out is None:
+        out = alloc_dense(rows, cols, src.device)
+    ws = workspace if workspace is not None else _workspace(_lib.nvfp4_fp6_workspace_bytes(), src.device)
+    co = out.c()
+    _check(_lib.nvfp4_fp6_quantize(_ptr(src), rows, cols, src.stride(0), rounding, seed, stream_id, ctypes.byref(co), _ptr(ws),
+                                   ws.numel(), _stream_ptr()), "nvfp4_fp6_quantize")
+    return out
+
+
+def nvfp4_fp6_requantize_t(inp: DenseOperand, rounding: int = ROUND_SR, seed: int = 0, stream_id: int = 0,
+                           out: DenseOperand | None = None, workspace: torch.Tensor | None = None) -> DenseOperand:
+    if out is None:
+        out = alloc_dense(inp.K, inp.R, inp.vals.device)
+    ws = workspace if workspace is not None else _workspace(_lib.nvfp4_fp6_workspace_bytes(), inp.vals.device)
+    ci, co = inp.c(), out.c()
+    _check(_lib.nvfp4_fp6_requantize_t(ctypes.byref(ci), rounding, seed, stream_id, ctypes.byref(co), _ptr(ws), ws.numel(),
+                                       _stream_ptr()), "nvfp4_fp6_requantize_t")
+    return out
+
+
+def nvfp4_expand_operand(inp: Operand, out: DenseOperand | None = None) -> DenseOperand:
+    if out is None:
+        out = alloc_dense(inp.R, inp.K, inp.codes.device)
+    ci, co = inp.c(), out.c()
+    _check(_lib.nvfp4_expand_operand(ctypes.byref(ci), ctypes.byref(co), _stream_ptr()), "nvfp4_expand_operand")
+    return out
+
+
+def nvfp4_dense_gemm(A: DenseOperand, B: DenseOperand, c_dtype: int = DT_F32, out: torch.Tensor | None = None,
+                     dev_status: torch.Tensor | None = None) -> torch.Tensor:
+    if out is None:
+        out = _matrix(A.R, B.R, c_dtype, A.vals.device)
+    ca, cb = A.c(), B.c()
+    _check(_lib.nvfp4_dense_gemm(ctypes.byref(ca), ctypes.byref(cb), _ptr(out), c_dtype, out.stride(0), _ptr(dev_status),
+                                 _stream_ptr()), "nvfp4_dense_gemm")
+    return out
+
+
+def fp6_linear_fwd(X: torch.Tensor, W: torch.Tensor, c_dtype: int = DT_BF16):
+    """Y = Q6_D(X) Q4_D(W^T): the calls of the simulated layer in order (sequencing only; every step is a library call).
+    Returns (Y, saved = (dense X-hat operand, FP4 operand of W))."""
+    qx6 = nvfp4_fp6_quantize(X, ROUND_RTN, 0, 1)
+    qw = nvfp4_quantize(W, AXIS_ROW, ROUND_RTN, 0, 2, GS_TENSOR)
+    Y = nvfp4_dense_gemm(qx6, nvfp4_expand_operand(qw), c_dtype)
+    return Y, (qx6, qw)
+
+
+def fp6_linear_bwd(dY: torch.Tensor, saved, seed: int = 0, dx_dtype: int = DT_BF16, dw_dtype: int = DT_F32):
+    """dX = Q6_S(dY) Q4_S(W-hat), dW = Q4_S(dY^T) Q6_S(X-hat). Returns (dX, dW, the four backward operands)."""
+    qx6, qw = saved
+    q3 = nvfp4_fp6_quantize(dY, ROUND_SR, seed, 3)
+    q4 = nvfp4_requantize_t(qw, ROUND_SR, seed, 4)
+    dX = nvfp4_dense_gemm(q3, nvfp4_expand_operand(q4), dx_dtype)
+    q5 = nvfp4_quantize(dY, AXIS_COL, ROUND_SR, seed, 5, GS_TENSOR)
+    q6 = nvfp4_fp6_requantize_t(qx6, ROUND_SR, seed, 6)
+    dW = nvfp4_dense_gemm(nvfp4_expand_operand(q5), q6, dw_dtype)
+    return dX, dW, (q3, q4, q5, q6)

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnvfp4_b200.so")
-SOURCES = ["api.cu", "quantize.cu", "gemm.cu", "hp.cu", "noalloc.cu", "calib.cu", "osci.cu", "w16.cu"]
+SOURCES = ["api.cu", "quantize.cu", "gemm.cu", "hp.cu", "noalloc.cu", "calib.cu", "osci.cu", "w16.cu", "fp6.cu"]
 # measurement aids (the tensor-core issue loop): a library of their own, loaded by the benchmark only
 MEASURE_LIB = os.path.join(HERE, "libnvfp4_measure.so")
 MEASURE_SOURCES = ["probe.cu"]

@@ -455,6 +455,79 @@ nvfp4_status nvfp4_gemm_ex(const nvfp4_operand* A, const nvfp4_operand* B, void*
   return do_gemm(A, B, C, c_dtype, ldc, accumulate, dev_status, static_cast<cudaStream_t>(stream), nullptr, nullptr, 0, opts);
 }
 
+int64_t nvfp4_dense_ld(int64_t K) { return (K + 63) & ~(int64_t)63; }
+size_t nvfp4_fp6_workspace_bytes(void) { return 16; }
+
+static nvfp4_status check_dense(const nvfp4_dense_operand* o) {
+  if (!o || !o->vals || !o->gscale) return NVFP4_ERR_NULL;
+  if (o->R <= 0 || o->K <= 0 || o->ld != nvfp4_dense_ld(o->K)) return NVFP4_ERR_SHAPE;
+  if (!aligned16(o->vals) || (reinterpret_cast<uintptr_t>(o->gscale) & 3u)) return NVFP4_ERR_ALIGN;
+  return NVFP4_OK;
+}
+
+nvfp4_status nvfp4_fp6_quantize(const void* src_bf16, int64_t rows, int64_t cols, int64_t ld, int32_t rounding, uint64_t seed,
+                                uint32_t stream_id, const nvfp4_dense_operand* out, void* workspace, size_t ws_bytes, void* stream) {
+  if (!src_bf16) return NVFP4_ERR_NULL;
+  nvfp4_status s;
+  if ((s = check_dense(out)) != NVFP4_OK) return s;
+  if (rows <= 0 || cols <= 0 || ld < cols || out->R != rows || out->K != cols) return NVFP4_ERR_SHAPE;
+  if (rounding != NVFP4_ROUND_RTN && rounding != NVFP4_ROUND_SR) return NVFP4_ERR_ENUM;
+  if (bad_matrix(src_bf16, ld, cols, 2)) return NVFP4_ERR_ALIGN;  // 16-byte aligned rows, as for nvfp4_quantize
+  if (!workspace || !aligned16(workspace) || ws_bytes < nvfp4_fp6_workspace_bytes()) return NVFP4_ERR_WORKSPACE;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  return launch_fp6_quantize_rows(static_cast<const uint16_t*>(src_bf16), rows, cols, ld, rounding == NVFP4_ROUND_SR, seed, stream_id,
+                                  static_cast<uint32_t*>(workspace), static_cast<uint16_t*>(out->vals), out->ld, out->gscale,
+                                  static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? NVFP4_OK
+             : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_fp6_requantize_t(const nvfp4_dense_operand* in, int32_t rounding, uint64_t seed, uint32_t stream_id,
+                                    const nvfp4_dense_operand* out, void* workspace, size_t ws_bytes, void* stream) {
+  nvfp4_status s;
+  if ((s = check_dense(in)) != NVFP4_OK) return s;
+  if ((s = check_dense(out)) != NVFP4_OK) return s;
+  if (out->R != in->K || out->K != in->R) return NVFP4_ERR_SHAPE;
+  if (rounding != NVFP4_ROUND_RTN && rounding != NVFP4_ROUND_SR) return NVFP4_ERR_ENUM;
+  if (!workspace || !aligned16(workspace) || ws_bytes < nvfp4_fp6_workspace_bytes()) return NVFP4_ERR_WORKSPACE;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  return launch_fp6_requantize_t(static_cast<const uint16_t*>(in->vals), in->R, in->K, in->ld, in->gscale, rounding == NVFP4_ROUND_SR, seed,
+                                 stream_id, static_cast<uint32_t*>(workspace), static_cast<uint16_t*>(out->vals), out->ld, out->gscale,
+                                 static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? NVFP4_OK
+             : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_expand_operand(const nvfp4_operand* in, const nvfp4_dense_operand* out, void* stream) {
+  nvfp4_status s;
+  if (!in) return NVFP4_ERR_NULL;
+  if ((s = check_operand_ptrs(in)) != NVFP4_OK) return s;
+  if ((s = check_dense(out)) != NVFP4_OK) return s;
+  if (in->R != out->R || in->K != out->K) return NVFP4_ERR_SHAPE;
+  if (in->gs_mode != NVFP4_GS_TENSOR) return NVFP4_ERR_ENUM;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  return launch_expand_operand(in->codes, in->sf, in->sf_layout == NVFP4_SF_TILED128x4, in->R, in->K, in->gscale,
+                               static_cast<uint16_t*>(out->vals), out->ld, out->gscale, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? NVFP4_OK
+             : NVFP4_ERR_CUDA;
+}
+
+nvfp4_status nvfp4_dense_gemm(const nvfp4_dense_operand* A, const nvfp4_dense_operand* B, void* C, int32_t c_dtype, int64_t ldc,
+                              int32_t* dev_status, void* stream) {
+  nvfp4_status s;
+  if (!C) return NVFP4_ERR_NULL;
+  if ((s = check_dense(A)) != NVFP4_OK) return s;
+  if ((s = check_dense(B)) != NVFP4_OK) return s;
+  if (A->K != B->K) return NVFP4_ERR_SHAPE;
+  if (c_dtype < 0 || c_dtype > 1) return NVFP4_ERR_ENUM;
+  if (bad_matrix(C, ldc, B->R, c_dtype == NVFP4_DT_F32 ? 4 : 2)) return NVFP4_ERR_ALIGN;
+  if ((s = check_arch()) != NVFP4_OK) return s;
+  return launch_dense_gemm(A->vals, B->vals, A->R, B->R, A->ld, A->gscale, B->gscale, C, c_dtype == NVFP4_DT_F32, ldc, dev_status,
+                           static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? NVFP4_OK
+             : NVFP4_ERR_CUDA;
+}
+
 size_t nvfp4_linear_workspace_bytes(int32_t op_kind, int64_t N_tok, int64_t D, int64_t C, int64_t n_out,
                                     int32_t gs_mode) {
   size_t total = 0;

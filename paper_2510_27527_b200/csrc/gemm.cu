@@ -366,8 +366,13 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             if (hp_cols) {
               tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + hp_tmem_col + c0, v);
               tc_wait_ld();
+              if (p.k_tiles > 0) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) o[j] += __uint_as_float(v[j]);
+                for (int j = 0; j < 32; ++j) o[j] += __uint_as_float(v[j]);
+              } else {  // dense BF16 product alone (no FP4 part: the main accumulator was never written): scaled like one
+#pragma unroll
+                for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(v[j]) * alpha;
+              }
             }
             if (p.accumulate && m < p.M) {
               if (n0 + 32 <= p.N) {
@@ -423,10 +428,18 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
               tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + hp_tmem_col + c0, v);
               tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + hp_tmem_col + c0 + 32, v2);
               tc_wait_ld();
+              if (p.k_tiles > 0) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                o[j] += __uint_as_float(v[j]);
-                o[32 + j] += __uint_as_float(v2[j]);
+                for (int j = 0; j < 32; ++j) {
+                  o[j] += __uint_as_float(v[j]);
+                  o[32 + j] += __uint_as_float(v2[j]);
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  o[j] = __uint_as_float(v[j]) * alpha;
+                  o[32 + j] = __uint_as_float(v2[j]) * alpha;
+                }
               }
             }
             if (p.accumulate && m < p.M) {
@@ -1416,6 +1429,39 @@ cudaError_t launch_hp_dw_mma(const uint16_t* dY, int64_t lddy, const uint16_t* X
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   return cudaSuccess;
+}
+
+// Dense BF16 product (the simulated FP6 x FP4 layer): C = (SgA SgB) * A B^T with A [M, ld], B [N, ld] BF16 row-major, ld a
+// multiple of 64 and the same for both. It is the 128 x 128 kernel with no FP4 k tiles at all: only its BF16 side-product path
+// runs (64-wide k tiles, kind::f16, FP32 accumulation in the side accumulator) and the epilogue scales that accumulator.
+cudaError_t launch_dense_gemm(const void* A, const void* B, int64_t M, int64_t N, int64_t ld, const float* a_gscale,
+                              const float* b_gscale, void* Cp, int c_is_f32, int64_t ldc, int32_t* dev_status, cudaStream_t st) {
+  using C = Cfg;
+  if (M == 0 || N == 0) return cudaSuccess;
+  CUtensorMap tmAh, tmBh, tmC;
+  if (!make_hp_map(&tmAh, A, M, ld) || !make_hp_map(&tmBh, B, N, ld) || !make_c_map(&tmC, Cp, M, N, ldc, c_is_f32 != 0))
+    return cudaErrorInvalidValue;
+  Params p{};
+  p.use_tma_store = 1;
+  p.wait_limit = DEFAULT_WAIT_LIMIT_CYCLES;
+  p.hp_k_tiles = (int32_t)(ld / 64);
+  p.a_gscale = a_gscale;
+  p.b_gscale = b_gscale;
+  p.C = Cp;
+  p.ldc = ldc;
+  p.M = M;
+  p.N = N;
+  p.k_tiles = 0;
+  p.m_tiles = (int32_t)((M + BM - 1) / BM);
+  p.n_tiles = (int32_t)((N + BN - 1) / BN);
+  p.c_is_f32 = c_is_f32;
+  p.dev_status = dev_status;
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(gemm_nvfp4_kernel<kGsTensor>), C::SMEM_BYTES);
+  if (e != cudaSuccess) return e;
+  const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
+  const unsigned grid = (unsigned)std::min<int64_t>(tiles, sm_count());
+  launch_kernel(gemm_nvfp4_kernel<kGsTensor>, dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, tmAh, tmBh, tmC, tmAh, tmBh, p);
+  return cudaGetLastError();
 }
 
 size_t gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }

@@ -135,6 +135,18 @@ struct GemmArgs {
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
 int64_t gemm_block128_max_k();  // largest K the BLOCK128 GEMM variant takes
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
+// C = (*a_gscale * *b_gscale) A B^T, A [M, ld] and B [N, ld] BF16 row-major (ld a multiple of 64), FP32 accumulation
+cudaError_t launch_dense_gemm(const void* A, const void* B, int64_t M, int64_t N, int64_t ld, const float* a_gscale,
+                              const float* b_gscale, void* C, int c_is_f32, int64_t ldc, int32_t* dev_status, cudaStream_t st);
+
+// Simulated FP6 (E2M3) quantizers and the FP4 -> dense expansion (fp6.cu). cell: one workspace word.
+cudaError_t launch_fp6_quantize_rows(const uint16_t* src, int64_t rows, int64_t K, int64_t ld, int sr, uint64_t seed, uint32_t stream_id,
+                                     uint32_t* cell, uint16_t* out, int64_t ld_out, float* gscale, cudaStream_t st);
+cudaError_t launch_fp6_requantize_t(const uint16_t* in, int64_t rowsK, int64_t D, int64_t ld_in, const float* in_gscale, int sr,
+                                    uint64_t seed, uint32_t stream_id, uint32_t* cell, uint16_t* out, int64_t ld_out, float* gscale,
+                                    cudaStream_t st);
+cudaError_t launch_expand_operand(const uint8_t* codes, const uint8_t* sf, int sf_tiled, int64_t R, int64_t K, const float* in_gscale,
+                                  uint16_t* out, int64_t ld_out, float* gscale, cudaStream_t st);
 
 // High-precision (BF16 inputs, FP32 accumulate) products over OutControl's outlier channels.
 //   fwd: Y[m, n] (+)= sum_j X[m, outl[j]] * W[n, outl[j]]
