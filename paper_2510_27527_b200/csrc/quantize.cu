@@ -1240,17 +1240,20 @@ quantize_transpose_kernel(TransposeSrc s, int64_t rowsK, int64_t D, uint64_t see
 
 // =========================================================================================================
 // Column-axis quantize from BF16 without a shared-memory transposition (Q5 of Sec. 2.3: the operand is dY^T, its blocks
-// run along the tokens). A lane owns FOUR neighbouring source columns (= operand rows) and 64 consecutive source rows
-// (= operand k). It reads 8 bytes per source row, so one warp instruction covers two source rows of 128 contiguous bytes
-// (lanes 0..15: rows k .. , lanes 16..31: rows k + 64 ..), and the 16 values of an inner block are the same half of 16 loaded
-// words: the transposition is the choice of that half. Per 16 source rows the lane quantizes four blocks (one per column)
-// and stores 8 code bytes to each of its four operand rows; the four scale bytes of an operand row (64 k) are one aligned
-// word of either scale layout. The two lanes that share a 128-wide outer group exchange their maxima with one shuffle;
-// BLOCK128 therefore walks its 64 rows twice (maxima, then codes; the second walk is served by L2). No barrier, no shared
-// memory, and the index arithmetic is paid once per 256 elements.
-//   RMODE  0 round to nearest, 1 stochastic rounding, 2 stochastic rounding with the block scale rounded up.
+// run along the tokens), for the TENSOR and ROW scale modes. A lane owns FOUR neighbouring source columns (= operand rows)
+// and 64 consecutive source rows (= operand k). It reads 8 bytes per source row, so one warp instruction covers two source
+// rows of 128 contiguous bytes (lanes 0..15: rows k .. , lanes 16..31: rows k + 64 ..), and the 16 values of an inner block
+// are the same half of 16 loaded words: the transposition is the choice of that half. Per 16 source rows the lane quantizes
+// four blocks (one per column) and stores 8 code bytes to each of its four operand rows; the four scale bytes of an operand
+// row (64 k) are one aligned word of either scale layout. No barrier, no shared memory, and the index arithmetic is paid
+// once per 256 elements.
+//   RMODE      0 round to nearest, 1 stochastic rounding, 2 stochastic rounding with the block scale rounded up.
+//   RHT        every block is replaced by (x S) H_16 first (Sec. 4.1): the lane's 64 sign bits are half of one generator
+//              block, the butterflies run on the 16 values it holds anyway.
+//   AMAX_ONLY  the pre-pass of RHT: only the maximum of the transformed values, folded into gs_cells (one cell, or one per
+//              operand row in ROW mode); nothing else is written.
 // Preconditions (the launcher falls back to the staged kernel otherwise): D and ld multiples of 4, src 8-byte aligned,
-// identity row order, no Hadamard transformation.
+// identity row order.
 // =========================================================================================================
 __device__ __forceinline__ uint2 ld_nc_8(const uint16_t* p) {
   uint2 v;
@@ -1258,11 +1261,12 @@ __device__ __forceinline__ uint2 ld_nc_8(const uint16_t* p) {
   return v;
 }
 
-template <int GS, int RMODE, bool TILED>
+template <int GS, int RMODE, bool TILED, bool RHT, bool AMAX_ONLY>
 __global__ void __launch_bounds__(128, 4)
-quantize_cols4_kernel(const uint16_t* __restrict__ src, uint32_t K, uint32_t D, uint32_t ld, uint32_t stream_id,
-                      const uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
+quantize_cols4_kernel(const uint16_t* __restrict__ src, uint32_t K, uint32_t D, uint32_t ld, uint64_t seed, uint32_t stream_id,
+                      uint32_t rht_stream, uint32_t* __restrict__ gs_cells, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf,
                       float* __restrict__ gscale, const __grid_constant__ PhiloxKeys pk) {
+  static_assert(GS != kGsBlock128, "the outer-block mode has a kernel of its own");
   pdl_prologue();
   constexpr bool SR = RMODE != 0;
   const uint32_t Kp = (K + 127u) & ~127u;
@@ -1274,80 +1278,103 @@ quantize_cols4_kernel(const uint16_t* __restrict__ src, uint32_t K, uint32_t D, 
   const bool live = d0 < D && k_start < Kp;  // (all four rows exist or none: D is a multiple of 4)
   const uint16_t* p = src + (size_t)k_start * ld + d0;
 
-  float Sg[4];
-  if (GS == kGsBlock128) {
-    uint32_t mx = 0, my = 0;
-    if (live) {
-#pragma unroll 16
-      for (uint32_t t = 0; t < 64; ++t) {
-        if (k_start + t < K) {
-          const uint2 v = ld_nc_8(p + (size_t)t * ld);
-          mx = amax16x2(mx, v.x);
-          my = amax16x2(my, v.y);
+  float Sg[4] = {1.0f, 1.0f, 1.0f, 1.0f};
+  if (!AMAX_ONLY) {
+    if (GS == kGsRow) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        Sg[c] = global_scale_from_amax(live ? __uint_as_float(gs_cells[d0 + c]) : 0.0f);
+        if (live && k_start == 0) gscale[d0 + c] = Sg[c];
+      }
+    } else {
+      Sg[0] = Sg[1] = Sg[2] = Sg[3] = global_scale_from_amax(__uint_as_float(gs_cells[0]));
+      if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) gscale[0] = Sg[0];
+    }
+  }
+  // the 64 sign bits of this lane's k range (one half of a 128-group's generator block)
+  uint32_t sgn_lo = 0, sgn_hi = 0;
+  if (RHT && live) {
+    const uint4 sw = rht_sign_words(seed, rht_stream, (uint64_t)(k_start >> 7));
+    sgn_lo = (k_start & 64u) ? sw.z : sw.x;
+    sgn_hi = (k_start & 64u) ? sw.w : sw.y;
+  }
+  float am_run[4] = {0.0f, 0.0f, 0.0f, 0.0f};  // AMAX_ONLY: running maxima of the four operand rows
+
+  uint32_t sfw[4] = {0u, 0u, 0u, 0u};
+  if (live) {
+#pragma unroll 1
+    for (uint32_t tb = 0; tb < 4; ++tb) {
+      const uint32_t k0 = k_start + 16u * tb;
+      if (AMAX_ONLY && k0 >= K16) break;  // layout padding: zeros
+      uint2 w[16];
+      if (k0 + 16u <= K) {
+#pragma unroll
+        for (int t = 0; t < 16; ++t) w[t] = ld_nc_8(p + (size_t)(16u * tb + t) * ld);
+      } else {
+#pragma unroll
+        for (int t = 0; t < 16; ++t) w[t] = k0 + t < K ? ld_nc_8(p + (size_t)(16u * tb + t) * ld) : make_uint2(0u, 0u);
+      }
+      float am[4];
+      if (!RHT) {
+        uint32_t mx = 0, my = 0;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          mx = amax16x2(mx, w[t].x);
+          my = amax16x2(my, w[t].y);
+        }
+        mx = bf16x2_abs_bits(mx);
+        my = bf16x2_abs_bits(my);
+        am[0] = __uint_as_float(mx << 16);
+        am[1] = __uint_as_float(mx & 0xFFFF0000u);
+        am[2] = __uint_as_float(my << 16);
+        am[3] = __uint_as_float(my & 0xFFFF0000u);
+      }
+      // signs of rows k0 .. k0 + 15; rows past K rounded up to 16 are layout padding and take none (they stay +0)
+      const uint32_t s16 = RHT && k0 < K16 ? ((((tb & 2u) ? sgn_hi : sgn_lo) >> (16u * (tb & 1u))) & 0xFFFFu) : 0u;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float x[16];
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          const uint32_t word = c < 2 ? w[t].x : w[t].y;
+          x[t] = (c & 1) ? bf16_hi(word) : bf16_lo(word);
+        }
+        if (RHT) {
+          rht_scale16(x, s16);
+          hadamard16_butterflies(x);
+          float m = 0.0f;
+#pragma unroll
+          for (int t = 0; t < 16; ++t) m = fmaxf(m, fabsf(x[t]));
+          am[c] = m;
+        }
+        if (AMAX_ONLY) {
+          am_run[c] = fmaxf(am_run[c], am[c]);
+        } else {
+          float rcp;
+          const uint32_t sb = block_scale(am[c], Sg[c], rcp, RMODE == 2);
+          sfw[c] |= sb << (8u * tb);
+          const uint2 packed = quantize_block16<SR>(x, rcp, pk, stream_id, ((uint64_t)(d0 + c) * K16 + k0) >> 3);
+          *reinterpret_cast<uint2*>(codes + (size_t)(d0 + c) * (Kp >> 1) + (k0 >> 1)) = packed;
         }
       }
     }
-    mx = amax16x2(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 16));  // the other half of the 128-wide group
-    my = amax16x2(my, __shfl_xor_sync(0xFFFFFFFFu, my, 16));
-    mx = bf16x2_abs_bits(mx);
-    my = bf16x2_abs_bits(my);
-    Sg[0] = global_scale_from_amax(__uint_as_float(mx << 16));
-    Sg[1] = global_scale_from_amax(__uint_as_float(mx & 0xFFFF0000u));
-    Sg[2] = global_scale_from_amax(__uint_as_float(my << 16));
-    Sg[3] = global_scale_from_amax(__uint_as_float(my & 0xFFFF0000u));
-    if (live && (lane >> 4) == 0) {
+  }
+  if (AMAX_ONLY) {
+    if (GS == kGsRow) {  // one cell per operand row; the two lanes that share the rows first combine
 #pragma unroll
-      for (int c = 0; c < 4; ++c) gscale[(size_t)(d0 + c) * (Kp >> 7) + (k_start >> 7)] = Sg[c];
-    }
-  } else if (GS == kGsRow) {
+      for (int c = 0; c < 4; ++c) {
+        const float m = fmaxf(am_run[c], __shfl_xor_sync(0xFFFFFFFFu, am_run[c], 16));
+        if (live && lane < 16 && m > 0.0f) atomicMax(gs_cells + d0 + c, __float_as_uint(m));
+      }
+    } else {
+      float m = fmaxf(fmaxf(am_run[0], am_run[1]), fmaxf(am_run[2], am_run[3]));
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      Sg[c] = global_scale_from_amax(live ? __uint_as_float(gs_cells[d0 + c]) : 0.0f);
-      if (live && k_start == 0) gscale[d0 + c] = Sg[c];
+      for (int q = 16; q; q >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, q));
+      if (lane == 0 && m > 0.0f) atomicMax(gs_cells, __float_as_uint(m));
     }
-  } else {
-    Sg[0] = Sg[1] = Sg[2] = Sg[3] = global_scale_from_amax(__uint_as_float(gs_cells[0]));
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) gscale[0] = Sg[0];
+    return;
   }
   if (!live) return;
-
-  uint32_t sfw[4] = {0u, 0u, 0u, 0u};
-#pragma unroll 1
-  for (uint32_t tb = 0; tb < 4; ++tb) {
-    const uint32_t k0 = k_start + 16u * tb;
-    uint2 w[16];
-    if (k0 + 16u <= K) {
-#pragma unroll
-      for (int t = 0; t < 16; ++t) w[t] = ld_nc_8(p + (size_t)(16u * tb + t) * ld);
-    } else {
-#pragma unroll
-      for (int t = 0; t < 16; ++t) w[t] = k0 + t < K ? ld_nc_8(p + (size_t)(16u * tb + t) * ld) : make_uint2(0u, 0u);
-    }
-    uint32_t mx = 0, my = 0;
-#pragma unroll
-    for (int t = 0; t < 16; ++t) {
-      mx = amax16x2(mx, w[t].x);
-      my = amax16x2(my, w[t].y);
-    }
-    mx = bf16x2_abs_bits(mx);
-    my = bf16x2_abs_bits(my);
-    const float am[4] = {__uint_as_float(mx << 16), __uint_as_float(mx & 0xFFFF0000u), __uint_as_float(my << 16),
-                         __uint_as_float(my & 0xFFFF0000u)};
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      float rcp;
-      const uint32_t sb = block_scale(am[c], Sg[c], rcp, RMODE == 2);
-      sfw[c] |= sb << (8u * tb);
-      float x[16];
-#pragma unroll
-      for (int t = 0; t < 16; ++t) {
-        const uint32_t word = c < 2 ? w[t].x : w[t].y;
-        x[t] = (c & 1) ? bf16_hi(word) : bf16_lo(word);
-      }
-      const uint2 packed = quantize_block16<SR>(x, rcp, pk, stream_id, ((uint64_t)(d0 + c) * K16 + k0) >> 3);
-      *reinterpret_cast<uint2*>(codes + (size_t)(d0 + c) * (Kp >> 1) + (k0 >> 1)) = packed;
-    }
-  }
   const uint32_t b = k_start >> 4;  // first of this lane's four k blocks: a multiple of 4
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
@@ -1361,11 +1388,13 @@ quantize_cols4_kernel(const uint16_t* __restrict__ src, uint32_t K, uint32_t D, 
 // The same for the 1 x 128 outer block (BLOCK128), where the scale of a block depends on all 128 k of its group: a lane owns
 // TWO neighbouring source columns and keeps its 64 source rows in registers (one 32-bit word per row), so the data is read
 // once; the two lanes of a group exchange the group maximum with one shuffle. A warp instruction covers two source rows of
-// 64 contiguous bytes.
-template <int RMODE, bool TILED>
+// 64 contiguous bytes. With RHT the group maximum is that of the transformed values: the eight blocks are transformed once
+// for their maxima and once more when they are quantized (80 floating-point operations per block and pass; holding the 128
+// transformed values beside the 64 raw words does not fit the register file at a useful occupancy).
+template <int RMODE, bool TILED, bool RHT>
 __global__ void __launch_bounds__(128, 3)
-quantize_cols2_block128_kernel(const uint16_t* __restrict__ src, uint32_t K, uint32_t D, uint32_t ld, uint32_t stream_id,
-                               uint8_t* __restrict__ codes, uint8_t* __restrict__ sf, float* __restrict__ gscale,
+quantize_cols2_block128_kernel(const uint16_t* __restrict__ src, uint32_t K, uint32_t D, uint32_t ld, uint64_t seed, uint32_t stream_id,
+                               uint32_t rht_stream, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf, float* __restrict__ gscale,
                                const __grid_constant__ PhiloxKeys pk) {
   pdl_prologue();
   constexpr bool SR = RMODE != 0;
@@ -1389,18 +1418,54 @@ quantize_cols2_block128_kernel(const uint16_t* __restrict__ src, uint32_t K, uin
       if (live && k_start + t < K) asm volatile("ld.global.nc.L1::no_allocate.b32 %0, [%1];" : "=r"(w[t]) : "l"(p + (size_t)t * ld));
     }
   }
-  uint32_t bm[4];  // packed block maxima (sign bits meaningless until masked)
-#pragma unroll
-  for (int tb = 0; tb < 4; ++tb) {
-    uint32_t m = 0;
-#pragma unroll
-    for (int t = 0; t < 16; ++t) m = amax16x2(m, w[16 * tb + t]);
-    bm[tb] = m;
+  // the 64 sign bits of this lane's k range; rows past K rounded up to 16 are layout padding and take none (they stay +0)
+  uint32_t sgn[2] = {0u, 0u};
+  if (RHT && live) {
+    const uint4 sw = rht_sign_words(seed, rht_stream, (uint64_t)(k_start >> 7));
+    sgn[0] = (k_start & 64u) ? sw.z : sw.x;
+    sgn[1] = (k_start & 64u) ? sw.w : sw.y;
   }
-  uint32_t g = amax16x2(amax16x2(bm[0], bm[1]), amax16x2(bm[2], bm[3]));
-  g = bf16x2_abs_bits(amax16x2(g, __shfl_xor_sync(0xFFFFFFFFu, g, 16)));  // the other half of the 128-wide group
+  auto sign16 = [&](int tb) -> uint32_t { return k_start + 16u * tb < K16 ? ((sgn[tb >> 1] >> (16 * (tb & 1))) & 0xFFFFu) : 0u; };
+
+  float Sg[2];
+  float bam[RHT ? 4 : 1][2];  // RHT: block maxima of the transformed values
+  uint32_t bm[4];             // otherwise: packed block maxima (sign bits meaningless until masked)
+  if (RHT) {
+    float g0 = 0.0f, g1 = 0.0f;
+#pragma unroll
+    for (int tb = 0; tb < 4; ++tb) {
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        float x[16];
+#pragma unroll
+        for (int t = 0; t < 16; ++t) x[t] = c ? bf16_hi(w[16 * tb + t]) : bf16_lo(w[16 * tb + t]);
+        rht_scale16(x, sign16(tb));
+        hadamard16_butterflies(x);
+        float m = 0.0f;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) m = fmaxf(m, fabsf(x[t]));
+        bam[RHT ? tb : 0][c] = m;
+        if (c) g1 = fmaxf(g1, m); else g0 = fmaxf(g0, m);
+      }
+    }
+    g0 = fmaxf(g0, __shfl_xor_sync(0xFFFFFFFFu, g0, 16));  // the other half of the 128-wide group
+    g1 = fmaxf(g1, __shfl_xor_sync(0xFFFFFFFFu, g1, 16));
+    Sg[0] = global_scale_from_amax(g0);
+    Sg[1] = global_scale_from_amax(g1);
+  } else {
+#pragma unroll
+    for (int tb = 0; tb < 4; ++tb) {
+      uint32_t m = 0;
+#pragma unroll
+      for (int t = 0; t < 16; ++t) m = amax16x2(m, w[16 * tb + t]);
+      bm[tb] = m;
+    }
+    uint32_t g = amax16x2(amax16x2(bm[0], bm[1]), amax16x2(bm[2], bm[3]));
+    g = bf16x2_abs_bits(amax16x2(g, __shfl_xor_sync(0xFFFFFFFFu, g, 16)));
+    Sg[0] = global_scale_from_amax(__uint_as_float(g << 16));
+    Sg[1] = global_scale_from_amax(__uint_as_float(g & 0xFFFF0000u));
+  }
   if (!live) return;
-  const float Sg[2] = {global_scale_from_amax(__uint_as_float(g << 16)), global_scale_from_amax(__uint_as_float(g & 0xFFFF0000u))};
   if ((lane >> 4) == 0) {
     gscale[(size_t)d0 * (Kp >> 7) + (k_start >> 7)] = Sg[0];
     gscale[(size_t)(d0 + 1) * (Kp >> 7) + (k_start >> 7)] = Sg[1];
@@ -1409,16 +1474,20 @@ quantize_cols2_block128_kernel(const uint16_t* __restrict__ src, uint32_t K, uin
 #pragma unroll
   for (int tb = 0; tb < 4; ++tb) {
     const uint32_t k0 = k_start + 16u * tb;
-    const uint32_t m = bf16x2_abs_bits(bm[tb]);
-    const float am[2] = {__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u)};
+    const uint32_t m = RHT ? 0u : bf16x2_abs_bits(bm[tb]);
 #pragma unroll
     for (int c = 0; c < 2; ++c) {
+      const float am = RHT ? bam[RHT ? tb : 0][c] : __uint_as_float(c ? (m & 0xFFFF0000u) : (m << 16));
       float rcp;
-      const uint32_t sb = block_scale(am[c], Sg[c], rcp, RMODE == 2);
+      const uint32_t sb = block_scale(am, Sg[c], rcp, RMODE == 2);
       sfw[c] |= sb << (8 * tb);
       float x[16];
 #pragma unroll
       for (int t = 0; t < 16; ++t) x[t] = c ? bf16_hi(w[16 * tb + t]) : bf16_lo(w[16 * tb + t]);
+      if (RHT) {
+        rht_scale16(x, sign16(tb));
+        hadamard16_butterflies(x);
+      }
       const uint2 packed = quantize_block16<SR>(x, rcp, pk, stream_id, ((uint64_t)(d0 + c) * K16 + k0) >> 3);
       *reinterpret_cast<uint2*>(codes + (size_t)(d0 + c) * (Kp >> 1) + (k0 >> 1)) = packed;
     }
@@ -1605,11 +1674,11 @@ static bool transpose_fast_path(const TransposeSrc& s, int from_codes) {
   return (s.ld & 7) == 0 && (reinterpret_cast<uintptr_t>(s.bf16) & 15u) == 0;
 }
 
-// The register-transposing kernel takes a plain BF16 source whose rows can be read in 8-byte pieces: identity row order, no
-// Hadamard transformation, no closed-form maximum handed in by OutControl's two-pass W-hat.
+// The register-transposing kernels take a plain BF16 source whose rows can be read in 8-byte pieces: identity row order, no
+// closed-form maximum handed in by OutControl's two-pass W-hat.
 static bool cols4_path(const QuantTransposeArgs& a) {
   const TransposeSrc& s = a.src;
-  return !a.rht_stream && !s.out_rows && !s.closed_form_sg && !a.tensor_closed_form && (a.D & 3) == 0 && (s.ld & 3) == 0 &&
+  return !s.out_rows && !s.closed_form_sg && !a.tensor_closed_form && (a.D & 3) == 0 && (s.ld & 3) == 0 &&
          (reinterpret_cast<uintptr_t>(s.bf16) & 7u) == 0 && s.ld < ((int64_t)1 << 31) && a.rowsK < ((int64_t)1 << 31) - 1024 &&
          a.D < ((int64_t)1 << 31) - 64;
 }
@@ -1618,25 +1687,26 @@ template <int SRC, int GS, int RMODE>
 static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
   const dim3 grid(blocks_for(a.rowsK, 128), blocks_for(a.D, 64));
   const bool fast = transpose_fast_path(a.src, SRC);
-  if (SRC == 0 && GS == kGsBlock128 && cols4_path(a)) {
-    const dim3 g2(blocks_for(a.rowsK, 512), blocks_for(a.D, 32));
-    if (a.sf_tiled)
-      launch_kernel(quantize_cols2_block128_kernel<RMODE, true>, g2, dim3(128), 0, st, a.src.bf16, (uint32_t)a.rowsK, (uint32_t)a.D,
-                    (uint32_t)a.src.ld, a.stream_id, a.codes, a.sf, a.gscale, make_philox_keys(a.seed));
-    else
-      launch_kernel(quantize_cols2_block128_kernel<RMODE, false>, g2, dim3(128), 0, st, a.src.bf16, (uint32_t)a.rowsK, (uint32_t)a.D,
-                    (uint32_t)a.src.ld, a.stream_id, a.codes, a.sf, a.gscale, make_philox_keys(a.seed));
-    return cudaGetLastError();
-  }
-  if (SRC == 0 && cols4_path(a)) {
-    const dim3 g4(blocks_for(a.rowsK, 512), blocks_for(a.D, 64));
-    if (a.sf_tiled)
-      launch_kernel(quantize_cols4_kernel<GS, RMODE, true>, g4, dim3(128), 0, st, a.src.bf16, (uint32_t)a.rowsK, (uint32_t)a.D,
-                    (uint32_t)a.src.ld, a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, make_philox_keys(a.seed));
-    else
-      launch_kernel(quantize_cols4_kernel<GS, RMODE, false>, g4, dim3(128), 0, st, a.src.bf16, (uint32_t)a.rowsK, (uint32_t)a.D,
-                    (uint32_t)a.src.ld, a.stream_id, a.gs_cells, a.codes, a.sf, a.gscale, make_philox_keys(a.seed));
-    return cudaGetLastError();
+  if constexpr (SRC == 0) {
+    if (cols4_path(a)) {
+      const PhiloxKeys keys = make_philox_keys(a.seed);
+      const uint32_t K32 = (uint32_t)a.rowsK, D32 = (uint32_t)a.D, ld32 = (uint32_t)a.src.ld;
+#define NVFP4_LAUNCH_COLS(TILED_, RHT_)                                                                                             \
+  if constexpr (GS == kGsBlock128)                                                                                                  \
+    launch_kernel(quantize_cols2_block128_kernel<RMODE, TILED_, RHT_>, dim3(blocks_for(a.rowsK, 512), blocks_for(a.D, 32)),         \
+                  dim3(128), 0, st, a.src.bf16, K32, D32, ld32, a.seed, a.stream_id, a.rht_stream, a.codes, a.sf, a.gscale, keys);  \
+  else                                                                                                                              \
+    launch_kernel(quantize_cols4_kernel<GS, RMODE, TILED_, RHT_, false>, dim3(blocks_for(a.rowsK, 512), blocks_for(a.D, 64)),       \
+                  dim3(128), 0, st, a.src.bf16, K32, D32, ld32, a.seed, a.stream_id, a.rht_stream, a.gs_cells, a.codes, a.sf,       \
+                  a.gscale, keys)
+      if (a.sf_tiled) {
+        if (a.rht_stream) { NVFP4_LAUNCH_COLS(true, true); } else { NVFP4_LAUNCH_COLS(true, false); }
+      } else {
+        if (a.rht_stream) { NVFP4_LAUNCH_COLS(false, true); } else { NVFP4_LAUNCH_COLS(false, false); }
+      }
+#undef NVFP4_LAUNCH_COLS
+      return cudaGetLastError();
+    }
   }
 #define NVFP4_LAUNCH_TR(TILED_, RHT_)                                                                                                  \
   if (fast)                                                                                                                            \
@@ -1665,6 +1735,16 @@ static cudaError_t launch_tr_amax_rht(const TransposeSrc& src, int64_t rowsK, in
   const dim3 grid(blocks_for(rowsK, 128), blocks_for(D, 64));
   uint8_t* const no_bytes = nullptr;
   float* const no_floats = nullptr;
+  if constexpr (SRC == 0 && GS != kGsBlock128) {
+    // the register-transposing kernel's own pre-pass (same conditions as cols4_path)
+    if (rht_stream && !src.out_rows && (D & 3) == 0 && (src.ld & 3) == 0 && (reinterpret_cast<uintptr_t>(src.bf16) & 7u) == 0 &&
+        src.ld < ((int64_t)1 << 31) && rowsK < ((int64_t)1 << 31) - 1024 && D < ((int64_t)1 << 31) - 64) {
+      launch_kernel(quantize_cols4_kernel<GS, 0, false, true, true>, dim3(blocks_for(rowsK, 512), blocks_for(D, 64)), dim3(128), 0, st,
+                    src.bf16, (uint32_t)rowsK, (uint32_t)D, (uint32_t)src.ld, seed, 0u, rht_stream, cells, no_bytes, no_bytes, no_floats,
+                    make_philox_keys(seed));
+      return cudaGetLastError();
+    }
+  }
   if (transpose_fast_path(src, SRC)) {
     if (rht_stream)
       launch_kernel(quantize_transpose_kernel<SRC, GS, 0, false, true, true>, dim3(grid), dim3(256), 0, st, src, rowsK, D, seed, 0u, cells, 0,

@@ -112,3 +112,15 @@ def test_bench_parses_gpus_and_would_spawn(monkeypatch):
         bench.main()
     assert e.value.code == 0
     assert calls == [(4, os.path.join(ROOT, "bench.py"), ["--gpus", "4", "--steps", "2"])]
+
+
+def test_module_keys_differ_between_layers_and_calls():
+    """Two modules built from the same configuration, and two calls of one module, must not share their stochastic-rounding
+    key (the draws of equal-shaped layers would otherwise be identical element for element)."""
+    from paper_2510_27527_b200 import module
+
+    keys = {module.call_seed(0, layer, call) for layer in range(24) for call in range(50)}
+    assert len(keys) == 24 * 50
+    assert all(0 <= k < 1 << 64 for k in keys)
+    assert module.call_seed(0, 0, 0) != module.call_seed(1, 0, 0)
+    assert module.call_seed(7, 3, 5) == module.call_seed(7, 3, 5)
