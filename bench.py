@@ -640,6 +640,25 @@ def run_aux(args):
         out[f"osci_sparse_update_8192x8192_{name}"] = {"us": sec * 1e6, "state_bytes_per_param": 20.0 * n_track / (C * D),
                                                         "GBps_upper_bound_bytes": alg / sec / 1e9}
         del ws0
+    # simulated FP6 x FP4 layer (Sec. 5.4) on the QKV linear of the 370M model, beside the FP4 layer on the same inputs
+    T, D2, C2 = 16384, 1024, 3072
+    Xs, Ws, dYs, _ = synth.layer_inputs(4, T, D2, C2, n_outlier=10, factor=30.0, grad_scale=1e-4, weight_id=10)
+    Xd, Wd, dYd = b.upload_bf16(Xs, dev), b.upload_bf16(Ws, dev), b.upload_bf16(dYs, dev)
+
+    def fp6_step():
+        _, saved6 = b.fp6_linear_fwd(Xd, Wd, b.DT_BF16)
+        b.fp6_linear_bwd(dYd, saved6, 0)
+
+    cfg4 = b.LayerConfig(gs_mode=b.GS_TENSOR, seed=0)
+
+    def fp4_step():
+        _, saved4 = b.nvfp4_linear_fwd(Xd, Wd, cfg4)
+        b.nvfp4_linear_bwd(dYd, saved4, cfg4)
+
+    fl = 6.0 * T * D2 * C2
+    for name, fn in (("fp6_sim_layer_qkv_tokens16384", fp6_step), ("fp4_layer_qkv_tokens16384_same_call_pattern", fp4_step)):
+        sec = t_of(fn, max(3, args.steps // 2))
+        out[name] = {"us": sec * 1e6, "TFLOPs": fl / sec / 1e12}
     print(json.dumps({"aux": out, "peaks": pk}))
 
 
