@@ -1502,6 +1502,149 @@ quantize_cols2_block128_kernel(const uint16_t* __restrict__ src, uint32_t K, uin
   }
 }
 
+// Transposing re-quantize of a forward operand (Q4, Q6 of Sec. 2.3) without a shared-memory transposition, for the TENSOR
+// and ROW scale modes of the output. A lane owns EIGHT neighbouring source columns (one 32-bit word of codes per source row,
+// all under one source scale byte) and 64 consecutive source rows; a warp instruction covers two source rows of 64
+// contiguous code bytes. Per 16 source rows the lane keeps the 16 code words and walks its four column pairs in a ROLLED loop
+// (the loop body -- decode one byte per row into P * S_block as an FP16 pair, exact, then two blocks of 16 values down the
+// rows -- stays small enough for the instruction cache, which a fully unrolled version did not). x_hat = (P * S_block) *
+// S_global of the source row is the same single binary32 rounding as everywhere else. The scale bytes of a lane (8 rows x 4
+// blocks) are collected in a private strip of shared memory and written as one aligned word per operand row.
+//   UNIFORM  the source has one global scale (TENSOR mode); otherwise it is fetched per source row (ROW) or per source row and
+//            128-column group (BLOCK128; a lane's eight columns lie in one group).
+//   TBT      16-row blocks per lane: 4 (64 source rows, CTA tile 512 x 128) for operands large enough to fill the chip with such
+//            tiles, 1 (CTA tile 128 x 128; scale bytes stored one by one) for the model's 16384 x 1024 activations.
+// Preconditions (else the staged kernel runs): identity row order, no row map, no Hadamard transformation.
+template <int GS, int RMODE, bool TILED, bool UNIFORM, int TBT>
+__global__ void __launch_bounds__(128, 4)
+requantize_cols8_kernel(const TransposeSrc s, uint32_t K, uint32_t D, uint32_t stream_id, const uint32_t* __restrict__ gs_cells,
+                        int tensor_closed_form, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf, float* __restrict__ gscale,
+                        const __grid_constant__ PhiloxKeys pk) {
+  static_assert(GS != kGsBlock128, "the outer-block mode keeps the staged kernel");
+  pdl_prologue();
+  constexpr bool SR = RMODE != 0;
+  __shared__ __align__(4) uint8_t sf_strip[128][36];  // per thread: 8 operand rows x 4 k blocks (+4: spreads the banks)
+  const uint32_t Kp = (K + 127u) & ~127u;
+  const uint32_t K16 = (K + 15u) & ~15u;
+  const uint32_t nb = Kp >> 4;
+  const uint32_t in_Kp = ((uint32_t)s.in_K + 127u) & ~127u;
+  const uint32_t in_nb = in_Kp >> 4;
+  const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+  const uint32_t d0 = blockIdx.y * 128u + (lane & 15u) * 8u;                       // first of this lane's operand rows
+  const uint32_t k_start = (blockIdx.x * 8u + warp * 2u + (lane >> 4)) * (16u * TBT);  // first of its 16 * TBT k
+  if (d0 >= D || k_start >= Kp) return;
+  // (d0 + 7 < in_Kp always: the source rows are padded to 128 columns with zero codes and zero scales)
+  const uint8_t* cp = s.in_codes + (size_t)k_start * (in_Kp >> 1) + (d0 >> 1);
+  const uint32_t kb_in = d0 >> 4;
+  const uint32_t in_tile_stride = ((in_nb + 15u) & ~15u) >> 2;
+
+  float Sg_t = 1.0f;
+  if (GS == kGsTensor) {
+    // (tensor_closed_form == 2: the cell carries nothing and may be uninitialised; otherwise it covers what the closed form
+    // does not. The closed form: the source's maximum is float32(2688 * S_global), its largest block has scale 448 and a
+    // magnitude-6 element.)
+    float amax = tensor_closed_form == 2 ? 0.0f : __uint_as_float(gs_cells[0]);
+    if (tensor_closed_form) amax = fmaxf(amax, __fmul_rn(2688.0f, s.in_gscale[0]));
+    Sg_t = global_scale_from_amax(amax);
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) gscale[0] = Sg_t;
+  }
+  const float sg_uniform = UNIFORM ? s.in_gscale[0] : 1.0f;
+  uint8_t* my_sf = &sf_strip[threadIdx.x][0];
+
+#pragma unroll 1
+  for (uint32_t tb = 0; tb < (uint32_t)TBT; ++tb) {
+    const uint32_t k0 = k_start + 16u * tb;
+    // the 16 scale bytes of rows k0 .. k0 + 15 (k0 a multiple of 16) lie at a constant stride in either layout
+    const size_t sf0 = s.in_sf_tiled ? (size_t)((k0 >> 7) * in_tile_stride + (kb_in >> 2)) * 512u +
+                                           ((k0 & 31u) * 16u + ((k0 >> 5) & 3u) * 4u + (kb_in & 3u))
+                                     : (size_t)k0 * in_nb + kb_in;
+    const uint32_t sf_step = s.in_sf_tiled ? 16u : in_nb;
+    const uint8_t* crow = cp + (size_t)(16u * tb) * (in_Kp >> 1);
+    uint32_t cw[16], s2[16];
+    float sgk[UNIFORM ? 1 : 16];
+    {
+      uint32_t sbv[16];
+      if (k0 + 16u <= K) {
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          cw[t] = *reinterpret_cast<const uint32_t*>(crow + (size_t)t * (in_Kp >> 1));
+          sbv[t] = s.in_sf[sf0 + (size_t)t * sf_step];
+        }
+      } else {
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          cw[t] = sbv[t] = 0u;
+          if (k0 + t < K) {
+            cw[t] = *reinterpret_cast<const uint32_t*>(crow + (size_t)t * (in_Kp >> 1));
+            sbv[t] = s.in_sf[sf0 + (size_t)t * sf_step];
+          }
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < 16; ++t)  // the row's block scale as an FP16 pair (both halves equal)
+        asm("{.reg .b16 q; cvt.u16.u32 q, %1; cvt.rn.f16x2.e4m3x2 %0, q;}" : "=r"(s2[t]) : "r"(sbv[t] | (sbv[t] << 8)));
+    }
+    if (!UNIFORM) {
+#pragma unroll
+      for (int t = 0; t < 16; ++t) {
+        const uint32_t k = k0 + t;
+        sgk[UNIFORM ? 0 : t] = k >= K ? 0.0f : s.in_gs_mode == kGsRow ? s.in_gscale[k] : s.in_gscale[(size_t)k * (in_Kp >> 7) + (d0 >> 7)];
+      }
+    }
+#pragma unroll 1
+    for (uint32_t j = 0; j < 4; ++j) {  // column pair (d0 + 2j, d0 + 2j + 1) = byte j of every code word
+      float xs[2][16];
+#pragma unroll
+      for (int t = 0; t < 16; ++t) {
+        uint32_t h2;
+        asm("{\n.reg .b8 b0, b1, b2, b3;\nmov.b32 {b0, b1, b2, b3}, %1;\ncvt.rn.f16x2.e2m1x2 %0, b0;\n}" : "=r"(h2) : "r"(__byte_perm(cw[t], 0u, j)));
+        const __half2 pv = __hmul2(*reinterpret_cast<const __half2*>(&h2), *reinterpret_cast<const __half2*>(&s2[t]));  // exact
+        const float2 f = __half22float2(pv);
+        const float g = UNIFORM ? sg_uniform : sgk[UNIFORM ? 0 : t];
+        xs[0][t] = __fmul_rn(f.x, g);
+        xs[1][t] = __fmul_rn(f.y, g);
+      }
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {
+        const uint32_t o = d0 + 2u * j + c;
+        float m = 0.0f;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) m = fmaxf(m, fabsf(xs[c][t]));
+        float Sg = Sg_t;
+        if (GS == kGsRow) {
+          Sg = global_scale_from_amax(o < D ? __uint_as_float(gs_cells[o]) : 0.0f);
+          if (o < D && k0 == 0) gscale[o] = Sg;
+        }
+        float rcp;
+        const uint32_t sb = block_scale(m, Sg, rcp, RMODE == 2);
+        if (TBT == 4) {
+          my_sf[(2u * j + c) * 4u + tb] = (uint8_t)sb;
+        } else if (o < D) {
+          const uint32_t bk = k0 >> 4;
+          const size_t off1 = TILED ? (size_t)((o >> 7) * (((nb + 15u) & ~15u) >> 2) + (bk >> 2)) * 512u +
+                                          ((o & 31u) * 16u + ((o >> 5) & 3u) * 4u + (bk & 3u))
+                                    : (size_t)o * nb + bk;
+          sf[off1] = (uint8_t)sb;
+        }
+        const uint2 packed = quantize_block16<SR>(xs[c], rcp, pk, stream_id, ((uint64_t)o * K16 + k0) >> 3);
+        if (o < D) *reinterpret_cast<uint2*>(codes + (size_t)o * (Kp >> 1) + (k0 >> 1)) = packed;
+      }
+    }
+  }
+  if (TBT != 4) return;
+  // (the strip is private to the thread: its own byte stores are ordered before its word loads)
+  const uint32_t b = k_start >> 4;
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    const uint32_t o = d0 + c;
+    if (o < D) {
+      const size_t off = TILED ? (size_t)((o >> 7) * (((nb + 15u) & ~15u) >> 2) + (b >> 2)) * 512u + ((o & 31u) * 16u + ((o >> 5) & 3u) * 4u)
+                               : (size_t)o * nb + b;
+      *reinterpret_cast<uint32_t*>(sf + off) = *reinterpret_cast<const uint32_t*>(my_sf + 4 * c);
+    }
+  }
+}
+
 // =========================================================================================================
 // Host-side launchers
 // =========================================================================================================
@@ -1683,10 +1826,40 @@ static bool cols4_path(const QuantTransposeArgs& a) {
          a.D < ((int64_t)1 << 31) - 64;
 }
 
+// ... and its counterpart for a forward operand as the source, from 8 M elements on (smaller operands, such as a layer's
+// weights, do not fill the chip with its 128 x 128 tiles of 128 threads and stay with the staged kernel).
+static bool cols8_path(const QuantTransposeArgs& a) {
+  const TransposeSrc& s = a.src;
+  return a.rowsK * a.D >= ((int64_t)8 << 20) && !a.rht_stream && !s.out_rows && !s.closed_form_sg && !s.row_map && s.in_K < ((int64_t)1 << 31) - 128 &&
+         a.rowsK < ((int64_t)1 << 31) - 1024 && a.D < ((int64_t)1 << 31) - 128;
+}
+
 template <int SRC, int GS, int RMODE>
 static cudaError_t launch_tr_t(const QuantTransposeArgs& a, cudaStream_t st) {
   const dim3 grid(blocks_for(a.rowsK, 128), blocks_for(a.D, 64));
   const bool fast = transpose_fast_path(a.src, SRC);
+  if constexpr (SRC == 1 && GS != kGsBlock128) {
+    if (cols8_path(a)) {
+      // 512 x 128 tiles when they fill the chip about twice over, else 128 x 128 tiles
+      const bool big = (int64_t)blocks_for(a.rowsK, 512) * blocks_for(a.D, 128) >= 8 * (int64_t)device_sm_count();
+      const dim3 g8(blocks_for(a.rowsK, big ? 512 : 128), blocks_for(a.D, 128));
+      const bool uniform = a.src.in_gs_mode == kGsTensor;
+      const PhiloxKeys keys = make_philox_keys(a.seed);
+#define NVFP4_LAUNCH_C8(TILED_, UNI_, TBT_)                                                                                          \
+  launch_kernel(requantize_cols8_kernel<GS, RMODE, TILED_, UNI_, TBT_>, g8, dim3(128), 0, st, a.src, (uint32_t)a.rowsK,                \
+                (uint32_t)a.D, a.stream_id, (const uint32_t*)a.gs_cells, a.tensor_closed_form, a.codes, a.sf, a.gscale, keys)
+#define NVFP4_LAUNCH_C8B(TILED_, UNI_)                                                                                               \
+  if (big) NVFP4_LAUNCH_C8(TILED_, UNI_, 4); else NVFP4_LAUNCH_C8(TILED_, UNI_, 1)
+      if (a.sf_tiled) {
+        if (uniform) { NVFP4_LAUNCH_C8B(true, true); } else { NVFP4_LAUNCH_C8B(true, false); }
+      } else {
+        if (uniform) { NVFP4_LAUNCH_C8B(false, true); } else { NVFP4_LAUNCH_C8B(false, false); }
+      }
+#undef NVFP4_LAUNCH_C8B
+#undef NVFP4_LAUNCH_C8
+      return cudaGetLastError();
+    }
+  }
   if constexpr (SRC == 0) {
     if (cols4_path(a)) {
       const PhiloxKeys keys = make_philox_keys(a.seed);

@@ -195,3 +195,28 @@ def test_variants_at_the_qkv_size():
     A64 = np.concatenate([orc.dequantize(q1), f8.snap(X[:, outl])[0].astype(np.float64)], axis=1)
     B64 = np.concatenate([orc.dequantize(q2), f8.snap(W[:, outl])[0].astype(np.float64)], axis=1)
     check_sampled(Y8, A64, B64, rng, True, "Y with FP8 outlier channels")
+
+
+@pytest.mark.parametrize("case", [
+    # (source rows = operand k, source columns = operand rows, scale mode, source scale layout, rounding)
+    (4100, 2100, 0, 1, 1),   # 8.6 M elements, 128 x 128 CTA tiles; ragged in rows (inside a 16-block) and in columns (not a multiple of 8)
+    (4100, 2100, 1, 0, 2),   # ROW scales of source and result, linear source scale layout, rounded-up block scales
+    (16400, 9300, 0, 1, 1),  # 153 M elements: 512 x 128 CTA tiles, ragged in both directions
+    (16400, 9300, 1, 1, 1),
+])
+def test_register_transposing_requantizer_on_large_ragged_operands(case):
+    """Q4 / Q6 from 8 M elements on take the kernel that transposes in registers (smaller operands keep the staged kernel, which
+    the small-shape tests cover): both of its tile sizes, both scale modes it handles, bit for bit."""
+    b = B()
+    rows, cols, gs_mode, in_layout, rounding = case
+    x, _ = synth.activations(rows, cols, 400 + rows, n_outlier=5, factor=40.0)
+    cols8 = (cols + 7) // 8 * 8
+    full = np.zeros((rows, cols8), dtype=np.float32)
+    full[:, :cols] = x
+    fwd_ref = orc.quantize(x, orc.AXIS_ROW, orc.RTN, gs_mode)
+    ref = orc.quantize(orc.rematerialize_f32(fwd_ref), orc.AXIS_COL, rounding, gs_mode, seed=17, stream_id=6)
+    fwd = b.nvfp4_quantize(to_dev_bf16(full)[:, :cols], b.AXIS_ROW, b.ROUND_RTN, 0, 1, gs_mode, in_layout)
+    assert_operand_equal(fwd, fwd_ref, f"forward operand {case}")
+    out = b.alloc_operand(cols, rows, gs_mode, poison=True)
+    b.nvfp4_requantize_t(fwd, rounding, 17, 6, out=out)
+    assert_operand_equal(out, ref, f"requantize_t {case}")
