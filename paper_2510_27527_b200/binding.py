@@ -116,6 +116,7 @@ EXPORTS = {
 MEASURE_EXPORTS = {
     "nvfp4_launch_count": (ctypes.c_longlong, []),
     "nvfp4_mma_issue_probe": (c_i32, [c_i32, c_vp, ctypes.POINTER(ctypes.c_double), c_vp]),
+    "nvfp4_mma_issue_probe_n": (c_i32, [c_i32, c_i32, c_i32, c_i32, c_i32, c_i32, c_vp, c_vp, ctypes.POINTER(ctypes.c_double), c_vp]),
 }
 for _name, (_res, _args) in list(EXPORTS.items()) + [("nvfp4_launch_count", MEASURE_EXPORTS["nvfp4_launch_count"])]:
     _f = getattr(_lib, _name)
@@ -134,9 +135,10 @@ def measure_lib():
         if not os.path.exists(MEASURE_LIB_PATH):
             raise ImportError(f"{MEASURE_LIB_PATH} is missing: build it with `python -m paper_2510_27527_b200.build`")
         _measure_lib = ctypes.CDLL(MEASURE_LIB_PATH)
-        res, args = MEASURE_EXPORTS["nvfp4_mma_issue_probe"]
-        _measure_lib.nvfp4_mma_issue_probe.restype = res
-        _measure_lib.nvfp4_mma_issue_probe.argtypes = args
+        for name in ("nvfp4_mma_issue_probe", "nvfp4_mma_issue_probe_n"):
+            res, args = MEASURE_EXPORTS[name]
+            getattr(_measure_lib, name).restype = res
+            getattr(_measure_lib, name).argtypes = args
     return _measure_lib
 
 
@@ -340,10 +342,16 @@ def nvfp4_outlier_select(acc: torch.Tensor, n_out: int):
     return outl, keep, cmap
 
 
-def nvfp4_mma_issue_probe(iters: int, dev_status: torch.Tensor | None = None) -> float:
-    """Enqueues the tensor-core issue loop (no memory traffic); returns the FP4 flops the launch performs."""
+def nvfp4_mma_issue_probe(iters: int, dev_status: torch.Tensor | None = None, n: int = 256, side_warps: int = 0,
+                          side_kind: int = 0, random_data: bool = False, dev_bytes_moved: torch.Tensor | None = None,
+                          loop_kind: int = 0) -> float:
+    """Enqueues the tensor-core issue loop (instructions of M = 128, N = n, K = 64; side_warps further warps per SM storing to
+    shared memory (side_kind 0), loading the accumulator (1) or bulk-copying from L2 into shared memory (2) meanwhile, their
+    bytes added to the int64 device counters dev_bytes_moved[0], loop cycles to [1]; loop_kind 1 adds the scale copies of a GEMM
+    to every group of four MMAs, 2 a commit as well); returns the FP4 flops the launch performs."""
     fl = ctypes.c_double(0.0)
-    _check(measure_lib().nvfp4_mma_issue_probe(iters, _ptr(dev_status), ctypes.byref(fl), _stream_ptr()), "nvfp4_mma_issue_probe")
+    _check(measure_lib().nvfp4_mma_issue_probe_n(iters, n, loop_kind, side_warps, side_kind, int(random_data), _ptr(dev_status),
+                                                 _ptr(dev_bytes_moved), ctypes.byref(fl), _stream_ptr()), "nvfp4_mma_issue_probe_n")
     return fl.value
 
 

@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(binding):
     assert declared == set(binding.EXPORTS)
     # the measurement aids: the launch counter in the main library, the issue loop in a library of its own
     aids = _declared("nvfp4_measure.h")
-    assert aids == set(binding.MEASURE_EXPORTS) == {"nvfp4_launch_count", "nvfp4_mma_issue_probe"}
+    assert aids == set(binding.MEASURE_EXPORTS) == {"nvfp4_launch_count", "nvfp4_mma_issue_probe", "nvfp4_mma_issue_probe_n"}
     assert hasattr(binding.lib, "nvfp4_launch_count") and not hasattr(binding.lib, "nvfp4_mma_issue_probe")
     assert hasattr(binding.measure_lib(), "nvfp4_mma_issue_probe")
     # headers of the include directory are exactly these two
