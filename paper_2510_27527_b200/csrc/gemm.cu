@@ -224,16 +224,14 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
   if (warp == 0) {
     // ===================================== TMA producer (warp stays converged) ===============================
     const uint32_t leader = elect_leader();
-    uint32_t it = 0;
+    uint32_t it = 0, s = 0, wait_parity = 1;  // running stage and the parity its "empty" barrier is waited with
     bool ok = true;
     for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
       const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
       const uint8_t* sfa_src = p.a_sf + (size_t)mt * p.sf_tiles_a * 512;
       const uint8_t* sfb_src = p.b_sf + (size_t)nt * p.sf_tiles_b * 512;
-      for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
-        const int s = it % C::STAGES;
-        const uint32_t round = it / C::STAGES;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), (round & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
+      for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it, s = (s + 1 == (uint32_t)C::STAGES ? 0u : s + 1), wait_parity ^= (s == 0)) {
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), wait_parity, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
         // (test hook of the bounded waits: with `starve` the very first stage never completes)
@@ -244,9 +242,8 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         bulk_load(st + A_BYTES + C::B_BYTES + SFA_BYTES, sfb_src + (size_t)kt * 2048, 2048, full_bar(s), leader);
       }
       // OutControl: the BF16 outlier channels of both operands, 64 per stage, into the same stage buffers
-      for (int32_t h = 0; h < p.hp_k_tiles && ok; ++h, ++it) {
-        const int s = it % C::STAGES;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / C::STAGES) & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
+      for (int32_t h = 0; h < p.hp_k_tiles && ok; ++h, ++it, s = (s + 1 == (uint32_t)C::STAGES ? 0u : s + 1), wait_parity ^= (s == 0)) {
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), wait_parity, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         const uint32_t st = smem_base + s * C::STAGE_BYTES;
         mbar_expect_tx(full_bar(s), A_BYTES + C::B_BYTES, leader);
@@ -268,8 +265,17 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     // ===================================== MMA issuer (warp stays converged) =================================
     const uint32_t leader = elect_leader();
     const uint32_t idesc = instr_desc<BN>();
-    uint32_t it = 0, tile_it = 0;
+    // The issuing warp's own instruction stream is what limits a 128 x 128 tile (13 tensor-core instructions per 256 cycles of
+    // math), so the loop keeps it short: running stage / phase counters instead of divisions, descriptors formed by adding
+    // to the low word of the first stage's (an address enters as address >> 4 in the low 14 bits; the high words are
+    // constants), and the try on the NEXT stage's barrier issued before this stage's instructions so that its latency
+    // overlaps them.
+    uint32_t it = 0, tile_it = 0, stage = 0, phase = 0;
     bool ok = true;
+    bool ready = false;
+    constexpr uint32_t SW_HI = (uint32_t)((((uint64_t)64 << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61)) >> 32);
+    constexpr uint32_t SF_HI = (uint32_t)((((uint64_t)8 << 32) | ((uint64_t)1 << 46)) >> 32);
+    const uint32_t a_lo0 = (uint32_t)desc_sw128(smem_base), sfa_lo0 = (uint32_t)desc_sf(smem_base + A_BYTES + C::B_BYTES);
     for (int64_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
       const uint32_t ab = tile_it % C::ACC_BUFS;
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar(ab), ((tile_it / C::ACC_BUFS) & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
@@ -277,24 +283,32 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + ab * C::ACC_COLS;
       for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
-        const int s = it % C::STAGES;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / C::STAGES) & 1, abort_flag, p.dev_status, p.wait_limit));
-        if (!ok) break;
+        if (!ready) {
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(stage), phase, abort_flag, p.dev_status, p.wait_limit));
+          if (!ok) break;
+        }
         tc_fence_after();
-        const uint32_t st = smem_base + s * C::STAGE_BYTES;
+        const uint32_t st16 = stage * (uint32_t)(C::STAGE_BYTES >> 4);
+        const uint32_t this_empty = empty_bar(stage);
+        if (++stage == (uint32_t)C::STAGES) {
+          stage = 0;
+          phase ^= 1u;
+        }
+        const uint32_t next_try = mbar_test(full_bar(stage), phase);
         const uint32_t sf_tmem = tmem_base + sf_tmem_col + (it & 3) * C::SF_COLS;
         // Scales of this k tile: shared memory -> tensor memory. Per 64-wide k step: 4 columns for the 128 rows
         // of A, 4 per 128 rows of B.
 #pragma unroll
         for (int kk = 0; kk < BK / 64; ++kk) {
-          tc_cp_sf(sf_tmem + kk * 4, desc_sf(st + A_BYTES + C::B_BYTES + kk * 512), leader);
-          tc_cp_sf(sf_tmem + 16 + kk * 4, desc_sf(st + A_BYTES + C::B_BYTES + SFA_BYTES + kk * 512), leader);
+          tc_cp_sf(sf_tmem + kk * 4, ((uint64_t)SF_HI << 32) | (sfa_lo0 + st16 + kk * 32), leader);
+          tc_cp_sf(sf_tmem + 16 + kk * 4, ((uint64_t)SF_HI << 32) | (sfa_lo0 + st16 + (SFA_BYTES >> 4) + kk * 32), leader);
         }
 #pragma unroll
         for (int kk = 0; kk < BK / 64; ++kk)
-          tc_mma_nvf4(d_tmem, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc, sf_tmem + kk * 4,
-                      sf_tmem + 16 + kk * 4, (kt | kk) != 0, leader);
-        tc_commit(empty_bar(s), leader);  // stage reusable once these MMAs have read it
+          tc_mma_nvf4(d_tmem, ((uint64_t)SW_HI << 32) | (a_lo0 + st16 + kk * 2), ((uint64_t)SW_HI << 32) | (a_lo0 + st16 + (A_BYTES >> 4) + kk * 2),
+                      idesc, sf_tmem + kk * 4, sf_tmem + 16 + kk * 4, (kt | kk) != 0, leader);
+        tc_commit(this_empty, leader);  // stage reusable once these MMAs have read it
+        ready = __all_sync(0xFFFFFFFFu, next_try);
       }
       if (p.hp_k_tiles > 0 && ok) {
         // high-precision side product into its own accumulator (single buffer: wait until the previous tile's epilogue
@@ -304,16 +318,24 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         tc_fence_after();
         const uint32_t idesc_bf16 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
         for (int32_t h = 0; h < p.hp_k_tiles; ++h, ++it) {
-          const int s = it % C::STAGES;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / C::STAGES) & 1, abort_flag, p.dev_status, p.wait_limit));
-          if (!ok) break;
+          if (!ready) {
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(stage), phase, abort_flag, p.dev_status, p.wait_limit));
+            if (!ok) break;
+          }
           tc_fence_after();
-          const uint32_t st = smem_base + s * C::STAGE_BYTES;
+          const uint32_t st = smem_base + stage * C::STAGE_BYTES;
+          const uint32_t this_empty = empty_bar(stage);
+          if (++stage == (uint32_t)C::STAGES) {
+            stage = 0;
+            phase ^= 1u;
+          }
+          const uint32_t next_try = mbar_test(full_bar(stage), phase);
 #pragma unroll
           for (int kk = 0; kk < 4; ++kk)  // 64 BF16 = one 128-byte swizzle row = four K = 16 steps of 32 bytes
             tc_mma_bf16(tmem_base + hp_tmem_col, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc_bf16,
                         (h | kk) != 0, leader);
-          tc_commit(empty_bar(s), leader);
+          tc_commit(this_empty, leader);
+          ready = __all_sync(0xFFFFFFFFu, next_try);
         }
         if (!ok) break;
       }
@@ -851,13 +873,16 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
 //   - tcgen05.commit multicasts the "stage free" / "accumulator ready" arrivals to the same barrier in both CTAs;
 //   - both CTAs' epilogue warps arrive on the leader's "accumulator free" barrier (a remote arrive for the peer).
 // No load uses cluster multicast. Accumulator: 128 lanes x 256 columns per CTA, drained into registers by eight
-// epilogue warps before it is handed back (see the 128 x 256 variant above).
+// epilogue warps, which hand it back at once and then scale, stage 128-byte row pieces in shared memory (one 4 KB buffer
+// per warp, 128-byte swizzle) and let the bulk-tensor engine write them as full lines while the next tile's MMAs run
+// (plain 16-byte stores from the registers, a lane per row, cost 16384 x 3072 x 1024 with FP32 output 112 instead of 56 us).
 // =========================================================================================================
 constexpr int C2_STAGES = 5;
 constexpr uint32_t C2_B_BYTES = 16384;                                  // this CTA's 128 rows of the B tile
 constexpr uint32_t C2_SFB_BYTES = 4096;                                 // scales of all 256 B rows
 constexpr uint32_t C2_STAGE_BYTES = A_BYTES + C2_B_BYTES + SFA_BYTES + C2_SFB_BYTES;  // 38 KB
-constexpr uint32_t C2_SMEM_BYTES = C2_STAGES * C2_STAGE_BYTES + 1024 + 256;
+constexpr uint32_t C2_STAGING_BYTES = 8 * 4096;
+constexpr uint32_t C2_SMEM_BYTES = C2_STAGES * C2_STAGE_BYTES + C2_STAGING_BYTES + 1024 + 256;
 constexpr int C2_THREADS = 64 + 256;
 constexpr uint32_t C2_SF_COLS = 16 + 32;
 
@@ -911,14 +936,65 @@ __device__ __forceinline__ void tc2_mma_nvf4(uint32_t d_tmem, uint64_t a_desc, u
       : "memory");
 }
 
+// One 128-byte-wide piece (W = 32 FP32 or 64 BF16 columns) of a warp's 32 output rows, values final except for the old C:
+// accumulate, then either plain stores (a chunk that sticks out past N) or a swizzled copy into the warp's 4 KB staging
+// buffer that the bulk-tensor engine writes as full lines. m0 is the first of the 32 rows, m this lane's row.
+template <int W>
+__device__ __forceinline__ void stage_and_store(const Params& p, const CUtensorMap* tmC, uint32_t buf, int lane, int64_t m, int64_t m0,
+                                                int64_t n0, float (&o)[W]) {
+  if (p.accumulate && m < p.M) {
+    if (n0 + W <= p.N) {
+      add_existing<W>(p, m, n0, o);
+    } else if (p.c_is_f32) {
+#pragma unroll
+      for (int j = 0; j < W; ++j)
+        if (n0 + j < p.N) o[j] += reinterpret_cast<const float*>(p.C)[m * p.ldc + n0 + j];
+    } else {
+#pragma unroll
+      for (int j = 0; j < W; ++j)
+        if (n0 + j < p.N) o[j] += __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.C)[m * p.ldc + n0 + j]);
+    }
+  }
+  if (n0 + W > p.N) {  // ragged last chunk of the row
+    if (m < p.M) store_ragged<W>(p, m, n0, o);
+    return;
+  }
+  if (lane == 0) bulk_wait_read<0>();  // the previous store from this buffer has read it
+  __syncwarp();
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    uint32_t q[4];
+    if (W == 32) {
+#pragma unroll
+      for (int h = 0; h < 4; ++h) q[h] = __float_as_uint(o[4 * j + h]);
+    } else {
+#pragma unroll
+      for (int h = 0; h < 4; ++h) {
+        const __nv_bfloat162 hh = __floats2bfloat162_rn(o[(8 * j + 2 * h) % W], o[(8 * j + 2 * h + 1) % W]);
+        q[h] = *reinterpret_cast<const uint32_t*>(&hh);
+      }
+    }
+    const uint32_t dst = buf + (uint32_t)lane * 128u + (uint32_t)((j ^ (lane & 7)) << 4);
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(q[0]), "r"(q[1]), "r"(q[2]), "r"(q[3]) : "memory");
+  }
+  fence_async_smem();
+  __syncwarp();
+  if (lane == 0) {
+    tma_store_2d(tmC, buf, (int32_t)n0, (int32_t)m0);
+    bulk_commit();
+  }
+}
+
 template <int GS>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(C2_THREADS, 1)
 gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                       const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB, const Params p) {
+                       const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB,
+                       const __grid_constant__ CUtensorMap tmC, const Params p) {
   constexpr int STAGES = C2_STAGES;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = smem_base + STAGES * C2_STAGE_BYTES;
+  const uint32_t staging_base = smem_base + STAGES * C2_STAGE_BYTES;  // eight 4 KB buffers, one per epilogue warp
+  const uint32_t bar_base = staging_base + C2_STAGING_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };             // used in the leader CTA only
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };  // one per CTA
   const uint32_t acc_full_bar = bar_base + 8u * (2 * STAGES);            // one per CTA
@@ -959,16 +1035,15 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   if (warp == 0) {
     // ===================================== TMA producer (both CTAs) ========================================
     const uint32_t leader = elect_leader();
-    uint32_t it = 0;
+    uint32_t it = 0, s = 0, wait_parity = 1;
     bool ok = true;
     for (int64_t t = pair; t < num_tiles && ok; t += num_pairs) {
       const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
       const int32_t a_row = mt * 256 + (int32_t)rank * 128, b_row = nt * 256 + (int32_t)rank * 128;
       const int32_t sfa_row = ((mt * 2 + (int32_t)rank) * p.sf_tiles_a) * 4;  // in units of 128 bytes
       const int32_t sfb_row0 = ((nt * 2) * p.sf_tiles_b) * 4, sfb_row1 = ((nt * 2 + 1) * p.sf_tiles_b) * 4;
-      for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
-        const int s = it % STAGES;
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), ((it / STAGES) & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
+      for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it, s = (s + 1 == (uint32_t)STAGES ? 0u : s + 1), wait_parity ^= (s == 0)) {
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), wait_parity, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         const uint32_t st = smem_base + s * C2_STAGE_BYTES;
         const uint32_t full0 = map_to_cta(full_bar(s), 0);
@@ -992,30 +1067,44 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     if (rank == 0) {
       const uint32_t leader = elect_leader();
       const uint32_t idesc = (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-      uint32_t it = 0, tile_it = 0;
+      // issue loop kept short as in the 128 x 128 kernel: running stage / phase counters, descriptors by addition to the low
+      // word, the next stage's barrier tried before this stage's instructions
+      uint32_t it = 0, tile_it = 0, stage = 0, phase = 0;
       bool ok = true;
+      bool ready = false;
+      constexpr uint32_t SW_HI = (uint32_t)((((uint64_t)64 << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61)) >> 32);
+      constexpr uint32_t SF_HI = (uint32_t)((((uint64_t)8 << 32) | ((uint64_t)1 << 46)) >> 32);
+      const uint32_t a_lo0 = (uint32_t)desc_sw128(smem_base), sfa_lo0 = (uint32_t)desc_sf(smem_base + A_BYTES + C2_B_BYTES);
       for (int64_t t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
         ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar, (tile_it & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         tc_fence_after();
         for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
-          const int s = it % STAGES;
-          ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(s), (it / STAGES) & 1, abort_flag, p.dev_status, p.wait_limit));
-          if (!ok) break;
+          if (!ready) {
+            ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(stage), phase, abort_flag, p.dev_status, p.wait_limit));
+            if (!ok) break;
+          }
           tc_fence_after();
-          const uint32_t st = smem_base + s * C2_STAGE_BYTES;
+          const uint32_t st16 = stage * (uint32_t)(C2_STAGE_BYTES >> 4);
+          const uint32_t this_empty = empty_bar(stage);
+          if (++stage == (uint32_t)STAGES) {
+            stage = 0;
+            phase ^= 1u;
+          }
+          const uint32_t next_try = mbar_test(full_bar(stage), phase);
           const uint32_t sf_tmem = tmem_base + 256 + (it & 3) * C2_SF_COLS;
 #pragma unroll
           for (int kk = 0; kk < BK / 64; ++kk) {
-            tc2_cp_sf(sf_tmem + kk * 4, desc_sf(st + A_BYTES + C2_B_BYTES + kk * 512), leader);
-            tc2_cp_sf(sf_tmem + 16 + kk * 8, desc_sf(st + A_BYTES + C2_B_BYTES + SFA_BYTES + kk * 512), leader);
-            tc2_cp_sf(sf_tmem + 16 + kk * 8 + 4, desc_sf(st + A_BYTES + C2_B_BYTES + SFA_BYTES + 2048 + kk * 512), leader);
+            tc2_cp_sf(sf_tmem + kk * 4, ((uint64_t)SF_HI << 32) | (sfa_lo0 + st16 + kk * 32), leader);
+            tc2_cp_sf(sf_tmem + 16 + kk * 8, ((uint64_t)SF_HI << 32) | (sfa_lo0 + st16 + (SFA_BYTES >> 4) + kk * 32), leader);
+            tc2_cp_sf(sf_tmem + 16 + kk * 8 + 4, ((uint64_t)SF_HI << 32) | (sfa_lo0 + st16 + ((SFA_BYTES + 2048) >> 4) + kk * 32), leader);
           }
 #pragma unroll
           for (int kk = 0; kk < BK / 64; ++kk)
-            tc2_mma_nvf4(tmem_base, desc_sw128(st + kk * 32), desc_sw128(st + A_BYTES + kk * 32), idesc, sf_tmem + kk * 4,
-                         sf_tmem + 16 + kk * 8, (kt | kk) != 0, leader);
-          tc2_commit_both(empty_bar(s), leader);
+            tc2_mma_nvf4(tmem_base, ((uint64_t)SW_HI << 32) | (a_lo0 + st16 + kk * 2), ((uint64_t)SW_HI << 32) | (a_lo0 + st16 + (A_BYTES >> 4) + kk * 2),
+                         idesc, sf_tmem + kk * 4, sf_tmem + 16 + kk * 8, (kt | kk) != 0, leader);
+          tc2_commit_both(this_empty, leader);
+          ready = __all_sync(0xFFFFFFFFu, next_try);
         }
         if (ok) tc2_commit_both(acc_full_bar, leader);
       }
@@ -1054,22 +1143,38 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
+      // The accumulator is free again (the pair's next tile may start); scale, stage and store from the registers.
+      const uint32_t my_stage = staging_base + (uint32_t)(warp - 2) * 4096u;
+      const int64_t m0 = (int64_t)mt * 256 + rank * 128 + quad * 32;
+      if (m0 >= p.M) continue;
+      if (p.c_is_f32) {
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int64_t n0 = (int64_t)nt * 256 + half * 128 + q * 32;
-        if (m < p.M && n0 < p.N) {
+        for (int q = 0; q < 4; ++q) {
+          const int64_t n0 = (int64_t)nt * 256 + half * 128 + q * 32;
+          if (n0 >= p.N) break;
           float o[32], sgb[32];
           if (GS == kGsRow) load_sgb32(p.b_gscale, n0, p.N, sgb);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            float sc = alpha;
-            if (GS == kGsRow) sc = __fmul_rn(sa, sgb[j]);
-            o[j] = __uint_as_float(v[q][j]) * sc;
-          }
-          store_row_chunk(p, m, n0, o);
+          for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(v[q][j]) * (GS == kGsRow ? __fmul_rn(sa, sgb[j]) : alpha);
+          stage_and_store<32>(p, &tmC, my_stage, lane, m, m0, n0, o);
+        }
+      } else {
+#pragma unroll
+        for (int qq = 0; qq < 2; ++qq) {
+          const int64_t n0 = (int64_t)nt * 256 + half * 128 + qq * 64;
+          if (n0 >= p.N) break;
+          float o[64], sgb[32];
+          if (GS == kGsRow) load_sgb32(p.b_gscale, n0, p.N, sgb);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(v[2 * qq][j]) * (GS == kGsRow ? __fmul_rn(sa, sgb[j]) : alpha);
+          if (GS == kGsRow) load_sgb32(p.b_gscale, n0 + 32, p.N, sgb);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[32 + j] = __uint_as_float(v[2 * qq + 1][j]) * (GS == kGsRow ? __fmul_rn(sa, sgb[j]) : alpha);
+          stage_and_store<64>(p, &tmC, my_stage, lane, m, m0, n0, o);
         }
       }
     }
+    if (lane == 0) bulk_wait_all();  // this lane's bulk stores are complete before the CTA may exit
   }
 
   // ===================================== teardown ============================================================
@@ -1324,9 +1429,10 @@ cudaError_t launch_2cta(const GemmArgs& a, cudaStream_t st) {
   const int64_t Kp = (a.K + 127) & ~(int64_t)127;
   const int64_t kb_padded = ((Kp >> 4) + 15) & ~(int64_t)15;
   const int64_t sfa_bytes = ((a.M + 127) / 128) * 128 * kb_padded, sfb_bytes = ((a.N + 127) / 128) * 128 * kb_padded;
-  CUtensorMap tmA, tmB, tmSFA, tmSFB;
+  CUtensorMap tmA, tmB, tmSFA, tmSFB, tmC;
   if (!make_codes_map(&tmA, a.a_codes, a.M, Kp, 128) || !make_codes_map(&tmB, a.b_codes, a.N, Kp, 128) ||
-      !make_sf_map(&tmSFA, a.a_sf, sfa_bytes) || !make_sf_map(&tmSFB, a.b_sf, sfb_bytes))
+      !make_sf_map(&tmSFA, a.a_sf, sfa_bytes) || !make_sf_map(&tmSFB, a.b_sf, sfb_bytes) ||
+      !make_c_map(&tmC, a.C, a.M, a.N, a.ldc, a.c_is_f32 != 0))
     return cudaErrorInvalidValue;
   Params p{};
   p.a_sf = a.a_sf;
@@ -1350,7 +1456,7 @@ cudaError_t launch_2cta(const GemmArgs& a, cudaStream_t st) {
   if (e != cudaSuccess) return e;
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned pairs = (unsigned)std::min<int64_t>(tiles, sm_count() / 2);
-  launch_kernel(gemm_nvfp4_2cta_kernel<GS>, dim3(2 * pairs), dim3(C2_THREADS), C2_SMEM_BYTES, st, tmA, tmB, tmSFA, tmSFB, p);
+  launch_kernel(gemm_nvfp4_2cta_kernel<GS>, dim3(2 * pairs), dim3(C2_THREADS), C2_SMEM_BYTES, st, tmA, tmB, tmSFA, tmSFB, tmC, p);
   return cudaGetLastError();
 }
 
@@ -1467,21 +1573,24 @@ cudaError_t launch_dense_gemm(const void* A, const void* B, int64_t M, int64_t N
 size_t gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
 int64_t gemm_block128_max_k() { return (int64_t)B128_MAX_CHUNKS * 128; }
 
-// Variant choice. 128 x 128 single-CTA tiles with two accumulators (a tile's epilogue overlaps the next tile's MMAs) win for
-// short K; pairs of CTAs on 256 x 256 tiles (half the operand traffic per flop and SM, which is what bounds the long-K
-// products: the 128 x 128 kernel pulls 36 KB per k tile and SM out of L2) win once K is long: from K = 4096 when there are
-// two tiles for every pair, from K = 8192 already when half of the pairs get a tile (the weight gradients of a model:
-// few tiles, K = tokens). Measured, FP32 output, 128 x 128 against pairs: 16384 x 1024 x 3072 -> 36.9 / 45.0 us,
-// 8192 x 8192 x 3072 -> 129 / 138, 16384 x 14336 x 4096 -> 541 / 524, 4096 x 8192 x 8192 -> 139 / 110,
-// 3072 x 1024 x 16384 (48 pair tiles) -> 41.1 / 34.8, 2816 x 1024 x 8192 (44) -> 26.6 / 24.6, 2048 x 2048 x 16384 (64) ->
-// 44.9 / 36.8, 1024 x 1024 x 16384 (16) -> 24.6 / 32.8; BF16 output: 16384 x 8192 x 8192 -> 477 / 380.
+// Variant choice. Both kernels are bound by what the L2 delivers to the SMs (about 13 - 16 TB/s over all SMs): the 128 x 128
+// kernel pulls 36 KB per k tile and SM, a pair on a 256 x 256 tile 38 KB per SM for twice the math. The 128 x 128 kernel has
+// two accumulators (a tile's epilogue overlaps the next tile's MMAs entirely); the pair kernel has one and hands it over once
+// its sixteen epilogue warps hold the tile in registers, which costs a few hundred cycles per tile and 256-wide tiles fill
+// the last wave worse. Pairs therefore run from K = 2048 when there are two tiles for every pair, and from K = 8192 already
+// when half of the pairs get a tile (the weight gradients of a model: few tiles, K = tokens). Measured, BF16 / FP32 output,
+// 128 x 128 against pairs, us: 16384 x 3072 x 1024 -> 41.0 / 44.0 and 52.0 / 56.3; 16384 x 1024 x 3072 -> 33.8 / 33.8 and
+// 37.0 / 37.8; 16384 x 3072 x 2048 -> 64.5 / 59.4 and 75.8 / 71.9; 8192 x 8192 x 3072 -> 105.5 / 90.9 and 122.8 / 109.6;
+// 4096 x 4096 x 4096 -> 41.0 / 38.8 and 46.0 / 45.9; 16384 x 14336 x 4096 -> 428 / 373 and 531 / 443; 3072 x 1024 x 16384 (48
+// pair tiles) -> 41.9 / 33.8 and 43.9 / 35.9; 1024 x 1024 x 16384 (16) -> 24.8 / 31.7; 16384 x 8192 x 8192 -> 459 / 370 and
+// 498 / 401.
 // A 256-row tile of an operand spans two 128-row scale tiles, and rows are padded to 128 in the scale layout, so any M, N
 // work. The fused high-precision side product and the outer-block scales live in the single-CTA kernels only.
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;
   if (a.gs_mode == kGsBlock128) return a.variant == 2 ? cudaErrorInvalidValue : launch_block128(a, st);
   const int64_t tiles256 = ((a.M + 255) / 256) * ((a.N + 255) / 256), n_pairs = sm_count() / 2;
-  bool pairs = (a.K >= 4096 && tiles256 >= 2 * n_pairs) || (a.K >= 8192 && 2 * tiles256 >= n_pairs);
+  bool pairs = (a.K >= 2048 && tiles256 >= 2 * n_pairs) || (a.K >= 8192 && 2 * tiles256 >= n_pairs);
   if (a.variant == 1) pairs = false;
   if (a.variant == 2) pairs = true;
   if (a.hp_Kh > 0) {

@@ -18,12 +18,13 @@ constexpr uint32_t PROBE_SCRATCH_PER_WARP = 24576;
 constexpr uint32_t PROBE_BULK_PIECE = 8192;  // three pieces per side warp and round
 constexpr int PROBE_MAX_STORE_WARPS = 6;
 constexpr uint32_t PROBE_SMEM_BYTES = PROBE_SCRATCH_OFFSET + PROBE_MAX_STORE_WARPS * PROBE_SCRATCH_PER_WARP + 1024;
+__device__ __align__(128) uint8_t probe_bulk_sink[PROBE_SCRATCH_PER_WARP];    // what the bulk-store side warps write (all to the same lines)
 __device__ __align__(128) uint8_t probe_bulk_source[PROBE_SCRATCH_PER_WARP];  // what the bulk-copy side warps read (stays in L2)
 constexpr uint32_t PROBE_SIDE_ROUNDS_LIMIT = 1u << 24;  // bounds the side warps' loop whatever happens to the flag
 
-template <int PN, int SIDE>
+template <int PN, int SIDE, int LOOP>
 __global__ void __launch_bounds__(64 + 32 * PROBE_MAX_STORE_WARPS, 1)
-    mma_issue_probe_kernel(int32_t iters, int32_t loop_kind, int32_t random_data, int32_t* dev_status, unsigned long long* dev_bytes_moved) {
+    mma_issue_probe_kernel(int32_t iters, int32_t stage_stride, int32_t random_data, int32_t* dev_status, unsigned long long* dev_bytes_moved) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -32,6 +33,8 @@ __global__ void __launch_bounds__(64 + 32 * PROBE_MAX_STORE_WARPS, 1)
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ volatile int loop_done_s;
+  constexpr int RING = 5;
+  __shared__ __align__(8) uint64_t ring_full_s[RING], ring_empty_s[RING];
   const int warp = threadIdx.x >> 5;
   __shared__ __align__(8) uint64_t side_bar_s[PROBE_MAX_STORE_WARPS];
   // operands: the E2M1 code of 1.0 everywhere (0x22), scales: the E4M3 byte of 1.0 (0x38); or hashed codes (all 16 values,
@@ -51,6 +54,10 @@ __global__ void __launch_bounds__(64 + 32 * PROBE_MAX_STORE_WARPS, 1)
     loop_done_s = 0;
     mbar_init(done_bar, 1);
     mbar_init(group_bar, 1);
+    for (int r = 0; r < RING; ++r) {
+      mbar_init(smem_u32(&ring_full_s[r]), 1);
+      mbar_init(smem_u32(&ring_empty_s[r]), 1);
+    }
     for (int w = 0; w < PROBE_MAX_STORE_WARPS; ++w) mbar_init(smem_u32(&side_bar_s[w]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -65,6 +72,17 @@ __global__ void __launch_bounds__(64 + 32 * PROBE_MAX_STORE_WARPS, 1)
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
   pdl_prologue();
+  if (warp == 0 && LOOP >= 3) {
+    // stand-in for a GEMM's producer: waits for a free stage and declares it full at once (no copy)
+    const uint32_t leader = elect_leader();
+    bool ok = true;
+    for (int32_t it = 0; it < iters && ok; ++it) {
+      const int s = it % RING;
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ring_empty_s[s]), ((it / RING) & 1) ^ 1, &abort_flag_s, dev_status, DEFAULT_WAIT_LIMIT_CYCLES));
+      if (!ok) break;
+      mbar_expect_tx(smem_u32(&ring_full_s[s]), 0, leader);
+    }
+  }
   if (warp == 1) {
     const uint32_t leader = elect_leader();
     const uint32_t idesc = instr_desc<PN>();
@@ -76,23 +94,77 @@ __global__ void __launch_bounds__(64 + 32 * PROBE_MAX_STORE_WARPS, 1)
       tc_cp_sf(sf_tmem + 16 + kk * 8 + 4, desc_sf(sfb + 2048 + kk * 512), leader);
     }
     const long long t_loop = clock64();
+    uint32_t stage = 0, phase = 0;
+    bool next_ready = false;
+    const uint32_t full0 = smem_u32(&ring_full_s[0]), empty0 = smem_u32(&ring_empty_s[0]);
+    // low words of the descriptors of stage 0 (the high words are constants): an address enters as (address >> 4) in the low
+    // 14 bits, so the descriptor of a later stage or k step is one 32-bit addition away
+    const uint32_t a_lo0 = (uint32_t)desc_sw128(a_tile), b_lo0 = (uint32_t)desc_sw128(b_tile);
+    const uint32_t sfa_lo0 = (uint32_t)desc_sf(sfa), sfb_lo0 = (uint32_t)desc_sf(sfb);
+    constexpr uint32_t SW_HI = (uint32_t)(((uint64_t)64 << 32 | (uint64_t)1 << 46 | (uint64_t)2 << 61) >> 32);
+    constexpr uint32_t SF_HI = (uint32_t)(((uint64_t)8 << 32 | (uint64_t)1 << 46) >> 32);
     for (int32_t it = 0; it < iters; ++it) {
-      // loop_kind 0: only the MMAs; 1: the group's scale copies first, as a GEMM issues them (four sets of scale columns in
-      // rotation); 2: and a commit to a barrier after the group, as a GEMM releases its operand stage
-      const uint32_t sf_set = loop_kind ? sf_tmem + (uint32_t)(it & 3) * 48u : sf_tmem;
-      if (loop_kind) {
+      // LOOP 0: only the MMAs; 1: the group's scale copies first, as a GEMM issues them (four sets of scale columns in
+      // rotation); 2: and a commit to a barrier after the group; 3: a five-stage ring with a producer warp that declares a
+      // released stage full at once, stage addresses and barrier waits written as in a straightforward GEMM main loop;
+      // 4: the same ring as the library's GEMMs walk it: running stage / phase counters, descriptors by addition, and a
+      // non-blocking look at the next stage's barrier issued before this stage's instructions
+      const uint32_t sf_set = LOOP ? sf_tmem + (uint32_t)(it & 3) * 48u : sf_tmem;
+      if constexpr (LOOP == 3) {
+        const int sidx = it % RING;
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait(smem_u32(&ring_full_s[sidx]), (it / RING) & 1, &abort_flag_s, dev_status, DEFAULT_WAIT_LIMIT_CYCLES))) break;
+        tc_fence_after();
+        const uint32_t st = (uint32_t)(sidx * stage_stride);  // stage_stride is 0: all stages share the tiles; the compiler cannot know
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
-          tc_cp_sf(sf_set + kk * 4, desc_sf(sfa + kk * 512), leader);
-          tc_cp_sf(sf_set + 16 + kk * 8, desc_sf(sfb + kk * 512), leader);
-          if (PN == 256) tc_cp_sf(sf_set + 16 + kk * 8 + 4, desc_sf(sfb + 2048 + kk * 512), leader);
+          tc_cp_sf(sf_set + kk * 4, desc_sf(sfa + st + kk * 512), leader);
+          tc_cp_sf(sf_set + 16 + kk * 8, desc_sf(sfb + st + kk * 512), leader);
+          if (PN == 256) tc_cp_sf(sf_set + 16 + kk * 8 + 4, desc_sf(sfb + st + 2048 + kk * 512), leader);
         }
-      }
 #pragma unroll
-      for (int kk = 0; kk < 4; ++kk)
-        tc_mma_nvf4(tmem_base, desc_sw128(a_tile + kk * 32), desc_sw128(b_tile + kk * 32), idesc, sf_set + kk * 4,
-                    sf_set + 16 + kk * 8, (it | kk) != 0, leader);
-      if (loop_kind == 2) tc_commit(group_bar, leader);
+        for (int kk = 0; kk < 4; ++kk)
+          tc_mma_nvf4(tmem_base, desc_sw128(a_tile + st + kk * 32), desc_sw128(b_tile + st + kk * 32), idesc, sf_set + kk * 4,
+                      sf_set + 16 + kk * 8, (it | kk) != 0, leader);
+        tc_commit(smem_u32(&ring_empty_s[sidx]), leader);
+      } else if constexpr (LOOP == 4) {
+        if (!next_ready) {
+          if (!__all_sync(0xFFFFFFFFu, mbar_wait(full0 + 8u * stage, phase, &abort_flag_s, dev_status, DEFAULT_WAIT_LIMIT_CYCLES))) break;
+        }
+        tc_fence_after();
+        const uint32_t st16 = stage * (uint32_t)stage_stride;  // in 16-byte units
+        const uint32_t this_empty = empty0 + 8u * stage;
+        if (++stage == (uint32_t)RING) {
+          stage = 0;
+          phase ^= 1;
+        }
+        const uint32_t next_look = mbar_test(full0 + 8u * stage, phase);
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          tc_cp_sf(sf_set + kk * 4, ((uint64_t)SF_HI << 32) | (sfa_lo0 + st16 + kk * 32), leader);
+          tc_cp_sf(sf_set + 16 + kk * 8, ((uint64_t)SF_HI << 32) | (sfb_lo0 + st16 + kk * 32), leader);
+          if (PN == 256) tc_cp_sf(sf_set + 16 + kk * 8 + 4, ((uint64_t)SF_HI << 32) | (sfb_lo0 + st16 + 128 + kk * 32), leader);
+        }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          tc_mma_nvf4(tmem_base, ((uint64_t)SW_HI << 32) | (a_lo0 + st16 + kk * 2), ((uint64_t)SW_HI << 32) | (b_lo0 + st16 + kk * 2), idesc,
+                      sf_set + kk * 4, sf_set + 16 + kk * 8, (it | kk) != 0, leader);
+        tc_commit(this_empty, leader);
+        next_ready = __all_sync(0xFFFFFFFFu, next_look);
+      } else {
+        if constexpr (LOOP >= 1) {
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            tc_cp_sf(sf_set + kk * 4, desc_sf(sfa + kk * 512), leader);
+            tc_cp_sf(sf_set + 16 + kk * 8, desc_sf(sfb + kk * 512), leader);
+            if (PN == 256) tc_cp_sf(sf_set + 16 + kk * 8 + 4, desc_sf(sfb + 2048 + kk * 512), leader);
+          }
+        }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk)
+          tc_mma_nvf4(tmem_base, desc_sw128(a_tile + kk * 32), desc_sw128(b_tile + kk * 32), idesc, sf_set + kk * 4,
+                      sf_set + 16 + kk * 8, (it | kk) != 0, leader);
+        if constexpr (LOOP == 2) tc_commit(group_bar, leader);
+      }
     }
     tc_commit(done_bar, leader);
     __all_sync(0xFFFFFFFFu, mbar_wait(done_bar, 0, &abort_flag_s, dev_status, DEFAULT_WAIT_LIMIT_CYCLES));  // bounded
@@ -127,6 +199,21 @@ __global__ void __launch_bounds__(64 + 32 * PROBE_MAX_STORE_WARPS, 1)
         ++rounds;
       }
       if (keep == 0x12345678u && dev_status) atomicAdd(dev_status, 0);  // keeps the loaded values alive
+    } else if constexpr (SIDE == 3) {  // three bulk stores of 8 KB from the warp's scratch to global (L2) per round
+      per_round = 3ull * PROBE_BULK_PIECE;
+      const uint32_t leader = elect_leader();
+      while (rounds < PROBE_SIDE_ROUNDS_LIMIT && !loop_done_s) {
+#pragma unroll
+        for (int j = 0; j < 3; ++j)
+          asm volatile("{\n.reg .pred q;\nsetp.ne.b32 q, %3, 0;\n@q cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;\n}" ::"l"(
+                           probe_bulk_sink + j * PROBE_BULK_PIECE),
+                       "r"(mine + j * PROBE_BULK_PIECE), "r"(PROBE_BULK_PIECE), "r"(leader)
+                       : "memory");
+        bulk_commit();
+        bulk_wait_read<0>();  // the engine has read the scratch (the global writes may still be in flight)
+        ++rounds;
+      }
+      bulk_wait_all();
     } else {  // three bulk copies of 8 KB from global (L2) into the warp's scratch per round, one barrier phase per round
       per_round = 3ull * PROBE_BULK_PIECE;
       const uint32_t bar = smem_u32(&side_bar_s[warp - 2]);
@@ -157,8 +244,8 @@ __global__ void __launch_bounds__(64 + 32 * PROBE_MAX_STORE_WARPS, 1)
 static int32_t issue_probe(int32_t iters, int32_t n, int32_t loop_kind, int32_t side_warps, int32_t side_kind, int32_t random_data, int32_t* dev_status,
                            unsigned long long* dev_bytes_moved, double* flops_out, void* stream) {
   using namespace nvfp4;
-  if (iters <= 0 || iters > (1 << 20) || (n != 128 && n != 256) || side_warps < 0 || side_warps > PROBE_MAX_STORE_WARPS ||
-      side_kind < 0 || side_kind > 2 || loop_kind < 0 || loop_kind > 2)
+  if (iters <= 0 || iters > (1 << 20) || (n != 128 && n != 256 && n != 32) || side_warps < 0 || side_warps > PROBE_MAX_STORE_WARPS ||
+      side_kind < 0 || side_kind > 3 || loop_kind < 0 || loop_kind > 4)
     return 2;  // NVFP4_ERR_SHAPE
   int dev = 0, major = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
@@ -166,14 +253,17 @@ static int32_t issue_probe(int32_t iters, int32_t n, int32_t loop_kind, int32_t 
     return 7;  // NVFP4_ERR_CUDA
   if (major != 10) return 6;  // NVFP4_ERR_ARCH
   using kernel_t = void (*)(int32_t, int32_t, int32_t, int32_t*, unsigned long long*);
-  static const kernel_t kernels[2][3] = {
-      {mma_issue_probe_kernel<128, 0>, mma_issue_probe_kernel<128, 1>, mma_issue_probe_kernel<128, 2>},
-      {mma_issue_probe_kernel<256, 0>, mma_issue_probe_kernel<256, 1>, mma_issue_probe_kernel<256, 2>}};
-  const kernel_t kernel = kernels[n == 256][side_kind];
+#define PROBE_ROW(N, S) {mma_issue_probe_kernel<N, S, 0>, mma_issue_probe_kernel<N, S, 1>, mma_issue_probe_kernel<N, S, 2>, \
+                         mma_issue_probe_kernel<N, S, 3>, mma_issue_probe_kernel<N, S, 4>}
+  static const kernel_t kernels[3][4][5] = {{PROBE_ROW(128, 0), PROBE_ROW(128, 1), PROBE_ROW(128, 2), PROBE_ROW(128, 3)},
+                                            {PROBE_ROW(256, 0), PROBE_ROW(256, 1), PROBE_ROW(256, 2), PROBE_ROW(256, 3)},
+                                            {PROBE_ROW(32, 0), PROBE_ROW(32, 1), PROBE_ROW(32, 2), PROBE_ROW(32, 3)}};
+#undef PROBE_ROW
+  const kernel_t kernel = kernels[n == 256 ? 1 : n == 32 ? 2 : 0][side_kind][loop_kind];
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PROBE_SMEM_BYTES) != cudaSuccess) return 7;
   if (flops_out) *flops_out = (double)sms * (double)iters * 4.0 * 2.0 * 128.0 * (double)n * 64.0;
   kernel<<<dim3((unsigned)sms), dim3(64 + 32 * (unsigned)side_warps), PROBE_SMEM_BYTES, static_cast<cudaStream_t>(stream)>>>(
-      iters, loop_kind, random_data != 0, dev_status, dev_bytes_moved);
+      iters, /*stage_stride=*/0, random_data != 0, dev_status, dev_bytes_moved);
   return cudaGetLastError() == cudaSuccess ? 0 : 7;
 }
 
