@@ -244,8 +244,16 @@ def measure_large_shapes(b, dev, pk, timer, shapes, gs_names, n_iter):
     probe_flops = b.nvfp4_mma_issue_probe(2048, status)
     sec = timer.median_s(lambda: b.nvfp4_mma_issue_probe(2048, status), 10)
     issue_loop = probe_flops / sec / 1e12 if int(status.item()) == 0 else None
+    # the same loop on hashed operand codes and scales (the arithmetic is the same, the power drawn is not): as a burst of
+    # about the duration of one large GEMM, and held for about 12 ms (the clock the power cap settles at)
+    rnd = {}
+    for name, iters, reps in (("burst", 2048, 10), ("sustained", 32768, 4)):
+        fl_r = b.nvfp4_mma_issue_probe(iters, status, 256, 0, 0, True)
+        sec_r = timer.median_s(lambda: b.nvfp4_mma_issue_probe(iters, status, 256, 0, 0, True), reps)
+        rnd[name] = fl_r / sec_r / 1e12 if int(status.item()) == 0 else None
     fp4_peak = 4.0 * pk["bf16"]
-    out = {"mma_issue_loop_TFLOPs": issue_loop, "fp4_peak_TFLOPs_4x_measured_bf16": fp4_peak, "hbm_peak_GBps": pk["hbm"], "shapes": []}
+    out = {"mma_issue_loop_TFLOPs": issue_loop, "mma_issue_loop_random_data_TFLOPs": rnd, "fp4_peak_TFLOPs_4x_measured_bf16": fp4_peak,
+           "hbm_peak_GBps": pk["hbm"], "shapes": []}
     cache = {}
 
     def operand_source(rows, K, tensor_id):
@@ -274,6 +282,7 @@ def measure_large_shapes(b, dev, pk, timer, shapes, gs_names, n_iter):
                                   "frac_of_4x_bf16_measured": fl / med / 1e12 / fp4_peak,
                                   "frac_of_9PF_nominal": fl / med / 1e12 / 9000.0,
                                   "frac_of_issue_loop": (fl / med / 1e12 / issue_loop) if issue_loop else None,
+                                  "frac_of_issue_loop_random_data_burst": (fl / med / 1e12 / rnd["burst"]) if rnd["burst"] else None,
                                   "bound_us_max_tensor_hbm": max(t_tensor, t_hbm) * 1e6}
 
             def both():

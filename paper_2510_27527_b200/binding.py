@@ -345,10 +345,12 @@ def nvfp4_outlier_select(acc: torch.Tensor, n_out: int):
 def nvfp4_mma_issue_probe(iters: int, dev_status: torch.Tensor | None = None, n: int = 256, side_warps: int = 0,
                           side_kind: int = 0, random_data: bool = False, dev_bytes_moved: torch.Tensor | None = None,
                           loop_kind: int = 0) -> float:
-    """Enqueues the tensor-core issue loop (instructions of M = 128, N = n, K = 64; side_warps further warps per SM storing to
-    shared memory (side_kind 0), loading the accumulator (1) or bulk-copying from L2 into shared memory (2) meanwhile, their
-    bytes added to the int64 device counters dev_bytes_moved[0], loop cycles to [1]; loop_kind 1 adds the scale copies of a GEMM
-    to every group of four MMAs, 2 a commit as well); returns the FP4 flops the launch performs."""
+    """Enqueues the tensor-core issue loop (instructions of M = 128, N = n, K = 64; loop_kind 0 = only MMAs, 1 = with the
+    scale copies of a GEMM, 2 = and a commit per group, 3 / 4 = a five-stage ring walked the straightforward way / as the
+    library's GEMMs walk it; side_warps further warps per SM storing to shared memory (side_kind 0), loading the accumulator
+    (1), bulk-copying from L2 into shared memory (2) or from shared memory to global (3) meanwhile; random_data = hashed
+    operand codes and scales instead of 1.0). dev_bytes_moved: int64[2] device counters, [0] += side bytes, [1] = loop
+    cycles. Returns the FP4 flops the launch performs."""
     fl = ctypes.c_double(0.0)
     _check(measure_lib().nvfp4_mma_issue_probe_n(iters, n, loop_kind, side_warps, side_kind, int(random_data), _ptr(dev_status),
                                                  _ptr(dev_bytes_moved), ctypes.byref(fl), _stream_ptr()), "nvfp4_mma_issue_probe_n")
