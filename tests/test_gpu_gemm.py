@@ -169,3 +169,51 @@ def test_mma_issue_probe_runs_and_reports_its_work():
     assert int(st.item()) == 0
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     assert fl == sms * 8 * 4 * 2.0 * 128 * 256 * 64
+
+
+@pytest.mark.parametrize("n", [32, 128, 256])
+@pytest.mark.parametrize("loop_kind", [0, 1, 2, 3, 4])
+def test_mma_issue_probe_loop_kinds_complete(n, loop_kind):
+    """Every loop structure of the probe (plain, with scale copies, with commits, the two ring walks) drains with status 0,
+    reports the flops of its instruction shape and a plausible cycle count: at least n / 2 cycles per 128 x n x 64 MMA for
+    n >= 128 (the tensor pipe's rate), and not absurdly more."""
+    from paper_2510_27527_b200 import binding as b
+
+    iters = 64
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(2, dtype=torch.int64, device="cuda")
+    fl = b.nvfp4_mma_issue_probe(iters, st, n, 0, 0, loop_kind == 4, cnt, loop_kind)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    assert fl == sms * iters * 4 * 2.0 * 128 * n * 64
+    per_mma = int(cnt[1].item()) / (iters * 4)
+    assert per_mma < 2000
+    if n >= 128:
+        assert per_mma >= 0.9 * n / 2
+    assert int(cnt[0].item()) == 0  # no side warps
+
+
+@pytest.mark.parametrize("side_kind", [0, 1, 2, 3])
+def test_mma_issue_probe_side_warps_count_their_bytes(side_kind):
+    from paper_2510_27527_b200 import binding as b
+
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(2, dtype=torch.int64, device="cuda")
+    b.nvfp4_mma_issue_probe(256, st, 128, 3, side_kind, False, cnt, 1)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    moved = int(cnt[0].item())
+    unit = {0: 4096, 1: 32 * 128 * 4, 2: 3 * 8192, 3: 3 * 8192}[side_kind]
+    assert moved > 0 and moved % unit == 0
+
+
+def test_mma_issue_probe_refuses_values_outside_its_ranges():
+    from paper_2510_27527_b200 import binding as b
+
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for kw in (dict(n=64), dict(loop_kind=5), dict(side_warps=7), dict(side_kind=4)):
+        with pytest.raises(b.Nvfp4Error):
+            b.nvfp4_mma_issue_probe(8, st, **kw)
+    with pytest.raises(b.Nvfp4Error):
+        b.nvfp4_mma_issue_probe(0, st)
