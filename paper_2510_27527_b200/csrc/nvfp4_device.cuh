@@ -231,18 +231,23 @@ __device__ __forceinline__ uint32_t e2m1x8_rtn(const float (&y)[8]) {
 // in below the ones already collected, so that element 0 ends in the lowest nibble.
 __device__ __forceinline__ uint32_t e2m1x8_sr(const float (&y)[8], const uint4& w) {
   const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-  uint32_t out = 0;
+  uint32_t out = 0, u_odd = 0;
 #pragma unroll
   for (int e = 7; e >= 0; --e) {
     // The draw u of element e (the even element is the low half of its word), then c6 = ((0xFFFF - u) << 12) | 0x400007C0
     // = 0x4FFFF7C0 - u * 4096. Multiply-adds are written as such on purpose: the logic / shift / min-max pipe is the one
     // this code saturates (half the rate of the multiply-add pipe), so shifts and adds that can be a multiply-add are one.
-    uint32_t u, c6, v;
-    if (e & 1)
-      asm("mul.hi.u32 %0, %1, 65536;" : "=r"(u) : "r"(ww[e >> 1]));
-    else
-      u = ww[e >> 1] & 0xFFFFu;
-    asm("mad.lo.u32 %0, %1, 0xFFFFF000, 0x4FFFF7C0;" : "=r"(c6) : "r"(u));
+    uint32_t c6, v;
+    if (e & 1) {
+      asm("mul.hi.u32 %0, %1, 65536;" : "=r"(u_odd) : "r"(ww[e >> 1]));
+      asm("mad.lo.u32 %0, %1, 0xFFFFF000, 0x4FFFF7C0;" : "=r"(c6) : "r"(u_odd));
+    } else {
+      // the even element's draw is the low half of the same word: w * -4096 = u_even * -4096 - u_odd * 2^28 (mod 2^32),
+      // so adding u_odd * 2^28 back gives its c6 without a mask (two multiply-adds instead of a logic op and one)
+      uint32_t t;
+      asm("mad.lo.u32 %0, %1, 0xFFFFF000, 0x4FFFF7C0;" : "=r"(t) : "r"(ww[e >> 1]));
+      asm("mad.lo.u32 %0, %1, 0x10000000, %2;" : "=r"(c6) : "r"(u_odd), "r"(t));
+    }
     const float a = fminf(fabsf(y[e]), 6.0f);
     const float z = fmaxf(a, __fmaf_ru(a, 0.5f, 0.5f));
     asm("mad.lo.u32 %0, %1, 64, %2;" : "=r"(v) : "r"(__float_as_uint(z)), "r"(c6));
