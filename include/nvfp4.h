@@ -202,8 +202,9 @@ nvfp4_status nvfp4_requantize_t(const nvfp4_operand* in, const void* hp_bf16, in
  * nvfp4_gemm_ex is the same product with explicit control over what nvfp4_gemm chooses by itself (opts == NULL gives
  * nvfp4_gemm). It exists for tests and for measurements:
  *   variant  AUTO: chosen from the shape. TILE128: one CTA per 128 x 128 output tile, two accumulators. PAIR256: a pair of
- *            CTAs on neighbouring SMs per 256 x 256 tile (cta_group::2; TENSOR and ROW scale modes only, NVFP4_ERR_ENUM
- *            with BLOCK128).
+ *            CTAs on neighbouring SMs per 256 x 256 tile (cta_group::2), one accumulator. PAIR192: the same pair on
+ *            256 x 192 tiles with two accumulators. The pair variants take the TENSOR and ROW scale modes only
+ *            (NVFP4_ERR_ENUM with BLOCK128).
  *   wait_limit_cycles  bound of every device-side wait, in SM clock cycles (0: the default, about two seconds).
  *   starve_first_stage  test hook of the bounded waits: when non-zero, the barrier of the first operand stage expects 16
  *            bytes more than will ever arrive, so the first wait of the MMA warp runs out; the kernel then reports
@@ -213,7 +214,7 @@ size_t nvfp4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
 nvfp4_status nvfp4_gemm(const nvfp4_operand* A, const nvfp4_operand* B, void* C, int32_t c_dtype, int64_t ldc,
                         int32_t accumulate, int32_t* dev_status, void* workspace, size_t ws_bytes, void* stream);
 
-typedef enum { NVFP4_GEMM_AUTO = 0, NVFP4_GEMM_TILE128 = 1, NVFP4_GEMM_PAIR256 = 2 } nvfp4_gemm_variant;
+typedef enum { NVFP4_GEMM_AUTO = 0, NVFP4_GEMM_TILE128 = 1, NVFP4_GEMM_PAIR256 = 2, NVFP4_GEMM_PAIR192 = 3 } nvfp4_gemm_variant;
 typedef struct {
   int32_t variant;           /* nvfp4_gemm_variant */
   int32_t starve_first_stage;

@@ -28,7 +28,7 @@ GS_TENSOR, GS_ROW, GS_BLOCK128 = 0, 1, 2
 SF_LINEAR, SF_TILED128x4 = 0, 1
 DT_BF16, DT_F32 = 0, 1
 OP_FWD, OP_BWD_DX, OP_BWD_DW, OP_BWD = 0, 1, 2, 3
-GEMM_AUTO, GEMM_TILE128, GEMM_PAIR256 = 0, 1, 2
+GEMM_AUTO, GEMM_TILE128, GEMM_PAIR256, GEMM_PAIR192 = 0, 1, 2, 3
 ERR_TIMEOUT = 8
 
 c_i64, c_i32, c_u64, c_u32, c_vp, c_sz = (ctypes.c_int64, ctypes.c_int32, ctypes.c_uint64, ctypes.c_uint32,

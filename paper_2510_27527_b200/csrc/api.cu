@@ -438,8 +438,8 @@ nvfp4_status nvfp4_gemm_ex(const nvfp4_operand* A, const nvfp4_operand* B, void*
                            int32_t accumulate, int32_t* dev_status, const nvfp4_gemm_opts* opts, void* workspace,
                            size_t ws_bytes, void* stream) {
   if (!A || !B || !C) return NVFP4_ERR_NULL;
-  if (opts && (opts->variant < 0 || opts->variant > 2 || opts->wait_limit_cycles < 0 ||
-               (opts->variant == NVFP4_GEMM_PAIR256 && A->gs_mode == NVFP4_GS_BLOCK128)))
+  if (opts && (opts->variant < 0 || opts->variant > 3 || opts->wait_limit_cycles < 0 ||
+               (opts->variant >= NVFP4_GEMM_PAIR256 && A->gs_mode == NVFP4_GS_BLOCK128)))
     return NVFP4_ERR_ENUM;
   nvfp4_status s;
   if ((s = check_operand_ptrs(A)) != NVFP4_OK) return s;

@@ -877,14 +877,29 @@ gemm_nvfp4_block128_kernel(const __grid_constant__ CUtensorMap tmA, const __grid
 // per warp, 128-byte swizzle) and let the bulk-tensor engine write them as full lines while the next tile's MMAs run
 // (plain 16-byte stores from the registers, a lane per row, cost 16384 x 3072 x 1024 with FP32 output 112 instead of 56 us).
 // =========================================================================================================
-constexpr int C2_STAGES = 5;
-constexpr uint32_t C2_B_BYTES = 16384;                                  // this CTA's 128 rows of the B tile
-constexpr uint32_t C2_SFB_BYTES = 4096;                                 // scales of all 256 B rows
-constexpr uint32_t C2_STAGE_BYTES = A_BYTES + C2_B_BYTES + SFA_BYTES + C2_SFB_BYTES;  // 38 KB
-constexpr uint32_t C2_STAGING_BYTES = 8 * 4096;
-constexpr uint32_t C2_SMEM_BYTES = C2_STAGES * C2_STAGE_BYTES + C2_STAGING_BYTES + 1024 + 256;
+// Two tile widths. PN = 256: one accumulator of 256 columns per CTA and four sets of scale columns. PN = 192: two
+// accumulators of 192 columns (a tile's epilogue runs entirely under the next tile's MMAs) and two sets of scale columns;
+// each CTA loads 96 rows of B. A 192-wide tile starts at a multiple of 64 B rows, i.e. possibly in the middle of a 128-row
+// scale tile: the two scale tiles it touches are copied whole and the MMA's scale address starts two columns later (one
+// tensor-memory column holds the scales of 32 rows).
+template <int PN>
+struct Cfg2 {
+  static constexpr int STAGES = 5;
+  static constexpr uint32_t B_ROWS = PN / 2;                                   // this CTA's rows of the B tile
+  static constexpr uint32_t B_BYTES = B_ROWS * 128;
+  static constexpr uint32_t SFB_BYTES = 4096;                                  // scales of the two 128-row scale tiles touched
+  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;  // 38 KB / 34 KB
+  // staging buffers of 4 KB: one per epilogue warp; with 192-wide tiles (room for it) the four warps that own 128 columns
+  // alternate between two, so that a chunk does not wait for the previous chunk's bulk store to have read the buffer
+  static constexpr uint32_t STAGING_BYTES = (PN == 256 ? 8 : 12) * 4096;
+  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 + 256;
+  static constexpr int ACC_BUFS = PN == 256 ? 1 : 2;
+  static constexpr uint32_t SF_COLS = 16 + 32;
+  static constexpr uint32_t SF_SETS = PN == 256 ? 4 : 2;
+  static constexpr uint32_t SF_TMEM_COL = ACC_BUFS * PN;                       // 256 / 384; + SF_SETS * 48 <= 512
+  static constexpr int COLS_HALF0 = 128;                                       // columns the first four epilogue warps own
+};
 constexpr int C2_THREADS = 64 + 256;
-constexpr uint32_t C2_SF_COLS = 16 + 32;
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -939,9 +954,11 @@ __device__ __forceinline__ void tc2_mma_nvf4(uint32_t d_tmem, uint64_t a_desc, u
 // One 128-byte-wide piece (W = 32 FP32 or 64 BF16 columns) of a warp's 32 output rows, values final except for the old C:
 // accumulate, then either plain stores (a chunk that sticks out past N) or a swizzled copy into the warp's 4 KB staging
 // buffer that the bulk-tensor engine writes as full lines. m0 is the first of the 32 rows, m this lane's row.
+// pending: how many of this lane's earlier bulk stores may still be reading shared memory when `buf` is written again (0 with
+// one staging buffer per warp, 1 when the warp alternates between two).
 template <int W>
 __device__ __forceinline__ void stage_and_store(const Params& p, const CUtensorMap* tmC, uint32_t buf, int lane, int64_t m, int64_t m0,
-                                                int64_t n0, float (&o)[W]) {
+                                                int64_t n0, float (&o)[W], int pending = 0) {
   if (p.accumulate && m < p.M) {
     if (n0 + W <= p.N) {
       add_existing<W>(p, m, n0, o);
@@ -959,7 +976,12 @@ __device__ __forceinline__ void stage_and_store(const Params& p, const CUtensorM
     if (m < p.M) store_ragged<W>(p, m, n0, o);
     return;
   }
-  if (lane == 0) bulk_wait_read<0>();  // the previous store from this buffer has read it
+  if (lane == 0) {  // the previous store from this buffer has read it
+    if (pending)
+      bulk_wait_read<1>();
+    else
+      bulk_wait_read<0>();
+  }
   __syncwarp();
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
@@ -985,21 +1007,24 @@ __device__ __forceinline__ void stage_and_store(const Params& p, const CUtensorM
   }
 }
 
-template <int GS>
+template <int GS, int PN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(C2_THREADS, 1)
 gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                        const __grid_constant__ CUtensorMap tmSFA, const __grid_constant__ CUtensorMap tmSFB,
                        const __grid_constant__ CUtensorMap tmC, const Params p) {
-  constexpr int STAGES = C2_STAGES;
+  using C2 = Cfg2<PN>;
+  constexpr int STAGES = C2::STAGES;
+  constexpr uint32_t C2_STAGE_BYTES = C2::STAGE_BYTES, C2_B_BYTES = C2::B_BYTES, C2_SF_COLS = C2::SF_COLS;
+  constexpr int ACC_BUFS = C2::ACC_BUFS;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t staging_base = smem_base + STAGES * C2_STAGE_BYTES;  // eight 4 KB buffers, one per epilogue warp
-  const uint32_t bar_base = staging_base + C2_STAGING_BYTES;
+  const uint32_t bar_base = staging_base + C2::STAGING_BYTES;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };             // used in the leader CTA only
   auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };  // one per CTA
-  const uint32_t acc_full_bar = bar_base + 8u * (2 * STAGES);            // one per CTA
-  const uint32_t acc_empty_bar = bar_base + 8u * (2 * STAGES + 1);       // leader CTA only (16 arrivals)
-  const uint32_t drain_bar = bar_base + 8u * (2 * STAGES + 2);
+  auto acc_full_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };       // one pair per CTA
+  auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };  // leader CTA only (16 arrivals)
+  const uint32_t drain_bar = bar_base + 8u * (2 * STAGES + 4);
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   volatile int* abort_flag = &abort_flag_s;
@@ -1012,8 +1037,10 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
     }
-    mbar_init(acc_full_bar, 1);
-    mbar_init(acc_empty_bar, 16);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(acc_full_bar(b), 1);
+      mbar_init(acc_empty_bar(b), 16);
+    }
     mbar_init(drain_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -1029,7 +1056,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
   const uint32_t tmem_base = tmem_base_slot;
   pdl_prologue();
 
-  const int64_t num_tiles = (int64_t)p.m_tiles * p.n_tiles;  // 256 x 256 tiles
+  const int64_t num_tiles = (int64_t)p.m_tiles * p.n_tiles;  // 256 x PN tiles
   const int64_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
   if (warp == 0) {
@@ -1039,9 +1066,10 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     bool ok = true;
     for (int64_t t = pair; t < num_tiles && ok; t += num_pairs) {
       const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
-      const int32_t a_row = mt * 256 + (int32_t)rank * 128, b_row = nt * 256 + (int32_t)rank * 128;
+      const int32_t a_row = mt * 256 + (int32_t)rank * 128, b_row = nt * PN + (int32_t)rank * (PN / 2);
       const int32_t sfa_row = ((mt * 2 + (int32_t)rank) * p.sf_tiles_a) * 4;  // in units of 128 bytes
-      const int32_t sfb_row0 = ((nt * 2) * p.sf_tiles_b) * 4, sfb_row1 = ((nt * 2 + 1) * p.sf_tiles_b) * 4;
+      const int32_t sfb_tile0 = (nt * PN) >> 7;  // first 128-row scale tile the B tile touches (it touches this one and the next)
+      const int32_t sfb_row0 = (sfb_tile0 * p.sf_tiles_b) * 4, sfb_row1 = ((sfb_tile0 + 1) * p.sf_tiles_b) * 4;
       for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it, s = (s + 1 == (uint32_t)STAGES ? 0u : s + 1), wait_parity ^= (s == 0)) {
         ok = __all_sync(0xFFFFFFFFu, mbar_wait(empty_bar(s), wait_parity, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
@@ -1066,7 +1094,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     // ===================================== MMA issuer (leader CTA only) ====================================
     if (rank == 0) {
       const uint32_t leader = elect_leader();
-      const uint32_t idesc = (1u << 7) | (1u << 10) | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+      const uint32_t idesc = (1u << 7) | (1u << 10) | ((uint32_t)(PN >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
       // issue loop kept short as in the 128 x 128 kernel: running stage / phase counters, descriptors by addition to the low
       // word, the next stage's barrier tried before this stage's instructions
       uint32_t it = 0, tile_it = 0, stage = 0, phase = 0;
@@ -1076,9 +1104,13 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
       constexpr uint32_t SF_HI = (uint32_t)((((uint64_t)8 << 32) | ((uint64_t)1 << 46)) >> 32);
       const uint32_t a_lo0 = (uint32_t)desc_sw128(smem_base), sfa_lo0 = (uint32_t)desc_sf(smem_base + A_BYTES + C2_B_BYTES);
       for (int64_t t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
-        ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar, (tile_it & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
+        const uint32_t ab = tile_it % ACC_BUFS;
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar(ab), ((tile_it / ACC_BUFS) & 1) ^ 1, abort_flag, p.dev_status, p.wait_limit));
         if (!ok) break;
         tc_fence_after();
+        const uint32_t d_tmem = tmem_base + ab * PN;
+        // scales of the B rows: the tile may start 64 rows into its first scale tile, i.e. two columns later
+        const uint32_t sfb_col = (uint32_t)((((int32_t)(t % p.n_tiles) * PN) & 127) >> 5);
         for (int32_t kt = 0; kt < p.k_tiles; ++kt, ++it) {
           if (!ready) {
             ok = __all_sync(0xFFFFFFFFu, mbar_wait(full_bar(stage), phase, abort_flag, p.dev_status, p.wait_limit));
@@ -1092,7 +1124,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
             phase ^= 1u;
           }
           const uint32_t next_try = mbar_test(full_bar(stage), phase);
-          const uint32_t sf_tmem = tmem_base + 256 + (it & 3) * C2_SF_COLS;
+          const uint32_t sf_tmem = tmem_base + C2::SF_TMEM_COL + (it % C2::SF_SETS) * C2_SF_COLS;
 #pragma unroll
           for (int kk = 0; kk < BK / 64; ++kk) {
             tc2_cp_sf(sf_tmem + kk * 4, ((uint64_t)SF_HI << 32) | (sfa_lo0 + st16 + kk * 32), leader);
@@ -1101,12 +1133,12 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           }
 #pragma unroll
           for (int kk = 0; kk < BK / 64; ++kk)
-            tc2_mma_nvf4(tmem_base, ((uint64_t)SW_HI << 32) | (a_lo0 + st16 + kk * 2), ((uint64_t)SW_HI << 32) | (a_lo0 + st16 + (A_BYTES >> 4) + kk * 2),
-                         idesc, sf_tmem + kk * 4, sf_tmem + 16 + kk * 8, (kt | kk) != 0, leader);
+            tc2_mma_nvf4(d_tmem, ((uint64_t)SW_HI << 32) | (a_lo0 + st16 + kk * 2), ((uint64_t)SW_HI << 32) | (a_lo0 + st16 + (A_BYTES >> 4) + kk * 2),
+                         idesc, sf_tmem + kk * 4, sf_tmem + 16 + kk * 8 + sfb_col, (kt | kk) != 0, leader);
           tc2_commit_both(this_empty, leader);
           ready = __all_sync(0xFFFFFFFFu, next_try);
         }
-        if (ok) tc2_commit_both(acc_full_bar, leader);
+        if (ok) tc2_commit_both(acc_full_bar(ab), leader);
       }
       // nothing issued may still be running when tensor memory is freed; the commit covers both CTAs' work
       asm volatile(
@@ -1124,45 +1156,50 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
     // ===================================== epilogue (both CTAs, eight warps) ================================
     const int quad = warp & 3;
     const int half = (warp - 2) >> 2;
-    const uint32_t acc_empty_leader = map_to_cta(acc_empty_bar, 0);
+    // columns of the tile this warp owns: [half * 128, half * 128 + 32 * nq): the first four warps 128, the others the rest
+    const int nq = half == 0 ? 4 : (PN - 128) / 32;
     uint32_t tile_it = 0;
     bool ok = true;
     float alpha = 1.0f;
     if (GS == kGsTensor) alpha = __fmul_rn(p.a_gscale[0], p.b_gscale[0]);
     for (int64_t t = pair; t < num_tiles && ok; t += num_pairs, ++tile_it) {
       const int32_t mt = (int32_t)(t / p.n_tiles), nt = (int32_t)(t % p.n_tiles);
-      if (!(ok = mbar_wait(acc_full_bar, tile_it & 1, abort_flag, p.dev_status, p.wait_limit))) break;
+      const uint32_t ab = tile_it % ACC_BUFS;
+      const uint32_t acc_empty_leader = map_to_cta(acc_empty_bar(ab), 0);
+      if (!(ok = mbar_wait(acc_full_bar(ab), (tile_it / ACC_BUFS) & 1, abort_flag, p.dev_status, p.wait_limit))) break;
       tc_fence_after();
       const int64_t m = (int64_t)mt * 256 + rank * 128 + quad * 32 + lane;
       float sa = 1.0f;
       if (GS == kGsRow && m < p.M) sa = p.a_gscale[m];
       uint32_t v[4][32];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + half * 128 + q * 32, v[q]);
+      for (int q = 0; q < 4; ++q)
+        if (q < nq) tc_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) + ab * PN + half * 128 + q * 32, v[q]);
       tc_wait_ld();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
       // The accumulator is free again (the pair's next tile may start); scale, stage and store from the registers.
-      const uint32_t my_stage = staging_base + (uint32_t)(warp - 2) * 4096u;
+      const bool two_bufs = PN == 192 && half == 0;
+      const uint32_t my_stage = staging_base + (PN == 256 ? (uint32_t)(warp - 2) : (half == 0 ? 2u * (uint32_t)(warp - 2) : 4u + (uint32_t)(warp - 2))) * 4096u;
       const int64_t m0 = (int64_t)mt * 256 + rank * 128 + quad * 32;
       if (m0 >= p.M) continue;
       if (p.c_is_f32) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          const int64_t n0 = (int64_t)nt * 256 + half * 128 + q * 32;
-          if (n0 >= p.N) break;
+          const int64_t n0 = (int64_t)nt * PN + half * 128 + q * 32;
+          if (q >= nq || n0 >= p.N) break;
           float o[32], sgb[32];
           if (GS == kGsRow) load_sgb32(p.b_gscale, n0, p.N, sgb);
 #pragma unroll
           for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(v[q][j]) * (GS == kGsRow ? __fmul_rn(sa, sgb[j]) : alpha);
-          stage_and_store<32>(p, &tmC, my_stage, lane, m, m0, n0, o);
+          stage_and_store<32>(p, &tmC, my_stage + (two_bufs ? (uint32_t)(q & 1) * 4096u : 0u), lane, m, m0, n0, o, two_bufs ? 1 : 0);
         }
       } else {
 #pragma unroll
         for (int qq = 0; qq < 2; ++qq) {
-          const int64_t n0 = (int64_t)nt * 256 + half * 128 + qq * 64;
-          if (n0 >= p.N) break;
+          const int64_t n0 = (int64_t)nt * PN + half * 128 + qq * 64;
+          if (2 * qq >= nq || n0 >= p.N) break;
           float o[64], sgb[32];
           if (GS == kGsRow) load_sgb32(p.b_gscale, n0, p.N, sgb);
 #pragma unroll
@@ -1170,7 +1207,7 @@ gemm_nvfp4_2cta_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_con
           if (GS == kGsRow) load_sgb32(p.b_gscale, n0 + 32, p.N, sgb);
 #pragma unroll
           for (int j = 0; j < 32; ++j) o[32 + j] = __uint_as_float(v[2 * qq + 1][j]) * (GS == kGsRow ? __fmul_rn(sa, sgb[j]) : alpha);
-          stage_and_store<64>(p, &tmC, my_stage, lane, m, m0, n0, o);
+          stage_and_store<64>(p, &tmC, my_stage + (two_bufs ? (uint32_t)(qq & 1) * 4096u : 0u), lane, m, m0, n0, o, two_bufs ? 1 : 0);
         }
       }
     }
@@ -1424,13 +1461,14 @@ bool make_sf_map(CUtensorMap* tm, const uint8_t* sf, int64_t total_bytes) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int GS>
+template <int GS, int PN>
 cudaError_t launch_2cta(const GemmArgs& a, cudaStream_t st) {
+  using C2 = Cfg2<PN>;
   const int64_t Kp = (a.K + 127) & ~(int64_t)127;
   const int64_t kb_padded = ((Kp >> 4) + 15) & ~(int64_t)15;
   const int64_t sfa_bytes = ((a.M + 127) / 128) * 128 * kb_padded, sfb_bytes = ((a.N + 127) / 128) * 128 * kb_padded;
   CUtensorMap tmA, tmB, tmSFA, tmSFB, tmC;
-  if (!make_codes_map(&tmA, a.a_codes, a.M, Kp, 128) || !make_codes_map(&tmB, a.b_codes, a.N, Kp, 128) ||
+  if (!make_codes_map(&tmA, a.a_codes, a.M, Kp, 128) || !make_codes_map(&tmB, a.b_codes, a.N, Kp, PN / 2) ||
       !make_sf_map(&tmSFA, a.a_sf, sfa_bytes) || !make_sf_map(&tmSFB, a.b_sf, sfb_bytes) ||
       !make_c_map(&tmC, a.C, a.M, a.N, a.ldc, a.c_is_f32 != 0))
     return cudaErrorInvalidValue;
@@ -1446,17 +1484,17 @@ cudaError_t launch_2cta(const GemmArgs& a, cudaStream_t st) {
   p.k_tiles = (int32_t)((Kp + BK - 1) / BK);
   p.sf_tiles_a = p.sf_tiles_b = (int32_t)(kb_padded >> 2);
   p.m_tiles = (int32_t)((a.M + 255) / 256);
-  p.n_tiles = (int32_t)((a.N + 255) / 256);
+  p.n_tiles = (int32_t)((a.N + PN - 1) / PN);
   p.c_is_f32 = a.c_is_f32;
   p.accumulate = a.accumulate;
   p.dev_status = a.dev_status;
   p.starve = a.starve_first_stage;
   p.wait_limit = wait_limit_of(a);
-  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(gemm_nvfp4_2cta_kernel<GS>), C2_SMEM_BYTES);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(gemm_nvfp4_2cta_kernel<GS, PN>), C2::SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const int64_t tiles = (int64_t)p.m_tiles * p.n_tiles;
   const unsigned pairs = (unsigned)std::min<int64_t>(tiles, sm_count() / 2);
-  launch_kernel(gemm_nvfp4_2cta_kernel<GS>, dim3(2 * pairs), dim3(C2_THREADS), C2_SMEM_BYTES, st, tmA, tmB, tmSFA, tmSFB, tmC, p);
+  launch_kernel(gemm_nvfp4_2cta_kernel<GS, PN>, dim3(2 * pairs), dim3(C2_THREADS), C2::SMEM_BYTES, st, tmA, tmB, tmSFA, tmSFB, tmC, p);
   return cudaGetLastError();
 }
 
@@ -1588,16 +1626,34 @@ int64_t gemm_block128_max_k() { return (int64_t)B128_MAX_CHUNKS * 128; }
 // work. The fused high-precision side product and the outer-block scales live in the single-CTA kernels only.
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;
-  if (a.gs_mode == kGsBlock128) return a.variant == 2 ? cudaErrorInvalidValue : launch_block128(a, st);
+  if (a.gs_mode == kGsBlock128) return a.variant >= 2 ? cudaErrorInvalidValue : launch_block128(a, st);
   const int64_t tiles256 = ((a.M + 255) / 256) * ((a.N + 255) / 256), n_pairs = sm_count() / 2;
   bool pairs = (a.K >= 2048 && tiles256 >= 2 * n_pairs) || (a.K >= 8192 && 2 * tiles256 >= n_pairs);
-  if (a.variant == 1) pairs = false;
-  if (a.variant == 2) pairs = true;
-  if (a.hp_Kh > 0) {
-    if (a.variant == 2) return cudaErrorInvalidValue;
-    pairs = false;
+  // Between the two pair kernels, by a cost model in units of one 256-wide k tile: rounds of the pair grid x (k tiles x the
+  // relative cost of a k tile + the per-tile cost). 256-wide tiles: 1 per k tile, about 3.5 per tile (single accumulator:
+  // its hand-over is exposed); 192-wide tiles: 0.82 per k tile (three quarters of the math, but 9 % more operand traffic
+  // per flop), about 1 per tile (two accumulators), and a finer last wave. Measured, BF16 output, 256 / 192 wide, us:
+  // 16384 x 3072 x 2048 59.3 / 51.3, 8192 x 8192 x 3072 88.0 / 84.1, 16384 x 4096 x 4096 112.7 / 106.5, 16384 x 14336 x 4096
+  // 374 / 365, 4096^3 37.0 / 36.9, 3072 x 1024 x 16384 33.7 / 32.8 (48 / 72 tiles for 74 pairs), 2048 x 2048 x 16384 32.8 /
+  // 47.1 (64 / 88 tiles), 4096 x 8192 x 8192 96.4 / 106.5, 16384 x 8192 x 8192 365 / 397.
+  bool pairs192 = false;
+  if (pairs) {
+    const int64_t tiles192 = ((a.M + 255) / 256) * ((a.N + 191) / 192);
+    const double k_tiles = (double)((a.K + BK - 1) / BK);
+    const double cost256 = (double)((tiles256 + n_pairs - 1) / n_pairs) * (k_tiles + 3.5);
+    const double cost192 = (double)((tiles192 + n_pairs - 1) / n_pairs) * (0.82 * k_tiles + 1.0);
+    pairs192 = cost192 < cost256;
   }
-  if (pairs) return a.gs_mode == kGsTensor ? launch_2cta<kGsTensor>(a, st) : launch_2cta<kGsRow>(a, st);
+  if (pairs192) pairs = false;
+  if (a.variant == 1) pairs = pairs192 = false;
+  if (a.variant == 2) { pairs = true; pairs192 = false; }
+  if (a.variant == 3) { pairs192 = true; pairs = false; }
+  if (a.hp_Kh > 0) {
+    if (a.variant == 2 || a.variant == 3) return cudaErrorInvalidValue;
+    pairs = pairs192 = false;
+  }
+  if (pairs192) return a.gs_mode == kGsTensor ? launch_2cta<kGsTensor, 192>(a, st) : launch_2cta<kGsRow, 192>(a, st);
+  if (pairs) return a.gs_mode == kGsTensor ? launch_2cta<kGsTensor, 256>(a, st) : launch_2cta<kGsRow, 256>(a, st);
   return a.gs_mode == kGsTensor ? launch_tile128<kGsTensor>(a, st) : launch_tile128<kGsRow>(a, st);
 }
 
