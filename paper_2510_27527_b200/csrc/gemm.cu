@@ -897,7 +897,6 @@ struct Cfg2 {
   static constexpr uint32_t SF_COLS = 16 + 32;
   static constexpr uint32_t SF_SETS = PN == 256 ? 4 : 2;
   static constexpr uint32_t SF_TMEM_COL = ACC_BUFS * PN;                       // 256 / 384; + SF_SETS * 48 <= 512
-  static constexpr int COLS_HALF0 = 128;                                       // columns the first four epilogue warps own
 };
 constexpr int C2_THREADS = 64 + 256;
 
@@ -916,8 +915,12 @@ __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// Arrive on a barrier of a CTA of the cluster (possibly this one). Relaxed: what it announces -- this warp's tensor-memory
+// loads of the accumulator are complete -- is ordered by tcgen05.wait::ld and the tcgen05 fence before it; with release
+// semantics at cluster scope the arrive took about 2500 cycles (it waits for the thread's earlier shared-memory and bulk
+// traffic), and that, not the loads, was the cost of handing the accumulator over.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // Bulk-tensor load of one CTA of a pair; completes on an mbarrier that may live in the peer CTA.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, int32_t c0, int32_t c1,
@@ -1611,37 +1614,35 @@ cudaError_t launch_dense_gemm(const void* A, const void* B, int64_t M, int64_t N
 size_t gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
 int64_t gemm_block128_max_k() { return (int64_t)B128_MAX_CHUNKS * 128; }
 
-// Variant choice. Both kernels are bound by what the L2 delivers to the SMs (about 13 - 16 TB/s over all SMs): the 128 x 128
+// Variant choice. All kernels are bound by what the L2 delivers to the SMs (about 13 - 16 TB/s over all SMs): the 128 x 128
 // kernel pulls 36 KB per k tile and SM, a pair on a 256 x 256 tile 38 KB per SM for twice the math. The 128 x 128 kernel has
-// two accumulators (a tile's epilogue overlaps the next tile's MMAs entirely); the pair kernel has one and hands it over once
-// its sixteen epilogue warps hold the tile in registers, which costs a few hundred cycles per tile and 256-wide tiles fill
-// the last wave worse. Pairs therefore run from K = 2048 when there are two tiles for every pair, and from K = 8192 already
-// when half of the pairs get a tile (the weight gradients of a model: few tiles, K = tokens). Measured, BF16 / FP32 output,
-// 128 x 128 against pairs, us: 16384 x 3072 x 1024 -> 41.0 / 44.0 and 52.0 / 56.3; 16384 x 1024 x 3072 -> 33.8 / 33.8 and
-// 37.0 / 37.8; 16384 x 3072 x 2048 -> 64.5 / 59.4 and 75.8 / 71.9; 8192 x 8192 x 3072 -> 105.5 / 90.9 and 122.8 / 109.6;
-// 4096 x 4096 x 4096 -> 41.0 / 38.8 and 46.0 / 45.9; 16384 x 14336 x 4096 -> 428 / 373 and 531 / 443; 3072 x 1024 x 16384 (48
-// pair tiles) -> 41.9 / 33.8 and 43.9 / 35.9; 1024 x 1024 x 16384 (16) -> 24.8 / 31.7; 16384 x 8192 x 8192 -> 459 / 370 and
-// 498 / 401.
+// two accumulators (a tile's epilogue overlaps the next tile's MMAs entirely); the 256-wide pair kernel has one and hands it
+// over once its sixteen epilogue warps hold the tile in registers (a few hundred cycles per tile), and 256-wide tiles fill
+// the last wave worse. Pairs therefore run when there are enough tiles: from K = 1024 with five tiles per pair, from
+// K = 2048 with two, and from K = 8192 already when half of the pairs get a tile (the weight gradients of a model: few
+// tiles, K = tokens). Measured, BF16 output, 128 x 128 / 256 x 256 / 256 x 192, us: 16384 x 3072 x 1024 38.9 / 34.8 / 36.9;
+// 16384 x 1024 x 1024 (256 pair tiles) 18.5 / 19.2 / 22.4; 8192 x 3072 x 1024 (384) 24.5 / 22.7 / 22.5; 4096 x 4096 x 1024
+// (256) 18.4 / 18.5 / 20.4; 16384 x 1024 x 2816 31.6 / 28.8 / 32.8; 16384 x 3072 x 2048 61.4 / 51.2 / 55.8; 8192 x 8192 x 3072
+// 100.4 / 77.8 / 87.9; 4096^3 38.9 / 34.8 / 34.8; 16384 x 14336 x 4096 426 / 342 / 387; 4096 x 8192 x 8192 114.8 / 88.1 /
+// 104.4; 16384 x 8192 x 8192 455 / 352 / 408; 3072 x 1024 x 16384 (48 / 72 pair tiles) 38.9 / 30.8 / 30.7, FP32 output 40.9 /
+// 32.7 / 30.7; 1024 x 1024 x 16384 (16 / 24) 22.6 / 30.8 / 28.7; 2048 x 2048 x 16384 (64 / 88) 38.9 / 32.8 / 46.9.
 // A 256-row tile of an operand spans two 128-row scale tiles, and rows are padded to 128 in the scale layout, so any M, N
 // work. The fused high-precision side product and the outer-block scales live in the single-CTA kernels only.
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;
   if (a.gs_mode == kGsBlock128) return a.variant >= 2 ? cudaErrorInvalidValue : launch_block128(a, st);
   const int64_t tiles256 = ((a.M + 255) / 256) * ((a.N + 255) / 256), n_pairs = sm_count() / 2;
-  bool pairs = (a.K >= 2048 && tiles256 >= 2 * n_pairs) || (a.K >= 8192 && 2 * tiles256 >= n_pairs);
+  bool pairs = (a.K >= 1024 && tiles256 >= 5 * n_pairs) || (a.K >= 2048 && tiles256 >= 2 * n_pairs) ||
+               (a.K >= 8192 && 2 * tiles256 >= n_pairs);
   // Between the two pair kernels, by a cost model in units of one 256-wide k tile: rounds of the pair grid x (k tiles x the
-  // relative cost of a k tile + the per-tile cost). 256-wide tiles: 1 per k tile, about 3.5 per tile (single accumulator:
-  // its hand-over is exposed); 192-wide tiles: 0.82 per k tile (three quarters of the math, but 9 % more operand traffic
-  // per flop), about 1 per tile (two accumulators), and a finer last wave. Measured, BF16 output, 256 / 192 wide, us:
-  // 16384 x 3072 x 2048 59.3 / 51.3, 8192 x 8192 x 3072 88.0 / 84.1, 16384 x 4096 x 4096 112.7 / 106.5, 16384 x 14336 x 4096
-  // 374 / 365, 4096^3 37.0 / 36.9, 3072 x 1024 x 16384 33.7 / 32.8 (48 / 72 tiles for 74 pairs), 2048 x 2048 x 16384 32.8 /
-  // 47.1 (64 / 88 tiles), 4096 x 8192 x 8192 96.4 / 106.5, 16384 x 8192 x 8192 365 / 397.
+  // relative cost of a k tile + 1 per tile). A 192-wide k tile costs 0.85 (three quarters of the math, but more operand
+  // traffic per flop); what the 192-wide tiles have is the finer last wave, which decides when tiles are few.
   bool pairs192 = false;
   if (pairs) {
     const int64_t tiles192 = ((a.M + 255) / 256) * ((a.N + 191) / 192);
     const double k_tiles = (double)((a.K + BK - 1) / BK);
-    const double cost256 = (double)((tiles256 + n_pairs - 1) / n_pairs) * (k_tiles + 3.5);
-    const double cost192 = (double)((tiles192 + n_pairs - 1) / n_pairs) * (0.82 * k_tiles + 1.0);
+    const double cost256 = (double)((tiles256 + n_pairs - 1) / n_pairs) * (k_tiles + 1.0);
+    const double cost192 = (double)((tiles192 + n_pairs - 1) / n_pairs) * (0.85 * k_tiles + 1.0);
     pairs192 = cost192 < cost256;
   }
   if (pairs192) pairs = false;
