@@ -1632,7 +1632,11 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.M == 0 || a.N == 0) return cudaSuccess;
   if (a.gs_mode == kGsBlock128) return a.variant >= 2 ? cudaErrorInvalidValue : launch_block128(a, st);
   const int64_t tiles256 = ((a.M + 255) / 256) * ((a.N + 255) / 256), n_pairs = sm_count() / 2;
-  bool pairs = (a.K >= 1024 && tiles256 >= 5 * n_pairs) || (a.K >= 2048 && tiles256 >= 2 * n_pairs) ||
+  // (ROW scales: the pair kernels' epilogue holds a quarter tile in registers and has two more multiplies per element to do,
+  // it spills and becomes the bound at short K -- 16384 x 3072 x 1024, BF16 output: 40.9 / 53.4 / 74.7 us -- so pairs start at
+  // K = 2048 there and the 192-wide kernel, which has the least time per tile to hide it in, is not used.)
+  const bool row_scales = a.gs_mode == kGsRow;
+  bool pairs = (!row_scales && a.K >= 1024 && tiles256 >= 5 * n_pairs) || (a.K >= 2048 && tiles256 >= 2 * n_pairs) ||
                (a.K >= 8192 && 2 * tiles256 >= n_pairs);
   // Between the two pair kernels, by a cost model in units of one 256-wide k tile: rounds of the pair grid x (k tiles x the
   // relative cost of a k tile + 1 per tile). A 192-wide k tile costs 0.85 (three quarters of the math, but more operand
@@ -1643,7 +1647,7 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
     const double k_tiles = (double)((a.K + BK - 1) / BK);
     const double cost256 = (double)((tiles256 + n_pairs - 1) / n_pairs) * (k_tiles + 1.0);
     const double cost192 = (double)((tiles192 + n_pairs - 1) / n_pairs) * (0.85 * k_tiles + 1.0);
-    pairs192 = cost192 < cost256;
+    pairs192 = !row_scales && cost192 < cost256;
   }
   if (pairs192) pairs = false;
   if (a.variant == 1) pairs = pairs192 = false;
